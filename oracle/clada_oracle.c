@@ -1,0 +1,295 @@
+/*
+ * CLADA oracle -- TEST INFRASTRUCTURE, not the product.
+ *
+ * A plain, slow CPU restatement of what the cognitive-load-aware sparse gated
+ * FFN computes, written from the paper's definitions.  Every sum is a plain
+ * loop in double precision in the order the definition states; there is no
+ * blocking, fusion or reordering.  It shares no code with the CUDA library and
+ * is only ever called by the tests, the smoke check and the CPU-baseline leg
+ * of the benchmark.
+ *
+ * Weight layout here is the paper's own: W_in and V_in are [d_ff, d_model]
+ * with neuron j in row j; W_out is [d_model, d_ff] with neuron j in COLUMN j
+ * (Section 3.2.1, text under Eq. neuron_activation).
+ *
+ * Pins (tests/test_oracle_pins.py): entropy/surprisal closed forms, literal
+ * Frobenius form of the score, brute-force selection on tiny layers, dense
+ * FFN against an independent float64 matrix formulation, zero-sparsity
+ * identity, CETT identity.  The whole of Algorithm 2 end to end has no
+ * published trace: parity unpinned beyond those per-step pins.
+ *
+ * Element types: 0 = IEEE fp32, 1 = bfloat16 (uint16 bit patterns).  Both
+ * widen to double exactly.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+enum { OR_F32 = 0, OR_BF16 = 1 };
+
+static double elem(const void *p, int dtype, size_t i)
+{
+    if (dtype == OR_F32)
+        return (double)((const float *)p)[i];
+    uint32_t bits = ((uint32_t)((const uint16_t *)p)[i]) << 16;
+    float f;
+    memcpy(&f, &bits, sizeof f);
+    return (double)f;
+}
+
+/* sigma of Eq. neuron_activation read as SiLU: g * logistic(g). */
+static double silu(double g) { return g / (1.0 + exp(-g)); }
+
+int oracle_num_threads(void)
+{
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
+
+/* ------------------------------------------------------------------ *
+ * Eq. neuron_activation, factored form.
+ *
+ * For sequence b with prefix rows [off[b], off[b+1]) of X and neuron j:
+ *   z_t = silu(W_in,j . x_t) * (V_in,j . x_t)
+ *   A_j = || z_{:,j} (outer) W_out,j ||  =  sqrt(sum_t z_t^2) * sqrt(sum_i W_out[i,j]^2)
+ * (the matrix inside the norm has rank one, so its Frobenius and spectral
+ * norms are the same number).
+ * scores: [B, d_ff] double.
+ * ------------------------------------------------------------------ */
+void oracle_neuron_scores(int dtype, const void *X, const int64_t *off, int B,
+                          int d_model, int d_ff, const void *W_in,
+                          const void *V_in, const void *W_out, double *scores)
+{
+#pragma omp parallel for schedule(dynamic, 8)
+    for (int j = 0; j < d_ff; ++j) {
+        double wnorm2 = 0.0;
+        for (int i = 0; i < d_model; ++i) {
+            double w = elem(W_out, dtype, (size_t)i * d_ff + j);
+            wnorm2 += w * w;
+        }
+        for (int b = 0; b < B; ++b) {
+            double zz = 0.0;
+            for (int64_t t = off[b]; t < off[b + 1]; ++t) {
+                double g = 0.0, u = 0.0;
+                for (int k = 0; k < d_model; ++k) {
+                    double x = elem(X, dtype, (size_t)t * d_model + k);
+                    g += elem(W_in, dtype, (size_t)j * d_model + k) * x;
+                    u += elem(V_in, dtype, (size_t)j * d_model + k) * x;
+                }
+                double z = silu(g) * u;
+                zz += z * z;
+            }
+            scores[(size_t)b * d_ff + j] = sqrt(zz) * sqrt(wnorm2);
+        }
+    }
+}
+
+/* Eq. neuron_activation, literal form for ONE sequence of T rows: build the
+ * T x d_model matrix M[t,i] = z_t * W_out[i,j] and take its Frobenius norm.
+ * Tiny sizes only (allocates T*d_model doubles per neuron). */
+void oracle_neuron_scores_literal(int dtype, const void *X, int T, int d_model,
+                                  int d_ff, const void *W_in, const void *V_in,
+                                  const void *W_out, double *scores)
+{
+    double *M = (double *)malloc((size_t)T * d_model * sizeof(double));
+    for (int j = 0; j < d_ff; ++j) {
+        for (int t = 0; t < T; ++t) {
+            double g = 0.0, u = 0.0;
+            for (int k = 0; k < d_model; ++k) {
+                double x = elem(X, dtype, (size_t)t * d_model + k);
+                g += elem(W_in, dtype, (size_t)j * d_model + k) * x;
+                u += elem(V_in, dtype, (size_t)j * d_model + k) * x;
+            }
+            double z = silu(g) * u;
+            for (int i = 0; i < d_model; ++i)
+                M[(size_t)t * d_model + i] = z * elem(W_out, dtype, (size_t)i * d_ff + j);
+        }
+        double fro2 = 0.0;
+        for (size_t q = 0; q < (size_t)T * d_model; ++q)
+            fro2 += M[q] * M[q];
+        scores[j] = sqrt(fro2);
+    }
+    free(M);
+}
+
+/* Eq. base_threshold, last line: S_cut = { j : A_j < eps }.  A neuron is kept
+ * iff A_j >= tau (equality keeps).  idx lists the kept neurons ascending.
+ * Returns the number kept. */
+int oracle_select(const double *scores, int d_ff, double tau, uint8_t *mask,
+                  int32_t *idx)
+{
+    int count = 0;
+    for (int j = 0; j < d_ff; ++j) {
+        int keep = !(scores[j] < tau);
+        if (mask)
+            mask[j] = (uint8_t)keep;
+        if (keep) {
+            if (idx)
+                idx[count] = j;
+            ++count;
+        }
+    }
+    return count;
+}
+
+/* Eqs. surprisal and entropy for one vocabulary row of logits (natural log):
+ *   P = softmax(logits); s = -log P[token]; H = -sum_w P[w] log P[w]
+ * with 0 log 0 := 0, so a logit of -inf contributes nothing.
+ * Returns 0, or 1 if token is outside [0, V) (then s = NaN). */
+int oracle_cogload(int dtype, const void *logits, int64_t V, int64_t token,
+                   double *surprisal, double *entropy)
+{
+    double m = -INFINITY;
+    for (int64_t w = 0; w < V; ++w) {
+        double l = elem(logits, dtype, (size_t)w);
+        if (l > m)
+            m = l;
+    }
+    double Z = 0.0;
+    for (int64_t w = 0; w < V; ++w)
+        Z += exp(elem(logits, dtype, (size_t)w) - m);
+    double logZ = log(Z);
+    double H = 0.0;
+    for (int64_t w = 0; w < V; ++w) {
+        double logp = elem(logits, dtype, (size_t)w) - m - logZ;
+        if (logp > -INFINITY)
+            H -= exp(logp) * logp;
+    }
+    *entropy = H;
+    if (token < 0 || token >= V) {
+        *surprisal = NAN;
+        return 1;
+    }
+    *surprisal = -(elem(logits, dtype, (size_t)token) - m - logZ);
+    return 0;
+}
+
+/* Eq. final_threshold for B sequences and L layers:
+ *   tau_final[b,l] = tau_base[b,l] * (1 + lambda[l]*I(s_b > tau_s) + gamma[l]*I(H_b > tau_H)).
+ * The multiplier and the product are taken in fp32, left to right, with no
+ * fused multiply-add (this file is compiled with -ffp-contract=off), so the
+ * result is a definite fp32 number.  The indicators compare in double. */
+void oracle_adjust_threshold(const float *tau_base, const float *lambda,
+                             const float *gamma, float tau_s, float tau_H,
+                             const double *surprisal, const double *entropy,
+                             int B, int L, float *tau_final)
+{
+    for (int b = 0; b < B; ++b) {
+        int hi_s = surprisal[b] > (double)tau_s;
+        int hi_H = entropy[b] > (double)tau_H;
+        for (int l = 0; l < L; ++l) {
+            volatile float mult = 1.0f;
+            if (hi_s)
+                mult = mult + lambda[l];
+            if (hi_H)
+                mult = mult + gamma[l];
+            volatile float t = tau_base[(size_t)b * L + l] * mult;
+            tau_final[(size_t)b * L + l] = t;
+        }
+    }
+}
+
+/* Algorithm 2, mask regeneration + sparse forward pass, one token x:
+ *   mask_j = (A_j >= tau);   y = sum_{j kept, ascending} silu(W_in,j.x) (V_in,j.x) W_out[:,j]
+ * No bias, no rescaling of the kept neurons.  mask_out may be NULL.
+ * Returns the number of kept neurons. */
+int oracle_sparse_ffn(int dtype, const void *x, int d_model, int d_ff,
+                      const void *W_in, const void *V_in, const void *W_out,
+                      const double *scores, double tau, double *y,
+                      uint8_t *mask_out)
+{
+    double *h = (double *)calloc((size_t)d_ff, sizeof(double));
+    uint8_t *keep = (uint8_t *)malloc((size_t)d_ff);
+    int count = 0;
+    for (int j = 0; j < d_ff; ++j) {
+        keep[j] = (uint8_t)!(scores[j] < tau);
+        count += keep[j];
+        if (mask_out)
+            mask_out[j] = keep[j];
+    }
+#pragma omp parallel for schedule(static)
+    for (int j = 0; j < d_ff; ++j) {
+        if (!keep[j])
+            continue;
+        double g = 0.0, u = 0.0;
+        for (int k = 0; k < d_model; ++k) {
+            double xv = elem(x, dtype, (size_t)k);
+            g += elem(W_in, dtype, (size_t)j * d_model + k) * xv;
+            u += elem(V_in, dtype, (size_t)j * d_model + k) * xv;
+        }
+        h[j] = silu(g) * u;
+    }
+#pragma omp parallel for schedule(static)
+    for (int i = 0; i < d_model; ++i) {
+        double acc = 0.0;
+        for (int j = 0; j < d_ff; ++j)
+            if (keep[j])
+                acc += h[j] * elem(W_out, dtype, (size_t)i * d_ff + j);
+        y[i] = acc;
+    }
+    free(h);
+    free(keep);
+    return count;
+}
+
+/* The dense gated FFN, y = W_out (silu(W_in x) * (V_in x)): the
+ * zero-sparsity reference the sparse pass must reduce to. */
+void oracle_dense_ffn(int dtype, const void *x, int d_model, int d_ff,
+                      const void *W_in, const void *V_in, const void *W_out,
+                      double *y)
+{
+    double *h = (double *)malloc((size_t)d_ff * sizeof(double));
+#pragma omp parallel for schedule(static)
+    for (int j = 0; j < d_ff; ++j) {
+        double g = 0.0, u = 0.0;
+        for (int k = 0; k < d_model; ++k) {
+            double xv = elem(x, dtype, (size_t)k);
+            g += elem(W_in, dtype, (size_t)j * d_model + k) * xv;
+            u += elem(V_in, dtype, (size_t)j * d_model + k) * xv;
+        }
+        h[j] = silu(g) * u;
+    }
+#pragma omp parallel for schedule(static)
+    for (int i = 0; i < d_model; ++i) {
+        double acc = 0.0;
+        for (int j = 0; j < d_ff; ++j)
+            acc += h[j] * elem(W_out, dtype, (size_t)i * d_ff + j);
+        y[i] = acc;
+    }
+    free(h);
+}
+
+/* Harness helper (stands in for the offline threshold search, which is an
+ * input to the path): the threshold that cuts exactly k_cut = floor(rho*F+0.5)
+ * neurons of an fp32 score vector, placed midway between the k_cut-th and
+ * (k_cut+1)-th smallest scores.  Midpoint taken in fp32 as 0.5f*a + 0.5f*b.
+ * k_cut == 0 gives 0 (keep all); k_cut == F gives +inf (cut all). */
+static int cmp_float(const void *a, const void *b)
+{
+    float x = *(const float *)a, y = *(const float *)b;
+    return (x > y) - (x < y);
+}
+
+float oracle_tau_from_sparsity(const float *scores, int d_ff, double rho)
+{
+    int k_cut = (int)floor(rho * d_ff + 0.5);
+    if (k_cut <= 0)
+        return 0.0f;
+    if (k_cut >= d_ff)
+        return INFINITY;
+    float *s = (float *)malloc((size_t)d_ff * sizeof(float));
+    memcpy(s, scores, (size_t)d_ff * sizeof(float));
+    qsort(s, (size_t)d_ff, sizeof(float), cmp_float);
+    volatile float lo = 0.5f * s[k_cut - 1];
+    volatile float hi = 0.5f * s[k_cut];
+    volatile float mid = lo + hi;
+    free(s);
+    return mid;
+}

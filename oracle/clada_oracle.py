@@ -1,0 +1,172 @@
+"""ctypes front end of the CLADA CPU oracle (TEST INFRASTRUCTURE, not the product).
+
+Loads ``libclada_oracle.so`` built from ``clada_oracle.c`` in this folder (``build()``
+compiles it with gcc).  Arrays are numpy; bf16 tensors travel as uint16 bit patterns.
+Nothing here imports the CUDA package, and the CUDA package never imports this.
+Weight layout is the paper's: W_in, V_in are [d_ff, d_model]; W_out is [d_model, d_ff].
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "clada_oracle.c")
+_LIB = os.path.join(_HERE, "libclada_oracle.so")
+
+F32, BF16 = 0, 1
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with gcc (plain C, OpenMP for the row loops, no FMA contraction)."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        cmd = ["gcc", "-O2", "-std=c99", "-fopenmp", "-ffp-contract=off", "-fno-fast-math",
+               "-shared", "-fPIC", _SRC, "-o", _LIB, "-lm"]
+        subprocess.run(cmd, check=True)
+    return _LIB
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        build()
+        L = ctypes.CDLL(_LIB)
+        vp, i32, i64, dbl, f32 = (ctypes.c_void_p, ctypes.c_int, ctypes.c_int64,
+                                  ctypes.c_double, ctypes.c_float)
+        L.oracle_num_threads.restype = ctypes.c_int
+        L.oracle_neuron_scores.argtypes = [i32, vp, vp, i32, i32, i32, vp, vp, vp, vp]
+        L.oracle_neuron_scores.restype = None
+        L.oracle_neuron_scores_literal.argtypes = [i32, vp, i32, i32, i32, vp, vp, vp, vp]
+        L.oracle_neuron_scores_literal.restype = None
+        L.oracle_select.argtypes = [vp, i32, dbl, vp, vp]
+        L.oracle_select.restype = ctypes.c_int
+        L.oracle_cogload.argtypes = [i32, vp, i64, i64, vp, vp]
+        L.oracle_cogload.restype = ctypes.c_int
+        L.oracle_adjust_threshold.argtypes = [vp, vp, vp, f32, f32, vp, vp, i32, i32, vp]
+        L.oracle_adjust_threshold.restype = None
+        L.oracle_sparse_ffn.argtypes = [i32, vp, i32, i32, vp, vp, vp, vp, dbl, vp, vp]
+        L.oracle_sparse_ffn.restype = ctypes.c_int
+        L.oracle_dense_ffn.argtypes = [i32, vp, i32, i32, vp, vp, vp, vp]
+        L.oracle_dense_ffn.restype = None
+        L.oracle_tau_from_sparsity.argtypes = [vp, i32, dbl]
+        L.oracle_tau_from_sparsity.restype = f32
+        _lib = L
+    return _lib
+
+
+def num_threads() -> int:
+    return int(lib().oracle_num_threads())
+
+
+def _dt(a: np.ndarray) -> int:
+    if a.dtype == np.float32:
+        return F32
+    if a.dtype == np.uint16:
+        return BF16
+    raise TypeError(f"oracle takes float32 or uint16 (bf16 bits) arrays, got {a.dtype}")
+
+
+def _c(a: np.ndarray, dtype=None) -> np.ndarray:
+    a = np.ascontiguousarray(a) if dtype is None else np.ascontiguousarray(a, dtype=dtype)
+    return a
+
+
+def _p(a: np.ndarray):
+    return a.ctypes.data_as(ctypes.c_void_p)
+
+
+def _check_weights(X, W_in, V_in, W_out):
+    d_ff, d_model = W_in.shape
+    assert V_in.shape == (d_ff, d_model), "V_in must be [d_ff, d_model]"
+    assert W_out.shape == (d_model, d_ff), "W_out must be [d_model, d_ff] (neuron j = column j)"
+    assert X.shape[-1] == d_model
+    assert X.dtype == W_in.dtype == V_in.dtype == W_out.dtype
+    return d_model, d_ff
+
+
+def neuron_scores(X, seq_offsets, W_in, V_in, W_out) -> np.ndarray:
+    """A[b, j] of Eq. neuron_activation for each prefix b = rows seq_offsets[b]:seq_offsets[b+1] of X."""
+    X, W_in, V_in, W_out = _c(X), _c(W_in), _c(V_in), _c(W_out)
+    d_model, d_ff = _check_weights(X, W_in, V_in, W_out)
+    off = _c(np.asarray(seq_offsets), np.int64)
+    B = off.size - 1
+    assert off[0] >= 0 and off[-1] <= X.shape[0] and np.all(np.diff(off) >= 0)
+    out = np.empty((B, d_ff), dtype=np.float64)
+    lib().oracle_neuron_scores(_dt(X), _p(X), _p(off), B, d_model, d_ff,
+                               _p(W_in), _p(V_in), _p(W_out), _p(out))
+    return out
+
+
+def neuron_scores_literal(X, W_in, V_in, W_out) -> np.ndarray:
+    """Same quantity for one prefix X [T, d_model], by the Frobenius norm of the explicit T x d_model matrix."""
+    X, W_in, V_in, W_out = _c(X), _c(W_in), _c(V_in), _c(W_out)
+    d_model, d_ff = _check_weights(X, W_in, V_in, W_out)
+    out = np.empty(d_ff, dtype=np.float64)
+    lib().oracle_neuron_scores_literal(_dt(X), _p(X), X.shape[0], d_model, d_ff,
+                                       _p(W_in), _p(V_in), _p(W_out), _p(out))
+    return out
+
+
+def select(scores, tau):
+    """(mask u8 [d_ff], idx int32 [count] ascending, count) with neuron j kept iff scores[j] >= tau."""
+    scores = _c(scores, np.float64)
+    d_ff = scores.size
+    mask = np.empty(d_ff, dtype=np.uint8)
+    idx = np.empty(d_ff, dtype=np.int32)
+    count = lib().oracle_select(_p(scores), d_ff, float(tau), _p(mask), _p(idx))
+    return mask, idx[:count].copy(), int(count)
+
+
+def cogload(logits, token_id):
+    """(surprisal, entropy) in nats of softmax(logits) for one vocabulary row; token out of range -> s = nan."""
+    logits = _c(logits)
+    assert logits.ndim == 1
+    s = ctypes.c_double()
+    h = ctypes.c_double()
+    lib().oracle_cogload(_dt(logits), _p(logits), logits.size, int(token_id),
+                         ctypes.byref(s), ctypes.byref(h))
+    return s.value, h.value
+
+
+def adjust_threshold(tau_base, lam, gam, tau_s, tau_H, surprisal, entropy) -> np.ndarray:
+    """tau_final [B, L] fp32 of Eq. final_threshold."""
+    tau_base = _c(tau_base, np.float32)
+    B, L = tau_base.shape
+    lam, gam = _c(lam, np.float32), _c(gam, np.float32)
+    s, h = _c(surprisal, np.float64), _c(entropy, np.float64)
+    assert lam.size == L and gam.size == L and s.size == B and h.size == B
+    out = np.empty((B, L), dtype=np.float32)
+    lib().oracle_adjust_threshold(_p(tau_base), _p(lam), _p(gam), float(np.float32(tau_s)), float(np.float32(tau_H)),
+                                  _p(s), _p(h), B, L, _p(out))
+    return out
+
+
+def sparse_ffn(x, W_in, V_in, W_out, scores, tau):
+    """(y [d_model] float64, mask u8 [d_ff], count) of the masked gated FFN for one token x."""
+    x, W_in, V_in, W_out = _c(x), _c(W_in), _c(V_in), _c(W_out)
+    d_model, d_ff = _check_weights(x, W_in, V_in, W_out)
+    scores = _c(scores, np.float64)
+    assert scores.size == d_ff and x.size == d_model
+    y = np.empty(d_model, dtype=np.float64)
+    mask = np.empty(d_ff, dtype=np.uint8)
+    count = lib().oracle_sparse_ffn(_dt(x), _p(x), d_model, d_ff, _p(W_in), _p(V_in), _p(W_out),
+                                    _p(scores), float(tau), _p(y), _p(mask))
+    return y, mask, int(count)
+
+
+def dense_ffn(x, W_in, V_in, W_out) -> np.ndarray:
+    x, W_in, V_in, W_out = _c(x), _c(W_in), _c(V_in), _c(W_out)
+    d_model, d_ff = _check_weights(x, W_in, V_in, W_out)
+    y = np.empty(d_model, dtype=np.float64)
+    lib().oracle_dense_ffn(_dt(x), _p(x), d_model, d_ff, _p(W_in), _p(V_in), _p(W_out), _p(y))
+    return y
+
+
+def tau_from_sparsity(scores_f32, rho) -> np.float32:
+    """Harness helper: fp32 midpoint threshold that cuts floor(rho*F + 0.5) neurons of an fp32 score vector."""
+    s = _c(scores_f32, np.float32)
+    return np.float32(lib().oracle_tau_from_sparsity(_p(s), s.size, float(rho)))

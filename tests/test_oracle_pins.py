@@ -1,0 +1,340 @@
+"""Pins for the CPU oracle: closed forms, invariants, brute force and library routines.
+
+Each test fixes the oracle to something other than itself, so that a dropped term, a wrong sign
+or index, or a transposed operand in oracle/clada_oracle.c fails here.  No GPU involved.
+"""
+import math
+import os
+
+import numpy as np
+import pytest
+import scipy.special
+import torch
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def _bf16_bits(a: np.ndarray) -> np.ndarray:
+    t = torch.from_numpy(np.asarray(a, dtype=np.float32)).to(torch.bfloat16)
+    return t.view(torch.int16).numpy().view(np.uint16)
+
+
+def _bf16_to_f64(bits: np.ndarray) -> np.ndarray:
+    return (bits.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+
+
+def _layer(rng, d, F, T, dtype="f32"):
+    Wg = (rng.standard_normal((F, d)) * 0.3).astype(np.float32)
+    Wu = (rng.standard_normal((F, d)) * 0.3).astype(np.float32)
+    Wd = (rng.standard_normal((d, F)) * 0.3).astype(np.float32)
+    X = rng.standard_normal((T, d)).astype(np.float32)
+    if dtype == "bf16":
+        return tuple(_bf16_bits(a) for a in (X, Wg, Wu, Wd))
+    return X, Wg, Wu, Wd
+
+
+def _f64(a):
+    return _bf16_to_f64(a) if a.dtype == np.uint16 else a.astype(np.float64)
+
+
+# ----------------------------------------------------------------------------------------------
+# Cognitive load: Eqs. surprisal / entropy
+# ----------------------------------------------------------------------------------------------
+
+def _golden_ln_vocab():
+    rows = {}
+    with open(os.path.join(GOLDEN, "ln_vocab.txt")) as f:
+        for line in f:
+            if line.startswith("#") or not line.strip():
+                continue
+            v, val = line.split()
+            rows[int(v)] = float(val)
+    return rows
+
+
+@pytest.mark.parametrize("V", [2, 4096, 32000, 128256])
+def test_entropy_uniform_is_ln_V(oracle, V):
+    golden = _golden_ln_vocab()
+    logits = np.full(V, 1.75, dtype=np.float32)
+    s, H = oracle.cogload(logits, V // 3)
+    assert abs(H - golden[V]) < 1e-10
+    assert abs(s - golden[V]) < 1e-10
+    assert abs(golden[V] - math.log(V)) < 1e-12
+
+
+def test_entropy_one_hot_is_zero(oracle):
+    logits = np.full(1000, -np.inf, dtype=np.float32)
+    logits[417] = 3.25
+    s, H = oracle.cogload(logits, 417)
+    assert H == 0.0 and s == 0.0
+    s_other, _ = oracle.cogload(logits, 3)
+    assert s_other == np.inf
+
+
+@pytest.mark.parametrize("a,V", [(5.0, 4096), (-2.0, 100), (12.0, 32000)])
+def test_two_level_closed_form(oracle, a, V):
+    logits = np.zeros(V, dtype=np.float32)
+    logits[7] = a
+    p = math.exp(a) / (math.exp(a) + V - 1)
+    q = (1 - p) / (V - 1)
+    H_ref = -p * math.log(p) - (V - 1) * q * math.log(q)
+    s_peak, H = oracle.cogload(logits, 7)
+    s_rest, _ = oracle.cogload(logits, 8)
+    assert abs(H - H_ref) < 1e-10
+    assert abs(s_peak + math.log(p)) < 1e-10
+    assert abs(s_rest + math.log(q)) < 1e-10
+
+
+def test_cogload_matches_library_log_softmax(oracle):
+    rng = np.random.default_rng(3)
+    for V in (17, 1000, 32000):
+        logits = (rng.standard_normal(V) * 3).astype(np.float32)
+        tok = int(rng.integers(V))
+        lp = scipy.special.log_softmax(logits.astype(np.float64))
+        s, H = oracle.cogload(logits, tok)
+        assert abs(s + lp[tok]) < 1e-10
+        assert abs(H + np.sum(np.exp(lp) * lp)) < 1e-10
+        assert 0.0 <= H <= math.log(V) + 1e-12 and s >= 0.0
+
+
+def test_cogload_shift_invariance_and_bf16(oracle):
+    rng = np.random.default_rng(4)
+    logits = (rng.standard_normal(5000) * 2).astype(np.float32)
+    s0, H0 = oracle.cogload(logits, 11)
+    s1, H1 = oracle.cogload(logits + np.float32(8.0), 11)
+    assert abs(s0 - s1) < 1e-5 and abs(H0 - H1) < 1e-5   # the shift itself rounds in fp32
+    bits = _bf16_bits(logits)
+    lp = scipy.special.log_softmax(_bf16_to_f64(bits))
+    s, H = oracle.cogload(bits, 11)
+    assert abs(s + lp[11]) < 1e-10 and abs(H + np.sum(np.exp(lp) * lp)) < 1e-10
+
+
+def test_cogload_token_out_of_range(oracle):
+    logits = np.zeros(10, dtype=np.float32)
+    s, H = oracle.cogload(logits, 10)
+    assert math.isnan(s) and abs(H - math.log(10)) < 1e-12
+    s, _ = oracle.cogload(logits, -1)
+    assert math.isnan(s)
+
+
+# ----------------------------------------------------------------------------------------------
+# Neuron scores: Eq. neuron_activation
+# ----------------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_scores_literal_frobenius_equals_factored(oracle, dtype):
+    rng = np.random.default_rng(0)
+    X, Wg, Wu, Wd = _layer(rng, d=12, F=9, T=7, dtype=dtype)
+    A = oracle.neuron_scores(X, [0, 7], Wg, Wu, Wd)[0]
+    A_lit = oracle.neuron_scores_literal(X, Wg, Wu, Wd)
+    np.testing.assert_allclose(A, A_lit, rtol=1e-12)
+
+
+def test_scores_against_explicit_matrix_norms(oracle):
+    """numpy builds the matrix [sigma(W_in,j x) * V_in,j x] W_out,j and takes library norms of it."""
+    rng = np.random.default_rng(1)
+    X, Wg, Wu, Wd = _layer(rng, d=10, F=6, T=5)
+    A = oracle.neuron_scores(X, [0, 5], Wg, Wu, Wd)[0]
+    X64, Wg64, Wu64, Wd64 = (a.astype(np.float64) for a in (X, Wg, Wu, Wd))
+    for j in range(6):
+        g = X64 @ Wg64[j]
+        z = g * scipy.special.expit(g) * (X64 @ Wu64[j])
+        M = np.outer(z, Wd64[:, j])            # column j of W_out, T x d_model
+        assert abs(A[j] - np.linalg.norm(M, "fro")) < 1e-12 * max(1.0, A[j])
+        assert abs(A[j] - np.linalg.norm(M, 2)) < 1e-10 * max(1.0, A[j])   # rank one: same number
+
+
+def test_scores_single_token_special_case(oracle):
+    rng = np.random.default_rng(2)
+    X, Wg, Wu, Wd = _layer(rng, d=16, F=8, T=1)
+    A = oracle.neuron_scores(X, [0, 1], Wg, Wu, Wd)[0]
+    x = X[0].astype(np.float64)
+    g = Wg.astype(np.float64) @ x
+    z = g * scipy.special.expit(g) * (Wu.astype(np.float64) @ x)
+    ref = np.abs(z) * np.linalg.norm(Wd.astype(np.float64), axis=0)
+    np.testing.assert_allclose(A, ref, rtol=1e-12)
+
+
+def test_scores_invariances(oracle):
+    rng = np.random.default_rng(5)
+    X, Wg, Wu, Wd = _layer(rng, d=8, F=11, T=12)
+    A = oracle.neuron_scores(X, [0, 12], Wg, Wu, Wd)[0]
+    # token order does not matter
+    perm = rng.permutation(12)
+    np.testing.assert_allclose(oracle.neuron_scores(X[perm], [0, 12], Wg, Wu, Wd)[0], A, rtol=1e-12)
+    # squares add across token chunks; ragged offsets index the right rows
+    parts = oracle.neuron_scores(X, [0, 5, 5, 12], Wg, Wu, Wd)
+    assert np.all(parts[1] == 0.0)
+    np.testing.assert_allclose(np.sqrt(parts[0] ** 2 + parts[2] ** 2), A, rtol=1e-12)
+    # permuting neurons permutes scores
+    q = rng.permutation(11)
+    Aq = oracle.neuron_scores(X, [0, 12], Wg[q], Wu[q], Wd[:, q])[0]
+    np.testing.assert_allclose(Aq, A[q], rtol=1e-12)
+    # gate and up are not interchangeable (silu acts on the gate only)
+    A_swapped = oracle.neuron_scores(X, [0, 12], Wu, Wg, Wd)[0]
+    assert np.max(np.abs(A_swapped - A) / A) > 1e-3
+
+
+def test_scores_tie_to_per_token_neuron_outputs(oracle):
+    """sum_t ||n_j(x_t)||^2 = A_j^2, n_j(x_t) obtained from the sparse FFN with only neuron j kept."""
+    rng = np.random.default_rng(6)
+    X, Wg, Wu, Wd = _layer(rng, d=8, F=5, T=6)
+    A = oracle.neuron_scores(X, [0, 6], Wg, Wu, Wd)[0]
+    for j in range(5):
+        only_j = np.zeros(5)
+        only_j[j] = 1.0
+        tot = 0.0
+        for t in range(6):
+            n_j, mask, cnt = oracle.sparse_ffn(X[t], Wg, Wu, Wd, only_j, 0.5)
+            assert cnt == 1 and mask[j] == 1
+            tot += float(np.sum(n_j ** 2))
+        assert abs(math.sqrt(tot) - A[j]) < 1e-12 * max(1.0, A[j])
+
+
+# ----------------------------------------------------------------------------------------------
+# Selection: S_cut = { j : A_j < eps }
+# ----------------------------------------------------------------------------------------------
+
+def test_select_brute_force_tiny(oracle):
+    rng = np.random.default_rng(7)
+    for F in (1, 2, 7, 16):
+        A = rng.random(F) + 0.1
+        order = np.sort(A)
+        cuts = [0.0, order[0]] + [0.5 * (order[i] + order[i + 1]) for i in range(F - 1)] + [order[-1], np.inf]
+        prev = None
+        for tau in cuts:
+            mask, idx, count = oracle.select(A, tau)
+            keep = [j for j in range(F) if A[j] >= tau]
+            assert list(idx) == keep and count == len(keep)
+            assert list(np.nonzero(mask)[0]) == keep
+            if prev is not None:
+                assert set(keep) <= prev          # nested as tau grows
+            prev = set(keep)
+        assert oracle.select(A, order[0])[2] == F          # tau <= min keeps all; equality keeps
+        assert oracle.select(A, np.inf)[2] == 0
+
+
+def test_select_rank_count(oracle):
+    rng = np.random.default_rng(8)
+    A = rng.random(16)
+    order = np.sort(A)
+    for r in range(15):
+        tau = 0.5 * (order[r] + order[r + 1])
+        assert oracle.select(A, tau)[2] == 16 - (r + 1)
+
+
+def test_tau_from_sparsity_cuts_k(oracle):
+    rng = np.random.default_rng(9)
+    A = rng.random(1376).astype(np.float32)
+    for rho in (0.0, 0.3, 0.4, 0.5, 0.6, 1.0):
+        tau = oracle.tau_from_sparsity(A, rho)
+        k_cut = int(math.floor(rho * 1376 + 0.5))
+        assert oracle.select(A.astype(np.float64), float(tau))[2] == 1376 - k_cut
+
+
+# ----------------------------------------------------------------------------------------------
+# Threshold adjustment: Eq. final_threshold
+# ----------------------------------------------------------------------------------------------
+
+def test_adjust_four_cases(oracle):
+    tb = np.array([[0.37, 1.5, 2.25]] * 4, dtype=np.float32)
+    lam = np.full(3, 0.80, dtype=np.float32)
+    gam = np.full(3, 0.12, dtype=np.float32)
+    s = np.array([1.0, 3.0, 1.0, 3.0])
+    H = np.array([1.0, 1.0, 5.0, 5.0])
+    out = oracle.adjust_threshold(tb, lam, gam, 2.0, 4.0, s, H)
+    one = np.float32(1.0)
+    mults = [one, one + np.float32(0.80), one + np.float32(0.12),
+             (one + np.float32(0.80)) + np.float32(0.12)]
+    for b in range(4):
+        np.testing.assert_array_equal(out[b], tb[b] * mults[b])
+    # against the exact rationals 1, 1.8, 1.12, 1.92 to fp32 rounding
+    np.testing.assert_allclose(out[:, 0].astype(np.float64) / 0.37,
+                               [1.0, 1.8, 1.12, 1.92], rtol=3e-7)
+
+
+def test_adjust_strict_and_signed(oracle):
+    tb = np.array([[2.0]], dtype=np.float32)
+    lam = np.array([0.80], dtype=np.float32)
+    gam = np.array([0.12], dtype=np.float32)
+    # equality does not trigger: I(s > tau_s)
+    assert oracle.adjust_threshold(tb, lam, gam, 2.0, 4.0, [2.0], [4.0])[0, 0] == np.float32(2.0)
+    # coefficients are signed inputs
+    out = oracle.adjust_threshold(tb, -lam, -gam, 2.0, 4.0, [2.5], [4.5])
+    assert out[0, 0] == np.float32(2.0) * ((np.float32(1.0) - np.float32(0.80)) - np.float32(0.12))
+    # lambda = gamma = 0: thresholds unchanged
+    z = np.zeros(1, dtype=np.float32)
+    assert oracle.adjust_threshold(tb, z, z, 2.0, 4.0, [9.0], [9.0])[0, 0] == np.float32(2.0)
+    # per-layer coefficients index by layer, thresholds by (sequence, layer)
+    tb2 = np.array([[1.0, 2.0], [3.0, 4.0]], dtype=np.float32)
+    lam2 = np.array([0.5, 0.25], dtype=np.float32)
+    out = oracle.adjust_threshold(tb2, lam2, np.zeros(2, np.float32), 0.0, 0.0, [1.0, -1.0], [0.0, 0.0])
+    np.testing.assert_array_equal(out, np.array([[1.5, 2.5], [3.0, 4.0]], dtype=np.float32))
+
+
+# ----------------------------------------------------------------------------------------------
+# FFN: Algorithm 2, sparse forward pass
+# ----------------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_dense_ffn_matches_matrix_formulation(oracle, dtype):
+    rng = np.random.default_rng(10)
+    X, Wg, Wu, Wd = _layer(rng, d=24, F=40, T=3, dtype=dtype)
+    tX, tWg, tWu, tWd = (torch.from_numpy(_f64(a)) for a in (X, Wg, Wu, Wd))
+    ref = (torch.nn.functional.silu(tX @ tWg.T) * (tX @ tWu.T)) @ tWd.T
+    for t in range(3):
+        y = oracle.dense_ffn(X[t], Wg, Wu, Wd)
+        np.testing.assert_allclose(y, ref[t].numpy(), rtol=1e-11, atol=1e-13)
+
+
+def test_zero_sparsity_is_dense_bit_for_bit(oracle):
+    rng = np.random.default_rng(11)
+    X, Wg, Wu, Wd = _layer(rng, d=16, F=30, T=4)
+    A = oracle.neuron_scores(X, [0, 4], Wg, Wu, Wd)[0]
+    for t in range(4):
+        y_s, mask, cnt = oracle.sparse_ffn(X[t], Wg, Wu, Wd, A, A.min())
+        assert cnt == 30 and mask.all()
+        assert np.array_equal(y_s, oracle.dense_ffn(X[t], Wg, Wu, Wd))
+    y_none, mask, cnt = oracle.sparse_ffn(X[0], Wg, Wu, Wd, A, np.inf)
+    assert cnt == 0 and not mask.any() and np.all(y_none == 0.0)
+
+
+def test_sparse_ffn_is_masked_matrix_product(oracle):
+    rng = np.random.default_rng(12)
+    X, Wg, Wu, Wd = _layer(rng, d=16, F=30, T=8)
+    A = oracle.neuron_scores(X, [0, 8], Wg, Wu, Wd)[0]
+    tau = float(np.median(A))
+    keep = torch.from_numpy(A >= tau)
+    tX, tWg, tWu, tWd = (torch.from_numpy(a.astype(np.float64)) for a in (X, Wg, Wu, Wd))
+    h = torch.nn.functional.silu(tX @ tWg.T) * (tX @ tWu.T)
+    ref = (h * keep) @ tWd.T
+    for t in range(8):
+        y, mask, cnt = oracle.sparse_ffn(X[t], Wg, Wu, Wd, A, tau)
+        assert cnt == int(keep.sum()) and np.array_equal(mask.astype(bool), keep.numpy())
+        np.testing.assert_allclose(y, ref[t].numpy(), rtol=1e-11, atol=1e-13)
+
+
+def test_cett_identity_and_prefix_bound(oracle):
+    """dense - sparse = sum of the cut neurons' outputs, so CETT = ||dense - sparse|| / ||dense||;
+    over the prefix, ||Y_dense - Y_sparse||_F <= sum_{cut} A_j (triangle inequality)."""
+    rng = np.random.default_rng(13)
+    T, F = 6, 20
+    X, Wg, Wu, Wd = _layer(rng, d=12, F=F, T=T)
+    A = oracle.neuron_scores(X, [0, T], Wg, Wu, Wd)[0]
+    tau = float(np.sort(A)[8] * 0.5 + np.sort(A)[9] * 0.5)
+    cut = np.nonzero(A < tau)[0]
+    assert len(cut) == 9
+    diff_fro2 = 0.0
+    for t in range(T):
+        y_d = oracle.dense_ffn(X[t], Wg, Wu, Wd)
+        y_s, _, _ = oracle.sparse_ffn(X[t], Wg, Wu, Wd, A, tau)
+        n_cut = np.zeros(12)
+        for j in cut:
+            e = np.zeros(F)
+            e[j] = 1.0
+            n_cut += oracle.sparse_ffn(X[t], Wg, Wu, Wd, e, 0.5)[0]
+        np.testing.assert_allclose(y_d - y_s, n_cut, rtol=1e-9, atol=1e-12)
+        cett = np.linalg.norm(n_cut) / np.linalg.norm(y_d)
+        assert abs(cett - np.linalg.norm(y_d - y_s) / np.linalg.norm(y_d)) < 1e-9
+        diff_fro2 += float(np.sum((y_d - y_s) ** 2))
+    assert math.sqrt(diff_fro2) <= float(np.sum(A[cut])) * (1 + 1e-12)
