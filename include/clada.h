@@ -1,0 +1,199 @@
+/*
+ * clada.h -- C ABI of the B200 (sm_100a) CLADA sparse gated FFN decode path.
+ *
+ * The library realises the data-parallel hot path of "Cognitive-Load-Aware
+ * Dynamic Activation" (Algorithm 2 of the paper):
+ *
+ *   prefill :  per-neuron activation magnitudes A_j over the prompt
+ *              (Eq. neuron_activation) and the baseline neuron subset
+ *              { j : A_j >= tau_base } (Eq. base_threshold, last line);
+ *   per step:  surprisal s_t and entropy H_t of the previous step's
+ *              vocabulary distribution (Eqs. surprisal, entropy);
+ *              tau_final = tau_base * (1 + lambda I(s_t > tau_s) + gamma I(H_t > tau_H))
+ *              (Eq. final_threshold);
+ *              mask regeneration A_j >= tau_final and the gated FFN over the
+ *              kept neurons only (Algorithm 2, generation phase).
+ *
+ * Conventions
+ * -----------
+ *  - Unless a parameter says "host", every pointer is a DEVICE pointer owned
+ *    by the caller.  The library allocates no device memory; scratch comes
+ *    from a caller-provided workspace (clada_workspace_bytes / clada_workspace_init).
+ *  - Calls validate on the host, enqueue their kernels on `stream`
+ *    (a cudaStream_t passed as void*, NULL = default stream) and return
+ *    without synchronising.
+ *  - Matrices are row-major and dense.  Weight rows and x / X rows must start
+ *    on 16-byte boundaries and d_model must be a multiple of 8.
+ *  - Return value: CLADA_OK, or a negative clada_error; on error nothing was
+ *    enqueued.  Conditions only the device can see (token id out of range,
+ *    non-finite logit, a bounded wait that expired) OR bits of clada_status
+ *    into the optional device word `status`; kernels never trap.
+ *  - Two calls may run concurrently only with distinct workspaces.
+ */
+#ifndef CLADA_H_
+#define CLADA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum { CLADA_F32 = 0, CLADA_BF16 = 1 } clada_dtype;
+
+typedef enum {
+    CLADA_OK = 0,
+    CLADA_ERR_NULL = -1,      /* a required pointer is NULL */
+    CLADA_ERR_SHAPE = -2,     /* a size is <= 0, d_model % 8 != 0, offsets not ascending, ... */
+    CLADA_ERR_ALIGN = -3,     /* a row base is not 16-byte aligned */
+    CLADA_ERR_DTYPE = -4,     /* unknown or unsupported clada_dtype */
+    CLADA_ERR_WORKSPACE = -5, /* workspace missing, misaligned or too small */
+    CLADA_ERR_CUDA = -6,      /* a CUDA runtime call failed: see clada_last_cuda_error() */
+    CLADA_ERR_UNSUPPORTED = -7 /* sizes beyond what the kernels were built for */
+} clada_error;
+
+typedef enum {
+    CLADA_STATUS_BAD_TOKEN = 1,        /* token_id outside [0, V): surprisal = NaN */
+    CLADA_STATUS_NONFINITE_LOGIT = 2,  /* +inf or NaN logit: surprisal = entropy = NaN */
+    CLADA_STATUS_TIMEOUT = 4           /* a bounded device-side wait gave up; outputs invalid,
+                                          re-initialise the workspace before reusing it */
+} clada_status;
+
+/* One gated FFN layer.  Neuron j owns row j of each matrix, so its three
+ * vectors are contiguous: w_gate row j = W_in,j, w_up row j = V_in,j,
+ * w_down_t row j = column j of the output projection W_out
+ * (text under Eq. neuron_activation). */
+typedef struct clada_layer {
+    int32_t d_model;          /* multiple of 8; <= 8192 (bf16) or 4096 (fp32) */
+    int32_t d_ff;
+    int32_t dtype;            /* clada_dtype of the weights and of x / X */
+    int32_t reserved;         /* set to 0 */
+    const void *w_gate;       /* [d_ff, d_model] */
+    const void *w_up;         /* [d_ff, d_model] */
+    const void *w_down_t;     /* [d_ff, d_model] */
+    const float *w_down_norm; /* [d_ff] ||W_out,j||_2 (clada_down_norms); needed by the prefix calls only */
+} clada_layer;
+
+int clada_version(void);
+const char *clada_status_string(int code);
+/* Text of the last CUDA error seen by this thread's calls ("" if none). Host. */
+const char *clada_last_cuda_error(void);
+
+/* Bytes of workspace that suffice for any call on this layer with B
+ * sequences and T_total prefix tokens in all (T_total = 0 for decode-only use).
+ * 0 on invalid arguments. */
+size_t clada_workspace_bytes(const clada_layer *layer, int32_t B, int64_t T_total);
+
+/* Zero the workspace's control words.  Once after allocation, and again after
+ * a CLADA_STATUS_TIMEOUT.  ws must be 256-byte aligned. */
+int clada_workspace_init(void *ws, size_t ws_bytes, void *stream);
+
+/* out[j] = ||W_out,j||_2 = the l2 norm of row j of w_down_t, fp32.  Once per
+ * layer; the second factor of Eq. neuron_activation. */
+int clada_down_norms(const clada_layer *layer, float *out /*[d_ff]*/, void *stream);
+
+/* Eq. neuron_activation over B prompts (B <= 128).
+ *   X            [T_total, d_model], the layer's input hidden states of all
+ *                prompts back to back, in the weights' dtype
+ *   seq_offsets  HOST int64 [B+1], ascending; prompt b = rows
+ *                [seq_offsets[b], seq_offsets[b+1]); an empty prompt scores 0
+ *   scores       out [B, d_ff] fp32:
+ *                A[b,j] = sqrt(sum_t z_tj^2) * w_down_norm[j],
+ *                z_tj = silu(w_gate_j . x_t) * (w_up_j . x_t)
+ * Products of the stored values are exact; accumulation is fp32. */
+int clada_prefix_scores(const clada_layer *layer, const void *X, const int64_t *seq_offsets,
+                        int32_t B, float *scores, void *ws, size_t ws_bytes,
+                        int32_t *status, void *stream);
+
+/* Guard band.  Every neuron whose fp32 score lies within rel_band (relative)
+ * of tau_base[b] * guard_mults[g] for some g gets its score recomputed with
+ * fp64 accumulation and stored back rounded to fp32, so that the later
+ * comparisons A_j >= tau are taken on correctly rounded scores where it
+ * matters.  guard_mults: HOST [n_guard] (the multipliers decode will apply,
+ * e.g. 1, 1+lambda, 1+gamma, 1+lambda+gamma), n_guard <= 8.
+ * The paper has no counterpart; it only removes rounding noise from the
+ * comparison the paper defines. */
+int clada_refine_scores(const clada_layer *layer, const void *X, const int64_t *seq_offsets,
+                        int32_t B, const float *tau_base /*[B]*/, const float *guard_mults,
+                        int32_t n_guard, float rel_band, float *scores /*[B,d_ff] in/out*/,
+                        void *ws, size_t ws_bytes, int32_t *status, void *stream);
+
+/* Eq. base_threshold, last line, and Algorithm 2's mask generation: neuron j
+ * of sequence b is kept iff scores[b,j] >= tau[b*tau_stride] (equality keeps;
+ * NaN scores are cut).
+ *   mask  out [B, d_ff] u8 (1 = kept), may be NULL
+ *   idx   out [B, d_ff] int32, the kept neurons of b ascending in
+ *         idx[b*d_ff .. b*d_ff+count[b]); the rest is left untouched; may be NULL
+ *   count out [B] int32, may be NULL */
+int clada_select(const float *scores, int32_t B, int32_t d_ff, const float *tau,
+                 int64_t tau_stride, uint8_t *mask, int32_t *idx, int32_t *count,
+                 void *stream);
+
+/* Prefill phase of Algorithm 2 in one call: clada_prefix_scores, then (if
+ * n_guard > 0) clada_refine_scores with rel_band 1e-4, then clada_select
+ * against tau_base.  tau_base == NULL stops after the scores (used to
+ * calibrate a threshold first). */
+int clada_prefix_select(const clada_layer *layer, const void *X, const int64_t *seq_offsets,
+                        int32_t B, const float *tau_base /*[B] or NULL*/,
+                        const float *guard_mults /*host, may be NULL*/, int32_t n_guard,
+                        float *scores, uint8_t *mask, int32_t *idx, int32_t *count,
+                        void *ws, size_t ws_bytes, int32_t *status, void *stream);
+
+/* Harness helper standing in for the offline threshold search (which is an
+ * input to this path): tau_base[b] = 0.5*a + 0.5*b in fp32, a and b the
+ * k_cut-th and (k_cut+1)-th smallest of scores[b,:], k_cut = floor(rho*d_ff + 0.5),
+ * i.e. the threshold that cuts exactly k_cut neurons.  k_cut = 0 gives 0,
+ * k_cut = d_ff gives +inf.  Scores must be non-negative (they are norms). */
+int clada_tau_from_sparsity(const float *scores, int32_t B, int32_t d_ff, float rho,
+                            float *tau_base /*[B]*/, void *stream);
+
+/* Eqs. surprisal and entropy, natural log, for B vocabulary rows:
+ *   P = softmax(logits[b,:]);  surprisal[b] = -log P[token_id[b]];
+ *   entropy[b] = -sum_w P[w] log P[w]   (0 log 0 = 0: -inf logits allowed).
+ *   logits     [B, V] with row stride row_stride elements, fp32 or bf16
+ *   token_id   [B] int32
+ * Out-of-range token -> surprisal NaN + CLADA_STATUS_BAD_TOKEN;
+ * +inf / NaN logit -> both NaN + CLADA_STATUS_NONFINITE_LOGIT. */
+int clada_cogload(const void *logits, int32_t logits_dtype, int32_t B, int64_t V,
+                  int64_t row_stride, const int32_t *token_id, float *surprisal,
+                  float *entropy, int32_t *status, void *stream);
+
+/* Eq. final_threshold for B sequences and L layers, fp32, evaluated left to
+ * right without fused multiply-add:
+ *   m = 1; if (surprisal[b] > tau_s) m += lambda[l]; if (entropy[b] > tau_H) m += gamma[l];
+ *   tau_final[b,l] = tau_base[b,l] * m
+ * lambda, gamma: [L] signed per-layer coefficients (the paper picks 0.80, 0.12). */
+int clada_adjust_threshold(const float *tau_base /*[B,L]*/, const float *lambda,
+                           const float *gamma, float tau_s, float tau_H,
+                           const float *surprisal /*[B]*/, const float *entropy /*[B]*/,
+                           int32_t B, int32_t L, float *tau_final /*[B,L]*/, void *stream);
+
+/* clada_cogload followed by clada_adjust_threshold in one launch (the two
+ * per-step scalar stages of Algorithm 2's generation loop).  surprisal and
+ * entropy are still written. */
+int clada_cogload_adjust(const void *logits, int32_t logits_dtype, int32_t B, int64_t V,
+                         int64_t row_stride, const int32_t *token_id,
+                         const float *tau_base, const float *lambda, const float *gamma,
+                         float tau_s, float tau_H, int32_t L, float *surprisal,
+                         float *entropy, float *tau_final, int32_t *status, void *stream);
+
+/* Algorithm 2, generation phase, one layer, one token per sequence:
+ *   kept_b = { j : scores[b,j] >= tau_final[b*tau_stride] }
+ *   y[b,:] = sum_{j in kept_b} silu(w_gate_j . x_b) * (w_up_j . x_b) * w_down_t[j,:]
+ * Only the kept neurons' rows are read.  No bias, no rescaling.
+ *   x        [B, d_model] in the layer's dtype
+ *   y        out [B, d_model], y_dtype fp32 or bf16
+ *   mask_out / idx_out / count_out: optional (NULL), as in clada_select
+ * Accumulation is fp32 in a fixed order: results are bit-identical run to run.
+ * The workspace must have been initialised with clada_workspace_init. */
+int clada_sparse_ffn_decode(const clada_layer *layer, const void *x, int32_t B,
+                            const float *scores /*[B,d_ff]*/, const float *tau_final,
+                            int64_t tau_stride, void *y, int32_t y_dtype,
+                            uint8_t *mask_out, int32_t *idx_out, int32_t *count_out,
+                            void *ws, size_t ws_bytes, int32_t *status, void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CLADA_H_ */
