@@ -1,0 +1,245 @@
+// Per-token cognitive load (Eqs. surprisal, entropy) and the token-aware threshold
+// (Eq. final_threshold).
+//
+// One CTA per vocabulary row.  Each thread streams 16-byte vectors of logits and keeps a running
+// (max m, Z = sum e^{l-m}, W = sum e^{l-m}(l-m)); triples are merged by warp shuffles, then across
+// warps through shared memory, always in the same order.  With logZ = log Z:
+//   surprisal = m + logZ - l[token],   entropy = logZ - W / Z.
+#include <math.h>
+
+#include "common.cuh"
+
+namespace clada {
+
+struct SoftStat {
+    float m, z, w;
+};
+
+__device__ __forceinline__ SoftStat stat_empty() { return SoftStat{-INFINITY, 0.f, 0.f}; }
+
+// Move a statistic to a new (not smaller) reference maximum.
+__device__ __forceinline__ void stat_rebase(SoftStat &a, float m_new) {
+    if (a.m == -INFINITY) {
+        a.m = m_new;  // nothing accumulated yet
+        return;
+    }
+    const float dm = a.m - m_new;  // <= 0
+    const float sc = expf(dm);
+    a.w = (a.w + dm * a.z) * sc;
+    a.z = a.z * sc;
+    a.m = m_new;
+}
+
+__device__ __forceinline__ SoftStat stat_merge(SoftStat a, SoftStat b) {
+    const float m = fmaxf(a.m, b.m);
+    if (m == -INFINITY) return a;
+    stat_rebase(a, m);
+    stat_rebase(b, m);
+    return SoftStat{m, a.z + b.z, a.w + b.w};
+}
+
+template <int N>
+__device__ __forceinline__ void stat_add(SoftStat &a, const float (&l)[N], bool &bad) {
+    float cm = -INFINITY;
+#pragma unroll
+    for (int i = 0; i < N; ++i) {
+        bad |= !(l[i] < INFINITY);  // +inf or NaN
+        cm = fmaxf(cm, l[i]);
+    }
+    if (cm == -INFINITY) return;  // the whole chunk has probability zero
+    if (cm > a.m) stat_rebase(a, cm);
+#pragma unroll
+    for (int i = 0; i < N; ++i) {
+        const float t = l[i] - a.m;
+        const float e = expf(t);
+        a.z += e;
+        a.w += (t == -INFINITY) ? 0.f : e * t;
+    }
+}
+
+template <typename T>
+__device__ __forceinline__ float load_logit(const T *row, int64_t i) {
+    return Elem<T>::to_float(row[i]);
+}
+
+constexpr int kCogThreads = 1024;
+
+// tau_base == nullptr: cognitive load only.
+template <typename T>
+__global__ void __launch_bounds__(kCogThreads)
+cogload_kernel(const T *__restrict__ logits, int64_t V, int64_t row_stride,
+               const int32_t *__restrict__ token_id, float *__restrict__ surprisal,
+               float *__restrict__ entropy, int32_t *__restrict__ status,
+               const float *__restrict__ tau_base, const float *__restrict__ lambda,
+               const float *__restrict__ gamma, float tau_s, float tau_H, int L,
+               float *__restrict__ tau_final) {
+    constexpr int E = Elem<T>::kPerVec;
+    const int b = blockIdx.x;
+    const T *row = logits + (size_t)b * row_stride;
+    const int tid = threadIdx.x;
+
+    SoftStat st = stat_empty();
+    bool bad = false;
+
+    // Scalar head up to the first 16-byte boundary, vector body, scalar tail.
+    const uintptr_t addr = reinterpret_cast<uintptr_t>(row);
+    int64_t head = ((16 - (addr & 15)) & 15) / sizeof(T);
+    if (head > V) head = V;
+    const int64_t nvec = (V - head) / E;
+    const int64_t tail0 = head + nvec * E;
+    if (tid < head) {
+        float l[1] = {load_logit(row, tid)};
+        stat_add(st, l, bad);
+    }
+    const uint4 *vrow = reinterpret_cast<const uint4 *>(row + head);
+    int64_t v = tid;
+    // four vectors in flight per thread
+    for (; v + 3 * (int64_t)kCogThreads < nvec; v += 4 * (int64_t)kCogThreads) {
+        uint4 q[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) q[u] = ldg_stream(vrow + v + u * (int64_t)kCogThreads);
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            float l[E];
+            Elem<T>::unpack(q[u], l);
+            stat_add(st, l, bad);
+        }
+    }
+    for (; v < nvec; v += kCogThreads) {
+        float l[E];
+        Elem<T>::unpack(ldg_stream(vrow + v), l);
+        stat_add(st, l, bad);
+    }
+    if (tail0 + tid < V) {
+        float l[1] = {load_logit(row, tail0 + tid)};
+        stat_add(st, l, bad);
+    }
+
+    // warp, then CTA merge in a fixed order
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        SoftStat other;
+        other.m = __shfl_xor_sync(0xffffffffu, st.m, o);
+        other.z = __shfl_xor_sync(0xffffffffu, st.z, o);
+        other.w = __shfl_xor_sync(0xffffffffu, st.w, o);
+        st = ((tid & o) == 0) ? stat_merge(st, other) : stat_merge(other, st);
+    }
+    __shared__ SoftStat s_stat[kCogThreads / kWarp];
+    __shared__ int s_bad;
+    __shared__ float s_out[2];
+    if (tid == 0) s_bad = 0;
+    __syncthreads();
+    if (bad) atomicOr(&s_bad, 1);
+    if ((tid & 31) == 0) s_stat[tid >> 5] = st;
+    __syncthreads();
+    if (tid == 0) {
+        SoftStat tot = s_stat[0];
+        for (int w = 1; w < kCogThreads / kWarp; ++w) tot = stat_merge(tot, s_stat[w]);
+        int flags = 0;
+        float s, h;
+        if (s_bad || !(tot.z > 0.f)) {  // a +inf / NaN logit, or no finite logit at all
+            flags |= CLADA_STATUS_NONFINITE_LOGIT;
+            s = h = NAN;
+        } else {
+            const float logz = logf(tot.z);
+            h = logz - tot.w / tot.z;
+            const int32_t tok = token_id[b];
+            if (tok < 0 || tok >= V) {
+                flags |= CLADA_STATUS_BAD_TOKEN;
+                s = NAN;
+            } else {
+                s = (tot.m + logz) - load_logit(row, tok);
+            }
+        }
+        surprisal[b] = s;
+        entropy[b] = h;
+        s_out[0] = s;
+        s_out[1] = h;
+        if (flags && status) atomicOr(status, flags);
+    }
+    if (tau_base == nullptr) return;
+    __syncthreads();
+    const float s = s_out[0], h = s_out[1];
+    for (int l = tid; l < L; l += kCogThreads) {
+        float mult = 1.0f;
+        if (s > tau_s) mult = __fadd_rn(mult, lambda[l]);
+        if (h > tau_H) mult = __fadd_rn(mult, gamma[l]);
+        tau_final[(size_t)b * L + l] = __fmul_rn(tau_base[(size_t)b * L + l], mult);
+    }
+}
+
+__global__ void adjust_threshold_kernel(const float *__restrict__ tau_base,
+                                        const float *__restrict__ lambda,
+                                        const float *__restrict__ gamma, float tau_s, float tau_H,
+                                        const float *__restrict__ surprisal,
+                                        const float *__restrict__ entropy, int B, int L,
+                                        float *__restrict__ tau_final) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= B * L) return;
+    const int b = i / L, l = i % L;
+    float mult = 1.0f;
+    if (surprisal[b] > tau_s) mult = __fadd_rn(mult, lambda[l]);
+    if (entropy[b] > tau_H) mult = __fadd_rn(mult, gamma[l]);
+    tau_final[i] = __fmul_rn(tau_base[i], mult);
+}
+
+static int launch_cogload(const void *logits, int32_t dtype, int32_t B, int64_t V, int64_t row_stride,
+                          const int32_t *token_id, float *surprisal, float *entropy,
+                          int32_t *status, const float *tau_base, const float *lambda,
+                          const float *gamma, float tau_s, float tau_H, int L, float *tau_final,
+                          void *stream) {
+    if (!logits || !token_id || !surprisal || !entropy) return CLADA_ERR_NULL;
+    if (dtype != CLADA_F32 && dtype != CLADA_BF16) return CLADA_ERR_DTYPE;
+    if (B <= 0 || V <= 0 || row_stride < V) return CLADA_ERR_SHAPE;
+    if (reinterpret_cast<uintptr_t>(logits) % elem_size(dtype)) return CLADA_ERR_ALIGN;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (dtype == CLADA_F32)
+        cogload_kernel<float><<<B, kCogThreads, 0, st>>>(
+            static_cast<const float *>(logits), V, row_stride, token_id, surprisal, entropy, status,
+            tau_base, lambda, gamma, tau_s, tau_H, L, tau_final);
+    else
+        cogload_kernel<__nv_bfloat16><<<B, kCogThreads, 0, st>>>(
+            static_cast<const __nv_bfloat16 *>(logits), V, row_stride, token_id, surprisal, entropy,
+            status, tau_base, lambda, gamma, tau_s, tau_H, L, tau_final);
+    CLADA_CUDA_TRY(cudaGetLastError());
+    return CLADA_OK;
+}
+
+}  // namespace clada
+
+using namespace clada;
+
+extern "C" {
+
+int clada_cogload(const void *logits, int32_t logits_dtype, int32_t B, int64_t V, int64_t row_stride,
+                  const int32_t *token_id, float *surprisal, float *entropy, int32_t *status,
+                  void *stream) {
+    return launch_cogload(logits, logits_dtype, B, V, row_stride, token_id, surprisal, entropy, status,
+                          nullptr, nullptr, nullptr, 0.f, 0.f, 0, nullptr, stream);
+}
+
+int clada_adjust_threshold(const float *tau_base, const float *lambda, const float *gamma, float tau_s,
+                           float tau_H, const float *surprisal, const float *entropy, int32_t B,
+                           int32_t L, float *tau_final, void *stream) {
+    if (!tau_base || !lambda || !gamma || !surprisal || !entropy || !tau_final) return CLADA_ERR_NULL;
+    if (B <= 0 || L <= 0) return CLADA_ERR_SHAPE;
+    const int threads = 128;
+    const int blocks = (B * L + threads - 1) / threads;
+    adjust_threshold_kernel<<<blocks, threads, 0, static_cast<cudaStream_t>(stream)>>>(
+        tau_base, lambda, gamma, tau_s, tau_H, surprisal, entropy, B, L, tau_final);
+    CLADA_CUDA_TRY(cudaGetLastError());
+    return CLADA_OK;
+}
+
+int clada_cogload_adjust(const void *logits, int32_t logits_dtype, int32_t B, int64_t V,
+                         int64_t row_stride, const int32_t *token_id, const float *tau_base,
+                         const float *lambda, const float *gamma, float tau_s, float tau_H, int32_t L,
+                         float *surprisal, float *entropy, float *tau_final, int32_t *status,
+                         void *stream) {
+    if (!tau_base || !lambda || !gamma || !tau_final) return CLADA_ERR_NULL;
+    if (L <= 0) return CLADA_ERR_SHAPE;
+    return launch_cogload(logits, logits_dtype, B, V, row_stride, token_id, surprisal, entropy, status,
+                          tau_base, lambda, gamma, tau_s, tau_H, L, tau_final, stream);
+}
+
+}  // extern "C"

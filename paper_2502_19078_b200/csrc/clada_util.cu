@@ -1,0 +1,140 @@
+// Library plumbing: version, error strings, device info, workspace, down-projection norms.
+#include <stdio.h>
+#include <string.h>
+
+#include "common.cuh"
+
+namespace clada {
+
+static thread_local char g_last_error[512] = "";
+
+void set_last_cuda_error(cudaError_t e, const char *where) {
+    snprintf(g_last_error, sizeof g_last_error, "%s: %s (%s)", where, cudaGetErrorName(e),
+             cudaGetErrorString(e));
+}
+
+int cuda_fail(cudaError_t e, const char *where) {
+    set_last_cuda_error(e, where);
+    (void)cudaGetLastError();  // clear a non-sticky error so the next call starts clean
+    return CLADA_ERR_CUDA;
+}
+
+int validate_layer(const clada_layer *layer, bool need_norm) {
+    if (!layer || !layer->w_gate || !layer->w_up || !layer->w_down_t) return CLADA_ERR_NULL;
+    if (need_norm && !layer->w_down_norm) return CLADA_ERR_NULL;
+    if (layer->dtype != CLADA_F32 && layer->dtype != CLADA_BF16) return CLADA_ERR_DTYPE;
+    if (layer->d_model <= 0 || layer->d_ff <= 0 || layer->d_model % 8 != 0) return CLADA_ERR_SHAPE;
+    const int max_d = layer->dtype == CLADA_BF16 ? kMaxDModel : kMaxDModel / 2;
+    if (layer->d_model > max_d) return CLADA_ERR_UNSUPPORTED;
+    if (!aligned16(layer->w_gate) || !aligned16(layer->w_up) || !aligned16(layer->w_down_t))
+        return CLADA_ERR_ALIGN;
+    return CLADA_OK;
+}
+
+int device_info(DeviceInfo *out) {
+    constexpr int kMaxDev = 64;
+    static DeviceInfo cache[kMaxDev];
+    static bool have[kMaxDev] = {};
+    int dev = 0;
+    CLADA_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev >= 0 && dev < kMaxDev && have[dev]) {
+        *out = cache[dev];
+        return CLADA_OK;
+    }
+    DeviceInfo di;
+    di.device = dev;
+    CLADA_CUDA_TRY(cudaDeviceGetAttribute(&di.num_sms, cudaDevAttrMultiProcessorCount, dev));
+    CLADA_CUDA_TRY(cudaDeviceGetAttribute(&di.max_smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev));
+    if (dev >= 0 && dev < kMaxDev) {
+        cache[dev] = di;
+        have[dev] = true;
+    }
+    *out = di;
+    return CLADA_OK;
+}
+
+// Row norms of w_down_t: one warp per row, 16-byte loads, fp32 accumulation.
+template <typename T>
+__global__ void down_norms_kernel(const T *__restrict__ w, int d_model, int d_ff, float *__restrict__ out) {
+    constexpr int E = Elem<T>::kPerVec;
+    const int warp = (blockIdx.x * blockDim.x + threadIdx.x) / kWarp;
+    const int lane = threadIdx.x % kWarp;
+    if (warp >= d_ff) return;
+    const uint4 *row = reinterpret_cast<const uint4 *>(w + (size_t)warp * d_model);
+    const int nvec = d_model / E;
+    float acc = 0.f;
+    for (int v = lane; v < nvec; v += kWarp) {
+        float f[E];
+        Elem<T>::unpack(ldg_stream(row + v), f);
+#pragma unroll
+        for (int i = 0; i < E; ++i) acc = fmaf(f[i], f[i], acc);
+    }
+    acc = warp_sum(acc);
+    if (lane == 0) out[warp] = sqrtf(acc);
+}
+
+}  // namespace clada
+
+using namespace clada;
+
+extern "C" {
+
+int clada_version(void) { return 100; }
+
+const char *clada_status_string(int code) {
+    switch (code) {
+        case CLADA_OK: return "ok";
+        case CLADA_ERR_NULL: return "a required pointer is NULL";
+        case CLADA_ERR_SHAPE: return "invalid size or shape";
+        case CLADA_ERR_ALIGN: return "pointer not 16-byte aligned";
+        case CLADA_ERR_DTYPE: return "unknown or unsupported dtype";
+        case CLADA_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+        case CLADA_ERR_CUDA: return "CUDA runtime error (see clada_last_cuda_error)";
+        case CLADA_ERR_UNSUPPORTED: return "size beyond what the kernels support";
+        default: return "unknown status";
+    }
+}
+
+const char *clada_last_cuda_error(void) { return g_last_error; }
+
+size_t clada_workspace_bytes(const clada_layer *layer, int32_t B, int64_t T_total) {
+    if (!layer || B <= 0 || T_total < 0 || layer->d_model <= 0 || layer->d_ff <= 0) return 0;
+    DeviceInfo di;
+    int sms = 148;
+    if (device_info(&di) == CLADA_OK) sms = di.num_sms;
+    // decode: one fp32 partial output row per persistent CTA (at most 4 CTAs per SM)
+    size_t decode = (size_t)sms * 4 * (size_t)layer->d_model * sizeof(float);
+    // prefix: one fp32 partial sum of squares per (token tile, neuron); tiles hold 64 tokens
+    size_t tiles = (size_t)(T_total / 64) + (size_t)B + 1;
+    size_t prefix = (tiles * (size_t)layer->d_ff * sizeof(float) + 255) & ~(size_t)255;
+    // guard band: candidate list (int32 pairs) per (sequence, neuron), worst case all of them
+    size_t refine = (size_t)B * (size_t)layer->d_ff * 2 * sizeof(int32_t) + 256;
+    size_t scratch = decode > prefix + refine ? decode : prefix + refine;
+    return kWsCtrlBytes + ((scratch + 255) & ~(size_t)255);
+}
+
+int clada_workspace_init(void *ws, size_t ws_bytes, void *stream) {
+    if (!ws) return CLADA_ERR_NULL;
+    if (ws_bytes < kWsCtrlBytes || (reinterpret_cast<uintptr_t>(ws) & 255u)) return CLADA_ERR_WORKSPACE;
+    CLADA_CUDA_TRY(cudaMemsetAsync(ws, 0, kWsCtrlBytes, static_cast<cudaStream_t>(stream)));
+    return CLADA_OK;
+}
+
+int clada_down_norms(const clada_layer *layer, float *out, void *stream) {
+    int rc = validate_layer(layer, false);
+    if (rc != CLADA_OK) return rc;
+    if (!out) return CLADA_ERR_NULL;
+    const int threads = 256;
+    const int blocks = (layer->d_ff + threads / kWarp - 1) / (threads / kWarp);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (layer->dtype == CLADA_F32)
+        down_norms_kernel<float><<<blocks, threads, 0, st>>>(
+            static_cast<const float *>(layer->w_down_t), layer->d_model, layer->d_ff, out);
+    else
+        down_norms_kernel<__nv_bfloat16><<<blocks, threads, 0, st>>>(
+            static_cast<const __nv_bfloat16 *>(layer->w_down_t), layer->d_model, layer->d_ff, out);
+    CLADA_CUDA_TRY(cudaGetLastError());
+    return CLADA_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,96 @@
+// Shared host/device helpers of the CLADA CUDA library (sm_100a only).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "clada.h"
+
+namespace clada {
+
+constexpr int kWarp = 32;
+constexpr int kMaxDModel = 8192;
+
+// ---- host-side error plumbing -------------------------------------------------------------
+void set_last_cuda_error(cudaError_t e, const char *where);
+int cuda_fail(cudaError_t e, const char *where);  // records and returns CLADA_ERR_CUDA
+
+#define CLADA_CUDA_TRY(expr)                                           \
+    do {                                                               \
+        cudaError_t e__ = (expr);                                      \
+        if (e__ != cudaSuccess) return ::clada::cuda_fail(e__, #expr); \
+    } while (0)
+
+inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+inline size_t elem_size(int dtype) { return dtype == CLADA_F32 ? 4 : 2; }
+int validate_layer(const clada_layer *layer, bool need_norm);
+
+struct DeviceInfo {
+    int device;
+    int num_sms;
+    int max_smem_optin;
+};
+// Properties of the current device (cached per device).
+int device_info(DeviceInfo *out);
+
+// ---- workspace layout ---------------------------------------------------------------------
+// [0, 256)            control words (grid-barrier counters), zeroed by clada_workspace_init
+// [256, ...)          per-call scratch
+constexpr size_t kWsCtrlBytes = 256;
+struct WsCtrl {
+    unsigned int arrive;  // grid barrier: CTAs that reached it
+    unsigned int depart;  // CTAs that left it; the last one resets both
+};
+
+// ---- device helpers -----------------------------------------------------------------------
+#ifdef __CUDACC__
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+__device__ __forceinline__ double warp_sum(double v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+// 16-byte read-only global load that does not allocate in L1 (weights are streamed once).
+__device__ __forceinline__ uint4 ldg_stream(const void *p) {
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "l"(p));
+    return v;
+}
+
+// The two bf16 halves of a 32-bit word as fp32 (exact).
+__device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
+
+template <typename T> struct Elem;
+template <> struct Elem<float> {
+    static constexpr int kPerVec = 4;  // elements per 16-byte vector
+    __device__ static __forceinline__ void unpack(const uint4 &v, float (&f)[4]) {
+        f[0] = __uint_as_float(v.x); f[1] = __uint_as_float(v.y);
+        f[2] = __uint_as_float(v.z); f[3] = __uint_as_float(v.w);
+    }
+    __device__ static __forceinline__ float to_float(float v) { return v; }
+};
+template <> struct Elem<__nv_bfloat16> {
+    static constexpr int kPerVec = 8;
+    __device__ static __forceinline__ void unpack(const uint4 &v, float (&f)[8]) {
+        f[0] = bf16_lo(v.x); f[1] = bf16_hi(v.x); f[2] = bf16_lo(v.y); f[3] = bf16_hi(v.y);
+        f[4] = bf16_lo(v.z); f[5] = bf16_hi(v.z); f[6] = bf16_lo(v.w); f[7] = bf16_hi(v.w);
+    }
+    __device__ static __forceinline__ float to_float(__nv_bfloat16 v) { return __bfloat162float(v); }
+};
+
+// silu(g) = g / (1 + exp(-g)); expf keeps full fp32 accuracy.
+__device__ __forceinline__ float silu_f(float g) { return g / (1.0f + expf(-g)); }
+
+#endif  // __CUDACC__
+
+}  // namespace clada
