@@ -1,0 +1,338 @@
+// Prefill statistics (Eq. neuron_activation) on CUDA cores, fp32 accumulation, any dtype:
+//   z[t,j] = silu(x_t . w_gate_j) * (x_t . w_up_j),   A[b,j] = sqrt(sum_{t in b} z[t,j]^2) * ||W_out,j||
+// plus the fp64 guard-band refinement and the one-call prefill entry point.
+//
+// The GEMM never writes z: each CTA owns a (token tile, neuron tile) pair that lies inside one
+// prompt, keeps both accumulators (gate and up) in registers, and its epilogue squares and sums
+// over the tile's tokens into one fp32 partial per neuron.  A second kernel adds a prompt's
+// partials in tile order, so scores are bit-identical run to run.
+#include <math.h>
+
+#include "common.cuh"
+
+namespace clada {
+
+constexpr int kMaxSeqs = 128;
+struct SeqTable {
+    int B;
+    long long off[kMaxSeqs + 1];
+};
+
+constexpr int BM = 64, BN = 64, BK = 32, kPfThreads = 256;
+
+__host__ __device__ inline int tiles_of(long long rows) { return (int)((rows + BM - 1) / BM); }
+
+// Which prompt and which token range a global token-tile index falls in.
+__device__ inline void locate_tile(const SeqTable &tab, int mtile, int &b, long long &t0, long long &t1) {
+    int first = 0;
+    for (b = 0; b < tab.B - 1; ++b) {
+        const int n = tiles_of(tab.off[b + 1] - tab.off[b]);
+        if (mtile < first + n) break;
+        first += n;
+    }
+    t0 = tab.off[b] + (long long)(mtile - first) * BM;
+    t1 = min(t0 + BM, tab.off[b + 1]);
+}
+
+template <typename T>
+__global__ void __launch_bounds__(kPfThreads)
+prefix_partials_kernel(const T *__restrict__ X, const T *__restrict__ Wg, const T *__restrict__ Wu,
+                       int d_model, int d_ff, const SeqTable tab, float *__restrict__ partials) {
+    constexpr int E = Elem<T>::kPerVec;
+    __shared__ __align__(16) float Xs[BK][BM + 4];
+    __shared__ __align__(16) float Gs[BK][BN + 4];
+    __shared__ __align__(16) float Us[BK][BN + 4];
+    __shared__ float s_red[16][BN + 1];
+
+    const int tid = threadIdx.x;
+    const int tx = tid & 15, ty = tid >> 4;  // 16 x 16 threads, 4 x 4 outputs each
+    const int n0 = blockIdx.x * BN;
+    int b;
+    long long t0, t1;
+    locate_tile(tab, blockIdx.y, b, t0, t1);
+
+    float ag[4][4], au[4][4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) ag[i][j] = au[i][j] = 0.f;
+
+    constexpr int kVecPerRow = BK / E;            // 16-byte vectors per tile row
+    constexpr int kVecPerTile = BM * kVecPerRow;  // BM == BN
+    for (int k0 = 0; k0 < d_model; k0 += BK) {
+        for (int v = tid; v < kVecPerTile; v += kPfThreads) {
+            const int r = v / kVecPerRow, c = (v % kVecPerRow) * E;
+            const bool kin = k0 + c < d_model;  // d_model % 8 == 0, so a vector is all in or all out
+            float fx[E], fg[E], fu[E];
+            uint4 qx = make_uint4(0, 0, 0, 0), qg = qx, qu = qx;
+            if (kin && t0 + r < t1) qx = *reinterpret_cast<const uint4 *>(X + (size_t)(t0 + r) * d_model + k0 + c);
+            if (kin && n0 + r < d_ff) {
+                qg = *reinterpret_cast<const uint4 *>(Wg + (size_t)(n0 + r) * d_model + k0 + c);
+                qu = *reinterpret_cast<const uint4 *>(Wu + (size_t)(n0 + r) * d_model + k0 + c);
+            }
+            Elem<T>::unpack(qx, fx);
+            Elem<T>::unpack(qg, fg);
+            Elem<T>::unpack(qu, fu);
+#pragma unroll
+            for (int e = 0; e < E; ++e) {
+                Xs[c + e][r] = fx[e];
+                Gs[c + e][r] = fg[e];
+                Us[c + e][r] = fu[e];
+            }
+        }
+        __syncthreads();
+#pragma unroll
+        for (int k = 0; k < BK; ++k) {
+            const float4 a = *reinterpret_cast<const float4 *>(&Xs[k][ty * 4]);
+            const float4 g = *reinterpret_cast<const float4 *>(&Gs[k][tx * 4]);
+            const float4 u = *reinterpret_cast<const float4 *>(&Us[k][tx * 4]);
+            const float av[4] = {a.x, a.y, a.z, a.w};
+            const float gv[4] = {g.x, g.y, g.z, g.w};
+            const float uv[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    ag[i][j] = fmaf(av[i], gv[j], ag[i][j]);
+                    au[i][j] = fmaf(av[i], uv[j], au[i][j]);
+                }
+        }
+        __syncthreads();
+    }
+    // epilogue: z^2 summed over this thread's 4 tokens, then over the 16 thread rows in order
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        float s = 0.f;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const float z = silu_f(ag[i][j]) * au[i][j];  // padded token rows give exactly 0
+            s = fmaf(z, z, s);
+        }
+        s_red[ty][tx * 4 + j] = s;
+    }
+    __syncthreads();
+    if (tid < BN && n0 + tid < d_ff) {
+        float s = 0.f;
+#pragma unroll
+        for (int r = 0; r < 16; ++r) s += s_red[r][tid];
+        partials[(size_t)blockIdx.y * d_ff + n0 + tid] = s;
+    }
+}
+
+__global__ void prefix_finalize_kernel(const float *__restrict__ partials, const SeqTable tab, int d_ff,
+                                       const float *__restrict__ w_down_norm, float *__restrict__ scores) {
+    const int j = blockIdx.x * blockDim.x + threadIdx.x;
+    const int b = blockIdx.y;
+    if (j >= d_ff) return;
+    int first = 0;
+    for (int q = 0; q < b; ++q) first += tiles_of(tab.off[q + 1] - tab.off[q]);
+    const int n = tiles_of(tab.off[b + 1] - tab.off[b]);
+    float s = 0.f;
+    for (int t = 0; t < n; ++t) s += partials[(size_t)(first + t) * d_ff + j];
+    scores[(size_t)b * d_ff + j] = __fmul_rn(sqrtf(s), w_down_norm[j]);
+}
+
+// ---- guard band -----------------------------------------------------------------------------
+
+struct GuardMults {
+    int n;
+    float m[8];
+};
+
+__global__ void guard_candidates_kernel(const float *__restrict__ scores, int B, int d_ff,
+                                        const float *__restrict__ tau_base, const GuardMults gm,
+                                        float rel_band, int *__restrict__ n_cand, int2 *__restrict__ cand) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= B * d_ff) return;
+    const int b = i / d_ff, j = i % d_ff;
+    const float a = scores[i];
+    bool near = false;
+#pragma unroll
+    for (int g = 0; g < 8; ++g) {
+        if (g < gm.n) {
+            const float thr = tau_base[b] * gm.m[g];
+            near |= fabsf(a - thr) <= rel_band * fabsf(thr);
+        }
+    }
+    if (near) cand[atomicAdd(n_cand, 1)] = make_int2(b, j);
+}
+
+constexpr int kRefThreads = 256;
+
+// One CTA per candidate (grid-stride).  Warps take tokens round-robin; lanes split d_model.
+template <typename T>
+__global__ void __launch_bounds__(kRefThreads)
+guard_refine_kernel(const T *__restrict__ X, const T *__restrict__ Wg, const T *__restrict__ Wu,
+                    const T *__restrict__ Wd_t, int d_model, int d_ff, const SeqTable tab,
+                    const int *__restrict__ n_cand, const int2 *__restrict__ cand,
+                    float *__restrict__ scores) {
+    __shared__ double s_zz[kRefThreads / kWarp];
+    __shared__ double s_nn[kRefThreads / kWarp];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    constexpr int kWarps = kRefThreads / kWarp;
+    const int total = *n_cand;
+    for (int c = blockIdx.x; c < total; c += gridDim.x) {
+        const int b = cand[c].x, j = cand[c].y;
+        const T *wg = Wg + (size_t)j * d_model, *wu = Wu + (size_t)j * d_model, *wd = Wd_t + (size_t)j * d_model;
+        double zz = 0.0;
+        for (long long t = tab.off[b] + warp; t < tab.off[b + 1]; t += kWarps) {
+            const T *x = X + (size_t)t * d_model;
+            double g = 0.0, u = 0.0;
+            for (int k = lane; k < d_model; k += kWarp) {
+                const double xv = (double)Elem<T>::to_float(x[k]);
+                g = fma((double)Elem<T>::to_float(wg[k]), xv, g);
+                u = fma((double)Elem<T>::to_float(wu[k]), xv, u);
+            }
+            g = warp_sum(g);
+            u = warp_sum(u);
+            const double z = g / (1.0 + exp(-g)) * u;
+            zz += z * z;
+        }
+        double nn = 0.0;
+        for (int k = threadIdx.x; k < d_model; k += kRefThreads) {
+            const double w = (double)Elem<T>::to_float(wd[k]);
+            nn = fma(w, w, nn);
+        }
+        nn = warp_sum(nn);
+        if (lane == 0) {
+            s_zz[warp] = zz;
+            s_nn[warp] = nn;
+        }
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            double a = 0.0, n2 = 0.0;
+            for (int w = 0; w < kWarps; ++w) {
+                a += s_zz[w];
+                n2 += s_nn[w];
+            }
+            scores[(size_t)b * d_ff + j] = (float)(sqrt(a) * sqrt(n2));
+        }
+        __syncthreads();
+    }
+}
+
+// ---- host side ------------------------------------------------------------------------------
+
+static int build_table(const int64_t *seq_offsets, int32_t B, SeqTable *tab, int *n_mtiles) {
+    if (!seq_offsets) return CLADA_ERR_NULL;
+    if (B <= 0) return CLADA_ERR_SHAPE;
+    if (B > kMaxSeqs) return CLADA_ERR_UNSUPPORTED;
+    tab->B = B;
+    long long tiles = 0;
+    for (int b = 0; b <= B; ++b) {
+        tab->off[b] = seq_offsets[b];
+        if (seq_offsets[b] < 0 || (b > 0 && seq_offsets[b] < seq_offsets[b - 1])) return CLADA_ERR_SHAPE;
+        if (b > 0) tiles += tiles_of(seq_offsets[b] - seq_offsets[b - 1]);
+    }
+    if (tiles > 65535) return CLADA_ERR_UNSUPPORTED;
+    *n_mtiles = (int)tiles;
+    return CLADA_OK;
+}
+
+static size_t partials_bytes(int n_mtiles, int d_ff) {
+    return (((size_t)n_mtiles * d_ff * sizeof(float)) + 255) & ~(size_t)255;
+}
+
+template <typename T>
+static int run_scores(const clada_layer *L, const void *X, const SeqTable &tab, int n_mtiles, float *scores,
+                      float *partials, cudaStream_t st) {
+    if (n_mtiles > 0) {
+        dim3 grid((L->d_ff + BN - 1) / BN, n_mtiles);
+        prefix_partials_kernel<T><<<grid, kPfThreads, 0, st>>>(
+            static_cast<const T *>(X), static_cast<const T *>(L->w_gate), static_cast<const T *>(L->w_up),
+            L->d_model, L->d_ff, tab, partials);
+        CLADA_CUDA_TRY(cudaGetLastError());
+    }
+    dim3 fgrid((L->d_ff + 255) / 256, tab.B);
+    prefix_finalize_kernel<<<fgrid, 256, 0, st>>>(partials, tab, L->d_ff, L->w_down_norm, scores);
+    CLADA_CUDA_TRY(cudaGetLastError());
+    return CLADA_OK;
+}
+
+}  // namespace clada
+
+using namespace clada;
+
+extern "C" {
+
+int clada_prefix_scores(const clada_layer *layer, const void *X, const int64_t *seq_offsets, int32_t B,
+                        float *scores, void *ws, size_t ws_bytes, int32_t *status, void *stream) {
+    (void)status;
+    int rc = validate_layer(layer, true);
+    if (rc != CLADA_OK) return rc;
+    if (!X || !scores) return CLADA_ERR_NULL;
+    if (!aligned16(X)) return CLADA_ERR_ALIGN;
+    SeqTable tab;
+    int n_mtiles = 0;
+    rc = build_table(seq_offsets, B, &tab, &n_mtiles);
+    if (rc != CLADA_OK) return rc;
+    if (!ws || (reinterpret_cast<uintptr_t>(ws) & 255u)) return CLADA_ERR_WORKSPACE;
+    if (ws_bytes < kWsCtrlBytes + partials_bytes(n_mtiles, layer->d_ff)) return CLADA_ERR_WORKSPACE;
+    float *partials = reinterpret_cast<float *>(static_cast<char *>(ws) + kWsCtrlBytes);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    return layer->dtype == CLADA_F32 ? run_scores<float>(layer, X, tab, n_mtiles, scores, partials, st)
+                                     : run_scores<__nv_bfloat16>(layer, X, tab, n_mtiles, scores, partials, st);
+}
+
+int clada_refine_scores(const clada_layer *layer, const void *X, const int64_t *seq_offsets, int32_t B,
+                        const float *tau_base, const float *guard_mults, int32_t n_guard, float rel_band,
+                        float *scores, void *ws, size_t ws_bytes, int32_t *status, void *stream) {
+    (void)status;
+    int rc = validate_layer(layer, false);
+    if (rc != CLADA_OK) return rc;
+    if (!X || !scores || !tau_base || !guard_mults) return CLADA_ERR_NULL;
+    if (n_guard <= 0 || n_guard > 8 || !(rel_band >= 0.f)) return CLADA_ERR_SHAPE;
+    if (!aligned16(X)) return CLADA_ERR_ALIGN;
+    SeqTable tab;
+    int n_mtiles = 0;
+    rc = build_table(seq_offsets, B, &tab, &n_mtiles);
+    if (rc != CLADA_OK) return rc;
+    if (!ws || (reinterpret_cast<uintptr_t>(ws) & 255u)) return CLADA_ERR_WORKSPACE;
+    // candidate counter + list live behind the partials region of clada_prefix_scores
+    const size_t off = kWsCtrlBytes + partials_bytes(n_mtiles, layer->d_ff);
+    const size_t need = off + 256 + (size_t)B * layer->d_ff * sizeof(int2);
+    if (ws_bytes < need) return CLADA_ERR_WORKSPACE;
+    int *n_cand = reinterpret_cast<int *>(static_cast<char *>(ws) + off);
+    int2 *cand = reinterpret_cast<int2 *>(static_cast<char *>(ws) + off + 256);
+    GuardMults gm;
+    gm.n = n_guard;
+    for (int g = 0; g < 8; ++g) gm.m[g] = g < n_guard ? guard_mults[g] : 0.f;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    CLADA_CUDA_TRY(cudaMemsetAsync(n_cand, 0, sizeof(int), st));
+    const int n = B * layer->d_ff;
+    guard_candidates_kernel<<<(n + 255) / 256, 256, 0, st>>>(scores, B, layer->d_ff, tau_base, gm, rel_band,
+                                                             n_cand, cand);
+    CLADA_CUDA_TRY(cudaGetLastError());
+    DeviceInfo di;
+    rc = device_info(&di);
+    if (rc != CLADA_OK) return rc;
+    const int grid = di.num_sms * 4;
+    if (layer->dtype == CLADA_F32)
+        guard_refine_kernel<float><<<grid, kRefThreads, 0, st>>>(
+            static_cast<const float *>(X), static_cast<const float *>(layer->w_gate),
+            static_cast<const float *>(layer->w_up), static_cast<const float *>(layer->w_down_t),
+            layer->d_model, layer->d_ff, tab, n_cand, cand, scores);
+    else
+        guard_refine_kernel<__nv_bfloat16><<<grid, kRefThreads, 0, st>>>(
+            static_cast<const __nv_bfloat16 *>(X), static_cast<const __nv_bfloat16 *>(layer->w_gate),
+            static_cast<const __nv_bfloat16 *>(layer->w_up), static_cast<const __nv_bfloat16 *>(layer->w_down_t),
+            layer->d_model, layer->d_ff, tab, n_cand, cand, scores);
+    CLADA_CUDA_TRY(cudaGetLastError());
+    return CLADA_OK;
+}
+
+int clada_prefix_select(const clada_layer *layer, const void *X, const int64_t *seq_offsets, int32_t B,
+                        const float *tau_base, const float *guard_mults, int32_t n_guard, float *scores,
+                        uint8_t *mask, int32_t *idx, int32_t *count, void *ws, size_t ws_bytes,
+                        int32_t *status, void *stream) {
+    int rc = clada_prefix_scores(layer, X, seq_offsets, B, scores, ws, ws_bytes, status, stream);
+    if (rc != CLADA_OK || !tau_base) return rc;
+    if (n_guard > 0 && guard_mults) {
+        rc = clada_refine_scores(layer, X, seq_offsets, B, tau_base, guard_mults, n_guard, 1e-4f, scores, ws,
+                                 ws_bytes, status, stream);
+        if (rc != CLADA_OK) return rc;
+    }
+    return clada_select(scores, B, layer->d_ff, tau_base, 1, mask, idx, count, stream);
+}
+
+}  // extern "C"
