@@ -1,0 +1,282 @@
+"""Thin ctypes binding of ``libclada.so``: the same call names as ``include/clada.h``.
+
+Argument marshalling only -- every step of the path runs in the CUDA library.  Tensors are
+torch CUDA tensors (torch provides device memory and streams, nothing else); each wrapper checks
+dtype / contiguity, passes raw pointers and raises ``CladaError`` on a negative return code.
+There is no fallback: if the shared library is missing or cannot be loaded, loading raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Sequence
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libclada.so")
+
+CLADA_F32, CLADA_BF16 = 0, 1
+STATUS_BAD_TOKEN, STATUS_NONFINITE_LOGIT, STATUS_TIMEOUT = 1, 2, 4
+
+_INT_RETURNING = [
+    "clada_workspace_init", "clada_down_norms", "clada_prefix_scores", "clada_refine_scores",
+    "clada_select", "clada_prefix_select", "clada_tau_from_sparsity", "clada_cogload",
+    "clada_adjust_threshold", "clada_cogload_adjust", "clada_sparse_ffn_decode",
+]
+
+
+class CladaError(RuntimeError):
+    pass
+
+
+class _CLayer(ctypes.Structure):
+    _fields_ = [("d_model", ctypes.c_int32), ("d_ff", ctypes.c_int32), ("dtype", ctypes.c_int32),
+                ("reserved", ctypes.c_int32), ("w_gate", ctypes.c_void_p), ("w_up", ctypes.c_void_p),
+                ("w_down_t", ctypes.c_void_p), ("w_down_norm", ctypes.c_void_p)]
+
+
+_lib = None
+
+
+def load() -> ctypes.CDLL:
+    """Load libclada.so (built in-tree by ``build.build()``); raises if it is not there."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise CladaError(f"{LIB_PATH} not found: build it with "
+                         f"`python -m paper_2502_19078_b200.build` (there is no CPU fallback)")
+    L = ctypes.CDLL(LIB_PATH)
+    vp, i32, i64, f32, sz = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_float, ctypes.c_size_t
+    lp = ctypes.POINTER(_CLayer)
+    L.clada_version.restype = ctypes.c_int
+    L.clada_status_string.argtypes = [ctypes.c_int]
+    L.clada_status_string.restype = ctypes.c_char_p
+    L.clada_last_cuda_error.restype = ctypes.c_char_p
+    L.clada_workspace_bytes.argtypes = [lp, i32, i64]
+    L.clada_workspace_bytes.restype = sz
+    L.clada_workspace_init.argtypes = [vp, sz, vp]
+    L.clada_down_norms.argtypes = [lp, vp, vp]
+    L.clada_prefix_scores.argtypes = [lp, vp, vp, i32, vp, vp, sz, vp, vp]
+    L.clada_refine_scores.argtypes = [lp, vp, vp, i32, vp, vp, i32, f32, vp, vp, sz, vp, vp]
+    L.clada_select.argtypes = [vp, i32, i32, vp, i64, vp, vp, vp, vp]
+    L.clada_prefix_select.argtypes = [lp, vp, vp, i32, vp, vp, i32, vp, vp, vp, vp, vp, sz, vp, vp]
+    L.clada_tau_from_sparsity.argtypes = [vp, i32, i32, f32, vp, vp]
+    L.clada_cogload.argtypes = [vp, i32, i32, i64, i64, vp, vp, vp, vp, vp]
+    L.clada_adjust_threshold.argtypes = [vp, vp, vp, f32, f32, vp, vp, i32, i32, vp, vp]
+    L.clada_cogload_adjust.argtypes = [vp, i32, i32, i64, i64, vp, vp, vp, vp, f32, f32, i32, vp, vp, vp, vp, vp]
+    L.clada_sparse_ffn_decode.argtypes = [lp, vp, i32, vp, vp, i64, vp, i32, vp, vp, vp, vp, sz, vp, vp]
+    for name in _INT_RETURNING:
+        getattr(L, name).restype = ctypes.c_int
+    _lib = L
+    return L
+
+
+def _check(rc: int, what: str) -> None:
+    if rc != 0:
+        L = load()
+        msg = L.clada_status_string(rc).decode()
+        if rc == -6:
+            msg += ": " + L.clada_last_cuda_error().decode()
+        raise CladaError(f"{what} failed ({rc}): {msg}")
+
+
+def _dtype_code(t: torch.dtype) -> int:
+    if t == torch.float32:
+        return CLADA_F32
+    if t == torch.bfloat16:
+        return CLADA_BF16
+    raise CladaError(f"unsupported dtype {t}")
+
+
+def _ptr(t: Optional[torch.Tensor], dtype=None, name="tensor") -> Optional[int]:
+    if t is None:
+        return None
+    if not t.is_cuda:
+        raise CladaError(f"{name} must be a CUDA tensor")
+    if not t.is_contiguous():
+        raise CladaError(f"{name} must be contiguous")
+    if dtype is not None and t.dtype != dtype:
+        raise CladaError(f"{name} must be {dtype}, got {t.dtype}")
+    return t.data_ptr()
+
+
+def _stream(stream) -> Optional[int]:
+    if stream is None:
+        return torch.cuda.current_stream().cuda_stream
+    if isinstance(stream, int):
+        return stream
+    return stream.cuda_stream
+
+
+class Layer:
+    """One gated FFN layer in the library's neuron-major layout (keeps the tensors alive)."""
+
+    def __init__(self, w_gate: torch.Tensor, w_up: torch.Tensor, w_down_t: torch.Tensor,
+                 w_down_norm: Optional[torch.Tensor] = None):
+        d_ff, d_model = w_gate.shape
+        if w_up.shape != (d_ff, d_model) or w_down_t.shape != (d_ff, d_model):
+            raise CladaError("w_gate, w_up, w_down_t must all be [d_ff, d_model]")
+        if not (w_gate.dtype == w_up.dtype == w_down_t.dtype):
+            raise CladaError("weights must share one dtype")
+        self.d_model, self.d_ff = int(d_model), int(d_ff)
+        self.dtype = w_gate.dtype
+        self.w_gate, self.w_up, self.w_down_t = w_gate, w_up, w_down_t
+        self.w_down_norm = w_down_norm
+        self.c = _CLayer(self.d_model, self.d_ff, _dtype_code(self.dtype), 0,
+                         _ptr(w_gate, name="w_gate"), _ptr(w_up, name="w_up"),
+                         _ptr(w_down_t, name="w_down_t"),
+                         _ptr(w_down_norm, torch.float32, "w_down_norm"))
+
+    def set_down_norm(self, w_down_norm: torch.Tensor) -> None:
+        self.w_down_norm = w_down_norm
+        self.c.w_down_norm = _ptr(w_down_norm, torch.float32, "w_down_norm")
+
+    @property
+    def ref(self):
+        return ctypes.byref(self.c)
+
+
+def _offsets(seq_offsets: Sequence[int]):
+    arr = (ctypes.c_int64 * len(seq_offsets))(*[int(v) for v in seq_offsets])
+    return arr, len(seq_offsets) - 1
+
+
+def _floats(vals):
+    arr = (ctypes.c_float * len(vals))(*[float(v) for v in vals])
+    return arr
+
+
+def clada_version() -> int:
+    return int(load().clada_version())
+
+
+def clada_workspace_bytes(layer: Layer, B: int, T_total: int) -> int:
+    n = int(load().clada_workspace_bytes(layer.ref, B, T_total))
+    if n == 0:
+        raise CladaError("clada_workspace_bytes: invalid arguments")
+    return n
+
+
+def clada_workspace_init(ws: torch.Tensor, stream=None) -> None:
+    _check(load().clada_workspace_init(_ptr(ws, torch.uint8, "ws"), ws.numel(), _stream(stream)),
+           "clada_workspace_init")
+
+
+def new_workspace(layer: Layer, B: int, T_total: int, stream=None) -> torch.Tensor:
+    """Allocate (through torch) and initialise a workspace for this layer shape."""
+    ws = torch.empty(clada_workspace_bytes(layer, B, T_total), dtype=torch.uint8, device=layer.w_gate.device)
+    clada_workspace_init(ws, stream)
+    return ws
+
+
+def clada_down_norms(layer: Layer, out: torch.Tensor, stream=None) -> None:
+    _check(load().clada_down_norms(layer.ref, _ptr(out, torch.float32, "out"), _stream(stream)),
+           "clada_down_norms")
+
+
+def clada_prefix_scores(layer: Layer, X, seq_offsets, scores, ws, status=None, stream=None) -> None:
+    off, B = _offsets(seq_offsets)
+    _check(load().clada_prefix_scores(layer.ref, _ptr(X, layer.dtype, "X"), ctypes.addressof(off), B,
+                                      _ptr(scores, torch.float32, "scores"), _ptr(ws, torch.uint8, "ws"),
+                                      ws.numel(), _ptr(status, torch.int32, "status"), _stream(stream)),
+           "clada_prefix_scores")
+
+
+def clada_refine_scores(layer: Layer, X, seq_offsets, tau_base, guard_mults, rel_band, scores, ws,
+                        status=None, stream=None) -> None:
+    off, B = _offsets(seq_offsets)
+    gm = _floats(guard_mults)
+    _check(load().clada_refine_scores(layer.ref, _ptr(X, layer.dtype, "X"), ctypes.addressof(off), B,
+                                      _ptr(tau_base, torch.float32, "tau_base"), ctypes.addressof(gm),
+                                      len(guard_mults), float(rel_band),
+                                      _ptr(scores, torch.float32, "scores"), _ptr(ws, torch.uint8, "ws"),
+                                      ws.numel(), _ptr(status, torch.int32, "status"), _stream(stream)),
+           "clada_refine_scores")
+
+
+def clada_select(scores, tau, tau_stride=1, mask=None, idx=None, count=None, stream=None) -> None:
+    B, d_ff = scores.shape
+    _check(load().clada_select(_ptr(scores, torch.float32, "scores"), B, d_ff, _ptr(tau, torch.float32, "tau"),
+                               tau_stride, _ptr(mask, torch.uint8, "mask"), _ptr(idx, torch.int32, "idx"),
+                               _ptr(count, torch.int32, "count"), _stream(stream)), "clada_select")
+
+
+def clada_prefix_select(layer: Layer, X, seq_offsets, tau_base, guard_mults, scores, mask, idx, count, ws,
+                        status=None, stream=None) -> None:
+    off, B = _offsets(seq_offsets)
+    gm, gm_ptr, n_guard = None, None, 0
+    if guard_mults is not None and len(guard_mults) > 0:
+        gm = _floats(guard_mults)
+        gm_ptr, n_guard = ctypes.addressof(gm), len(guard_mults)
+    _check(load().clada_prefix_select(layer.ref, _ptr(X, layer.dtype, "X"), ctypes.addressof(off), B,
+                                      _ptr(tau_base, torch.float32, "tau_base"), gm_ptr, n_guard,
+                                      _ptr(scores, torch.float32, "scores"), _ptr(mask, torch.uint8, "mask"),
+                                      _ptr(idx, torch.int32, "idx"), _ptr(count, torch.int32, "count"),
+                                      _ptr(ws, torch.uint8, "ws"), ws.numel(),
+                                      _ptr(status, torch.int32, "status"), _stream(stream)),
+           "clada_prefix_select")
+
+
+def clada_tau_from_sparsity(scores, rho, tau_base, stream=None) -> None:
+    B, d_ff = scores.shape
+    _check(load().clada_tau_from_sparsity(_ptr(scores, torch.float32, "scores"), B, d_ff, float(rho),
+                                          _ptr(tau_base, torch.float32, "tau_base"), _stream(stream)),
+           "clada_tau_from_sparsity")
+
+
+def _logits_args(logits):
+    if not logits.is_cuda or logits.dim() != 2 or logits.stride(1) != 1:
+        raise CladaError("logits must be a 2-D CUDA tensor with contiguous rows")
+    B, V = logits.shape
+    return logits.data_ptr(), _dtype_code(logits.dtype), B, V, logits.stride(0)
+
+
+def clada_cogload(logits, token_id, surprisal, entropy, status=None, stream=None) -> None:
+    _check(load().clada_cogload(*_logits_args(logits), _ptr(token_id, torch.int32, "token_id"),
+                                _ptr(surprisal, torch.float32, "surprisal"),
+                                _ptr(entropy, torch.float32, "entropy"),
+                                _ptr(status, torch.int32, "status"), _stream(stream)), "clada_cogload")
+
+
+def clada_adjust_threshold(tau_base, lam, gam, tau_s, tau_H, surprisal, entropy, tau_final, stream=None) -> None:
+    B, L = tau_base.shape
+    _check(load().clada_adjust_threshold(_ptr(tau_base, torch.float32, "tau_base"), _ptr(lam, torch.float32, "lambda"),
+                                         _ptr(gam, torch.float32, "gamma"), float(tau_s), float(tau_H),
+                                         _ptr(surprisal, torch.float32, "surprisal"),
+                                         _ptr(entropy, torch.float32, "entropy"), B, L,
+                                         _ptr(tau_final, torch.float32, "tau_final"), _stream(stream)),
+           "clada_adjust_threshold")
+
+
+def clada_cogload_adjust(logits, token_id, tau_base, lam, gam, tau_s, tau_H, surprisal, entropy, tau_final,
+                         status=None, stream=None) -> None:
+    L = tau_base.shape[1]
+    _check(load().clada_cogload_adjust(*_logits_args(logits), _ptr(token_id, torch.int32, "token_id"),
+                                       _ptr(tau_base, torch.float32, "tau_base"),
+                                       _ptr(lam, torch.float32, "lambda"), _ptr(gam, torch.float32, "gamma"),
+                                       float(tau_s), float(tau_H), L,
+                                       _ptr(surprisal, torch.float32, "surprisal"),
+                                       _ptr(entropy, torch.float32, "entropy"),
+                                       _ptr(tau_final, torch.float32, "tau_final"),
+                                       _ptr(status, torch.int32, "status"), _stream(stream)),
+           "clada_cogload_adjust")
+
+
+def clada_sparse_ffn_decode(layer: Layer, x, scores, tau_final, tau_stride, y, ws, mask_out=None, idx_out=None,
+                            count_out=None, status=None, stream=None) -> None:
+    """tau_final may be a view into a larger [B, L] array: pass the element for (b=0, this layer) and
+    tau_stride = L."""
+    B = x.shape[0]
+    if not tau_final.is_cuda or tau_final.dtype != torch.float32:
+        raise CladaError("tau_final must be a CUDA float32 tensor")
+    _check(load().clada_sparse_ffn_decode(layer.ref, _ptr(x, layer.dtype, "x"), B,
+                                          _ptr(scores, torch.float32, "scores"), tau_final.data_ptr(),
+                                          int(tau_stride), _ptr(y, name="y"), _dtype_code(y.dtype),
+                                          _ptr(mask_out, torch.uint8, "mask_out"),
+                                          _ptr(idx_out, torch.int32, "idx_out"),
+                                          _ptr(count_out, torch.int32, "count_out"),
+                                          _ptr(ws, torch.uint8, "ws"), ws.numel(),
+                                          _ptr(status, torch.int32, "status"), _stream(stream)),
+           "clada_sparse_ffn_decode")
