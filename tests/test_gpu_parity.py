@@ -1,0 +1,465 @@
+"""GPU parity: every C-ABI call against the CPU oracle on the same seeded inputs.
+
+Tolerances (the ones the path is held to):
+  * masks / index lists / counts: bit-exact, except neurons whose oracle score lies within 1e-6
+    relative of the threshold (counted separately);
+  * FFN outputs: max |y - y_oracle| / max |y_oracle| <= 1e-5 with fp32 output (both weight dtypes:
+    bf16 products are exact in fp32), <= 2e-2 with bf16 output;
+  * surprisal / entropy: 1e-4 absolute;
+  * tau_final, tau_from_sparsity: bit-exact given the same fp32 inputs.
+"""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from paper_2502_19078_b200 import workloads as wl
+from tests._util import compare_masks, gpu_layer, oracle_weights, rel_inf
+
+pytestmark = pytest.mark.gpu
+
+FFN_TOL_F32 = 1e-5
+FFN_TOL_BF16_OUT = 2e-2
+COG_TOL = 1e-4
+SCORE_TOL = 2e-6   # fp32-accumulated scores vs fp64 (relative); selection is checked separately
+
+
+@pytest.fixture(scope="module")
+def clada():
+    from paper_2502_19078_b200 import binding, build
+    build.build()
+    binding.load()
+    return binding
+
+
+def _dev(a, dtype=None):
+    t = torch.as_tensor(a)
+    if dtype is not None:
+        t = t.to(dtype)
+    return t.cuda().contiguous()
+
+
+# ------------------------------------------------------------------------------------------------
+# cognitive load
+# ------------------------------------------------------------------------------------------------
+
+def _cogload_gpu(clada, logits_dev, tokens):
+    B = logits_dev.shape[0]
+    s = torch.empty(B, dtype=torch.float32, device="cuda")
+    h = torch.empty(B, dtype=torch.float32, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    clada.clada_cogload(logits_dev, _dev(tokens, torch.int32), s, h, status)
+    torch.cuda.synchronize()
+    return s.cpu().numpy(), h.cpu().numpy(), int(status.item())
+
+
+@pytest.mark.parametrize("V", [1, 3, 17, 4096, 32000, 128256])
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_cogload_parity(clada, oracle, V, dtype):
+    g = torch.Generator().manual_seed(V)
+    B = 5
+    logits = 3.0 * torch.randn(B, V, generator=g)
+    logits[1] /= 0.5
+    logits[2] /= 4.0
+    if V > 8:
+        logits[3, ::3] = -float("inf")
+    tdt = torch.float32 if dtype == "f32" else torch.bfloat16
+    logits = logits.to(tdt)
+    tokens = torch.randint(0, V, (B,), generator=g)
+    tokens[0] = int(torch.argmax(logits[0].float()))
+    s, h, status = _cogload_gpu(clada, logits.cuda(), tokens)
+    assert status == 0
+    for b in range(B):
+        s_or, h_or = oracle.cogload(wl.to_numpy_bits(logits[b]), int(tokens[b]))
+        if math.isinf(s_or):
+            assert math.isinf(s[b]) and s[b] > 0
+        else:
+            assert abs(s[b] - s_or) <= COG_TOL, (b, s[b], s_or)
+        assert abs(h[b] - h_or) <= COG_TOL, (b, h[b], h_or)
+
+
+def test_cogload_closed_forms_on_gpu(clada):
+    for V in (4096, 32000, 128256):
+        uni = torch.full((1, V), 0.25, device="cuda")
+        s, h, _ = _cogload_gpu(clada, uni, [V - 1])
+        assert abs(h[0] - math.log(V)) <= COG_TOL and abs(s[0] - math.log(V)) <= COG_TOL
+        one = torch.full((1, V), -float("inf"), device="cuda")
+        one[0, 5] = 2.0
+        s, h, status = _cogload_gpu(clada, one, [5])
+        assert s[0] == 0.0 and h[0] == 0.0 and status == 0
+
+
+def test_cogload_unaligned_and_strided_rows(clada, oracle):
+    g = torch.Generator().manual_seed(1)
+    big = (2.0 * torch.randn(4, 1003, generator=g)).cuda()
+    view = big[:, 3:1000]            # rows start off a 16-byte boundary, stride 1003
+    tokens = [0, 10, 500, 996]
+    s, h, status = _cogload_gpu(clada, view, tokens)
+    assert status == 0
+    for b in range(4):
+        s_or, h_or = oracle.cogload(view[b].cpu().numpy(), tokens[b])
+        assert abs(s[b] - s_or) <= COG_TOL and abs(h[b] - h_or) <= COG_TOL
+
+
+def test_cogload_status_bits(clada):
+    logits = torch.zeros(3, 100, device="cuda")
+    logits[1, 7] = float("nan")
+    logits[2, 9] = float("inf")
+    s, h, status = _cogload_gpu(clada, logits, [100, 0, 0])
+    assert status == (clada.STATUS_BAD_TOKEN | clada.STATUS_NONFINITE_LOGIT)
+    assert math.isnan(s[0]) and abs(h[0] - math.log(100)) <= COG_TOL
+    assert math.isnan(s[1]) and math.isnan(h[1]) and math.isnan(s[2]) and math.isnan(h[2])
+    s, h, status = _cogload_gpu(clada, torch.full((1, 64), -float("inf"), device="cuda"), [0])
+    assert status == clada.STATUS_NONFINITE_LOGIT and math.isnan(h[0])
+
+
+# ------------------------------------------------------------------------------------------------
+# threshold adjustment, selection, order statistic
+# ------------------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("sign", [1.0, -1.0])
+def test_adjust_threshold_bit_exact(clada, oracle, sign):
+    rng = np.random.default_rng(0)
+    B, L = 7, 40
+    tau_base = (rng.random((B, L)) + 0.1).astype(np.float32)
+    lam = (sign * (0.80 + 0.01 * rng.standard_normal(L))).astype(np.float32)
+    gam = (sign * (0.12 + 0.01 * rng.standard_normal(L))).astype(np.float32)
+    s = np.array([0.5, 2.0, 3.0, 2.0, 9.0, 0.0, 2.0000002], dtype=np.float32)
+    h = np.array([1.0, 4.0, 4.5, 7.0, 0.1, 4.0, 4.0000005], dtype=np.float32)
+    out = torch.empty(B, L, dtype=torch.float32, device="cuda")
+    clada.clada_adjust_threshold(_dev(tau_base), _dev(lam), _dev(gam), 2.0, 4.0, _dev(s), _dev(h), out)
+    ref = oracle.adjust_threshold(tau_base, lam, gam, 2.0, 4.0, s.astype(np.float64), h.astype(np.float64))
+    np.testing.assert_array_equal(out.cpu().numpy(), ref)
+
+
+def test_cogload_adjust_fused_equals_separate(clada):
+    g = torch.Generator().manual_seed(2)
+    B, V, L = 4, 5000, 33
+    logits = (3.0 * torch.randn(B, V, generator=g)).cuda()
+    tokens = _dev(torch.randint(0, V, (B,), generator=g), torch.int32)
+    tau_base = (torch.rand(B, L, generator=g) + 0.5).cuda()
+    lam = torch.full((L,), 0.80, device="cuda")
+    gam = torch.full((L,), 0.12, device="cuda")
+    s1, h1, s2, h2 = (torch.empty(B, device="cuda") for _ in range(4))
+    t1, t2 = torch.empty(B, L, device="cuda"), torch.empty(B, L, device="cuda")
+    clada.clada_cogload(logits, tokens, s1, h1)
+    tau_s, tau_H = float(s1.median()) + 1e-3, float(h1.median()) + 1e-3
+    clada.clada_adjust_threshold(tau_base, lam, gam, tau_s, tau_H, s1, h1, t1)
+    clada.clada_cogload_adjust(logits, tokens, tau_base, lam, gam, tau_s, tau_H, s2, h2, t2)
+    torch.cuda.synchronize()
+    assert torch.equal(s1, s2) and torch.equal(h1, h2) and torch.equal(t1, t2)
+    assert not torch.equal(t1, tau_base)
+
+
+@pytest.mark.parametrize("F", [1, 31, 32, 33, 1376, 11008, 14336])
+def test_select_bit_exact(clada, oracle, F):
+    rng = np.random.default_rng(F)
+    B = 3
+    scores = rng.random((B, F)).astype(np.float32)
+    taus = np.array([0.0, 0.4, np.inf], dtype=np.float32)
+    if F > 4:
+        taus[1] = scores[1, F // 2]                 # equality keeps
+    mask = torch.empty(B, F, dtype=torch.uint8, device="cuda")
+    idx = torch.full((B, F), -1, dtype=torch.int32, device="cuda")
+    count = torch.empty(B, dtype=torch.int32, device="cuda")
+    clada.clada_select(_dev(scores), _dev(taus), 1, mask, idx, count)
+    torch.cuda.synchronize()
+    for b in range(B):
+        m_or, idx_or, n_or = oracle.select(scores[b].astype(np.float64), float(taus[b]))
+        assert int(count[b]) == n_or
+        np.testing.assert_array_equal(mask[b].cpu().numpy(), m_or)
+        np.testing.assert_array_equal(idx[b, :n_or].cpu().numpy(), idx_or)
+        assert bool((idx[b, n_or:] == -1).all())
+
+
+@pytest.mark.parametrize("F,rho", [(1376, 0.4), (11008, 0.4), (11008, 0.5), (13824, 0.3), (13824, 0.6),
+                                   (100, 0.0), (100, 1.0), (7, 0.5)])
+def test_tau_from_sparsity_bit_exact(clada, oracle, F, rho):
+    rng = np.random.default_rng(F)
+    B = 2
+    scores = (rng.random((B, F)) * 3).astype(np.float32)
+    scores[1, : F // 2] = scores[1, 0]            # heavy ties
+    tau = torch.empty(B, dtype=torch.float32, device="cuda")
+    clada.clada_tau_from_sparsity(_dev(scores), rho, tau)
+    for b in range(B):
+        ref = oracle.tau_from_sparsity(scores[b], float(np.float32(rho)))
+        assert np.float32(tau[b].item()) == ref or (math.isinf(ref) and math.isinf(tau[b].item()))
+
+
+# ------------------------------------------------------------------------------------------------
+# prefix statistics
+# ------------------------------------------------------------------------------------------------
+
+def _small(name, **kw):
+    return wl.scaled(wl.WORKLOADS[name], **kw)
+
+
+def _prefix_inputs(w, lengths, dev="cpu"):
+    scale = wl.channel_scale(w, dev)
+    xs = [wl.hidden_states(w, 0, "prefix", b, n, dev, scale) for b, n in enumerate(lengths)]
+    return torch.cat(xs, dim=0) if xs else torch.empty(0, w.d_model, dtype=w.torch_dtype)
+
+
+@pytest.mark.parametrize("name,kw,lengths", [
+    ("c1_small_f32", {}, [64]),
+    ("c1_small_f32", {"d_model": 72, "d_ff": 130}, [70, 0, 129, 1]),
+    ("c2_llama2_7b_layer", {"d_model": 256, "d_ff": 300}, [200, 65]),
+])
+def test_prefix_scores_parity(clada, oracle, name, kw, lengths):
+    w = _small(name, **kw)
+    weights = wl.layer_weights(w, 0)
+    X = _prefix_inputs(w, lengths)
+    off = wl.seq_offsets(lengths)
+    layer = gpu_layer(weights, clada)
+    ws = clada.new_workspace(layer, len(lengths), off[-1])
+    scores = torch.empty(len(lengths), w.d_ff, dtype=torch.float32, device="cuda")
+    clada.clada_prefix_scores(layer, X.cuda(), off, scores, ws)
+    A_or = oracle.neuron_scores(wl.to_numpy_bits(X), off, *oracle_weights(weights))
+    A = scores.cpu().numpy().astype(np.float64)
+    for b, n in enumerate(lengths):
+        if n == 0:
+            assert np.all(A[b] == 0.0)
+        else:
+            assert np.max(np.abs(A[b] - A_or[b]) / A_or[b]) <= SCORE_TOL
+    # down norms against numpy
+    Wd = oracle_weights(weights)[2]
+    Wd64 = (Wd.astype(np.uint32) << 16).view(np.float32).astype(np.float64) if Wd.dtype == np.uint16 else Wd.astype(np.float64)
+    np.testing.assert_allclose(layer.w_down_norm.cpu().numpy(), np.linalg.norm(Wd64, axis=0), rtol=1e-6)
+
+
+def test_guard_band_refinement_rounds_correctly(clada, oracle):
+    """Inside the band the stored score is the fp64 result rounded to fp32; outside it is untouched."""
+    w = _small("c2_llama2_7b_layer", d_model=256, d_ff=300)
+    lengths = [90, 40]
+    weights = wl.layer_weights(w, 0)
+    X = _prefix_inputs(w, lengths)
+    off = wl.seq_offsets(lengths)
+    layer = gpu_layer(weights, clada)
+    ws = clada.new_workspace(layer, 2, off[-1])
+    scores = torch.empty(2, w.d_ff, dtype=torch.float32, device="cuda")
+    clada.clada_prefix_scores(layer, X.cuda(), off, scores, ws)
+    before = scores.clone()
+    tau = torch.empty(2, dtype=torch.float32, device="cuda")
+    clada.clada_tau_from_sparsity(scores, 0.4, tau)
+    band = 0.05       # wide, so that a fair number of neurons qualify
+    mults = [1.0, 1.8]
+    clada.clada_refine_scores(layer, X.cuda(), off, tau, mults, band, scores, ws)
+    A_or = oracle.neuron_scores(wl.to_numpy_bits(X), off, *oracle_weights(weights))
+    b4, after, t = before.cpu().numpy(), scores.cpu().numpy(), tau.cpu().numpy()
+    n_in = 0
+    for b in range(2):
+        inside = np.zeros(w.d_ff, dtype=bool)
+        for m in mults:
+            thr = np.float32(t[b] * np.float32(m))
+            inside |= np.abs(b4[b] - thr) <= np.float32(band) * abs(thr)
+        n_in += int(inside.sum())
+        assert np.array_equal(after[b][~inside], b4[b][~inside])
+        ref32 = A_or[b][inside].astype(np.float32)
+        ulp = np.spacing(ref32)
+        assert np.all(np.abs(after[b][inside].astype(np.float64) - A_or[b][inside]) <= 1.01 * ulp)
+    assert n_in > 10
+
+
+# ------------------------------------------------------------------------------------------------
+# sparse FFN decode
+# ------------------------------------------------------------------------------------------------
+
+def _ffn_case(clada, oracle, w, rho, n_steps, y_dtype=torch.float32, B=1, prefix=48):
+    """Prefill + n_steps decode tokens of one layer, both sides; returns worst errors."""
+    weights = wl.layer_weights(w, 0)
+    lengths = [prefix + 5 * b for b in range(B)]
+    X = _prefix_inputs(w, lengths)
+    off = wl.seq_offsets(lengths)
+    layer = gpu_layer(weights, clada)
+    ws = clada.new_workspace(layer, B, off[-1])
+    scores = torch.empty(B, w.d_ff, dtype=torch.float32, device="cuda")
+    clada.clada_prefix_scores(layer, X.cuda(), off, scores, ws)
+    tau_base = torch.empty(B, dtype=torch.float32, device="cuda")
+    clada.clada_tau_from_sparsity(scores, rho, tau_base)
+    mults = [1.0, 1.8, 1.12, 1.92]
+    clada.clada_refine_scores(layer, X.cuda(), off, tau_base, mults, 1e-4, scores, ws)
+    W_in, V_in, W_out = oracle_weights(weights)
+    A_or = oracle.neuron_scores(wl.to_numpy_bits(X), off, W_in, V_in, W_out)
+    scale = wl.channel_scale(w)
+    xs = torch.stack([wl.hidden_states(w, 0, "decode", b, n_steps, "cpu", scale) for b in range(B)], dim=1)
+    y = torch.empty(B, w.d_model, dtype=y_dtype, device="cuda")
+    mask = torch.empty(B, w.d_ff, dtype=torch.uint8, device="cuda")
+    idx = torch.empty(B, w.d_ff, dtype=torch.int32, device="cuda")
+    count = torch.empty(B, dtype=torch.int32, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    worst, excused, mismatched = 0.0, 0, 0
+    tb = tau_base.cpu().numpy()
+    for t in range(n_steps):
+        mult = np.float32(mults[t % 4])
+        tau_t = torch.from_numpy(tb * mult).cuda()
+        clada.clada_sparse_ffn_decode(layer, xs[t].cuda(), scores, tau_t, 1, y, ws, mask, idx, count, status)
+        torch.cuda.synchronize()
+        for b in range(B):
+            tau_b = float(tb[b] * mult)
+            y_or, m_or, n_or = oracle.sparse_ffn(wl.to_numpy_bits(xs[t, b]), W_in, V_in, W_out, A_or[b], tau_b)
+            m_gpu = mask[b].cpu().numpy()
+            e, m = compare_masks(m_gpu, A_or[b], tau_b)
+            excused += e
+            mismatched += m
+            n_gpu = int(count[b])
+            assert n_gpu == int(m_gpu.sum())
+            np.testing.assert_array_equal(idx[b, :n_gpu].cpu().numpy(), np.nonzero(m_gpu)[0])
+            if e == 0 and m == 0:
+                worst = max(worst, rel_inf(y[b].float().cpu().numpy(), y_or))
+    assert int(status.item()) == 0
+    return worst, excused, mismatched
+
+
+def test_sparse_ffn_config1_full(clada, oracle):
+    w = wl.WORKLOADS["c1_small_f32"]
+    worst, excused, mismatched = _ffn_case(clada, oracle, w, 0.40, w.n_decode, prefix=64)
+    assert mismatched == 0
+    assert worst <= FFN_TOL_F32
+
+
+@pytest.mark.parametrize("d,F", [(8, 5), (64, 100), (520, 777), (1024, 2500), (2048, 1500), (4096, 1200),
+                                 (5120, 900), (8192, 600)])
+def test_sparse_ffn_bf16_shapes(clada, oracle, d, F):
+    w = _small("c2_llama2_7b_layer", d_model=d, d_ff=F)
+    worst, excused, mismatched = _ffn_case(clada, oracle, w, 0.40, 4, prefix=20)
+    assert mismatched == 0
+    assert worst <= FFN_TOL_F32
+
+
+@pytest.mark.parametrize("d,F", [(16, 40), (512, 1376), (1032, 300), (4096, 300)])
+def test_sparse_ffn_f32_shapes(clada, oracle, d, F):
+    w = _small("c1_small_f32", d_model=d, d_ff=F)
+    worst, excused, mismatched = _ffn_case(clada, oracle, w, 0.50, 4, prefix=20)
+    assert mismatched == 0
+    assert worst <= FFN_TOL_F32
+
+
+def test_sparse_ffn_bf16_output_and_batch(clada, oracle):
+    w = _small("c4_llama3_8b_b8", d_model=1024, d_ff=1800)
+    worst, excused, mismatched = _ffn_case(clada, oracle, w, 0.40, 3, y_dtype=torch.bfloat16, B=3)
+    assert mismatched == 0
+    assert worst <= FFN_TOL_BF16_OUT
+    worst, _, mismatched = _ffn_case(clada, oracle, w, 0.60, 3, B=3)
+    assert mismatched == 0 and worst <= FFN_TOL_F32
+
+
+def test_sparse_ffn_degenerate_thresholds_and_determinism(clada, oracle):
+    w = _small("c2_llama2_7b_layer", d_model=512, d_ff=700)
+    weights = wl.layer_weights(w, 0)
+    layer = gpu_layer(weights, clada)
+    ws = clada.new_workspace(layer, 1, 0)
+    W_in, V_in, W_out = oracle_weights(weights)
+    x = wl.hidden_states(w, 0, "decode", 0, 1)
+    rng = np.random.default_rng(5)
+    scores = (rng.random((1, w.d_ff)) + 0.5).astype(np.float32)
+    y = torch.empty(1, w.d_model, dtype=torch.float32, device="cuda")
+    count = torch.empty(1, dtype=torch.int32, device="cuda")
+    # tau = 0 keeps everything: the dense FFN
+    clada.clada_sparse_ffn_decode(layer, x.cuda(), _dev(scores), _dev(np.zeros(1, np.float32)), 1, y, ws,
+                                  count_out=count)
+    y_dense = oracle.dense_ffn(wl.to_numpy_bits(x[0]), W_in, V_in, W_out)
+    assert int(count[0]) == w.d_ff and rel_inf(y[0].cpu().numpy(), y_dense) <= FFN_TOL_F32
+    # tau = +inf keeps nothing: y = 0 exactly
+    clada.clada_sparse_ffn_decode(layer, x.cuda(), _dev(scores), _dev(np.full(1, np.inf, np.float32)), 1, y, ws,
+                                  count_out=count)
+    assert int(count[0]) == 0 and bool((y == 0).all())
+    # one kept neuron
+    tau1 = np.float32(np.sort(scores[0])[-1])
+    clada.clada_sparse_ffn_decode(layer, x.cuda(), _dev(scores), _dev(np.array([tau1])), 1, y, ws, count_out=count)
+    y_or, _, n_or = oracle.sparse_ffn(wl.to_numpy_bits(x[0]), W_in, V_in, W_out, scores[0].astype(np.float64),
+                                      float(tau1))
+    assert int(count[0]) == n_or == 1 and rel_inf(y[0].cpu().numpy(), y_or) <= FFN_TOL_F32
+    # bit-identical run to run
+    tau = _dev(np.array([1.0], np.float32))
+    y2 = torch.empty_like(y)
+    clada.clada_sparse_ffn_decode(layer, x.cuda(), _dev(scores), tau, 1, y, ws)
+    clada.clada_sparse_ffn_decode(layer, x.cuda(), _dev(scores), tau, 1, y2, ws)
+    torch.cuda.synchronize()
+    assert torch.equal(y, y2)
+
+
+def test_host_side_errors(clada):
+    w = _small("c2_llama2_7b_layer", d_model=64, d_ff=50)
+    layer = gpu_layer(wl.layer_weights(w, 0), clada)
+    ws = clada.new_workspace(layer, 1, 0)
+    x = torch.zeros(1, 64, dtype=torch.bfloat16, device="cuda")
+    scores = torch.ones(1, 50, device="cuda")
+    tau = torch.ones(1, device="cuda")
+    y = torch.empty(1, 64, device="cuda")
+    small_ws = torch.empty(512, dtype=torch.uint8, device="cuda")
+    with pytest.raises(clada.CladaError, match="workspace"):
+        clada.clada_sparse_ffn_decode(layer, x, scores, tau, 1, y, small_ws)
+    with pytest.raises(clada.CladaError):
+        clada.clada_sparse_ffn_decode(layer, x.float(), scores, tau, 1, y, ws)      # wrong dtype for x
+    with pytest.raises(clada.CladaError, match="shape"):
+        clada.clada_prefix_scores(layer, x, [0, 5, 3], torch.empty(2, 50, device="cuda"), ws)   # descending offsets
+    bad = clada.Layer(layer.w_gate[:, :60].contiguous(), layer.w_up[:, :60].contiguous(),
+                      layer.w_down_t[:, :60].contiguous())                          # d_model % 8 != 0
+    with pytest.raises(clada.CladaError, match="shape"):
+        clada.clada_sparse_ffn_decode(bad, x, scores, tau, 1, y, ws)
+    torch.cuda.synchronize()
+
+
+# ------------------------------------------------------------------------------------------------
+# Algorithm 2 end to end on the small configuration
+# ------------------------------------------------------------------------------------------------
+
+def test_algorithm2_loop_config1(clada, oracle):
+    w = wl.WORKLOADS["c1_small_f32"]
+    rho = w.sparsities[0]
+    weights = wl.layer_weights(w, 0)
+    T = w.prefix_len[0]
+    X = _prefix_inputs(w, [T])
+    off = [0, T]
+    layer = gpu_layer(weights, clada)
+    ws = clada.new_workspace(layer, 1, T)
+    W_in, V_in, W_out = oracle_weights(weights)
+    logits = wl.decode_logits(w, 0)
+    tokens = wl.chosen_tokens(w, logits, 0)
+    xs = wl.hidden_states(w, 0, "decode", 0, w.n_decode)
+    lam = torch.full((1,), 0.80, device="cuda")
+    gam = torch.full((1,), 0.12, device="cuda")
+    mults = [1.0, 1.8, 1.12, 1.92]
+
+    # oracle side
+    A_or = oracle.neuron_scores(wl.to_numpy_bits(X), off, W_in, V_in, W_out)[0]
+    sh_or = [oracle.cogload(logits[t].numpy(), int(tokens[t])) for t in range(w.n_decode)]
+    tau_s = wl.universal_threshold([a for a, _ in sh_or])
+    tau_H = wl.universal_threshold([b for _, b in sh_or])
+
+    # GPU prefill: scores -> calibrated tau_base -> prefill entry point with guard band
+    scores = torch.empty(1, w.d_ff, dtype=torch.float32, device="cuda")
+    clada.clada_prefix_select(layer, X.cuda(), off, None, None, scores, None, None, None, ws)
+    tau_base = torch.empty(1, 1, dtype=torch.float32, device="cuda")
+    clada.clada_tau_from_sparsity(scores, rho, tau_base.view(1))
+    mask0 = torch.empty(1, w.d_ff, dtype=torch.uint8, device="cuda")
+    idx0 = torch.empty(1, w.d_ff, dtype=torch.int32, device="cuda")
+    cnt0 = torch.empty(1, dtype=torch.int32, device="cuda")
+    clada.clada_prefix_select(layer, X.cuda(), off, tau_base.view(1), mults, scores, mask0, idx0, cnt0, ws)
+    tb = float(tau_base.item())
+    assert int(cnt0[0]) == w.d_ff - w.k_cut(rho)
+    assert compare_masks(mask0[0].cpu().numpy(), A_or, tb) == (0, 0)
+
+    s = torch.empty(1, device="cuda")
+    h = torch.empty(1, device="cuda")
+    tau_final = torch.empty(1, 1, device="cuda")
+    y = torch.empty(1, w.d_model, device="cuda")
+    mask = torch.empty(1, w.d_ff, dtype=torch.uint8, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    seen = set()
+    for t in range(w.n_decode):
+        clada.clada_cogload_adjust(logits[t:t + 1].cuda(), tokens[t:t + 1].cuda(), tau_base, lam, gam, tau_s, tau_H,
+                                   s, h, tau_final, status)
+        clada.clada_sparse_ffn_decode(layer, xs[t:t + 1].cuda(), scores, tau_final, 1, y, ws, mask, status=status)
+        torch.cuda.synchronize()
+        s_or, h_or = sh_or[t]
+        assert abs(s.item() - s_or) <= COG_TOL and abs(h.item() - h_or) <= COG_TOL
+        tf_or = oracle.adjust_threshold(np.array([[tb]], np.float32), [0.80], [0.12], tau_s, tau_H, [s_or], [h_or])
+        assert np.float32(tau_final.item()) == tf_or[0, 0]
+        seen.add(round(float(tf_or[0, 0]) / tb, 2))
+        y_or, m_or, _ = oracle.sparse_ffn(xs[t].numpy(), W_in, V_in, W_out, A_or, float(tf_or[0, 0]))
+        assert compare_masks(mask[0].cpu().numpy(), A_or, float(tf_or[0, 0])) == (0, 0)
+        assert rel_inf(y[0].cpu().numpy(), y_or) <= FFN_TOL_F32
+    assert int(status.item()) == 0
+    assert len(seen) >= 3          # the loop exercised several of the four threshold levels
