@@ -1,0 +1,396 @@
+#!/usr/bin/env python
+"""Benchmark of the CLADA sparse-FFN hot path on the Llama-2-7B-shaped layer workload.
+
+One step = one pass of the whole path over one batch of synthetic input:
+    prefill statistics of the 512-token prompt (once), then for each baseline sparsity (40 %, 50 %):
+    guard-band refinement + baseline selection, then 128 decode tokens, each
+    cogload+threshold adjustment (one launch) and the sparse gated FFN (one launch).
+The layer exists in several identical copies at different addresses and decode step t reads copy
+t mod n, so that no step can be served from L2 (one copy's kept rows are 135-162 MB, L2 is 126 MB).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--no-graph]
+
+Prints ONE JSON line (rank 0).  `--impl reference` times the CPU oracle on a bounded sample.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import time
+
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2502_19078_b200 import workloads as wl  # noqa: E402
+
+WORKLOAD = "c2_llama2_7b_layer"
+METRIC = "sparse_ffn_decode_tokens_per_s"
+LAMBDA, GAMMA = 0.80, 0.12
+N_COPIES = 4
+
+
+def _peaks():
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """nvidia-smi sampling of SM clocks and throttle reasons while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100",
+                 "-i", str(self.gpu)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except Exception:
+            self.proc.kill()
+            out = ""
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.splitlines():
+            f = [c.strip() for c in line.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1]))
+                mx.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, val in zip(names, f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        sm.sort()
+        return {"sm_mhz": sm[len(sm) // 2] if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ------------------------------------------------------------------------------------------------
+# our arm
+# ------------------------------------------------------------------------------------------------
+
+class Job:
+    """Device-resident state of one workload instance and the launch sequence of one step."""
+
+    def __init__(self, clada, w, dev, rank: int):
+        self.clada, self.w, self.dev = clada, w, dev
+        T = w.prefix_len[0]
+        self.T, self.N = T, w.n_decode
+        weights = wl.layer_weights(w, 0, dev)
+        wdt = weights["w_down"].t().contiguous()
+        del weights["w_down"]
+        self.layers = []
+        for c in range(N_COPIES):
+            if c == 0:
+                lay = clada.Layer(weights["w_gate"], weights["w_up"], wdt)
+            else:
+                lay = clada.Layer(weights["w_gate"].clone(), weights["w_up"].clone(), wdt.clone())
+            self.layers.append(lay)
+        norms = torch.empty(w.d_ff, dtype=torch.float32, device=dev)
+        clada.clada_down_norms(self.layers[0], norms)
+        for lay in self.layers:
+            lay.set_down_norm(norms)
+        scale = wl.channel_scale(w, dev)
+        # a rank's sequence differs from the other ranks' (independent jobs, no exchange)
+        self.X = wl.hidden_states(w, 0, "prefix", rank, T, dev, scale)
+        self.xs = wl.hidden_states(w, 0, "decode", rank, self.N, dev, scale)
+        self.logits = wl.decode_logits(w, rank, self.N, dev)
+        self.tokens = wl.chosen_tokens(w, self.logits, rank).contiguous()
+        self.off = [0, T]
+        self.ws = clada.new_workspace(self.layers[0], 1, T)
+        f32 = dict(dtype=torch.float32, device=dev)
+        self.scores = torch.empty(1, w.d_ff, **f32)
+        self.mask = torch.empty(1, w.d_ff, dtype=torch.uint8, device=dev)
+        self.idx = torch.empty(1, w.d_ff, dtype=torch.int32, device=dev)
+        self.count = torch.empty(1, dtype=torch.int32, device=dev)
+        self.status = torch.zeros(1, dtype=torch.int32, device=dev)
+        self.lam = torch.full((1,), LAMBDA, **f32)
+        self.gam = torch.full((1,), GAMMA, **f32)
+        self.s = torch.empty(self.N, **f32)
+        self.h = torch.empty(self.N, **f32)
+        self.tau_final = torch.empty(1, 1, **f32)
+        self.y = torch.empty(len(w.sparsities), self.N, w.d_model, **f32)
+        self.guard = [1.0, 1.0 + LAMBDA, 1.0 + GAMMA, 1.0 + LAMBDA + GAMMA]
+        # calibration (stands in for the offline threshold search; not part of a step)
+        clada.clada_prefix_scores(self.layers[0], self.X, self.off, self.scores, self.ws)
+        self.tau_base = []
+        for rho in w.sparsities:
+            t = torch.empty(1, 1, **f32)
+            clada.clada_tau_from_sparsity(self.scores, rho, t.view(1))
+            self.tau_base.append(t)
+        clada.clada_cogload(self.logits, self.tokens, self.s, self.h)
+        torch.cuda.synchronize()
+        self.tau_s = wl.universal_threshold(self.s.tolist())
+        self.tau_H = wl.universal_threshold(self.h.tolist())
+        self.counts = {}
+
+    def step(self):
+        c, w = self.clada, self.w
+        L0 = self.layers[0]
+        c.clada_prefix_scores(L0, self.X, self.off, self.scores, self.ws, self.status)
+        for r, rho in enumerate(w.sparsities):
+            tb = self.tau_base[r]
+            c.clada_refine_scores(L0, self.X, self.off, tb.view(1), self.guard, 1e-4, self.scores, self.ws, self.status)
+            c.clada_select(self.scores, tb.view(1), 1, self.mask, self.idx, self.count)
+            for t in range(self.N):
+                c.clada_cogload_adjust(self.logits[t:t + 1], self.tokens[t:t + 1], tb, self.lam, self.gam,
+                                       self.tau_s, self.tau_H, self.s[t:t + 1], self.h[t:t + 1], self.tau_final,
+                                       self.status)
+                c.clada_sparse_ffn_decode(self.layers[t % N_COPIES], self.xs[t:t + 1], self.scores, self.tau_final, 1,
+                                          self.y[r, t:t + 1], self.ws, status=self.status)
+
+    @property
+    def launches_per_step(self) -> int:
+        return 2 + len(self.w.sparsities) * (3 + 2 * self.N)
+
+    def tokens_per_step(self) -> int:
+        return len(self.w.sparsities) * self.N
+
+    def kept_per_token(self):
+        """Average number of kept neurons per decode token over the step (for algorithmic bytes)."""
+        c = self.clada
+        cnt = torch.empty(1, dtype=torch.int32, device=self.dev)
+        tot = 0
+        for r in range(len(self.w.sparsities)):
+            tb = self.tau_base[r]
+            for t in range(self.N):
+                c.clada_cogload_adjust(self.logits[t:t + 1], self.tokens[t:t + 1], tb, self.lam, self.gam,
+                                       self.tau_s, self.tau_H, self.s[t:t + 1], self.h[t:t + 1], self.tau_final)
+                c.clada_select(self.scores, self.tau_final.view(1), 1, None, None, cnt)
+                tot += int(cnt.item())
+        return tot / self.tokens_per_step()
+
+    def ffn_only_loop(self):
+        """The FFN launches of one sparsity level back to back (for the kernel's own duration)."""
+        for t in range(self.N):
+            self.clada.clada_sparse_ffn_decode(self.layers[t % N_COPIES], self.xs[t:t + 1], self.scores,
+                                               self.tau_base[0], 1, self.y[0, t:t + 1], self.ws)
+
+
+def _timed(fn, steps, dist_barrier):
+    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    dist_barrier()
+    torch.cuda.synchronize()
+    start.record()
+    for _ in range(steps):
+        fn()
+    end.record()
+    torch.cuda.synchronize()
+    dist_barrier()
+    return start.elapsed_time(end)
+
+
+def run_ours(args):
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    import torch.distributed as dist
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+
+    from paper_2502_19078_b200 import binding as clada
+    from paper_2502_19078_b200 import build
+    if rank == 0:
+        build.build()
+    barrier()
+    clada.load()
+    w = wl.WORKLOADS[WORKLOAD]
+    job = Job(clada, w, dev, rank)
+
+    stream = torch.cuda.Stream()
+    graph = None
+    with torch.cuda.stream(stream):
+        for _ in range(max(args.warmup, 3) if not args.graph else 1):
+            job.step()
+        stream.synchronize()
+        if args.graph:
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=stream):
+                job.step()
+            run = graph.replay
+            for _ in range(max(args.warmup, 3)):
+                run()
+        else:
+            run = job.step
+        stream.synchronize()
+        sampler = ClockSampler(local)
+        if rank == 0:
+            sampler.start()
+        ms = _timed(run, args.steps, barrier)
+        clocks = sampler.stop() if rank == 0 else None
+
+        # the FFN kernel alone, same launches, for the roofline
+        job.ffn_only_loop()
+        ffn_ms = _timed(job.ffn_only_loop, 3, lambda: None) / (3 * job.N)
+        kept = job.kept_per_token()
+        kept_base = w.d_ff - w.k_cut(w.sparsities[0])
+
+        # end to end: inputs start in pinned host memory, outputs end there
+        hX, hxs, hlog, htok = (t.cpu().pin_memory() for t in (job.X, job.xs, job.logits, job.tokens))
+        hy = torch.empty(job.y.shape, dtype=job.y.dtype).pin_memory()
+
+        def e2e_step():
+            job.X.copy_(hX, non_blocking=True)
+            job.xs.copy_(hxs, non_blocking=True)
+            job.logits.copy_(hlog, non_blocking=True)
+            job.tokens.copy_(htok, non_blocking=True)
+            run()
+            hy.copy_(job.y, non_blocking=True)
+
+        e2e_step()
+        e2e_ms = _timed(e2e_step, args.steps, barrier)
+        status = int(job.status.item())
+
+    t = torch.tensor([ms, e2e_ms], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms, e2e_ms = float(t[0]), float(t[1])
+    tokens = job.tokens_per_step() * args.steps * world
+    value = tokens / (ms * 1e-3)
+    e2e_value = tokens / (e2e_ms * 1e-3)
+
+    peak, peak_kind = _peaks()
+    eb = w.elem_bytes
+    # algorithmic bytes of one FFN launch: three rows per kept neuron + scores + x in + y out
+    ffn_bytes = kept_base * 3 * w.d_model * eb + w.d_ff * 4 + w.d_model * eb + w.d_model * 4
+    achieved = ffn_bytes / (ffn_ms * 1e-3) / 1e9
+    h2d = sum(x.numel() * x.element_size() for x in (hX, hxs, hlog, htok))
+    d2h = hy.numel() * hy.element_size()
+
+    line = {
+        "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "d_model": w.d_model, "d_ff": w.d_ff, "prefix_tokens": job.T,
+                   "decode_tokens_per_sparsity": job.N, "sparsities": list(w.sparsities), "batch": 1,
+                   "l2": f"inputs larger than L2: {N_COPIES} rotating copies of the layer",
+                   "cuda_graph": bool(args.graph), "avg_kept_neurons_per_token": kept,
+                   "step": "prefix statistics + per sparsity (guard band, select, 128 x (cogload+adjust, sparse FFN))"},
+        "e2e": {"value": e2e_value, "unit": "tokens/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+        "gpu_launches": job.launches_per_step * args.steps,
+        "roofline": {"bound": "hbm", "kernel": "sparse_ffn_kernel", "achieved": achieved, "peak": peak,
+                     "unit": "GB/s", "frac": achieved / peak, "peak_kind": peak_kind, "traffic": None,
+                     "bytes_per_launch": ffn_bytes, "us_per_launch": ffn_ms * 1e3,
+                     "kept_neurons": kept_base},
+        "clocks": clocks, "device_status_word": status,
+    }
+    if rank == 0:
+        if world == 1:
+            line["cpu_baseline"] = cpu_baseline(w)
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+# ------------------------------------------------------------------------------------------------
+# CPU oracle arm (baseline, not a target)
+# ------------------------------------------------------------------------------------------------
+
+def oracle_sample(w, n_prefix=8, n_tokens=6):
+    """Times the oracle, as it stands, on a bounded sample of the workload: the statistics of the first
+    n_prefix prompt tokens, then n_tokens decode tokens (cogload, adjustment, sparse FFN) per sparsity."""
+    import numpy as np
+    from oracle import clada_oracle as orc
+    orc.build()
+    weights = wl.layer_weights(w, 0)
+    W_in, V_in, W_out = (wl.to_numpy_bits(weights[k]) for k in ("w_gate", "w_up", "w_down"))
+    scale = wl.channel_scale(w)
+    X = wl.to_numpy_bits(wl.hidden_states(w, 0, "prefix", 0, n_prefix, "cpu", scale))
+    xs = wl.to_numpy_bits(wl.hidden_states(w, 0, "decode", 0, n_tokens, "cpu", scale))
+    logits = wl.decode_logits(w, 0, n_tokens)
+    tokens = wl.chosen_tokens(w, logits, 0)
+    t0 = time.perf_counter()
+    A = orc.neuron_scores(X, [0, n_prefix], W_in, V_in, W_out)[0]
+    t_prefix = time.perf_counter() - t0
+    t1 = time.perf_counter()
+    n_done = 0
+    for rho in w.sparsities:
+        tau_base = orc.tau_from_sparsity(A.astype(np.float32), rho)
+        for t in range(n_tokens):
+            s, h = orc.cogload(logits[t].numpy(), int(tokens[t]))
+            tf = orc.adjust_threshold(np.array([[tau_base]], np.float32), [LAMBDA], [GAMMA], 6.0, 9.0, [s], [h])
+            orc.sparse_ffn(xs[t], W_in, V_in, W_out, A, float(tf[0, 0]))
+            n_done += 1
+    t_decode = time.perf_counter() - t1
+    return {"tokens": n_done, "decode_s": t_decode, "prefix_tokens": n_prefix, "prefix_s": t_prefix,
+            "cores": orc.num_threads()}
+
+
+def cpu_baseline(w):
+    r = oracle_sample(w)
+    return {"value": r["tokens"] / r["decode_s"], "unit": "tokens/s", "cores": r["cores"], "kind": "oracle",
+            "sample": (f"{r['tokens']} decode tokens ({r['tokens'] // len(w.sparsities)} per sparsity) of the "
+                       f"full-size layer: cogload + adjustment + sparse FFN, {r['decode_s']:.1f} s; scores from the "
+                       f"first {r['prefix_tokens']} prompt tokens ({r['prefix_s']:.1f} s, not in the rate)")}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    w = wl.WORKLOADS[WORKLOAD]
+    for _ in range(min(args.warmup, 1)):
+        oracle_sample(w, n_prefix=2, n_tokens=1)
+    tot_tokens, tot_s, last = 0, 0.0, None
+    for _ in range(args.steps):
+        last = oracle_sample(w, n_prefix=4, n_tokens=3)
+        tot_tokens += last["tokens"]
+        tot_s += last["decode_s"]
+    value = tot_tokens / tot_s
+    sample = (f"per step {last['tokens']} decode tokens of the full-size layer (cogload + adjustment + sparse FFN); "
+              f"scores from the first {last['prefix_tokens']} prompt tokens, outside the rate")
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": "tokens/s",
+        "n_gpus": int(os.environ.get("WORLD_SIZE", "1")), "steps": args.steps, "warmup": min(args.warmup, 1),
+        "ms_per_step": 1e3 * tot_s / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f64", "data": "synthetic", "config": {"workload": WORKLOAD, "sample": sample},
+        "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": last["cores"], "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-graph", dest="graph", action="store_false")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()
