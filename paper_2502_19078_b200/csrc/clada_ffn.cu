@@ -4,11 +4,11 @@
 // One persistent cooperative kernel per (layer, sequence):
 //   prologue  every CTA scans the F scores against tau (warp ballots), learns the number of kept
 //             neurons and takes an equal share [r0, r1) of the kept list in ascending order;
-//   stream    the CTA walks its share G neurons at a time.  Thread t owns the same 16-byte column
-//             vectors of every row (x and the partial y for those columns live in registers), so the
-//             three rows of a neuron are read with fully coalesced 128-bit loads.  The loads of the
-//             next group's gate/up rows are issued before the current group's down rows are consumed,
-//             which keeps HBM requests in flight across the CTA-wide dot-product reduction;
+//   stream    a producer thread copies the three contiguous rows of each kept neuron into a ring of
+//             shared-memory stages with bulk asynchronous copies (mbarrier-tracked), which keeps
+//             ~200 KB of HBM requests in flight per SM whatever the consumers are doing.  Consumer
+//             thread t owns the same 16-byte column vectors of every row (x and the partial y for
+//             those columns live in registers) and reads the staged rows from shared memory;
 //   epilogue  each CTA stores its fp32 partial y, all CTAs meet at a bounded grid barrier, then every
 //             CTA sums a slice of columns over all partials in CTA order (deterministic) and writes y.
 #include <math.h>
@@ -33,7 +33,6 @@ struct FfnParams {
     int d_model, d_ff;
 };
 
-constexpr int kFfnMaxWarps = 8;
 constexpr unsigned kBarrierSpinLimit = 1u << 20;  // polls ~100 ns apart: gives up after ~0.1 s
 
 // Bounded grid-wide barrier on two self-resetting counters in the workspace control block.
@@ -68,21 +67,87 @@ __device__ bool grid_barrier(WsCtrl *ctrl, unsigned n_ctas) {
     return s_ok != 0;
 }
 
+// ---- mbarrier / bulk-copy primitives (bounded waits) -------------------------------------------
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) {
+    return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+constexpr unsigned kMbarSpinLimit = 1u << 22;  // each failed try_wait already sleeps in hardware
+// Waits for the phase with the given parity; gives up (returns false) after kMbarSpinLimit tries.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+    for (unsigned i = 0; i < kMbarSpinLimit; ++i)
+        if (mbar_try_wait(bar, parity)) return true;
+    return false;
+}
+// One contiguous row, global -> this CTA's shared memory, completion counted on an mbarrier.
+// Both addresses are 16-byte aligned and bytes is a multiple of 16.
+__device__ __forceinline__ void bulk_load_row(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar)
+                 : "memory");
+}
+__device__ __forceinline__ uint4 lds128(uint32_t addr) {
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+    return v;
+}
+
+constexpr int kConsumers = 256;              // consumer threads (8 warps)
+constexpr int kFfnThreads = kConsumers + 32;  // + one producer warp
+constexpr int kMaxStages = 16;
+
+// One CTA per SM.  Warp 8 lane 0 streams the three rows of each kept neuron of this CTA's share into
+// a ring of shared-memory stages with bulk async copies (one stage = gate row | up row | down row);
+// the 8 consumer warps take stages G at a time: dot products from shared memory against x in
+// registers, CTA-wide sum, silu * up, then the down row is added into the register-resident partial y.
 template <typename T, int NV, int G>
-__global__ void __launch_bounds__(kFfnMaxWarps *kWarp, 2)
-sparse_ffn_kernel(const FfnParams p) {
+__global__ void __launch_bounds__(kFfnThreads, 1)
+sparse_ffn_kernel(const FfnParams p, const int n_stages) {
     constexpr int E = Elem<T>::kPerVec;
-    extern __shared__ __align__(16) unsigned char smem_raw[];
+    extern __shared__ __align__(128) unsigned char smem_raw[];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int nthreads = blockDim.x, nwarps = nthreads >> 5;
+    constexpr int nwarps = kFfnThreads / kWarp;
     const int cta = blockIdx.x, n_ctas = gridDim.x;
     const int F = p.d_ff, d = p.d_model;
-    const int vpr = d / E;  // 16-byte vectors per row
+    const int vpr = d / E;                       // 16-byte vectors per row
+    const uint32_t row_bytes = (uint32_t)vpr * 16u;
+    const uint32_t stage_bytes = 3u * row_bytes;
 
-    // shared: kept list of this CTA (dynamic), per-warp scan totals, dot-product exchange
-    int *s_list = reinterpret_cast<int *>(smem_raw);
-    __shared__ int s_wtot[kFfnMaxWarps];
-    __shared__ float s_dot[2][kFfnMaxWarps][2 * G];
+    // dynamic shared memory: ring | full[kMaxStages] | empty[kMaxStages] | kept list
+    const uint32_t ring = smem_u32(smem_raw);
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem_raw + (size_t)n_stages * stage_bytes);
+    const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + kMaxStages);
+    int *s_list = reinterpret_cast<int *>(bars + 2 * kMaxStages);
+    __shared__ int s_wtot[nwarps];
+    __shared__ float s_dot[2][kConsumers / kWarp][2 * G];
+
+    if (tid == 0) {
+        for (int s = 0; s < n_stages; ++s) {
+            mbar_init(full0 + 8 * s, 1);                      // the producer's expect_tx arrival
+            mbar_init(empty0 + 8 * s, kConsumers / kWarp);    // one arrival per consumer warp
+        }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
 
     // ---- prologue: threshold test and this CTA's share of the kept list -------------------------
     const float tau = *p.tau;
@@ -98,6 +163,7 @@ sparse_ffn_kernel(const FfnParams p) {
     if (lane == 0) s_wtot[warp] = n;
     __syncthreads();
     int base = 0, n_act = 0;
+#pragma unroll
     for (int w = 0; w < nwarps; ++w) {
         const int v = s_wtot[w];
         base += (w < warp) ? v : 0;
@@ -121,120 +187,127 @@ sparse_ffn_kernel(const FfnParams p) {
     }
     if (p.count_out && cta == 0 && tid == 0) *p.count_out = n_act;
     const int my_n = r1 - r0;
+    __syncthreads();  // s_list and the mbarriers are ready
 
-    // ---- x and the partial y of this thread's columns, in registers -----------------------------
-    float xr[NV][E], acc[NV][E];
-    bool vok[NV];
-#pragma unroll
-    for (int i = 0; i < NV; ++i) {
-        const int v = tid + i * nthreads;
-        vok[i] = v < vpr;
-        uint4 q = make_uint4(0, 0, 0, 0);
-        if (vok[i]) q = *(reinterpret_cast<const uint4 *>(p.x) + v);
-        Elem<T>::unpack(q, xr[i]);
-#pragma unroll
-        for (int e = 0; e < E; ++e) acc[i][e] = 0.f;
-    }
-    __syncthreads();  // s_list complete
+    float acc[NV][E];
+    bool timed_out = false;
 
-    const uint4 *Wg = reinterpret_cast<const uint4 *>(p.w_gate);
-    const uint4 *Wu = reinterpret_cast<const uint4 *>(p.w_up);
-    const uint4 *Wd = reinterpret_cast<const uint4 *>(p.w_down_t);
-
-    uint4 qg[G][NV], qu[G][NV], qd[G][NV];
-    int jn[G];  // neurons of the group whose gate/up rows are in flight
-
-    auto issue_gate_up = [&](int g0) {
-#pragma unroll
-        for (int g = 0; g < G; ++g) {
-            jn[g] = (g0 + g < my_n) ? s_list[g0 + g] : -1;
-#pragma unroll
-            for (int i = 0; i < NV; ++i) {
-                qg[g][i] = make_uint4(0, 0, 0, 0);
-                qu[g][i] = make_uint4(0, 0, 0, 0);
-                if (jn[g] >= 0 && vok[i]) {
-                    const size_t off = (size_t)jn[g] * vpr + tid + i * nthreads;
-                    qg[g][i] = ldg_stream(Wg + off);
-                    qu[g][i] = ldg_stream(Wu + off);
-                }
-            }
-        }
-    };
-
-    issue_gate_up(0);
-    int buf = 0;
-    for (int g0 = 0; g0 < my_n; g0 += G, buf ^= 1) {
-        // partial dot products over this thread's columns
-        float pd[2 * G];
-        int jcur[G];
-#pragma unroll
-        for (int g = 0; g < G; ++g) {
-            jcur[g] = jn[g];
-            float sg = 0.f, su = 0.f;
-#pragma unroll
-            for (int i = 0; i < NV; ++i) {
-                float fg[E], fu[E];
-                Elem<T>::unpack(qg[g][i], fg);
-                Elem<T>::unpack(qu[g][i], fu);
-#pragma unroll
-                for (int e = 0; e < E; ++e) {
-                    sg = fmaf(fg[e], xr[i][e], sg);
-                    su = fmaf(fu[e], xr[i][e], su);
-                }
-            }
-            pd[2 * g] = sg;
-            pd[2 * g + 1] = su;
-        }
-        // down rows of the same neurons: issue now, consume after the reduction
-#pragma unroll
-        for (int g = 0; g < G; ++g)
-#pragma unroll
-            for (int i = 0; i < NV; ++i) {
-                qd[g][i] = make_uint4(0, 0, 0, 0);
-                if (jcur[g] >= 0 && vok[i])
-                    qd[g][i] = ldg_stream(Wd + (size_t)jcur[g] * vpr + tid + i * nthreads);
-            }
-        // CTA-wide sums in a fixed order: lanes by butterfly, then warps 0..nwarps-1
-#pragma unroll
-        for (int k = 0; k < 2 * G; ++k) pd[k] = warp_sum(pd[k]);
+    if (warp == kConsumers / kWarp) {
+        // ---- producer ------------------------------------------------------------------------
         if (lane == 0) {
-#pragma unroll
-            for (int k = 0; k < 2 * G; ++k) s_dot[buf][warp][k] = pd[k];
-        }
-        __syncthreads();
-        // next group's gate/up rows go out before the FMAs below
-        issue_gate_up(g0 + G);
-        float h[G];
-#pragma unroll
-        for (int g = 0; g < G; ++g) {
-            float sg = 0.f, su = 0.f;
-            for (int w = 0; w < nwarps; ++w) {
-                sg += s_dot[buf][w][2 * g];
-                su += s_dot[buf][w][2 * g + 1];
+            const char *Wg = static_cast<const char *>(p.w_gate);
+            const char *Wu = static_cast<const char *>(p.w_up);
+            const char *Wd = static_cast<const char *>(p.w_down_t);
+            int issued = 0;
+            for (int i = 0; i < my_n; ++i) {
+                const int s = i % n_stages, use = i / n_stages;
+                if (!mbar_wait(empty0 + 8 * s, (use & 1) ^ 1)) {  // a fresh barrier passes parity 1 at once
+                    timed_out = true;
+                    break;
+                }
+                const size_t off = (size_t)s_list[i] * row_bytes;
+                const uint32_t dst = ring + (uint32_t)s * stage_bytes, bar = full0 + 8 * s;
+                mbar_expect_tx(bar, stage_bytes);
+                bulk_load_row(dst, Wg + off, row_bytes, bar);
+                bulk_load_row(dst + row_bytes, Wu + off, row_bytes, bar);
+                bulk_load_row(dst + 2 * row_bytes, Wd + off, row_bytes, bar);
+                issued = i + 1;
             }
-            h[g] = (jcur[g] >= 0) ? silu_f(sg) * su : 0.f;
+            // Never leave with copies in flight: the last use of every stage must have landed.
+            for (int i = max(0, issued - n_stages); i < issued; ++i)
+                if (!mbar_wait(full0 + 8 * (i % n_stages), (i / n_stages) & 1)) timed_out = true;
         }
+    } else {
+        // ---- consumers -----------------------------------------------------------------------
+        float xr[NV][E];
+        bool vok[NV];
 #pragma unroll
-        for (int g = 0; g < G; ++g)
+        for (int i = 0; i < NV; ++i) {
+            const int v = tid + i * kConsumers;
+            vok[i] = v < vpr;
+            uint4 q = make_uint4(0, 0, 0, 0);
+            if (vok[i]) q = *(reinterpret_cast<const uint4 *>(p.x) + v);
+            Elem<T>::unpack(q, xr[i]);
 #pragma unroll
-            for (int i = 0; i < NV; ++i) {
-                float fd[E];
-                Elem<T>::unpack(qd[g][i], fd);
+            for (int e = 0; e < E; ++e) acc[i][e] = 0.f;
+        }
+        int buf = 0;
+        for (int g0 = 0; g0 < my_n; g0 += G, buf ^= 1) {
+            float pd[2 * G];
+            uint32_t st_addr[G];
 #pragma unroll
-                for (int e = 0; e < E; ++e) acc[i][e] = fmaf(h[g], fd[e], acc[i][e]);
+            for (int g = 0; g < G; ++g) {
+                const int i = g0 + g;
+                float sg = 0.f, su = 0.f;
+                st_addr[g] = ring + (uint32_t)(i % n_stages) * stage_bytes;
+                if (i < my_n) {
+                    if (!timed_out && !mbar_wait(full0 + 8 * (i % n_stages), (i / n_stages) & 1)) timed_out = true;
+#pragma unroll
+                    for (int k = 0; k < NV; ++k) {
+                        if (!vok[k]) continue;
+                        const uint32_t a = st_addr[g] + (uint32_t)(tid + k * kConsumers) * 16u;
+                        float fg[E], fu[E];
+                        Elem<T>::unpack(lds128(a), fg);
+                        Elem<T>::unpack(lds128(a + row_bytes), fu);
+#pragma unroll
+                        for (int e = 0; e < E; ++e) {
+                            sg = fmaf(fg[e], xr[k][e], sg);
+                            su = fmaf(fu[e], xr[k][e], su);
+                        }
+                    }
+                }
+                pd[2 * g] = sg;
+                pd[2 * g + 1] = su;
             }
+            // CTA-wide sums in a fixed order: lanes by butterfly, then warps 0..7
+#pragma unroll
+            for (int k = 0; k < 2 * G; ++k) pd[k] = warp_sum(pd[k]);
+            if (lane == 0) {
+#pragma unroll
+                for (int k = 0; k < 2 * G; ++k) s_dot[buf][warp][k] = pd[k];
+            }
+            asm volatile("bar.sync 1, %0;" ::"n"(kConsumers) : "memory");
+#pragma unroll
+            for (int g = 0; g < G; ++g) {
+                if (g0 + g >= my_n) continue;
+                float sg = 0.f, su = 0.f;
+#pragma unroll
+                for (int w = 0; w < kConsumers / kWarp; ++w) {
+                    sg += s_dot[buf][w][2 * g];
+                    su += s_dot[buf][w][2 * g + 1];
+                }
+                const float h = silu_f(sg) * su;
+#pragma unroll
+                for (int k = 0; k < NV; ++k) {
+                    if (!vok[k]) continue;
+                    float fd[E];
+                    Elem<T>::unpack(lds128(st_addr[g] + 2 * row_bytes + (uint32_t)(tid + k * kConsumers) * 16u), fd);
+#pragma unroll
+                    for (int e = 0; e < E; ++e) acc[k][e] = fmaf(h, fd[e], acc[k][e]);
+                }
+            }
+            // hand the stages back to the producer
+            __syncwarp();
+            if (lane == 0) {
+#pragma unroll
+                for (int g = 0; g < G; ++g)
+                    if (g0 + g < my_n) mbar_arrive(empty0 + 8 * ((g0 + g) % n_stages));
+            }
+        }
+        // partial y of this CTA
+        float *mine = p.partials + (size_t)cta * d;
+#pragma unroll
+        for (int i = 0; i < NV; ++i) {
+            if (!vok[i]) continue;
+            float4 *dst = reinterpret_cast<float4 *>(mine + (size_t)(tid + i * kConsumers) * E);
+#pragma unroll
+            for (int e = 0; e < E; e += 4)
+                dst[e / 4] = make_float4(acc[i][e], acc[i][e + 1], acc[i][e + 2], acc[i][e + 3]);
+        }
     }
+    if (timed_out && p.status) atomicOr(p.status, CLADA_STATUS_TIMEOUT);
 
-    // ---- epilogue: partial rows, grid barrier, deterministic column reduction -------------------
-    float *mine = p.partials + (size_t)cta * d;
-#pragma unroll
-    for (int i = 0; i < NV; ++i) {
-        if (!vok[i]) continue;
-        float4 *dst = reinterpret_cast<float4 *>(mine + (size_t)(tid + i * nthreads) * E);
-#pragma unroll
-        for (int e = 0; e < E; e += 4)
-            dst[e / 4] = make_float4(acc[i][e], acc[i][e + 1], acc[i][e + 2], acc[i][e + 3]);
-    }
+    // ---- epilogue: grid barrier, deterministic column reduction ---------------------------------
     if (!grid_barrier(p.ctrl, (unsigned)n_ctas)) {
         if (tid == 0 && p.status) atomicOr(p.status, CLADA_STATUS_TIMEOUT);
         return;
@@ -244,7 +317,7 @@ sparse_ffn_kernel(const FfnParams p) {
     const int ngroups = d / 4;
     for (int q = cta + warp * n_ctas; q < ngroups; q += n_ctas * nwarps) {
         float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll 4
+#pragma unroll 5
         for (int r = lane; r < n_ctas; r += kWarp) {
             const float4 v = __ldcg(reinterpret_cast<const float4 *>(p.partials + (size_t)r * d) + q);
             s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
@@ -267,27 +340,30 @@ sparse_ffn_kernel(const FfnParams p) {
 // ---- host side ------------------------------------------------------------------------------
 
 template <typename T, int NV, int G>
-static int launch_variant(const FfnParams &p, int threads, cudaStream_t st) {
-    static int cached_ctas[64][kFfnMaxWarps + 1] = {};
+static int launch_variant(const FfnParams &p, cudaStream_t st) {
+    constexpr int E = Elem<T>::kPerVec;
+    static bool configured[64] = {};
     DeviceInfo di;
     int rc = device_info(&di);
     if (rc != CLADA_OK) return rc;
     auto kern = sparse_ffn_kernel<T, NV, G>;
-    // dynamic shared memory: the kept-list share of one CTA at the smallest grid we may use
-    const size_t smem = ((size_t)(p.d_ff / di.num_sms + 2) * sizeof(int) + 15) & ~(size_t)15;
-    int &per_sm = cached_ctas[di.device & 63][threads / kWarp];
-    if (per_sm == 0) {
-        int occ = 0;
-        CLADA_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kern, threads, smem));
-        if (occ < 1) return CLADA_ERR_UNSUPPORTED;
-        per_sm = occ > 4 ? 4 : occ;
+    const size_t stage_bytes = 3 * (size_t)(p.d_model / E) * 16;
+    const size_t tail = 2 * kMaxStages * sizeof(uint64_t) + (size_t)(p.d_ff / di.num_sms + 2) * sizeof(int);
+    const size_t budget = (size_t)di.max_smem_optin - 1024;  // leave room for the static arrays
+    if (budget < tail + 2 * G * stage_bytes) return CLADA_ERR_UNSUPPORTED;
+    int n_stages = (int)((budget - tail) / stage_bytes);
+    if (n_stages > kMaxStages) n_stages = kMaxStages;
+    const size_t smem = (size_t)n_stages * stage_bytes + tail;
+    if (!configured[di.device & 63]) {
+        CLADA_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, di.max_smem_optin - 1024));
+        configured[di.device & 63] = true;
     }
-    const int grid = di.num_sms * per_sm;
     FfnParams params = p;
-    void *args[] = {&params};
+    int stages_arg = n_stages;
+    void *args[] = {&params, &stages_arg};
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(grid);
-    cfg.blockDim = dim3(threads);
+    cfg.gridDim = dim3(di.num_sms);  // one CTA per SM: co-resident by construction, checked by the launch
+    cfg.blockDim = dim3(kFfnThreads);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
@@ -303,12 +379,10 @@ template <typename T>
 static int launch_ffn(const FfnParams &p, cudaStream_t st) {
     constexpr int E = Elem<T>::kPerVec;
     const int vpr = p.d_model / E;
-    // threads: enough to cover a row with at most 4 vectors each, a multiple of 32, at most 256
-    if (vpr <= 128) return launch_variant<T, 1, 4>(p, ((vpr + 31) / 32) * 32, st);
-    if (vpr <= 256) return launch_variant<T, 1, 4>(p, 256, st);
-    if (vpr <= 512) return launch_variant<T, 2, 2>(p, 256, st);
-    if (vpr <= 768) return launch_variant<T, 3, 1>(p, 256, st);
-    if (vpr <= 1024) return launch_variant<T, 4, 1>(p, 256, st);
+    if (vpr <= 256) return launch_variant<T, 1, 2>(p, st);
+    if (vpr <= 512) return launch_variant<T, 2, 2>(p, st);
+    if (vpr <= 768) return launch_variant<T, 3, 2>(p, st);
+    if (vpr <= 1024) return launch_variant<T, 4, 2>(p, st);
     return CLADA_ERR_UNSUPPORTED;
 }
 
@@ -331,7 +405,7 @@ extern "C" int clada_sparse_ffn_decode(const clada_layer *layer, const void *x, 
     DeviceInfo di;
     rc = device_info(&di);
     if (rc != CLADA_OK) return rc;
-    const size_t need = kWsCtrlBytes + (size_t)di.num_sms * 4 * layer->d_model * sizeof(float);
+    const size_t need = kWsCtrlBytes + (size_t)di.num_sms * layer->d_model * sizeof(float);
     if (ws_bytes < need) return CLADA_ERR_WORKSPACE;
 
     const size_t esz = elem_size(layer->dtype);
