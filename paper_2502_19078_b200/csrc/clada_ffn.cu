@@ -2,7 +2,7 @@
 //   kept = { j : A_j >= tau_final },  y = sum_{j in kept} silu(w_gate_j . x) (w_up_j . x) w_down_t[j,:]
 //
 // One persistent cooperative kernel per (layer, sequence):
-//   prologue  every CTA scans the F scores against tau (warp ballots), learns the number of kept
+//   prologue  every CTA scans the F scores against tau (batched loads, warp ballots), learns the number of kept
 //             neurons and takes an equal share [r0, r1) of the kept list in ascending order;
 //   stream    a producer thread copies the three contiguous rows of each kept neuron into a ring of
 //             shared-memory stages with bulk asynchronous copies (mbarrier-tracked), which keeps
@@ -137,7 +137,8 @@ sparse_ffn_kernel(const FfnParams p, const int n_stages) {
     const uint32_t ring = smem_u32(smem_raw);
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem_raw + (size_t)n_stages * stage_bytes);
     const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + kMaxStages);
-    int *s_list = reinterpret_cast<int *>(bars + 2 * kMaxStages);
+    unsigned *s_bal = reinterpret_cast<unsigned *>(bars + 2 * kMaxStages);  // one ballot word per chunk
+    int *s_list = reinterpret_cast<int *>(s_bal + (F + kWarp - 1) / kWarp);
     __shared__ int s_wtot[nwarps];
     __shared__ float s_dot[2][kConsumers / kWarp][2 * G];
 
@@ -150,15 +151,31 @@ sparse_ffn_kernel(const FfnParams p, const int n_stages) {
     }
 
     // ---- prologue: threshold test and this CTA's share of the kept list -------------------------
+    // Pass 1 reads the scores in batches of independent loads (one memory round trip per batch, not
+    // per chunk) and leaves one ballot word per 32-neuron chunk in shared memory; pass 2 ranks from
+    // those words without touching global memory again.
     const float tau = *p.tau;
     const int chunks = (F + kWarp - 1) / kWarp;
     const int per_warp = (chunks + nwarps - 1) / nwarps;
     const int c0 = warp * per_warp, c1 = min(chunks, c0 + per_warp);
     int n = 0;
-    for (int c = c0; c < c1; ++c) {
-        const int j = c * kWarp + lane;
-        const bool keep = j < F && p.scores[j] >= tau;
-        n += __popc(__ballot_sync(0xffffffffu, keep));
+    constexpr int kBatch = 16;
+    for (int c = c0; c < c1; c += kBatch) {
+        float v[kBatch];
+#pragma unroll
+        for (int u = 0; u < kBatch; ++u) {
+            const int j = (c + u) * kWarp + lane;
+            v[u] = (c + u < c1 && j < F) ? __ldg(p.scores + j) : -INFINITY;
+        }
+#pragma unroll
+        for (int u = 0; u < kBatch; ++u) {
+            if (c + u < c1) {  // warp-uniform
+                const int j = (c + u) * kWarp + lane;
+                const unsigned bal = __ballot_sync(0xffffffffu, j < F && v[u] >= tau);
+                if (lane == 0) s_bal[c + u] = bal;
+                n += __popc(bal);
+            }
+        }
     }
     if (lane == 0) s_wtot[warp] = n;
     __syncthreads();
@@ -175,8 +192,8 @@ sparse_ffn_kernel(const FfnParams p, const int n_stages) {
     const int m1 = (int)(((int64_t)F * (cta + 1)) / n_ctas);
     for (int c = c0; c < c1; ++c) {
         const int j = c * kWarp + lane;
-        const bool keep = j < F && p.scores[j] >= tau;
-        const unsigned bal = __ballot_sync(0xffffffffu, keep);
+        const unsigned bal = s_bal[c];
+        const bool keep = (bal >> lane) & 1u;
         const int rank = base + __popc(bal & ((1u << lane) - 1u));
         if (keep && rank >= r0 && rank < r1) {
             s_list[rank - r0] = j;
@@ -348,7 +365,8 @@ static int launch_variant(const FfnParams &p, cudaStream_t st) {
     if (rc != CLADA_OK) return rc;
     auto kern = sparse_ffn_kernel<T, NV, G>;
     const size_t stage_bytes = 3 * (size_t)(p.d_model / E) * 16;
-    const size_t tail = 2 * kMaxStages * sizeof(uint64_t) + (size_t)(p.d_ff / di.num_sms + 2) * sizeof(int);
+    const size_t tail = 2 * kMaxStages * sizeof(uint64_t) + (size_t)((p.d_ff + 31) / 32) * sizeof(unsigned) +
+                        (size_t)(p.d_ff / di.num_sms + 2) * sizeof(int);
     const size_t budget = (size_t)di.max_smem_optin - 1024;  // leave room for the static arrays
     if (budget < tail + 2 * G * stage_bytes) return CLADA_ERR_UNSUPPORTED;
     int n_stages = (int)((budget - tail) / stage_bytes);
