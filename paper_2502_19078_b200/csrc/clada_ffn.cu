@@ -1,14 +1,16 @@
 // Sparse gated FFN for one decode token per sequence (Algorithm 2, generation phase):
 //   kept = { j : A_j >= tau_final },  y = sum_{j in kept} silu(w_gate_j . x) (w_up_j . x) w_down_t[j,:]
 //
-// One persistent cooperative kernel per (layer, sequence):
-//   prologue  every CTA scans the F scores against tau (batched loads, warp ballots), learns the number of kept
-//             neurons and takes an equal share [r0, r1) of the kept list in ascending order;
+// One persistent cooperative kernel per (layer, sequence), one CTA per SM:
+//   prologue  every CTA tests all F scores against tau (each thread owns whole 32-neuron chunks, so all
+//             its loads are independent: one memory round trip), a block scan ranks the chunks, and the
+//             CTA takes an equal share [r0, r1) of the kept neurons in ascending order;
 //   stream    a producer thread copies the three contiguous rows of each kept neuron into a ring of
 //             shared-memory stages with bulk asynchronous copies (mbarrier-tracked), which keeps
 //             ~200 KB of HBM requests in flight per SM whatever the consumers are doing.  Consumer
 //             thread t owns the same 16-byte column vectors of every row (x and the partial y for
-//             those columns live in registers) and reads the staged rows from shared memory;
+//             those columns live in registers) and reads the staged rows from shared memory, four
+//             neurons per CTA-wide reduction;
 //   epilogue  each CTA stores its fp32 partial y, all CTAs meet at a bounded grid barrier, then every
 //             CTA sums a slice of columns over all partials in CTA order (deterministic) and writes y.
 #include <math.h>
@@ -33,7 +35,7 @@ struct FfnParams {
     int d_model, d_ff;
 };
 
-constexpr unsigned kBarrierSpinLimit = 1u << 20;  // polls ~100 ns apart: gives up after ~0.1 s
+constexpr unsigned kBarrierSpinLimit = 1u << 22;  // polls of an L2 word: gives up after ~1 s at most
 
 // Bounded grid-wide barrier on two self-resetting counters in the workspace control block.
 // Returns false if the wait expired.
@@ -43,16 +45,16 @@ __device__ bool grid_barrier(WsCtrl *ctrl, unsigned n_ctas) {
     if (threadIdx.x == 0) {
         __threadfence();
         atomicAdd(&ctrl->arrive, 1u);
-        unsigned spins = 0;
+        unsigned spins = 0, seen;
         int ok = 1;
-        while (*reinterpret_cast<volatile unsigned *>(&ctrl->arrive) < n_ctas) {
+        for (;;) {
+            asm volatile("ld.acquire.gpu.u32 %0, [%1];" : "=r"(seen) : "l"(&ctrl->arrive) : "memory");
+            if (seen >= n_ctas) break;
             if (++spins > kBarrierSpinLimit) {
                 ok = 0;
                 break;
             }
-            __nanosleep(64);
         }
-        __threadfence();
         s_ok = ok;
         if (ok) {
             const unsigned left = atomicAdd(&ctrl->depart, 1u);
@@ -112,104 +114,171 @@ __device__ __forceinline__ uint4 lds128(uint32_t addr) {
     return v;
 }
 
-constexpr int kConsumers = 256;              // consumer threads (8 warps)
-constexpr int kFfnThreads = kConsumers + 32;  // + one producer warp
-constexpr int kMaxStages = 16;
+// A 16-byte vector as E/2 pairs of fp32 (exact), ready for the packed two-wide FMA.
+template <typename T> struct Pairs;
+template <> struct Pairs<float> {
+    static constexpr int kPairs = 2;
+    __device__ static __forceinline__ void unpack(const uint4 &v, float2 (&f)[2]) {
+        f[0] = make_float2(__uint_as_float(v.x), __uint_as_float(v.y));
+        f[1] = make_float2(__uint_as_float(v.z), __uint_as_float(v.w));
+    }
+};
+template <> struct Pairs<__nv_bfloat16> {
+    static constexpr int kPairs = 4;
+    __device__ static __forceinline__ void unpack(const uint4 &v, float2 (&f)[4]) {
+        f[0] = make_float2(bf16_lo(v.x), bf16_hi(v.x));
+        f[1] = make_float2(bf16_lo(v.y), bf16_hi(v.y));
+        f[2] = make_float2(bf16_lo(v.z), bf16_hi(v.z));
+        f[3] = make_float2(bf16_lo(v.w), bf16_hi(v.w));
+    }
+};
 
-// One CTA per SM.  Warp 8 lane 0 streams the three rows of each kept neuron of this CTA's share into
-// a ring of shared-memory stages with bulk async copies (one stage = gate row | up row | down row);
-// the 8 consumer warps take stages G at a time: dot products from shared memory against x in
-// registers, CTA-wide sum, silu * up, then the down row is added into the register-resident partial y.
-template <typename T, int NV, int G>
+constexpr int kConsumers = 512;               // consumer threads (16 warps)
+constexpr int kConsWarps = kConsumers / kWarp;
+constexpr int kFfnThreads = kConsumers + 32;  // + one producer warp
+constexpr int kFfnWarps = kFfnThreads / kWarp;
+constexpr int kMaxStages = 16;
+constexpr int G = 4;                          // neurons per CTA-wide reduction
+
+template <typename T, int NV>
 __global__ void __launch_bounds__(kFfnThreads, 1)
 sparse_ffn_kernel(const FfnParams p, const int n_stages) {
     constexpr int E = Elem<T>::kPerVec;
+    constexpr int P = Pairs<T>::kPairs;
     extern __shared__ __align__(128) unsigned char smem_raw[];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    constexpr int nwarps = kFfnThreads / kWarp;
     const int cta = blockIdx.x, n_ctas = gridDim.x;
     const int F = p.d_ff, d = p.d_model;
-    const int vpr = d / E;                       // 16-byte vectors per row
+    const int vpr = d / E;  // 16-byte vectors per row
     const uint32_t row_bytes = (uint32_t)vpr * 16u;
     const uint32_t stage_bytes = 3u * row_bytes;
+    const int chunks = (F + kWarp - 1) / kWarp;
 
     // dynamic shared memory: ring | full[kMaxStages] | empty[kMaxStages] | kept list
     const uint32_t ring = smem_u32(smem_raw);
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem_raw + (size_t)n_stages * stage_bytes);
     const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + kMaxStages);
-    unsigned *s_bal = reinterpret_cast<unsigned *>(bars + 2 * kMaxStages);  // one ballot word per chunk
-    int *s_list = reinterpret_cast<int *>(s_bal + (F + kWarp - 1) / kWarp);
-    __shared__ int s_wtot[nwarps];
-    __shared__ float s_dot[2][kConsumers / kWarp][2 * G];
+    int *s_list = reinterpret_cast<int *>(bars + 2 * kMaxStages);
+    __shared__ int s_wtot[kFfnWarps];
+    __shared__ __align__(16) float s_dot[2][2 * G][kConsWarps];
 
     if (tid == 0) {
         for (int s = 0; s < n_stages; ++s) {
-            mbar_init(full0 + 8 * s, 1);                      // the producer's expect_tx arrival
-            mbar_init(empty0 + 8 * s, kConsumers / kWarp);    // one arrival per consumer warp
+            mbar_init(full0 + 8 * s, 1);            // the producer's expect_tx arrival
+            mbar_init(empty0 + 8 * s, kConsWarps);  // one arrival per consumer warp
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
 
-    // ---- prologue: threshold test and this CTA's share of the kept list -------------------------
-    // Pass 1 reads the scores in batches of independent loads (one memory round trip per batch, not
-    // per chunk) and leaves one ballot word per 32-neuron chunk in shared memory; pass 2 ranks from
-    // those words without touching global memory again.
+    // x of this thread's columns (consumers), requested before the scan so the latencies overlap
+    float2 xr[NV][P];
+    bool vok[NV];
+#pragma unroll
+    for (int i = 0; i < NV; ++i) {
+        const int v = tid + i * kConsumers;
+        vok[i] = tid < kConsumers && v < vpr;
+        uint4 q = make_uint4(0, 0, 0, 0);
+        if (vok[i]) q = *(reinterpret_cast<const uint4 *>(p.x) + v);
+        Pairs<T>::unpack(q, xr[i]);
+    }
+
+    // ---- prologue: threshold test, ranks, this CTA's share of the kept list ---------------------
     const float tau = *p.tau;
-    const int chunks = (F + kWarp - 1) / kWarp;
-    const int per_warp = (chunks + nwarps - 1) / nwarps;
-    const int c0 = warp * per_warp, c1 = min(chunks, c0 + per_warp);
-    int n = 0;
-    constexpr int kBatch = 16;
-    for (int c = c0; c < c1; c += kBatch) {
-        float v[kBatch];
-#pragma unroll
-        for (int u = 0; u < kBatch; ++u) {
-            const int j = (c + u) * kWarp + lane;
-            v[u] = (c + u < c1 && j < F) ? __ldg(p.scores + j) : -INFINITY;
-        }
-#pragma unroll
-        for (int u = 0; u < kBatch; ++u) {
-            if (c + u < c1) {  // warp-uniform
-                const int j = (c + u) * kWarp + lane;
-                const unsigned bal = __ballot_sync(0xffffffffu, j < F && v[u] >= tau);
-                if (lane == 0) s_bal[c + u] = bal;
-                n += __popc(bal);
-            }
-        }
-    }
-    if (lane == 0) s_wtot[warp] = n;
-    __syncthreads();
-    int base = 0, n_act = 0;
-#pragma unroll
-    for (int w = 0; w < nwarps; ++w) {
-        const int v = s_wtot[w];
-        base += (w < warp) ? v : 0;
-        n_act += v;
-    }
-    const int r0 = (int)(((int64_t)n_act * cta) / n_ctas);
-    const int r1 = (int)(((int64_t)n_act * (cta + 1)) / n_ctas);
+    const bool vec_ok = (reinterpret_cast<uintptr_t>(p.scores) & 15u) == 0;
+    int run = 0;  // kept neurons in the chunks of all earlier batches
+    int r0 = 0, r1 = 0, n_act = 0;
     const int m0 = (int)(((int64_t)F * cta) / n_ctas);  // slice of the mask this CTA writes
     const int m1 = (int)(((int64_t)F * (cta + 1)) / n_ctas);
-    for (int c = c0; c < c1; ++c) {
-        const int j = c * kWarp + lane;
-        const unsigned bal = s_bal[c];
-        const bool keep = (bal >> lane) & 1u;
-        const int rank = base + __popc(bal & ((1u << lane) - 1u));
-        if (keep && rank >= r0 && rank < r1) {
-            s_list[rank - r0] = j;
-            if (p.idx_out) p.idx_out[rank] = j;
+    // Two sweeps over the chunk batches: the first counts (n_act fixes r0, r1), the second ranks.
+    // A batch is one chunk per thread; F <= 32 * kFfnThreads needs a single batch.
+    unsigned my_bal[2] = {0u, 0u};
+    const int n_batches = (chunks + kFfnThreads - 1) / kFfnThreads;
+    for (int sweep = 0; sweep < 2; ++sweep) {
+        run = 0;
+        for (int bt = 0; bt < n_batches; ++bt) {
+            const int q = bt * kFfnThreads + tid;  // this thread's chunk
+            unsigned bal = 0;
+            if (sweep == 0 || bt >= 2) {
+                if (q < chunks) {
+                    const int j0 = q * kWarp;
+                    if (vec_ok && j0 + kWarp <= F) {
+                        float4 v[8];
+#pragma unroll
+                        for (int u = 0; u < 8; ++u) v[u] = __ldg(reinterpret_cast<const float4 *>(p.scores + j0) + u);
+#pragma unroll
+                        for (int u = 0; u < 8; ++u) {
+                            bal |= (v[u].x >= tau ? 1u : 0u) << (4 * u);
+                            bal |= (v[u].y >= tau ? 1u : 0u) << (4 * u + 1);
+                            bal |= (v[u].z >= tau ? 1u : 0u) << (4 * u + 2);
+                            bal |= (v[u].w >= tau ? 1u : 0u) << (4 * u + 3);
+                        }
+                    } else {
+                        float v[kWarp];
+#pragma unroll
+                        for (int u = 0; u < kWarp; ++u) v[u] = (j0 + u < F) ? __ldg(p.scores + j0 + u) : -INFINITY;
+#pragma unroll
+                        for (int u = 0; u < kWarp; ++u) bal |= (v[u] >= tau ? 1u : 0u) << u;
+                    }
+                }
+                if (bt < 2) my_bal[bt] = bal;
+            } else {
+                bal = my_bal[bt];
+            }
+            // block-wide exclusive scan of popc(bal) in thread order
+            const int cnt = __popc(bal);
+            int incl = cnt;
+#pragma unroll
+            for (int o = 1; o < kWarp; o <<= 1) {
+                const int t = __shfl_up_sync(0xffffffffu, incl, o);
+                if (lane >= o) incl += t;
+            }
+            __syncthreads();  // s_wtot free again
+            if (lane == kWarp - 1) s_wtot[warp] = incl;
+            __syncthreads();
+            int wbase = 0, btot = 0;
+#pragma unroll
+            for (int w = 0; w < kFfnWarps; ++w) {
+                const int v = s_wtot[w];
+                wbase += (w < warp) ? v : 0;
+                btot += v;
+            }
+            if (sweep == 1 && q < chunks) {
+                int rank = run + wbase + incl - cnt;  // rank of this chunk's first kept neuron
+                const int j0 = q * kWarp;
+                if (rank < r1 && rank + cnt > r0) {   // chunk holds part of this CTA's share
+                    unsigned b = bal;
+                    while (b) {
+                        const int u = __ffs(b) - 1;
+                        b &= b - 1;
+                        if (rank >= r0 && rank < r1) {
+                            s_list[rank - r0] = j0 + u;
+                            if (p.idx_out) p.idx_out[rank] = j0 + u;
+                        }
+                        ++rank;
+                    }
+                }
+                if (p.mask_out && j0 < m1 && j0 + kWarp > m0) {
+                    for (int u = 0; u < kWarp; ++u) {
+                        const int j = j0 + u;
+                        if (j >= m0 && j < m1) p.mask_out[j] = (bal >> u) & 1u;
+                    }
+                }
+            }
+            run += btot;
         }
-        if (p.mask_out && j >= m0 && j < m1) p.mask_out[j] = keep ? 1 : 0;
-        base += __popc(bal);
+        if (sweep == 0) {
+            n_act = run;
+            r0 = (int)(((int64_t)n_act * cta) / n_ctas);
+            r1 = (int)(((int64_t)n_act * (cta + 1)) / n_ctas);
+        }
     }
     if (p.count_out && cta == 0 && tid == 0) *p.count_out = n_act;
     const int my_n = r1 - r0;
     __syncthreads();  // s_list and the mbarriers are ready
 
-    float acc[NV][E];
     bool timed_out = false;
 
-    if (warp == kConsumers / kWarp) {
+    if (warp == kConsWarps) {
         // ---- producer ------------------------------------------------------------------------
         if (lane == 0) {
             const char *Wg = static_cast<const char *>(p.w_gate);
@@ -236,18 +305,12 @@ sparse_ffn_kernel(const FfnParams p, const int n_stages) {
         }
     } else {
         // ---- consumers -----------------------------------------------------------------------
-        float xr[NV][E];
-        bool vok[NV];
+        float2 acc[NV][P];
 #pragma unroll
-        for (int i = 0; i < NV; ++i) {
-            const int v = tid + i * kConsumers;
-            vok[i] = v < vpr;
-            uint4 q = make_uint4(0, 0, 0, 0);
-            if (vok[i]) q = *(reinterpret_cast<const uint4 *>(p.x) + v);
-            Elem<T>::unpack(q, xr[i]);
+        for (int i = 0; i < NV; ++i)
 #pragma unroll
-            for (int e = 0; e < E; ++e) acc[i][e] = 0.f;
-        }
+            for (int e = 0; e < P; ++e) acc[i][e] = make_float2(0.f, 0.f);
+        const bool b16 = lane & 16, b8 = lane & 8, b4 = lane & 4;
         int buf = 0;
         for (int g0 = 0; g0 < my_n; g0 += G, buf ^= 1) {
             float pd[2 * G];
@@ -255,7 +318,7 @@ sparse_ffn_kernel(const FfnParams p, const int n_stages) {
 #pragma unroll
             for (int g = 0; g < G; ++g) {
                 const int i = g0 + g;
-                float sg = 0.f, su = 0.f;
+                float2 sg = make_float2(0.f, 0.f), su = make_float2(0.f, 0.f);
                 st_addr[g] = ring + (uint32_t)(i % n_stages) * stage_bytes;
                 if (i < my_n) {
                     if (!timed_out && !mbar_wait(full0 + 8 * (i % n_stages), (i / n_stages) & 1)) timed_out = true;
@@ -263,44 +326,61 @@ sparse_ffn_kernel(const FfnParams p, const int n_stages) {
                     for (int k = 0; k < NV; ++k) {
                         if (!vok[k]) continue;
                         const uint32_t a = st_addr[g] + (uint32_t)(tid + k * kConsumers) * 16u;
-                        float fg[E], fu[E];
-                        Elem<T>::unpack(lds128(a), fg);
-                        Elem<T>::unpack(lds128(a + row_bytes), fu);
+                        float2 fg[P], fu[P];
+                        Pairs<T>::unpack(lds128(a), fg);
+                        Pairs<T>::unpack(lds128(a + row_bytes), fu);
 #pragma unroll
-                        for (int e = 0; e < E; ++e) {
-                            sg = fmaf(fg[e], xr[k][e], sg);
-                            su = fmaf(fu[e], xr[k][e], su);
+                        for (int e = 0; e < P; ++e) {
+                            sg = __ffma2_rn(fg[e], xr[k][e], sg);
+                            su = __ffma2_rn(fu[e], xr[k][e], su);
                         }
                     }
                 }
-                pd[2 * g] = sg;
-                pd[2 * g + 1] = su;
+                pd[2 * g] = sg.x + sg.y;
+                pd[2 * g + 1] = su.x + su.y;
             }
-            // CTA-wide sums in a fixed order: lanes by butterfly, then warps 0..7
+            // Warp sums of the 8 values by a halving butterfly (9 shuffles): after it every lane of
+            // quad q holds the warp total of value q.  Fixed order, so results repeat bit for bit.
+            float b[4], c[2], v8;
 #pragma unroll
-            for (int k = 0; k < 2 * G; ++k) pd[k] = warp_sum(pd[k]);
-            if (lane == 0) {
-#pragma unroll
-                for (int k = 0; k < 2 * G; ++k) s_dot[buf][warp][k] = pd[k];
+            for (int i = 0; i < 4; ++i) {
+                const float send = b16 ? pd[i] : pd[i + 4];
+                b[i] = (b16 ? pd[i + 4] : pd[i]) + __shfl_xor_sync(0xffffffffu, send, 16);
             }
+#pragma unroll
+            for (int i = 0; i < 2; ++i) {
+                const float send = b8 ? b[i] : b[i + 2];
+                c[i] = (b8 ? b[i + 2] : b[i]) + __shfl_xor_sync(0xffffffffu, send, 8);
+            }
+            v8 = (b4 ? c[1] : c[0]) + __shfl_xor_sync(0xffffffffu, b4 ? c[0] : c[1], 4);
+            v8 += __shfl_xor_sync(0xffffffffu, v8, 2);
+            v8 += __shfl_xor_sync(0xffffffffu, v8, 1);
+            // lane 4q holds value index: bit4 -> +4, bit3 -> +2, bit2 -> +1
+            if ((lane & 3) == 0) s_dot[buf][(b16 ? 4 : 0) + (b8 ? 2 : 0) + (b4 ? 1 : 0)][warp] = v8;
             asm volatile("bar.sync 1, %0;" ::"n"(kConsumers) : "memory");
+            // Cross-warp sums: lane l adds 4 consecutive warps of value l/4 (16 warps = 4 lanes per
+            // value), the quad finishes by butterfly; then gate lanes form h = silu(gate) * up.
+            float tot;
+            {
+                const float4 q4 = *reinterpret_cast<const float4 *>(&s_dot[buf][lane >> 2][(lane & 3) * 4]);
+                tot = (q4.x + q4.y) + (q4.z + q4.w);
+                tot += __shfl_xor_sync(0xffffffffu, tot, 1);
+                tot += __shfl_xor_sync(0xffffffffu, tot, 2);
+            }
+            const float up = __shfl_xor_sync(0xffffffffu, tot, 4);  // value 2g+1 sits 4 lanes above value 2g
+            const float hval = silu_f(tot) * up;                    // meaningful on lanes 8g..8g+3
 #pragma unroll
             for (int g = 0; g < G; ++g) {
+                const float h = __shfl_sync(0xffffffffu, hval, 8 * g);
                 if (g0 + g >= my_n) continue;
-                float sg = 0.f, su = 0.f;
-#pragma unroll
-                for (int w = 0; w < kConsumers / kWarp; ++w) {
-                    sg += s_dot[buf][w][2 * g];
-                    su += s_dot[buf][w][2 * g + 1];
-                }
-                const float h = silu_f(sg) * su;
+                const float2 h2 = make_float2(h, h);
 #pragma unroll
                 for (int k = 0; k < NV; ++k) {
                     if (!vok[k]) continue;
-                    float fd[E];
-                    Elem<T>::unpack(lds128(st_addr[g] + 2 * row_bytes + (uint32_t)(tid + k * kConsumers) * 16u), fd);
+                    float2 fd[P];
+                    Pairs<T>::unpack(lds128(st_addr[g] + 2 * row_bytes + (uint32_t)(tid + k * kConsumers) * 16u), fd);
 #pragma unroll
-                    for (int e = 0; e < E; ++e) acc[k][e] = fmaf(h, fd[e], acc[k][e]);
+                    for (int e = 0; e < P; ++e) acc[k][e] = __ffma2_rn(h2, fd[e], acc[k][e]);
                 }
             }
             // hand the stages back to the producer
@@ -318,8 +398,8 @@ sparse_ffn_kernel(const FfnParams p, const int n_stages) {
             if (!vok[i]) continue;
             float4 *dst = reinterpret_cast<float4 *>(mine + (size_t)(tid + i * kConsumers) * E);
 #pragma unroll
-            for (int e = 0; e < E; e += 4)
-                dst[e / 4] = make_float4(acc[i][e], acc[i][e + 1], acc[i][e + 2], acc[i][e + 3]);
+            for (int e = 0; e < P; e += 2)
+                dst[e / 2] = make_float4(acc[i][e].x, acc[i][e].y, acc[i][e + 1].x, acc[i][e + 1].y);
         }
     }
     if (timed_out && p.status) atomicOr(p.status, CLADA_STATUS_TIMEOUT);
@@ -330,14 +410,22 @@ sparse_ffn_kernel(const FfnParams p, const int n_stages) {
         return;
     }
     // columns in groups of 4 (float4); a warp sums one group: lane l adds partial rows l, l+32, ...
-    // in order, then the 32 lane sums combine by butterfly.
+    // in order (five loads in flight at a time), then the 32 lane sums combine by butterfly.
     const int ngroups = d / 4;
-    for (int q = cta + warp * n_ctas; q < ngroups; q += n_ctas * nwarps) {
+    for (int q = cta + warp * n_ctas; q < ngroups; q += n_ctas * kFfnWarps) {
         float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll 5
-        for (int r = lane; r < n_ctas; r += kWarp) {
-            const float4 v = __ldcg(reinterpret_cast<const float4 *>(p.partials + (size_t)r * d) + q);
-            s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
+        for (int rb = 0; rb < n_ctas; rb += 5 * kWarp) {
+            float4 v[5];
+#pragma unroll
+            for (int u = 0; u < 5; ++u) {
+                const int r = rb + u * kWarp + lane;
+                v[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (r < n_ctas) v[u] = __ldcg(reinterpret_cast<const float4 *>(p.partials + (size_t)r * d) + q);
+            }
+#pragma unroll
+            for (int u = 0; u < 5; ++u) {
+                s.x += v[u].x; s.y += v[u].y; s.z += v[u].z; s.w += v[u].w;
+            }
         }
         s.x = warp_sum(s.x); s.y = warp_sum(s.y); s.z = warp_sum(s.z); s.w = warp_sum(s.w);
         if (lane == 0) {
@@ -356,31 +444,30 @@ sparse_ffn_kernel(const FfnParams p, const int n_stages) {
 
 // ---- host side ------------------------------------------------------------------------------
 
-template <typename T, int NV, int G>
+template <typename T, int NV>
 static int launch_variant(const FfnParams &p, cudaStream_t st) {
     constexpr int E = Elem<T>::kPerVec;
     static bool configured[64] = {};
     DeviceInfo di;
     int rc = device_info(&di);
     if (rc != CLADA_OK) return rc;
-    auto kern = sparse_ffn_kernel<T, NV, G>;
+    auto kern = sparse_ffn_kernel<T, NV>;
     const size_t stage_bytes = 3 * (size_t)(p.d_model / E) * 16;
-    const size_t tail = 2 * kMaxStages * sizeof(uint64_t) + (size_t)((p.d_ff + 31) / 32) * sizeof(unsigned) +
-                        (size_t)(p.d_ff / di.num_sms + 2) * sizeof(int);
-    const size_t budget = (size_t)di.max_smem_optin - 1024;  // leave room for the static arrays
+    const size_t tail = 2 * kMaxStages * sizeof(uint64_t) + (size_t)(p.d_ff / di.num_sms + 2) * sizeof(int);
+    const size_t budget = (size_t)di.max_smem_optin - 2048;  // leave room for the static arrays
     if (budget < tail + 2 * G * stage_bytes) return CLADA_ERR_UNSUPPORTED;
     int n_stages = (int)((budget - tail) / stage_bytes);
     if (n_stages > kMaxStages) n_stages = kMaxStages;
     const size_t smem = (size_t)n_stages * stage_bytes + tail;
     if (!configured[di.device & 63]) {
-        CLADA_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, di.max_smem_optin - 1024));
+        CLADA_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)budget));
         configured[di.device & 63] = true;
     }
     FfnParams params = p;
     int stages_arg = n_stages;
     void *args[] = {&params, &stages_arg};
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(di.num_sms);  // one CTA per SM: co-resident by construction, checked by the launch
+    cfg.gridDim = dim3(di.num_sms);  // one CTA per SM
     cfg.blockDim = dim3(kFfnThreads);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = st;
@@ -397,10 +484,8 @@ template <typename T>
 static int launch_ffn(const FfnParams &p, cudaStream_t st) {
     constexpr int E = Elem<T>::kPerVec;
     const int vpr = p.d_model / E;
-    if (vpr <= 256) return launch_variant<T, 1, 2>(p, st);
-    if (vpr <= 512) return launch_variant<T, 2, 2>(p, st);
-    if (vpr <= 768) return launch_variant<T, 3, 2>(p, st);
-    if (vpr <= 1024) return launch_variant<T, 4, 2>(p, st);
+    if (vpr <= kConsumers) return launch_variant<T, 1>(p, st);
+    if (vpr <= 2 * kConsumers) return launch_variant<T, 2>(p, st);
     return CLADA_ERR_UNSUPPORTED;
 }
 
