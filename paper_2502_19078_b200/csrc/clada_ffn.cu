@@ -455,7 +455,7 @@ static int launch_variant(const FfnParams &p, cudaStream_t st) {
     const size_t stage_bytes = 3 * (size_t)(p.d_model / E) * 16;
     const size_t tail = 2 * kMaxStages * sizeof(uint64_t) + (size_t)(p.d_ff / di.num_sms + 2) * sizeof(int);
     const size_t budget = (size_t)di.max_smem_optin - 2048;  // leave room for the static arrays
-    if (budget < tail + 2 * G * stage_bytes) return CLADA_ERR_UNSUPPORTED;
+    if (budget < tail + G * stage_bytes) return CLADA_ERR_UNSUPPORTED;  // a group needs G stages at once
     int n_stages = (int)((budget - tail) / stage_bytes);
     if (n_stages > kMaxStages) n_stages = kMaxStages;
     const size_t smem = (size_t)n_stages * stage_bytes + tail;
