@@ -101,12 +101,38 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
         if (mbar_try_wait(bar, parity)) return true;
     return false;
 }
-// One contiguous row, global -> this CTA's shared memory, completion counted on an mbarrier.
-// Both addresses are 16-byte aligned and bytes is a multiple of 16.
-__device__ __forceinline__ void bulk_load_row(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar)
-                 : "memory");
+// Bulk copies move one contiguous row, global -> this CTA's shared memory, completion counted on an
+// mbarrier; both addresses are 16-byte aligned and the size is a multiple of 16.
+// L2 policies: weights are read once (evict first), the small per-call vectors are re-read by every
+// CTA and by the next call (evict last), so the streaming rows do not push them out of L2.
+__device__ __forceinline__ uint64_t policy_evict_first() {
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+__device__ __forceinline__ uint64_t policy_evict_last() {
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+__device__ __forceinline__ void bulk_load_row_hint(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar,
+                                                   uint64_t policy) {
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
+        ::"r"(dst), "l"(src), "r"(bytes), "r"(bar), "l"(policy)
+        : "memory");
+}
+__device__ __forceinline__ float ld_keep(const float *p, uint64_t policy) {
+    float v;
+    asm volatile("ld.global.L2::cache_hint.f32 %0, [%1], %2;" : "=f"(v) : "l"(p), "l"(policy));
+    return v;
+}
+__device__ __forceinline__ float4 ld_keep4(const float4 *p, uint64_t policy) {
+    float4 v;
+    asm volatile("ld.global.L2::cache_hint.v4.f32 {%0,%1,%2,%3}, [%4], %5;"
+                 : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w)
+                 : "l"(p), "l"(policy));
+    return v;
 }
 __device__ __forceinline__ uint4 lds128(uint32_t addr) {
     uint4 v;
@@ -139,6 +165,7 @@ constexpr int kFfnThreads = kConsumers + 32;  // + one producer warp
 constexpr int kFfnWarps = kFfnThreads / kWarp;
 constexpr int kMaxStages = 16;
 constexpr int G = 4;                          // neurons per CTA-wide reduction
+constexpr int kMaxBatches = 4;                // prologue batches: d_ff <= 4 * 32 * kFfnThreads
 
 template <typename T, int NV>
 __global__ void __launch_bounds__(kFfnThreads, 1)
@@ -170,6 +197,7 @@ sparse_ffn_kernel(const FfnParams p, const int n_stages) {
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
 
+    const uint64_t keep_policy = policy_evict_last();
     // x of this thread's columns (consumers), requested before the scan so the latencies overlap
     float2 xr[NV][P];
     bool vok[NV];
@@ -183,93 +211,90 @@ sparse_ffn_kernel(const FfnParams p, const int n_stages) {
     }
 
     // ---- prologue: threshold test, ranks, this CTA's share of the kept list ---------------------
-    const float tau = *p.tau;
+    // A batch is one 32-neuron chunk per thread (all its loads independent); F <= 32 * kFfnThreads
+    // needs a single batch.  Each batch: keep-bits word per thread, block-wide exclusive scan.
+    const float tau = ld_keep(p.tau, keep_policy);
     const bool vec_ok = (reinterpret_cast<uintptr_t>(p.scores) & 15u) == 0;
-    int run = 0;  // kept neurons in the chunks of all earlier batches
-    int r0 = 0, r1 = 0, n_act = 0;
+    unsigned bal[kMaxBatches];
+    int first_rank[kMaxBatches];  // rank of this thread's chunk's first kept neuron
+    int n_act = 0;
+    const int n_batches = (chunks + kFfnThreads - 1) / kFfnThreads;
+#pragma unroll
+    for (int bt = 0; bt < kMaxBatches; ++bt) {
+        bal[bt] = 0u;
+        first_rank[bt] = 0;
+        if (bt >= n_batches) continue;  // uniform
+        const int q = bt * kFfnThreads + tid;  // this thread's chunk
+        if (q < chunks) {
+            const int j0 = q * kWarp;
+            unsigned w = 0;
+            if (vec_ok && j0 + kWarp <= F) {
+                float4 v[8];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) v[u] = ld_keep4(reinterpret_cast<const float4 *>(p.scores + j0) + u, keep_policy);
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    w |= (v[u].x >= tau ? 1u : 0u) << (4 * u);
+                    w |= (v[u].y >= tau ? 1u : 0u) << (4 * u + 1);
+                    w |= (v[u].z >= tau ? 1u : 0u) << (4 * u + 2);
+                    w |= (v[u].w >= tau ? 1u : 0u) << (4 * u + 3);
+                }
+            } else {
+                float v[kWarp];
+#pragma unroll
+                for (int u = 0; u < kWarp; ++u) v[u] = (j0 + u < F) ? ld_keep(p.scores + j0 + u, keep_policy) : -INFINITY;
+#pragma unroll
+                for (int u = 0; u < kWarp; ++u) w |= (v[u] >= tau ? 1u : 0u) << u;
+            }
+            bal[bt] = w;
+        }
+        const int cnt = __popc(bal[bt]);
+        int incl = cnt;
+#pragma unroll
+        for (int o = 1; o < kWarp; o <<= 1) {
+            const int t = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += t;
+        }
+        if (bt > 0) __syncthreads();  // s_wtot free again
+        if (lane == kWarp - 1) s_wtot[warp] = incl;
+        __syncthreads();
+        int wbase = 0, btot = 0;
+#pragma unroll
+        for (int w = 0; w < kFfnWarps; ++w) {
+            const int v = s_wtot[w];
+            wbase += (w < warp) ? v : 0;
+            btot += v;
+        }
+        first_rank[bt] = n_act + wbase + incl - cnt;
+        n_act += btot;
+    }
+    const int r0 = (int)(((int64_t)n_act * cta) / n_ctas);
+    const int r1 = (int)(((int64_t)n_act * (cta + 1)) / n_ctas);
     const int m0 = (int)(((int64_t)F * cta) / n_ctas);  // slice of the mask this CTA writes
     const int m1 = (int)(((int64_t)F * (cta + 1)) / n_ctas);
-    // Two sweeps over the chunk batches: the first counts (n_act fixes r0, r1), the second ranks.
-    // A batch is one chunk per thread; F <= 32 * kFfnThreads needs a single batch.
-    unsigned my_bal[2] = {0u, 0u};
-    const int n_batches = (chunks + kFfnThreads - 1) / kFfnThreads;
-    for (int sweep = 0; sweep < 2; ++sweep) {
-        run = 0;
-        for (int bt = 0; bt < n_batches; ++bt) {
-            const int q = bt * kFfnThreads + tid;  // this thread's chunk
-            unsigned bal = 0;
-            if (sweep == 0 || bt >= 2) {
-                if (q < chunks) {
-                    const int j0 = q * kWarp;
-                    if (vec_ok && j0 + kWarp <= F) {
-                        float4 v[8];
 #pragma unroll
-                        for (int u = 0; u < 8; ++u) v[u] = __ldg(reinterpret_cast<const float4 *>(p.scores + j0) + u);
-#pragma unroll
-                        for (int u = 0; u < 8; ++u) {
-                            bal |= (v[u].x >= tau ? 1u : 0u) << (4 * u);
-                            bal |= (v[u].y >= tau ? 1u : 0u) << (4 * u + 1);
-                            bal |= (v[u].z >= tau ? 1u : 0u) << (4 * u + 2);
-                            bal |= (v[u].w >= tau ? 1u : 0u) << (4 * u + 3);
-                        }
-                    } else {
-                        float v[kWarp];
-#pragma unroll
-                        for (int u = 0; u < kWarp; ++u) v[u] = (j0 + u < F) ? __ldg(p.scores + j0 + u) : -INFINITY;
-#pragma unroll
-                        for (int u = 0; u < kWarp; ++u) bal |= (v[u] >= tau ? 1u : 0u) << u;
-                    }
+    for (int bt = 0; bt < kMaxBatches; ++bt) {
+        const int q = bt * kFfnThreads + tid;
+        if (bt >= n_batches || q >= chunks) continue;
+        const int j0 = q * kWarp;
+        int rank = first_rank[bt];
+        if (rank < r1 && rank + __popc(bal[bt]) > r0) {  // chunk holds part of this CTA's share
+            unsigned b = bal[bt];
+            while (b) {
+                const int u = __ffs(b) - 1;
+                b &= b - 1;
+                if (rank >= r0 && rank < r1) {
+                    s_list[rank - r0] = j0 + u;
+                    if (p.idx_out) p.idx_out[rank] = j0 + u;
                 }
-                if (bt < 2) my_bal[bt] = bal;
-            } else {
-                bal = my_bal[bt];
+                ++rank;
             }
-            // block-wide exclusive scan of popc(bal) in thread order
-            const int cnt = __popc(bal);
-            int incl = cnt;
-#pragma unroll
-            for (int o = 1; o < kWarp; o <<= 1) {
-                const int t = __shfl_up_sync(0xffffffffu, incl, o);
-                if (lane >= o) incl += t;
-            }
-            __syncthreads();  // s_wtot free again
-            if (lane == kWarp - 1) s_wtot[warp] = incl;
-            __syncthreads();
-            int wbase = 0, btot = 0;
-#pragma unroll
-            for (int w = 0; w < kFfnWarps; ++w) {
-                const int v = s_wtot[w];
-                wbase += (w < warp) ? v : 0;
-                btot += v;
-            }
-            if (sweep == 1 && q < chunks) {
-                int rank = run + wbase + incl - cnt;  // rank of this chunk's first kept neuron
-                const int j0 = q * kWarp;
-                if (rank < r1 && rank + cnt > r0) {   // chunk holds part of this CTA's share
-                    unsigned b = bal;
-                    while (b) {
-                        const int u = __ffs(b) - 1;
-                        b &= b - 1;
-                        if (rank >= r0 && rank < r1) {
-                            s_list[rank - r0] = j0 + u;
-                            if (p.idx_out) p.idx_out[rank] = j0 + u;
-                        }
-                        ++rank;
-                    }
-                }
-                if (p.mask_out && j0 < m1 && j0 + kWarp > m0) {
-                    for (int u = 0; u < kWarp; ++u) {
-                        const int j = j0 + u;
-                        if (j >= m0 && j < m1) p.mask_out[j] = (bal >> u) & 1u;
-                    }
-                }
-            }
-            run += btot;
         }
-        if (sweep == 0) {
-            n_act = run;
-            r0 = (int)(((int64_t)n_act * cta) / n_ctas);
-            r1 = (int)(((int64_t)n_act * (cta + 1)) / n_ctas);
+        if (p.mask_out && j0 < m1 && j0 + kWarp > m0) {
+            for (int u = 0; u < kWarp; ++u) {
+                const int j = j0 + u;
+                if (j >= m0 && j < m1) p.mask_out[j] = (bal[bt] >> u) & 1u;
+            }
         }
     }
     if (p.count_out && cta == 0 && tid == 0) *p.count_out = n_act;
@@ -284,6 +309,7 @@ sparse_ffn_kernel(const FfnParams p, const int n_stages) {
             const char *Wg = static_cast<const char *>(p.w_gate);
             const char *Wu = static_cast<const char *>(p.w_up);
             const char *Wd = static_cast<const char *>(p.w_down_t);
+            const uint64_t stream_policy = policy_evict_first();
             int issued = 0;
             for (int i = 0; i < my_n; ++i) {
                 const int s = i % n_stages, use = i / n_stages;
@@ -294,9 +320,9 @@ sparse_ffn_kernel(const FfnParams p, const int n_stages) {
                 const size_t off = (size_t)s_list[i] * row_bytes;
                 const uint32_t dst = ring + (uint32_t)s * stage_bytes, bar = full0 + 8 * s;
                 mbar_expect_tx(bar, stage_bytes);
-                bulk_load_row(dst, Wg + off, row_bytes, bar);
-                bulk_load_row(dst + row_bytes, Wu + off, row_bytes, bar);
-                bulk_load_row(dst + 2 * row_bytes, Wd + off, row_bytes, bar);
+                bulk_load_row_hint(dst, Wg + off, row_bytes, bar, stream_policy);
+                bulk_load_row_hint(dst + row_bytes, Wu + off, row_bytes, bar, stream_policy);
+                bulk_load_row_hint(dst + 2 * row_bytes, Wd + off, row_bytes, bar, stream_policy);
                 issued = i + 1;
             }
             // Never leave with copies in flight: the last use of every stage must have landed.
@@ -484,6 +510,7 @@ template <typename T>
 static int launch_ffn(const FfnParams &p, cudaStream_t st) {
     constexpr int E = Elem<T>::kPerVec;
     const int vpr = p.d_model / E;
+    if (p.d_ff > kMaxBatches * kWarp * kFfnThreads) return CLADA_ERR_UNSUPPORTED;
     if (vpr <= kConsumers) return launch_variant<T, 1>(p, st);
     if (vpr <= 2 * kConsumers) return launch_variant<T, 2>(p, st);
     return CLADA_ERR_UNSUPPORTED;
