@@ -77,6 +77,8 @@ cogload_kernel(const T *__restrict__ logits, int64_t V, int64_t row_stride,
     const int b = blockIdx.x;
     const T *row = logits + (size_t)b * row_stride;
     const int tid = threadIdx.x;
+    pdl_launch_dependents();
+    pdl_wait();
 
     SoftStat st = stat_empty();
     bool bad = false;
@@ -192,16 +194,24 @@ static int launch_cogload(const void *logits, int32_t dtype, int32_t B, int64_t 
     if (dtype != CLADA_F32 && dtype != CLADA_BF16) return CLADA_ERR_DTYPE;
     if (B <= 0 || V <= 0 || row_stride < V) return CLADA_ERR_SHAPE;
     if (reinterpret_cast<uintptr_t>(logits) % elem_size(dtype)) return CLADA_ERR_ALIGN;
-    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(B);
+    cfg.blockDim = dim3(kCogThreads);
+    cfg.stream = static_cast<cudaStream_t>(stream);
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
     if (dtype == CLADA_F32)
-        cogload_kernel<float><<<B, kCogThreads, 0, st>>>(
-            static_cast<const float *>(logits), V, row_stride, token_id, surprisal, entropy, status,
-            tau_base, lambda, gamma, tau_s, tau_H, L, tau_final);
+        CLADA_CUDA_TRY(cudaLaunchKernelEx(&cfg, cogload_kernel<float>, static_cast<const float *>(logits), V,
+                                          row_stride, token_id, surprisal, entropy, status, tau_base, lambda, gamma,
+                                          tau_s, tau_H, L, tau_final));
     else
-        cogload_kernel<__nv_bfloat16><<<B, kCogThreads, 0, st>>>(
-            static_cast<const __nv_bfloat16 *>(logits), V, row_stride, token_id, surprisal, entropy,
-            status, tau_base, lambda, gamma, tau_s, tau_H, L, tau_final);
-    CLADA_CUDA_TRY(cudaGetLastError());
+        CLADA_CUDA_TRY(cudaLaunchKernelEx(&cfg, cogload_kernel<__nv_bfloat16>,
+                                          static_cast<const __nv_bfloat16 *>(logits), V, row_stride, token_id,
+                                          surprisal, entropy, status, tau_base, lambda, gamma, tau_s, tau_H, L,
+                                          tau_final));
     return CLADA_OK;
 }
 

@@ -189,15 +189,18 @@ sparse_ffn_kernel(const FfnParams p, const int n_stages) {
     __shared__ int s_wtot[kFfnWarps];
     __shared__ __align__(16) float s_dot[2][2 * G][kConsWarps];
 
-    if (tid == 0) {
+    pdl_launch_dependents();  // the next kernel in the stream may be scheduled as SMs free up
+    if (tid == kConsumers) {  // the producer warp sets the ring up while the others start loading
         for (int s = 0; s < n_stages; ++s) {
             mbar_init(full0 + 8 * s, 1);            // the producer's expect_tx arrival
             mbar_init(empty0 + 8 * s, kConsWarps);  // one arrival per consumer warp
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
+    pdl_wait();  // everything below may read what the previous kernel wrote
 
     const uint64_t keep_policy = policy_evict_last();
+    const float tau = ld_keep(p.tau, keep_policy);
     // x of this thread's columns (consumers), requested before the scan so the latencies overlap
     float2 xr[NV][P];
     bool vok[NV];
@@ -213,7 +216,6 @@ sparse_ffn_kernel(const FfnParams p, const int n_stages) {
     // ---- prologue: threshold test, ranks, this CTA's share of the kept list ---------------------
     // A batch is one 32-neuron chunk per thread (all its loads independent); F <= 32 * kFfnThreads
     // needs a single batch.  Each batch: keep-bits word per thread, block-wide exclusive scan.
-    const float tau = ld_keep(p.tau, keep_policy);
     const bool vec_ok = (reinterpret_cast<uintptr_t>(p.scores) & 15u) == 0;
     unsigned bal[kMaxBatches];
     int first_rank[kMaxBatches];  // rank of this thread's chunk's first kept neuron
@@ -497,11 +499,13 @@ static int launch_variant(const FfnParams &p, cudaStream_t st) {
     cfg.blockDim = dim3(kFfnThreads);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = st;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeCooperative;  // all CTAs co-resident: the grid barrier cannot starve
     attr[0].val.cooperative = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;  // hide the launch latency
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = 2;
     CLADA_CUDA_TRY(cudaLaunchKernelExC(&cfg, reinterpret_cast<const void *>(kern), args));
     return CLADA_OK;
 }

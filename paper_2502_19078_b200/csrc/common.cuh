@@ -88,6 +88,13 @@ template <> struct Elem<__nv_bfloat16> {
     __device__ static __forceinline__ float to_float(__nv_bfloat16 v) { return __bfloat162float(v); }
 };
 
+// Programmatic dependent launch: a kernel launched with the stream-serialization attribute may start
+// while its predecessor in the stream drains; it must not touch global memory the predecessor may
+// write before pdl_wait() returns (the predecessor has then completed and flushed).  Both are
+// no-ops for a plain launch.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // silu(g) = g / (1 + exp(-g)); expf keeps full fp32 accuracy.
 __device__ __forceinline__ float silu_f(float g) { return g / (1.0f + expf(-g)); }
 
