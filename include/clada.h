@@ -193,6 +193,30 @@ int clada_sparse_ffn_decode(const clada_layer *layer, const void *x, int32_t B,
                             uint8_t *mask_out, int32_t *idx_out, int32_t *count_out,
                             void *ws, size_t ws_bytes, int32_t *status, void *stream);
 
+/* clada_sparse_ffn_decode for callers that cannot allocate device memory (the
+ * paper has no counterpart; this is a deployment variant of the call above).
+ * Think of a plug-in that runs inside another engine's execution step, where
+ * the host engine owns and budgets all device memory and allocation calls are
+ * forbidden there, or of a server whose memory plan is frozen after start-up.
+ * Same arguments and results as clada_sparse_ffn_decode, minus the workspace:
+ * the kernel's scratch is a fixed array inside the library (about 5 MiB, held
+ * by every GPU that loads the library until the process exits).  The call
+ * itself allocates nothing.
+ *  - Limits: d_model <= 8192 and a device with at most 160 SMs; beyond that the
+ *    call returns CLADA_ERR_UNSUPPORTED (clada_last_cuda_error() says why)
+ *    and enqueues nothing.
+ *  - The first call on a device looks up the array's device address; make that
+ *    first call outside any stream capture.
+ *  - All calls share the one array and it keeps the previous call's contents;
+ *    each call clears the control words it needs at zero, in stream order.
+ *    Two calls whose kernels overlap on the GPU (different streams) race on
+ *    the array: serialise them, or use the workspace variant. */
+int clada_sparse_ffn_decode_static(const clada_layer *layer, const void *x, int32_t B,
+                                   const float *scores /*[B,d_ff]*/, const float *tau_final,
+                                   int64_t tau_stride, void *y, int32_t y_dtype,
+                                   uint8_t *mask_out, int32_t *idx_out, int32_t *count_out,
+                                   int32_t *status, void *stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -23,6 +23,7 @@ _INT_RETURNING = [
     "clada_workspace_init", "clada_down_norms", "clada_prefix_scores", "clada_refine_scores",
     "clada_select", "clada_prefix_select", "clada_tau_from_sparsity", "clada_cogload",
     "clada_adjust_threshold", "clada_cogload_adjust", "clada_sparse_ffn_decode",
+    "clada_sparse_ffn_decode_static",
 ]
 
 
@@ -67,6 +68,7 @@ def load() -> ctypes.CDLL:
     L.clada_adjust_threshold.argtypes = [vp, vp, vp, f32, f32, vp, vp, i32, i32, vp, vp]
     L.clada_cogload_adjust.argtypes = [vp, i32, i32, i64, i64, vp, vp, vp, vp, f32, f32, i32, vp, vp, vp, vp, vp]
     L.clada_sparse_ffn_decode.argtypes = [lp, vp, i32, vp, vp, i64, vp, i32, vp, vp, vp, vp, sz, vp, vp]
+    L.clada_sparse_ffn_decode_static.argtypes = [lp, vp, i32, vp, vp, i64, vp, i32, vp, vp, vp, vp, vp]
     for name in _INT_RETURNING:
         getattr(L, name).restype = ctypes.c_int
     _lib = L
@@ -280,3 +282,21 @@ def clada_sparse_ffn_decode(layer: Layer, x, scores, tau_final, tau_stride, y, w
                                           _ptr(ws, torch.uint8, "ws"), ws.numel(),
                                           _ptr(status, torch.int32, "status"), _stream(stream)),
            "clada_sparse_ffn_decode")
+
+
+def clada_sparse_ffn_decode_static(layer: Layer, x, scores, tau_final, tau_stride, y, mask_out=None, idx_out=None,
+                                   count_out=None, status=None, stream=None) -> None:
+    """clada_sparse_ffn_decode without a workspace argument: the scratch is a fixed array inside the
+    library, for callers that are not allowed to allocate device memory.  Calls share that array, so
+    do not let two of them overlap on the GPU."""
+    B = x.shape[0]
+    if not tau_final.is_cuda or tau_final.dtype != torch.float32:
+        raise CladaError("tau_final must be a CUDA float32 tensor")
+    _check(load().clada_sparse_ffn_decode_static(layer.ref, _ptr(x, layer.dtype, "x"), B,
+                                                 _ptr(scores, torch.float32, "scores"), tau_final.data_ptr(),
+                                                 int(tau_stride), _ptr(y, name="y"), _dtype_code(y.dtype),
+                                                 _ptr(mask_out, torch.uint8, "mask_out"),
+                                                 _ptr(idx_out, torch.int32, "idx_out"),
+                                                 _ptr(count_out, torch.int32, "count_out"),
+                                                 _ptr(status, torch.int32, "status"), _stream(stream)),
+           "clada_sparse_ffn_decode_static")

@@ -524,11 +524,10 @@ static int launch_ffn(const FfnParams &p, cudaStream_t st) {
 
 using namespace clada;
 
-extern "C" int clada_sparse_ffn_decode(const clada_layer *layer, const void *x, int32_t B,
-                                       const float *scores, const float *tau_final, int64_t tau_stride,
-                                       void *y, int32_t y_dtype, uint8_t *mask_out, int32_t *idx_out,
-                                       int32_t *count_out, void *ws, size_t ws_bytes, int32_t *status,
-                                       void *stream) {
+static int decode_with_workspace(const clada_layer *layer, const void *x, int32_t B, const float *scores,
+                                 const float *tau_final, int64_t tau_stride, void *y, int32_t y_dtype,
+                                 uint8_t *mask_out, int32_t *idx_out, int32_t *count_out, void *ws,
+                                 size_t ws_bytes, int32_t *status, void *stream) {
     int rc = validate_layer(layer, false);
     if (rc != CLADA_OK) return rc;
     if (!x || !scores || !tau_final || !y) return CLADA_ERR_NULL;
@@ -567,4 +566,69 @@ extern "C" int clada_sparse_ffn_decode(const clada_layer *layer, const void *x, 
         if (rc != CLADA_OK) return rc;
     }
     return CLADA_OK;
+}
+
+extern "C" int clada_sparse_ffn_decode(const clada_layer *layer, const void *x, int32_t B,
+                                       const float *scores, const float *tau_final, int64_t tau_stride,
+                                       void *y, int32_t y_dtype, uint8_t *mask_out, int32_t *idx_out,
+                                       int32_t *count_out, void *ws, size_t ws_bytes, int32_t *status,
+                                       void *stream) {
+    return decode_with_workspace(layer, x, B, scores, tau_final, tau_stride, y, y_dtype, mask_out, idx_out,
+                                 count_out, ws, ws_bytes, status, stream);
+}
+
+// ---- the entry point that allocates nothing ---------------------------------------------------
+//
+// Some callers may not allocate device memory at all: a plug-in that runs inside another engine's
+// execution step, where the host engine owns and budgets every byte and forbids allocation calls in
+// the step; a serving process that froze its memory plan at start-up; code on a latency-critical path
+// where cudaMalloc would synchronise the whole device.  For them the decode kernel's scratch (its
+// control words and the per-CTA partial outputs) lives in the fixed array below instead of a
+// caller-provided workspace.  Every GPU that loads the library holds these kStaticScratchBytes until
+// the process exits.
+constexpr int kStaticMaxSms = 160;
+constexpr int kStaticMaxDModel = 8192;
+constexpr size_t kStaticScratchBytes = kWsCtrlBytes + (size_t)kStaticMaxSms * kStaticMaxDModel * sizeof(float);
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+// The array's name is only a host-side handle; kernels need its device address, which the runtime
+// gives per device.  Looked up once per device, with that device current, and cached.
+static int static_scratch_address(void **out) {
+    constexpr int kMaxDev = 64;
+    static void *cache[kMaxDev] = {};
+    int dev = 0;
+    CLADA_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDev) return CLADA_ERR_UNSUPPORTED;
+    if (!cache[dev]) {
+        void *ptr = nullptr;
+        CLADA_CUDA_TRY(cudaGetSymbolAddress(&ptr, g_static_scratch));
+        cache[dev] = ptr;
+    }
+    *out = cache[dev];
+    return CLADA_OK;
+}
+
+extern "C" int clada_sparse_ffn_decode_static(const clada_layer *layer, const void *x, int32_t B,
+                                              const float *scores, const float *tau_final,
+                                              int64_t tau_stride, void *y, int32_t y_dtype,
+                                              uint8_t *mask_out, int32_t *idx_out, int32_t *count_out,
+                                              int32_t *status, void *stream) {
+    if (!layer) return CLADA_ERR_NULL;
+    DeviceInfo di;
+    int rc = device_info(&di);
+    if (rc != CLADA_OK) return rc;
+    if (layer->d_model > kStaticMaxDModel || di.num_sms > kStaticMaxSms) {
+        set_last_cuda_error(cudaErrorInvalidValue,
+                            "clada_sparse_ffn_decode_static: d_model > 8192 or more than 160 SMs exceeds the "
+                            "built-in scratch; use clada_sparse_ffn_decode with a workspace");
+        return CLADA_ERR_UNSUPPORTED;
+    }
+    void *scratch = nullptr;
+    rc = static_scratch_address(&scratch);
+    if (rc != CLADA_OK) return rc;
+    // The array keeps whatever the last call left.  The control words must start at zero (they are
+    // zero after a clean call, not after one that timed out), so clear them in stream order.
+    CLADA_CUDA_TRY(cudaMemsetAsync(scratch, 0, kWsCtrlBytes, static_cast<cudaStream_t>(stream)));
+    return decode_with_workspace(layer, x, B, scores, tau_final, tau_stride, y, y_dtype, mask_out, idx_out,
+                                 count_out, scratch, kStaticScratchBytes, status, stream);
 }
