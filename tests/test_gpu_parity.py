@@ -393,7 +393,7 @@ def test_host_side_errors(clada):
     scores = torch.ones(1, 50, device="cuda")
     tau = torch.ones(1, device="cuda")
     y = torch.empty(1, 64, device="cuda")
-    small_ws = torch.empty(512, dtype=torch.uint8, device="cuda")
+    small_ws = torch.empty(256, dtype=torch.uint8, device="cuda")
     with pytest.raises(clada.CladaError, match="workspace"):
         clada.clada_sparse_ffn_decode(layer, x, scores, tau, 1, y, small_ws)
     with pytest.raises(clada.CladaError):
