@@ -474,17 +474,21 @@ sparse_ffn_kernel(const FfnParams p, const int n_stages) {
         }
         // All slices of y must have been cleared before anyone adds: the barrier every CTA arrived at
         // right after its prologue; by now it has normally long been complete.
-        if (!timed_out) {
+        // One thread looks (an acquire load per thread would queue 75 000 of them on one L2 word);
+        // the named barrier hands the answer to the other consumers.
+        if (tid == 0 && !*reinterpret_cast<volatile int *>(&s_abort)) {
             unsigned spins = 0, seen;
             for (;;) {
                 asm volatile("ld.acquire.gpu.u32 %0, [%1];" : "=r"(seen) : "l"(&p.ctrl->arrive) : "memory");
                 if (seen >= (unsigned)n_ctas) break;
                 if (++spins > kBarrierSpinLimit) {
-                    timed_out = true;
+                    *reinterpret_cast<volatile int *>(&s_abort) = 1;
                     break;
                 }
             }
         }
+        asm volatile("bar.sync 1, %0;" ::"n"(kConsumers) : "memory");
+        if (*reinterpret_cast<volatile int *>(&s_abort)) timed_out = true;
         if (!timed_out) {
 #pragma unroll
             for (int i = 0; i < NV; ++i) {
