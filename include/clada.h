@@ -185,9 +185,7 @@ int clada_cogload_adjust(const void *logits, int32_t logits_dtype, int32_t B, in
  *   x        [B, d_model] in the layer's dtype
  *   y        out [B, d_model], y_dtype fp32 or bf16
  *   mask_out / idx_out / count_out: optional (NULL), as in clada_select
- * Accumulation is fp32; the per-SM partial outputs are combined with atomic
- * adds whose order is not fixed, so y may differ in its last bits from run to
- * run (masks, index lists and counts never do).  d_ff <= 69632.
+ * Accumulation is fp32 in a fixed order: results are bit-identical run to run.
  * The workspace must have been initialised with clada_workspace_init. */
 int clada_sparse_ffn_decode(const clada_layer *layer, const void *x, int32_t B,
                             const float *scores /*[B,d_ff]*/, const float *tau_final,

@@ -15,8 +15,6 @@
 //             CTA sums a slice of columns over all partials in CTA order (deterministic) and writes y.
 #include <math.h>
 
-#include <algorithm>
-
 #include "common.cuh"
 
 namespace clada {
@@ -31,13 +29,45 @@ struct FfnParams {
     uint8_t *mask_out;    // [d_ff] or null
     int32_t *idx_out;     // [d_ff] or null
     int32_t *count_out;   // one int or null
-    float *yacc;          // [d_model] fp32 accumulation target: y itself (fp32 output) or scratch
+    float *partials;      // [gridDim.x, d_model]
     WsCtrl *ctrl;
     int32_t *status;
     int d_model, d_ff;
 };
 
 constexpr unsigned kBarrierSpinLimit = 1u << 22;  // polls of an L2 word: gives up after ~1 s at most
+
+// Bounded grid-wide barrier on two self-resetting counters in the workspace control block.
+// Returns false if the wait expired.
+__device__ bool grid_barrier(WsCtrl *ctrl, unsigned n_ctas) {
+    __shared__ int s_ok;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        __threadfence();
+        atomicAdd(&ctrl->arrive, 1u);
+        unsigned spins = 0, seen;
+        int ok = 1;
+        for (;;) {
+            asm volatile("ld.acquire.gpu.u32 %0, [%1];" : "=r"(seen) : "l"(&ctrl->arrive) : "memory");
+            if (seen >= n_ctas) break;
+            if (++spins > kBarrierSpinLimit) {
+                ok = 0;
+                break;
+            }
+        }
+        s_ok = ok;
+        if (ok) {
+            const unsigned left = atomicAdd(&ctrl->depart, 1u);
+            if (left == n_ctas - 1) {  // last one out: everyone has seen arrive == n_ctas
+                ctrl->arrive = 0;
+                ctrl->depart = 0;
+                __threadfence();
+            }
+        }
+    }
+    __syncthreads();
+    return s_ok != 0;
+}
 
 // ---- mbarrier / bulk-copy primitives (bounded waits) -------------------------------------------
 
@@ -104,9 +134,6 @@ __device__ __forceinline__ float4 ld_keep4(const float4 *p, uint64_t policy) {
                  : "l"(p), "l"(policy));
     return v;
 }
-__device__ __forceinline__ void red_add_v4(float *dst, float a, float b, float c, float d) {
-    asm volatile("red.global.add.v4.f32 [%0], {%1,%2,%3,%4};" ::"l"(dst), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
-}
 __device__ __forceinline__ uint4 lds128(uint32_t addr) {
     uint4 v;
     asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
@@ -139,9 +166,6 @@ constexpr int kFfnWarps = kFfnThreads / kWarp;
 constexpr int kMaxStages = 16;
 constexpr int G = 4;                          // neurons per CTA-wide reduction
 constexpr int kMaxBatches = 4;                // prologue batches: d_ff <= 4 * 32 * kFfnThreads
-constexpr int kMaxPool = 2048;                // neurons handed out dynamically, at most
-constexpr int kPoolChunk = 2;                 // ... this many per grab
-constexpr int kGroupRing = 32;                // group descriptors in flight (> stages)
 
 template <typename T, int NV>
 __global__ void __launch_bounds__(kFfnThreads, 1)
@@ -161,13 +185,9 @@ sparse_ffn_kernel(const FfnParams p, const int n_stages) {
     const uint32_t ring = smem_u32(smem_raw);
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem_raw + (size_t)n_stages * stage_bytes);
     const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + kMaxStages);
-    int *s_list = reinterpret_cast<int *>(bars + 2 * kMaxStages);  // this CTA's static share
-    int *s_pool = s_list + (F / n_ctas + 2);                        // the shared pool (same in every CTA)
+    int *s_list = reinterpret_cast<int *>(bars + 2 * kMaxStages);
     __shared__ int s_wtot[kFfnWarps];
     __shared__ __align__(16) float s_dot[2][2 * G][kConsWarps];
-    __shared__ int s_gend[kGroupRing];  // group descriptors, producer -> consumers
-    __shared__ int s_ngroups;
-    __shared__ int s_abort;
 
     pdl_launch_dependents();  // the next kernel in the stream may be scheduled as SMs free up
     if (tid == kConsumers) {  // the producer warp sets the ring up while the others start loading
@@ -250,16 +270,9 @@ sparse_ffn_kernel(const FfnParams p, const int n_stages) {
         first_rank[bt] = n_act + wbase + incl - cnt;
         n_act += btot;
     }
-    // The kept list splits into a static part [0, n_stat), shared out equally and contiguously, and a
-    // pool [n_stat, n_act) at its end that CTAs drain two neurons at a time through an atomic counter:
-    // SMs that the memory system serves faster take more of it, so all finish together.
-    const int n_pool = min(n_act / 8, kMaxPool);
-    const int n_stat = n_act - n_pool;
-    const int r0 = (int)(((int64_t)n_stat * cta) / n_ctas);
-    const int r1 = (int)(((int64_t)n_stat * (cta + 1)) / n_ctas);
-    const int o0 = (int)(((int64_t)n_act * cta) / n_ctas);  // slice of idx_out this CTA writes
-    const int o1 = (int)(((int64_t)n_act * (cta + 1)) / n_ctas);
-    const int m0 = (int)(((int64_t)F * cta) / n_ctas);      // slice of mask_out this CTA writes
+    const int r0 = (int)(((int64_t)n_act * cta) / n_ctas);
+    const int r1 = (int)(((int64_t)n_act * (cta + 1)) / n_ctas);
+    const int m0 = (int)(((int64_t)F * cta) / n_ctas);  // slice of the mask this CTA writes
     const int m1 = (int)(((int64_t)F * (cta + 1)) / n_ctas);
 #pragma unroll
     for (int bt = 0; bt < kMaxBatches; ++bt) {
@@ -267,17 +280,15 @@ sparse_ffn_kernel(const FfnParams p, const int n_stages) {
         if (bt >= n_batches || q >= chunks) continue;
         const int j0 = q * kWarp;
         int rank = first_rank[bt];
-        const int rend = rank + __popc(bal[bt]);
-        const bool mine = rank < r1 && rend > r0, pool = rend > n_stat;
-        const bool out = p.idx_out && rank < o1 && rend > o0;
-        if (mine || pool || out) {
+        if (rank < r1 && rank + __popc(bal[bt]) > r0) {  // chunk holds part of this CTA's share
             unsigned b = bal[bt];
             while (b) {
                 const int u = __ffs(b) - 1;
                 b &= b - 1;
-                if (rank >= r0 && rank < r1) s_list[rank - r0] = j0 + u;
-                if (rank >= n_stat) s_pool[rank - n_stat] = j0 + u;
-                if (out && rank >= o0 && rank < o1) p.idx_out[rank] = j0 + u;
+                if (rank >= r0 && rank < r1) {
+                    s_list[rank - r0] = j0 + u;
+                    if (p.idx_out) p.idx_out[rank] = j0 + u;
+                }
                 ++rank;
             }
         }
@@ -290,21 +301,7 @@ sparse_ffn_kernel(const FfnParams p, const int n_stages) {
     }
     if (p.count_out && cta == 0 && tid == 0) *p.count_out = n_act;
     const int my_n = r1 - r0;
-    // y is accumulated with atomic adds, so it must be zero before any CTA adds: every CTA clears a
-    // slice now and arrives at the grid barrier; nobody waits for it until its own stream is done.
-    {
-        const int z0 = (int)(((int64_t)d * cta) / n_ctas), z1 = (int)(((int64_t)d * (cta + 1)) / n_ctas);
-        for (int i = z0 + tid; i < z1; i += kFfnThreads) p.yacc[i] = 0.f;
-    }
-    if (tid == 0) {
-        s_ngroups = 0;
-        s_abort = 0;
-    }
-    __syncthreads();  // s_list, s_pool, the mbarriers and the zeroed slice are done
-    if (tid == 0) {
-        __threadfence();
-        atomicAdd(&p.ctrl->arrive, 1u);
-    }
+    __syncthreads();  // s_list and the mbarriers are ready
 
     bool timed_out = false;
 
@@ -315,48 +312,23 @@ sparse_ffn_kernel(const FfnParams p, const int n_stages) {
             const char *Wu = static_cast<const char *>(p.w_up);
             const char *Wd = static_cast<const char *>(p.w_down_t);
             const uint64_t stream_policy = policy_evict_first();
-            int seq = 0;     // neurons issued so far by this CTA; neuron i uses stage i % n_stages
-            int ngroups = 0;
-            auto issue = [&](int j) -> bool {
-                const int s = seq % n_stages, use = seq / n_stages;
-                if (!mbar_wait(empty0 + 8 * s, (use & 1) ^ 1)) return false;  // fresh barrier: parity 1 passes
-                const size_t off = (size_t)j * row_bytes;
+            int issued = 0;
+            for (int i = 0; i < my_n; ++i) {
+                const int s = i % n_stages, use = i / n_stages;
+                if (!mbar_wait(empty0 + 8 * s, (use & 1) ^ 1)) {  // a fresh barrier passes parity 1 at once
+                    timed_out = true;
+                    break;
+                }
+                const size_t off = (size_t)s_list[i] * row_bytes;
                 const uint32_t dst = ring + (uint32_t)s * stage_bytes, bar = full0 + 8 * s;
                 mbar_expect_tx(bar, stage_bytes);
                 bulk_load_row_hint(dst, Wg + off, row_bytes, bar, stream_policy);
                 bulk_load_row_hint(dst + row_bytes, Wu + off, row_bytes, bar, stream_policy);
                 bulk_load_row_hint(dst + 2 * row_bytes, Wd + off, row_bytes, bar, stream_policy);
-                ++seq;
-                return true;
-            };
-            auto publish = [&](int end_seq) {  // group descriptor: the consumers' next group ends here
-                s_gend[ngroups % kGroupRing] = end_seq;
-                __threadfence_block();
-                ++ngroups;
-                *reinterpret_cast<volatile int *>(&s_ngroups) = ngroups;
-            };
-            // static share, G neurons per group
-            for (int i0 = 0; i0 < my_n && !timed_out; i0 += G) {
-                const int cnt = min(G, my_n - i0);
-                for (int g = 0; g < cnt && !timed_out; ++g) timed_out = !issue(s_list[i0 + g]);
-                if (!timed_out) publish(seq);
+                issued = i + 1;
             }
-            // pool, kPoolChunk neurons per grab, the next grab requested one chunk ahead
-            if (n_pool > 0 && !timed_out) {
-                unsigned c_next = atomicAdd(&p.ctrl->next, 1u);
-                for (;;) {
-                    const int r = (int)c_next * kPoolChunk;
-                    if (r >= n_pool) break;
-                    c_next = atomicAdd(&p.ctrl->next, 1u);
-                    const int cnt = min(kPoolChunk, n_pool - r);
-                    for (int g = 0; g < cnt && !timed_out; ++g) timed_out = !issue(s_pool[r + g]);
-                    if (timed_out) break;
-                    publish(seq);
-                }
-            }
-            publish(-1);  // no more groups
             // Never leave with copies in flight: the last use of every stage must have landed.
-            for (int i = max(0, seq - n_stages); i < seq; ++i)
+            for (int i = max(0, issued - n_stages); i < issued; ++i)
                 if (!mbar_wait(full0 + 8 * (i % n_stages), (i / n_stages) & 1)) timed_out = true;
         }
     } else {
@@ -367,51 +339,28 @@ sparse_ffn_kernel(const FfnParams p, const int n_stages) {
 #pragma unroll
             for (int e = 0; e < P; ++e) acc[i][e] = make_float2(0.f, 0.f);
         const bool b16 = lane & 16, b8 = lane & 8, b4 = lane & 4;
-        int buf = 0, seq0 = 0;
-        for (int k = 0;; ++k, buf ^= 1) {
-            // The producer's descriptor for group k.  A thread whose wait expires raises s_abort and
-            // keeps walking to the named barrier below, after which all consumers leave together:
-            // nobody is ever left alone at a barrier.
-            int gend = -1;
-            if (!timed_out) {
-                unsigned spins = 0;
-                while (*reinterpret_cast<volatile int *>(&s_ngroups) <= k) {
-                    if (++spins > kMbarSpinLimit) {
-                        timed_out = true;
-                        break;
-                    }
-                }
-            }
-            if (!timed_out) {
-                __threadfence_block();
-                gend = *reinterpret_cast<volatile int *>(&s_gend[k % kGroupRing]);
-            } else {
-                *reinterpret_cast<volatile int *>(&s_abort) = 1;
-            }
-            const int cnt = gend < 0 ? 0 : gend - seq0;  // 1..G neurons in this group; 0 at the end marker
+        int buf = 0;
+        for (int g0 = 0; g0 < my_n; g0 += G, buf ^= 1) {
             float pd[2 * G];
             uint32_t st_addr[G];
 #pragma unroll
             for (int g = 0; g < G; ++g) {
-                const int i = seq0 + g;
+                const int i = g0 + g;
                 float2 sg = make_float2(0.f, 0.f), su = make_float2(0.f, 0.f);
                 st_addr[g] = ring + (uint32_t)(i % n_stages) * stage_bytes;
-                if (g < cnt) {
-                    if (!timed_out && !mbar_wait(full0 + 8 * (i % n_stages), (i / n_stages) & 1)) {
-                        timed_out = true;
-                        *reinterpret_cast<volatile int *>(&s_abort) = 1;
-                    }
+                if (i < my_n) {
+                    if (!timed_out && !mbar_wait(full0 + 8 * (i % n_stages), (i / n_stages) & 1)) timed_out = true;
 #pragma unroll
-                    for (int kk = 0; kk < NV; ++kk) {
-                        if (!vok[kk]) continue;
-                        const uint32_t a = st_addr[g] + (uint32_t)(tid + kk * kConsumers) * 16u;
+                    for (int k = 0; k < NV; ++k) {
+                        if (!vok[k]) continue;
+                        const uint32_t a = st_addr[g] + (uint32_t)(tid + k * kConsumers) * 16u;
                         float2 fg[P], fu[P];
                         Pairs<T>::unpack(lds128(a), fg);
                         Pairs<T>::unpack(lds128(a + row_bytes), fu);
 #pragma unroll
                         for (int e = 0; e < P; ++e) {
-                            sg = __ffma2_rn(fg[e], xr[kk][e], sg);
-                            su = __ffma2_rn(fu[e], xr[kk][e], su);
+                            sg = __ffma2_rn(fg[e], xr[k][e], sg);
+                            su = __ffma2_rn(fu[e], xr[k][e], su);
                         }
                     }
                 }
@@ -419,7 +368,7 @@ sparse_ffn_kernel(const FfnParams p, const int n_stages) {
                 pd[2 * g + 1] = su.x + su.y;
             }
             // Warp sums of the 8 values by a halving butterfly (9 shuffles): after it every lane of
-            // quad q holds the warp total of value q.
+            // quad q holds the warp total of value q.  Fixed order, so results repeat bit for bit.
             float b[4], c[2], v8;
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
@@ -437,7 +386,6 @@ sparse_ffn_kernel(const FfnParams p, const int n_stages) {
             // lane 4q holds value index: bit4 -> +4, bit3 -> +2, bit2 -> +1
             if ((lane & 3) == 0) s_dot[buf][(b16 ? 4 : 0) + (b8 ? 2 : 0) + (b4 ? 1 : 0)][warp] = v8;
             asm volatile("bar.sync 1, %0;" ::"n"(kConsumers) : "memory");
-            if (*reinterpret_cast<volatile int *>(&s_abort) || gend < 0) break;  // same for all consumers
             // Cross-warp sums: lane l adds 4 consecutive warps of value l/4 (16 warps = 4 lanes per
             // value), the quad finishes by butterfly; then gate lanes form h = silu(gate) * up.
             float tot;
@@ -452,15 +400,15 @@ sparse_ffn_kernel(const FfnParams p, const int n_stages) {
 #pragma unroll
             for (int g = 0; g < G; ++g) {
                 const float h = __shfl_sync(0xffffffffu, hval, 8 * g);
-                if (g >= cnt) continue;
+                if (g0 + g >= my_n) continue;
                 const float2 h2 = make_float2(h, h);
 #pragma unroll
-                for (int kk = 0; kk < NV; ++kk) {
-                    if (!vok[kk]) continue;
+                for (int k = 0; k < NV; ++k) {
+                    if (!vok[k]) continue;
                     float2 fd[P];
-                    Pairs<T>::unpack(lds128(st_addr[g] + 2 * row_bytes + (uint32_t)(tid + kk * kConsumers) * 16u), fd);
+                    Pairs<T>::unpack(lds128(st_addr[g] + 2 * row_bytes + (uint32_t)(tid + k * kConsumers) * 16u), fd);
 #pragma unroll
-                    for (int e = 0; e < P; ++e) acc[kk][e] = __ffma2_rn(h2, fd[e], acc[kk][e]);
+                    for (int e = 0; e < P; ++e) acc[k][e] = __ffma2_rn(h2, fd[e], acc[k][e]);
                 }
             }
             // hand the stages back to the producer
@@ -468,58 +416,57 @@ sparse_ffn_kernel(const FfnParams p, const int n_stages) {
             if (lane == 0) {
 #pragma unroll
                 for (int g = 0; g < G; ++g)
-                    if (g < cnt) mbar_arrive(empty0 + 8 * ((seq0 + g) % n_stages));
-            }
-            seq0 = gend;
-        }
-        // All slices of y must have been cleared before anyone adds: the barrier every CTA arrived at
-        // right after its prologue; by now it has normally long been complete.
-        // One thread looks (an acquire load per thread would queue 75 000 of them on one L2 word);
-        // the named barrier hands the answer to the other consumers.
-        if (tid == 0 && !*reinterpret_cast<volatile int *>(&s_abort)) {
-            unsigned spins = 0, seen;
-            for (;;) {
-                asm volatile("ld.acquire.gpu.u32 %0, [%1];" : "=r"(seen) : "l"(&p.ctrl->arrive) : "memory");
-                if (seen >= (unsigned)n_ctas) break;
-                if (++spins > kBarrierSpinLimit) {
-                    *reinterpret_cast<volatile int *>(&s_abort) = 1;
-                    break;
-                }
+                    if (g0 + g < my_n) mbar_arrive(empty0 + 8 * ((g0 + g) % n_stages));
             }
         }
-        asm volatile("bar.sync 1, %0;" ::"n"(kConsumers) : "memory");
-        if (*reinterpret_cast<volatile int *>(&s_abort)) timed_out = true;
-        if (!timed_out) {
+        // partial y of this CTA
+        float *mine = p.partials + (size_t)cta * d;
 #pragma unroll
-            for (int i = 0; i < NV; ++i) {
-                if (!vok[i]) continue;
-                float *dst = p.yacc + (size_t)(tid + i * kConsumers) * E;
+        for (int i = 0; i < NV; ++i) {
+            if (!vok[i]) continue;
+            float4 *dst = reinterpret_cast<float4 *>(mine + (size_t)(tid + i * kConsumers) * E);
 #pragma unroll
-                for (int e = 0; e < P; e += 2)
-                    red_add_v4(dst + 2 * e, acc[i][e].x, acc[i][e].y, acc[i][e + 1].x, acc[i][e + 1].y);
-            }
+            for (int e = 0; e < P; e += 2)
+                dst[e / 2] = make_float4(acc[i][e].x, acc[i][e].y, acc[i][e + 1].x, acc[i][e + 1].y);
         }
     }
     if (timed_out && p.status) atomicOr(p.status, CLADA_STATUS_TIMEOUT);
 
-    // ---- epilogue: the last CTA to finish converts (bf16 output) and re-arms the control words ---
-    __shared__ int s_last;
-    __syncthreads();
-    if (tid == 0) {
-        __threadfence();
-        s_last = atomicAdd(&p.ctrl->depart, 1u) == (unsigned)n_ctas - 1u;
+    // ---- epilogue: grid barrier, deterministic column reduction ---------------------------------
+    if (!grid_barrier(p.ctrl, (unsigned)n_ctas)) {
+        if (tid == 0 && p.status) atomicOr(p.status, CLADA_STATUS_TIMEOUT);
+        return;
     }
-    __syncthreads();
-    if (!s_last) return;
-    __threadfence();
-    if (p.y_dtype == CLADA_BF16) {
-        __nv_bfloat16 *yb = static_cast<__nv_bfloat16 *>(p.y);
-        for (int i = tid; i < d; i += kFfnThreads) yb[i] = __float2bfloat16_rn(__ldcg(p.yacc + i));
-    }
-    if (tid == 0) {
-        p.ctrl->arrive = 0;
-        p.ctrl->next = 0;
-        p.ctrl->depart = 0;
+    // columns in groups of 4 (float4); a warp sums one group: lane l adds partial rows l, l+32, ...
+    // in order (five loads in flight at a time), then the 32 lane sums combine by butterfly.
+    const int ngroups = d / 4;
+    for (int q = cta + warp * n_ctas; q < ngroups; q += n_ctas * kFfnWarps) {
+        float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int rb = 0; rb < n_ctas; rb += 5 * kWarp) {
+            float4 v[5];
+#pragma unroll
+            for (int u = 0; u < 5; ++u) {
+                const int r = rb + u * kWarp + lane;
+                v[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (r < n_ctas) v[u] = __ldcg(reinterpret_cast<const float4 *>(p.partials + (size_t)r * d) + q);
+            }
+#pragma unroll
+            for (int u = 0; u < 5; ++u) {
+                s.x += v[u].x; s.y += v[u].y; s.z += v[u].z; s.w += v[u].w;
+            }
+        }
+        s.x = warp_sum(s.x); s.y = warp_sum(s.y); s.z = warp_sum(s.z); s.w = warp_sum(s.w);
+        if (lane == 0) {
+            if (p.y_dtype == CLADA_F32) {
+                reinterpret_cast<float4 *>(p.y)[q] = s;
+            } else {
+                __nv_bfloat162 lo = __floats2bfloat162_rn(s.x, s.y), hi = __floats2bfloat162_rn(s.z, s.w);
+                uint2 o;
+                o.x = *reinterpret_cast<uint32_t *>(&lo);
+                o.y = *reinterpret_cast<uint32_t *>(&hi);
+                reinterpret_cast<uint2 *>(p.y)[q] = o;
+            }
+        }
     }
 }
 
@@ -534,8 +481,7 @@ static int launch_variant(const FfnParams &p, cudaStream_t st) {
     if (rc != CLADA_OK) return rc;
     auto kern = sparse_ffn_kernel<T, NV>;
     const size_t stage_bytes = 3 * (size_t)(p.d_model / E) * 16;
-    const size_t tail = 2 * kMaxStages * sizeof(uint64_t) +
-                        ((size_t)(p.d_ff / di.num_sms + 2) + (size_t)std::min(p.d_ff / 8, kMaxPool)) * sizeof(int);
+    const size_t tail = 2 * kMaxStages * sizeof(uint64_t) + (size_t)(p.d_ff / di.num_sms + 2) * sizeof(int);
     const size_t budget = (size_t)di.max_smem_optin - 2048;  // leave room for the static arrays
     if (budget < tail + G * stage_bytes) return CLADA_ERR_UNSUPPORTED;  // a group needs G stages at once
     int n_stages = (int)((budget - tail) / stage_bytes);
@@ -592,7 +538,7 @@ static int decode_with_workspace(const clada_layer *layer, const void *x, int32_
     DeviceInfo di;
     rc = device_info(&di);
     if (rc != CLADA_OK) return rc;
-    const size_t need = kWsCtrlBytes + (size_t)layer->d_model * sizeof(float);
+    const size_t need = kWsCtrlBytes + (size_t)di.num_sms * layer->d_model * sizeof(float);
     if (ws_bytes < need) return CLADA_ERR_WORKSPACE;
 
     const size_t esz = elem_size(layer->dtype);
@@ -611,8 +557,7 @@ static int decode_with_workspace(const clada_layer *layer, const void *x, int32_
         p.mask_out = mask_out ? mask_out + (size_t)b * layer->d_ff : nullptr;
         p.idx_out = idx_out ? idx_out + (size_t)b * layer->d_ff : nullptr;
         p.count_out = count_out ? count_out + b : nullptr;
-        p.yacc = y_dtype == CLADA_F32 ? static_cast<float *>(p.y)
-                                      : reinterpret_cast<float *>(static_cast<char *>(ws) + kWsCtrlBytes);
+        p.partials = reinterpret_cast<float *>(static_cast<char *>(ws) + kWsCtrlBytes);
         p.ctrl = static_cast<WsCtrl *>(ws);
         p.status = status;
         p.d_model = layer->d_model;

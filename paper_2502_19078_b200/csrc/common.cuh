@@ -39,9 +39,8 @@ int device_info(DeviceInfo *out);
 // [256, ...)          per-call scratch
 constexpr size_t kWsCtrlBytes = 256;
 struct WsCtrl {
-    unsigned int arrive;  // CTAs that have cleared their slice of y (early grid barrier)
-    unsigned int depart;  // CTAs that have finished; the last one resets all three
-    unsigned int next;    // next chunk of the dynamically shared pool
+    unsigned int arrive;  // grid barrier: CTAs that reached it
+    unsigned int depart;  // CTAs that left it; the last one resets both
 };
 
 // ---- device helpers -----------------------------------------------------------------------

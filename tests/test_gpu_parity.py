@@ -376,13 +376,13 @@ def test_sparse_ffn_degenerate_thresholds_and_determinism(clada, oracle):
     y_or, _, n_or = oracle.sparse_ffn(wl.to_numpy_bits(x[0]), W_in, V_in, W_out, scores[0].astype(np.float64),
                                       float(tau1))
     assert int(count[0]) == n_or == 1 and rel_inf(y[0].cpu().numpy(), y_or) <= FFN_TOL_F32
-    # run to run only the order of the fp32 atomic adds into y may differ
+    # bit-identical run to run
     tau = _dev(np.array([1.0], np.float32))
     y2 = torch.empty_like(y)
     clada.clada_sparse_ffn_decode(layer, x.cuda(), _dev(scores), tau, 1, y, ws)
     clada.clada_sparse_ffn_decode(layer, x.cuda(), _dev(scores), tau, 1, y2, ws)
     torch.cuda.synchronize()
-    assert rel_inf(y2[0].cpu().numpy(), y[0].cpu().numpy().astype(np.float64)) <= 2e-6
+    assert torch.equal(y, y2)
 
 
 def test_host_side_errors(clada):
@@ -393,7 +393,7 @@ def test_host_side_errors(clada):
     scores = torch.ones(1, 50, device="cuda")
     tau = torch.ones(1, device="cuda")
     y = torch.empty(1, 64, device="cuda")
-    small_ws = torch.empty(256, dtype=torch.uint8, device="cuda")
+    small_ws = torch.empty(512, dtype=torch.uint8, device="cuda")
     with pytest.raises(clada.CladaError, match="workspace"):
         clada.clada_sparse_ffn_decode(layer, x, scores, tau, 1, y, small_ws)
     with pytest.raises(clada.CladaError):
