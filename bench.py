@@ -249,8 +249,15 @@ def run_ours(args):
         clocks = sampler.stop() if rank == 0 else None
 
         # the FFN kernel alone, same launches, for the roofline
+        ffn_run = job.ffn_only_loop
         job.ffn_only_loop()
-        ffn_ms = _timed(job.ffn_only_loop, 3, lambda: None) / (3 * job.N)
+        if args.graph:
+            ffn_graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(ffn_graph, stream=stream):
+                job.ffn_only_loop()
+            ffn_run = ffn_graph.replay
+        ffn_run()
+        ffn_ms = _timed(ffn_run, 5, lambda: None) / (5 * job.N)
         kept = job.kept_per_token()
         kept_base = w.d_ff - w.k_cut(w.sparsities[0])
 

@@ -181,11 +181,12 @@ sparse_ffn_kernel(const FfnParams p, const int n_stages) {
     const uint32_t stage_bytes = 3u * row_bytes;
     const int chunks = (F + kWarp - 1) / kWarp;
 
-    // dynamic shared memory: ring | full[kMaxStages] | empty[kMaxStages] | kept list
+    // dynamic shared memory: ring | full[kMaxStages] | empty[kMaxStages] | keep-bits | kept list
     const uint32_t ring = smem_u32(smem_raw);
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem_raw + (size_t)n_stages * stage_bytes);
     const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + kMaxStages);
-    int *s_list = reinterpret_cast<int *>(bars + 2 * kMaxStages);
+    unsigned *s_bal = reinterpret_cast<unsigned *>(bars + 2 * kMaxStages);  // keep-bits word per chunk
+    int *s_list = reinterpret_cast<int *>(s_bal + chunks);
     __shared__ int s_wtot[kFfnWarps];
     __shared__ __align__(16) float s_dot[2][2 * G][kConsWarps];
 
@@ -214,20 +215,19 @@ sparse_ffn_kernel(const FfnParams p, const int n_stages) {
     }
 
     // ---- prologue: threshold test, ranks, this CTA's share of the kept list ---------------------
-    // A batch is one 32-neuron chunk per thread (all its loads independent); F <= 32 * kFfnThreads
-    // needs a single batch.  Each batch: keep-bits word per thread, block-wide exclusive scan.
+    // A batch is one 32-neuron chunk per thread (eight independent 16-byte loads); F <= 32 * kFfnThreads
+    // needs a single batch.  Which chunk a thread LOADS is rotated by the CTA index, so that the 148
+    // CTAs do not all ask L2 for the same line at the same moment; the keep-bits words go through
+    // shared memory and are ranked in natural order by a block-wide scan.
     const bool vec_ok = (reinterpret_cast<uintptr_t>(p.scores) & 15u) == 0;
-    unsigned bal[kMaxBatches];
-    int first_rank[kMaxBatches];  // rank of this thread's chunk's first kept neuron
-    int n_act = 0;
     const int n_batches = (chunks + kFfnThreads - 1) / kFfnThreads;
+    {
+        int slot = tid + (cta * 37) % kFfnThreads;
+        if (slot >= kFfnThreads) slot -= kFfnThreads;
 #pragma unroll
-    for (int bt = 0; bt < kMaxBatches; ++bt) {
-        bal[bt] = 0u;
-        first_rank[bt] = 0;
-        if (bt >= n_batches) continue;  // uniform
-        const int q = bt * kFfnThreads + tid;  // this thread's chunk
-        if (q < chunks) {
+        for (int bt = 0; bt < kMaxBatches; ++bt) {
+            const int q = bt * kFfnThreads + slot;
+            if (bt >= n_batches || q >= chunks) continue;
             const int j0 = q * kWarp;
             unsigned w = 0;
             if (vec_ok && j0 + kWarp <= F) {
@@ -248,8 +248,20 @@ sparse_ffn_kernel(const FfnParams p, const int n_stages) {
 #pragma unroll
                 for (int u = 0; u < kWarp; ++u) w |= (v[u] >= tau ? 1u : 0u) << u;
             }
-            bal[bt] = w;
+            s_bal[q] = w;
         }
+    }
+    __syncthreads();
+    unsigned bal[kMaxBatches];
+    int first_rank[kMaxBatches];  // rank of this thread's chunk's first kept neuron
+    int n_act = 0;
+#pragma unroll
+    for (int bt = 0; bt < kMaxBatches; ++bt) {
+        bal[bt] = 0u;
+        first_rank[bt] = 0;
+        if (bt >= n_batches) continue;  // uniform
+        const int q = bt * kFfnThreads + tid;  // this thread's chunk
+        if (q < chunks) bal[bt] = s_bal[q];
         const int cnt = __popc(bal[bt]);
         int incl = cnt;
 #pragma unroll
@@ -274,29 +286,29 @@ sparse_ffn_kernel(const FfnParams p, const int n_stages) {
     const int r1 = (int)(((int64_t)n_act * (cta + 1)) / n_ctas);
     const int m0 = (int)(((int64_t)F * cta) / n_ctas);  // slice of the mask this CTA writes
     const int m1 = (int)(((int64_t)F * (cta + 1)) / n_ctas);
+    // Only two or three chunks hold this CTA's share: the warp that owns such a chunk writes it out
+    // with one lane per neuron.
 #pragma unroll
     for (int bt = 0; bt < kMaxBatches; ++bt) {
+        if (bt >= n_batches) continue;  // uniform
         const int q = bt * kFfnThreads + tid;
-        if (bt >= n_batches || q >= chunks) continue;
-        const int j0 = q * kWarp;
-        int rank = first_rank[bt];
-        if (rank < r1 && rank + __popc(bal[bt]) > r0) {  // chunk holds part of this CTA's share
-            unsigned b = bal[bt];
-            while (b) {
-                const int u = __ffs(b) - 1;
-                b &= b - 1;
-                if (rank >= r0 && rank < r1) {
-                    s_list[rank - r0] = j0 + u;
-                    if (p.idx_out) p.idx_out[rank] = j0 + u;
-                }
-                ++rank;
+        const int fr = first_rank[bt];
+        const bool in_share = q < chunks && fr < r1 && fr + __popc(bal[bt]) > r0;
+        const bool in_mask = p.mask_out && q < chunks && q * kWarp < m1 && q * kWarp + kWarp > m0;
+        unsigned todo = __ballot_sync(0xffffffffu, in_share || in_mask);
+        while (todo) {
+            const int t = __ffs(todo) - 1;
+            todo &= todo - 1;
+            const unsigned wb = __shfl_sync(0xffffffffu, bal[bt], t);
+            const int wfr = __shfl_sync(0xffffffffu, fr, t);
+            const int j = (bt * kFfnThreads + (warp * kWarp + t)) * kWarp + lane;
+            const bool keep = (wb >> lane) & 1u;
+            const int rank = wfr + __popc(wb & ((1u << lane) - 1u));
+            if (keep && rank >= r0 && rank < r1) {
+                s_list[rank - r0] = j;
+                if (p.idx_out) p.idx_out[rank] = j;
             }
-        }
-        if (p.mask_out && j0 < m1 && j0 + kWarp > m0) {
-            for (int u = 0; u < kWarp; ++u) {
-                const int j = j0 + u;
-                if (j >= m0 && j < m1) p.mask_out[j] = (bal[bt] >> u) & 1u;
-            }
+            if (p.mask_out && j >= m0 && j < m1) p.mask_out[j] = keep ? 1 : 0;
         }
     }
     if (p.count_out && cta == 0 && tid == 0) *p.count_out = n_act;
@@ -481,7 +493,8 @@ static int launch_variant(const FfnParams &p, cudaStream_t st) {
     if (rc != CLADA_OK) return rc;
     auto kern = sparse_ffn_kernel<T, NV>;
     const size_t stage_bytes = 3 * (size_t)(p.d_model / E) * 16;
-    const size_t tail = 2 * kMaxStages * sizeof(uint64_t) + (size_t)(p.d_ff / di.num_sms + 2) * sizeof(int);
+    const size_t tail = 2 * kMaxStages * sizeof(uint64_t) + (size_t)((p.d_ff + 31) / 32) * sizeof(unsigned) +
+                        (size_t)(p.d_ff / di.num_sms + 2) * sizeof(int);
     const size_t budget = (size_t)di.max_smem_optin - 2048;  // leave room for the static arrays
     if (budget < tail + G * stage_bytes) return CLADA_ERR_UNSUPPORTED;  // a group needs G stages at once
     int n_stages = (int)((budget - tail) / stage_bytes);
