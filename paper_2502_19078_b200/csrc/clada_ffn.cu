@@ -188,6 +188,7 @@ sparse_ffn_kernel(const FfnParams p, const int n_stages) {
     unsigned *s_bal = reinterpret_cast<unsigned *>(bars + 2 * kMaxStages);  // keep-bits word per chunk
     int *s_list = reinterpret_cast<int *>(s_bal + chunks);
     __shared__ int s_wtot[kFfnWarps];
+    __shared__ float s_tau;
     __shared__ __align__(16) float s_dot[2][2 * G][kConsWarps];
 
     pdl_launch_dependents();  // the next kernel in the stream may be scheduled as SMs free up
@@ -201,7 +202,7 @@ sparse_ffn_kernel(const FfnParams p, const int n_stages) {
     pdl_wait();  // everything below may read what the previous kernel wrote
 
     const uint64_t keep_policy = policy_evict_last();
-    const float tau = ld_keep(p.tau, keep_policy);
+    if (tid == 0) s_tau = ld_keep(p.tau, keep_policy);  // one request per CTA, not one per warp
     // x of this thread's columns (consumers), requested before the scan so the latencies overlap
     float2 xr[NV][P];
     bool vok[NV];
@@ -224,16 +225,36 @@ sparse_ffn_kernel(const FfnParams p, const int n_stages) {
     {
         int slot = tid + (cta * 37) % kFfnThreads;
         if (slot >= kFfnThreads) slot -= kFfnThreads;
+        float tau = 0.f;
 #pragma unroll
         for (int bt = 0; bt < kMaxBatches; ++bt) {
+            if (bt >= n_batches) continue;  // uniform
             const int q = bt * kFfnThreads + slot;
-            if (bt >= n_batches || q >= chunks) continue;
+            const bool has = q < chunks;
             const int j0 = q * kWarp;
-            unsigned w = 0;
-            if (vec_ok && j0 + kWarp <= F) {
-                float4 v[8];
+            float4 v[8];
+            if (has) {
+                if (vec_ok && j0 + kWarp <= F) {
 #pragma unroll
-                for (int u = 0; u < 8; ++u) v[u] = ld_keep4(reinterpret_cast<const float4 *>(p.scores + j0) + u, keep_policy);
+                    for (int u = 0; u < 8; ++u)
+                        v[u] = ld_keep4(reinterpret_cast<const float4 *>(p.scores + j0) + u, keep_policy);
+                } else {
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) {
+                        const int j = j0 + 4 * u;
+                        v[u].x = (j < F) ? ld_keep(p.scores + j, keep_policy) : -INFINITY;
+                        v[u].y = (j + 1 < F) ? ld_keep(p.scores + j + 1, keep_policy) : -INFINITY;
+                        v[u].z = (j + 2 < F) ? ld_keep(p.scores + j + 2, keep_policy) : -INFINITY;
+                        v[u].w = (j + 3 < F) ? ld_keep(p.scores + j + 3, keep_policy) : -INFINITY;
+                    }
+                }
+            }
+            if (bt == 0) {  // the threshold arrives while the score loads are in flight
+                __syncthreads();
+                tau = s_tau;
+            }
+            if (has) {
+                unsigned w = 0;
 #pragma unroll
                 for (int u = 0; u < 8; ++u) {
                     w |= (v[u].x >= tau ? 1u : 0u) << (4 * u);
@@ -241,14 +262,8 @@ sparse_ffn_kernel(const FfnParams p, const int n_stages) {
                     w |= (v[u].z >= tau ? 1u : 0u) << (4 * u + 2);
                     w |= (v[u].w >= tau ? 1u : 0u) << (4 * u + 3);
                 }
-            } else {
-                float v[kWarp];
-#pragma unroll
-                for (int u = 0; u < kWarp; ++u) v[u] = (j0 + u < F) ? ld_keep(p.scores + j0 + u, keep_policy) : -INFINITY;
-#pragma unroll
-                for (int u = 0; u < kWarp; ++u) w |= (v[u] >= tau ? 1u : 0u) << u;
+                s_bal[q] = w;
             }
-            s_bal[q] = w;
         }
     }
     __syncthreads();
