@@ -7,7 +7,11 @@
 //   surprisal = m + logZ - l[token],   entropy = logZ - W / Z.
 #include <math.h>
 
+#include <cooperative_groups.h>
+
 #include "common.cuh"
+
+namespace cg = cooperative_groups;
 
 namespace clada {
 
@@ -62,9 +66,12 @@ __device__ __forceinline__ float load_logit(const T *row, int64_t i) {
     return Elem<T>::to_float(row[i]);
 }
 
-constexpr int kCogThreads = 1024;
+constexpr int kCogThreads = 512;
+constexpr int kCogMaxCluster = 8;
 
-// tau_base == nullptr: cognitive load only.
+// Grid (cluster size, B): the CTAs of a cluster split one vocabulary row into equal slices, leave their
+// slice statistics in shared memory, and rank 0 reads them over distributed shared memory, merges them
+// in rank order and writes the row's outputs.  tau_base == nullptr: cognitive load only.
 template <typename T>
 __global__ void __launch_bounds__(kCogThreads)
 cogload_kernel(const T *__restrict__ logits, int64_t V, int64_t row_stride,
@@ -74,7 +81,9 @@ cogload_kernel(const T *__restrict__ logits, int64_t V, int64_t row_stride,
                const float *__restrict__ gamma, float tau_s, float tau_H, int L,
                float *__restrict__ tau_final) {
     constexpr int E = Elem<T>::kPerVec;
-    const int b = blockIdx.x;
+    cg::cluster_group cluster = cg::this_cluster();
+    const int n_slices = (int)cluster.num_blocks(), slice = (int)cluster.block_rank();
+    const int b = blockIdx.y;
     const T *row = logits + (size_t)b * row_stride;
     const int tid = threadIdx.x;
     pdl_launch_dependents();
@@ -83,41 +92,43 @@ cogload_kernel(const T *__restrict__ logits, int64_t V, int64_t row_stride,
     SoftStat st = stat_empty();
     bool bad = false;
 
-    // Scalar head up to the first 16-byte boundary, vector body, scalar tail.
+    // The row as scalar head (up to the first 16-byte boundary), 16-byte vectors, scalar tail; the
+    // vectors are dealt to the slices in contiguous runs, head and tail go to slice 0.
     const uintptr_t addr = reinterpret_cast<uintptr_t>(row);
     int64_t head = ((16 - (addr & 15)) & 15) / sizeof(T);
     if (head > V) head = V;
     const int64_t nvec = (V - head) / E;
     const int64_t tail0 = head + nvec * E;
-    if (tid < head) {
+    if (slice == 0 && tid < head) {
         float l[1] = {load_logit(row, tid)};
         stat_add(st, l, bad);
     }
     const uint4 *vrow = reinterpret_cast<const uint4 *>(row + head);
-    int64_t v = tid;
-    // four vectors in flight per thread
-    for (; v + 3 * (int64_t)kCogThreads < nvec; v += 4 * (int64_t)kCogThreads) {
-        uint4 q[4];
+    const int64_t v0 = nvec * slice / n_slices, v1 = nvec * (slice + 1) / n_slices;
+    // eight vectors in flight per thread
+    for (int64_t v = v0 + tid; v < v1; v += 8 * (int64_t)kCogThreads) {
+        uint4 q[8];
 #pragma unroll
-        for (int u = 0; u < 4; ++u) q[u] = ldg_stream(vrow + v + u * (int64_t)kCogThreads);
+        for (int u = 0; u < 8; ++u) {
+            const int64_t vi = v + u * (int64_t)kCogThreads;
+            q[u] = make_uint4(0, 0, 0, 0);
+            if (vi < v1) q[u] = ldg_stream(vrow + vi);
+        }
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            float l[E];
-            Elem<T>::unpack(q[u], l);
-            stat_add(st, l, bad);
+        for (int u = 0; u < 8; ++u) {
+            if (v + u * (int64_t)kCogThreads < v1) {
+                float l[E];
+                Elem<T>::unpack(q[u], l);
+                stat_add(st, l, bad);
+            }
         }
     }
-    for (; v < nvec; v += kCogThreads) {
-        float l[E];
-        Elem<T>::unpack(ldg_stream(vrow + v), l);
-        stat_add(st, l, bad);
-    }
-    if (tail0 + tid < V) {
+    if (slice == 0 && tail0 + tid < V) {
         float l[1] = {load_logit(row, tail0 + tid)};
         stat_add(st, l, bad);
     }
 
-    // warp, then CTA merge in a fixed order
+    // warp, CTA, then cluster merge, each in a fixed order
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
         SoftStat other;
@@ -127,6 +138,7 @@ cogload_kernel(const T *__restrict__ logits, int64_t V, int64_t row_stride,
         st = ((tid & o) == 0) ? stat_merge(st, other) : stat_merge(other, st);
     }
     __shared__ SoftStat s_stat[kCogThreads / kWarp];
+    __shared__ SoftStat s_slice;  // this CTA's slice, read by rank 0
     __shared__ int s_bad;
     __shared__ float s_out[2];
     if (tid == 0) s_bad = 0;
@@ -137,37 +149,51 @@ cogload_kernel(const T *__restrict__ logits, int64_t V, int64_t row_stride,
     if (tid == 0) {
         SoftStat tot = s_stat[0];
         for (int w = 1; w < kCogThreads / kWarp; ++w) tot = stat_merge(tot, s_stat[w]);
-        int flags = 0;
-        float s, h;
-        if (s_bad || !(tot.z > 0.f)) {  // a +inf / NaN logit, or no finite logit at all
-            flags |= CLADA_STATUS_NONFINITE_LOGIT;
-            s = h = NAN;
-        } else {
-            const float logz = logf(tot.z);
-            h = logz - tot.w / tot.z;
-            const int32_t tok = token_id[b];
-            if (tok < 0 || tok >= V) {
-                flags |= CLADA_STATUS_BAD_TOKEN;
-                s = NAN;
+        if (s_bad) tot.z = NAN;  // carries the non-finite flag to rank 0
+        s_slice = tot;
+    }
+    cluster.sync();
+    if (slice == 0) {
+        if (tid == 0) {
+            SoftStat tot = s_slice;
+            for (int r = 1; r < n_slices; ++r) {
+                const SoftStat *remote = cluster.map_shared_rank(&s_slice, r);
+                tot = stat_merge(tot, *remote);
+            }
+            int flags = 0;
+            float s, h;
+            if (!(tot.z > 0.f)) {  // a +inf / NaN logit (z is NaN), or no finite logit at all
+                flags |= CLADA_STATUS_NONFINITE_LOGIT;
+                s = h = NAN;
             } else {
-                s = (tot.m + logz) - load_logit(row, tok);
+                const float logz = logf(tot.z);
+                h = logz - tot.w / tot.z;
+                const int32_t tok = token_id[b];
+                if (tok < 0 || tok >= V) {
+                    flags |= CLADA_STATUS_BAD_TOKEN;
+                    s = NAN;
+                } else {
+                    s = (tot.m + logz) - load_logit(row, tok);
+                }
+            }
+            surprisal[b] = s;
+            entropy[b] = h;
+            s_out[0] = s;
+            s_out[1] = h;
+            if (flags && status) atomicOr(status, flags);
+        }
+        if (tau_base != nullptr) {
+            __syncthreads();
+            const float s = s_out[0], h = s_out[1];
+            for (int l = tid; l < L; l += kCogThreads) {
+                float mult = 1.0f;
+                if (s > tau_s) mult = __fadd_rn(mult, lambda[l]);
+                if (h > tau_H) mult = __fadd_rn(mult, gamma[l]);
+                tau_final[(size_t)b * L + l] = __fmul_rn(tau_base[(size_t)b * L + l], mult);
             }
         }
-        surprisal[b] = s;
-        entropy[b] = h;
-        s_out[0] = s;
-        s_out[1] = h;
-        if (flags && status) atomicOr(status, flags);
     }
-    if (tau_base == nullptr) return;
-    __syncthreads();
-    const float s = s_out[0], h = s_out[1];
-    for (int l = tid; l < L; l += kCogThreads) {
-        float mult = 1.0f;
-        if (s > tau_s) mult = __fadd_rn(mult, lambda[l]);
-        if (h > tau_H) mult = __fadd_rn(mult, gamma[l]);
-        tau_final[(size_t)b * L + l] = __fmul_rn(tau_base[(size_t)b * L + l], mult);
-    }
+    cluster.sync();  // no CTA leaves while rank 0 may still read its shared memory
 }
 
 __global__ void adjust_threshold_kernel(const float *__restrict__ tau_base,
@@ -195,14 +221,22 @@ static int launch_cogload(const void *logits, int32_t dtype, int32_t B, int64_t 
     if (B <= 0 || V <= 0 || row_stride < V) return CLADA_ERR_SHAPE;
     if (reinterpret_cast<uintptr_t>(logits) % elem_size(dtype)) return CLADA_ERR_ALIGN;
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(B);
+    // one CTA per 4096 logits of a row, at most a portable cluster of 8
+    int n_slices = 1;
+    while (n_slices < kCogMaxCluster && (int64_t)n_slices * 4096 < V) n_slices *= 2;
+    if (B > 65535) return CLADA_ERR_UNSUPPORTED;
+    cfg.gridDim = dim3(n_slices, B);
     cfg.blockDim = dim3(kCogThreads);
     cfg.stream = static_cast<cudaStream_t>(stream);
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
+    attr[1].id = cudaLaunchAttributeClusterDimension;
+    attr[1].val.clusterDim.x = n_slices;
+    attr[1].val.clusterDim.y = 1;
+    attr[1].val.clusterDim.z = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = 2;
     if (dtype == CLADA_F32)
         CLADA_CUDA_TRY(cudaLaunchKernelEx(&cfg, cogload_kernel<float>, static_cast<const float *>(logits), V,
                                           row_stride, token_id, surprisal, entropy, status, tau_base, lambda, gamma,

@@ -157,31 +157,49 @@ __global__ void guard_candidates_kernel(const float *__restrict__ scores, int B,
     if (near) cand[atomicAdd(n_cand, 1)] = make_int2(b, j);
 }
 
-constexpr int kRefThreads = 256;
+constexpr int kRefThreads = 1024;
 
-// One CTA per candidate (grid-stride).  Warps take tokens round-robin; lanes split d_model.
+// One CTA per candidate (grid-stride).  The candidate's gate and up rows sit in shared memory; each of
+// the 32 warps takes every 32nd token of the prompt, lanes split d_model by 16-byte vectors, products
+// and sums in fp64.  Warp and CTA sums are taken in a fixed order.
 template <typename T>
 __global__ void __launch_bounds__(kRefThreads)
 guard_refine_kernel(const T *__restrict__ X, const T *__restrict__ Wg, const T *__restrict__ Wu,
                     const T *__restrict__ Wd_t, int d_model, int d_ff, const SeqTable tab,
                     const int *__restrict__ n_cand, const int2 *__restrict__ cand,
                     float *__restrict__ scores) {
-    __shared__ double s_zz[kRefThreads / kWarp];
-    __shared__ double s_nn[kRefThreads / kWarp];
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    constexpr int E = Elem<T>::kPerVec;
     constexpr int kWarps = kRefThreads / kWarp;
+    extern __shared__ uint4 s_rows[];  // gate row | up row
+    __shared__ double s_zz[kWarps];
+    __shared__ double s_nn[kWarps];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int vpr = d_model / E;
     const int total = *n_cand;
     for (int c = blockIdx.x; c < total; c += gridDim.x) {
         const int b = cand[c].x, j = cand[c].y;
-        const T *wg = Wg + (size_t)j * d_model, *wu = Wu + (size_t)j * d_model, *wd = Wd_t + (size_t)j * d_model;
+        const uint4 *wg = reinterpret_cast<const uint4 *>(Wg + (size_t)j * d_model);
+        const uint4 *wu = reinterpret_cast<const uint4 *>(Wu + (size_t)j * d_model);
+        const uint4 *wd = reinterpret_cast<const uint4 *>(Wd_t + (size_t)j * d_model);
+        for (int v = threadIdx.x; v < vpr; v += kRefThreads) {
+            s_rows[v] = wg[v];
+            s_rows[vpr + v] = wu[v];
+        }
+        __syncthreads();
         double zz = 0.0;
         for (long long t = tab.off[b] + warp; t < tab.off[b + 1]; t += kWarps) {
-            const T *x = X + (size_t)t * d_model;
+            const uint4 *x = reinterpret_cast<const uint4 *>(X + (size_t)t * d_model);
             double g = 0.0, u = 0.0;
-            for (int k = lane; k < d_model; k += kWarp) {
-                const double xv = (double)Elem<T>::to_float(x[k]);
-                g = fma((double)Elem<T>::to_float(wg[k]), xv, g);
-                u = fma((double)Elem<T>::to_float(wu[k]), xv, u);
+            for (int v = lane; v < vpr; v += kWarp) {
+                float fx[E], fg[E], fu[E];
+                Elem<T>::unpack(x[v], fx);
+                Elem<T>::unpack(s_rows[v], fg);
+                Elem<T>::unpack(s_rows[vpr + v], fu);
+#pragma unroll
+                for (int e = 0; e < E; ++e) {
+                    g = fma((double)fg[e], (double)fx[e], g);
+                    u = fma((double)fu[e], (double)fx[e], u);
+                }
             }
             g = warp_sum(g);
             u = warp_sum(u);
@@ -189,9 +207,11 @@ guard_refine_kernel(const T *__restrict__ X, const T *__restrict__ Wg, const T *
             zz += z * z;
         }
         double nn = 0.0;
-        for (int k = threadIdx.x; k < d_model; k += kRefThreads) {
-            const double w = (double)Elem<T>::to_float(wd[k]);
-            nn = fma(w, w, nn);
+        for (int v = threadIdx.x; v < vpr; v += kRefThreads) {
+            float fd[E];
+            Elem<T>::unpack(wd[v], fd);
+#pragma unroll
+            for (int e = 0; e < E; ++e) nn = fma((double)fd[e], (double)fd[e], nn);
         }
         nn = warp_sum(nn);
         if (lane == 0) {
@@ -306,14 +326,15 @@ int clada_refine_scores(const clada_layer *layer, const void *X, const int64_t *
     DeviceInfo di;
     rc = device_info(&di);
     if (rc != CLADA_OK) return rc;
-    const int grid = di.num_sms * 4;
+    const int grid = di.num_sms;
+    const size_t rows_smem = 2 * (size_t)layer->d_model * elem_size(layer->dtype);
     if (layer->dtype == CLADA_F32)
-        guard_refine_kernel<float><<<grid, kRefThreads, 0, st>>>(
+        guard_refine_kernel<float><<<grid, kRefThreads, rows_smem, st>>>(
             static_cast<const float *>(X), static_cast<const float *>(layer->w_gate),
             static_cast<const float *>(layer->w_up), static_cast<const float *>(layer->w_down_t),
             layer->d_model, layer->d_ff, tab, n_cand, cand, scores);
     else
-        guard_refine_kernel<__nv_bfloat16><<<grid, kRefThreads, 0, st>>>(
+        guard_refine_kernel<__nv_bfloat16><<<grid, kRefThreads, rows_smem, st>>>(
             static_cast<const __nv_bfloat16 *>(X), static_cast<const __nv_bfloat16 *>(layer->w_gate),
             static_cast<const __nv_bfloat16 *>(layer->w_up), static_cast<const __nv_bfloat16 *>(layer->w_down_t),
             layer->d_model, layer->d_ff, tab, n_cand, cand, scores);
