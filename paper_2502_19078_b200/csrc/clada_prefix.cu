@@ -9,30 +9,11 @@
 #include <math.h>
 
 #include "common.cuh"
+#include "prefix_common.cuh"
 
 namespace clada {
 
-constexpr int kMaxSeqs = 128;
-struct SeqTable {
-    int B;
-    long long off[kMaxSeqs + 1];
-};
-
 constexpr int BM = 64, BN = 64, BK = 32, kPfThreads = 256;
-
-__host__ __device__ inline int tiles_of(long long rows) { return (int)((rows + BM - 1) / BM); }
-
-// Which prompt and which token range a global token-tile index falls in.
-__device__ inline void locate_tile(const SeqTable &tab, int mtile, int &b, long long &t0, long long &t1) {
-    int first = 0;
-    for (b = 0; b < tab.B - 1; ++b) {
-        const int n = tiles_of(tab.off[b + 1] - tab.off[b]);
-        if (mtile < first + n) break;
-        first += n;
-    }
-    t0 = tab.off[b] + (long long)(mtile - first) * BM;
-    t1 = min(t0 + BM, tab.off[b + 1]);
-}
 
 template <typename T>
 __global__ void __launch_bounds__(kPfThreads)
@@ -49,7 +30,7 @@ prefix_partials_kernel(const T *__restrict__ X, const T *__restrict__ Wg, const 
     const int n0 = blockIdx.x * BN;
     int b;
     long long t0, t1;
-    locate_tile(tab, blockIdx.y, b, t0, t1);
+    locate_tile(tab, blockIdx.y, BM, b, t0, t1);
 
     float ag[4][4], au[4][4];
 #pragma unroll
@@ -119,14 +100,14 @@ prefix_partials_kernel(const T *__restrict__ X, const T *__restrict__ Wg, const 
     }
 }
 
-__global__ void prefix_finalize_kernel(const float *__restrict__ partials, const SeqTable tab, int d_ff,
+__global__ void prefix_finalize_kernel(const float *__restrict__ partials, const SeqTable tab, int tile, int d_ff,
                                        const float *__restrict__ w_down_norm, float *__restrict__ scores) {
     const int j = blockIdx.x * blockDim.x + threadIdx.x;
     const int b = blockIdx.y;
     if (j >= d_ff) return;
     int first = 0;
-    for (int q = 0; q < b; ++q) first += tiles_of(tab.off[q + 1] - tab.off[q]);
-    const int n = tiles_of(tab.off[b + 1] - tab.off[b]);
+    for (int q = 0; q < b; ++q) first += tiles_of(tab.off[q + 1] - tab.off[q], tile);
+    const int n = tiles_of(tab.off[b + 1] - tab.off[b], tile);
     float s = 0.f;
     for (int t = 0; t < n; ++t) s += partials[(size_t)(first + t) * d_ff + j];
     scores[(size_t)b * d_ff + j] = __fmul_rn(sqrtf(s), w_down_norm[j]);
@@ -242,7 +223,7 @@ static int build_table(const int64_t *seq_offsets, int32_t B, SeqTable *tab, int
     for (int b = 0; b <= B; ++b) {
         tab->off[b] = seq_offsets[b];
         if (seq_offsets[b] < 0 || (b > 0 && seq_offsets[b] < seq_offsets[b - 1])) return CLADA_ERR_SHAPE;
-        if (b > 0) tiles += tiles_of(seq_offsets[b] - seq_offsets[b - 1]);
+        if (b > 0) tiles += tiles_of(seq_offsets[b] - seq_offsets[b - 1], BM);
     }
     if (tiles > 65535) return CLADA_ERR_UNSUPPORTED;
     *n_mtiles = (int)tiles;
@@ -263,8 +244,13 @@ static int run_scores(const clada_layer *L, const void *X, const SeqTable &tab, 
             L->d_model, L->d_ff, tab, partials);
         CLADA_CUDA_TRY(cudaGetLastError());
     }
-    dim3 fgrid((L->d_ff + 255) / 256, tab.B);
-    prefix_finalize_kernel<<<fgrid, 256, 0, st>>>(partials, tab, L->d_ff, L->w_down_norm, scores);
+    return launch_prefix_finalize(partials, tab, BM, L->d_ff, L->w_down_norm, scores, st);
+}
+
+int launch_prefix_finalize(const float *partials, const SeqTable &tab, int tile, int d_ff,
+                           const float *w_down_norm, float *scores, cudaStream_t st) {
+    dim3 fgrid((d_ff + 255) / 256, tab.B);
+    prefix_finalize_kernel<<<fgrid, 256, 0, st>>>(partials, tab, tile, d_ff, w_down_norm, scores);
     CLADA_CUDA_TRY(cudaGetLastError());
     return CLADA_OK;
 }
@@ -290,8 +276,11 @@ int clada_prefix_scores(const clada_layer *layer, const void *X, const int64_t *
     if (ws_bytes < kWsCtrlBytes + partials_bytes(n_mtiles, layer->d_ff)) return CLADA_ERR_WORKSPACE;
     float *partials = reinterpret_cast<float *>(static_cast<char *>(ws) + kWsCtrlBytes);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    return layer->dtype == CLADA_F32 ? run_scores<float>(layer, X, tab, n_mtiles, scores, partials, st)
-                                     : run_scores<__nv_bfloat16>(layer, X, tab, n_mtiles, scores, partials, st);
+    if (layer->dtype == CLADA_F32) return run_scores<float>(layer, X, tab, n_mtiles, scores, partials, st);
+    // bf16: tensor cores (128-token tiles: never more partial rows than the 64-token tiling above)
+    rc = run_prefix_partials_tc(layer, X, tab, seq_offsets[B], partials, status, st);
+    if (rc != CLADA_OK) return rc;
+    return launch_prefix_finalize(partials, tab, kTcTokenTile, layer->d_ff, layer->w_down_norm, scores, st);
 }
 
 int clada_refine_scores(const clada_layer *layer, const void *X, const int64_t *seq_offsets, int32_t B,

@@ -1,0 +1,41 @@
+// Shared by the two prefill-statistics paths (CUDA-core and tensor-core): the prompt table passed by
+// value to kernels, token-tile bookkeeping, and the finalize step.
+#pragma once
+
+#include "common.cuh"
+
+namespace clada {
+
+constexpr int kMaxSeqs = 128;
+struct SeqTable {
+    int B;
+    long long off[kMaxSeqs + 1];
+};
+
+// Token tiles of `tile` rows never straddle prompts: prompt b owns tiles_of(T_b, tile) of them.
+__host__ __device__ inline int tiles_of(long long rows, int tile) { return (int)((rows + tile - 1) / tile); }
+
+#ifdef __CUDACC__
+// Which prompt and which token range a global token-tile index falls in.
+__device__ inline void locate_tile(const SeqTable &tab, int ttile, int tile, int &b, long long &t0, long long &t1) {
+    int first = 0;
+    for (b = 0; b < tab.B - 1; ++b) {
+        const int n = tiles_of(tab.off[b + 1] - tab.off[b], tile);
+        if (ttile < first + n) break;
+        first += n;
+    }
+    t0 = tab.off[b] + (long long)(ttile - first) * tile;
+    t1 = min(t0 + tile, tab.off[b + 1]);
+}
+#endif
+
+// scores[b,j] = sqrt(sum over prompt b's tiles of partials[tile,j]) * w_down_norm[j], tiles in order.
+int launch_prefix_finalize(const float *partials, const SeqTable &tab, int tile, int d_ff,
+                           const float *w_down_norm, float *scores, cudaStream_t st);
+
+// Tensor-core partial sums (bf16 layers, 128-token tiles).  partials: [sum_b tiles_of(T_b, 128), d_ff].
+int run_prefix_partials_tc(const clada_layer *layer, const void *X, const SeqTable &tab, long long T_total,
+                           float *partials, int32_t *status, cudaStream_t st);
+constexpr int kTcTokenTile = 128;
+
+}  // namespace clada
