@@ -258,6 +258,10 @@ def run_ours(args):
             ffn_run = ffn_graph.replay
         ffn_run()
         ffn_ms = _timed(ffn_run, 5, lambda: None) / (5 * job.N)
+        # the prefix statistics alone (tensor-core contraction), for its own roofline line
+        pf = lambda: clada.clada_prefix_scores(job.layers[0], job.X, job.off, job.scores, job.ws, job.status)
+        pf()
+        prefix_ms = _timed(pf, 10, lambda: None) / 10
         kept = job.kept_per_token()
         kept_base = w.d_ff - w.k_cut(w.sparsities[0])
 
@@ -286,6 +290,13 @@ def run_ours(args):
     e2e_value = tokens / (e2e_ms * 1e-3)
 
     peak, peak_kind = _peaks()
+    prefix_flop = 4.0 * job.T * w.d_model * w.d_ff
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            bf16_peak = float(json.load(f)["bf16_tflops"])
+        bf16_kind = "measured (burst)"
+    except Exception:
+        bf16_peak, bf16_kind = 1590.0, "fallback"
     eb = w.elem_bytes
     # algorithmic bytes of one FFN launch: three rows per kept neuron + scores + x in + y out
     ffn_bytes = kept_base * 3 * w.d_model * eb + w.d_ff * 4 + w.d_model * eb + w.d_model * 4
@@ -308,6 +319,10 @@ def run_ours(args):
                      "unit": "GB/s", "frac": achieved / peak, "peak_kind": peak_kind, "traffic": None,
                      "bytes_per_launch": ffn_bytes, "us_per_launch": ffn_ms * 1e3,
                      "kept_neurons": kept_base},
+        "prefix_roofline": {"bound": "tensor", "kernel": "prefix_tc_kernel (+finalize)", "ms": prefix_ms,
+                            "achieved": prefix_flop / (prefix_ms * 1e-3) / 1e12, "peak": bf16_peak, "unit": "TFLOP/s",
+                            "frac": prefix_flop / (prefix_ms * 1e-3) / 1e12 / bf16_peak, "peak_kind": bf16_kind,
+                            "flop": prefix_flop},
         "clocks": clocks, "device_status_word": status,
     }
     if rank == 0:
