@@ -26,6 +26,7 @@ import torch
 ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
+from paper_2502_19078_b200 import sharding  # noqa: E402
 from paper_2502_19078_b200 import workloads as wl  # noqa: E402
 
 WORKLOAD = "c2_llama2_7b_layer"
@@ -281,13 +282,10 @@ def run_ours(args):
         e2e_ms = _timed(e2e_step, args.steps, barrier)
         status = int(job.status.item())
 
-    t = torch.tensor([ms, e2e_ms], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms, e2e_ms = float(t[0]), float(t[1])
-    tokens = job.tokens_per_step() * args.steps * world
-    value = tokens / (ms * 1e-3)
-    e2e_value = tokens / (e2e_ms * 1e-3)
+    # every rank ran its own sequence; the job's rate is all ranks' tokens over the slowest rank's time
+    tokens_rank = job.tokens_per_step() * args.steps
+    value, ms = sharding.whole_job_rate(tokens_rank, ms, dev)
+    e2e_value, e2e_ms = sharding.whole_job_rate(tokens_rank, e2e_ms, dev)
 
     peak, peak_kind = _peaks()
     prefix_flop = 4.0 * job.T * w.d_model * w.d_ff
