@@ -87,14 +87,14 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(ok)
-        : "r"(bar), "r"(parity)
+        : "r"(bar), "r"(parity), "r"(1000u)  // suspend for at most ~1 us per try
         : "memory");
     return ok != 0;
 }
-constexpr unsigned kMbarSpinLimit = 1u << 22;  // each failed try_wait already sleeps in hardware
+constexpr unsigned kMbarSpinLimit = 1u << 20;  // tries of at most ~1 us each: about a second
 // Waits for the phase with the given parity; gives up (returns false) after kMbarSpinLimit tries.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
     for (unsigned i = 0; i < kMbarSpinLimit; ++i)
