@@ -16,6 +16,7 @@
 #include <math.h>
 
 #include "common.cuh"
+#include "ffn_common.cuh"
 
 namespace clada {
 
@@ -35,135 +36,6 @@ struct FfnParams {
     int d_model, d_ff;
 };
 
-constexpr unsigned kBarrierSpinLimit = 1u << 22;  // polls of an L2 word: gives up after ~1 s at most
-
-// Bounded grid-wide barrier on two self-resetting counters in the workspace control block.
-// Returns false if the wait expired.
-__device__ bool grid_barrier(WsCtrl *ctrl, unsigned n_ctas) {
-    __shared__ int s_ok;
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        __threadfence();
-        atomicAdd(&ctrl->arrive, 1u);
-        unsigned spins = 0, seen;
-        int ok = 1;
-        for (;;) {
-            asm volatile("ld.acquire.gpu.u32 %0, [%1];" : "=r"(seen) : "l"(&ctrl->arrive) : "memory");
-            if (seen >= n_ctas) break;
-            if (++spins > kBarrierSpinLimit) {
-                ok = 0;
-                break;
-            }
-        }
-        s_ok = ok;
-        if (ok) {
-            const unsigned left = atomicAdd(&ctrl->depart, 1u);
-            if (left == n_ctas - 1) {  // last one out: everyone has seen arrive == n_ctas
-                ctrl->arrive = 0;
-                ctrl->depart = 0;
-                __threadfence();
-            }
-        }
-    }
-    __syncthreads();
-    return s_ok != 0;
-}
-
-// ---- mbarrier / bulk-copy primitives (bounded waits) -------------------------------------------
-
-__device__ __forceinline__ uint32_t smem_u32(const void *p) {
-    return static_cast<uint32_t>(__cvta_generic_to_shared(p));
-}
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(bar), "r"(parity), "r"(1000u)  // suspend for at most ~1 us per try
-        : "memory");
-    return ok != 0;
-}
-constexpr unsigned kMbarSpinLimit = 1u << 20;  // tries of at most ~1 us each: about a second
-// Waits for the phase with the given parity; gives up (returns false) after kMbarSpinLimit tries.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
-    for (unsigned i = 0; i < kMbarSpinLimit; ++i)
-        if (mbar_try_wait(bar, parity)) return true;
-    return false;
-}
-// Bulk copies move one contiguous row, global -> this CTA's shared memory, completion counted on an
-// mbarrier; both addresses are 16-byte aligned and the size is a multiple of 16.
-// L2 policies: weights are read once (evict first), the small per-call vectors are re-read by every
-// CTA and by the next call (evict last), so the streaming rows do not push them out of L2.
-__device__ __forceinline__ uint64_t policy_evict_first() {
-    uint64_t p;
-    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
-    return p;
-}
-__device__ __forceinline__ uint64_t policy_evict_last() {
-    uint64_t p;
-    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
-    return p;
-}
-__device__ __forceinline__ void bulk_load_row_hint(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar,
-                                                   uint64_t policy) {
-    asm volatile(
-        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
-        ::"r"(dst), "l"(src), "r"(bytes), "r"(bar), "l"(policy)
-        : "memory");
-}
-__device__ __forceinline__ float ld_keep(const float *p, uint64_t policy) {
-    float v;
-    asm volatile("ld.global.L2::cache_hint.f32 %0, [%1], %2;" : "=f"(v) : "l"(p), "l"(policy));
-    return v;
-}
-__device__ __forceinline__ float4 ld_keep4(const float4 *p, uint64_t policy) {
-    float4 v;
-    asm volatile("ld.global.L2::cache_hint.v4.f32 {%0,%1,%2,%3}, [%4], %5;"
-                 : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w)
-                 : "l"(p), "l"(policy));
-    return v;
-}
-__device__ __forceinline__ uint4 lds128(uint32_t addr) {
-    uint4 v;
-    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
-    return v;
-}
-
-// A 16-byte vector as E/2 pairs of fp32 (exact), ready for the packed two-wide FMA.
-template <typename T> struct Pairs;
-template <> struct Pairs<float> {
-    static constexpr int kPairs = 2;
-    __device__ static __forceinline__ void unpack(const uint4 &v, float2 (&f)[2]) {
-        f[0] = make_float2(__uint_as_float(v.x), __uint_as_float(v.y));
-        f[1] = make_float2(__uint_as_float(v.z), __uint_as_float(v.w));
-    }
-};
-template <> struct Pairs<__nv_bfloat16> {
-    static constexpr int kPairs = 4;
-    __device__ static __forceinline__ void unpack(const uint4 &v, float2 (&f)[4]) {
-        f[0] = make_float2(bf16_lo(v.x), bf16_hi(v.x));
-        f[1] = make_float2(bf16_lo(v.y), bf16_hi(v.y));
-        f[2] = make_float2(bf16_lo(v.z), bf16_hi(v.z));
-        f[3] = make_float2(bf16_lo(v.w), bf16_hi(v.w));
-    }
-};
-
-constexpr int kConsumers = 512;               // consumer threads (16 warps)
-constexpr int kConsWarps = kConsumers / kWarp;
-constexpr int kFfnThreads = kConsumers + 32;  // + one producer warp
-constexpr int kFfnWarps = kFfnThreads / kWarp;
-constexpr int kMaxStages = 16;
 constexpr int G = 4;                          // neurons per CTA-wide reduction
 constexpr int kMaxBatches = 4;                // prologue batches: d_ff <= 4 * 32 * kFfnThreads
 
@@ -566,13 +438,31 @@ static int decode_with_workspace(const clada_layer *layer, const void *x, int32_
     DeviceInfo di;
     rc = device_info(&di);
     if (rc != CLADA_OK) return rc;
-    const size_t need = kWsCtrlBytes + (size_t)di.num_sms * layer->d_model * sizeof(float);
+    const size_t need = kWsCtrlBytes + (size_t)di.num_sms * (B >= 4 ? 4 : B >= 2 ? 2 : 1) * layer->d_model * sizeof(float);
     if (ws_bytes < need) return CLADA_ERR_WORKSPACE;
 
     const size_t esz = elem_size(layer->dtype);
     const size_t ysz = elem_size(y_dtype);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    for (int b = 0; b < B; ++b) {
+    int b = 0;
+    while (b < B) {
+        // Tiles of 4 or 2 sequences read each row of the union of their kept sets once.
+        const int bt = ffn_batch_tile(layer, B - b);
+        if (bt > 1) {
+            if (mask_out || idx_out || count_out) {  // the tile kernel computes y only
+                rc = clada_select(scores + (size_t)b * layer->d_ff, bt, layer->d_ff, tau_final + (size_t)b * tau_stride,
+                                  tau_stride, mask_out ? mask_out + (size_t)b * layer->d_ff : nullptr,
+                                  idx_out ? idx_out + (size_t)b * layer->d_ff : nullptr,
+                                  count_out ? count_out + b : nullptr, stream);
+                if (rc != CLADA_OK) return rc;
+            }
+            rc = launch_ffn_batch(layer, bt, static_cast<const char *>(x) + (size_t)b * layer->d_model * esz,
+                                  scores + (size_t)b * layer->d_ff, tau_final + (size_t)b * tau_stride, tau_stride,
+                                  static_cast<char *>(y) + (size_t)b * layer->d_model * ysz, y_dtype, ws, status, st);
+            if (rc != CLADA_OK) return rc;
+            b += bt;
+            continue;
+        }
         FfnParams p;
         p.w_gate = layer->w_gate;
         p.w_up = layer->w_up;
@@ -592,6 +482,7 @@ static int decode_with_workspace(const clada_layer *layer, const void *x, int32_
         p.d_ff = layer->d_ff;
         rc = layer->dtype == CLADA_F32 ? launch_ffn<float>(p, st) : launch_ffn<__nv_bfloat16>(p, st);
         if (rc != CLADA_OK) return rc;
+        ++b;
     }
     return CLADA_OK;
 }

@@ -1,0 +1,447 @@
+// Sparse gated FFN decode for a tile of BT sequences at once (per-sequence masks):
+//   kept_b = { j : A_bj >= tau_b },   y_b = sum_{j in kept_b} silu(w_gate_j . x_b) (w_up_j . x_b) w_down_t[j,:]
+//
+// The rows of a neuron are read ONCE for the whole tile: the CTAs share out the UNION of the tile's kept
+// sets, stream each union neuron's three rows through the same bulk-copy ring as the single-sequence
+// kernel, and every consumer thread keeps x and the partial y of its columns for all BT sequences in
+// registers.  A sequence that does not keep a neuron of the union gets h = 0 for it, so each y_b is
+// exactly the sum over its own kept set.  8 dot products share one CTA-wide reduction (BT = 4: one
+// neuron per reduction, BT = 2: two).  Partial outputs are reduced across CTAs in a fixed order.
+#include <math.h>
+
+#include "common.cuh"
+#include "ffn_common.cuh"
+
+namespace clada {
+
+struct FfnBatchParams {
+    const void *w_gate, *w_up, *w_down_t;
+    const void *x;           // sequence b at x + b * x_stride (bytes)
+    size_t x_stride;
+    const float *scores;     // [BT, d_ff]
+    const float *tau;        // sequence b at tau[b * tau_stride]
+    long long tau_stride;
+    void *y;                 // sequence b at y + b * y_stride (bytes)
+    size_t y_stride;
+    int y_dtype;
+    float *partials;         // [gridDim.x, BT, d_model]
+    WsCtrl *ctrl;
+    int32_t *status;
+    int d_model, d_ff;
+};
+
+constexpr int kBatchMaxBatches = 4;  // prologue batches: d_ff <= 4 * 32 * kFfnThreads
+
+template <typename T, int NV, int BT>
+__global__ void __launch_bounds__(kFfnThreads, 1)
+sparse_ffn_batch_kernel(const FfnBatchParams p, const int n_stages) {
+    constexpr int E = Elem<T>::kPerVec;
+    constexpr int P = Pairs<T>::kPairs;
+    constexpr int GB = 4 / BT;  // neurons per CTA-wide reduction: 8 dot products each time
+    static_assert(BT == 2 || BT == 4, "tile of 2 or 4 sequences");
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int cta = blockIdx.x, n_ctas = gridDim.x;
+    const int F = p.d_ff, d = p.d_model;
+    const int vpr = d / E;
+    const uint32_t row_bytes = (uint32_t)vpr * 16u;
+    const uint32_t stage_bytes = 3u * row_bytes;
+    const int chunks = (F + kWarp - 1) / kWarp;
+    const int list_cap = F / n_ctas + 2;
+
+    // dynamic shared memory: ring | full | empty | union keep-bits | per-sequence keep-bits | list | keep nibbles
+    const uint32_t ring = smem_u32(smem_raw);
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem_raw + (size_t)n_stages * stage_bytes);
+    const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + kMaxStages);
+    unsigned *s_bal = reinterpret_cast<unsigned *>(bars + 2 * kMaxStages);
+    unsigned *s_balb = s_bal + chunks;                      // [BT][chunks]
+    int *s_list = reinterpret_cast<int *>(s_balb + BT * chunks);
+    int *s_keep = s_list + list_cap;                        // bit b: sequence b keeps this neuron
+    __shared__ int s_wtot[kFfnWarps];
+    __shared__ float s_tau[BT];
+    __shared__ __align__(16) float s_dot[2][8][kConsWarps];
+
+    pdl_launch_dependents();
+    if (tid == kConsumers) {
+        for (int s = 0; s < n_stages; ++s) {
+            mbar_init(full0 + 8 * s, 1);
+            mbar_init(empty0 + 8 * s, kConsWarps);
+        }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    pdl_wait();
+
+    const uint64_t keep_policy = policy_evict_last();
+    if (tid < BT) s_tau[tid] = ld_keep(p.tau + (size_t)tid * p.tau_stride, keep_policy);
+    float2 xr[BT][NV][P];
+    bool vok[NV];
+#pragma unroll
+    for (int i = 0; i < NV; ++i) {
+        const int v = tid + i * kConsumers;
+        vok[i] = tid < kConsumers && v < vpr;
+#pragma unroll
+        for (int b = 0; b < BT; ++b) {
+            uint4 q = make_uint4(0, 0, 0, 0);
+            if (vok[i]) q = *(reinterpret_cast<const uint4 *>(static_cast<const char *>(p.x) + b * p.x_stride) + v);
+            Pairs<T>::unpack(q, xr[b][i]);
+        }
+    }
+    __syncthreads();  // thresholds are in shared memory
+
+    // ---- prologue: keep-bits per sequence, their union, ranks of the union -----------------------
+    const int n_batches = (chunks + kFfnThreads - 1) / kFfnThreads;
+    {
+        int slot = tid + (cta * 37) % kFfnThreads;
+        if (slot >= kFfnThreads) slot -= kFfnThreads;
+        for (int bt = 0; bt < n_batches; ++bt) {
+            const int q = bt * kFfnThreads + slot;
+            if (q >= chunks) continue;
+            const int j0 = q * kWarp;
+            unsigned wu = 0;
+#pragma unroll
+            for (int b = 0; b < BT; ++b) {
+                const float *sc = p.scores + (size_t)b * F;
+                const float tau = s_tau[b];
+                unsigned w = 0;
+                if (((reinterpret_cast<uintptr_t>(sc) & 15u) == 0) && j0 + kWarp <= F) {
+                    float4 v[8];
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) v[u] = ld_keep4(reinterpret_cast<const float4 *>(sc + j0) + u, keep_policy);
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) {
+                        w |= (v[u].x >= tau ? 1u : 0u) << (4 * u);
+                        w |= (v[u].y >= tau ? 1u : 0u) << (4 * u + 1);
+                        w |= (v[u].z >= tau ? 1u : 0u) << (4 * u + 2);
+                        w |= (v[u].w >= tau ? 1u : 0u) << (4 * u + 3);
+                    }
+                } else {
+                    for (int u = 0; u < kWarp; ++u)
+                        if (j0 + u < F && ld_keep(sc + j0 + u, keep_policy) >= tau) w |= 1u << u;
+                }
+                s_balb[b * chunks + q] = w;
+                wu |= w;
+            }
+            s_bal[q] = wu;
+        }
+    }
+    __syncthreads();
+    unsigned bal[kBatchMaxBatches];
+    int first_rank[kBatchMaxBatches];
+    int n_act = 0;
+#pragma unroll
+    for (int bt = 0; bt < kBatchMaxBatches; ++bt) {
+        bal[bt] = 0u;
+        first_rank[bt] = 0;
+        if (bt >= n_batches) continue;  // uniform
+        const int q = bt * kFfnThreads + tid;
+        if (q < chunks) bal[bt] = s_bal[q];
+        const int cnt = __popc(bal[bt]);
+        int incl = cnt;
+#pragma unroll
+        for (int o = 1; o < kWarp; o <<= 1) {
+            const int t = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += t;
+        }
+        if (bt > 0) __syncthreads();
+        if (lane == kWarp - 1) s_wtot[warp] = incl;
+        __syncthreads();
+        int wbase = 0, btot = 0;
+#pragma unroll
+        for (int w = 0; w < kFfnWarps; ++w) {
+            const int v = s_wtot[w];
+            wbase += (w < warp) ? v : 0;
+            btot += v;
+        }
+        first_rank[bt] = n_act + wbase + incl - cnt;
+        n_act += btot;
+    }
+    const int r0 = (int)(((int64_t)n_act * cta) / n_ctas);
+    const int r1 = (int)(((int64_t)n_act * (cta + 1)) / n_ctas);
+#pragma unroll
+    for (int bt = 0; bt < kBatchMaxBatches; ++bt) {
+        if (bt >= n_batches) continue;  // uniform
+        const int q = bt * kFfnThreads + tid;
+        const int fr = first_rank[bt];
+        const bool in_share = q < chunks && fr < r1 && fr + __popc(bal[bt]) > r0;
+        unsigned todo = __ballot_sync(0xffffffffu, in_share);
+        while (todo) {
+            const int t = __ffs(todo) - 1;
+            todo &= todo - 1;
+            const unsigned wb = __shfl_sync(0xffffffffu, bal[bt], t);
+            const int wfr = __shfl_sync(0xffffffffu, fr, t);
+            const int qq = bt * kFfnThreads + warp * kWarp + t;
+            const int rank = wfr + __popc(wb & ((1u << lane) - 1u));
+            if (((wb >> lane) & 1u) && rank >= r0 && rank < r1) {
+                int bits = 0;
+#pragma unroll
+                for (int b = 0; b < BT; ++b) bits |= (int)((s_balb[b * chunks + qq] >> lane) & 1u) << b;
+                s_list[rank - r0] = qq * kWarp + lane;
+                s_keep[rank - r0] = bits;
+            }
+        }
+    }
+    const int my_n = r1 - r0;
+    __syncthreads();  // list, keep bits and the mbarriers are ready
+
+    bool timed_out = false;
+
+    if (warp == kConsWarps) {
+        // ---- producer (as in the single-sequence kernel) -------------------------------------------
+        if (lane == 0) {
+            const char *Wg = static_cast<const char *>(p.w_gate);
+            const char *Wu = static_cast<const char *>(p.w_up);
+            const char *Wd = static_cast<const char *>(p.w_down_t);
+            const uint64_t stream_policy = policy_evict_first();
+            int issued = 0;
+            for (int i = 0; i < my_n; ++i) {
+                const int s = i % n_stages, use = i / n_stages;
+                if (!mbar_wait(empty0 + 8 * s, (use & 1) ^ 1)) {
+                    timed_out = true;
+                    break;
+                }
+                const size_t off = (size_t)s_list[i] * row_bytes;
+                const uint32_t dst = ring + (uint32_t)s * stage_bytes, bar = full0 + 8 * s;
+                mbar_expect_tx(bar, stage_bytes);
+                bulk_load_row_hint(dst, Wg + off, row_bytes, bar, stream_policy);
+                bulk_load_row_hint(dst + row_bytes, Wu + off, row_bytes, bar, stream_policy);
+                bulk_load_row_hint(dst + 2 * row_bytes, Wd + off, row_bytes, bar, stream_policy);
+                issued = i + 1;
+            }
+            for (int i = max(0, issued - n_stages); i < issued; ++i)
+                if (!mbar_wait(full0 + 8 * (i % n_stages), (i / n_stages) & 1)) timed_out = true;
+        }
+    } else {
+        // ---- consumers ---------------------------------------------------------------------------
+        float2 acc[BT][NV][P];
+#pragma unroll
+        for (int b = 0; b < BT; ++b)
+#pragma unroll
+            for (int i = 0; i < NV; ++i)
+#pragma unroll
+                for (int e = 0; e < P; ++e) acc[b][i][e] = make_float2(0.f, 0.f);
+        const bool b16 = lane & 16, b8 = lane & 8, b4 = lane & 4;
+        int buf = 0;
+        for (int g0 = 0; g0 < my_n; g0 += GB, buf ^= 1) {
+            float pd[8];  // value (g * BT + b) * 2 + {0: gate, 1: up}
+            uint32_t st_addr[GB];
+#pragma unroll
+            for (int g = 0; g < GB; ++g) {
+                const int i = g0 + g;
+                float2 sg[BT], su[BT];
+#pragma unroll
+                for (int b = 0; b < BT; ++b) sg[b] = su[b] = make_float2(0.f, 0.f);
+                st_addr[g] = ring + (uint32_t)(i % n_stages) * stage_bytes;
+                if (i < my_n) {
+                    if (!timed_out && !mbar_wait(full0 + 8 * (i % n_stages), (i / n_stages) & 1)) timed_out = true;
+#pragma unroll
+                    for (int k = 0; k < NV; ++k) {
+                        if (!vok[k]) continue;
+                        const uint32_t a = st_addr[g] + (uint32_t)(tid + k * kConsumers) * 16u;
+                        float2 fg[P], fu[P];
+                        Pairs<T>::unpack(lds128(a), fg);
+                        Pairs<T>::unpack(lds128(a + row_bytes), fu);
+#pragma unroll
+                        for (int b = 0; b < BT; ++b)
+#pragma unroll
+                            for (int e = 0; e < P; ++e) {
+                                sg[b] = __ffma2_rn(fg[e], xr[b][k][e], sg[b]);
+                                su[b] = __ffma2_rn(fu[e], xr[b][k][e], su[b]);
+                            }
+                    }
+                }
+#pragma unroll
+                for (int b = 0; b < BT; ++b) {
+                    pd[(g * BT + b) * 2] = sg[b].x + sg[b].y;
+                    pd[(g * BT + b) * 2 + 1] = su[b].x + su[b].y;
+                }
+            }
+            // warp sums of the 8 values by a halving butterfly, then across warps (fixed order)
+            float bb[4], c[2], v8;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const float send = b16 ? pd[i] : pd[i + 4];
+                bb[i] = (b16 ? pd[i + 4] : pd[i]) + __shfl_xor_sync(0xffffffffu, send, 16);
+            }
+#pragma unroll
+            for (int i = 0; i < 2; ++i) {
+                const float send = b8 ? bb[i] : bb[i + 2];
+                c[i] = (b8 ? bb[i + 2] : bb[i]) + __shfl_xor_sync(0xffffffffu, send, 8);
+            }
+            v8 = (b4 ? c[1] : c[0]) + __shfl_xor_sync(0xffffffffu, b4 ? c[0] : c[1], 4);
+            v8 += __shfl_xor_sync(0xffffffffu, v8, 2);
+            v8 += __shfl_xor_sync(0xffffffffu, v8, 1);
+            if ((lane & 3) == 0) s_dot[buf][(b16 ? 4 : 0) + (b8 ? 2 : 0) + (b4 ? 1 : 0)][warp] = v8;
+            asm volatile("bar.sync 1, %0;" ::"n"(kConsumers) : "memory");
+            float tot;
+            {
+                const float4 q4 = *reinterpret_cast<const float4 *>(&s_dot[buf][lane >> 2][(lane & 3) * 4]);
+                tot = (q4.x + q4.y) + (q4.z + q4.w);
+                tot += __shfl_xor_sync(0xffffffffu, tot, 1);
+                tot += __shfl_xor_sync(0xffffffffu, tot, 2);
+            }
+            const float up = __shfl_xor_sync(0xffffffffu, tot, 4);
+            const float hval = silu_f(tot) * up;  // pair m = g * BT + b sits on lanes 8m .. 8m+3
+#pragma unroll
+            for (int g = 0; g < GB; ++g) {
+                float h[BT];
+#pragma unroll
+                for (int b = 0; b < BT; ++b) h[b] = __shfl_sync(0xffffffffu, hval, 8 * (g * BT + b));
+                if (g0 + g >= my_n) continue;
+                const int bits = s_keep[g0 + g];
+#pragma unroll
+                for (int k = 0; k < NV; ++k) {
+                    if (!vok[k]) continue;
+                    float2 fd[P];
+                    Pairs<T>::unpack(lds128(st_addr[g] + 2 * row_bytes + (uint32_t)(tid + k * kConsumers) * 16u), fd);
+#pragma unroll
+                    for (int b = 0; b < BT; ++b) {
+                        const float hb = ((bits >> b) & 1) ? h[b] : 0.f;  // not kept by sequence b: no contribution
+                        const float2 h2 = make_float2(hb, hb);
+#pragma unroll
+                        for (int e = 0; e < P; ++e) acc[b][k][e] = __ffma2_rn(h2, fd[e], acc[b][k][e]);
+                    }
+                }
+            }
+            __syncwarp();
+            if (lane == 0) {
+#pragma unroll
+                for (int g = 0; g < GB; ++g)
+                    if (g0 + g < my_n) mbar_arrive(empty0 + 8 * ((g0 + g) % n_stages));
+            }
+        }
+#pragma unroll
+        for (int b = 0; b < BT; ++b) {
+            float *mine = p.partials + ((size_t)cta * BT + b) * d;
+#pragma unroll
+            for (int i = 0; i < NV; ++i) {
+                if (!vok[i]) continue;
+                float4 *dst = reinterpret_cast<float4 *>(mine + (size_t)(tid + i * kConsumers) * E);
+#pragma unroll
+                for (int e = 0; e < P; e += 2)
+                    dst[e / 2] = make_float4(acc[b][i][e].x, acc[b][i][e].y, acc[b][i][e + 1].x, acc[b][i][e + 1].y);
+            }
+        }
+    }
+    if (timed_out && p.status) atomicOr(p.status, CLADA_STATUS_TIMEOUT);
+
+    // ---- epilogue: grid barrier, deterministic column reduction per sequence ----------------------
+    if (!grid_barrier(p.ctrl, (unsigned)n_ctas)) {
+        if (tid == 0 && p.status) atomicOr(p.status, CLADA_STATUS_TIMEOUT);
+        return;
+    }
+    const int ngroups = d / 4;
+    for (int it = cta + warp * n_ctas; it < BT * ngroups; it += n_ctas * kFfnWarps) {
+        const int b = it / ngroups, q = it % ngroups;
+        float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int rb = 0; rb < n_ctas; rb += 5 * kWarp) {
+            float4 v[5];
+#pragma unroll
+            for (int u = 0; u < 5; ++u) {
+                const int r = rb + u * kWarp + lane;
+                v[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (r < n_ctas)
+                    v[u] = __ldcg(reinterpret_cast<const float4 *>(p.partials + ((size_t)r * BT + b) * d) + q);
+            }
+#pragma unroll
+            for (int u = 0; u < 5; ++u) {
+                s.x += v[u].x; s.y += v[u].y; s.z += v[u].z; s.w += v[u].w;
+            }
+        }
+        s.x = warp_sum(s.x); s.y = warp_sum(s.y); s.z = warp_sum(s.z); s.w = warp_sum(s.w);
+        if (lane == 0) {
+            char *yb = static_cast<char *>(p.y) + b * p.y_stride;
+            if (p.y_dtype == CLADA_F32) {
+                reinterpret_cast<float4 *>(yb)[q] = s;
+            } else {
+                __nv_bfloat162 lo = __floats2bfloat162_rn(s.x, s.y), hi = __floats2bfloat162_rn(s.z, s.w);
+                uint2 o;
+                o.x = *reinterpret_cast<uint32_t *>(&lo);
+                o.y = *reinterpret_cast<uint32_t *>(&hi);
+                reinterpret_cast<uint2 *>(yb)[q] = o;
+            }
+        }
+    }
+}
+
+
+// ---- host side ------------------------------------------------------------------------------
+
+template <typename T, int NV, int BT>
+static int launch_batch_variant(const FfnBatchParams &p, cudaStream_t st) {
+    constexpr int E = Elem<T>::kPerVec;
+    static bool configured[64] = {};
+    DeviceInfo di;
+    int rc = device_info(&di);
+    if (rc != CLADA_OK) return rc;
+    auto kern = sparse_ffn_batch_kernel<T, NV, BT>;
+    const size_t stage_bytes = 3 * (size_t)(p.d_model / E) * 16;
+    const size_t chunks = (size_t)(p.d_ff + 31) / 32;
+    const size_t tail = 2 * kMaxStages * sizeof(uint64_t) + (1 + BT) * chunks * sizeof(unsigned) +
+                        2 * (size_t)(p.d_ff / di.num_sms + 2) * sizeof(int);
+    const size_t budget = (size_t)di.max_smem_optin - 2048;
+    if (budget < tail + 4 * stage_bytes) return CLADA_ERR_UNSUPPORTED;
+    int n_stages = (int)((budget - tail) / stage_bytes);
+    if (n_stages > kMaxStages) n_stages = kMaxStages;
+    const size_t smem = (size_t)n_stages * stage_bytes + tail;
+    if (!configured[di.device & 63]) {
+        CLADA_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)budget));
+        configured[di.device & 63] = true;
+    }
+    FfnBatchParams params = p;
+    int stages_arg = n_stages;
+    void *args[] = {&params, &stages_arg};
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(di.num_sms);
+    cfg.blockDim = dim3(kFfnThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeCooperative;  // all CTAs co-resident: the grid barrier cannot starve
+    attr[0].val.cooperative = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 2;
+    CLADA_CUDA_TRY(cudaLaunchKernelExC(&cfg, reinterpret_cast<const void *>(kern), args));
+    return CLADA_OK;
+}
+
+int ffn_batch_tile(const clada_layer *layer, int remaining) {
+    const int vpr = layer->d_model / (layer->dtype == CLADA_F32 ? 4 : 8);
+    if (layer->d_ff > kBatchMaxBatches * kWarp * kFfnThreads) return 1;
+    if (remaining >= 4 && vpr <= kConsumers) return 4;
+    if (remaining >= 2 && vpr <= 2 * kConsumers) return 2;
+    return 1;
+}
+
+int launch_ffn_batch(const clada_layer *layer, int bt, const void *x, const float *scores, const float *tau,
+                     long long tau_stride, void *y, int y_dtype, void *ws, int32_t *status, cudaStream_t st) {
+    FfnBatchParams p;
+    p.w_gate = layer->w_gate;
+    p.w_up = layer->w_up;
+    p.w_down_t = layer->w_down_t;
+    p.x = x;
+    p.x_stride = (size_t)layer->d_model * elem_size(layer->dtype);
+    p.scores = scores;
+    p.tau = tau;
+    p.tau_stride = tau_stride;
+    p.y = y;
+    p.y_stride = (size_t)layer->d_model * elem_size(y_dtype);
+    p.y_dtype = y_dtype;
+    p.partials = reinterpret_cast<float *>(static_cast<char *>(ws) + kWsCtrlBytes);
+    p.ctrl = static_cast<WsCtrl *>(ws);
+    p.status = status;
+    p.d_model = layer->d_model;
+    p.d_ff = layer->d_ff;
+    const bool f32 = layer->dtype == CLADA_F32;
+    const int vpr = layer->d_model / (f32 ? 4 : 8);
+    if (bt == 4 && vpr <= kConsumers)
+        return f32 ? launch_batch_variant<float, 1, 4>(p, st) : launch_batch_variant<__nv_bfloat16, 1, 4>(p, st);
+    if (bt == 2 && vpr <= kConsumers)
+        return f32 ? launch_batch_variant<float, 1, 2>(p, st) : launch_batch_variant<__nv_bfloat16, 1, 2>(p, st);
+    if (bt == 2 && vpr <= 2 * kConsumers)
+        return f32 ? launch_batch_variant<float, 2, 2>(p, st) : launch_batch_variant<__nv_bfloat16, 2, 2>(p, st);
+    return CLADA_ERR_UNSUPPORTED;
+}
+
+}  // namespace clada

@@ -469,3 +469,49 @@ def test_algorithm2_loop_config1(clada, oracle):
         assert rel_inf(y[0].cpu().numpy(), y_or) <= FFN_TOL_F32
     assert int(status.item()) == 0
     assert len(seen) >= 3          # the loop exercised several of the four threshold levels
+
+
+# ------------------------------------------------------------------------------------------------
+# batched decode: tiles of 4 / 2 sequences read the union of their kept rows once
+# ------------------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("name,d,F,B", [("c4_llama3_8b_b8", 1024, 1800, 7), ("c5_13b_b16", 5120, 700, 5),
+                                        ("c1_small_f32", 512, 1376, 6), ("c4_llama3_8b_b8", 4096, 1000, 4)])
+def test_sparse_ffn_batched_tiles(clada, oracle, name, d, F, B):
+    """Per-sequence scores and thresholds, including a sequence that keeps nothing and one that keeps all:
+    every y_b must be the sum over its own kept set although the tile streams the union."""
+    w = _small(name, d_model=d, d_ff=F, batch=B)
+    weights = wl.layer_weights(w, 0)
+    layer = gpu_layer(weights, clada)
+    W_in, V_in, W_out = oracle_weights(weights)
+    rng = np.random.default_rng(B * 1000 + d)
+    scores = (rng.random((B, F)) + 0.5).astype(np.float32)
+    taus = (0.7 + 0.6 * rng.random(B)).astype(np.float32)
+    taus[1] = np.inf          # keeps nothing
+    taus[2] = 0.0             # keeps everything
+    xs = torch.stack([wl.hidden_states(w, 0, "decode", b, 1)[0] for b in range(B)])
+    ws = clada.new_workspace(layer, B, 0)
+    for y_dtype, tol in ((torch.float32, FFN_TOL_F32), (torch.bfloat16, FFN_TOL_BF16_OUT)):
+        y = torch.empty(B, d, dtype=y_dtype, device="cuda")
+        mask = torch.empty(B, F, dtype=torch.uint8, device="cuda")
+        idx = torch.full((B, F), -1, dtype=torch.int32, device="cuda")
+        count = torch.empty(B, dtype=torch.int32, device="cuda")
+        status = torch.zeros(1, dtype=torch.int32, device="cuda")
+        clada.clada_sparse_ffn_decode(layer, xs.cuda(), _dev(scores), _dev(taus), 1, y, ws, mask, idx, count, status)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        for b in range(B):
+            y_or, m_or, n_or = oracle.sparse_ffn(wl.to_numpy_bits(xs[b]), W_in, V_in, W_out,
+                                                 scores[b].astype(np.float64), float(taus[b]))
+            assert int(count[b]) == n_or
+            np.testing.assert_array_equal(mask[b].cpu().numpy(), m_or)
+            np.testing.assert_array_equal(idx[b, :n_or].cpu().numpy(), np.nonzero(m_or)[0])
+            if n_or == 0:
+                assert bool((y[b] == 0).all())
+            else:
+                assert rel_inf(y[b].float().cpu().numpy(), y_or) <= tol, (b, y_dtype)
+        # without the optional outputs the same y comes back bit for bit
+        y2 = torch.empty_like(y)
+        clada.clada_sparse_ffn_decode(layer, xs.cuda(), _dev(scores), _dev(taus), 1, y2, ws)
+        torch.cuda.synchronize()
+        assert torch.equal(y, y2)
