@@ -5,8 +5,8 @@
 // sets, stream each union neuron's three rows through the same bulk-copy ring as the single-sequence
 // kernel, and every consumer thread keeps x and the partial y of its columns for all BT sequences in
 // registers.  A sequence that does not keep a neuron of the union gets h = 0 for it, so each y_b is
-// exactly the sum over its own kept set.  8 dot products share one CTA-wide reduction (BT = 4: one
-// neuron per reduction, BT = 2: two).  Partial outputs are reduced across CTAs in a fixed order.
+// exactly the sum over its own kept set.  16 dot products share one CTA-wide reduction (BT = 4: two
+// neurons per reduction, BT = 2: four).  Partial outputs are reduced across CTAs in a fixed order.
 #include <math.h>
 
 #include "common.cuh"
@@ -37,7 +37,7 @@ __global__ void __launch_bounds__(kFfnThreads, 1)
 sparse_ffn_batch_kernel(const FfnBatchParams p, const int n_stages) {
     constexpr int E = Elem<T>::kPerVec;
     constexpr int P = Pairs<T>::kPairs;
-    constexpr int GB = 4 / BT;  // neurons per CTA-wide reduction: 8 dot products each time
+    constexpr int GB = 8 / BT;  // neurons per CTA-wide reduction: 16 dot products each time
     static_assert(BT == 2 || BT == 4, "tile of 2 or 4 sequences");
     extern __shared__ __align__(128) unsigned char smem_raw[];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -59,7 +59,7 @@ sparse_ffn_batch_kernel(const FfnBatchParams p, const int n_stages) {
     int *s_keep = s_list + list_cap;                        // bit b: sequence b keeps this neuron
     __shared__ int s_wtot[kFfnWarps];
     __shared__ float s_tau[BT];
-    __shared__ __align__(16) float s_dot[2][8][kConsWarps];
+    __shared__ __align__(16) float s_dot[2][16][kConsWarps];
 
     pdl_launch_dependents();
     if (tid == kConsumers) {
@@ -219,10 +219,10 @@ sparse_ffn_batch_kernel(const FfnBatchParams p, const int n_stages) {
             for (int i = 0; i < NV; ++i)
 #pragma unroll
                 for (int e = 0; e < P; ++e) acc[b][i][e] = make_float2(0.f, 0.f);
-        const bool b16 = lane & 16, b8 = lane & 8, b4 = lane & 4;
+        const bool b16 = lane & 16, b8 = lane & 8, b4 = lane & 4, b2 = lane & 2;
         int buf = 0;
         for (int g0 = 0; g0 < my_n; g0 += GB, buf ^= 1) {
-            float pd[8];  // value (g * BT + b) * 2 + {0: gate, 1: up}
+            float pd[16];  // value (g * BT + b) * 2 + {0: gate, 1: up}
             uint32_t st_addr[GB];
 #pragma unroll
             for (int g = 0; g < GB; ++g) {
@@ -255,37 +255,44 @@ sparse_ffn_batch_kernel(const FfnBatchParams p, const int n_stages) {
                     pd[(g * BT + b) * 2 + 1] = su[b].x + su[b].y;
                 }
             }
-            // warp sums of the 8 values by a halving butterfly, then across warps (fixed order)
-            float bb[4], c[2], v8;
+            // Warp sums of the 16 values by a halving butterfly (16 shuffles): afterwards both lanes of pair
+            // v hold the warp total of value v.  Then across the 16 warps through shared memory: lane l adds
+            // 8 warps of value l / 2, the pair finishes.  Fixed order throughout.
+            float b8v[8], b4v[4], b2v[2], v16;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const float send = b16 ? pd[i] : pd[i + 8];
+                b8v[i] = (b16 ? pd[i + 8] : pd[i]) + __shfl_xor_sync(0xffffffffu, send, 16);
+            }
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
-                const float send = b16 ? pd[i] : pd[i + 4];
-                bb[i] = (b16 ? pd[i + 4] : pd[i]) + __shfl_xor_sync(0xffffffffu, send, 16);
+                const float send = b8 ? b8v[i] : b8v[i + 4];
+                b4v[i] = (b8 ? b8v[i + 4] : b8v[i]) + __shfl_xor_sync(0xffffffffu, send, 8);
             }
 #pragma unroll
             for (int i = 0; i < 2; ++i) {
-                const float send = b8 ? bb[i] : bb[i + 2];
-                c[i] = (b8 ? bb[i + 2] : bb[i]) + __shfl_xor_sync(0xffffffffu, send, 8);
+                const float send = b4 ? b4v[i] : b4v[i + 2];
+                b2v[i] = (b4 ? b4v[i + 2] : b4v[i]) + __shfl_xor_sync(0xffffffffu, send, 4);
             }
-            v8 = (b4 ? c[1] : c[0]) + __shfl_xor_sync(0xffffffffu, b4 ? c[0] : c[1], 4);
-            v8 += __shfl_xor_sync(0xffffffffu, v8, 2);
-            v8 += __shfl_xor_sync(0xffffffffu, v8, 1);
-            if ((lane & 3) == 0) s_dot[buf][(b16 ? 4 : 0) + (b8 ? 2 : 0) + (b4 ? 1 : 0)][warp] = v8;
+            v16 = (b2 ? b2v[1] : b2v[0]) + __shfl_xor_sync(0xffffffffu, b2 ? b2v[0] : b2v[1], 2);
+            v16 += __shfl_xor_sync(0xffffffffu, v16, 1);
+            // value index: bit4 -> +8, bit3 -> +4, bit2 -> +2, bit1 -> +1  ( = lane >> 1 )
+            if ((lane & 1) == 0) s_dot[buf][lane >> 1][warp] = v16;
             asm volatile("bar.sync 1, %0;" ::"n"(kConsumers) : "memory");
             float tot;
             {
-                const float4 q4 = *reinterpret_cast<const float4 *>(&s_dot[buf][lane >> 2][(lane & 3) * 4]);
-                tot = (q4.x + q4.y) + (q4.z + q4.w);
+                const float4 *src = reinterpret_cast<const float4 *>(&s_dot[buf][lane >> 1][(lane & 1) * 8]);
+                const float4 q0 = src[0], q1 = src[1];
+                tot = ((q0.x + q0.y) + (q0.z + q0.w)) + ((q1.x + q1.y) + (q1.z + q1.w));
                 tot += __shfl_xor_sync(0xffffffffu, tot, 1);
-                tot += __shfl_xor_sync(0xffffffffu, tot, 2);
             }
-            const float up = __shfl_xor_sync(0xffffffffu, tot, 4);
-            const float hval = silu_f(tot) * up;  // pair m = g * BT + b sits on lanes 8m .. 8m+3
+            const float up = __shfl_xor_sync(0xffffffffu, tot, 2);  // value 2m+1 sits 2 lanes above value 2m
+            const float hval = silu_f(tot) * up;                    // pair m = g * BT + b sits on lanes 4m, 4m+1
 #pragma unroll
             for (int g = 0; g < GB; ++g) {
                 float h[BT];
 #pragma unroll
-                for (int b = 0; b < BT; ++b) h[b] = __shfl_sync(0xffffffffu, hval, 8 * (g * BT + b));
+                for (int b = 0; b < BT; ++b) h[b] = __shfl_sync(0xffffffffu, hval, 4 * (g * BT + b));
                 if (g0 + g >= my_n) continue;
                 const int bits = s_keep[g0 + g];
 #pragma unroll
@@ -379,7 +386,7 @@ static int launch_batch_variant(const FfnBatchParams &p, cudaStream_t st) {
     const size_t tail = 2 * kMaxStages * sizeof(uint64_t) + (1 + BT) * chunks * sizeof(unsigned) +
                         2 * (size_t)(p.d_ff / di.num_sms + 2) * sizeof(int);
     const size_t budget = (size_t)di.max_smem_optin - 2048;
-    if (budget < tail + 4 * stage_bytes) return CLADA_ERR_UNSUPPORTED;
+    if (budget < tail + 4 * stage_bytes) return CLADA_ERR_UNSUPPORTED;  // a reduction group needs up to 4 stages
     int n_stages = (int)((budget - tail) / stage_bytes);
     if (n_stages > kMaxStages) n_stages = kMaxStages;
     const size_t smem = (size_t)n_stages * stage_bytes + tail;
