@@ -385,7 +385,7 @@ static int launch_batch_variant(const FfnBatchParams &p, cudaStream_t st) {
     const size_t chunks = (size_t)(p.d_ff + 31) / 32;
     const size_t tail = 2 * kMaxStages * sizeof(uint64_t) + (1 + BT) * chunks * sizeof(unsigned) +
                         2 * (size_t)(p.d_ff / di.num_sms + 2) * sizeof(int);
-    const size_t budget = (size_t)di.max_smem_optin - 2048;
+    const size_t budget = (size_t)di.max_smem_optin - 4096;  // leave room for the static arrays
     if (budget < tail + 4 * stage_bytes) return CLADA_ERR_UNSUPPORTED;  // a reduction group needs up to 4 stages
     int n_stages = (int)((budget - tail) / stage_bytes);
     if (n_stages > kMaxStages) n_stages = kMaxStages;
