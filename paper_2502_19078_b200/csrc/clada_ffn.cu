@@ -212,9 +212,10 @@ sparse_ffn_kernel(const FfnParams p, const int n_stages) {
             const char *Wd = static_cast<const char *>(p.w_down_t);
             const uint64_t stream_policy = policy_evict_first();
             int issued = 0;
+            int s = 0;            // ring position and the parity of its current use, kept incrementally
+            uint32_t par = 0;
             for (int i = 0; i < my_n; ++i) {
-                const int s = i % n_stages, use = i / n_stages;
-                if (!mbar_wait(empty0 + 8 * s, (use & 1) ^ 1)) {  // a fresh barrier passes parity 1 at once
+                if (!mbar_wait(empty0 + 8 * s, par ^ 1)) {  // a fresh barrier passes parity 1 at once
                     timed_out = true;
                     break;
                 }
@@ -225,6 +226,10 @@ sparse_ffn_kernel(const FfnParams p, const int n_stages) {
                 bulk_load_row_hint(dst + row_bytes, Wu + off, row_bytes, bar, stream_policy);
                 bulk_load_row_hint(dst + 2 * row_bytes, Wd + off, row_bytes, bar, stream_policy);
                 issued = i + 1;
+                if (++s == n_stages) {
+                    s = 0;
+                    par ^= 1;
+                }
             }
             // Never leave with copies in flight: the last use of every stage must have landed.
             for (int i = max(0, issued - n_stages); i < issued; ++i)
@@ -239,16 +244,24 @@ sparse_ffn_kernel(const FfnParams p, const int n_stages) {
             for (int e = 0; e < P; ++e) acc[i][e] = make_float2(0.f, 0.f);
         const bool b16 = lane & 16, b8 = lane & 8, b4 = lane & 4;
         int buf = 0;
+        int cs = 0;           // ring position of the next neuron to consume, and the parity of its use
+        uint32_t cpar = 0;
         for (int g0 = 0; g0 < my_n; g0 += G, buf ^= 1) {
             float pd[2 * G];
             uint32_t st_addr[G];
+            int st_idx[G];
 #pragma unroll
             for (int g = 0; g < G; ++g) {
                 const int i = g0 + g;
                 float2 sg = make_float2(0.f, 0.f), su = make_float2(0.f, 0.f);
-                st_addr[g] = ring + (uint32_t)(i % n_stages) * stage_bytes;
+                st_idx[g] = cs;
+                st_addr[g] = ring + (uint32_t)cs * stage_bytes;
                 if (i < my_n) {
-                    if (!timed_out && !mbar_wait(full0 + 8 * (i % n_stages), (i / n_stages) & 1)) timed_out = true;
+                    if (!timed_out && !mbar_wait(full0 + 8 * cs, cpar)) timed_out = true;
+                    if (++cs == n_stages) {
+                        cs = 0;
+                        cpar ^= 1;
+                    }
 #pragma unroll
                     for (int k = 0; k < NV; ++k) {
                         if (!vok[k]) continue;
@@ -315,7 +328,7 @@ sparse_ffn_kernel(const FfnParams p, const int n_stages) {
             if (lane == 0) {
 #pragma unroll
                 for (int g = 0; g < G; ++g)
-                    if (g0 + g < my_n) mbar_arrive(empty0 + 8 * ((g0 + g) % n_stages));
+                    if (g0 + g < my_n) mbar_arrive(empty0 + 8 * st_idx[g]);
             }
         }
         // partial y of this CTA

@@ -193,9 +193,10 @@ sparse_ffn_batch_kernel(const FfnBatchParams p, const int n_stages) {
             const char *Wd = static_cast<const char *>(p.w_down_t);
             const uint64_t stream_policy = policy_evict_first();
             int issued = 0;
+            int s = 0;            // ring position and the parity of its current use, kept incrementally
+            uint32_t par = 0;
             for (int i = 0; i < my_n; ++i) {
-                const int s = i % n_stages, use = i / n_stages;
-                if (!mbar_wait(empty0 + 8 * s, (use & 1) ^ 1)) {
+                if (!mbar_wait(empty0 + 8 * s, par ^ 1)) {
                     timed_out = true;
                     break;
                 }
@@ -206,6 +207,10 @@ sparse_ffn_batch_kernel(const FfnBatchParams p, const int n_stages) {
                 bulk_load_row_hint(dst + row_bytes, Wu + off, row_bytes, bar, stream_policy);
                 bulk_load_row_hint(dst + 2 * row_bytes, Wd + off, row_bytes, bar, stream_policy);
                 issued = i + 1;
+                if (++s == n_stages) {
+                    s = 0;
+                    par ^= 1;
+                }
             }
             for (int i = max(0, issued - n_stages); i < issued; ++i)
                 if (!mbar_wait(full0 + 8 * (i % n_stages), (i / n_stages) & 1)) timed_out = true;
@@ -221,18 +226,26 @@ sparse_ffn_batch_kernel(const FfnBatchParams p, const int n_stages) {
                 for (int e = 0; e < P; ++e) acc[b][i][e] = make_float2(0.f, 0.f);
         const bool b16 = lane & 16, b8 = lane & 8, b4 = lane & 4, b2 = lane & 2;
         int buf = 0;
+        int cs = 0;           // ring position of the next neuron to consume, and the parity of its use
+        uint32_t cpar = 0;
         for (int g0 = 0; g0 < my_n; g0 += GB, buf ^= 1) {
             float pd[16];  // value (g * BT + b) * 2 + {0: gate, 1: up}
             uint32_t st_addr[GB];
+            int st_idx[GB];
 #pragma unroll
             for (int g = 0; g < GB; ++g) {
                 const int i = g0 + g;
                 float2 sg[BT], su[BT];
 #pragma unroll
                 for (int b = 0; b < BT; ++b) sg[b] = su[b] = make_float2(0.f, 0.f);
-                st_addr[g] = ring + (uint32_t)(i % n_stages) * stage_bytes;
+                st_idx[g] = cs;
+                st_addr[g] = ring + (uint32_t)cs * stage_bytes;
                 if (i < my_n) {
-                    if (!timed_out && !mbar_wait(full0 + 8 * (i % n_stages), (i / n_stages) & 1)) timed_out = true;
+                    if (!timed_out && !mbar_wait(full0 + 8 * cs, cpar)) timed_out = true;
+                    if (++cs == n_stages) {
+                        cs = 0;
+                        cpar ^= 1;
+                    }
 #pragma unroll
                     for (int k = 0; k < NV; ++k) {
                         if (!vok[k]) continue;
@@ -295,25 +308,28 @@ sparse_ffn_batch_kernel(const FfnBatchParams p, const int n_stages) {
                 for (int b = 0; b < BT; ++b) h[b] = __shfl_sync(0xffffffffu, hval, 4 * (g * BT + b));
                 if (g0 + g >= my_n) continue;
                 const int bits = s_keep[g0 + g];
+                float2 h2[BT];
+#pragma unroll
+                for (int b = 0; b < BT; ++b) {
+                    const float hb = ((bits >> b) & 1) ? h[b] : 0.f;  // not kept by sequence b: no contribution
+                    h2[b] = make_float2(hb, hb);
+                }
 #pragma unroll
                 for (int k = 0; k < NV; ++k) {
                     if (!vok[k]) continue;
                     float2 fd[P];
                     Pairs<T>::unpack(lds128(st_addr[g] + 2 * row_bytes + (uint32_t)(tid + k * kConsumers) * 16u), fd);
 #pragma unroll
-                    for (int b = 0; b < BT; ++b) {
-                        const float hb = ((bits >> b) & 1) ? h[b] : 0.f;  // not kept by sequence b: no contribution
-                        const float2 h2 = make_float2(hb, hb);
+                    for (int b = 0; b < BT; ++b)
 #pragma unroll
-                        for (int e = 0; e < P; ++e) acc[b][k][e] = __ffma2_rn(h2, fd[e], acc[b][k][e]);
-                    }
+                        for (int e = 0; e < P; ++e) acc[b][k][e] = __ffma2_rn(h2[b], fd[e], acc[b][k][e]);
                 }
             }
             __syncwarp();
             if (lane == 0) {
 #pragma unroll
                 for (int g = 0; g < GB; ++g)
-                    if (g0 + g < my_n) mbar_arrive(empty0 + 8 * ((g0 + g) % n_stages));
+                    if (g0 + g < my_n) mbar_arrive(empty0 + 8 * st_idx[g]);
             }
         }
 #pragma unroll
