@@ -146,41 +146,56 @@ cogload_kernel(const T *__restrict__ logits, int64_t V, int64_t row_stride,
     if (bad) atomicOr(&s_bad, 1);
     if ((tid & 31) == 0) s_stat[tid >> 5] = st;
     __syncthreads();
-    if (tid == 0) {
-        SoftStat tot = s_stat[0];
-        for (int w = 1; w < kCogThreads / kWarp; ++w) tot = stat_merge(tot, s_stat[w]);
+    if (tid < kWarp) {  // warp 0 merges the 16 warp statistics by butterfly (same bits on every lane)
+        SoftStat tot = tid < kCogThreads / kWarp ? s_stat[tid] : stat_empty();
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            SoftStat other;
+            other.m = __shfl_xor_sync(0xffffffffu, tot.m, o);
+            other.z = __shfl_xor_sync(0xffffffffu, tot.z, o);
+            other.w = __shfl_xor_sync(0xffffffffu, tot.w, o);
+            tot = ((tid & o) == 0) ? stat_merge(tot, other) : stat_merge(other, tot);
+        }
         if (s_bad) tot.z = NAN;  // carries the non-finite flag to rank 0
-        s_slice = tot;
+        if (tid == 0) s_slice = tot;
     }
     cluster.sync();
     if (slice == 0) {
-        if (tid == 0) {
-            SoftStat tot = s_slice;
-            for (int r = 1; r < n_slices; ++r) {
-                const SoftStat *remote = cluster.map_shared_rank(&s_slice, r);
-                tot = stat_merge(tot, *remote);
+        if (tid < kWarp) {
+            // lane r fetches slice r's statistic over distributed shared memory, then a butterfly merges them
+            SoftStat tot = stat_empty();
+            if (tid < n_slices) tot = *cluster.map_shared_rank(&s_slice, tid);
+#pragma unroll
+            for (int o = kCogMaxCluster / 2; o > 0; o >>= 1) {
+                SoftStat other;
+                other.m = __shfl_xor_sync(0xffffffffu, tot.m, o);
+                other.z = __shfl_xor_sync(0xffffffffu, tot.z, o);
+                other.w = __shfl_xor_sync(0xffffffffu, tot.w, o);
+                tot = ((tid & o) == 0) ? stat_merge(tot, other) : stat_merge(other, tot);
             }
-            int flags = 0;
-            float s, h;
-            if (!(tot.z > 0.f)) {  // a +inf / NaN logit (z is NaN), or no finite logit at all
-                flags |= CLADA_STATUS_NONFINITE_LOGIT;
-                s = h = NAN;
-            } else {
-                const float logz = logf(tot.z);
-                h = logz - tot.w / tot.z;
-                const int32_t tok = token_id[b];
-                if (tok < 0 || tok >= V) {
-                    flags |= CLADA_STATUS_BAD_TOKEN;
-                    s = NAN;
+            if (tid == 0) {
+                int flags = 0;
+                float s, h;
+                if (!(tot.z > 0.f)) {  // a +inf / NaN logit (z is NaN), or no finite logit at all
+                    flags |= CLADA_STATUS_NONFINITE_LOGIT;
+                    s = h = NAN;
                 } else {
-                    s = (tot.m + logz) - load_logit(row, tok);
+                    const float logz = logf(tot.z);
+                    h = logz - tot.w / tot.z;
+                    const int32_t tok = token_id[b];
+                    if (tok < 0 || tok >= V) {
+                        flags |= CLADA_STATUS_BAD_TOKEN;
+                        s = NAN;
+                    } else {
+                        s = (tot.m + logz) - load_logit(row, tok);
+                    }
                 }
+                surprisal[b] = s;
+                entropy[b] = h;
+                s_out[0] = s;
+                s_out[1] = h;
+                if (flags && status) atomicOr(status, flags);
             }
-            surprisal[b] = s;
-            entropy[b] = h;
-            s_out[0] = s;
-            s_out[1] = h;
-            if (flags && status) atomicOr(status, flags);
         }
         if (tau_base != nullptr) {
             __syncthreads();

@@ -200,6 +200,19 @@ sparse_ffn_kernel(const FfnParams p, const int n_stages) {
     }
     if (p.count_out && cta == 0 && tid == 0) *p.count_out = n_act;
     const int my_n = r1 - r0;
+    if (n_act == 0) {
+        // Nothing is kept (every CTA sees the same count): y = 0, written slice by slice, and there are
+        // no partial sums to combine, so the grid barrier is skipped as well.
+        const int ng = d / 4;  // output in groups of 4 columns
+        const int q0 = (int)(((int64_t)ng * cta) / n_ctas), q1 = (int)(((int64_t)ng * (cta + 1)) / n_ctas);
+        for (int q = q0 + tid; q < q1; q += kFfnThreads) {
+            if (p.y_dtype == CLADA_F32)
+                reinterpret_cast<float4 *>(p.y)[q] = make_float4(0.f, 0.f, 0.f, 0.f);
+            else
+                reinterpret_cast<uint2 *>(p.y)[q] = make_uint2(0u, 0u);
+        }
+        return;
+    }
     __syncthreads();  // s_list and the mbarriers are ready
 
     bool timed_out = false;

@@ -140,9 +140,34 @@ __global__ void guard_candidates_kernel(const float *__restrict__ scores, int B,
 
 constexpr int kRefThreads = 1024;
 
-// One CTA per candidate (grid-stride).  The candidate's gate and up rows sit in shared memory; each of
-// the 32 warps takes every 32nd token of the prompt, lanes split d_model by 16-byte vectors, products
-// and sums in fp64.  Warp and CTA sums are taken in a fixed order.
+// A 16-byte vector widened to fp64 (exact).  For bf16 the double is assembled from the bit fields with
+// integer operations: converting through the float-to-double instruction runs at a sixteenth of the ALU
+// rate and was the guard band's bottleneck.  Zeros, denormals, inf and NaN take the conversion.
+template <typename T> struct Widen;
+template <> struct Widen<float> {
+    __device__ static __forceinline__ void run(const uint4 &v, double (&o)[4]) {
+        o[0] = (double)__uint_as_float(v.x); o[1] = (double)__uint_as_float(v.y);
+        o[2] = (double)__uint_as_float(v.z); o[3] = (double)__uint_as_float(v.w);
+    }
+};
+__device__ __forceinline__ double bf16_bits_to_double(uint32_t b) {  // b: 16 significant bits
+    const uint32_t ex = (b >> 7) & 0xffu;
+    if (ex == 0u || ex == 255u) return (double)__uint_as_float(b << 16);
+    const uint32_t hi = ((b & 0x8000u) << 16) | ((ex + 896u) << 20) | ((b & 0x7fu) << 13);
+    return __hiloint2double((int)hi, 0);
+}
+template <> struct Widen<__nv_bfloat16> {
+    __device__ static __forceinline__ void run(const uint4 &v, double (&o)[8]) {
+        o[0] = bf16_bits_to_double(v.x & 0xffffu); o[1] = bf16_bits_to_double(v.x >> 16);
+        o[2] = bf16_bits_to_double(v.y & 0xffffu); o[3] = bf16_bits_to_double(v.y >> 16);
+        o[4] = bf16_bits_to_double(v.z & 0xffffu); o[5] = bf16_bits_to_double(v.z >> 16);
+        o[6] = bf16_bits_to_double(v.w & 0xffffu); o[7] = bf16_bits_to_double(v.w >> 16);
+    }
+};
+
+// One CTA per candidate (grid-stride).  The candidate's gate and up rows are widened to fp64 once into
+// shared memory; each of the 32 warps takes every 32nd token of the prompt, lanes split d_model by
+// 16-byte vectors, products and sums in fp64.  Warp and CTA sums are taken in a fixed order.
 template <typename T>
 __global__ void __launch_bounds__(kRefThreads)
 guard_refine_kernel(const T *__restrict__ X, const T *__restrict__ Wg, const T *__restrict__ Wu,
@@ -151,7 +176,7 @@ guard_refine_kernel(const T *__restrict__ X, const T *__restrict__ Wg, const T *
                     float *__restrict__ scores) {
     constexpr int E = Elem<T>::kPerVec;
     constexpr int kWarps = kRefThreads / kWarp;
-    extern __shared__ uint4 s_rows[];  // gate row | up row
+    extern __shared__ __align__(16) double s_rows[];  // gate row | up row, fp64
     __shared__ double s_zz[kWarps];
     __shared__ double s_nn[kWarps];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -163,8 +188,14 @@ guard_refine_kernel(const T *__restrict__ X, const T *__restrict__ Wg, const T *
         const uint4 *wu = reinterpret_cast<const uint4 *>(Wu + (size_t)j * d_model);
         const uint4 *wd = reinterpret_cast<const uint4 *>(Wd_t + (size_t)j * d_model);
         for (int v = threadIdx.x; v < vpr; v += kRefThreads) {
-            s_rows[v] = wg[v];
-            s_rows[vpr + v] = wu[v];
+            double g[E], u[E];
+            Widen<T>::run(wg[v], g);
+            Widen<T>::run(wu[v], u);
+#pragma unroll
+            for (int e = 0; e < E; ++e) {
+                s_rows[v * E + e] = g[e];
+                s_rows[d_model + v * E + e] = u[e];
+            }
         }
         __syncthreads();
         double zz = 0.0;
@@ -172,14 +203,12 @@ guard_refine_kernel(const T *__restrict__ X, const T *__restrict__ Wg, const T *
             const uint4 *x = reinterpret_cast<const uint4 *>(X + (size_t)t * d_model);
             double g = 0.0, u = 0.0;
             for (int v = lane; v < vpr; v += kWarp) {
-                float fx[E], fg[E], fu[E];
-                Elem<T>::unpack(x[v], fx);
-                Elem<T>::unpack(s_rows[v], fg);
-                Elem<T>::unpack(s_rows[vpr + v], fu);
+                double fx[E];
+                Widen<T>::run(x[v], fx);
 #pragma unroll
                 for (int e = 0; e < E; ++e) {
-                    g = fma((double)fg[e], (double)fx[e], g);
-                    u = fma((double)fu[e], (double)fx[e], u);
+                    g = fma(s_rows[v * E + e], fx[e], g);
+                    u = fma(s_rows[d_model + v * E + e], fx[e], u);
                 }
             }
             g = warp_sum(g);
@@ -189,10 +218,10 @@ guard_refine_kernel(const T *__restrict__ X, const T *__restrict__ Wg, const T *
         }
         double nn = 0.0;
         for (int v = threadIdx.x; v < vpr; v += kRefThreads) {
-            float fd[E];
-            Elem<T>::unpack(wd[v], fd);
+            double fd[E];
+            Widen<T>::run(wd[v], fd);
 #pragma unroll
-            for (int e = 0; e < E; ++e) nn = fma((double)fd[e], (double)fd[e], nn);
+            for (int e = 0; e < E; ++e) nn = fma(fd[e], fd[e], nn);
         }
         nn = warp_sum(nn);
         if (lane == 0) {
@@ -316,7 +345,16 @@ int clada_refine_scores(const clada_layer *layer, const void *X, const int64_t *
     rc = device_info(&di);
     if (rc != CLADA_OK) return rc;
     const int grid = di.num_sms;
-    const size_t rows_smem = 2 * (size_t)layer->d_model * elem_size(layer->dtype);
+    const size_t rows_smem = 2 * (size_t)layer->d_model * sizeof(double);
+    static bool configured[64] = {};
+    if (!configured[di.device & 63]) {  // up to 128 KB of dynamic shared memory
+        CLADA_CUDA_TRY(cudaFuncSetAttribute(guard_refine_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                            2 * kMaxDModel * (int)sizeof(double)));
+        CLADA_CUDA_TRY(cudaFuncSetAttribute(guard_refine_kernel<__nv_bfloat16>,
+                                            cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                            2 * kMaxDModel * (int)sizeof(double)));
+        configured[di.device & 63] = true;
+    }
     if (layer->dtype == CLADA_F32)
         guard_refine_kernel<float><<<grid, kRefThreads, rows_smem, st>>>(
             static_cast<const float *>(X), static_cast<const float *>(layer->w_gate),
