@@ -192,9 +192,9 @@ guard_refine_kernel(const T *__restrict__ X, const T *__restrict__ Wg, const T *
             Widen<T>::run(wg[v], g);
             Widen<T>::run(wu[v], u);
 #pragma unroll
-            for (int e = 0; e < E; ++e) {
-                s_rows[v * E + e] = g[e];
-                s_rows[d_model + v * E + e] = u[e];
+            for (int e = 0; e < E; ++e) {  // element-major: lanes then read consecutive doubles
+                s_rows[e * vpr + v] = g[e];
+                s_rows[d_model + e * vpr + v] = u[e];
             }
         }
         __syncthreads();
@@ -202,13 +202,14 @@ guard_refine_kernel(const T *__restrict__ X, const T *__restrict__ Wg, const T *
         for (long long t = tab.off[b] + warp; t < tab.off[b + 1]; t += kWarps) {
             const uint4 *x = reinterpret_cast<const uint4 *>(X + (size_t)t * d_model);
             double g = 0.0, u = 0.0;
-            for (int v = lane; v < vpr; v += kWarp) {
+#pragma unroll 4
+            for (int v = lane; v < vpr; v += kWarp) {  // four independent 16-byte loads in flight
                 double fx[E];
                 Widen<T>::run(x[v], fx);
 #pragma unroll
                 for (int e = 0; e < E; ++e) {
-                    g = fma(s_rows[v * E + e], fx[e], g);
-                    u = fma(s_rows[d_model + v * E + e], fx[e], u);
+                    g = fma(s_rows[e * vpr + v], fx[e], g);
+                    u = fma(s_rows[d_model + e * vpr + v], fx[e], u);
                 }
             }
             g = warp_sum(g);
