@@ -8,7 +8,7 @@ One step = one pass of the whole path over one batch of synthetic input:
 The layer exists in several identical copies at different addresses and decode step t reads copy
 t mod n, so that no step can be served from L2 (one copy's kept rows are 135-162 MB, L2 is 126 MB).
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--no-graph]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--no-graph] [--workload NAME]
 
 Prints ONE JSON line (rank 0).  `--impl reference` times the CPU oracle on a bounded sample.
 """
@@ -184,11 +184,120 @@ class Job:
                 tot += int(cnt.item())
         return tot / self.tokens_per_step()
 
+    ffn_launches_per_loop = property(lambda self: self.N)
+    prefix_flop = property(lambda self: 4.0 * self.T * self.w.d_model * self.w.d_ff)
+    l2_note = f"inputs larger than L2: {N_COPIES} rotating copies of the layer"
+    step_note = "prefix statistics + per sparsity (guard band, select, 128 x (cogload+adjust, sparse FFN))"
+
+    def prefix_once(self):
+        self.clada.clada_prefix_scores(self.layers[0], self.X, self.off, self.scores, self.ws, self.status)
+
+    def io_tensors(self):
+        return [self.X, self.xs, self.logits, self.tokens], self.y
+
     def ffn_only_loop(self):
         """The FFN launches of one sparsity level back to back (for the kernel's own duration)."""
         for t in range(self.N):
             self.clada.clada_sparse_ffn_decode(self.layers[t % N_COPIES], self.xs[t:t + 1], self.scores,
                                                self.tau_base[0], 1, self.y[0, t:t + 1], self.ws)
+
+
+class StackJob:
+    """A whole FFN stack (workload c3: 32 Llama-2-7B-shaped layers, one sequence): per token one
+    cogload+adjust launch for all layers, then the native per-layer loop of the library."""
+
+    def __init__(self, clada, w, dev, rank: int):
+        self.clada, self.w, self.dev = clada, w, dev
+        L, T = w.n_layers, w.prefix_len[0]
+        self.L, self.T, self.N = L, T, w.n_decode
+        scale = wl.channel_scale(w, dev)
+        f32 = dict(dtype=torch.float32, device=dev)
+        self.layers, Xs, xs = [], [], []
+        for l in range(L):
+            wt = wl.layer_weights(w, l, dev)
+            lay = clada.Layer(wt["w_gate"], wt["w_up"], wt["w_down"].t().contiguous())
+            norms = torch.empty(w.d_ff, **f32)
+            clada.clada_down_norms(lay, norms)
+            lay.set_down_norm(norms)
+            self.layers.append(lay)
+            Xs.append(wl.hidden_states(w, l, "prefix", rank, T, dev, scale))
+            xs.append(wl.hidden_states(w, l, "decode", rank, self.N, dev, scale))
+        self.stack = clada.LayerStack(self.layers)
+        self.X = torch.stack(Xs)                                   # [L, T, d]
+        self.xs = torch.stack(xs, dim=1).unsqueeze(2).contiguous()  # [N, L, 1, d]
+        self.logits = wl.decode_logits(w, rank, self.N, dev)
+        self.tokens = wl.chosen_tokens(w, self.logits, rank).contiguous()
+        self.off = [0, T]
+        self.ws = clada.new_workspace(self.layers[0], 1, T)
+        self.scores = torch.empty(L, 1, w.d_ff, **f32)
+        self.mask = torch.empty(1, w.d_ff, dtype=torch.uint8, device=dev)
+        self.idx = torch.empty(1, w.d_ff, dtype=torch.int32, device=dev)
+        self.count = torch.empty(1, dtype=torch.int32, device=dev)
+        self.status = torch.zeros(1, dtype=torch.int32, device=dev)
+        self.lam = torch.full((L,), LAMBDA, **f32)
+        self.gam = torch.full((L,), GAMMA, **f32)
+        self.s = torch.empty(self.N, **f32)
+        self.h = torch.empty(self.N, **f32)
+        self.tau_final = torch.empty(1, L, **f32)
+        self.tau_base = torch.empty(1, L, **f32)
+        self.y = torch.empty(self.N, L, 1, w.d_model, **f32)
+        self.guard = [1.0, 1.0 + LAMBDA, 1.0 + GAMMA, 1.0 + LAMBDA + GAMMA]
+        self.rho = w.sparsities[0]
+        for l in range(L):   # calibration, outside the step
+            clada.clada_prefix_scores(self.layers[l], self.X[l], self.off, self.scores[l], self.ws)
+            clada.clada_tau_from_sparsity(self.scores[l], self.rho, self.tau_base[:, l])
+        clada.clada_cogload(self.logits, self.tokens, self.s, self.h)
+        torch.cuda.synchronize()
+        self.tau_s = wl.universal_threshold(self.s.tolist())
+        self.tau_H = wl.universal_threshold(self.h.tolist())
+
+    ffn_launches_per_loop = property(lambda self: self.L * 8)
+    prefix_flop = property(lambda self: 4.0 * self.T * self.w.d_model * self.w.d_ff)
+    l2_note = "inputs larger than L2: 32 layers, 8.7 GB of weights per token"
+    step_note = "per layer: prefix statistics, guard band, select; then 256 x (cogload+adjust for 32 layers, 32 sparse FFNs)"
+
+    def step(self):
+        c = self.clada
+        for l in range(self.L):
+            c.clada_prefix_select(self.layers[l], self.X[l], self.off, self.tau_base[:, l].contiguous(), self.guard,
+                                  self.scores[l], self.mask, self.idx, self.count, self.ws, self.status)
+        for t in range(self.N):
+            c.clada_cogload_adjust(self.logits[t:t + 1], self.tokens[t:t + 1], self.tau_base, self.lam, self.gam,
+                                   self.tau_s, self.tau_H, self.s[t:t + 1], self.h[t:t + 1], self.tau_final, self.status)
+            c.clada_sparse_ffn_decode_layers(self.stack, self.xs[t], self.scores, self.tau_final, self.y[t], self.ws,
+                                             self.status)
+
+    @property
+    def launches_per_step(self) -> int:
+        return self.L * 6 + self.N * (1 + self.L)
+
+    def tokens_per_step(self) -> int:
+        return self.N
+
+    def kept_per_token(self):
+        """Average kept neurons per (token, layer) over the step."""
+        c = self.clada
+        cnt = torch.empty(1, dtype=torch.int32, device=self.dev)
+        tot, n = 0, 0
+        for t in range(0, self.N, 8):
+            c.clada_cogload_adjust(self.logits[t:t + 1], self.tokens[t:t + 1], self.tau_base, self.lam, self.gam,
+                                   self.tau_s, self.tau_H, self.s[t:t + 1], self.h[t:t + 1], self.tau_final)
+            for l in (0, self.L // 2, self.L - 1):
+                c.clada_select(self.scores[l], self.tau_final[:, l].contiguous(), 1, None, None, cnt)
+                tot += int(cnt.item())
+                n += 1
+        return tot / n
+
+    def prefix_once(self):
+        self.clada.clada_prefix_scores(self.layers[0], self.X[0], self.off, self.scores[0], self.ws, self.status)
+
+    def io_tensors(self):
+        return [self.X, self.xs, self.logits, self.tokens], self.y
+
+    def ffn_only_loop(self):
+        """Eight tokens x 32 layers at the baseline thresholds."""
+        for t in range(8):
+            self.clada.clada_sparse_ffn_decode_layers(self.stack, self.xs[t], self.scores, self.tau_base, self.y[t], self.ws)
 
 
 def _timed(fn, steps, dist_barrier):
@@ -224,8 +333,8 @@ def run_ours(args):
         build.build()
     barrier()
     clada.load()
-    w = wl.WORKLOADS[WORKLOAD]
-    job = Job(clada, w, dev, rank)
+    w = wl.WORKLOADS[args.workload]
+    job = (StackJob if w.n_layers > 1 else Job)(clada, w, dev, rank)
 
     stream = torch.cuda.Stream()
     graph = None
@@ -258,25 +367,24 @@ def run_ours(args):
                 job.ffn_only_loop()
             ffn_run = ffn_graph.replay
         ffn_run()
-        ffn_ms = _timed(ffn_run, 5, lambda: None) / (5 * job.N)
+        ffn_ms = _timed(ffn_run, 5, lambda: None) / (5 * job.ffn_launches_per_loop)
         # the prefix statistics alone (tensor-core contraction), for its own roofline line
-        pf = lambda: clada.clada_prefix_scores(job.layers[0], job.X, job.off, job.scores, job.ws, job.status)
+        pf = job.prefix_once
         pf()
         prefix_ms = _timed(pf, 10, lambda: None) / 10
         kept = job.kept_per_token()
         kept_base = w.d_ff - w.k_cut(w.sparsities[0])
 
         # end to end: inputs start in pinned host memory, outputs end there
-        hX, hxs, hlog, htok = (t.cpu().pin_memory() for t in (job.X, job.xs, job.logits, job.tokens))
-        hy = torch.empty(job.y.shape, dtype=job.y.dtype).pin_memory()
+        dev_in, dev_out = job.io_tensors()
+        host_in = [t.cpu().pin_memory() for t in dev_in]
+        hy = torch.empty(dev_out.shape, dtype=dev_out.dtype).pin_memory()
 
         def e2e_step():
-            job.X.copy_(hX, non_blocking=True)
-            job.xs.copy_(hxs, non_blocking=True)
-            job.logits.copy_(hlog, non_blocking=True)
-            job.tokens.copy_(htok, non_blocking=True)
+            for dt, ht in zip(dev_in, host_in):
+                dt.copy_(ht, non_blocking=True)
             run()
-            hy.copy_(job.y, non_blocking=True)
+            hy.copy_(dev_out, non_blocking=True)
 
         e2e_step()
         e2e_ms = _timed(e2e_step, args.steps, barrier)
@@ -288,7 +396,7 @@ def run_ours(args):
     e2e_value, e2e_ms = sharding.whole_job_rate(tokens_rank, e2e_ms, dev)
 
     peak, peak_kind = _peaks()
-    prefix_flop = 4.0 * job.T * w.d_model * w.d_ff
+    prefix_flop = job.prefix_flop
     try:
         with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
             bf16_peak = float(json.load(f)["bf16_tflops"])
@@ -299,18 +407,17 @@ def run_ours(args):
     # algorithmic bytes of one FFN launch: three rows per kept neuron + scores + x in + y out
     ffn_bytes = kept_base * 3 * w.d_model * eb + w.d_ff * 4 + w.d_model * eb + w.d_model * 4
     achieved = ffn_bytes / (ffn_ms * 1e-3) / 1e9
-    h2d = sum(x.numel() * x.element_size() for x in (hX, hxs, hlog, htok))
+    h2d = sum(x.numel() * x.element_size() for x in host_in)
     d2h = hy.numel() * hy.element_size()
 
     line = {
         "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": WORKLOAD, "d_model": w.d_model, "d_ff": w.d_ff, "prefix_tokens": job.T,
+        "config": {"workload": w.name, "d_model": w.d_model, "d_ff": w.d_ff, "layers": w.n_layers, "prefix_tokens": job.T,
                    "decode_tokens_per_sparsity": job.N, "sparsities": list(w.sparsities), "batch": 1,
-                   "l2": f"inputs larger than L2: {N_COPIES} rotating copies of the layer",
-                   "cuda_graph": bool(args.graph), "avg_kept_neurons_per_token": kept,
-                   "step": "prefix statistics + per sparsity (guard band, select, 128 x (cogload+adjust, sparse FFN))"},
+                   "l2": job.l2_note, "cuda_graph": bool(args.graph), "avg_kept_neurons_per_token": kept,
+                   "step": job.step_note},
         "e2e": {"value": e2e_value, "unit": "tokens/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
         "gpu_launches": job.launches_per_step * args.steps,
         "roofline": {"bound": "hbm", "kernel": "sparse_ffn_kernel", "achieved": achieved, "peak": peak,
@@ -324,7 +431,7 @@ def run_ours(args):
         "clocks": clocks, "device_status_word": status,
     }
     if rank == 0:
-        if world == 1:
+        if world == 1 and w.name == WORKLOAD:
             line["cpu_baseline"] = cpu_baseline(w)
         print(json.dumps(line), flush=True)
     if world > 1:
@@ -422,6 +529,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-graph", dest="graph", action="store_false")
+    ap.add_argument("--workload", default=WORKLOAD, choices=[WORKLOAD, "c3_llama2_7b_stack"],
+                    help="the metric's workload (default), or the 32-layer stack for information")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

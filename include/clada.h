@@ -193,6 +193,20 @@ int clada_sparse_ffn_decode(const clada_layer *layer, const void *x, int32_t B,
                             uint8_t *mask_out, int32_t *idx_out, int32_t *count_out,
                             void *ws, size_t ws_bytes, int32_t *status, void *stream);
 
+/* Algorithm 2's sparse forward pass over a stack of L layers for one decode
+ * step: clada_sparse_ffn_decode for l = 0 .. L-1 in one call.
+ *   layers     HOST array of L layers of one shape and dtype
+ *   x          [L, B, d_model]: the input hidden state of every layer (this path has
+ *              no attention, residual or norm between FFNs, so each layer's input is given)
+ *   scores     [L, B, d_ff]
+ *   tau_final  [B, L] as clada_adjust_threshold writes it
+ *   y          out [L, B, d_model]
+ * All layers are validated before anything is enqueued. */
+int clada_sparse_ffn_decode_layers(const clada_layer *layers, int32_t L, const void *x, int32_t B,
+                                   const float *scores, const float *tau_final, void *y,
+                                   int32_t y_dtype, void *ws, size_t ws_bytes, int32_t *status,
+                                   void *stream);
+
 /* clada_sparse_ffn_decode for callers that cannot allocate device memory (the
  * paper has no counterpart; this is a deployment variant of the call above).
  * Think of a plug-in that runs inside another engine's execution step, where

@@ -23,7 +23,7 @@ _INT_RETURNING = [
     "clada_workspace_init", "clada_down_norms", "clada_prefix_scores", "clada_refine_scores",
     "clada_select", "clada_prefix_select", "clada_tau_from_sparsity", "clada_cogload",
     "clada_adjust_threshold", "clada_cogload_adjust", "clada_sparse_ffn_decode",
-    "clada_sparse_ffn_decode_static",
+    "clada_sparse_ffn_decode_static", "clada_sparse_ffn_decode_layers",
 ]
 
 
@@ -69,6 +69,7 @@ def load() -> ctypes.CDLL:
     L.clada_cogload_adjust.argtypes = [vp, i32, i32, i64, i64, vp, vp, vp, vp, f32, f32, i32, vp, vp, vp, vp, vp]
     L.clada_sparse_ffn_decode.argtypes = [lp, vp, i32, vp, vp, i64, vp, i32, vp, vp, vp, vp, sz, vp, vp]
     L.clada_sparse_ffn_decode_static.argtypes = [lp, vp, i32, vp, vp, i64, vp, i32, vp, vp, vp, vp, vp]
+    L.clada_sparse_ffn_decode_layers.argtypes = [vp, i32, vp, i32, vp, vp, vp, i32, vp, sz, vp, vp]
     for name in _INT_RETURNING:
         getattr(L, name).restype = ctypes.c_int
     _lib = L
@@ -300,3 +301,27 @@ def clada_sparse_ffn_decode_static(layer: Layer, x, scores, tau_final, tau_strid
                                                  _ptr(count_out, torch.int32, "count_out"),
                                                  _ptr(status, torch.int32, "status"), _stream(stream)),
            "clada_sparse_ffn_decode_static")
+
+
+class LayerStack:
+    """L layers of one shape as the contiguous host array clada_sparse_ffn_decode_layers takes."""
+
+    def __init__(self, layers):
+        self.layers = list(layers)
+        self.array = (_CLayer * len(self.layers))(*[l.c for l in self.layers])
+
+    def __len__(self):
+        return len(self.layers)
+
+
+def clada_sparse_ffn_decode_layers(stack: LayerStack, x, scores, tau_final, y, ws, status=None, stream=None) -> None:
+    """x [L, B, d], scores [L, B, F], tau_final [B, L], y [L, B, d]."""
+    L, B = x.shape[0], x.shape[1]
+    if L != len(stack):
+        raise CladaError("x must have one [B, d_model] slab per layer")
+    _check(load().clada_sparse_ffn_decode_layers(ctypes.addressof(stack.array), L, _ptr(x, stack.layers[0].dtype, "x"), B,
+                                                 _ptr(scores, torch.float32, "scores"),
+                                                 _ptr(tau_final, torch.float32, "tau_final"), _ptr(y, name="y"),
+                                                 _dtype_code(y.dtype), _ptr(ws, torch.uint8, "ws"), ws.numel(),
+                                                 _ptr(status, torch.int32, "status"), _stream(stream)),
+           "clada_sparse_ffn_decode_layers")

@@ -522,6 +522,34 @@ extern "C" int clada_sparse_ffn_decode(const clada_layer *layer, const void *x, 
                                  count_out, ws, ws_bytes, status, stream);
 }
 
+// One decode step of a whole stack: the per-layer call in a native loop (one C call per token instead
+// of one per layer); the launches chain with programmatic dependent launch.
+extern "C" int clada_sparse_ffn_decode_layers(const clada_layer *layers, int32_t L, const void *x, int32_t B,
+                                              const float *scores, const float *tau_final, void *y,
+                                              int32_t y_dtype, void *ws, size_t ws_bytes, int32_t *status,
+                                              void *stream) {
+    if (!layers || !x || !scores || !tau_final || !y) return CLADA_ERR_NULL;
+    if (L <= 0 || B <= 0) return CLADA_ERR_SHAPE;
+    if (y_dtype != CLADA_F32 && y_dtype != CLADA_BF16) return CLADA_ERR_DTYPE;
+    for (int l = 0; l < L; ++l) {  // validate everything before enqueueing anything
+        int rc = validate_layer(&layers[l], false);
+        if (rc != CLADA_OK) return rc;
+        if (layers[l].d_model != layers[0].d_model || layers[l].d_ff != layers[0].d_ff ||
+            layers[l].dtype != layers[0].dtype)
+            return CLADA_ERR_SHAPE;
+    }
+    const size_t d = (size_t)layers[0].d_model, F = (size_t)layers[0].d_ff;
+    const size_t x_layer = (size_t)B * d * elem_size(layers[0].dtype), y_layer = (size_t)B * d * elem_size(y_dtype);
+    for (int l = 0; l < L; ++l) {
+        int rc = decode_with_workspace(&layers[l], static_cast<const char *>(x) + l * x_layer, B,
+                                       scores + (size_t)l * B * F, tau_final + l, L,
+                                       static_cast<char *>(y) + l * y_layer, y_dtype, nullptr, nullptr, nullptr, ws,
+                                       ws_bytes, status, stream);
+        if (rc != CLADA_OK) return rc;
+    }
+    return CLADA_OK;
+}
+
 // ---- the entry point that allocates nothing ---------------------------------------------------
 //
 // Some callers may not allocate device memory at all: a plug-in that runs inside another engine's

@@ -515,3 +515,28 @@ def test_sparse_ffn_batched_tiles(clada, oracle, name, d, F, B):
         clada.clada_sparse_ffn_decode(layer, xs.cuda(), _dev(scores), _dev(taus), 1, y2, ws)
         torch.cuda.synchronize()
         assert torch.equal(y, y2)
+
+
+def test_decode_layers_equals_per_layer_calls(clada):
+    """The stack call is the per-layer call in a loop: same bits, with tau_final read at stride L."""
+    L, B = 3, 2
+    w = _small("c3_llama2_7b_stack", d_model=1024, d_ff=900, batch=B)
+    layers = [gpu_layer(wl.layer_weights(w, l), clada) for l in range(L)]
+    stack = clada.LayerStack(layers)
+    ws = clada.new_workspace(layers[0], B, 0)
+    g = torch.Generator(device="cuda").manual_seed(11)
+    scores = torch.rand(L, B, w.d_ff, generator=g, device="cuda") + 0.5
+    tau = torch.rand(B, L, generator=g, device="cuda") * 0.5 + 0.75
+    x = torch.stack([torch.stack([wl.hidden_states(w, l, "decode", b, 1)[0] for b in range(B)]) for l in range(L)]).cuda()
+    y_stack = torch.empty(L, B, w.d_model, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    clada.clada_sparse_ffn_decode_layers(stack, x, scores, tau, y_stack, ws, status)
+    y_ref = torch.empty_like(y_stack)
+    for l in range(L):
+        clada.clada_sparse_ffn_decode(layers[l], x[l], scores[l], tau[:, l], L, y_ref[l], ws)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0 and torch.equal(y_stack, y_ref)
+    assert float(y_stack.abs().max()) > 0
+    bad = clada.LayerStack([layers[0], gpu_layer(wl.layer_weights(_small("c3_llama2_7b_stack", d_model=1024, d_ff=800), 0), clada)])
+    with pytest.raises(clada.CladaError, match="shape"):
+        clada.clada_sparse_ffn_decode_layers(bad, x[:2], scores[:2], tau[:, :2].contiguous(), y_stack[:2], ws)
