@@ -33,6 +33,9 @@ WORKLOAD = "c2_llama2_7b_layer"
 METRIC = "sparse_ffn_decode_tokens_per_s"
 LAMBDA, GAMMA = 0.80, 0.12
 N_COPIES = 4
+# DRAM read + write bytes of one sparse_ffn_kernel launch at the baseline threshold of this workload, from the ncu
+# capture summarised in profiles/sparse_ffn_kernel_c2_full.md.  Must go back to None whenever that kernel changes.
+FFN_NCU_TRAFFIC_BYTES = 166.06e6
 
 
 def _peaks():
@@ -421,7 +424,8 @@ def run_ours(args):
         "e2e": {"value": e2e_value, "unit": "tokens/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
         "gpu_launches": job.launches_per_step * args.steps,
         "roofline": {"bound": "hbm", "kernel": "sparse_ffn_kernel", "achieved": achieved, "peak": peak,
-                     "unit": "GB/s", "frac": achieved / peak, "peak_kind": peak_kind, "traffic": None,
+                     "unit": "GB/s", "frac": achieved / peak, "peak_kind": peak_kind,
+                     "traffic": FFN_NCU_TRAFFIC_BYTES if w.name == WORKLOAD else None,
                      "bytes_per_launch": ffn_bytes, "us_per_launch": ffn_ms * 1e3,
                      "kept_neurons": kept_base},
         "prefix_roofline": {"bound": "tensor", "kernel": "prefix_tc_kernel (+finalize)", "ms": prefix_ms,
