@@ -293,3 +293,114 @@ float oracle_tau_from_sparsity(const float *scores, int d_ff, double rho)
     free(s);
     return mid;
 }
+
+/* ------------------------------------------------------------------ *
+ * Layer-wise base threshold (Eq. base_threshold), offline search.
+ *
+ *   tau_base = argmax eps  s.t.  E_{x in D_val}[ CETT(x; eps) ] <= bound,
+ *   CETT(x; eps) = || sum_{j in S_cut} n_j(x) ||_2 / || MLP(x) ||_2,   S_cut = { j : A_j(x) < eps }.
+ *
+ * A validation sample x is one sequence of T tokens; A_j(x) is its score of
+ * Eq. neuron_activation; n_j(x) is neuron j's contribution to the FFN output over
+ * all T tokens (a T x d_model matrix), MLP(x) the dense output, norms Frobenius.
+ *
+ * oracle_cett_curve: for ONE sample, cett[k] = CETT when exactly the k
+ * lowest-scored neurons are cut, k = 0 .. d_ff (cett[0] = 0, cett[d_ff] = 1),
+ * by accumulating the cut neurons' outputs in ascending score order (ties in
+ * index order).  Also returns the scores and that order.
+ * ------------------------------------------------------------------ */
+typedef struct { double a; int j; } or_pair;
+static int cmp_pair(const void *p, const void *q)
+{
+    const or_pair *x = (const or_pair *)p, *y = (const or_pair *)q;
+    if (x->a < y->a) return -1;
+    if (x->a > y->a) return 1;
+    return (x->j > y->j) - (x->j < y->j);
+}
+
+void oracle_cett_curve(int dtype, const void *X, int T, int d_model, int d_ff,
+                       const void *W_in, const void *V_in, const void *W_out,
+                       double *scores, int32_t *order, double *cett)
+{
+    double *z = (double *)malloc((size_t)T * d_ff * sizeof(double));      /* z[t, j] */
+    double *cut = (double *)calloc((size_t)T * d_model, sizeof(double));  /* running sum of cut outputs */
+    or_pair *pr = (or_pair *)malloc((size_t)d_ff * sizeof(or_pair));
+#pragma omp parallel for schedule(static)
+    for (int j = 0; j < d_ff; ++j) {
+        double wnorm2 = 0.0, zz = 0.0;
+        for (int i = 0; i < d_model; ++i) {
+            double w = elem(W_out, dtype, (size_t)i * d_ff + j);
+            wnorm2 += w * w;
+        }
+        for (int t = 0; t < T; ++t) {
+            double g = 0.0, u = 0.0;
+            for (int k = 0; k < d_model; ++k) {
+                double x = elem(X, dtype, (size_t)t * d_model + k);
+                g += elem(W_in, dtype, (size_t)j * d_model + k) * x;
+                u += elem(V_in, dtype, (size_t)j * d_model + k) * x;
+            }
+            double zt = silu(g) * u;
+            z[(size_t)t * d_ff + j] = zt;
+            zz += zt * zt;
+        }
+        scores[j] = sqrt(zz) * sqrt(wnorm2);
+        pr[j].a = scores[j];
+        pr[j].j = j;
+    }
+    qsort(pr, (size_t)d_ff, sizeof(or_pair), cmp_pair);
+    cett[0] = 0.0;
+    for (int k = 0; k < d_ff; ++k) {
+        const int j = pr[k].j;
+        order[k] = j;
+        double norm2 = 0.0;
+#pragma omp parallel for schedule(static) reduction(+ : norm2)
+        for (int t = 0; t < T; ++t) {
+            const double zt = z[(size_t)t * d_ff + j];
+            for (int i = 0; i < d_model; ++i) {
+                double *c = &cut[(size_t)t * d_model + i];
+                *c += zt * elem(W_out, dtype, (size_t)i * d_ff + j);
+                norm2 += (*c) * (*c);
+            }
+        }
+        cett[k + 1] = sqrt(norm2);  /* numerator; divided by the dense norm below */
+    }
+    const double dense = cett[d_ff];  /* all neurons cut = the dense output */
+    for (int k = 1; k <= d_ff; ++k)
+        cett[k] = dense > 0.0 ? cett[k] / dense : 0.0;
+    free(z);
+    free(cut);
+    free(pr);
+}
+
+/* The search itself, given every sample's scores [B, d_ff] and curve [B, d_ff+1]:
+ * CETT(x; eps) is constant between consecutive scores of x, so the candidates
+ * are the scores of all samples; the answer is the largest candidate whose mean
+ * CETT over the samples is within the bound.  The smallest score of all always
+ * qualifies (nothing is cut).  mean_out receives the mean CETT at the answer. */
+double oracle_threshold_search(const double *scores, const double *cett, int B, int d_ff,
+                               double bound, double *mean_out)
+{
+    double *sorted = (double *)malloc((size_t)B * d_ff * sizeof(double));
+    for (int b = 0; b < B; ++b) {
+        or_pair *pr = (or_pair *)malloc((size_t)d_ff * sizeof(or_pair));
+        for (int j = 0; j < d_ff; ++j) { pr[j].a = scores[(size_t)b * d_ff + j]; pr[j].j = j; }
+        qsort(pr, (size_t)d_ff, sizeof(or_pair), cmp_pair);
+        for (int j = 0; j < d_ff; ++j) sorted[(size_t)b * d_ff + j] = pr[j].a;
+        free(pr);
+    }
+    double best = -1.0, best_mean = 0.0;
+    for (size_t c = 0; c < (size_t)B * d_ff; ++c) {
+        const double eps = scores[c];
+        double mean = 0.0;
+        for (int b = 0; b < B; ++b) {
+            int k = 0;  /* neurons of sample b with score < eps */
+            while (k < d_ff && sorted[(size_t)b * d_ff + k] < eps) ++k;
+            mean += cett[(size_t)b * (d_ff + 1) + k];
+        }
+        mean /= B;
+        if (mean <= bound && eps > best) { best = eps; best_mean = mean; }
+    }
+    if (mean_out) *mean_out = best_mean;
+    free(sorted);
+    return best;
+}

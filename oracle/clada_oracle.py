@@ -52,6 +52,10 @@ def lib():
         L.oracle_sparse_ffn.restype = ctypes.c_int
         L.oracle_dense_ffn.argtypes = [i32, vp, i32, i32, vp, vp, vp, vp]
         L.oracle_dense_ffn.restype = None
+        L.oracle_cett_curve.argtypes = [i32, vp, i32, i32, i32, vp, vp, vp, vp, vp, vp]
+        L.oracle_cett_curve.restype = None
+        L.oracle_threshold_search.argtypes = [vp, vp, i32, i32, dbl, vp]
+        L.oracle_threshold_search.restype = dbl
         L.oracle_tau_from_sparsity.argtypes = [vp, i32, dbl]
         L.oracle_tau_from_sparsity.restype = f32
         _lib = L
@@ -170,3 +174,27 @@ def tau_from_sparsity(scores_f32, rho) -> np.float32:
     """Harness helper: fp32 midpoint threshold that cuts floor(rho*F + 0.5) neurons of an fp32 score vector."""
     s = _c(scores_f32, np.float32)
     return np.float32(lib().oracle_tau_from_sparsity(_p(s), s.size, float(rho)))
+
+
+def cett_curve(X, W_in, V_in, W_out):
+    """For one validation sample X [T, d_model]: (scores [d_ff], order int32 [d_ff] ascending by score,
+    cett [d_ff + 1]) with cett[k] = CETT of Eq. base_threshold when the k lowest-scored neurons are cut."""
+    X, W_in, V_in, W_out = _c(X), _c(W_in), _c(V_in), _c(W_out)
+    d_model, d_ff = _check_weights(X, W_in, V_in, W_out)
+    scores = np.empty(d_ff, dtype=np.float64)
+    order = np.empty(d_ff, dtype=np.int32)
+    cett = np.empty(d_ff + 1, dtype=np.float64)
+    lib().oracle_cett_curve(_dt(X), _p(X), X.shape[0], d_model, d_ff, _p(W_in), _p(V_in), _p(W_out),
+                            _p(scores), _p(order), _p(cett))
+    return scores, order, cett
+
+
+def threshold_search(scores, cett, bound=0.2):
+    """(tau_base, mean CETT at tau_base): the largest score value eps over all samples with
+    mean_x CETT(x; eps) <= bound (Eq. base_threshold).  scores [B, d_ff], cett [B, d_ff + 1]."""
+    scores, cett = _c(scores, np.float64), _c(cett, np.float64)
+    B, d_ff = scores.shape
+    assert cett.shape == (B, d_ff + 1)
+    mean = ctypes.c_double()
+    tau = lib().oracle_threshold_search(_p(scores), _p(cett), B, d_ff, float(bound), ctypes.byref(mean))
+    return float(tau), mean.value

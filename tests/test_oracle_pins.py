@@ -338,3 +338,71 @@ def test_cett_identity_and_prefix_bound(oracle):
         assert abs(cett - np.linalg.norm(y_d - y_s) / np.linalg.norm(y_d)) < 1e-9
         diff_fro2 += float(np.sum((y_d - y_s) ** 2))
     assert math.sqrt(diff_fro2) <= float(np.sum(A[cut])) * (1 + 1e-12)
+
+
+# ----------------------------------------------------------------------------------------------
+# Offline threshold search: Eq. base_threshold
+# ----------------------------------------------------------------------------------------------
+
+def _cett_by_definition(oracle, X, Wg, Wu, Wd, A, eps):
+    """||sum_{A_j < eps} n_j(x)||_F / ||MLP(x)||_F through the (separately pinned) per-token FFN routines."""
+    num = den = 0.0
+    for t in range(X.shape[0]):
+        y_d = oracle.dense_ffn(X[t], Wg, Wu, Wd)
+        y_s, _, _ = oracle.sparse_ffn(X[t], Wg, Wu, Wd, A, eps)     # keeps A_j >= eps
+        num += float(np.sum((y_d - y_s) ** 2))
+        den += float(np.sum(y_d ** 2))
+    return math.sqrt(num / den)
+
+
+def test_cett_curve_matches_definition(oracle):
+    rng = np.random.default_rng(20)
+    T, F = 5, 9
+    X, Wg, Wu, Wd = _layer(rng, d=8, F=F, T=T)
+    A, order, cett = oracle.cett_curve(X, Wg, Wu, Wd)
+    np.testing.assert_allclose(A, oracle.neuron_scores(X, [0, T], Wg, Wu, Wd)[0], rtol=1e-12)
+    assert list(order) == list(np.argsort(A, kind="stable"))
+    assert cett[0] == 0.0 and abs(cett[F] - 1.0) < 1e-12
+    a = np.sort(A)
+    for k in range(F + 1):
+        eps = a[0] * 0.5 if k == 0 else (np.inf if k == F else 0.5 * (a[k - 1] + a[k]))
+        assert abs(cett[k] - _cett_by_definition(oracle, X, Wg, Wu, Wd, A, eps)) < 1e-10
+    # at eps equal to a score that neuron is still kept (S_cut uses strict <)
+    assert abs(cett[3] - _cett_by_definition(oracle, X, Wg, Wu, Wd, A, a[3])) < 1e-10
+
+
+def test_cett_curve_orthogonal_outputs_closed_form(oracle):
+    """W_out diagonal: the neurons' outputs are orthogonal, so ||sum_cut n_j||^2 = sum_cut A_j^2."""
+    rng = np.random.default_rng(21)
+    d = F = 7
+    X, Wg, Wu, _ = _layer(rng, d=d, F=F, T=6)
+    Wd = np.diag(rng.random(F) + 0.5).astype(np.float32)
+    A, order, cett = oracle.cett_curve(X, Wg, Wu, Wd)
+    a2 = np.sort(A) ** 2
+    ref = np.sqrt(np.concatenate([[0.0], np.cumsum(a2)]) / np.sum(a2))
+    np.testing.assert_allclose(cett, ref, rtol=1e-10, atol=1e-12)
+
+
+def test_threshold_search_brute_force(oracle):
+    rng = np.random.default_rng(22)
+    B, F, d = 3, 6, 8
+    Wg = (rng.standard_normal((F, d)) * 0.3).astype(np.float32)
+    Wu = (rng.standard_normal((F, d)) * 0.3).astype(np.float32)
+    Wd = (rng.standard_normal((d, F)) * 0.3).astype(np.float32)
+    Xs = [rng.standard_normal((T, d)).astype(np.float32) for T in (4, 7, 5)]
+    curves = [oracle.cett_curve(X, Wg, Wu, Wd) for X in Xs]
+    scores = np.stack([c[0] for c in curves])
+    cett = np.stack([c[2] for c in curves])
+    for bound in (0.0, 0.05, 0.2, 0.5, 1.0):
+        tau, mean = oracle.threshold_search(scores, cett, bound)
+        best, best_mean = None, None
+        for eps in np.sort(scores.ravel()):
+            m = np.mean([_cett_by_definition(oracle, Xs[b], Wg, Wu, Wd, scores[b], eps) for b in range(B)])
+            if m <= bound + 1e-12:
+                best, best_mean = eps, m
+        assert tau == best and abs(mean - best_mean) < 1e-10
+    assert oracle.threshold_search(scores, cett, 0.0)[0] == scores.min()      # nothing may be cut
+    assert oracle.threshold_search(scores, cett, 1.0)[0] == scores.max()      # everything but the top neuron
+    # a looser bound never lowers the threshold
+    taus = [oracle.threshold_search(scores, cett, b)[0] for b in (0.01, 0.1, 0.2, 0.4, 0.8)]
+    assert all(x <= y for x, y in zip(taus, taus[1:]))
