@@ -148,6 +148,33 @@ int clada_prefix_select(const clada_layer *layer, const void *X, const int64_t *
 int clada_tau_from_sparsity(const float *scores, int32_t B, int32_t d_ff, float rho,
                             float *tau_base /*[B]*/, void *stream);
 
+/* Offline error-controlled threshold search (Eq. base_threshold) on a set of
+ * validation prompts:
+ *   tau_base = the largest eps with  mean_x CETT(x; eps) <= bound   (the paper uses 0.2),
+ *   CETT(x; eps) = || sum_{A_j(x) < eps} n_j(x) ||_F / || MLP(x) ||_F,
+ * where sample x is prompt b of X (rows seq_offsets[b] .. seq_offsets[b+1]), A_j(x)
+ * its score, n_j(x) neuron j's contribution to the FFN output over the prompt's
+ * tokens and MLP(x) the dense output.  CETT(x; .) only changes at scores of x, so
+ * the candidates are the scores of all samples; the smallest one always
+ * qualifies (nothing cut).
+ *   X, seq_offsets, B   as in clada_prefix_scores (seq_offsets on the HOST, B <= 128)
+ *   tau_base   out [1] device;  mean_cett  out [1] device, the mean CETT at tau_base, may be NULL
+ *   scores     out [B, d_ff] fp32 (CUDA-core accumulation for every dtype)
+ *   ws         clada_cett_workspace_bytes() bytes, 256-byte aligned; d_ff <= 16384
+ * Not on the decode path: run once per layer before serving. */
+size_t clada_cett_workspace_bytes(const clada_layer *layer, const int64_t *seq_offsets, int32_t B);
+int clada_cett_threshold_search(const clada_layer *layer, const void *X, const int64_t *seq_offsets,
+                                int32_t B, float bound, float *tau_base, float *mean_cett,
+                                float *scores, void *ws, size_t ws_bytes, int32_t *status,
+                                void *stream);
+/* After a search, sample `sample`'s curve from the same workspace:
+ * cum_out [d_ff+1] fp64 device, cum_out[k] = || sum of the k lowest-scored neurons' outputs ||_F^2
+ * (so CETT with k neurons cut = sqrt(cum_out[k] / cum_out[d_ff])); order_out [d_ff]
+ * int32 device, the neurons in ascending score order (ties by index); may be NULL. */
+int clada_cett_curve(const clada_layer *layer, const int64_t *seq_offsets, int32_t B, int32_t sample,
+                     const void *ws, size_t ws_bytes, double *cum_out, int32_t *order_out,
+                     void *stream);
+
 /* Eqs. surprisal and entropy, natural log, for B vocabulary rows:
  *   P = softmax(logits[b,:]);  surprisal[b] = -log P[token_id[b]];
  *   entropy[b] = -sum_w P[w] log P[w]   (0 log 0 = 0: -inf logits allowed).

@@ -23,7 +23,8 @@ _INT_RETURNING = [
     "clada_workspace_init", "clada_down_norms", "clada_prefix_scores", "clada_refine_scores",
     "clada_select", "clada_prefix_select", "clada_tau_from_sparsity", "clada_cogload",
     "clada_adjust_threshold", "clada_cogload_adjust", "clada_sparse_ffn_decode",
-    "clada_sparse_ffn_decode_static", "clada_sparse_ffn_decode_layers",
+    "clada_sparse_ffn_decode_static", "clada_sparse_ffn_decode_layers", "clada_cett_threshold_search",
+    "clada_cett_curve",
 ]
 
 
@@ -70,6 +71,10 @@ def load() -> ctypes.CDLL:
     L.clada_sparse_ffn_decode.argtypes = [lp, vp, i32, vp, vp, i64, vp, i32, vp, vp, vp, vp, sz, vp, vp]
     L.clada_sparse_ffn_decode_static.argtypes = [lp, vp, i32, vp, vp, i64, vp, i32, vp, vp, vp, vp, vp]
     L.clada_sparse_ffn_decode_layers.argtypes = [vp, i32, vp, i32, vp, vp, vp, i32, vp, sz, vp, vp]
+    L.clada_cett_workspace_bytes.argtypes = [lp, vp, i32]
+    L.clada_cett_workspace_bytes.restype = sz
+    L.clada_cett_threshold_search.argtypes = [lp, vp, vp, i32, f32, vp, vp, vp, vp, sz, vp, vp]
+    L.clada_cett_curve.argtypes = [lp, vp, i32, i32, vp, sz, vp, vp, vp]
     for name in _INT_RETURNING:
         getattr(L, name).restype = ctypes.c_int
     _lib = L
@@ -325,3 +330,29 @@ def clada_sparse_ffn_decode_layers(stack: LayerStack, x, scores, tau_final, y, w
                                                  _dtype_code(y.dtype), _ptr(ws, torch.uint8, "ws"), ws.numel(),
                                                  _ptr(status, torch.int32, "status"), _stream(stream)),
            "clada_sparse_ffn_decode_layers")
+
+
+def clada_cett_workspace_bytes(layer: Layer, seq_offsets) -> int:
+    off, B = _offsets(seq_offsets)
+    n = int(load().clada_cett_workspace_bytes(layer.ref, ctypes.addressof(off), B))
+    if n == 0:
+        raise CladaError("clada_cett_workspace_bytes: invalid arguments")
+    return n
+
+
+def clada_cett_threshold_search(layer: Layer, X, seq_offsets, bound, tau_base, mean_cett, scores, ws, status=None,
+                                stream=None) -> None:
+    off, B = _offsets(seq_offsets)
+    _check(load().clada_cett_threshold_search(layer.ref, _ptr(X, layer.dtype, "X"), ctypes.addressof(off), B,
+                                              float(bound), _ptr(tau_base, torch.float32, "tau_base"),
+                                              _ptr(mean_cett, torch.float32, "mean_cett"),
+                                              _ptr(scores, torch.float32, "scores"), _ptr(ws, torch.uint8, "ws"),
+                                              ws.numel(), _ptr(status, torch.int32, "status"), _stream(stream)),
+           "clada_cett_threshold_search")
+
+
+def clada_cett_curve(layer: Layer, seq_offsets, sample, ws, cum_out, order_out=None, stream=None) -> None:
+    off, B = _offsets(seq_offsets)
+    _check(load().clada_cett_curve(layer.ref, ctypes.addressof(off), B, int(sample), _ptr(ws, torch.uint8, "ws"),
+                                   ws.numel(), _ptr(cum_out, torch.float64, "cum_out"),
+                                   _ptr(order_out, torch.int32, "order_out"), _stream(stream)), "clada_cett_curve")

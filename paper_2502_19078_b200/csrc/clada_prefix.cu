@@ -18,7 +18,8 @@ constexpr int BM = 64, BN = 64, BK = 32, kPfThreads = 256;
 template <typename T>
 __global__ void __launch_bounds__(kPfThreads)
 prefix_partials_kernel(const T *__restrict__ X, const T *__restrict__ Wg, const T *__restrict__ Wu,
-                       int d_model, int d_ff, const SeqTable tab, float *__restrict__ partials) {
+                       int d_model, int d_ff, const SeqTable tab, float *__restrict__ partials,
+                       float *__restrict__ zt, long long zt_stride) {
     constexpr int E = Elem<T>::kPerVec;
     __shared__ __align__(16) float Xs[BK][BM + 4];
     __shared__ __align__(16) float Gs[BK][BN + 4];
@@ -81,6 +82,7 @@ prefix_partials_kernel(const T *__restrict__ X, const T *__restrict__ Wg, const 
         __syncthreads();
     }
     // epilogue: z^2 summed over this thread's 4 tokens, then over the 16 thread rows in order
+    // (the offline threshold search also wants z itself, neuron-major: zt[j, t])
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
         float s = 0.f;
@@ -88,6 +90,8 @@ prefix_partials_kernel(const T *__restrict__ X, const T *__restrict__ Wg, const 
         for (int i = 0; i < 4; ++i) {
             const float z = silu_f(ag[i][j]) * au[i][j];  // padded token rows give exactly 0
             s = fmaf(z, z, s);
+            const long long t = t0 + ty * 4 + i;
+            if (zt && t < t1 && n0 + tx * 4 + j < d_ff) zt[(size_t)(n0 + tx * 4 + j) * zt_stride + t] = z;
         }
         s_red[ty][tx * 4 + j] = s;
     }
@@ -266,15 +270,32 @@ static size_t partials_bytes(int n_mtiles, int d_ff) {
 
 template <typename T>
 static int run_scores(const clada_layer *L, const void *X, const SeqTable &tab, int n_mtiles, float *scores,
-                      float *partials, cudaStream_t st) {
+                      float *partials, cudaStream_t st, float *zt = nullptr, long long zt_stride = 0) {
     if (n_mtiles > 0) {
         dim3 grid((L->d_ff + BN - 1) / BN, n_mtiles);
         prefix_partials_kernel<T><<<grid, kPfThreads, 0, st>>>(
             static_cast<const T *>(X), static_cast<const T *>(L->w_gate), static_cast<const T *>(L->w_up),
-            L->d_model, L->d_ff, tab, partials);
+            L->d_model, L->d_ff, tab, partials, zt, zt_stride);
         CLADA_CUDA_TRY(cudaGetLastError());
     }
     return launch_prefix_finalize(partials, tab, BM, L->d_ff, L->w_down_norm, scores, st);
+}
+
+int run_prefix_scores_with_z(const clada_layer *layer, const void *X, const int64_t *seq_offsets, int32_t B,
+                             float *scores, float *partials, float *zt, cudaStream_t st) {
+    SeqTable tab;
+    int n_mtiles = 0;
+    int rc = build_table(seq_offsets, B, &tab, &n_mtiles);
+    if (rc != CLADA_OK) return rc;
+    return layer->dtype == CLADA_F32
+               ? run_scores<float>(layer, X, tab, n_mtiles, scores, partials, st, zt, seq_offsets[B])
+               : run_scores<__nv_bfloat16>(layer, X, tab, n_mtiles, scores, partials, st, zt, seq_offsets[B]);
+}
+
+size_t prefix_partials_bytes_cuda_core(const int64_t *seq_offsets, int32_t B, int d_ff) {
+    long long tiles = 0;
+    for (int b = 0; b < B; ++b) tiles += tiles_of(seq_offsets[b + 1] - seq_offsets[b], BM);
+    return partials_bytes((int)tiles, d_ff);
 }
 
 int launch_prefix_finalize(const float *partials, const SeqTable &tab, int tile, int d_ff,

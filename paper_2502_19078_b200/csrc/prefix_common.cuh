@@ -33,6 +33,12 @@ __device__ inline void locate_tile(const SeqTable &tab, int ttile, int tile, int
 int launch_prefix_finalize(const float *partials, const SeqTable &tab, int tile, int d_ff,
                            const float *w_down_norm, float *scores, cudaStream_t st);
 
+// CUDA-core scores for any dtype that also leave z, neuron-major (zt[j, t], row stride T_total), for the
+// offline threshold search; partials must hold prefix_partials_bytes_cuda_core() bytes.
+int run_prefix_scores_with_z(const clada_layer *layer, const void *X, const int64_t *seq_offsets, int32_t B,
+                             float *scores, float *partials, float *zt, cudaStream_t st);
+size_t prefix_partials_bytes_cuda_core(const int64_t *seq_offsets, int32_t B, int d_ff);
+
 // Tensor-core partial sums (bf16 layers, 128-token tiles).  partials: [sum_b tiles_of(T_b, 128), d_ff].
 int run_prefix_partials_tc(const clada_layer *layer, const void *X, const SeqTable &tab, long long T_total,
                            float *partials, int32_t *status, cudaStream_t st);

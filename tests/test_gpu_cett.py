@@ -1,0 +1,96 @@
+"""GPU parity of the offline threshold search (Eq. base_threshold) against the oracle.
+
+Tolerances: the curve CETT(k) within 1e-4 absolute (fp32 running sums over up to d_ff neurons against fp64);
+the chosen threshold must be the score of the same (sample, neuron) as the oracle's, or - when two candidates'
+mean CETT straddle the bound by less than the curve tolerance - a candidate the oracle finds feasible within it.
+"""
+import numpy as np
+import pytest
+import torch
+
+from paper_2502_19078_b200 import workloads as wl
+from tests._util import gpu_layer, oracle_weights
+
+pytestmark = pytest.mark.gpu
+
+CURVE_TOL = 1e-4
+
+
+@pytest.fixture(scope="module")
+def clada():
+    from paper_2502_19078_b200 import binding, build
+    build.build()
+    binding.load()
+    return binding
+
+
+@pytest.mark.parametrize("name,kw,lengths", [
+    ("c1_small_f32", {"d_model": 64, "d_ff": 96}, [40, 70, 33]),
+    ("c2_llama2_7b_layer", {"d_model": 256, "d_ff": 300}, [100, 60]),
+    ("c1_small_f32", {}, [64]),
+    ("c2_llama2_7b_layer", {"d_model": 136, "d_ff": 200}, [1, 35, 64, 7]),
+])
+def test_cett_threshold_search_parity(clada, oracle, name, kw, lengths):
+    w = wl.scaled(wl.WORKLOADS[name], **kw)
+    weights = wl.layer_weights(w, 0)
+    layer = gpu_layer(weights, clada)
+    W_in, V_in, W_out = oracle_weights(weights)
+    scale = wl.channel_scale(w)
+    Xs = [wl.hidden_states(w, 0, "prefix", b, n, "cpu", scale) for b, n in enumerate(lengths)]
+    X = torch.cat(Xs)
+    off = wl.seq_offsets(lengths)
+    B, F = len(lengths), w.d_ff
+    curves = [oracle.cett_curve(wl.to_numpy_bits(x), W_in, V_in, W_out) for x in Xs]
+    sc_or = np.stack([c[0] for c in curves])
+    cett_or = np.stack([c[2] for c in curves])
+
+    ws = torch.empty(clada.clada_cett_workspace_bytes(layer, off), dtype=torch.uint8, device="cuda")
+    tau = torch.empty(1, device="cuda")
+    mean = torch.empty(1, device="cuda")
+    scores = torch.empty(B, F, device="cuda")
+    for bound in (0.2, 0.05, 0.6):
+        clada.clada_cett_threshold_search(layer, X.cuda(), off, bound, tau, mean, scores, ws)
+        torch.cuda.synchronize()
+        sc = scores.cpu().numpy()
+        assert np.max(np.abs(sc - sc_or) / sc_or) <= 5e-6
+        # curves
+        for b in range(B):
+            cum = torch.empty(F + 1, dtype=torch.float64, device="cuda")
+            order = torch.empty(F, dtype=torch.int32, device="cuda")
+            clada.clada_cett_curve(layer, off, b, ws, cum, order)
+            torch.cuda.synchronize()
+            cum = cum.cpu().numpy()
+            cett = np.sqrt(cum / cum[F])
+            assert cett[0] == 0.0
+            assert np.max(np.abs(cett - cett_or[b])) <= CURVE_TOL, (b, np.max(np.abs(cett - cett_or[b])))
+            od = order.cpu().numpy()
+            assert sorted(od.tolist()) == list(range(F))
+            assert np.all(np.diff(sc[b][od]) >= 0)                      # ascending by the GPU's own scores
+        # the threshold
+        tau_or, mean_or = oracle.threshold_search(sc_or, cett_or, bound)
+        t = np.float32(tau.item())
+        where = np.argwhere(sc == t)
+        assert where.size > 0                                            # tau is one of the scores
+        where_or = np.argwhere(sc_or == tau_or)[0]
+        if not any((wb == where_or).all() for wb in where):
+            # another candidate: acceptable only if the oracle's own mean CETT there is within tolerance of the bound
+            b_, j_ = where[0]
+            m_there = np.mean([cett_or[x][np.sum(sc_or[x] < sc_or[b_, j_])] for x in range(B)])
+            assert m_there <= bound + CURVE_TOL and abs(sc_or[b_, j_] - tau_or) / tau_or < 0.05, (bound, m_there)
+        assert abs(mean.item() - mean_or) <= 3 * CURVE_TOL or not any((wb == where_or).all() for wb in where)
+        assert mean.item() <= bound + 1e-6
+
+
+def test_cett_search_host_errors(clada):
+    w = wl.scaled(wl.WORKLOADS["c2_llama2_7b_layer"], d_model=64, d_ff=50)
+    layer = gpu_layer(wl.layer_weights(w, 0), clada)
+    X = torch.zeros(10, 64, dtype=torch.bfloat16, device="cuda")
+    out = torch.empty(1, device="cuda")
+    scores = torch.empty(1, 50, device="cuda")
+    small = torch.empty(1024, dtype=torch.uint8, device="cuda")
+    with pytest.raises(clada.CladaError, match="workspace"):
+        clada.clada_cett_threshold_search(layer, X, [0, 10], 0.2, out, None, scores, small)
+    ws = torch.empty(clada.clada_cett_workspace_bytes(layer, [0, 10]), dtype=torch.uint8, device="cuda")
+    with pytest.raises(clada.CladaError, match="shape"):
+        clada.clada_cett_threshold_search(layer, X, [0, 10], -1.0, out, None, scores, ws)
+    torch.cuda.synchronize()
