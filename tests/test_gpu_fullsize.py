@@ -204,3 +204,54 @@ def test_c5_batch16_ragged(clada, oracle):
     for rho in (0.30, 0.60):
         _ffn_synthetic_scores(clada, oracle, w, 2, seqs=[3], n_steps=1, rho=rho)
     _cogload_all_rows(clada, oracle, w, n_steps=1)
+
+
+def test_c2_threshold_search_full_width(clada, oracle):
+    """Offline threshold search on the full-width layer (11008 neurons, two short validation prompts):
+    sampled points of the curve against the definition, and the optimality of the chosen threshold."""
+    w = wl.WORKLOADS["c2_llama2_7b_layer"]
+    layer, weights = _layer_on_gpu(clada, w, 0)
+    W_in, V_in, W_out = (wl.to_numpy_bits(weights[k]) for k in ("w_gate", "w_up", "w_down"))
+    scale = wl.channel_scale(w, "cuda")
+    lengths = [16, 24]
+    off = wl.seq_offsets(lengths)
+    X = torch.cat([wl.hidden_states(w, 0, "prefix", b, n, "cuda", scale) for b, n in enumerate(lengths)])
+    F, bound = w.d_ff, 0.2
+    ws = torch.empty(clada.clada_cett_workspace_bytes(layer, off), dtype=torch.uint8, device="cuda")
+    tau = torch.empty(1, device="cuda")
+    mean = torch.empty(1, device="cuda")
+    scores = torch.empty(2, F, device="cuda")
+    clada.clada_cett_threshold_search(layer, X, off, bound, tau, mean, scores, ws)
+    cums = []
+    for b in range(2):
+        cum = torch.empty(F + 1, dtype=torch.float64, device="cuda")
+        clada.clada_cett_curve(layer, off, b, ws, cum)
+        cums.append(cum.cpu().numpy())
+    torch.cuda.synchronize()
+    sc = scores.cpu().numpy()
+    cett = [np.sqrt(c / c[F]) for c in cums]
+    # the curve of sample 0 at three cut sizes, by the definition (dense minus sparse output over the prompt)
+    X0 = wl.to_numpy_bits(X[:16])
+    A0 = oracle.neuron_scores(X0, [0, 16], W_in, V_in, W_out)[0]
+    a_sorted = np.sort(A0)
+    for k in (F // 4, F // 2, (3 * F) // 4):
+        eps = 0.5 * (a_sorted[k - 1] + a_sorted[k])
+        num = den = 0.0
+        for t in range(16):
+            y_d = oracle.dense_ffn(X0[t], W_in, V_in, W_out)
+            y_s, _, n_kept = oracle.sparse_ffn(X0[t], W_in, V_in, W_out, A0, eps)
+            assert n_kept == F - k
+            num += float(np.sum((y_d - y_s) ** 2))
+            den += float(np.sum(y_d ** 2))
+        assert abs(cett[0][k] - np.sqrt(num / den)) <= 1e-4
+    # optimality on the GPU's own curves: tau is a score, feasible, and every larger candidate is infeasible
+    t = np.float32(tau.item())
+    assert np.any(sc == t) and mean.item() <= bound + 1e-6
+    srt = [np.sort(sc[b]) for b in range(2)]
+    def mean_at(eps):
+        return np.mean([cett[b][np.searchsorted(srt[b], eps, side="left")] for b in range(2)])
+    assert abs(mean_at(t) - mean.item()) <= 1e-5
+    larger = np.sort(sc[sc > t])
+    assert larger.size > 0
+    assert all(mean_at(e) > bound - 1e-6 for e in larger[:64])
+    assert mean_at(larger[0]) > bound - 1e-6
