@@ -15,7 +15,9 @@
  * Pins (tests/test_oracle_pins.py): entropy/surprisal closed forms, literal
  * Frobenius form of the score, brute-force selection on tiny layers, dense
  * FFN against an independent float64 matrix formulation, zero-sparsity
- * identity, CETT identity.  The whole of Algorithm 2 end to end has no
+ * identity, CETT identity; the offline threshold search against the definition
+ * evaluated through the per-token FFN routines, a closed form for orthogonal
+ * neuron outputs, and brute force over all candidates.  The whole of Algorithm 2 end to end has no
  * published trace: parity unpinned beyond those per-step pins.
  *
  * Element types: 0 = IEEE fp32, 1 = bfloat16 (uint16 bit patterns).  Both
