@@ -17,7 +17,9 @@
  * FFN against an independent float64 matrix formulation, zero-sparsity
  * identity, CETT identity; the offline threshold search against the definition
  * evaluated through the per-token FFN routines, a closed form for orthogonal
- * neuron outputs, and brute force over all candidates.  The whole of Algorithm 2 end to end has no
+ * neuron outputs, and brute force over all candidates; the GELU-gated and
+ * non-gated ReLU forms against a library formulation, a worked two-neuron
+ * example and the tanh formula typed out.  The whole of Algorithm 2 end to end has no
  * published trace: parity unpinned beyond those per-step pins.
  *
  * Element types: 0 = IEEE fp32, 1 = bfloat16 (uint16 bit patterns).  Both
@@ -46,6 +48,34 @@ static double elem(const void *p, int dtype, size_t i)
 /* sigma of Eq. neuron_activation read as SiLU: g * logistic(g). */
 static double silu(double g) { return g / (1.0 + exp(-g)); }
 
+/* The FFN forms of the model families the paper evaluates (Section 4.1):
+ *   OR_SILU_GATED  z = silu(g) * u                       (LLaMA, Mistral)
+ *   OR_GELU_GATED  z = gelu(g) * u, tanh form of GELU    (Gemma)
+ *   OR_RELU        z = max(g, 0), no V_in factor         (OPT)
+ * with g = W_in,j . x and u = V_in,j . x.  The gated forms are Eq.
+ * neuron_activation with that sigma; the non-gated one is the same equation
+ * with the V_in factor absent, the only reading an FFN without a gate
+ * projection admits.  Biases are not part of the equation and are left out. */
+#define OR_PI 3.14159265358979323846
+enum { OR_SILU_GATED = 0, OR_GELU_GATED = 1, OR_RELU = 2 };
+
+static int is_gated(int act) { return act != OR_RELU; }
+
+static double neuron_value(int act, double g, double u)
+{
+    switch (act) {
+    case OR_GELU_GATED: {
+        /* 0.5 g (1 + tanh(sqrt(2/pi) (g + 0.044715 g^3))) */
+        double inner = sqrt(2.0 / OR_PI) * (g + 0.044715 * g * g * g);
+        return 0.5 * g * (1.0 + tanh(inner)) * u;
+    }
+    case OR_RELU:
+        return g > 0.0 ? g : 0.0;
+    default:
+        return silu(g) * u;
+    }
+}
+
 int oracle_num_threads(void)
 {
 #ifdef _OPENMP
@@ -67,7 +97,7 @@ int oracle_num_threads(void)
  * ------------------------------------------------------------------ */
 void oracle_neuron_scores(int dtype, const void *X, const int64_t *off, int B,
                           int d_model, int d_ff, const void *W_in,
-                          const void *V_in, const void *W_out, double *scores)
+                          const void *V_in, const void *W_out, double *scores, int act)
 {
 #pragma omp parallel for schedule(dynamic, 8)
     for (int j = 0; j < d_ff; ++j) {
@@ -83,9 +113,10 @@ void oracle_neuron_scores(int dtype, const void *X, const int64_t *off, int B,
                 for (int k = 0; k < d_model; ++k) {
                     double x = elem(X, dtype, (size_t)t * d_model + k);
                     g += elem(W_in, dtype, (size_t)j * d_model + k) * x;
-                    u += elem(V_in, dtype, (size_t)j * d_model + k) * x;
+                    if (is_gated(act))
+                        u += elem(V_in, dtype, (size_t)j * d_model + k) * x;
                 }
-                double z = silu(g) * u;
+                double z = neuron_value(act, g, u);
                 zz += z * z;
             }
             scores[(size_t)b * d_ff + j] = sqrt(zz) * sqrt(wnorm2);
@@ -98,7 +129,7 @@ void oracle_neuron_scores(int dtype, const void *X, const int64_t *off, int B,
  * Tiny sizes only (allocates T*d_model doubles per neuron). */
 void oracle_neuron_scores_literal(int dtype, const void *X, int T, int d_model,
                                   int d_ff, const void *W_in, const void *V_in,
-                                  const void *W_out, double *scores)
+                                  const void *W_out, double *scores, int act)
 {
     double *M = (double *)malloc((size_t)T * d_model * sizeof(double));
     for (int j = 0; j < d_ff; ++j) {
@@ -107,9 +138,10 @@ void oracle_neuron_scores_literal(int dtype, const void *X, int T, int d_model,
             for (int k = 0; k < d_model; ++k) {
                 double x = elem(X, dtype, (size_t)t * d_model + k);
                 g += elem(W_in, dtype, (size_t)j * d_model + k) * x;
-                u += elem(V_in, dtype, (size_t)j * d_model + k) * x;
+                if (is_gated(act))
+                    u += elem(V_in, dtype, (size_t)j * d_model + k) * x;
             }
-            double z = silu(g) * u;
+            double z = neuron_value(act, g, u);
             for (int i = 0; i < d_model; ++i)
                 M[(size_t)t * d_model + i] = z * elem(W_out, dtype, (size_t)i * d_ff + j);
         }
@@ -205,7 +237,7 @@ void oracle_adjust_threshold(const float *tau_base, const float *lambda,
 int oracle_sparse_ffn(int dtype, const void *x, int d_model, int d_ff,
                       const void *W_in, const void *V_in, const void *W_out,
                       const double *scores, double tau, double *y,
-                      uint8_t *mask_out)
+                      uint8_t *mask_out, int act)
 {
     double *h = (double *)calloc((size_t)d_ff, sizeof(double));
     uint8_t *keep = (uint8_t *)malloc((size_t)d_ff);
@@ -224,9 +256,10 @@ int oracle_sparse_ffn(int dtype, const void *x, int d_model, int d_ff,
         for (int k = 0; k < d_model; ++k) {
             double xv = elem(x, dtype, (size_t)k);
             g += elem(W_in, dtype, (size_t)j * d_model + k) * xv;
-            u += elem(V_in, dtype, (size_t)j * d_model + k) * xv;
+            if (is_gated(act))
+                u += elem(V_in, dtype, (size_t)j * d_model + k) * xv;
         }
-        h[j] = silu(g) * u;
+        h[j] = neuron_value(act, g, u);
     }
 #pragma omp parallel for schedule(static)
     for (int i = 0; i < d_model; ++i) {
@@ -245,7 +278,7 @@ int oracle_sparse_ffn(int dtype, const void *x, int d_model, int d_ff,
  * zero-sparsity reference the sparse pass must reduce to. */
 void oracle_dense_ffn(int dtype, const void *x, int d_model, int d_ff,
                       const void *W_in, const void *V_in, const void *W_out,
-                      double *y)
+                      double *y, int act)
 {
     double *h = (double *)malloc((size_t)d_ff * sizeof(double));
 #pragma omp parallel for schedule(static)
@@ -254,9 +287,10 @@ void oracle_dense_ffn(int dtype, const void *x, int d_model, int d_ff,
         for (int k = 0; k < d_model; ++k) {
             double xv = elem(x, dtype, (size_t)k);
             g += elem(W_in, dtype, (size_t)j * d_model + k) * xv;
-            u += elem(V_in, dtype, (size_t)j * d_model + k) * xv;
+            if (is_gated(act))
+                u += elem(V_in, dtype, (size_t)j * d_model + k) * xv;
         }
-        h[j] = silu(g) * u;
+        h[j] = neuron_value(act, g, u);
     }
 #pragma omp parallel for schedule(static)
     for (int i = 0; i < d_model; ++i) {
@@ -322,7 +356,7 @@ static int cmp_pair(const void *p, const void *q)
 
 void oracle_cett_curve(int dtype, const void *X, int T, int d_model, int d_ff,
                        const void *W_in, const void *V_in, const void *W_out,
-                       double *scores, int32_t *order, double *cett)
+                       double *scores, int32_t *order, double *cett, int act)
 {
     double *z = (double *)malloc((size_t)T * d_ff * sizeof(double));      /* z[t, j] */
     double *cut = (double *)calloc((size_t)T * d_model, sizeof(double));  /* running sum of cut outputs */
@@ -339,9 +373,10 @@ void oracle_cett_curve(int dtype, const void *X, int T, int d_model, int d_ff,
             for (int k = 0; k < d_model; ++k) {
                 double x = elem(X, dtype, (size_t)t * d_model + k);
                 g += elem(W_in, dtype, (size_t)j * d_model + k) * x;
-                u += elem(V_in, dtype, (size_t)j * d_model + k) * x;
+                if (is_gated(act))
+                    u += elem(V_in, dtype, (size_t)j * d_model + k) * x;
             }
-            double zt = silu(g) * u;
+            double zt = neuron_value(act, g, u);
             z[(size_t)t * d_ff + j] = zt;
             zz += zt * zt;
         }

@@ -18,6 +18,8 @@ _SRC = os.path.join(_HERE, "clada_oracle.c")
 _LIB = os.path.join(_HERE, "libclada_oracle.so")
 
 F32, BF16 = 0, 1
+# FFN forms (Section 4.1 model families): z = silu(g)*u, z = gelu_tanh(g)*u, z = relu(g) without V_in
+SILU_GATED, GELU_GATED, RELU = 0, 1, 2
 _lib = None
 
 
@@ -38,9 +40,9 @@ def lib():
         vp, i32, i64, dbl, f32 = (ctypes.c_void_p, ctypes.c_int, ctypes.c_int64,
                                   ctypes.c_double, ctypes.c_float)
         L.oracle_num_threads.restype = ctypes.c_int
-        L.oracle_neuron_scores.argtypes = [i32, vp, vp, i32, i32, i32, vp, vp, vp, vp]
+        L.oracle_neuron_scores.argtypes = [i32, vp, vp, i32, i32, i32, vp, vp, vp, vp, i32]
         L.oracle_neuron_scores.restype = None
-        L.oracle_neuron_scores_literal.argtypes = [i32, vp, i32, i32, i32, vp, vp, vp, vp]
+        L.oracle_neuron_scores_literal.argtypes = [i32, vp, i32, i32, i32, vp, vp, vp, vp, i32]
         L.oracle_neuron_scores_literal.restype = None
         L.oracle_select.argtypes = [vp, i32, dbl, vp, vp]
         L.oracle_select.restype = ctypes.c_int
@@ -48,11 +50,11 @@ def lib():
         L.oracle_cogload.restype = ctypes.c_int
         L.oracle_adjust_threshold.argtypes = [vp, vp, vp, f32, f32, vp, vp, i32, i32, vp]
         L.oracle_adjust_threshold.restype = None
-        L.oracle_sparse_ffn.argtypes = [i32, vp, i32, i32, vp, vp, vp, vp, dbl, vp, vp]
+        L.oracle_sparse_ffn.argtypes = [i32, vp, i32, i32, vp, vp, vp, vp, dbl, vp, vp, i32]
         L.oracle_sparse_ffn.restype = ctypes.c_int
-        L.oracle_dense_ffn.argtypes = [i32, vp, i32, i32, vp, vp, vp, vp]
+        L.oracle_dense_ffn.argtypes = [i32, vp, i32, i32, vp, vp, vp, vp, i32]
         L.oracle_dense_ffn.restype = None
-        L.oracle_cett_curve.argtypes = [i32, vp, i32, i32, i32, vp, vp, vp, vp, vp, vp]
+        L.oracle_cett_curve.argtypes = [i32, vp, i32, i32, i32, vp, vp, vp, vp, vp, vp, i32]
         L.oracle_cett_curve.restype = None
         L.oracle_threshold_search.argtypes = [vp, vp, i32, i32, dbl, vp]
         L.oracle_threshold_search.restype = dbl
@@ -83,35 +85,45 @@ def _p(a: np.ndarray):
     return a.ctypes.data_as(ctypes.c_void_p)
 
 
-def _check_weights(X, W_in, V_in, W_out):
+def _check_weights(X, W_in, V_in, W_out, act=SILU_GATED):
     d_ff, d_model = W_in.shape
-    assert V_in.shape == (d_ff, d_model), "V_in must be [d_ff, d_model]"
+    if act == RELU:
+        assert V_in is None, "the non-gated form has no V_in"
+    else:
+        assert V_in.shape == (d_ff, d_model), "V_in must be [d_ff, d_model]"
+        assert V_in.dtype == W_in.dtype
     assert W_out.shape == (d_model, d_ff), "W_out must be [d_model, d_ff] (neuron j = column j)"
     assert X.shape[-1] == d_model
-    assert X.dtype == W_in.dtype == V_in.dtype == W_out.dtype
+    assert X.dtype == W_in.dtype == W_out.dtype
     return d_model, d_ff
 
 
-def neuron_scores(X, seq_offsets, W_in, V_in, W_out) -> np.ndarray:
+def _pv(V_in):
+    return None if V_in is None else _p(V_in)
+
+
+def neuron_scores(X, seq_offsets, W_in, V_in, W_out, act=SILU_GATED) -> np.ndarray:
     """A[b, j] of Eq. neuron_activation for each prefix b = rows seq_offsets[b]:seq_offsets[b+1] of X."""
-    X, W_in, V_in, W_out = _c(X), _c(W_in), _c(V_in), _c(W_out)
-    d_model, d_ff = _check_weights(X, W_in, V_in, W_out)
+    X, W_in, W_out = _c(X), _c(W_in), _c(W_out)
+    V_in = None if V_in is None else _c(V_in)
+    d_model, d_ff = _check_weights(X, W_in, V_in, W_out, act)
     off = _c(np.asarray(seq_offsets), np.int64)
     B = off.size - 1
     assert off[0] >= 0 and off[-1] <= X.shape[0] and np.all(np.diff(off) >= 0)
     out = np.empty((B, d_ff), dtype=np.float64)
     lib().oracle_neuron_scores(_dt(X), _p(X), _p(off), B, d_model, d_ff,
-                               _p(W_in), _p(V_in), _p(W_out), _p(out))
+                               _p(W_in), _pv(V_in), _p(W_out), _p(out), int(act))
     return out
 
 
-def neuron_scores_literal(X, W_in, V_in, W_out) -> np.ndarray:
+def neuron_scores_literal(X, W_in, V_in, W_out, act=SILU_GATED) -> np.ndarray:
     """Same quantity for one prefix X [T, d_model], by the Frobenius norm of the explicit T x d_model matrix."""
-    X, W_in, V_in, W_out = _c(X), _c(W_in), _c(V_in), _c(W_out)
-    d_model, d_ff = _check_weights(X, W_in, V_in, W_out)
+    X, W_in, W_out = _c(X), _c(W_in), _c(W_out)
+    V_in = None if V_in is None else _c(V_in)
+    d_model, d_ff = _check_weights(X, W_in, V_in, W_out, act)
     out = np.empty(d_ff, dtype=np.float64)
     lib().oracle_neuron_scores_literal(_dt(X), _p(X), X.shape[0], d_model, d_ff,
-                                       _p(W_in), _p(V_in), _p(W_out), _p(out))
+                                       _p(W_in), _pv(V_in), _p(W_out), _p(out), int(act))
     return out
 
 
@@ -149,24 +161,26 @@ def adjust_threshold(tau_base, lam, gam, tau_s, tau_H, surprisal, entropy) -> np
     return out
 
 
-def sparse_ffn(x, W_in, V_in, W_out, scores, tau):
+def sparse_ffn(x, W_in, V_in, W_out, scores, tau, act=SILU_GATED):
     """(y [d_model] float64, mask u8 [d_ff], count) of the masked gated FFN for one token x."""
-    x, W_in, V_in, W_out = _c(x), _c(W_in), _c(V_in), _c(W_out)
-    d_model, d_ff = _check_weights(x, W_in, V_in, W_out)
+    x, W_in, W_out = _c(x), _c(W_in), _c(W_out)
+    V_in = None if V_in is None else _c(V_in)
+    d_model, d_ff = _check_weights(x, W_in, V_in, W_out, act)
     scores = _c(scores, np.float64)
     assert scores.size == d_ff and x.size == d_model
     y = np.empty(d_model, dtype=np.float64)
     mask = np.empty(d_ff, dtype=np.uint8)
-    count = lib().oracle_sparse_ffn(_dt(x), _p(x), d_model, d_ff, _p(W_in), _p(V_in), _p(W_out),
-                                    _p(scores), float(tau), _p(y), _p(mask))
+    count = lib().oracle_sparse_ffn(_dt(x), _p(x), d_model, d_ff, _p(W_in), _pv(V_in), _p(W_out),
+                                    _p(scores), float(tau), _p(y), _p(mask), int(act))
     return y, mask, int(count)
 
 
-def dense_ffn(x, W_in, V_in, W_out) -> np.ndarray:
-    x, W_in, V_in, W_out = _c(x), _c(W_in), _c(V_in), _c(W_out)
-    d_model, d_ff = _check_weights(x, W_in, V_in, W_out)
+def dense_ffn(x, W_in, V_in, W_out, act=SILU_GATED) -> np.ndarray:
+    x, W_in, W_out = _c(x), _c(W_in), _c(W_out)
+    V_in = None if V_in is None else _c(V_in)
+    d_model, d_ff = _check_weights(x, W_in, V_in, W_out, act)
     y = np.empty(d_model, dtype=np.float64)
-    lib().oracle_dense_ffn(_dt(x), _p(x), d_model, d_ff, _p(W_in), _p(V_in), _p(W_out), _p(y))
+    lib().oracle_dense_ffn(_dt(x), _p(x), d_model, d_ff, _p(W_in), _pv(V_in), _p(W_out), _p(y), int(act))
     return y
 
 
@@ -176,16 +190,17 @@ def tau_from_sparsity(scores_f32, rho) -> np.float32:
     return np.float32(lib().oracle_tau_from_sparsity(_p(s), s.size, float(rho)))
 
 
-def cett_curve(X, W_in, V_in, W_out):
+def cett_curve(X, W_in, V_in, W_out, act=SILU_GATED):
     """For one validation sample X [T, d_model]: (scores [d_ff], order int32 [d_ff] ascending by score,
     cett [d_ff + 1]) with cett[k] = CETT of Eq. base_threshold when the k lowest-scored neurons are cut."""
-    X, W_in, V_in, W_out = _c(X), _c(W_in), _c(V_in), _c(W_out)
-    d_model, d_ff = _check_weights(X, W_in, V_in, W_out)
+    X, W_in, W_out = _c(X), _c(W_in), _c(W_out)
+    V_in = None if V_in is None else _c(V_in)
+    d_model, d_ff = _check_weights(X, W_in, V_in, W_out, act)
     scores = np.empty(d_ff, dtype=np.float64)
     order = np.empty(d_ff, dtype=np.int32)
     cett = np.empty(d_ff + 1, dtype=np.float64)
-    lib().oracle_cett_curve(_dt(X), _p(X), X.shape[0], d_model, d_ff, _p(W_in), _p(V_in), _p(W_out),
-                            _p(scores), _p(order), _p(cett))
+    lib().oracle_cett_curve(_dt(X), _p(X), X.shape[0], d_model, d_ff, _p(W_in), _pv(V_in), _p(W_out),
+                            _p(scores), _p(order), _p(cett), int(act))
     return scores, order, cett
 
 

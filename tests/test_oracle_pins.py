@@ -406,3 +406,89 @@ def test_threshold_search_brute_force(oracle):
     # a looser bound never lowers the threshold
     taus = [oracle.threshold_search(scores, cett, b)[0] for b in (0.01, 0.1, 0.2, 0.4, 0.8)]
     assert all(x <= y for x, y in zip(taus, taus[1:]))
+
+
+# ----------------------------------------------------------------------------------------------
+# FFN forms of the other model families (Section 4.1): GELU-gated and non-gated ReLU
+# ----------------------------------------------------------------------------------------------
+
+def _torch_h(act, tX, tWg, tWu):
+    """Library formulation of the per-neuron value for every token: [T, d_ff] float64."""
+    g = tX @ tWg.T
+    if act == 1:
+        return torch.nn.functional.gelu(g, approximate="tanh") * (tX @ tWu.T)
+    if act == 2:
+        return torch.relu(g)
+    return torch.nn.functional.silu(g) * (tX @ tWu.T)
+
+
+@pytest.mark.parametrize("act", [1, 2])
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_variant_dense_and_masked_ffn_match_library(oracle, act, dtype):
+    rng = np.random.default_rng(30 + act)
+    T, F = 5, 40
+    X, Wg, Wu, Wd = _layer(rng, d=24, F=F, T=T, dtype=dtype)
+    V = None if act == 2 else Wu
+    tX, tWg, tWu, tWd = (torch.from_numpy(_f64(a)) for a in (X, Wg, Wu, Wd))
+    h = _torch_h(act, tX, tWg, tWu)
+    A = oracle.neuron_scores(X, [0, T], Wg, V, Wd, act=act)[0]
+    # scores against explicit norms of the library's h and of W_out's columns
+    ref_A = torch.linalg.norm(h, dim=0) * torch.linalg.norm(tWd, dim=0)
+    np.testing.assert_allclose(A, ref_A.numpy(), rtol=1e-11, atol=1e-14)
+    np.testing.assert_allclose(oracle.neuron_scores_literal(X, Wg, V, Wd, act=act), A, rtol=1e-11, atol=1e-14)
+    tau = float(np.median(A))
+    keep = torch.from_numpy(A >= tau)
+    for t in range(T):
+        np.testing.assert_allclose(oracle.dense_ffn(X[t], Wg, V, Wd, act=act), (h[t] @ tWd.T).numpy(),
+                                   rtol=1e-11, atol=1e-13)
+        y, mask, cnt = oracle.sparse_ffn(X[t], Wg, V, Wd, A, tau, act=act)
+        assert cnt == int(keep.sum()) and np.array_equal(mask.astype(bool), keep.numpy())
+        np.testing.assert_allclose(y, ((h[t] * keep) @ tWd.T).numpy(), rtol=1e-11, atol=1e-13)
+        y0, _, c0 = oracle.sparse_ffn(X[t], Wg, V, Wd, A, 0.0, act=act)
+        assert c0 == F and np.array_equal(y0, oracle.dense_ffn(X[t], Wg, V, Wd, act=act))
+
+
+def test_relu_form_worked_example(oracle):
+    """Two neurons reading +x0 and -x0: only the one whose pre-activation is positive contributes,
+    and it contributes its pre-activation times its W_out column; V_in plays no part."""
+    W_in = np.array([[1.0, 0.0], [-1.0, 0.0]], np.float32)
+    W_out = np.array([[2.0, 5.0], [3.0, 7.0]], np.float32)       # columns are the neurons' outputs
+    x = np.array([2.0, 3.0], np.float32)
+    assert np.array_equal(oracle.dense_ffn(x, W_in, None, W_out, act=2), [4.0, 6.0])
+    assert np.array_equal(oracle.dense_ffn(-x, W_in, None, W_out, act=2), [10.0, 14.0])
+    X = np.stack([x, -x, 2 * x])
+    A = oracle.neuron_scores(X, [0, 3], W_in, None, W_out, act=2)[0]
+    np.testing.assert_allclose(A, [math.sqrt(4 + 16) * math.sqrt(13), 2.0 * math.sqrt(74)], rtol=1e-14)
+
+
+def test_gelu_form_scalar_values(oracle):
+    """One neuron, one input: y = gelu(g) * u.  Checked against the tanh formula typed out for a few
+    points, and against the erf form of GELU, which the tanh form approximates to within 5e-4."""
+    for g in (-3.0, -1.0, -0.25, 0.0, 0.5, 1.0, 2.5):
+        W_in = np.array([[g]], np.float32)
+        V_in = np.array([[1.5]], np.float32)
+        W_out = np.array([[1.0]], np.float32)
+        y = oracle.dense_ffn(np.array([1.0], np.float32), W_in, V_in, W_out, act=1)[0]
+        tanh_form = 0.5 * g * (1.0 + math.tanh(math.sqrt(2.0 / math.pi) * (g + 0.044715 * g ** 3))) * 1.5
+        erf_form = 0.5 * g * (1.0 + math.erf(g / math.sqrt(2.0))) * 1.5
+        assert abs(y - tanh_form) < 1e-15 and abs(y - erf_form) < 7.5e-4
+
+
+@pytest.mark.parametrize("act", [1, 2])
+def test_variant_cett_curve_matches_definition(oracle, act):
+    rng = np.random.default_rng(40 + act)
+    T, F = 5, 9
+    X, Wg, Wu, Wd = _layer(rng, d=8, F=F, T=T)
+    V = None if act == 2 else Wu
+    A, order, cett = oracle.cett_curve(X, Wg, V, Wd, act=act)
+    np.testing.assert_allclose(A, oracle.neuron_scores(X, [0, T], Wg, V, Wd, act=act)[0], rtol=1e-12)
+    a = np.sort(A)
+    for k in range(F + 1):
+        eps = a[0] * 0.5 if k == 0 else (np.inf if k == F else 0.5 * (a[k - 1] + a[k]))
+        num = den = 0.0
+        for t in range(T):
+            y_d = oracle.dense_ffn(X[t], Wg, V, Wd, act=act)
+            y_s, _, _ = oracle.sparse_ffn(X[t], Wg, V, Wd, A, eps, act=act)
+            num += float(np.sum((y_d - y_s) ** 2))
+            den += float(np.sum(y_d ** 2))
+        assert abs(cett[k] - math.sqrt(num / den)) < 1e-10
