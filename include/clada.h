@@ -60,7 +60,17 @@ typedef enum {
                                           re-initialise the workspace before reusing it */
 } clada_status;
 
-/* One gated FFN layer.  Neuron j owns row j of each matrix, so its three
+/* FFN form of a layer: the value z of neuron j for a token x from g = w_gate_j . x
+ * and u = w_up_j . x (Eq. neuron_activation with the sigma of the model family,
+ * Section 4.1).  The non-gated form has no w_up (pass NULL) and streams one
+ * row fewer per neuron; biases are not part of the equation and are not applied. */
+typedef enum {
+    CLADA_ACT_SILU_GATED = 0, /* z = silu(g) * u                      (LLaMA, Mistral) */
+    CLADA_ACT_GELU_GATED = 1, /* z = gelu(g) * u, tanh form of GELU   (Gemma)          */
+    CLADA_ACT_RELU = 2        /* z = max(g, 0)                        (OPT)            */
+} clada_activation;
+
+/* One FFN layer.  Neuron j owns row j of each matrix, so its three
  * vectors are contiguous: w_gate row j = W_in,j, w_up row j = V_in,j,
  * w_down_t row j = column j of the output projection W_out
  * (text under Eq. neuron_activation). */
@@ -68,9 +78,9 @@ typedef struct clada_layer {
     int32_t d_model;          /* multiple of 8; <= 8192 (bf16) or 4096 (fp32) */
     int32_t d_ff;
     int32_t dtype;            /* clada_dtype of the weights and of x / X */
-    int32_t reserved;         /* set to 0 */
+    int32_t activation;       /* clada_activation; 0 = SiLU-gated */
     const void *w_gate;       /* [d_ff, d_model] */
-    const void *w_up;         /* [d_ff, d_model] */
+    const void *w_up;         /* [d_ff, d_model]; NULL for CLADA_ACT_RELU */
     const void *w_down_t;     /* [d_ff, d_model] */
     const float *w_down_norm; /* [d_ff] ||W_out,j||_2 (clada_down_norms); needed by the prefix calls only */
 } clada_layer;

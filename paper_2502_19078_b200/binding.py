@@ -34,7 +34,7 @@ class CladaError(RuntimeError):
 
 class _CLayer(ctypes.Structure):
     _fields_ = [("d_model", ctypes.c_int32), ("d_ff", ctypes.c_int32), ("dtype", ctypes.c_int32),
-                ("reserved", ctypes.c_int32), ("w_gate", ctypes.c_void_p), ("w_up", ctypes.c_void_p),
+                ("activation", ctypes.c_int32), ("w_gate", ctypes.c_void_p), ("w_up", ctypes.c_void_p),
                 ("w_down_t", ctypes.c_void_p), ("w_down_norm", ctypes.c_void_p)]
 
 
@@ -118,21 +118,32 @@ def _stream(stream) -> Optional[int]:
     return stream.cuda_stream
 
 
-class Layer:
-    """One gated FFN layer in the library's neuron-major layout (keeps the tensors alive)."""
+# clada_activation of include/clada.h
+ACT_SILU_GATED, ACT_GELU_GATED, ACT_RELU = 0, 1, 2
 
-    def __init__(self, w_gate: torch.Tensor, w_up: torch.Tensor, w_down_t: torch.Tensor,
-                 w_down_norm: Optional[torch.Tensor] = None):
+
+class Layer:
+    """One FFN layer in the library's neuron-major layout (keeps the tensors alive).
+    ``activation`` is a clada_activation; the non-gated ReLU form takes ``w_up=None``."""
+
+    def __init__(self, w_gate: torch.Tensor, w_up: Optional[torch.Tensor], w_down_t: torch.Tensor,
+                 w_down_norm: Optional[torch.Tensor] = None, activation: int = ACT_SILU_GATED):
         d_ff, d_model = w_gate.shape
-        if w_up.shape != (d_ff, d_model) or w_down_t.shape != (d_ff, d_model):
+        if activation == ACT_RELU:
+            if w_up is not None:
+                raise CladaError("the non-gated form has no w_up")
+        elif w_up is None or w_up.shape != (d_ff, d_model) or w_up.dtype != w_gate.dtype:
+            raise CladaError("w_up must be [d_ff, d_model] of the weights' dtype")
+        if w_down_t.shape != (d_ff, d_model):
             raise CladaError("w_gate, w_up, w_down_t must all be [d_ff, d_model]")
-        if not (w_gate.dtype == w_up.dtype == w_down_t.dtype):
+        if w_gate.dtype != w_down_t.dtype:
             raise CladaError("weights must share one dtype")
         self.d_model, self.d_ff = int(d_model), int(d_ff)
         self.dtype = w_gate.dtype
+        self.activation = int(activation)
         self.w_gate, self.w_up, self.w_down_t = w_gate, w_up, w_down_t
         self.w_down_norm = w_down_norm
-        self.c = _CLayer(self.d_model, self.d_ff, _dtype_code(self.dtype), 0,
+        self.c = _CLayer(self.d_model, self.d_ff, _dtype_code(self.dtype), self.activation,
                          _ptr(w_gate, name="w_gate"), _ptr(w_up, name="w_up"),
                          _ptr(w_down_t, name="w_down_t"),
                          _ptr(w_down_norm, torch.float32, "w_down_norm"))

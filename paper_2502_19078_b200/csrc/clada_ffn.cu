@@ -34,12 +34,13 @@ struct FfnParams {
     WsCtrl *ctrl;
     int32_t *status;
     int d_model, d_ff;
+    int act;              // clada_activation of the layer
 };
 
 constexpr int G = 4;                          // neurons per CTA-wide reduction
 constexpr int kMaxBatches = 4;                // prologue batches: d_ff <= 4 * 32 * kFfnThreads
 
-template <typename T, int NV>
+template <typename T, int NV, bool GATED>
 __global__ void __launch_bounds__(kFfnThreads, 1)
 sparse_ffn_kernel(const FfnParams p, const int n_stages) {
     constexpr int E = Elem<T>::kPerVec;
@@ -50,7 +51,9 @@ sparse_ffn_kernel(const FfnParams p, const int n_stages) {
     const int F = p.d_ff, d = p.d_model;
     const int vpr = d / E;  // 16-byte vectors per row
     const uint32_t row_bytes = (uint32_t)vpr * 16u;
-    const uint32_t stage_bytes = 3u * row_bytes;
+    constexpr uint32_t kRows = GATED ? 3u : 2u;  // gate | up | down, or gate | down without a gate projection
+    const uint32_t stage_bytes = kRows * row_bytes;
+    const uint32_t down_off = (kRows - 1u) * row_bytes;
     const int chunks = (F + kWarp - 1) / kWarp;
 
     // dynamic shared memory: ring | full[kMaxStages] | empty[kMaxStages] | keep-bits | kept list
@@ -236,8 +239,8 @@ sparse_ffn_kernel(const FfnParams p, const int n_stages) {
                 const uint32_t dst = ring + (uint32_t)s * stage_bytes, bar = full0 + 8 * s;
                 mbar_expect_tx(bar, stage_bytes);
                 bulk_load_row_hint(dst, Wg + off, row_bytes, bar, stream_policy);
-                bulk_load_row_hint(dst + row_bytes, Wu + off, row_bytes, bar, stream_policy);
-                bulk_load_row_hint(dst + 2 * row_bytes, Wd + off, row_bytes, bar, stream_policy);
+                if (GATED) bulk_load_row_hint(dst + row_bytes, Wu + off, row_bytes, bar, stream_policy);
+                bulk_load_row_hint(dst + down_off, Wd + off, row_bytes, bar, stream_policy);
                 issued = i + 1;
                 if (++s == n_stages) {
                     s = 0;
@@ -281,11 +284,11 @@ sparse_ffn_kernel(const FfnParams p, const int n_stages) {
                         const uint32_t a = st_addr[g] + (uint32_t)(tid + k * kConsumers) * 16u;
                         float2 fg[P], fu[P];
                         Pairs<T>::unpack(lds128(a), fg);
-                        Pairs<T>::unpack(lds128(a + row_bytes), fu);
+                        if (GATED) Pairs<T>::unpack(lds128(a + row_bytes), fu);
 #pragma unroll
                         for (int e = 0; e < P; ++e) {
                             sg = __ffma2_rn(fg[e], xr[k][e], sg);
-                            su = __ffma2_rn(fu[e], xr[k][e], su);
+                            if (GATED) su = __ffma2_rn(fu[e], xr[k][e], su);
                         }
                     }
                 }
@@ -321,7 +324,7 @@ sparse_ffn_kernel(const FfnParams p, const int n_stages) {
                 tot += __shfl_xor_sync(0xffffffffu, tot, 2);
             }
             const float up = __shfl_xor_sync(0xffffffffu, tot, 4);  // value 2g+1 sits 4 lanes above value 2g
-            const float hval = silu_f(tot) * up;                    // meaningful on lanes 8g..8g+3
+            const float hval = neuron_value_f(p.act, tot, up);          // meaningful on lanes 8g..8g+3
 #pragma unroll
             for (int g = 0; g < G; ++g) {
                 const float h = __shfl_sync(0xffffffffu, hval, 8 * g);
@@ -331,7 +334,7 @@ sparse_ffn_kernel(const FfnParams p, const int n_stages) {
                 for (int k = 0; k < NV; ++k) {
                     if (!vok[k]) continue;
                     float2 fd[P];
-                    Pairs<T>::unpack(lds128(st_addr[g] + 2 * row_bytes + (uint32_t)(tid + k * kConsumers) * 16u), fd);
+                    Pairs<T>::unpack(lds128(st_addr[g] + down_off + (uint32_t)(tid + k * kConsumers) * 16u), fd);
 #pragma unroll
                     for (int e = 0; e < P; ++e) acc[k][e] = __ffma2_rn(h2, fd[e], acc[k][e]);
                 }
@@ -397,15 +400,15 @@ sparse_ffn_kernel(const FfnParams p, const int n_stages) {
 
 // ---- host side ------------------------------------------------------------------------------
 
-template <typename T, int NV>
+template <typename T, int NV, bool GATED>
 static int launch_variant(const FfnParams &p, cudaStream_t st) {
     constexpr int E = Elem<T>::kPerVec;
     static bool configured[64] = {};
     DeviceInfo di;
     int rc = device_info(&di);
     if (rc != CLADA_OK) return rc;
-    auto kern = sparse_ffn_kernel<T, NV>;
-    const size_t stage_bytes = 3 * (size_t)(p.d_model / E) * 16;
+    auto kern = sparse_ffn_kernel<T, NV, GATED>;
+    const size_t stage_bytes = (GATED ? 3 : 2) * (size_t)(p.d_model / E) * 16;
     const size_t tail = 2 * kMaxStages * sizeof(uint64_t) + (size_t)((p.d_ff + 31) / 32) * sizeof(unsigned) +
                         (size_t)(p.d_ff / di.num_sms + 2) * sizeof(int);
     const size_t budget = (size_t)di.max_smem_optin - 2048;  // leave room for the static arrays
@@ -441,8 +444,9 @@ static int launch_ffn(const FfnParams &p, cudaStream_t st) {
     constexpr int E = Elem<T>::kPerVec;
     const int vpr = p.d_model / E;
     if (p.d_ff > kMaxBatches * kWarp * kFfnThreads) return CLADA_ERR_UNSUPPORTED;
-    if (vpr <= kConsumers) return launch_variant<T, 1>(p, st);
-    if (vpr <= 2 * kConsumers) return launch_variant<T, 2>(p, st);
+    const bool gated = act_is_gated(p.act);
+    if (vpr <= kConsumers) return gated ? launch_variant<T, 1, true>(p, st) : launch_variant<T, 1, false>(p, st);
+    if (vpr <= 2 * kConsumers) return gated ? launch_variant<T, 2, true>(p, st) : launch_variant<T, 2, false>(p, st);
     return CLADA_ERR_UNSUPPORTED;
 }
 
@@ -506,6 +510,7 @@ static int decode_with_workspace(const clada_layer *layer, const void *x, int32_
         p.status = status;
         p.d_model = layer->d_model;
         p.d_ff = layer->d_ff;
+        p.act = layer->activation;
         rc = layer->dtype == CLADA_F32 ? launch_ffn<float>(p, st) : launch_ffn<__nv_bfloat16>(p, st);
         if (rc != CLADA_OK) return rc;
         ++b;

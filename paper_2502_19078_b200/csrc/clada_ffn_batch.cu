@@ -28,6 +28,7 @@ struct FfnBatchParams {
     WsCtrl *ctrl;
     int32_t *status;
     int d_model, d_ff;
+    int act;                 // clada_activation of the layer
 };
 
 constexpr int kBatchMaxBatches = 4;  // prologue batches: d_ff <= 4 * 32 * kFfnThreads
@@ -45,7 +46,10 @@ sparse_ffn_batch_kernel(const FfnBatchParams p, const int n_stages) {
     const int F = p.d_ff, d = p.d_model;
     const int vpr = d / E;
     const uint32_t row_bytes = (uint32_t)vpr * 16u;
-    const uint32_t stage_bytes = 3u * row_bytes;
+    const bool gated = act_is_gated(p.act);
+    const uint32_t n_rows = gated ? 3u : 2u;  // gate | up | down, or gate | down without a gate projection
+    const uint32_t stage_bytes = n_rows * row_bytes;
+    const uint32_t down_off = (n_rows - 1u) * row_bytes;
     const int chunks = (F + kWarp - 1) / kWarp;
     const int list_cap = F / n_ctas + 2;
 
@@ -204,8 +208,8 @@ sparse_ffn_batch_kernel(const FfnBatchParams p, const int n_stages) {
                 const uint32_t dst = ring + (uint32_t)s * stage_bytes, bar = full0 + 8 * s;
                 mbar_expect_tx(bar, stage_bytes);
                 bulk_load_row_hint(dst, Wg + off, row_bytes, bar, stream_policy);
-                bulk_load_row_hint(dst + row_bytes, Wu + off, row_bytes, bar, stream_policy);
-                bulk_load_row_hint(dst + 2 * row_bytes, Wd + off, row_bytes, bar, stream_policy);
+                if (gated) bulk_load_row_hint(dst + row_bytes, Wu + off, row_bytes, bar, stream_policy);
+                bulk_load_row_hint(dst + down_off, Wd + off, row_bytes, bar, stream_policy);
                 issued = i + 1;
                 if (++s == n_stages) {
                     s = 0;
@@ -252,14 +256,21 @@ sparse_ffn_batch_kernel(const FfnBatchParams p, const int n_stages) {
                         const uint32_t a = st_addr[g] + (uint32_t)(tid + k * kConsumers) * 16u;
                         float2 fg[P], fu[P];
                         Pairs<T>::unpack(lds128(a), fg);
-                        Pairs<T>::unpack(lds128(a + row_bytes), fu);
+                        if (gated) {
+                            Pairs<T>::unpack(lds128(a + row_bytes), fu);
 #pragma unroll
-                        for (int b = 0; b < BT; ++b)
+                            for (int b = 0; b < BT; ++b)
 #pragma unroll
-                            for (int e = 0; e < P; ++e) {
-                                sg[b] = __ffma2_rn(fg[e], xr[b][k][e], sg[b]);
-                                su[b] = __ffma2_rn(fu[e], xr[b][k][e], su[b]);
-                            }
+                                for (int e = 0; e < P; ++e) {
+                                    sg[b] = __ffma2_rn(fg[e], xr[b][k][e], sg[b]);
+                                    su[b] = __ffma2_rn(fu[e], xr[b][k][e], su[b]);
+                                }
+                        } else {
+#pragma unroll
+                            for (int b = 0; b < BT; ++b)
+#pragma unroll
+                                for (int e = 0; e < P; ++e) sg[b] = __ffma2_rn(fg[e], xr[b][k][e], sg[b]);
+                        }
                     }
                 }
 #pragma unroll
@@ -300,7 +311,7 @@ sparse_ffn_batch_kernel(const FfnBatchParams p, const int n_stages) {
                 tot += __shfl_xor_sync(0xffffffffu, tot, 1);
             }
             const float up = __shfl_xor_sync(0xffffffffu, tot, 2);  // value 2m+1 sits 2 lanes above value 2m
-            const float hval = silu_f(tot) * up;                    // pair m = g * BT + b sits on lanes 4m, 4m+1
+            const float hval = neuron_value_f(p.act, tot, up);                    // pair m = g * BT + b sits on lanes 4m, 4m+1
 #pragma unroll
             for (int g = 0; g < GB; ++g) {
                 float h[BT];
@@ -318,7 +329,7 @@ sparse_ffn_batch_kernel(const FfnBatchParams p, const int n_stages) {
                 for (int k = 0; k < NV; ++k) {
                     if (!vok[k]) continue;
                     float2 fd[P];
-                    Pairs<T>::unpack(lds128(st_addr[g] + 2 * row_bytes + (uint32_t)(tid + k * kConsumers) * 16u), fd);
+                    Pairs<T>::unpack(lds128(st_addr[g] + down_off + (uint32_t)(tid + k * kConsumers) * 16u), fd);
 #pragma unroll
                     for (int b = 0; b < BT; ++b)
 #pragma unroll
@@ -397,7 +408,7 @@ static int launch_batch_variant(const FfnBatchParams &p, cudaStream_t st) {
     int rc = device_info(&di);
     if (rc != CLADA_OK) return rc;
     auto kern = sparse_ffn_batch_kernel<T, NV, BT>;
-    const size_t stage_bytes = 3 * (size_t)(p.d_model / E) * 16;
+    const size_t stage_bytes = (act_is_gated(p.act) ? 3 : 2) * (size_t)(p.d_model / E) * 16;
     const size_t chunks = (size_t)(p.d_ff + 31) / 32;
     const size_t tail = 2 * kMaxStages * sizeof(uint64_t) + (1 + BT) * chunks * sizeof(unsigned) +
                         2 * (size_t)(p.d_ff / di.num_sms + 2) * sizeof(int);
@@ -456,6 +467,7 @@ int launch_ffn_batch(const clada_layer *layer, int bt, const void *x, const floa
     p.status = status;
     p.d_model = layer->d_model;
     p.d_ff = layer->d_ff;
+    p.act = layer->activation;
     const bool f32 = layer->dtype == CLADA_F32;
     const int vpr = layer->d_model / (f32 ? 4 : 8);
     if (bt == 4 && vpr <= kConsumers)

@@ -19,7 +19,7 @@ template <typename T>
 __global__ void __launch_bounds__(kPfThreads)
 prefix_partials_kernel(const T *__restrict__ X, const T *__restrict__ Wg, const T *__restrict__ Wu,
                        int d_model, int d_ff, const SeqTable tab, float *__restrict__ partials,
-                       float *__restrict__ zt, long long zt_stride) {
+                       float *__restrict__ zt, long long zt_stride, int act) {
     constexpr int E = Elem<T>::kPerVec;
     __shared__ __align__(16) float Xs[BK][BM + 4];
     __shared__ __align__(16) float Gs[BK][BN + 4];
@@ -50,7 +50,7 @@ prefix_partials_kernel(const T *__restrict__ X, const T *__restrict__ Wg, const 
             if (kin && t0 + r < t1) qx = *reinterpret_cast<const uint4 *>(X + (size_t)(t0 + r) * d_model + k0 + c);
             if (kin && n0 + r < d_ff) {
                 qg = *reinterpret_cast<const uint4 *>(Wg + (size_t)(n0 + r) * d_model + k0 + c);
-                qu = *reinterpret_cast<const uint4 *>(Wu + (size_t)(n0 + r) * d_model + k0 + c);
+                if (Wu) qu = *reinterpret_cast<const uint4 *>(Wu + (size_t)(n0 + r) * d_model + k0 + c);  // null: no gate projection
             }
             Elem<T>::unpack(qx, fx);
             Elem<T>::unpack(qg, fg);
@@ -88,7 +88,7 @@ prefix_partials_kernel(const T *__restrict__ X, const T *__restrict__ Wg, const 
         float s = 0.f;
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-            const float z = silu_f(ag[i][j]) * au[i][j];  // padded token rows give exactly 0
+            const float z = neuron_value_f(act, ag[i][j], au[i][j]);  // padded token rows give exactly 0
             s = fmaf(z, z, s);
             const long long t = t0 + ty * 4 + i;
             if (zt && t < t1 && n0 + tx * 4 + j < d_ff) zt[(size_t)(n0 + tx * 4 + j) * zt_stride + t] = z;
@@ -177,7 +177,7 @@ __global__ void __launch_bounds__(kRefThreads)
 guard_refine_kernel(const T *__restrict__ X, const T *__restrict__ Wg, const T *__restrict__ Wu,
                     const T *__restrict__ Wd_t, int d_model, int d_ff, const SeqTable tab,
                     const int *__restrict__ n_cand, const int2 *__restrict__ cand,
-                    float *__restrict__ scores) {
+                    float *__restrict__ scores, int act) {
     constexpr int E = Elem<T>::kPerVec;
     constexpr int kWarps = kRefThreads / kWarp;
     extern __shared__ __align__(16) double s_rows[];  // gate row | up row, fp64
@@ -194,7 +194,12 @@ guard_refine_kernel(const T *__restrict__ X, const T *__restrict__ Wg, const T *
         for (int v = threadIdx.x; v < vpr; v += kRefThreads) {
             double g[E], u[E];
             Widen<T>::run(wg[v], g);
-            Widen<T>::run(wu[v], u);
+            if (Wu) {
+                Widen<T>::run(wu[v], u);
+            } else {  // no gate projection: the u factor is not used
+#pragma unroll
+                for (int e = 0; e < E; ++e) u[e] = 0.0;
+            }
 #pragma unroll
             for (int e = 0; e < E; ++e) {  // element-major: lanes then read consecutive doubles
                 s_rows[e * vpr + v] = g[e];
@@ -218,7 +223,7 @@ guard_refine_kernel(const T *__restrict__ X, const T *__restrict__ Wg, const T *
             }
             g = warp_sum(g);
             u = warp_sum(u);
-            const double z = g / (1.0 + exp(-g)) * u;
+            const double z = neuron_value_d(act, g, u);
             zz += z * z;
         }
         double nn = 0.0;
@@ -275,7 +280,7 @@ static int run_scores(const clada_layer *L, const void *X, const SeqTable &tab, 
         dim3 grid((L->d_ff + BN - 1) / BN, n_mtiles);
         prefix_partials_kernel<T><<<grid, kPfThreads, 0, st>>>(
             static_cast<const T *>(X), static_cast<const T *>(L->w_gate), static_cast<const T *>(L->w_up),
-            L->d_model, L->d_ff, tab, partials, zt, zt_stride);
+            L->d_model, L->d_ff, tab, partials, zt, zt_stride, L->activation);
         CLADA_CUDA_TRY(cudaGetLastError());
     }
     return launch_prefix_finalize(partials, tab, BM, L->d_ff, L->w_down_norm, scores, st);
@@ -381,12 +386,12 @@ int clada_refine_scores(const clada_layer *layer, const void *X, const int64_t *
         guard_refine_kernel<float><<<grid, kRefThreads, rows_smem, st>>>(
             static_cast<const float *>(X), static_cast<const float *>(layer->w_gate),
             static_cast<const float *>(layer->w_up), static_cast<const float *>(layer->w_down_t),
-            layer->d_model, layer->d_ff, tab, n_cand, cand, scores);
+            layer->d_model, layer->d_ff, tab, n_cand, cand, scores, layer->activation);
     else
         guard_refine_kernel<__nv_bfloat16><<<grid, kRefThreads, rows_smem, st>>>(
             static_cast<const __nv_bfloat16 *>(X), static_cast<const __nv_bfloat16 *>(layer->w_gate),
             static_cast<const __nv_bfloat16 *>(layer->w_up), static_cast<const __nv_bfloat16 *>(layer->w_down_t),
-            layer->d_model, layer->d_ff, tab, n_cand, cand, scores);
+            layer->d_model, layer->d_ff, tab, n_cand, cand, scores, layer->activation);
     CLADA_CUDA_TRY(cudaGetLastError());
     return CLADA_OK;
 }

@@ -42,6 +42,7 @@ struct TcParams {
     int n_ttiles;   // token tiles over all prompts
     float *partials;  // [n_ttiles, d_ff]
     int32_t *status;
+    int act;        // clada_activation; the non-gated form skips the w_up tiles and their MMAs
     SeqTable tab;
 };
 
@@ -132,6 +133,7 @@ prefix_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int n_items = p.n_ntiles * p.n_ttiles;
     const int n_kblocks = (p.d_model + kTcTileK - 1) / kTcTileK;
+    const bool gated = act_is_gated(p.act);
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kTcStages; ++s) {
@@ -175,9 +177,9 @@ prefix_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                     }
                     const uint32_t bar = tc_smem_u32(&s_full[s]);
                     const uint32_t dst = smem0 + (uint32_t)s * kTcStageBytes;
-                    tc_mbar_expect_tx(bar, kTcStageBytes);
+                    tc_mbar_expect_tx(bar, gated ? kTcStageBytes : 2 * kTcTileBytes);
                     tc_tma_load(dst, &map_wg, kb * kTcTileK, ntile * kTcTileM, bar);
-                    tc_tma_load(dst + kTcTileBytes, &map_wu, kb * kTcTileK, ntile * kTcTileM, bar);
+                    if (gated) tc_tma_load(dst + kTcTileBytes, &map_wu, kb * kTcTileK, ntile * kTcTileM, bar);
                     tc_tma_load(dst + 2 * kTcTileBytes, &map_x, kb * kTcTileK, (int)t0, bar);
                 }
             }
@@ -218,7 +220,7 @@ prefix_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                         // advancing K by 16 bf16 = 32 bytes = 2 descriptor units inside the swizzled row
                         const uint32_t acc = (kb > 0 || k > 0) ? 1u : 0u;
                         tc_mma(d_gate, dg + 2 * k, dx + 2 * k, acc);
-                        tc_mma(d_up, du + 2 * k, dx + 2 * k, acc);
+                        if (gated) tc_mma(d_up, du + 2 * k, dx + 2 * k, acc);
                     }
                     tc_commit(tc_smem_u32(&s_empty[s]));  // the stage is free once these MMAs have read it
                 }
@@ -249,12 +251,17 @@ prefix_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
             for (int c0 = 0; c0 < ncols; c0 += 16) {  // uniform per warp: ncols is
                 uint32_t rg[16], ru[16];
                 tc_ld16(t_gate + c0, rg);
-                tc_ld16(t_up + c0, ru);
+                if (gated) {
+                    tc_ld16(t_up + c0, ru);
+                } else {
+#pragma unroll
+                    for (int c = 0; c < 16; ++c) ru[c] = 0u;
+                }
                 tc_wait_ld();
 #pragma unroll
                 for (int c = 0; c < 16; ++c) {
                     if (c0 + c < ncols) {
-                        const float z = silu_f(__uint_as_float(rg[c])) * __uint_as_float(ru[c]);
+                        const float z = neuron_value_f(p.act, __uint_as_float(rg[c]), __uint_as_float(ru[c]));
                         sum = fmaf(z, z, sum);
                     }
                 }
@@ -330,7 +337,9 @@ int run_prefix_partials_tc(const clada_layer *layer, const void *X, const SeqTab
     CUtensorMap map_x, map_wg, map_wu;
     if ((rc = make_map(enc, &map_x, X, T_total, layer->d_model)) != CLADA_OK) return rc;
     if ((rc = make_map(enc, &map_wg, layer->w_gate, layer->d_ff, layer->d_model)) != CLADA_OK) return rc;
-    if ((rc = make_map(enc, &map_wu, layer->w_up, layer->d_ff, layer->d_model)) != CLADA_OK) return rc;
+    // without a gate projection the w_up map is never used by the kernel: give it w_gate's address
+    const void *wu = act_is_gated(layer->activation) ? layer->w_up : layer->w_gate;
+    if ((rc = make_map(enc, &map_wu, wu, layer->d_ff, layer->d_model)) != CLADA_OK) return rc;
     TcParams p;
     p.d_model = layer->d_model;
     p.d_ff = layer->d_ff;
@@ -338,6 +347,7 @@ int run_prefix_partials_tc(const clada_layer *layer, const void *X, const SeqTab
     p.n_ttiles = n_ttiles;
     p.partials = partials;
     p.status = status;
+    p.act = layer->activation;
     p.tab = tab;
     const size_t smem = (size_t)kTcStages * kTcStageBytes + 1024;
     if (!configured[di.device & 63]) {

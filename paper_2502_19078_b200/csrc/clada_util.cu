@@ -20,13 +20,16 @@ int cuda_fail(cudaError_t e, const char *where) {
 }
 
 int validate_layer(const clada_layer *layer, bool need_norm) {
-    if (!layer || !layer->w_gate || !layer->w_up || !layer->w_down_t) return CLADA_ERR_NULL;
+    if (!layer || !layer->w_gate || !layer->w_down_t) return CLADA_ERR_NULL;
+    if (layer->activation < CLADA_ACT_SILU_GATED || layer->activation > CLADA_ACT_RELU) return CLADA_ERR_UNSUPPORTED;
+    const bool gated = layer->activation != CLADA_ACT_RELU;
+    if (gated && !layer->w_up) return CLADA_ERR_NULL;
     if (need_norm && !layer->w_down_norm) return CLADA_ERR_NULL;
     if (layer->dtype != CLADA_F32 && layer->dtype != CLADA_BF16) return CLADA_ERR_DTYPE;
     if (layer->d_model <= 0 || layer->d_ff <= 0 || layer->d_model % 8 != 0) return CLADA_ERR_SHAPE;
     const int max_d = layer->dtype == CLADA_BF16 ? kMaxDModel : kMaxDModel / 2;
     if (layer->d_model > max_d) return CLADA_ERR_UNSUPPORTED;
-    if (!aligned16(layer->w_gate) || !aligned16(layer->w_up) || !aligned16(layer->w_down_t))
+    if (!aligned16(layer->w_gate) || (gated && !aligned16(layer->w_up)) || !aligned16(layer->w_down_t))
         return CLADA_ERR_ALIGN;
     return CLADA_OK;
 }

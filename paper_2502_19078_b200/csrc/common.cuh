@@ -98,6 +98,31 @@ __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepc
 // silu(g) = g / (1 + exp(-g)); expf keeps full fp32 accuracy.
 __device__ __forceinline__ float silu_f(float g) { return g / (1.0f + expf(-g)); }
 
+// tanh form of GELU: 0.5 g (1 + tanh(sqrt(2/pi) (g + 0.044715 g^3))).
+__device__ __forceinline__ float gelu_tanh_f(float g) {
+    const float inner = 0.7978845608028654f * (g + 0.044715f * g * g * g);
+    return 0.5f * g * (1.0f + tanhf(inner));
+}
+
+// Value of one neuron for one token from g = w_gate_j . x and u = w_up_j . x in the layer's FFN form
+// (Eq. neuron_activation with the family's sigma; the non-gated form has no u factor).
+__device__ __forceinline__ float neuron_value_f(int act, float g, float u) {
+    if (act == CLADA_ACT_GELU_GATED) return gelu_tanh_f(g) * u;
+    if (act == CLADA_ACT_RELU) return g > 0.f ? g : 0.f;
+    return silu_f(g) * u;
+}
+
+__device__ __forceinline__ double neuron_value_d(int act, double g, double u) {
+    if (act == CLADA_ACT_GELU_GATED) {
+        const double inner = 0.79788456080286535588 * (g + 0.044715 * g * g * g);
+        return 0.5 * g * (1.0 + tanh(inner)) * u;
+    }
+    if (act == CLADA_ACT_RELU) return g > 0.0 ? g : 0.0;
+    return g / (1.0 + exp(-g)) * u;
+}
+
+__host__ __device__ __forceinline__ bool act_is_gated(int act) { return act != CLADA_ACT_RELU; }
+
 #endif  // __CUDACC__
 
 }  // namespace clada

@@ -6,7 +6,7 @@ no softmax, no SiLU, no thresholds.  Both the CUDA library's tests/benchmark and
 oracle's tests take their inputs from here, so that the two sides see the same bits.
 
 Shapes follow the FFN dimensions of the models the paper evaluates (LLaMA-2-7B 4096x11008,
-LLaMA-3-8B 4096x14336, a 13B shape 5120x13824; Section 4.1) and its prompt / generation
+LLaMA-3-8B 4096x14336, a 13B shape 5120x13824, OPT-2.7B 2560x10240, Gemma-2B 2048x16384; Section 4.1) and its prompt / generation
 lengths (Section 4.2, long-context table).  The paper's trained weights and datasets are
 replaced by these draws:
 
@@ -46,6 +46,7 @@ class Workload:
     vocab: int
     logit_recipe: str        # "gauss2" | "gauss3_peak" | "temp_mix" | "gauss3"
     sparsities: Tuple[float, ...]
+    activation: int = 0      # FFN form: 0 SiLU-gated, 1 GELU-gated, 2 ReLU without a gate projection
 
     @property
     def torch_dtype(self) -> torch.dtype:
@@ -71,6 +72,11 @@ WORKLOADS: Dict[str, Workload] = {
                  "gauss3", (0.40,)),
         Workload("c5_13b_b16", 5120, 13824, "bf16", 40, 16, (256, 4096), 512, 32000,
                  "gauss3", (0.30, 0.40, 0.50, 0.60)),
+        # the other FFN forms among the evaluated families: OPT-2.7B (ReLU, no gate) and Gemma-2B (GELU-gated)
+        Workload("v1_opt_2p7b_layer", 2560, 10240, "bf16", 1, 1, (512, 512), 128, 50272, "gauss3_peak",
+                 (0.40, 0.50), activation=2),
+        Workload("v2_gemma_2b_layer", 2048, 16384, "bf16", 1, 1, (512, 512), 128, 256000, "gauss3_peak",
+                 (0.40, 0.50), activation=1),
     ]
 }
 

@@ -7,21 +7,23 @@ import torch
 from paper_2502_19078_b200 import workloads as wl
 
 
-def gpu_layer(weights, binding, dev="cuda"):
-    """binding.Layer (neuron-major, on the GPU) from a workloads.layer_weights() draw, norms included."""
+def gpu_layer(weights, binding, dev="cuda", activation=0):
+    """binding.Layer (neuron-major, on the GPU) from a workloads.layer_weights() draw, norms included.
+    The non-gated form (activation 2) leaves the drawn w_up out."""
     wg = weights["w_gate"].to(dev).contiguous()
-    wu = weights["w_up"].to(dev).contiguous()
+    wu = None if activation == 2 else weights["w_up"].to(dev).contiguous()
     wdt = weights["w_down"].to(dev).t().contiguous()      # row j = column j of W_out
-    layer = binding.Layer(wg, wu, wdt)
+    layer = binding.Layer(wg, wu, wdt, activation=activation)
     norms = torch.empty(layer.d_ff, dtype=torch.float32, device=dev)
     binding.clada_down_norms(layer, norms)
     layer.set_down_norm(norms)
     return layer
 
 
-def oracle_weights(weights):
-    """(W_in, V_in, W_out) numpy arrays in the paper's layout for the oracle."""
-    return (wl.to_numpy_bits(weights["w_gate"]), wl.to_numpy_bits(weights["w_up"]),
+def oracle_weights(weights, activation=0):
+    """(W_in, V_in, W_out) numpy arrays in the paper's layout for the oracle (V_in None when non-gated)."""
+    return (wl.to_numpy_bits(weights["w_gate"]),
+            None if activation == 2 else wl.to_numpy_bits(weights["w_up"]),
             wl.to_numpy_bits(weights["w_down"]))
 
 
