@@ -108,10 +108,13 @@ class Job:
         del weights["w_down"]
         self.layers = []
         for c in range(N_COPIES):
+            gated = w.activation != clada.ACT_RELU
+            wu = weights["w_up"] if gated else None
             if c == 0:
-                lay = clada.Layer(weights["w_gate"], weights["w_up"], wdt)
+                lay = clada.Layer(weights["w_gate"], wu, wdt, activation=w.activation)
             else:
-                lay = clada.Layer(weights["w_gate"].clone(), weights["w_up"].clone(), wdt.clone())
+                lay = clada.Layer(weights["w_gate"].clone(), wu.clone() if gated else None, wdt.clone(),
+                                  activation=w.activation)
             self.layers.append(lay)
         norms = torch.empty(w.d_ff, dtype=torch.float32, device=dev)
         clada.clada_down_norms(self.layers[0], norms)
@@ -188,7 +191,8 @@ class Job:
         return tot / self.tokens_per_step()
 
     ffn_launches_per_loop = property(lambda self: self.N)
-    prefix_flop = property(lambda self: 4.0 * self.T * self.w.d_model * self.w.d_ff)
+    # two contractions per (token, neuron) with a gate projection, one without
+    prefix_flop = property(lambda self: (2.0 if self.w.activation == 2 else 4.0) * self.T * self.w.d_model * self.w.d_ff)
     l2_note = f"inputs larger than L2: {N_COPIES} rotating copies of the layer"
     step_note = "prefix statistics + per sparsity (guard band, select, 128 x (cogload+adjust, sparse FFN))"
 
@@ -407,8 +411,10 @@ def run_ours(args):
     except Exception:
         bf16_peak, bf16_kind = 1590.0, "fallback"
     eb = w.elem_bytes
-    # algorithmic bytes of one FFN launch: three rows per kept neuron + scores + x in + y out
-    ffn_bytes = kept_base * 3 * w.d_model * eb + w.d_ff * 4 + w.d_model * eb + w.d_model * 4
+    # algorithmic bytes of one FFN launch: three rows per kept neuron (two without a gate projection)
+    # + scores + x in + y out
+    rows = 2 if w.activation == 2 else 3
+    ffn_bytes = kept_base * rows * w.d_model * eb + w.d_ff * 4 + w.d_model * eb + w.d_model * 4
     achieved = ffn_bytes / (ffn_ms * 1e-3) / 1e9
     h2d = sum(x.numel() * x.element_size() for x in host_in)
     d2h = hy.numel() * hy.element_size()
@@ -461,6 +467,9 @@ def oracle_sample(w, n_prefix, n_tokens):
         weights = wl.layer_weights(w, 0)
         _ORACLE_WEIGHTS[w.name] = tuple(wl.to_numpy_bits(weights[k]) for k in ("w_gate", "w_up", "w_down"))
     W_in, V_in, W_out = _ORACLE_WEIGHTS[w.name]
+    act = w.activation
+    if act == 2:
+        V_in = None
     scale = wl.channel_scale(w)
     T, N = w.prefix_len[0], w.n_decode
     X = wl.to_numpy_bits(wl.hidden_states(w, 0, "prefix", 0, n_prefix, "cpu", scale))
@@ -468,7 +477,7 @@ def oracle_sample(w, n_prefix, n_tokens):
     logits = wl.decode_logits(w, 0, n_tokens)
     tokens = wl.chosen_tokens(w, logits, 0)
     t0 = time.perf_counter()
-    A = orc.neuron_scores(X, [0, n_prefix], W_in, V_in, W_out)[0]
+    A = orc.neuron_scores(X, [0, n_prefix], W_in, V_in, W_out, act=act)[0]
     t_prefix = time.perf_counter() - t0
     t1 = time.perf_counter()
     sh = [orc.cogload(logits[t].numpy(), int(tokens[t])) for t in range(n_tokens)]
@@ -482,7 +491,7 @@ def oracle_sample(w, n_prefix, n_tokens):
         for t in range(n_tokens):
             tf = orc.adjust_threshold(np.array([[tau_base]], np.float32), [LAMBDA], [GAMMA], tau_s, tau_H,
                                       [sh[t][0]], [sh[t][1]])
-            orc.sparse_ffn(xs[t], W_in, V_in, W_out, A, float(tf[0, 0]))
+            orc.sparse_ffn(xs[t], W_in, V_in, W_out, A, float(tf[0, 0]), act=act)
             n_done += 1
     t_decode = time.perf_counter() - t2 + t_cog * len(w.sparsities)
     step_s = t_decode + t_prefix * (T / n_prefix) * (n_tokens / N)
@@ -533,8 +542,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-graph", dest="graph", action="store_false")
-    ap.add_argument("--workload", default=WORKLOAD, choices=[WORKLOAD, "c3_llama2_7b_stack"],
-                    help="the metric's workload (default), or the 32-layer stack for information")
+    ap.add_argument("--workload", default=WORKLOAD, choices=[WORKLOAD, "c3_llama2_7b_stack", "v1_opt_2p7b_layer", "v2_gemma_2b_layer"],
+                    help="the metric's workload (default); the 32-layer stack or the OPT- / Gemma-shaped "
+                         "layers (other FFN forms) for information")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
