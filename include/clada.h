@@ -40,7 +40,7 @@
 extern "C" {
 #endif
 
-typedef enum { CLADA_F32 = 0, CLADA_BF16 = 1 } clada_dtype;
+typedef enum { CLADA_F32 = 0, CLADA_BF16 = 1, CLADA_F16 = 2 } clada_dtype;
 
 typedef enum {
     CLADA_OK = 0,
@@ -75,7 +75,7 @@ typedef enum {
  * w_down_t row j = column j of the output projection W_out
  * (text under Eq. neuron_activation). */
 typedef struct clada_layer {
-    int32_t d_model;          /* multiple of 8; <= 8192 (bf16) or 4096 (fp32) */
+    int32_t d_model;          /* multiple of 8; <= 8192 (bf16, fp16) or 4096 (fp32) */
     int32_t d_ff;
     int32_t dtype;            /* clada_dtype of the weights and of x / X */
     int32_t activation;       /* clada_activation; 0 = SiLU-gated */
@@ -188,7 +188,7 @@ int clada_cett_curve(const clada_layer *layer, const int64_t *seq_offsets, int32
 /* Eqs. surprisal and entropy, natural log, for B vocabulary rows:
  *   P = softmax(logits[b,:]);  surprisal[b] = -log P[token_id[b]];
  *   entropy[b] = -sum_w P[w] log P[w]   (0 log 0 = 0: -inf logits allowed).
- *   logits     [B, V] with row stride row_stride elements, fp32 or bf16
+ *   logits     [B, V] with row stride row_stride elements, fp32, bf16 or fp16
  *   token_id   [B] int32
  * Out-of-range token -> surprisal NaN + CLADA_STATUS_BAD_TOKEN;
  * +inf / NaN logit -> both NaN + CLADA_STATUS_NONFINITE_LOGIT. */
@@ -220,7 +220,7 @@ int clada_cogload_adjust(const void *logits, int32_t logits_dtype, int32_t B, in
  *   y[b,:] = sum_{j in kept_b} silu(w_gate_j . x_b) * (w_up_j . x_b) * w_down_t[j,:]
  * Only the kept neurons' rows are read.  No bias, no rescaling.
  *   x        [B, d_model] in the layer's dtype
- *   y        out [B, d_model], y_dtype fp32 or bf16
+ *   y        out [B, d_model], y_dtype fp32, bf16 or fp16
  *   mask_out / idx_out / count_out: optional (NULL), as in clada_select
  * Accumulation is fp32 in a fixed order: results are bit-identical run to run.
  * The workspace must have been initialised with clada_workspace_init. */

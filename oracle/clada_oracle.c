@@ -22,8 +22,9 @@
  * example and the tanh formula typed out.  The whole of Algorithm 2 end to end has no
  * published trace: parity unpinned beyond those per-step pins.
  *
- * Element types: 0 = IEEE fp32, 1 = bfloat16 (uint16 bit patterns).  Both
- * widen to double exactly.
+ * Element types: 0 = IEEE fp32, 1 = bfloat16 (uint16 bit patterns), 2 = IEEE
+ * fp16, the type of the paper's latency runs (Efficiency Evaluation).  All widen
+ * to double exactly.
  */
 #include <math.h>
 #include <stdint.h>
@@ -33,12 +34,30 @@
 #include <omp.h>
 #endif
 
-enum { OR_F32 = 0, OR_BF16 = 1 };
+enum { OR_F32 = 0, OR_BF16 = 1, OR_F16 = 2 };
+
+/* IEEE 754 binary16 from its bit pattern: 1 sign bit, 5 exponent bits (bias
+ * 15), 10 fraction bits; exponent 0 is zero / subnormal (fraction * 2^-24),
+ * exponent 31 is inf / NaN. */
+static double half_bits_to_double(uint16_t h)
+{
+    const int sign = (h >> 15) & 1, ex = (h >> 10) & 0x1f, frac = h & 0x3ff;
+    double v;
+    if (ex == 0)
+        v = ldexp((double)frac, -24);
+    else if (ex == 31)
+        v = frac ? NAN : INFINITY;
+    else
+        v = ldexp(1.0 + (double)frac / 1024.0, ex - 15);
+    return sign ? -v : v;
+}
 
 static double elem(const void *p, int dtype, size_t i)
 {
     if (dtype == OR_F32)
         return (double)((const float *)p)[i];
+    if (dtype == OR_F16)
+        return half_bits_to_double(((const uint16_t *)p)[i]);
     uint32_t bits = ((uint32_t)((const uint16_t *)p)[i]) << 16;
     float f;
     memcpy(&f, &bits, sizeof f);
@@ -74,6 +93,13 @@ static double neuron_value(int act, double g, double u)
     default:
         return silu(g) * u;
     }
+}
+
+/* The widening itself, exposed so that a test can check every bit pattern. */
+void oracle_widen(int dtype, const void *p, int64_t n, double *out)
+{
+    for (int64_t i = 0; i < n; ++i)
+        out[i] = elem(p, dtype, (size_t)i);
 }
 
 int oracle_num_threads(void)

@@ -17,7 +17,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "clada_oracle.c")
 _LIB = os.path.join(_HERE, "libclada_oracle.so")
 
-F32, BF16 = 0, 1
+F32, BF16, F16 = 0, 1, 2
 # FFN forms (Section 4.1 model families): z = silu(g)*u, z = gelu_tanh(g)*u, z = relu(g) without V_in
 SILU_GATED, GELU_GATED, RELU = 0, 1, 2
 _lib = None
@@ -40,6 +40,8 @@ def lib():
         vp, i32, i64, dbl, f32 = (ctypes.c_void_p, ctypes.c_int, ctypes.c_int64,
                                   ctypes.c_double, ctypes.c_float)
         L.oracle_num_threads.restype = ctypes.c_int
+        L.oracle_widen.argtypes = [i32, vp, i64, vp]
+        L.oracle_widen.restype = None
         L.oracle_neuron_scores.argtypes = [i32, vp, vp, i32, i32, i32, vp, vp, vp, vp, i32]
         L.oracle_neuron_scores.restype = None
         L.oracle_neuron_scores_literal.argtypes = [i32, vp, i32, i32, i32, vp, vp, vp, vp, i32]
@@ -64,6 +66,14 @@ def lib():
     return _lib
 
 
+def widen(a: np.ndarray) -> np.ndarray:
+    """The oracle's own element widening to float64 (for the pin that checks every 16-bit pattern)."""
+    a = np.ascontiguousarray(a)
+    out = np.empty(a.size, dtype=np.float64)
+    lib().oracle_widen(_dt(a), _p(a), a.size, _p(out))
+    return out.reshape(a.shape)
+
+
 def num_threads() -> int:
     return int(lib().oracle_num_threads())
 
@@ -73,7 +83,9 @@ def _dt(a: np.ndarray) -> int:
         return F32
     if a.dtype == np.uint16:
         return BF16
-    raise TypeError(f"oracle takes float32 or uint16 (bf16 bits) arrays, got {a.dtype}")
+    if a.dtype == np.float16:
+        return F16
+    raise TypeError(f"oracle takes float32, float16 or uint16 (bf16 bits) arrays, got {a.dtype}")
 
 
 def _c(a: np.ndarray, dtype=None) -> np.ndarray:

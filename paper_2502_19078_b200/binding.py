@@ -16,7 +16,7 @@ import torch
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libclada.so")
 
-CLADA_F32, CLADA_BF16 = 0, 1
+CLADA_F32, CLADA_BF16, CLADA_F16 = 0, 1, 2
 STATUS_BAD_TOKEN, STATUS_NONFINITE_LOGIT, STATUS_TIMEOUT = 1, 2, 4
 
 _INT_RETURNING = [
@@ -95,6 +95,8 @@ def _dtype_code(t: torch.dtype) -> int:
         return CLADA_F32
     if t == torch.bfloat16:
         return CLADA_BF16
+    if t == torch.float16:
+        return CLADA_F16
     raise CladaError(f"unsupported dtype {t}")
 
 

@@ -272,10 +272,14 @@ int clada_cett_threshold_search(const clada_layer *layer, const void *X, const i
                 cett_cumulative_kernel<float><<<grid, kCumThreads, 0, st>>>(
                     zt, T_total, static_cast<const float *>(layer->w_down_t), d, F, order + (size_t)b * F, t0, t1,
                     tile_partials);
-            else
+            else if (layer->dtype == CLADA_BF16)
                 cett_cumulative_kernel<__nv_bfloat16><<<grid, kCumThreads, 0, st>>>(
                     zt, T_total, static_cast<const __nv_bfloat16 *>(layer->w_down_t), d, F, order + (size_t)b * F, t0,
                     t1, tile_partials);
+            else
+                cett_cumulative_kernel<__half><<<grid, kCumThreads, 0, st>>>(
+                    zt, T_total, static_cast<const __half *>(layer->w_down_t), d, F, order + (size_t)b * F, t0, t1,
+                    tile_partials);
             CLADA_CUDA_TRY(cudaGetLastError());
         }
         cett_reduce_kernel<<<(F + 255) / 256, 256, 0, st>>>(tile_partials, n_tiles, F, cum_b);

@@ -232,7 +232,7 @@ static int launch_cogload(const void *logits, int32_t dtype, int32_t B, int64_t 
                           const float *gamma, float tau_s, float tau_H, int L, float *tau_final,
                           void *stream) {
     if (!logits || !token_id || !surprisal || !entropy) return CLADA_ERR_NULL;
-    if (dtype != CLADA_F32 && dtype != CLADA_BF16) return CLADA_ERR_DTYPE;
+    if (!dtype_ok(dtype)) return CLADA_ERR_DTYPE;
     if (B <= 0 || V <= 0 || row_stride < V) return CLADA_ERR_SHAPE;
     if (reinterpret_cast<uintptr_t>(logits) % elem_size(dtype)) return CLADA_ERR_ALIGN;
     cudaLaunchConfig_t cfg = {};
@@ -256,11 +256,15 @@ static int launch_cogload(const void *logits, int32_t dtype, int32_t B, int64_t 
         CLADA_CUDA_TRY(cudaLaunchKernelEx(&cfg, cogload_kernel<float>, static_cast<const float *>(logits), V,
                                           row_stride, token_id, surprisal, entropy, status, tau_base, lambda, gamma,
                                           tau_s, tau_H, L, tau_final));
-    else
+    else if (dtype == CLADA_BF16)
         CLADA_CUDA_TRY(cudaLaunchKernelEx(&cfg, cogload_kernel<__nv_bfloat16>,
                                           static_cast<const __nv_bfloat16 *>(logits), V, row_stride, token_id,
                                           surprisal, entropy, status, tau_base, lambda, gamma, tau_s, tau_H, L,
                                           tau_final));
+    else
+        CLADA_CUDA_TRY(cudaLaunchKernelEx(&cfg, cogload_kernel<__half>, static_cast<const __half *>(logits), V,
+                                          row_stride, token_id, surprisal, entropy, status, tau_base, lambda, gamma,
+                                          tau_s, tau_H, L, tau_final));
     return CLADA_OK;
 }
 

@@ -388,11 +388,7 @@ sparse_ffn_kernel(const FfnParams p, const int n_stages) {
             if (p.y_dtype == CLADA_F32) {
                 reinterpret_cast<float4 *>(p.y)[q] = s;
             } else {
-                __nv_bfloat162 lo = __floats2bfloat162_rn(s.x, s.y), hi = __floats2bfloat162_rn(s.z, s.w);
-                uint2 o;
-                o.x = *reinterpret_cast<uint32_t *>(&lo);
-                o.y = *reinterpret_cast<uint32_t *>(&hi);
-                reinterpret_cast<uint2 *>(p.y)[q] = o;
+                reinterpret_cast<uint2 *>(p.y)[q] = pack4_16bit(p.y_dtype, s);
             }
         }
     }
@@ -462,7 +458,7 @@ static int decode_with_workspace(const clada_layer *layer, const void *x, int32_
     if (rc != CLADA_OK) return rc;
     if (!x || !scores || !tau_final || !y) return CLADA_ERR_NULL;
     if (B <= 0 || tau_stride < 0) return CLADA_ERR_SHAPE;
-    if (y_dtype != CLADA_F32 && y_dtype != CLADA_BF16) return CLADA_ERR_DTYPE;
+    if (!dtype_ok(y_dtype)) return CLADA_ERR_DTYPE;
     if (!aligned16(x) || !aligned16(y)) return CLADA_ERR_ALIGN;
     if (!ws || (reinterpret_cast<uintptr_t>(ws) & 255u)) return CLADA_ERR_WORKSPACE;
     DeviceInfo di;
@@ -511,7 +507,9 @@ static int decode_with_workspace(const clada_layer *layer, const void *x, int32_
         p.d_model = layer->d_model;
         p.d_ff = layer->d_ff;
         p.act = layer->activation;
-        rc = layer->dtype == CLADA_F32 ? launch_ffn<float>(p, st) : launch_ffn<__nv_bfloat16>(p, st);
+        rc = layer->dtype == CLADA_F32    ? launch_ffn<float>(p, st)
+             : layer->dtype == CLADA_BF16 ? launch_ffn<__nv_bfloat16>(p, st)
+                                          : launch_ffn<__half>(p, st);
         if (rc != CLADA_OK) return rc;
         ++b;
     }
@@ -535,7 +533,7 @@ extern "C" int clada_sparse_ffn_decode_layers(const clada_layer *layers, int32_t
                                               void *stream) {
     if (!layers || !x || !scores || !tau_final || !y) return CLADA_ERR_NULL;
     if (L <= 0 || B <= 0) return CLADA_ERR_SHAPE;
-    if (y_dtype != CLADA_F32 && y_dtype != CLADA_BF16) return CLADA_ERR_DTYPE;
+    if (!dtype_ok(y_dtype)) return CLADA_ERR_DTYPE;
     for (int l = 0; l < L; ++l) {  // validate everything before enqueueing anything
         int rc = validate_layer(&layers[l], false);
         if (rc != CLADA_OK) return rc;

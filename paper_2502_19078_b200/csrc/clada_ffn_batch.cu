@@ -387,11 +387,7 @@ sparse_ffn_batch_kernel(const FfnBatchParams p, const int n_stages) {
             if (p.y_dtype == CLADA_F32) {
                 reinterpret_cast<float4 *>(yb)[q] = s;
             } else {
-                __nv_bfloat162 lo = __floats2bfloat162_rn(s.x, s.y), hi = __floats2bfloat162_rn(s.z, s.w);
-                uint2 o;
-                o.x = *reinterpret_cast<uint32_t *>(&lo);
-                o.y = *reinterpret_cast<uint32_t *>(&hi);
-                reinterpret_cast<uint2 *>(yb)[q] = o;
+                reinterpret_cast<uint2 *>(yb)[q] = pack4_16bit(p.y_dtype, s);
             }
         }
     }
@@ -470,12 +466,19 @@ int launch_ffn_batch(const clada_layer *layer, int bt, const void *x, const floa
     p.act = layer->activation;
     const bool f32 = layer->dtype == CLADA_F32;
     const int vpr = layer->d_model / (f32 ? 4 : 8);
+    const bool f16 = layer->dtype == CLADA_F16;
     if (bt == 4 && vpr <= kConsumers)
-        return f32 ? launch_batch_variant<float, 1, 4>(p, st) : launch_batch_variant<__nv_bfloat16, 1, 4>(p, st);
+        return f32   ? launch_batch_variant<float, 1, 4>(p, st)
+               : f16 ? launch_batch_variant<__half, 1, 4>(p, st)
+                     : launch_batch_variant<__nv_bfloat16, 1, 4>(p, st);
     if (bt == 2 && vpr <= kConsumers)
-        return f32 ? launch_batch_variant<float, 1, 2>(p, st) : launch_batch_variant<__nv_bfloat16, 1, 2>(p, st);
+        return f32   ? launch_batch_variant<float, 1, 2>(p, st)
+               : f16 ? launch_batch_variant<__half, 1, 2>(p, st)
+                     : launch_batch_variant<__nv_bfloat16, 1, 2>(p, st);
     if (bt == 2 && vpr <= 2 * kConsumers)
-        return f32 ? launch_batch_variant<float, 2, 2>(p, st) : launch_batch_variant<__nv_bfloat16, 2, 2>(p, st);
+        return f32   ? launch_batch_variant<float, 2, 2>(p, st)
+               : f16 ? launch_batch_variant<__half, 2, 2>(p, st)
+                     : launch_batch_variant<__nv_bfloat16, 2, 2>(p, st);
     return CLADA_ERR_UNSUPPORTED;
 }
 

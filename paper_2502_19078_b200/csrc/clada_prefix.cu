@@ -160,6 +160,21 @@ __device__ __forceinline__ double bf16_bits_to_double(uint32_t b) {  // b: 16 si
     const uint32_t hi = ((b & 0x8000u) << 16) | ((ex + 896u) << 20) | ((b & 0x7fu) << 13);
     return __hiloint2double((int)hi, 0);
 }
+// IEEE half: 1 sign, 5 exponent (bias 15), 10 fraction bits -> double (bias 1023, fraction at bit 42 of 52).
+__device__ __forceinline__ double f16_bits_to_double(uint32_t b) {  // b: 16 significant bits
+    const uint32_t ex = (b >> 10) & 0x1fu;
+    if (ex == 0u || ex == 31u) return (double)__half2float(__ushort_as_half((unsigned short)b));
+    const uint32_t hi = ((b & 0x8000u) << 16) | ((ex + 1008u) << 20) | ((b & 0x3ffu) << 10);
+    return __hiloint2double((int)hi, 0);
+}
+template <> struct Widen<__half> {
+    __device__ static __forceinline__ void run(const uint4 &v, double (&o)[8]) {
+        o[0] = f16_bits_to_double(v.x & 0xffffu); o[1] = f16_bits_to_double(v.x >> 16);
+        o[2] = f16_bits_to_double(v.y & 0xffffu); o[3] = f16_bits_to_double(v.y >> 16);
+        o[4] = f16_bits_to_double(v.z & 0xffffu); o[5] = f16_bits_to_double(v.z >> 16);
+        o[6] = f16_bits_to_double(v.w & 0xffffu); o[7] = f16_bits_to_double(v.w >> 16);
+    }
+};
 template <> struct Widen<__nv_bfloat16> {
     __device__ static __forceinline__ void run(const uint4 &v, double (&o)[8]) {
         o[0] = bf16_bits_to_double(v.x & 0xffffu); o[1] = bf16_bits_to_double(v.x >> 16);
@@ -292,9 +307,11 @@ int run_prefix_scores_with_z(const clada_layer *layer, const void *X, const int6
     int n_mtiles = 0;
     int rc = build_table(seq_offsets, B, &tab, &n_mtiles);
     if (rc != CLADA_OK) return rc;
-    return layer->dtype == CLADA_F32
-               ? run_scores<float>(layer, X, tab, n_mtiles, scores, partials, st, zt, seq_offsets[B])
-               : run_scores<__nv_bfloat16>(layer, X, tab, n_mtiles, scores, partials, st, zt, seq_offsets[B]);
+    if (layer->dtype == CLADA_F32)
+        return run_scores<float>(layer, X, tab, n_mtiles, scores, partials, st, zt, seq_offsets[B]);
+    if (layer->dtype == CLADA_BF16)
+        return run_scores<__nv_bfloat16>(layer, X, tab, n_mtiles, scores, partials, st, zt, seq_offsets[B]);
+    return run_scores<__half>(layer, X, tab, n_mtiles, scores, partials, st, zt, seq_offsets[B]);
 }
 
 size_t prefix_partials_bytes_cuda_core(const int64_t *seq_offsets, int32_t B, int d_ff) {
@@ -333,7 +350,7 @@ int clada_prefix_scores(const clada_layer *layer, const void *X, const int64_t *
     float *partials = reinterpret_cast<float *>(static_cast<char *>(ws) + kWsCtrlBytes);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (layer->dtype == CLADA_F32) return run_scores<float>(layer, X, tab, n_mtiles, scores, partials, st);
-    // bf16: tensor cores (128-token tiles: never more partial rows than the 64-token tiling above)
+    // bf16 / fp16: tensor cores (128-token tiles: never more partial rows than the 64-token tiling above)
     rc = run_prefix_partials_tc(layer, X, tab, seq_offsets[B], partials, status, st);
     if (rc != CLADA_OK) return rc;
     return launch_prefix_finalize(partials, tab, kTcTokenTile, layer->d_ff, layer->w_down_norm, scores, st);
@@ -380,6 +397,8 @@ int clada_refine_scores(const clada_layer *layer, const void *X, const int64_t *
         CLADA_CUDA_TRY(cudaFuncSetAttribute(guard_refine_kernel<__nv_bfloat16>,
                                             cudaFuncAttributeMaxDynamicSharedMemorySize,
                                             2 * kMaxDModel * (int)sizeof(double)));
+        CLADA_CUDA_TRY(cudaFuncSetAttribute(guard_refine_kernel<__half>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                            2 * kMaxDModel * (int)sizeof(double)));
         configured[di.device & 63] = true;
     }
     if (layer->dtype == CLADA_F32)
@@ -387,10 +406,15 @@ int clada_refine_scores(const clada_layer *layer, const void *X, const int64_t *
             static_cast<const float *>(X), static_cast<const float *>(layer->w_gate),
             static_cast<const float *>(layer->w_up), static_cast<const float *>(layer->w_down_t),
             layer->d_model, layer->d_ff, tab, n_cand, cand, scores, layer->activation);
-    else
+    else if (layer->dtype == CLADA_BF16)
         guard_refine_kernel<__nv_bfloat16><<<grid, kRefThreads, rows_smem, st>>>(
             static_cast<const __nv_bfloat16 *>(X), static_cast<const __nv_bfloat16 *>(layer->w_gate),
             static_cast<const __nv_bfloat16 *>(layer->w_up), static_cast<const __nv_bfloat16 *>(layer->w_down_t),
+            layer->d_model, layer->d_ff, tab, n_cand, cand, scores, layer->activation);
+    else
+        guard_refine_kernel<__half><<<grid, kRefThreads, rows_smem, st>>>(
+            static_cast<const __half *>(X), static_cast<const __half *>(layer->w_gate),
+            static_cast<const __half *>(layer->w_up), static_cast<const __half *>(layer->w_down_t),
             layer->d_model, layer->d_ff, tab, n_cand, cand, scores, layer->activation);
     CLADA_CUDA_TRY(cudaGetLastError());
     return CLADA_OK;

@@ -42,6 +42,7 @@ struct TcParams {
     int n_ttiles;   // token tiles over all prompts
     float *partials;  // [n_ttiles, d_ff]
     int32_t *status;
+    uint32_t idesc; // instruction descriptor for the layer's element type
     int act;        // clada_activation; the non-gated form skips the w_up tiles and their MMAs
     SeqTable tab;
 };
@@ -93,15 +94,17 @@ __device__ __forceinline__ uint64_t tc_smem_desc(uint32_t addr) {
     d |= (uint64_t)2 << 61;                  // SWIZZLE_128B
     return d;
 }
-// Instruction descriptor, kind::f16: D fp32, A and B bf16, both K-major, N = 128, M = 128.
-constexpr uint32_t kTcInstrDesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kTcTileN >> 3) << 17) |
-                                  ((uint32_t)(kTcTileM >> 4) << 24);
-__device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t accumulate) {
+// Instruction descriptor, kind::f16: D fp32, A and B of one 16-bit type (format code 1 = bf16, 0 = fp16,
+// the same for both operands), both K-major, N = 128, M = 128.
+constexpr uint32_t kTcInstrDescF16 = (1u << 4) | ((uint32_t)(kTcTileN >> 3) << 17) | ((uint32_t)(kTcTileM >> 4) << 24);
+constexpr uint32_t kTcInstrDescBf16 = kTcInstrDescF16 | (1u << 7) | (1u << 10);
+__device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t accumulate,
+                                       uint32_t idesc) {
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
         "setp.ne.b32 p, %4, 0;\n\t"
         "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(kTcInstrDesc), "r"(accumulate)
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
         : "memory");
 }
 // Arrive on an mbarrier once all MMAs issued so far by this thread have completed.
@@ -219,8 +222,8 @@ prefix_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                     for (int k = 0; k < kTcTileK / 16; ++k) {
                         // advancing K by 16 bf16 = 32 bytes = 2 descriptor units inside the swizzled row
                         const uint32_t acc = (kb > 0 || k > 0) ? 1u : 0u;
-                        tc_mma(d_gate, dg + 2 * k, dx + 2 * k, acc);
-                        if (gated) tc_mma(d_up, du + 2 * k, dx + 2 * k, acc);
+                        tc_mma(d_gate, dg + 2 * k, dx + 2 * k, acc, p.idesc);
+                        if (gated) tc_mma(d_up, du + 2 * k, dx + 2 * k, acc, p.idesc);
                     }
                     tc_commit(tc_smem_u32(&s_empty[s]));  // the stage is free once these MMAs have read it
                 }
@@ -305,14 +308,15 @@ static int encode_fn(EncodeTiledFn *out) {
     return CLADA_OK;
 }
 
-// Row-major bf16 matrix [rows, cols] as a 2-D tensor map with a {64, 128} box and 128-byte swizzle;
+// Row-major bf16 or fp16 matrix [rows, cols] as a 2-D tensor map with a {64, 128} box and 128-byte swizzle;
 // out-of-range rows and columns read as zero.
-static int make_map(EncodeTiledFn enc, CUtensorMap *map, const void *base, long long rows, int cols) {
+static int make_map(EncodeTiledFn enc, CUtensorMap *map, const void *base, long long rows, int cols, int dtype) {
     const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
     const cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
     const cuuint32_t box[2] = {(cuuint32_t)kTcTileK, (cuuint32_t)kTcTileM};
     const cuuint32_t estr[2] = {1, 1};
-    const CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr,
+    const CUtensorMapDataType et = dtype == CLADA_F16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
+    const CUresult r = enc(map, et, 2, const_cast<void *>(base), dims, strides, box, estr,
                            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) {
@@ -335,11 +339,11 @@ int run_prefix_partials_tc(const clada_layer *layer, const void *X, const SeqTab
     rc = encode_fn(&enc);
     if (rc != CLADA_OK) return rc;
     CUtensorMap map_x, map_wg, map_wu;
-    if ((rc = make_map(enc, &map_x, X, T_total, layer->d_model)) != CLADA_OK) return rc;
-    if ((rc = make_map(enc, &map_wg, layer->w_gate, layer->d_ff, layer->d_model)) != CLADA_OK) return rc;
+    if ((rc = make_map(enc, &map_x, X, T_total, layer->d_model, layer->dtype)) != CLADA_OK) return rc;
+    if ((rc = make_map(enc, &map_wg, layer->w_gate, layer->d_ff, layer->d_model, layer->dtype)) != CLADA_OK) return rc;
     // without a gate projection the w_up map is never used by the kernel: give it w_gate's address
     const void *wu = act_is_gated(layer->activation) ? layer->w_up : layer->w_gate;
-    if ((rc = make_map(enc, &map_wu, wu, layer->d_ff, layer->d_model)) != CLADA_OK) return rc;
+    if ((rc = make_map(enc, &map_wu, wu, layer->d_ff, layer->d_model, layer->dtype)) != CLADA_OK) return rc;
     TcParams p;
     p.d_model = layer->d_model;
     p.d_ff = layer->d_ff;
@@ -348,6 +352,7 @@ int run_prefix_partials_tc(const clada_layer *layer, const void *X, const SeqTab
     p.partials = partials;
     p.status = status;
     p.act = layer->activation;
+    p.idesc = layer->dtype == CLADA_F16 ? kTcInstrDescF16 : kTcInstrDescBf16;
     p.tab = tab;
     const size_t smem = (size_t)kTcStages * kTcStageBytes + 1024;
     if (!configured[di.device & 63]) {

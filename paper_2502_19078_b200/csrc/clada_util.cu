@@ -25,9 +25,9 @@ int validate_layer(const clada_layer *layer, bool need_norm) {
     const bool gated = layer->activation != CLADA_ACT_RELU;
     if (gated && !layer->w_up) return CLADA_ERR_NULL;
     if (need_norm && !layer->w_down_norm) return CLADA_ERR_NULL;
-    if (layer->dtype != CLADA_F32 && layer->dtype != CLADA_BF16) return CLADA_ERR_DTYPE;
+    if (!dtype_ok(layer->dtype)) return CLADA_ERR_DTYPE;
     if (layer->d_model <= 0 || layer->d_ff <= 0 || layer->d_model % 8 != 0) return CLADA_ERR_SHAPE;
-    const int max_d = layer->dtype == CLADA_BF16 ? kMaxDModel : kMaxDModel / 2;
+    const int max_d = layer->dtype == CLADA_F32 ? kMaxDModel / 2 : kMaxDModel;
     if (layer->d_model > max_d) return CLADA_ERR_UNSUPPORTED;
     if (!aligned16(layer->w_gate) || (gated && !aligned16(layer->w_up)) || !aligned16(layer->w_down_t))
         return CLADA_ERR_ALIGN;
@@ -133,9 +133,12 @@ int clada_down_norms(const clada_layer *layer, float *out, void *stream) {
     if (layer->dtype == CLADA_F32)
         down_norms_kernel<float><<<blocks, threads, 0, st>>>(
             static_cast<const float *>(layer->w_down_t), layer->d_model, layer->d_ff, out);
-    else
+    else if (layer->dtype == CLADA_BF16)
         down_norms_kernel<__nv_bfloat16><<<blocks, threads, 0, st>>>(
             static_cast<const __nv_bfloat16 *>(layer->w_down_t), layer->d_model, layer->d_ff, out);
+    else
+        down_norms_kernel<__half><<<blocks, threads, 0, st>>>(
+            static_cast<const __half *>(layer->w_down_t), layer->d_model, layer->d_ff, out);
     CLADA_CUDA_TRY(cudaGetLastError());
     return CLADA_OK;
 }

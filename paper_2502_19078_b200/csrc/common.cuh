@@ -2,6 +2,7 @@
 #pragma once
 
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -24,6 +25,7 @@ int cuda_fail(cudaError_t e, const char *where);  // records and returns CLADA_E
 
 inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 inline size_t elem_size(int dtype) { return dtype == CLADA_F32 ? 4 : 2; }
+inline bool dtype_ok(int dtype) { return dtype == CLADA_F32 || dtype == CLADA_BF16 || dtype == CLADA_F16; }
 int validate_layer(const clada_layer *layer, bool need_norm);
 
 struct DeviceInfo {
@@ -87,6 +89,33 @@ template <> struct Elem<__nv_bfloat16> {
     }
     __device__ static __forceinline__ float to_float(__nv_bfloat16 v) { return __bfloat162float(v); }
 };
+__device__ __forceinline__ float2 half2_bits_to_float2(uint32_t w) {
+    return __half22float2(*reinterpret_cast<const __half2 *>(&w));
+}
+template <> struct Elem<__half> {
+    static constexpr int kPerVec = 8;
+    __device__ static __forceinline__ void unpack(const uint4 &v, float (&f)[8]) {
+        const float2 a = half2_bits_to_float2(v.x), b = half2_bits_to_float2(v.y), c = half2_bits_to_float2(v.z),
+                     d = half2_bits_to_float2(v.w);
+        f[0] = a.x; f[1] = a.y; f[2] = b.x; f[3] = b.y; f[4] = c.x; f[5] = c.y; f[6] = d.x; f[7] = d.y;
+    }
+    __device__ static __forceinline__ float to_float(__half v) { return __half2float(v); }
+};
+
+// Four fp32 values as four 16-bit elements of the given clada_dtype (round to nearest even).
+__device__ __forceinline__ uint2 pack4_16bit(int dtype, float4 s) {
+    uint2 o;
+    if (dtype == CLADA_BF16) {
+        __nv_bfloat162 lo = __floats2bfloat162_rn(s.x, s.y), hi = __floats2bfloat162_rn(s.z, s.w);
+        o.x = *reinterpret_cast<uint32_t *>(&lo);
+        o.y = *reinterpret_cast<uint32_t *>(&hi);
+    } else {
+        __half2 lo = __floats2half2_rn(s.x, s.y), hi = __floats2half2_rn(s.z, s.w);
+        o.x = *reinterpret_cast<uint32_t *>(&lo);
+        o.y = *reinterpret_cast<uint32_t *>(&hi);
+    }
+    return o;
+}
 
 // Programmatic dependent launch: a kernel launched with the stream-serialization attribute may start
 // while its predecessor in the stream drains; it must not touch global memory the predecessor may

@@ -130,6 +130,16 @@ template <> struct Pairs<__nv_bfloat16> {
     }
 };
 
+template <> struct Pairs<__half> {
+    static constexpr int kPairs = 4;
+    __device__ static __forceinline__ void unpack(const uint4 &v, float2 (&f)[4]) {
+        f[0] = half2_bits_to_float2(v.x);
+        f[1] = half2_bits_to_float2(v.y);
+        f[2] = half2_bits_to_float2(v.z);
+        f[3] = half2_bits_to_float2(v.w);
+    }
+};
+
 constexpr int kConsumers = 512;               // consumer threads (16 warps)
 constexpr int kConsWarps = kConsumers / kWarp;
 constexpr int kFfnThreads = kConsumers + 32;  // + one producer warp

@@ -38,7 +38,7 @@ class Workload:
     name: str
     d_model: int
     d_ff: int
-    dtype: str               # "f32" | "bf16": weights and hidden states
+    dtype: str               # "f32" | "bf16" | "f16": weights and hidden states
     n_layers: int
     batch: int
     prefix_len: Tuple[int, int]   # (lo, hi): every prefix has lo tokens if lo == hi, else U{lo..hi}
@@ -50,7 +50,7 @@ class Workload:
 
     @property
     def torch_dtype(self) -> torch.dtype:
-        return torch.float32 if self.dtype == "f32" else torch.bfloat16
+        return {"f32": torch.float32, "bf16": torch.bfloat16, "f16": torch.float16}[self.dtype]
 
     @property
     def elem_bytes(self) -> int:
@@ -195,7 +195,7 @@ def universal_threshold(values, margin: float = 1e-3) -> float:
 
 
 def to_numpy_bits(t: torch.Tensor):
-    """numpy view the oracle takes: float32 as is, bfloat16 as uint16 bit patterns."""
+    """numpy view the oracle takes: float32 and float16 as is, bfloat16 as uint16 bit patterns."""
     t = t.detach().cpu().contiguous()
     if t.dtype == torch.bfloat16:
         return t.view(torch.int16).numpy().view("uint16")

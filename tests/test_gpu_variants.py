@@ -221,3 +221,82 @@ def test_variant_layer_validation(clada):
     norms = torch.empty(w.d_ff, dtype=torch.float32, device="cuda")
     with pytest.raises(clada.CladaError):
         clada.clada_down_norms(layer, norms)
+
+
+# ---- fp16 weights and activations (the precision of the paper's latency runs) -------------------------
+
+@pytest.mark.parametrize("act", [0, 1, 2])
+@pytest.mark.parametrize("name,kw,lengths", [
+    ("c2_llama2_7b_layer", {"d_model": 256, "d_ff": 300}, [200, 0, 65, 1]),
+    ("c2_llama2_7b_layer", {"d_ff": 200}, [300]),
+])
+def test_fp16_prefix_scores(clada, oracle, act, name, kw, lengths):
+    test_variant_prefix_scores(clada, oracle, act, name, dict(kw, dtype="f16"), lengths)
+
+
+@pytest.mark.parametrize("act", [0, 1, 2])
+@pytest.mark.parametrize("name,kw,B", [
+    ("c2_llama2_7b_layer", {"d_model": 520, "d_ff": 777}, 1),
+    ("c2_llama2_7b_layer", {"d_ff": 1200}, 1),
+    ("c5_13b_b16", {"d_ff": 600}, 1),
+    ("c4_llama3_8b_b8", {"d_model": 1024, "d_ff": 1800}, 7),
+    ("c5_13b_b16", {"d_ff": 700}, 5),
+])
+def test_fp16_sparse_ffn(clada, oracle, act, name, kw, B):
+    w = wl.scaled(wl.WORKLOADS[name], dtype="f16", **kw)
+    worst, excused, mismatched, compared = _ffn_case(clada, oracle, w, act, rho=0.4, n_steps=4, B=B)
+    assert mismatched == 0 and excused <= 2
+    assert compared >= 3 * B and worst <= FFN_TOL_F32, worst
+
+
+def test_fp16_output_and_logits(clada, oracle):
+    """y written as fp16 (rounded once from the fp32 sums), and surprisal / entropy from fp16 logits."""
+    w = wl.scaled(wl.WORKLOADS["c2_llama2_7b_layer"], dtype="f16", d_model=512, d_ff=640)
+    weights = wl.layer_weights(w, 0)
+    layer = gpu_layer(weights, clada)
+    g = torch.Generator().manual_seed(3)
+    scores = (torch.rand(1, w.d_ff, generator=g) + 0.5).cuda()
+    tau = torch.empty(1, dtype=torch.float32, device="cuda")
+    clada.clada_tau_from_sparsity(scores, 0.4, tau)
+    x = wl.hidden_states(w, 0, "decode", 0, 1, "cpu", wl.channel_scale(w))
+    ws = clada.new_workspace(layer, 1, 0)
+    y32 = torch.empty(1, w.d_model, dtype=torch.float32, device="cuda")
+    y16 = torch.empty(1, w.d_model, dtype=torch.float16, device="cuda")
+    clada.clada_sparse_ffn_decode(layer, x.cuda(), scores, tau, 1, y32, ws)
+    clada.clada_sparse_ffn_decode(layer, x.cuda(), scores, tau, 1, y16, ws)
+    torch.cuda.synchronize()
+    assert torch.equal(y16, y32.to(torch.float16))            # same sums, one rounding to nearest even
+    y_or, _, _ = oracle.sparse_ffn(wl.to_numpy_bits(x[0]), *oracle_weights(weights),
+                                   scores[0].cpu().numpy().astype(np.float64), float(tau.item()))
+    assert rel_inf(y32[0].cpu().numpy(), y_or) <= FFN_TOL_F32
+    V = 50272
+    logits = (torch.randn(3, V, generator=g) * 3).to(torch.float16)
+    tokens = torch.tensor([0, V - 1, 12345], dtype=torch.int32)
+    s = torch.empty(3, device="cuda")
+    h = torch.empty(3, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    clada.clada_cogload(logits.cuda(), tokens.cuda(), s, h, status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    for b in range(3):
+        so, ho = oracle.cogload(logits[b].numpy(), int(tokens[b]))
+        assert abs(s[b].item() - so) <= 1e-4 and abs(h[b].item() - ho) <= 1e-4
+
+
+def test_fp16_threshold_search(clada, oracle):
+    w = wl.scaled(wl.WORKLOADS["c2_llama2_7b_layer"], dtype="f16", d_model=128, d_ff=200)
+    weights = wl.layer_weights(w, 0)
+    lengths = [40, 23]
+    X = _prompts(w, lengths)
+    off = wl.seq_offsets(lengths)
+    layer = gpu_layer(weights, clada)
+    ws = torch.empty(clada.clada_cett_workspace_bytes(layer, off), dtype=torch.uint8, device="cuda")
+    tau = torch.empty(1, dtype=torch.float32, device="cuda")
+    mean = torch.empty(1, dtype=torch.float32, device="cuda")
+    scores = torch.empty(len(lengths), w.d_ff, dtype=torch.float32, device="cuda")
+    clada.clada_cett_threshold_search(layer, X.cuda(), off, 0.2, tau, mean, scores, ws)
+    torch.cuda.synchronize()
+    W_in, V_in, W_out = oracle_weights(weights)
+    curves = [oracle.cett_curve(wl.to_numpy_bits(X[off[b]:off[b + 1]]), W_in, V_in, W_out) for b in range(2)]
+    tau_or, mean_or = oracle.threshold_search(np.stack([c[0] for c in curves]), np.stack([c[2] for c in curves]), 0.2)
+    assert abs(tau.item() - tau_or) <= 1e-5 * tau_or and abs(mean.item() - mean_or) <= 1e-4

@@ -492,3 +492,44 @@ def test_variant_cett_curve_matches_definition(oracle, act):
             num += float(np.sum((y_d - y_s) ** 2))
             den += float(np.sum(y_d ** 2))
         assert abs(cett[k] - math.sqrt(num / den)) < 1e-10
+
+
+# ----------------------------------------------------------------------------------------------
+# fp16 elements (the precision of the paper's latency runs)
+# ----------------------------------------------------------------------------------------------
+
+def test_fp16_and_bf16_widening_every_bit_pattern(oracle):
+    bits = np.arange(65536, dtype=np.uint32).astype(np.uint16)
+    halves = bits.view(np.float16)
+    got = oracle.widen(halves)
+    ref = halves.astype(np.float64)                       # numpy's own conversion
+    assert np.array_equal(np.isnan(got), np.isnan(ref))
+    ok = ~np.isnan(ref)
+    assert np.array_equal(got[ok], ref[ok]) and np.array_equal(np.signbit(got[ok]), np.signbit(ref[ok]))
+    got_b = oracle.widen(bits)                            # the same patterns read as bfloat16
+    ref_b = (bits.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+    okb = ~np.isnan(ref_b)
+    assert np.array_equal(np.isnan(got_b), np.isnan(ref_b)) and np.array_equal(got_b[okb], ref_b[okb])
+    # a few values typed out
+    assert oracle.widen(np.array([0x3C00, 0xC000, 0x0001, 0x7BFF, 0x3555], np.uint16).view(np.float16)).tolist() == \
+        [1.0, -2.0, 2.0 ** -24, 65504.0, 0.333251953125]
+
+
+@pytest.mark.parametrize("act", [0, 1, 2])
+def test_fp16_layer_matches_library_formulation(oracle, act):
+    rng = np.random.default_rng(50 + act)
+    T, F = 4, 36
+    X, Wg, Wu, Wd = (a.astype(np.float16) for a in _layer(rng, d=16, F=F, T=T))
+    V = None if act == 2 else Wu
+    tX, tWg, tWu, tWd = (torch.from_numpy(a.astype(np.float64)) for a in (X, Wg, Wu, Wd))
+    h = _torch_h(act, tX, tWg, tWu)
+    A = oracle.neuron_scores(X, [0, T], Wg, V, Wd, act=act)[0]
+    ref_A = torch.linalg.norm(h, dim=0) * torch.linalg.norm(tWd, dim=0)
+    np.testing.assert_allclose(A, ref_A.numpy(), rtol=1e-11, atol=1e-14)
+    for t in range(T):
+        np.testing.assert_allclose(oracle.dense_ffn(X[t], Wg, V, Wd, act=act), (h[t] @ tWd.T).numpy(),
+                                   rtol=1e-11, atol=1e-13)
+    lg = (rng.standard_normal(300) * 3).astype(np.float16)
+    s, H = oracle.cogload(lg, 7)
+    lp = torch.log_softmax(torch.from_numpy(lg.astype(np.float64)), dim=0)
+    assert abs(s + lp[7].item()) < 1e-12 and abs(H + float((lp.exp() * lp).sum())) < 1e-12
