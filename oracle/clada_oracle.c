@@ -328,6 +328,47 @@ void oracle_dense_ffn(int dtype, const void *x, int d_model, int d_ff,
     free(h);
 }
 
+/* Mask compression by nesting.  Eq. final_threshold can only produce
+ * tau_base * {1, 1+lambda, 1+gamma, 1+lambda+gamma}, and the kept set of any
+ * threshold is { j : A_j >= tau }, so every kept set is a leading part of ONE
+ * list: the neurons in descending order of score (equal scores in ascending
+ * index order).  order receives that list; counts[k] = |{ j : A_j >= taus[k] }|,
+ * so the kept set at level k is order[0 .. counts[k]).  (The paper names mask
+ * memory as a limitation and mask compression as future work; this is the
+ * plain definition of the compressed form, not an algorithm of the paper.) */
+typedef struct { double a; int32_t j; } or_rank;
+
+static int cmp_rank_desc(const void *x, const void *y)
+{
+    const or_rank *p = (const or_rank *)x, *q = (const or_rank *)y;
+    if (p->a > q->a) return -1;
+    if (p->a < q->a) return 1;
+    return (p->j > q->j) - (p->j < q->j);
+}
+
+void oracle_nested_lists(const double *scores, int d_ff, const double *taus, int n_levels,
+                         int32_t *order, int32_t *counts)
+{
+    or_rank *r = (or_rank *)malloc((size_t)d_ff * sizeof(or_rank));
+    for (int j = 0; j < d_ff; ++j) { r[j].a = scores[j]; r[j].j = j; }
+    qsort(r, (size_t)d_ff, sizeof(or_rank), cmp_rank_desc);
+    for (int j = 0; j < d_ff; ++j) order[j] = r[j].j;
+    free(r);
+    for (int k = 0; k < n_levels; ++k) {
+        int c = 0;
+        for (int j = 0; j < d_ff; ++j)
+            c += !(scores[j] < taus[k]);
+        counts[k] = c;
+    }
+}
+
+/* Which of the four thresholds Eq. final_threshold yields for a token:
+ * level = I(s > tau_s) + 2 I(H > tau_H). */
+int oracle_load_level(double surprisal, double entropy, double tau_s, double tau_H)
+{
+    return (surprisal > tau_s ? 1 : 0) + (entropy > tau_H ? 2 : 0);
+}
+
 /* Harness helper (stands in for the offline threshold search, which is an
  * input to the path): the threshold that cuts exactly k_cut = floor(rho*F+0.5)
  * neurons of an fp32 score vector, placed midway between the k_cut-th and

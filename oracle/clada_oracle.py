@@ -60,6 +60,10 @@ def lib():
         L.oracle_cett_curve.restype = None
         L.oracle_threshold_search.argtypes = [vp, vp, i32, i32, dbl, vp]
         L.oracle_threshold_search.restype = dbl
+        L.oracle_nested_lists.argtypes = [vp, i32, vp, i32, vp, vp]
+        L.oracle_nested_lists.restype = None
+        L.oracle_load_level.argtypes = [dbl, dbl, dbl, dbl]
+        L.oracle_load_level.restype = ctypes.c_int
         L.oracle_tau_from_sparsity.argtypes = [vp, i32, dbl]
         L.oracle_tau_from_sparsity.restype = f32
         _lib = L
@@ -225,3 +229,19 @@ def threshold_search(scores, cett, bound=0.2):
     mean = ctypes.c_double()
     tau = lib().oracle_threshold_search(_p(scores), _p(cett), B, d_ff, float(bound), ctypes.byref(mean))
     return float(tau), mean.value
+
+
+def nested_lists(scores, taus):
+    """(order int32 [d_ff], counts int32 [len(taus)]): neurons by descending score (ties by ascending index) and,
+    per threshold, how many of them satisfy A_j >= tau -- the kept set at level k is order[:counts[k]]."""
+    scores, taus = _c(scores, np.float64), _c(taus, np.float64)
+    order = np.empty(scores.size, dtype=np.int32)
+    counts = np.empty(taus.size, dtype=np.int32)
+    lib().oracle_nested_lists(_p(scores), scores.size, _p(taus), taus.size, _p(order), _p(counts))
+    return order, counts
+
+
+def load_level(surprisal, entropy, tau_s, tau_H) -> int:
+    """I(s > tau_s) + 2 I(H > tau_H): the index of the threshold Eq. final_threshold yields."""
+    return int(lib().oracle_load_level(float(surprisal), float(entropy), float(np.float32(tau_s)),
+                                       float(np.float32(tau_H))))

@@ -533,3 +533,62 @@ def test_fp16_layer_matches_library_formulation(oracle, act):
     s, H = oracle.cogload(lg, 7)
     lp = torch.log_softmax(torch.from_numpy(lg.astype(np.float64)), dim=0)
     assert abs(s + lp[7].item()) < 1e-12 and abs(H + float((lp.exp() * lp).sum())) < 1e-12
+
+
+# ----------------------------------------------------------------------------------------------
+# Nested index lists (the compressed form of the four masks)
+# ----------------------------------------------------------------------------------------------
+
+def test_nested_lists_equal_the_masks(oracle):
+    rng = np.random.default_rng(60)
+    for F in (1, 7, 64, 333):
+        A = rng.random(F) + 0.5
+        if F >= 7:
+            A[3] = A[5] = A[1]                       # equal scores
+        srt = np.sort(A)
+        taus = np.array([0.0, srt[F // 2], A[min(1, F - 1)], 0.5 * (srt[0] + srt[-1]), srt[-1], np.inf, srt[-1] * (1 + 1e-12)])
+        order, counts = oracle.nested_lists(A, taus)
+        assert sorted(order.tolist()) == list(range(F))                      # a permutation
+        a = A[order]
+        assert np.all(a[:-1] >= a[1:])                                       # descending
+        assert all(order[i] < order[i + 1] for i in range(F - 1) if a[i] == a[i + 1])   # ties by index
+        for k, tau in enumerate(taus):
+            mask, idx, cnt = oracle.select(A, tau)                           # the mask definition (pinned above)
+            assert counts[k] == cnt
+            assert sorted(order[:cnt].tolist()) == idx.tolist()
+        # nesting: a higher threshold keeps a leading part of a lower one's list
+        by_tau = np.argsort(taus)
+        assert all(counts[by_tau[i]] >= counts[by_tau[i + 1]] for i in range(len(taus) - 1))
+
+
+def test_load_level_indexes_the_four_thresholds(oracle):
+    lam, gam = np.float32(0.80), np.float32(0.12)
+    one = np.float32(1.0)
+    mults = [one, one + lam, one + gam, (one + lam) + gam]                   # fp32, left to right
+    tau_base = np.array([[0.731]], np.float32)
+    tau_s, tau_H = 2.0, 3.0
+    for s, H, level in [(1.0, 1.0, 0), (2.5, 1.0, 1), (1.0, 3.5, 2), (2.5, 3.5, 3),
+                        (2.0, 3.0, 0), (float("nan"), 4.0, 2)]:             # strict >, NaN compares false
+        assert oracle.load_level(s, H, tau_s, tau_H) == level
+        tf = oracle.adjust_threshold(tau_base, [lam], [gam], tau_s, tau_H, [s], [H])
+        assert tf[0, 0] == np.float32(tau_base[0, 0] * mults[level])
+    # negative coefficients (the prose reading) index the same way
+    tf = oracle.adjust_threshold(tau_base, [-0.3], [-0.1], tau_s, tau_H, [2.5], [3.5])
+    assert oracle.load_level(2.5, 3.5, tau_s, tau_H) == 3
+    assert tf[0, 0] == np.float32(tau_base[0, 0] * ((one + np.float32(-0.3)) + np.float32(-0.1)))
+
+
+def test_nested_ffn_equals_thresholded_ffn(oracle):
+    rng = np.random.default_rng(61)
+    T, F = 6, 50
+    X, Wg, Wu, Wd = _layer(rng, d=16, F=F, T=T)
+    A = oracle.neuron_scores(X, [0, T], Wg, Wu, Wd)[0]
+    tau_base = float(np.sort(A)[20])
+    taus = np.array([np.float32(tau_base) * m for m in (1.0, 1.8, 1.12, 1.92)], dtype=np.float64)
+    order, counts = oracle.nested_lists(A, taus)
+    for k in range(4):
+        y_tau, mask, cnt = oracle.sparse_ffn(X[0], Wg, Wu, Wd, A, taus[k])
+        marks = np.zeros(F)
+        marks[order[:counts[k]]] = 1.0                                       # keep exactly the listed neurons
+        y_list, mask2, cnt2 = oracle.sparse_ffn(X[0], Wg, Wu, Wd, marks, 0.5)
+        assert cnt == cnt2 == counts[k] and np.array_equal(mask, mask2) and np.array_equal(y_tau, y_list)
