@@ -56,8 +56,9 @@ typedef enum {
 typedef enum {
     CLADA_STATUS_BAD_TOKEN = 1,        /* token_id outside [0, V): surprisal = NaN */
     CLADA_STATUS_NONFINITE_LOGIT = 2,  /* +inf or NaN logit: surprisal = entropy = NaN */
-    CLADA_STATUS_TIMEOUT = 4           /* a bounded device-side wait gave up; outputs invalid,
+    CLADA_STATUS_TIMEOUT = 4,          /* a bounded device-side wait gave up; outputs invalid,
                                           re-initialise the workspace before reusing it */
+    CLADA_STATUS_BAD_INDEX = 8         /* a nested-list level, count or neuron index was out of range (clamped) */
 } clada_status;
 
 /* FFN form of a layer: the value z of neuron j for a token x from g = w_gate_j . x
@@ -267,6 +268,55 @@ int clada_sparse_ffn_decode_static(const clada_layer *layer, const void *x, int3
                                    int64_t tau_stride, void *y, int32_t y_dtype,
                                    uint8_t *mask_out, int32_t *idx_out, int32_t *count_out,
                                    int32_t *status, void *stream);
+
+/* ---- Nested index lists: the masks of Eq. final_threshold in compressed form ----
+ *
+ * The paper names mask memory as a limitation and mask compression as future
+ * work (Limitations; Conclusion).  Eq. final_threshold can only yield
+ * tau_base * m, m in {1, 1+lambda, 1+gamma, (1+lambda)+gamma}, and a kept set
+ * is { j : A_j >= tau }: all four kept sets of a sequence are leading parts of
+ * one list, its neurons in descending order of score.
+ *
+ * clada_nested_build, once per (sequence, layer) after the prefix statistics:
+ *   scores     [B, d_ff] fp32, device (clada_prefix_scores / clada_refine_scores)
+ *   tau_base   sequence b reads tau_base[b * tau_stride], device
+ *   lambda, gamma  the layer's coefficients (host values, signed)
+ *   order  out [B, d_ff] int32, device: neurons by descending score, equal
+ *              scores by ascending index
+ *   counts out [B, 4] int32, device: counts[b][k] = |{ j : A_bj >= tau_k }|,
+ *              tau_k = fl32(tau_base_b * m_k), m = {1, 1+lambda, 1+gamma,
+ *              (1+lambda)+gamma} in fp32 -- bit for bit the thresholds that
+ *              clada_adjust_threshold produces, so order[b][0 .. counts[b][k])
+ *              is exactly the kept set clada_select would give at level k.
+ *   d_ff <= 16384 (the sort runs in one CTA's shared memory); otherwise
+ *   CLADA_ERR_UNSUPPORTED.  Nothing is allocated.
+ *
+ * clada_cogload_level, per decode step: clada_cogload plus
+ *   level  out [B] int32, device: I(s > tau_s) + 2 I(H > tau_H), the same fp32
+ *              comparisons as the indicators of Eq. final_threshold (a NaN
+ *              surprisal compares false).
+ *
+ * clada_sparse_ffn_decode_nested, per decode step and layer: the sparse FFN over
+ * order[b][0 .. counts[b][level[b]]).  Same x / y / workspace / status rules as
+ * clada_sparse_ffn_decode (workspace of clada_workspace_bytes(layer, 1, 0) is
+ * enough); sequences run one launch each.  The sum over the kept neurons runs
+ * in list order split over the CTAs, so y agrees with clada_sparse_ffn_decode to
+ * rounding (fp32 sums in another order), not bit for bit.  count_out [B] or
+ * NULL receives the kept count.  A level outside 0..3, a count outside
+ * [0, d_ff] or an index outside [0, d_ff) is clamped into range, so no access
+ * leaves the layer, and CLADA_STATUS_BAD_INDEX is or-ed into *status. */
+int clada_nested_build(const float *scores, int32_t B, int32_t d_ff, const float *tau_base,
+                       int64_t tau_stride, float lambda, float gamma, int32_t *order,
+                       int32_t *counts, void *stream);
+int clada_cogload_level(const void *logits, int32_t logits_dtype, int32_t B, int64_t V,
+                        int64_t row_stride, const int32_t *token_id, float tau_s, float tau_H,
+                        float *surprisal, float *entropy, int32_t *level, int32_t *status,
+                        void *stream);
+int clada_sparse_ffn_decode_nested(const clada_layer *layer, const void *x, int32_t B,
+                                   const int32_t *order /*[B,d_ff]*/, const int32_t *counts /*[B,4]*/,
+                                   const int32_t *level /*[B]*/, void *y, int32_t y_dtype,
+                                   int32_t *count_out, void *ws, size_t ws_bytes, int32_t *status,
+                                   void *stream);
 
 #ifdef __cplusplus
 }

@@ -71,6 +71,9 @@ def load() -> ctypes.CDLL:
     L.clada_sparse_ffn_decode.argtypes = [lp, vp, i32, vp, vp, i64, vp, i32, vp, vp, vp, vp, sz, vp, vp]
     L.clada_sparse_ffn_decode_static.argtypes = [lp, vp, i32, vp, vp, i64, vp, i32, vp, vp, vp, vp, vp]
     L.clada_sparse_ffn_decode_layers.argtypes = [vp, i32, vp, i32, vp, vp, vp, i32, vp, sz, vp, vp]
+    L.clada_nested_build.argtypes = [vp, i32, i32, vp, i64, f32, f32, vp, vp, vp]
+    L.clada_cogload_level.argtypes = [vp, i32, i32, i64, i64, vp, f32, f32, vp, vp, vp, vp, vp]
+    L.clada_sparse_ffn_decode_nested.argtypes = [lp, vp, i32, vp, vp, vp, vp, i32, vp, vp, sz, vp, vp]
     L.clada_cett_workspace_bytes.argtypes = [lp, vp, i32]
     L.clada_cett_workspace_bytes.restype = sz
     L.clada_cett_threshold_search.argtypes = [lp, vp, vp, i32, f32, vp, vp, vp, vp, sz, vp, vp]
@@ -369,3 +372,33 @@ def clada_cett_curve(layer: Layer, seq_offsets, sample, ws, cum_out, order_out=N
     _check(load().clada_cett_curve(layer.ref, ctypes.addressof(off), B, int(sample), _ptr(ws, torch.uint8, "ws"),
                                    ws.numel(), _ptr(cum_out, torch.float64, "cum_out"),
                                    _ptr(order_out, torch.int32, "order_out"), _stream(stream)), "clada_cett_curve")
+
+
+def clada_nested_build(scores, tau_base, lam, gam, order, counts, tau_stride=1, stream=None) -> None:
+    """scores [B, F] fp32, tau_base (sequence b at b * tau_stride) -> order [B, F] int32, counts [B, 4] int32."""
+    B, F = scores.shape
+    _check(load().clada_nested_build(_ptr(scores, torch.float32, "scores"), B, F,
+                                     _ptr(tau_base, torch.float32, "tau_base"), int(tau_stride), float(lam),
+                                     float(gam), _ptr(order, torch.int32, "order"),
+                                     _ptr(counts, torch.int32, "counts"), _stream(stream)), "clada_nested_build")
+
+
+def clada_cogload_level(logits, token_id, tau_s, tau_H, surprisal, entropy, level, status=None, stream=None) -> None:
+    _check(load().clada_cogload_level(*_logits_args(logits), _ptr(token_id, torch.int32, "token_id"),
+                                      float(tau_s), float(tau_H), _ptr(surprisal, torch.float32, "surprisal"),
+                                      _ptr(entropy, torch.float32, "entropy"), _ptr(level, torch.int32, "level"),
+                                      _ptr(status, torch.int32, "status"), _stream(stream)), "clada_cogload_level")
+
+
+def clada_sparse_ffn_decode_nested(layer: Layer, x, order, counts, level, y, ws, count=None, status=None,
+                                   stream=None) -> None:
+    """x [B, d], order [B, F], counts [B, 4], level [B] -> y [B, d] over order[b][:counts[b][level[b]]]."""
+    B = x.shape[0] if x.dim() == 2 else 1
+    _check(load().clada_sparse_ffn_decode_nested(layer.ref, _ptr(x, layer.dtype, "x"), B,
+                                                 _ptr(order, torch.int32, "order"),
+                                                 _ptr(counts, torch.int32, "counts"),
+                                                 _ptr(level, torch.int32, "level"), _ptr(y, name="y"),
+                                                 _dtype_code(y.dtype), _ptr(count, torch.int32, "count"),
+                                                 _ptr(ws, torch.uint8, "ws"), ws.numel(),
+                                                 _ptr(status, torch.int32, "status"), _stream(stream)),
+           "clada_sparse_ffn_decode_nested")

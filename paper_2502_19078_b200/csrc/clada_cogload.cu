@@ -79,7 +79,7 @@ cogload_kernel(const T *__restrict__ logits, int64_t V, int64_t row_stride,
                float *__restrict__ entropy, int32_t *__restrict__ status,
                const float *__restrict__ tau_base, const float *__restrict__ lambda,
                const float *__restrict__ gamma, float tau_s, float tau_H, int L,
-               float *__restrict__ tau_final) {
+               float *__restrict__ tau_final, int32_t *__restrict__ level_out) {
     constexpr int E = Elem<T>::kPerVec;
     cg::cluster_group cluster = cg::this_cluster();
     const int n_slices = (int)cluster.num_blocks(), slice = (int)cluster.block_rank();
@@ -192,6 +192,8 @@ cogload_kernel(const T *__restrict__ logits, int64_t V, int64_t row_stride,
                 }
                 surprisal[b] = s;
                 entropy[b] = h;
+                // which of the four thresholds of Eq. final_threshold this token selects
+                if (level_out) level_out[b] = (s > tau_s ? 1 : 0) + (h > tau_H ? 2 : 0);
                 s_out[0] = s;
                 s_out[1] = h;
                 if (flags && status) atomicOr(status, flags);
@@ -230,7 +232,7 @@ static int launch_cogload(const void *logits, int32_t dtype, int32_t B, int64_t 
                           const int32_t *token_id, float *surprisal, float *entropy,
                           int32_t *status, const float *tau_base, const float *lambda,
                           const float *gamma, float tau_s, float tau_H, int L, float *tau_final,
-                          void *stream) {
+                          int32_t *level_out, void *stream) {
     if (!logits || !token_id || !surprisal || !entropy) return CLADA_ERR_NULL;
     if (!dtype_ok(dtype)) return CLADA_ERR_DTYPE;
     if (B <= 0 || V <= 0 || row_stride < V) return CLADA_ERR_SHAPE;
@@ -255,16 +257,16 @@ static int launch_cogload(const void *logits, int32_t dtype, int32_t B, int64_t 
     if (dtype == CLADA_F32)
         CLADA_CUDA_TRY(cudaLaunchKernelEx(&cfg, cogload_kernel<float>, static_cast<const float *>(logits), V,
                                           row_stride, token_id, surprisal, entropy, status, tau_base, lambda, gamma,
-                                          tau_s, tau_H, L, tau_final));
+                                          tau_s, tau_H, L, tau_final, level_out));
     else if (dtype == CLADA_BF16)
         CLADA_CUDA_TRY(cudaLaunchKernelEx(&cfg, cogload_kernel<__nv_bfloat16>,
                                           static_cast<const __nv_bfloat16 *>(logits), V, row_stride, token_id,
                                           surprisal, entropy, status, tau_base, lambda, gamma, tau_s, tau_H, L,
-                                          tau_final));
+                                          tau_final, level_out));
     else
         CLADA_CUDA_TRY(cudaLaunchKernelEx(&cfg, cogload_kernel<__half>, static_cast<const __half *>(logits), V,
                                           row_stride, token_id, surprisal, entropy, status, tau_base, lambda, gamma,
-                                          tau_s, tau_H, L, tau_final));
+                                          tau_s, tau_H, L, tau_final, level_out));
     return CLADA_OK;
 }
 
@@ -278,7 +280,17 @@ int clada_cogload(const void *logits, int32_t logits_dtype, int32_t B, int64_t V
                   const int32_t *token_id, float *surprisal, float *entropy, int32_t *status,
                   void *stream) {
     return launch_cogload(logits, logits_dtype, B, V, row_stride, token_id, surprisal, entropy, status,
-                          nullptr, nullptr, nullptr, 0.f, 0.f, 0, nullptr, stream);
+                          nullptr, nullptr, nullptr, 0.f, 0.f, 0, nullptr, nullptr, stream);
+}
+
+// Surprisal and entropy as clada_cogload, plus the load level I(s > tau_s) + 2 I(H > tau_H) that indexes
+// the nested lists' counts (the same comparisons as Eq. final_threshold's indicators).
+int clada_cogload_level(const void *logits, int32_t logits_dtype, int32_t B, int64_t V, int64_t row_stride,
+                        const int32_t *token_id, float tau_s, float tau_H, float *surprisal, float *entropy,
+                        int32_t *level, int32_t *status, void *stream) {
+    if (!level) return CLADA_ERR_NULL;
+    return launch_cogload(logits, logits_dtype, B, V, row_stride, token_id, surprisal, entropy, status,
+                          nullptr, nullptr, nullptr, tau_s, tau_H, 0, nullptr, level, stream);
 }
 
 int clada_adjust_threshold(const float *tau_base, const float *lambda, const float *gamma, float tau_s,
@@ -302,7 +314,7 @@ int clada_cogload_adjust(const void *logits, int32_t logits_dtype, int32_t B, in
     if (!tau_base || !lambda || !gamma || !tau_final) return CLADA_ERR_NULL;
     if (L <= 0) return CLADA_ERR_SHAPE;
     return launch_cogload(logits, logits_dtype, B, V, row_stride, token_id, surprisal, entropy, status,
-                          tau_base, lambda, gamma, tau_s, tau_H, L, tau_final, stream);
+                          tau_base, lambda, gamma, tau_s, tau_H, L, tau_final, nullptr, stream);
 }
 
 }  // extern "C"

@@ -35,6 +35,11 @@ struct FfnParams {
     int32_t *status;
     int d_model, d_ff;
     int act;              // clada_activation of the layer
+    // Nested index lists instead of scores and a threshold (order != null): the kept set is
+    // order[0 .. counts[*level]), neurons in descending order of score.
+    const int32_t *order;   // [d_ff]
+    const int32_t *counts;  // [4]
+    const int32_t *level;   // one int in 0..3
 };
 
 constexpr int G = 4;                          // neurons per CTA-wide reduction
@@ -77,7 +82,14 @@ sparse_ffn_kernel(const FfnParams p, const int n_stages) {
     pdl_wait();  // everything below may read what the previous kernel wrote
 
     const uint64_t keep_policy = policy_evict_last();
-    if (tid == 0) s_tau = ld_keep(p.tau, keep_policy);  // one request per CTA, not one per warp
+    const bool nested = p.order != nullptr;
+    __shared__ int s_cnt[5];
+    if (nested) {  // the four counts and the level are independent loads: one round trip
+        if (tid < 4) s_cnt[tid] = p.counts[tid];
+        if (tid == 4) s_cnt[4] = *p.level;
+    } else if (tid == 0) {
+        s_tau = ld_keep(p.tau, keep_policy);  // one request per CTA, not one per warp
+    }
     // x of this thread's columns (consumers), requested before the scan so the latencies overlap
     float2 xr[NV][P];
     bool vok[NV];
@@ -95,6 +107,25 @@ sparse_ffn_kernel(const FfnParams p, const int n_stages) {
     // needs a single batch.  Which chunk a thread LOADS is rotated by the CTA index, so that the 148
     // CTAs do not all ask L2 for the same line at the same moment; the keep-bits words go through
     // shared memory and are ranked in natural order by a block-wide scan.
+    int n_act_o = 0, r0_o = 0, r1_o = 0;
+    if (nested) {
+        // The list exists already: this CTA copies its share of the leading n_act entries.  A count or
+        // an index outside its range is clamped (no access leaves the layer) and reported.
+        __syncthreads();
+        const int lv = s_cnt[4];
+        int n = s_cnt[lv & 3];
+        bool bad = lv < 0 || lv > 3 || n < 0 || n > F;
+        n = min(max(n, 0), F);
+        n_act_o = n;
+        r0_o = (int)(((int64_t)n * cta) / n_ctas);
+        r1_o = (int)(((int64_t)n * (cta + 1)) / n_ctas);
+        for (int i = tid; i < r1_o - r0_o; i += kFfnThreads) {
+            const int j = p.order[r0_o + i];
+            bad |= j < 0 || j >= F;
+            s_list[i] = min(max(j, 0), F - 1);
+        }
+        if (bad && p.status) atomicOr(p.status, CLADA_STATUS_BAD_INDEX);
+    } else {
     const bool vec_ok = (reinterpret_cast<uintptr_t>(p.scores) & 15u) == 0;
     const int n_batches = (chunks + kFfnThreads - 1) / kFfnThreads;
     {
@@ -201,6 +232,11 @@ sparse_ffn_kernel(const FfnParams p, const int n_stages) {
             if (p.mask_out && j >= m0 && j < m1) p.mask_out[j] = keep ? 1 : 0;
         }
     }
+    n_act_o = n_act;
+    r0_o = r0;
+    r1_o = r1;
+    }  // scores + threshold
+    const int n_act = n_act_o, r0 = r0_o, r1 = r1_o;
     if (p.count_out && cta == 0 && tid == 0) *p.count_out = n_act;
     const int my_n = r1 - r0;
     if (n_act == 0) {
@@ -507,6 +543,9 @@ static int decode_with_workspace(const clada_layer *layer, const void *x, int32_
         p.d_model = layer->d_model;
         p.d_ff = layer->d_ff;
         p.act = layer->activation;
+        p.order = nullptr;
+        p.counts = nullptr;
+        p.level = nullptr;
         rc = layer->dtype == CLADA_F32    ? launch_ffn<float>(p, st)
              : layer->dtype == CLADA_BF16 ? launch_ffn<__nv_bfloat16>(p, st)
                                           : launch_ffn<__half>(p, st);
@@ -523,6 +562,51 @@ extern "C" int clada_sparse_ffn_decode(const clada_layer *layer, const void *x, 
                                        void *stream) {
     return decode_with_workspace(layer, x, B, scores, tau_final, tau_stride, y, y_dtype, mask_out, idx_out,
                                  count_out, ws, ws_bytes, status, stream);
+}
+
+// Decode from nested index lists (clada_nested_build): no scores, no threshold, no compaction -- the
+// kept set of sequence b is the leading counts[b][level[b]] entries of order[b].  One launch per sequence.
+extern "C" int clada_sparse_ffn_decode_nested(const clada_layer *layer, const void *x, int32_t B,
+                                              const int32_t *order, const int32_t *counts, const int32_t *level,
+                                              void *y, int32_t y_dtype, int32_t *count_out, void *ws,
+                                              size_t ws_bytes, int32_t *status, void *stream) {
+    int rc = validate_layer(layer, false);
+    if (rc != CLADA_OK) return rc;
+    if (!x || !order || !counts || !level || !y) return CLADA_ERR_NULL;
+    if (B <= 0) return CLADA_ERR_SHAPE;
+    if (!dtype_ok(y_dtype)) return CLADA_ERR_DTYPE;
+    if (!aligned16(x) || !aligned16(y)) return CLADA_ERR_ALIGN;
+    if (!ws || (reinterpret_cast<uintptr_t>(ws) & 255u)) return CLADA_ERR_WORKSPACE;
+    DeviceInfo di;
+    rc = device_info(&di);
+    if (rc != CLADA_OK) return rc;
+    if (ws_bytes < kWsCtrlBytes + (size_t)di.num_sms * layer->d_model * sizeof(float)) return CLADA_ERR_WORKSPACE;
+    const size_t esz = elem_size(layer->dtype), ysz = elem_size(y_dtype);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    for (int b = 0; b < B; ++b) {
+        FfnParams p = {};
+        p.w_gate = layer->w_gate;
+        p.w_up = layer->w_up;
+        p.w_down_t = layer->w_down_t;
+        p.x = static_cast<const char *>(x) + (size_t)b * layer->d_model * esz;
+        p.y = static_cast<char *>(y) + (size_t)b * layer->d_model * ysz;
+        p.y_dtype = y_dtype;
+        p.count_out = count_out ? count_out + b : nullptr;
+        p.partials = reinterpret_cast<float *>(static_cast<char *>(ws) + kWsCtrlBytes);
+        p.ctrl = static_cast<WsCtrl *>(ws);
+        p.status = status;
+        p.d_model = layer->d_model;
+        p.d_ff = layer->d_ff;
+        p.act = layer->activation;
+        p.order = order + (size_t)b * layer->d_ff;
+        p.counts = counts + (size_t)b * 4;
+        p.level = level + b;
+        rc = layer->dtype == CLADA_F32    ? launch_ffn<float>(p, st)
+             : layer->dtype == CLADA_BF16 ? launch_ffn<__nv_bfloat16>(p, st)
+                                          : launch_ffn<__half>(p, st);
+        if (rc != CLADA_OK) return rc;
+    }
+    return CLADA_OK;
 }
 
 // One decode step of a whole stack: the per-layer call in a native loop (one C call per token instead
