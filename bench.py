@@ -35,7 +35,7 @@ LAMBDA, GAMMA = 0.80, 0.12
 N_COPIES = 4
 # DRAM read + write bytes of one sparse_ffn_kernel launch at the baseline threshold of this workload, from the ncu
 # capture summarised in profiles/sparse_ffn_kernel_c2_full.md.  Must go back to None whenever that kernel changes.
-FFN_NCU_TRAFFIC_BYTES = 166.06e6
+FFN_NCU_TRAFFIC_BYTES = None
 
 
 def _peaks():
@@ -153,6 +153,35 @@ class Job:
         self.tau_s = wl.universal_threshold(self.s.tolist())
         self.tau_H = wl.universal_threshold(self.h.tolist())
         self.counts = {}
+        # nested index lists (the masks' compressed form): per sparsity one list + four counts
+        i32 = dict(dtype=torch.int32, device=dev)
+        self.order = torch.empty(len(w.sparsities), 1, w.d_ff, **i32)
+        self.ncounts = torch.empty(len(w.sparsities), 1, 4, **i32)
+        self.level = torch.zeros(1, **i32)
+
+    def step_nested(self):
+        """The same step with the kept sets held as nested index lists: the selection builds one list and
+        four counts per sparsity, a decode token takes its load level and the FFN reads the list's head."""
+        c, w = self.clada, self.w
+        L0 = self.layers[0]
+        c.clada_prefix_scores(L0, self.X, self.off, self.scores, self.ws, self.status)
+        for r, rho in enumerate(w.sparsities):
+            tb = self.tau_base[r]
+            c.clada_refine_scores(L0, self.X, self.off, tb.view(1), self.guard, 1e-4, self.scores, self.ws, self.status)
+            c.clada_nested_build(self.scores, tb.view(1), LAMBDA, GAMMA, self.order[r], self.ncounts[r])
+            for t in range(self.N):
+                c.clada_cogload_level(self.logits[t:t + 1], self.tokens[t:t + 1], self.tau_s, self.tau_H,
+                                      self.s[t:t + 1], self.h[t:t + 1], self.level, self.status)
+                c.clada_sparse_ffn_decode_nested(self.layers[t % N_COPIES], self.xs[t:t + 1], self.order[r],
+                                                 self.ncounts[r], self.level, self.y[r, t:t + 1], self.ws,
+                                                 status=self.status)
+
+    def ffn_only_loop_nested(self):
+        """Nested-list FFN launches at the baseline level back to back (call after step_nested)."""
+        self.level.zero_()
+        for t in range(self.N):
+            self.clada.clada_sparse_ffn_decode_nested(self.layers[t % N_COPIES], self.xs[t:t + 1], self.order[0],
+                                                      self.ncounts[0], self.level, self.y[0, t:t + 1], self.ws)
 
     def step(self):
         c, w = self.clada, self.w
@@ -395,12 +424,38 @@ def run_ours(args):
 
         e2e_step()
         e2e_ms = _timed(e2e_step, args.steps, barrier)
+
+        # the same step over nested index lists, reported beside the headline (not in place of it)
+        nested_ms = nested_ffn_ms = None
+        if hasattr(job, "step_nested"):
+            job.step_nested()
+            n_run = job.step_nested
+            nf_run = job.ffn_only_loop_nested
+            if args.graph:
+                n_graph = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(n_graph, stream=stream):
+                    job.step_nested()
+                n_run = n_graph.replay
+            for _ in range(3):
+                n_run()
+            nested_ms = _timed(n_run, args.steps, barrier)
+            job.ffn_only_loop_nested()
+            if args.graph:
+                nf_graph = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(nf_graph, stream=stream):
+                    job.ffn_only_loop_nested()
+                nf_run = nf_graph.replay
+            nf_run()
+            nested_ffn_ms = _timed(nf_run, 5, lambda: None) / (5 * job.ffn_launches_per_loop)
         status = int(job.status.item())
 
     # every rank ran its own sequence; the job's rate is all ranks' tokens over the slowest rank's time
     tokens_rank = job.tokens_per_step() * args.steps
     value, ms = sharding.whole_job_rate(tokens_rank, ms, dev)
     e2e_value, e2e_ms = sharding.whole_job_rate(tokens_rank, e2e_ms, dev)
+    nested_value = None
+    if nested_ms is not None:
+        nested_value, nested_ms = sharding.whole_job_rate(tokens_rank, nested_ms, dev)
 
     peak, peak_kind = _peaks()
     prefix_flop = job.prefix_flop
@@ -440,6 +495,15 @@ def run_ours(args):
                             "flop": prefix_flop},
         "clocks": clocks, "device_status_word": status,
     }
+    if nested_value is not None:
+        # list entries instead of the score vector: 4 bytes per kept neuron
+        nb = kept_base * rows * w.d_model * eb + kept_base * 4 + w.d_model * eb + w.d_model * 4
+        line["nested_lists"] = {
+            "value": nested_value, "unit": "tokens/s", "ms_per_step": nested_ms / args.steps,
+            "step": "prefix statistics + per sparsity (guard band, nested lists, 128 x (cogload+level, sparse FFN "
+                    "over the list's head))",
+            "ffn_us_per_launch": nested_ffn_ms * 1e3, "ffn_bytes_per_launch": nb,
+            "ffn_achieved_gbs": nb / (nested_ffn_ms * 1e-3) / 1e9, "ffn_frac": nb / (nested_ffn_ms * 1e-3) / 1e9 / peak}
     if rank == 0:
         if world == 1 and w.name == WORKLOAD:
             line["cpu_baseline"] = cpu_baseline(w)
