@@ -328,6 +328,79 @@ void oracle_dense_ffn(int dtype, const void *x, int d_model, int d_ff,
     free(h);
 }
 
+/* ------------------------------------------------------------------ *
+ * The dense prefill FFN whose by-product the statistics are (Algorithm 2,
+ * prefill phase: the prompt runs through the dense layer).
+ *
+ * Half-precision models keep the hidden activation z in the storage type
+ * between the two projections; round_z != 0 reproduces that: z is computed in
+ * double, rounded to fp32 (the accumulator type) and then to the storage type,
+ * both to nearest even, before the down projection.  round_z == 0 keeps z in
+ * double (then Y[t] equals oracle_dense_ffn of row t).
+ * ------------------------------------------------------------------ */
+
+/* v rounded to nearest even in a binary format with p significand bits (hidden
+ * bit included), minimum normal exponent emin and largest finite value vmax. */
+static double round_to_format(double v, int p, int emin, double vmax)
+{
+    if (v == 0.0 || isnan(v) || isinf(v))
+        return v;
+    int e;
+    (void)frexp(fabs(v), &e);            /* |v| = f * 2^e, f in [0.5, 1)  ->  exponent e - 1 */
+    int ex = e - 1;
+    if (ex < emin)
+        ex = emin;                       /* subnormal range: fixed quantum */
+    const double quantum = ldexp(1.0, ex - (p - 1));
+    const double r = nearbyint(v / quantum) * quantum;   /* default rounding mode: ties to even */
+    if (fabs(r) > vmax)
+        return v > 0 ? INFINITY : -INFINITY;
+    return r;
+}
+
+double oracle_round_storage(int dtype, double v)
+{
+    const double f = (double)(float)v;   /* the fp32 accumulator value */
+    if (dtype == OR_BF16)
+        return round_to_format(f, 8, -126, 3.3895313892515355e38);
+    if (dtype == OR_F16)
+        return round_to_format(f, 11, -14, 65504.0);
+    return f;
+}
+
+/* Z[t, j] = value of neuron j for token t (rounded to the storage type if round_z). */
+void oracle_prefill_hidden(int dtype, const void *X, int T, int d_model, int d_ff,
+                           const void *W_in, const void *V_in, int act, int round_z, double *Z)
+{
+#pragma omp parallel for schedule(static)
+    for (int j = 0; j < d_ff; ++j) {
+        for (int t = 0; t < T; ++t) {
+            double g = 0.0, u = 0.0;
+            for (int k = 0; k < d_model; ++k) {
+                double x = elem(X, dtype, (size_t)t * d_model + k);
+                g += elem(W_in, dtype, (size_t)j * d_model + k) * x;
+                if (is_gated(act))
+                    u += elem(V_in, dtype, (size_t)j * d_model + k) * x;
+            }
+            double z = neuron_value(act, g, u);
+            Z[(size_t)t * d_ff + j] = round_z ? oracle_round_storage(dtype, z) : z;
+        }
+    }
+}
+
+/* Y[t, i] = sum_j Z[t, j] W_out[i, j]: the down projection of given hidden activations. */
+void oracle_down_proj(int dtype, const double *Z, int T, int d_model, int d_ff, const void *W_out, double *Y)
+{
+#pragma omp parallel for schedule(static)
+    for (int i = 0; i < d_model; ++i) {
+        for (int t = 0; t < T; ++t) {
+            double acc = 0.0;
+            for (int j = 0; j < d_ff; ++j)
+                acc += Z[(size_t)t * d_ff + j] * elem(W_out, dtype, (size_t)i * d_ff + j);
+            Y[(size_t)t * d_model + i] = acc;
+        }
+    }
+}
+
 /* Mask compression by nesting.  Eq. final_threshold can only produce
  * tau_base * {1, 1+lambda, 1+gamma, 1+lambda+gamma}, and the kept set of any
  * threshold is { j : A_j >= tau }, so every kept set is a leading part of ONE

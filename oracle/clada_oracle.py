@@ -60,6 +60,12 @@ def lib():
         L.oracle_cett_curve.restype = None
         L.oracle_threshold_search.argtypes = [vp, vp, i32, i32, dbl, vp]
         L.oracle_threshold_search.restype = dbl
+        L.oracle_round_storage.argtypes = [i32, dbl]
+        L.oracle_round_storage.restype = dbl
+        L.oracle_prefill_hidden.argtypes = [i32, vp, i32, i32, i32, vp, vp, i32, i32, vp]
+        L.oracle_prefill_hidden.restype = None
+        L.oracle_down_proj.argtypes = [i32, vp, i32, i32, i32, vp, vp]
+        L.oracle_down_proj.restype = None
         L.oracle_nested_lists.argtypes = [vp, i32, vp, i32, vp, vp]
         L.oracle_nested_lists.restype = None
         L.oracle_load_level.argtypes = [dbl, dbl, dbl, dbl]
@@ -245,3 +251,31 @@ def load_level(surprisal, entropy, tau_s, tau_H) -> int:
     """I(s > tau_s) + 2 I(H > tau_H): the index of the threshold Eq. final_threshold yields."""
     return int(lib().oracle_load_level(float(surprisal), float(entropy), float(np.float32(tau_s)),
                                        float(np.float32(tau_H))))
+
+
+def round_storage(dtype_code: int, v: float) -> float:
+    """v rounded to fp32 and then to the storage type (F32 / BF16 / F16), both to nearest even."""
+    return float(lib().oracle_round_storage(int(dtype_code), float(v)))
+
+
+def prefill_hidden(X, W_in, V_in, act=SILU_GATED, round_z=True) -> np.ndarray:
+    """Z [T, d_ff] float64: every neuron's value for every prompt token, rounded to the storage type of X
+    (as half-precision models keep it between the two projections) unless round_z is False."""
+    X, W_in = _c(X), _c(W_in)
+    V_in = None if V_in is None else _c(V_in)
+    d_ff, d_model = W_in.shape
+    assert X.shape[1] == d_model and X.dtype == W_in.dtype
+    Z = np.empty((X.shape[0], d_ff), dtype=np.float64)
+    lib().oracle_prefill_hidden(_dt(X), _p(X), X.shape[0], d_model, d_ff, _p(W_in), _pv(V_in), int(act),
+                                1 if round_z else 0, _p(Z))
+    return Z
+
+
+def down_proj(Z, W_out) -> np.ndarray:
+    """Y [T, d_model] float64 = Z W_out^T for hidden activations Z [T, d_ff] (float64) and W_out [d_model, d_ff]."""
+    Z, W_out = _c(Z, np.float64), _c(W_out)
+    d_model, d_ff = W_out.shape
+    assert Z.shape[1] == d_ff
+    Y = np.empty((Z.shape[0], d_model), dtype=np.float64)
+    lib().oracle_down_proj(_dt(W_out), _p(Z), Z.shape[0], d_model, d_ff, _p(W_out), _p(Y))
+    return Y

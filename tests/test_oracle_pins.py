@@ -592,3 +592,59 @@ def test_nested_ffn_equals_thresholded_ffn(oracle):
         marks[order[:counts[k]]] = 1.0                                       # keep exactly the listed neurons
         y_list, mask2, cnt2 = oracle.sparse_ffn(X[0], Wg, Wu, Wd, marks, 0.5)
         assert cnt == cnt2 == counts[k] and np.array_equal(mask, mask2) and np.array_equal(y_tau, y_list)
+
+
+# ----------------------------------------------------------------------------------------------
+# Dense prefill FFN (the pass the statistics are a by-product of)
+# ----------------------------------------------------------------------------------------------
+
+def test_round_storage_matches_library_casts(oracle):
+    rng = np.random.default_rng(70)
+    vals = np.concatenate([rng.standard_normal(2000) * 10.0 ** rng.integers(-9, 6, 2000),
+                           [0.0, -0.0, 1.0, 65504.0, 65519.9, 65520.0, 7e4, 6.0e-8, 2.98e-8, 2.9e-8, 1e-45,
+                            1.00390625, 1.001953125, 1.005859375, 3.4e38, 3.39e38, -2.5]])
+    f32 = vals.astype(np.float32)
+    ref16 = f32.astype(np.float16).astype(np.float64)                         # numpy: nearest even
+    ref_b = torch.from_numpy(f32).to(torch.bfloat16).to(torch.float64).numpy()   # torch: nearest even
+    with np.errstate(over="ignore"):
+        for v, r16, rb in zip(vals, ref16, ref_b):
+            assert oracle.round_storage(2, v) == r16, v
+            assert oracle.round_storage(1, v) == rb, v
+            assert oracle.round_storage(0, v) == float(np.float32(v))
+    # ties go to even: 1 + 2^-8 is halfway between two bf16 values, 1 + 2^-11 between two fp16 values
+    assert oracle.round_storage(1, 1.00390625) == 1.0 and oracle.round_storage(1, 1.01171875) == 1.015625
+    assert oracle.round_storage(2, 1.00048828125) == 1.0 and oracle.round_storage(2, 1.00146484375) == 1.001953125
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16", "f16"])
+@pytest.mark.parametrize("act", [0, 1, 2])
+def test_prefill_ffn_matches_library_formulation(oracle, dtype, act):
+    rng = np.random.default_rng(71 + act)
+    T, F, d = 7, 33, 24
+    X, Wg, Wu, Wd = _layer(rng, d=d, F=F, T=T, dtype="bf16" if dtype == "bf16" else "f32")
+    if dtype == "f16":
+        X, Wg, Wu, Wd = (a.astype(np.float16) for a in (X, Wg, Wu, Wd))
+    V = None if act == 2 else Wu
+    tX, tWg, tWu, tWd = (torch.from_numpy(_f64(a) if a.dtype == np.uint16 else a.astype(np.float64)) for a in (X, Wg, Wu, Wd))
+    h = _torch_h(act, tX, tWg, tWu)                                       # [T, F] float64
+    # without rounding: row t is the (separately pinned) per-token dense FFN
+    Z0 = oracle.prefill_hidden(X, Wg, V, act=act, round_z=False)
+    np.testing.assert_allclose(Z0, h.numpy(), rtol=1e-11, atol=1e-14)
+    Y0 = oracle.down_proj(Z0, Wd)
+    for t in range(T):
+        np.testing.assert_allclose(Y0[t], oracle.dense_ffn(X[t], Wg, V, Wd, act=act), rtol=1e-11, atol=1e-13)
+    # with rounding: the library's own casts, float64 -> float32 -> storage type
+    tdt = {"f32": torch.float32, "bf16": torch.bfloat16, "f16": torch.float16}[dtype]
+    h_r = h.to(torch.float32).to(tdt).to(torch.float64)
+    Z = oracle.prefill_hidden(X, Wg, V, act=act, round_z=True)
+    # the library's h differs from the oracle's in the last bits of float64, which can move a value across a
+    # rounding boundary only where it sits on one: allow one such element
+    assert np.sum(Z != h_r.numpy()) <= 1
+    np.testing.assert_allclose(oracle.down_proj(h_r.numpy(), Wd), (h_r @ tWd.T).numpy(), rtol=1e-11, atol=1e-13)
+
+
+def test_down_proj_worked_example(oracle):
+    """Y[t, i] = sum_j Z[t, j] W_out[i, j]: a transposed or mis-indexed operand changes these numbers."""
+    Z = np.array([[1.0, 2.0, 3.0], [0.0, -1.0, 0.5]])
+    W_out = np.array([[1.0, 0.0, 2.0], [0.0, 1.0, -1.0]], np.float32)        # [d_model = 2, d_ff = 3]
+    np.testing.assert_array_equal(oracle.down_proj(Z, W_out), [[7.0, -1.0], [1.0, -1.5]])
