@@ -269,6 +269,42 @@ int clada_sparse_ffn_decode_static(const clada_layer *layer, const void *x, int3
                                    uint8_t *mask_out, int32_t *idx_out, int32_t *count_out,
                                    int32_t *status, void *stream);
 
+/* ---- Dense prefill FFN with the statistics as a by-product, in chunks ----------
+ *
+ * Algorithm 2's prefill phase runs the prompt through the dense layer; the
+ * paper's Limitations name the pre-filling phase of long prompts (over 2048
+ * tokens) as a cost, and its long-context table reaches 32K-token prompts.  These three
+ * calls take the statistics from the prefill FFN itself and let a prompt arrive
+ * in chunks (chunked prefill):
+ *
+ * clada_prefix_accumulate: one chunk.  Arguments as clada_prefix_scores, but
+ *   sumsq  in/out [B, d_ff] fp32, device: running sum over the tokens seen so
+ *          far of z[t,j]^2 per (prompt, neuron); zero it before the first chunk.
+ *          seq_offsets describe THIS chunk's rows of X (a prompt may have no
+ *          rows in a chunk).
+ *   Z      out [T_chunk, d_ff] in the layer's element type, device, or NULL:
+ *          the hidden activations z[t,j] themselves, rounded once to the
+ *          element type (bf16 / fp16 layers only; CLADA_ERR_UNSUPPORTED for
+ *          fp32 layers with Z != NULL).  d_ff must then be a multiple of 8.
+ *   w_down_norm is not needed.  Workspace as for clada_prefix_scores of the chunk.
+ * clada_prefix_finish: scores[b,j] = sqrt(sumsq[b,j]) * w_down_norm[j] (fp32),
+ *   the same last step as clada_prefix_scores.  The guard band
+ *   (clada_refine_scores) needs the whole prompt's X; with chunks that are not
+ *   kept it is skipped and the scores carry the fp32 accumulation error.
+ * clada_prefill_down: Y [T, d_model] (y_dtype) = Z [T, d_ff] . w_down^T with
+ *   w_down [d_model, d_ff] in the paper's layout (W_out, neuron j = column j;
+ *   the decode path's w_down_t is its transpose), tensor cores, fp32
+ *   accumulation.  bf16 / fp16 layers; d_ff a multiple of 8; all pointers
+ *   16-byte aligned.  Together with Z from clada_prefix_accumulate this is the
+ *   layer's dense prefill output. */
+int clada_prefix_accumulate(const clada_layer *layer, const void *X, const int64_t *seq_offsets,
+                            int32_t B, float *sumsq, void *Z, void *ws, size_t ws_bytes,
+                            int32_t *status, void *stream);
+int clada_prefix_finish(const clada_layer *layer, const float *sumsq, int32_t B, float *scores,
+                        void *stream);
+int clada_prefill_down(const clada_layer *layer, const void *w_down, const void *Z, int64_t T,
+                       void *Y, int32_t y_dtype, int32_t *status, void *stream);
+
 /* ---- Nested index lists: the masks of Eq. final_threshold in compressed form ----
  *
  * The paper names mask memory as a limitation and mask compression as future

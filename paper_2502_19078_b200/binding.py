@@ -71,6 +71,9 @@ def load() -> ctypes.CDLL:
     L.clada_sparse_ffn_decode.argtypes = [lp, vp, i32, vp, vp, i64, vp, i32, vp, vp, vp, vp, sz, vp, vp]
     L.clada_sparse_ffn_decode_static.argtypes = [lp, vp, i32, vp, vp, i64, vp, i32, vp, vp, vp, vp, vp]
     L.clada_sparse_ffn_decode_layers.argtypes = [vp, i32, vp, i32, vp, vp, vp, i32, vp, sz, vp, vp]
+    L.clada_prefix_accumulate.argtypes = [lp, vp, vp, i32, vp, vp, vp, sz, vp, vp]
+    L.clada_prefix_finish.argtypes = [lp, vp, i32, vp, vp]
+    L.clada_prefill_down.argtypes = [lp, vp, vp, i64, vp, i32, vp, vp]
     L.clada_nested_build.argtypes = [vp, i32, i32, vp, i64, f32, f32, vp, vp, vp]
     L.clada_cogload_level.argtypes = [vp, i32, i32, i64, i64, vp, f32, f32, vp, vp, vp, vp, vp]
     L.clada_sparse_ffn_decode_nested.argtypes = [lp, vp, i32, vp, vp, vp, vp, i32, vp, vp, sz, vp, vp]
@@ -402,3 +405,25 @@ def clada_sparse_ffn_decode_nested(layer: Layer, x, order, counts, level, y, ws,
                                                  _ptr(ws, torch.uint8, "ws"), ws.numel(),
                                                  _ptr(status, torch.int32, "status"), _stream(stream)),
            "clada_sparse_ffn_decode_nested")
+
+
+def clada_prefix_accumulate(layer: Layer, X, seq_offsets, sumsq, ws, Z=None, status=None, stream=None) -> None:
+    """One chunk of prompts: sumsq [B, F] += sum_t z^2; Z [T_chunk, F] (layer dtype) receives the hidden activations."""
+    off, B = _offsets(seq_offsets)
+    _check(load().clada_prefix_accumulate(layer.ref, _ptr(X, layer.dtype, "X"), ctypes.addressof(off), B,
+                                          _ptr(sumsq, torch.float32, "sumsq"), _ptr(Z, layer.dtype, "Z"),
+                                          _ptr(ws, torch.uint8, "ws"), ws.numel(),
+                                          _ptr(status, torch.int32, "status"), _stream(stream)),
+           "clada_prefix_accumulate")
+
+
+def clada_prefix_finish(layer: Layer, sumsq, scores, stream=None) -> None:
+    _check(load().clada_prefix_finish(layer.ref, _ptr(sumsq, torch.float32, "sumsq"), sumsq.shape[0],
+                                      _ptr(scores, torch.float32, "scores"), _stream(stream)), "clada_prefix_finish")
+
+
+def clada_prefill_down(layer: Layer, w_down, Z, Y, status=None, stream=None) -> None:
+    """Y [T, d_model] = Z [T, d_ff] w_down^T, w_down [d_model, d_ff] in the paper's layout."""
+    _check(load().clada_prefill_down(layer.ref, _ptr(w_down, layer.dtype, "w_down"), _ptr(Z, layer.dtype, "Z"),
+                                     Z.shape[0], _ptr(Y, name="Y"), _dtype_code(Y.dtype),
+                                     _ptr(status, torch.int32, "status"), _stream(stream)), "clada_prefill_down")

@@ -117,6 +117,28 @@ __global__ void prefix_finalize_kernel(const float *__restrict__ partials, const
     scores[(size_t)b * d_ff + j] = __fmul_rn(sqrtf(s), w_down_norm[j]);
 }
 
+// Chunked prefill: the same tile sums added into a running sum of squares per (prompt, neuron) ...
+__global__ void prefix_accumulate_kernel(const float *__restrict__ partials, const SeqTable tab, int tile, int d_ff,
+                                         float *__restrict__ sumsq) {
+    const int j = blockIdx.x * blockDim.x + threadIdx.x;
+    const int b = blockIdx.y;
+    if (j >= d_ff) return;
+    int first = 0;
+    for (int q = 0; q < b; ++q) first += tiles_of(tab.off[q + 1] - tab.off[q], tile);
+    const int n = tiles_of(tab.off[b + 1] - tab.off[b], tile);
+    float s = sumsq[(size_t)b * d_ff + j];
+    for (int t = 0; t < n; ++t) s += partials[(size_t)(first + t) * d_ff + j];
+    sumsq[(size_t)b * d_ff + j] = s;
+}
+
+// ... and, after the last chunk, the scores from it.
+__global__ void prefix_finish_kernel(const float *__restrict__ sumsq, int B, int d_ff,
+                                     const float *__restrict__ w_down_norm, float *__restrict__ scores) {
+    const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= (size_t)B * d_ff) return;
+    scores[i] = __fmul_rn(sqrtf(sumsq[i]), w_down_norm[i % d_ff]);
+}
+
 // ---- guard band -----------------------------------------------------------------------------
 
 struct GuardMults {
@@ -354,6 +376,67 @@ int clada_prefix_scores(const clada_layer *layer, const void *X, const int64_t *
     rc = run_prefix_partials_tc(layer, X, tab, seq_offsets[B], partials, status, st);
     if (rc != CLADA_OK) return rc;
     return launch_prefix_finalize(partials, tab, kTcTokenTile, layer->d_ff, layer->w_down_norm, scores, st);
+}
+
+int clada_prefix_accumulate(const clada_layer *layer, const void *X, const int64_t *seq_offsets, int32_t B,
+                            float *sumsq, void *Z, void *ws, size_t ws_bytes, int32_t *status, void *stream) {
+    int rc = validate_layer(layer, false);
+    if (rc != CLADA_OK) return rc;
+    if (!X || !sumsq) return CLADA_ERR_NULL;
+    if (!aligned16(X) || (Z && !aligned16(Z))) return CLADA_ERR_ALIGN;
+    if (Z && layer->dtype == CLADA_F32) return CLADA_ERR_UNSUPPORTED;  // hidden activations: tensor-core route only
+    SeqTable tab;
+    int n_mtiles = 0;
+    rc = build_table(seq_offsets, B, &tab, &n_mtiles);
+    if (rc != CLADA_OK) return rc;
+    if (!ws || (reinterpret_cast<uintptr_t>(ws) & 255u)) return CLADA_ERR_WORKSPACE;
+    if (ws_bytes < kWsCtrlBytes + partials_bytes(n_mtiles, layer->d_ff)) return CLADA_ERR_WORKSPACE;
+    float *partials = reinterpret_cast<float *>(static_cast<char *>(ws) + kWsCtrlBytes);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int tile = BM;
+    if (layer->dtype == CLADA_F32) {
+        if (n_mtiles > 0) {
+            dim3 grid((layer->d_ff + BN - 1) / BN, n_mtiles);
+            prefix_partials_kernel<float><<<grid, kPfThreads, 0, st>>>(
+                static_cast<const float *>(X), static_cast<const float *>(layer->w_gate),
+                static_cast<const float *>(layer->w_up), layer->d_model, layer->d_ff, tab, partials, nullptr, 0,
+                layer->activation);
+            CLADA_CUDA_TRY(cudaGetLastError());
+        }
+    } else {
+        rc = run_prefix_partials_tc(layer, X, tab, seq_offsets[B], partials, status, st, Z);
+        if (rc != CLADA_OK) return rc;
+        tile = kTcTokenTile;
+    }
+    dim3 agrid((layer->d_ff + 255) / 256, tab.B);
+    prefix_accumulate_kernel<<<agrid, 256, 0, st>>>(partials, tab, tile, layer->d_ff, sumsq);
+    CLADA_CUDA_TRY(cudaGetLastError());
+    return CLADA_OK;
+}
+
+int clada_prefix_finish(const clada_layer *layer, const float *sumsq, int32_t B, float *scores, void *stream) {
+    int rc = validate_layer(layer, true);
+    if (rc != CLADA_OK) return rc;
+    if (!sumsq || !scores) return CLADA_ERR_NULL;
+    if (B <= 0) return CLADA_ERR_SHAPE;
+    const size_t n = (size_t)B * layer->d_ff;
+    prefix_finish_kernel<<<(unsigned)((n + 255) / 256), 256, 0, static_cast<cudaStream_t>(stream)>>>(
+        sumsq, B, layer->d_ff, layer->w_down_norm, scores);
+    CLADA_CUDA_TRY(cudaGetLastError());
+    return CLADA_OK;
+}
+
+int clada_prefill_down(const clada_layer *layer, const void *w_down, const void *Z, int64_t T, void *Y,
+                       int32_t y_dtype, int32_t *status, void *stream) {
+    int rc = validate_layer(layer, false);
+    if (rc != CLADA_OK) return rc;
+    if (!w_down || !Z || !Y) return CLADA_ERR_NULL;
+    if (T < 0) return CLADA_ERR_SHAPE;
+    if (layer->dtype == CLADA_F32) return CLADA_ERR_UNSUPPORTED;  // tensor-core route: bf16 / fp16 layers
+    if (!dtype_ok(y_dtype)) return CLADA_ERR_DTYPE;
+    if (layer->d_ff % 8 != 0) return CLADA_ERR_SHAPE;  // rows of Z and of w_down must be 16-byte multiples
+    if (!aligned16(w_down) || !aligned16(Z) || !aligned16(Y)) return CLADA_ERR_ALIGN;
+    return run_down_tc(layer, w_down, Z, T, Y, y_dtype, status, static_cast<cudaStream_t>(stream));
 }
 
 int clada_refine_scores(const clada_layer *layer, const void *X, const int64_t *seq_offsets, int32_t B,

@@ -42,6 +42,8 @@ struct TcParams {
     int n_ttiles;   // token tiles over all prompts
     float *partials;  // [n_ttiles, d_ff]
     int32_t *status;
+    void *z_out;    // [T_total, d_ff] in the layer's element type, or null: the hidden activations themselves
+    int dtype;      // clada_dtype of the layer (for z_out)
     uint32_t idesc; // instruction descriptor for the layer's element type
     int act;        // clada_activation; the non-gated form skips the w_up tiles and their MMAs
     SeqTable tab;
@@ -251,6 +253,7 @@ prefix_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
             const uint32_t t_gate = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)a * 256u;
             const uint32_t t_up = t_gate + 128u;
             float sum = 0.f;
+            const int jrow = ntile * kTcTileM + quarter * 32 + lane;
             for (int c0 = 0; c0 < ncols; c0 += 16) {  // uniform per warp: ncols is
                 uint32_t rg[16], ru[16];
                 tc_ld16(t_gate + c0, rg);
@@ -266,6 +269,13 @@ prefix_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                     if (c0 + c < ncols) {
                         const float z = neuron_value_f(p.act, __uint_as_float(rg[c]), __uint_as_float(ru[c]));
                         sum = fmaf(z, z, sum);
+                        if (p.z_out && jrow < p.d_ff) {  // a warp writes 32 consecutive neurons of one token
+                            const size_t at = (size_t)(t0 + c0 + c) * p.d_ff + jrow;
+                            if (p.dtype == CLADA_BF16)
+                                static_cast<__nv_bfloat16 *>(p.z_out)[at] = __float2bfloat16_rn(z);
+                            else
+                                static_cast<__half *>(p.z_out)[at] = __float2half_rn(z);
+                        }
                     }
                 }
             }
@@ -327,7 +337,7 @@ static int make_map(EncodeTiledFn enc, CUtensorMap *map, const void *base, long 
 }
 
 int run_prefix_partials_tc(const clada_layer *layer, const void *X, const SeqTable &tab, long long T_total,
-                           float *partials, int32_t *status, cudaStream_t st) {
+                           float *partials, int32_t *status, cudaStream_t st, void *z_out) {
     static bool configured[64] = {};
     int n_ttiles = 0;
     for (int b = 0; b < tab.B; ++b) n_ttiles += tiles_of(tab.off[b + 1] - tab.off[b], kTcTileN);
@@ -352,6 +362,8 @@ int run_prefix_partials_tc(const clada_layer *layer, const void *X, const SeqTab
     p.partials = partials;
     p.status = status;
     p.act = layer->activation;
+    p.z_out = z_out;
+    p.dtype = layer->dtype;
     p.idesc = layer->dtype == CLADA_F16 ? kTcInstrDescF16 : kTcInstrDescBf16;
     p.tab = tab;
     const size_t smem = (size_t)kTcStages * kTcStageBytes + 1024;
@@ -362,6 +374,210 @@ int run_prefix_partials_tc(const clada_layer *layer, const void *X, const SeqTab
     const long long items = (long long)p.n_ntiles * n_ttiles;
     const int grid = (int)std::min<long long>(items, di.num_sms);
     prefix_tc_kernel<<<grid, kTcThreads, smem, st>>>(map_x, map_wg, map_wu, p);
+    CLADA_CUDA_TRY(cudaGetLastError());
+    return CLADA_OK;
+}
+
+// ---- down projection of the dense prefill FFN --------------------------------------------------
+//   Y[t, i] = sum_j Z[t, j] * W_out[i, j]      (Z: hidden activations, W_out in the paper's [d_model, d_ff] layout)
+// Both operands are K-major (d_ff contiguous), so the tiles, descriptors and the role split are those of
+// the statistics kernel: tokens are the M dimension (TMEM lanes), output columns the N dimension, one
+// accumulator per tile, two in flight.  The epilogue thread that owns token t writes its row of the tile.
+
+constexpr int kDnStages = 6;
+constexpr uint32_t kDnStageBytes = 2 * kTcTileBytes;  // Z tile | W_out tile
+constexpr uint32_t kDnTmemCols = 256;                 // two 128-column accumulators
+
+struct DownParams {
+    int d_model, d_ff;
+    long long T;
+    int n_ttiles, n_dtiles;
+    void *y;
+    int y_dtype;
+    uint32_t idesc;
+    int32_t *status;
+};
+
+__global__ void __launch_bounds__(kTcThreads, 1)
+down_tc_kernel(const __grid_constant__ CUtensorMap map_z, const __grid_constant__ CUtensorMap map_w,
+               const DownParams p) {
+    extern __shared__ unsigned char tc_smem_raw[];
+    const uint32_t smem0 = (tc_smem_u32(tc_smem_raw) + 1023u) & ~1023u;
+    __shared__ __align__(8) uint64_t s_full[kDnStages], s_empty[kDnStages], s_acc_full[2], s_acc_empty[2];
+    __shared__ uint32_t s_tmem_base;
+    __shared__ int s_abort;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int n_items = p.n_ttiles * p.n_dtiles;
+    const int n_kblocks = (p.d_ff + kTcTileK - 1) / kTcTileK;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kDnStages; ++s) {
+            tc_mbar_init(tc_smem_u32(&s_full[s]), 1);
+            tc_mbar_init(tc_smem_u32(&s_empty[s]), 1);
+        }
+        for (int a = 0; a < 2; ++a) {
+            tc_mbar_init(tc_smem_u32(&s_acc_full[a]), 1);
+            tc_mbar_init(tc_smem_u32(&s_acc_empty[a]), 4);
+        }
+        s_abort = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(tc_smem_u32(&s_tmem_base)),
+                     "r"(kDnTmemCols)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = s_tmem_base;
+    volatile int *abort_flag = &s_abort;
+
+    // items run token tile fastest, so the CTAs of a wave share the same W_out tiles in L2
+    if (warp == 0) {
+        if (lane == 0) {
+            int kc = 0;
+            bool ok = true;
+            for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
+                const int dtile = item / p.n_ttiles, ttile = item % p.n_ttiles;
+                for (int kb = 0; kb < n_kblocks; ++kb, ++kc) {
+                    const int s = kc % kDnStages;
+                    if (!tc_mbar_wait(tc_smem_u32(&s_empty[s]), ((kc / kDnStages) & 1) ^ 1, abort_flag)) {
+                        ok = false;
+                        break;
+                    }
+                    const uint32_t bar = tc_smem_u32(&s_full[s]);
+                    const uint32_t dst = smem0 + (uint32_t)s * kDnStageBytes;
+                    tc_mbar_expect_tx(bar, kDnStageBytes);
+                    tc_tma_load(dst, &map_z, kb * kTcTileK, ttile * kTcTileM, bar);
+                    tc_tma_load(dst + kTcTileBytes, &map_w, kb * kTcTileK, dtile * kTcTileN, bar);
+                }
+            }
+            if (!ok) *abort_flag = 1;
+            for (int i = max(0, kc - kDnStages); i < kc; ++i) {
+                int never = 0;  // these copies land by themselves: wait for them even after an abort
+                if (!tc_mbar_wait(tc_smem_u32(&s_full[i % kDnStages]), (i / kDnStages) & 1, &never)) *abort_flag = 1;
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            int kc = 0, it = 0;
+            bool ok = true;
+            for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++it) {
+                const int a = it & 1;
+                if (!tc_mbar_wait(tc_smem_u32(&s_acc_empty[a]), ((it >> 1) & 1) ^ 1, abort_flag)) {
+                    ok = false;
+                    break;
+                }
+                tc_fence_after();
+                const uint32_t d_acc = tmem_base + (uint32_t)a * 128u;
+                for (int kb = 0; kb < n_kblocks; ++kb, ++kc) {
+                    const int s = kc % kDnStages;
+                    if (!tc_mbar_wait(tc_smem_u32(&s_full[s]), (kc / kDnStages) & 1, abort_flag)) {
+                        ok = false;
+                        break;
+                    }
+                    tc_fence_after();
+                    const uint32_t base = smem0 + (uint32_t)s * kDnStageBytes;
+                    const uint64_t dz = tc_smem_desc(base), dw = tc_smem_desc(base + kTcTileBytes);
+#pragma unroll
+                    for (int k = 0; k < kTcTileK / 16; ++k)
+                        tc_mma(d_acc, dz + 2 * k, dw + 2 * k, (kb > 0 || k > 0) ? 1u : 0u, p.idesc);
+                    tc_commit(tc_smem_u32(&s_empty[s]));
+                }
+                if (ok) tc_commit(tc_smem_u32(&s_acc_full[a]));
+            }
+            if (!ok) *abort_flag = 1;
+        }
+    } else {
+        const int quarter = warp & 3;
+        int it = 0;
+        bool ok = true;
+        for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++it) {
+            const int a = it & 1;
+            const int dtile = item / p.n_ttiles, ttile = item % p.n_ttiles;
+            if (!tc_mbar_wait(tc_smem_u32(&s_acc_full[a]), (it >> 1) & 1, abort_flag)) {
+                ok = false;
+                break;
+            }
+            tc_fence_after();
+            const uint32_t t_acc = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)a * 128u;
+            const long long t = (long long)ttile * kTcTileM + quarter * 32 + lane;
+            const int i0 = dtile * kTcTileN;
+            const int ncols = min(kTcTileN, p.d_model - i0);  // a multiple of 8 (d_model is)
+            for (int c0 = 0; c0 < ncols; c0 += 16) {           // uniform per warp
+                uint32_t r[16];
+                tc_ld16(t_acc + c0, r);
+                tc_wait_ld();
+                if (t < p.T) {
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {              // two groups of 8 columns
+                        if (c0 + 8 * h >= ncols) continue;
+                        const float4 lo = make_float4(__uint_as_float(r[8 * h]), __uint_as_float(r[8 * h + 1]),
+                                                      __uint_as_float(r[8 * h + 2]), __uint_as_float(r[8 * h + 3]));
+                        const float4 hi = make_float4(__uint_as_float(r[8 * h + 4]), __uint_as_float(r[8 * h + 5]),
+                                                      __uint_as_float(r[8 * h + 6]), __uint_as_float(r[8 * h + 7]));
+                        const size_t at = (size_t)t * p.d_model + i0 + c0 + 8 * h;
+                        if (p.y_dtype == CLADA_F32) {
+                            float4 *dst = reinterpret_cast<float4 *>(static_cast<float *>(p.y) + at);
+                            dst[0] = lo;
+                            dst[1] = hi;
+                        } else {
+                            const uint2 a2 = pack4_16bit(p.y_dtype, lo), b2 = pack4_16bit(p.y_dtype, hi);
+                            *reinterpret_cast<uint4 *>(static_cast<uint16_t *>(p.y) + at) = make_uint4(a2.x, a2.y, b2.x, b2.y);
+                        }
+                    }
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) tc_mbar_arrive(tc_smem_u32(&s_acc_empty[a]));
+        }
+        if (!ok) *abort_flag = 1;
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (threadIdx.x == 0 && s_abort && p.status) atomicOr(p.status, CLADA_STATUS_TIMEOUT);
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kDnTmemCols) : "memory");
+    }
+}
+
+int run_down_tc(const clada_layer *layer, const void *w_down, const void *Z, long long T, void *Y, int y_dtype,
+                int32_t *status, cudaStream_t st) {
+    static bool configured[64] = {};
+    if (T <= 0) return CLADA_OK;
+    DeviceInfo di;
+    int rc = device_info(&di);
+    if (rc != CLADA_OK) return rc;
+    EncodeTiledFn enc;
+    rc = encode_fn(&enc);
+    if (rc != CLADA_OK) return rc;
+    CUtensorMap map_z, map_w;
+    if ((rc = make_map(enc, &map_z, Z, T, layer->d_ff, layer->dtype)) != CLADA_OK) return rc;
+    if ((rc = make_map(enc, &map_w, w_down, layer->d_model, layer->d_ff, layer->dtype)) != CLADA_OK) return rc;
+    DownParams p;
+    p.d_model = layer->d_model;
+    p.d_ff = layer->d_ff;
+    p.T = T;
+    p.n_ttiles = (int)((T + kTcTileM - 1) / kTcTileM);
+    p.n_dtiles = (layer->d_model + kTcTileN - 1) / kTcTileN;
+    p.y = Y;
+    p.y_dtype = y_dtype;
+    p.idesc = layer->dtype == CLADA_F16 ? kTcInstrDescF16 : kTcInstrDescBf16;
+    p.status = status;
+    const size_t smem = (size_t)kDnStages * kDnStageBytes + 1024;
+    if (!configured[di.device & 63]) {
+        CLADA_CUDA_TRY(cudaFuncSetAttribute(down_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        configured[di.device & 63] = true;
+    }
+    const long long items = (long long)p.n_ttiles * p.n_dtiles;
+    const int grid = (int)std::min<long long>(items, di.num_sms);
+    down_tc_kernel<<<grid, kTcThreads, smem, st>>>(map_z, map_w, p);
     CLADA_CUDA_TRY(cudaGetLastError());
     return CLADA_OK;
 }

@@ -40,8 +40,13 @@ int run_prefix_scores_with_z(const clada_layer *layer, const void *X, const int6
 size_t prefix_partials_bytes_cuda_core(const int64_t *seq_offsets, int32_t B, int d_ff);
 
 // Tensor-core partial sums (bf16 layers, 128-token tiles).  partials: [sum_b tiles_of(T_b, 128), d_ff].
+// z_out (optional): the hidden activations [T_total, d_ff] in the layer's element type.
 int run_prefix_partials_tc(const clada_layer *layer, const void *X, const SeqTable &tab, long long T_total,
-                           float *partials, int32_t *status, cudaStream_t st);
+                           float *partials, int32_t *status, cudaStream_t st, void *z_out = nullptr);
+
+// Y [T, d_model] = Z [T, d_ff] . w_down[d_model, d_ff]^T on the tensor cores (16-bit element types).
+int run_down_tc(const clada_layer *layer, const void *w_down, const void *Z, long long T, void *Y, int y_dtype,
+                int32_t *status, cudaStream_t st);
 constexpr int kTcTokenTile = 128;
 
 }  // namespace clada
