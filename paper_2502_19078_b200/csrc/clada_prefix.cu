@@ -385,6 +385,7 @@ int clada_prefix_accumulate(const clada_layer *layer, const void *X, const int64
     if (!X || !sumsq) return CLADA_ERR_NULL;
     if (!aligned16(X) || (Z && !aligned16(Z))) return CLADA_ERR_ALIGN;
     if (Z && layer->dtype == CLADA_F32) return CLADA_ERR_UNSUPPORTED;  // hidden activations: tensor-core route only
+    if (Z && layer->d_ff % 8 != 0) return CLADA_ERR_SHAPE;  // rows of Z are written as 16-byte vectors
     SeqTable tab;
     int n_mtiles = 0;
     rc = build_table(seq_offsets, B, &tab, &n_mtiles);

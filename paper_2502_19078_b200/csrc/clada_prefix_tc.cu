@@ -26,19 +26,24 @@
 
 namespace clada {
 
-constexpr int kTcTileM = 128;   // neurons per tile (TMEM lanes)
-constexpr int kTcTileN = 128;   // tokens per tile (TMEM columns per accumulator)
-constexpr int kTcTileK = 64;    // K block: 64 bf16 = 128 bytes = one swizzle row
-constexpr int kTcStages = 4;
+constexpr int kTcTileM = 128;   // rows of the A tile = TMEM lanes (tokens; also the most neurons per tile)
+constexpr int kTcTileN = 128;   // columns of a down-projection tile
+constexpr int kTcTileK = 64;    // K block: 64 16-bit elements = 128 bytes = one swizzle row
+constexpr int kTcMaxStages = 8;
 constexpr int kTcThreads = 192;
-constexpr uint32_t kTcTileBytes = kTcTileM * kTcTileK * 2;       // 16 KiB
-constexpr uint32_t kTcStageBytes = 3 * kTcTileBytes;             // w_gate | w_up | X
-constexpr uint32_t kTcTmemCols = 512;                            // 2 x (gate 128 + up 128)
+constexpr uint32_t kTcTileBytes = kTcTileM * kTcTileK * 2;       // 16 KiB: a 128-row tile
+constexpr uint32_t kTcRingBytes = 192 * 1024;                    // shared-memory ring of the statistics kernel
+constexpr uint32_t kTcTmemCols = 512;                            // two accumulators of up to 256 columns
 constexpr unsigned kTcSpinLimit = 1u << 20;
 
 struct TcParams {
     int d_model, d_ff;
-    int n_ntiles;   // neuron tiles
+    int n_full;     // work items of 128 neurons x 128 tokens, neuron tile major: item = ntile * n_ttiles + ttile
+    int n_half;     // the last (n_half / 2) such items are issued as two 64-neuron halves each, so that a last,
+                    // partly filled wave of CTAs takes half the time
+    int n_stages;   // ring depth
+    uint32_t idesc_half;  // instruction descriptor of a 64-neuron item
+    int n_ntiles;   // neuron tiles of 128
     int n_ttiles;   // token tiles over all prompts
     float *partials;  // [n_ttiles, d_ff]
     int32_t *status;
@@ -98,8 +103,10 @@ __device__ __forceinline__ uint64_t tc_smem_desc(uint32_t addr) {
 }
 // Instruction descriptor, kind::f16: D fp32, A and B of one 16-bit type (format code 1 = bf16, 0 = fp16,
 // the same for both operands), both K-major, N = 128, M = 128.
-constexpr uint32_t kTcInstrDescF16 = (1u << 4) | ((uint32_t)(kTcTileN >> 3) << 17) | ((uint32_t)(kTcTileM >> 4) << 24);
-constexpr uint32_t kTcInstrDescBf16 = kTcInstrDescF16 | (1u << 7) | (1u << 10);
+__host__ __device__ constexpr uint32_t tc_instr_desc(int dtype, int n_cols) {
+    return (1u << 4) | (dtype == CLADA_F16 ? 0u : ((1u << 7) | (1u << 10))) | ((uint32_t)(n_cols >> 3) << 17) |
+           ((uint32_t)(kTcTileM >> 4) << 24);
+}
 __device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t accumulate,
                                        uint32_t idesc) {
     asm volatile(
@@ -127,27 +134,45 @@ __device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sy
 
 __global__ void __launch_bounds__(kTcThreads, 1)
 prefix_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_wg,
-                 const __grid_constant__ CUtensorMap map_wu, const TcParams p) {
+                 const __grid_constant__ CUtensorMap map_wu, const __grid_constant__ CUtensorMap map_wg_half,
+                 const __grid_constant__ CUtensorMap map_wu_half, const TcParams p) {
     extern __shared__ unsigned char tc_smem_raw[];
     // stage tiles must sit on 1024-byte boundaries (the swizzle pattern is anchored to the address)
     const uint32_t smem0 = (tc_smem_u32(tc_smem_raw) + 1023u) & ~1023u;
-    __shared__ __align__(8) uint64_t s_full[kTcStages], s_empty[kTcStages], s_acc_full[2], s_acc_empty[2];
+    __shared__ __align__(8) uint64_t s_full[kTcMaxStages], s_empty[kTcMaxStages], s_acc_full[2], s_acc_empty[2], s_epi[2];
     __shared__ uint32_t s_tmem_base;
     __shared__ int s_abort;
+    __shared__ float s_col[2][4][kTcTileM];  // [tile parity][epilogue warp][neuron of the tile]
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int n_items = p.n_ntiles * p.n_ttiles;
+    const int n_items = p.n_full + p.n_half;
     const int n_kblocks = (p.d_model + kTcTileK - 1) / kTcTileK;
     const bool gated = act_is_gated(p.act);
+    const uint32_t stage_bytes = kTcTileBytes + (gated ? 2u : 1u) * kTcTileBytes;  // ring stride: a full item's stage
+    const int n_stages = p.n_stages;
+    // item -> (neurons per tile, first neuron, token tile)
+    auto decode = [&](int item, int &nt, int &j0, int &ttile) {
+        if (item < p.n_full) {
+            nt = 128;
+            j0 = (item / p.n_ttiles) * 128;
+            ttile = item % p.n_ttiles;
+        } else {
+            const int h = item - p.n_full, f = p.n_full + (h >> 1);
+            nt = 64;
+            j0 = (f / p.n_ttiles) * 128 + (h & 1) * 64;
+            ttile = f % p.n_ttiles;
+        }
+    };
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < kTcStages; ++s) {
+        for (int s = 0; s < n_stages; ++s) {
             tc_mbar_init(tc_smem_u32(&s_full[s]), 1);
             tc_mbar_init(tc_smem_u32(&s_empty[s]), 1);
         }
         for (int a = 0; a < 2; ++a) {
             tc_mbar_init(tc_smem_u32(&s_acc_full[a]), 1);
             tc_mbar_init(tc_smem_u32(&s_acc_empty[a]), 4);  // one arrival per epilogue warp
+            tc_mbar_init(tc_smem_u32(&s_epi[a]), 4);
         }
         s_abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -167,123 +192,161 @@ prefix_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
     if (warp == 0) {
         // ---- TMA producer ----------------------------------------------------------------------
         if (lane == 0) {
-            int kc = 0;  // K blocks issued so far (ring position)
+            int kc = 0;  // K blocks issued so far
+            int s = 0;   // ring position and the parity of its current use
+            uint32_t par = 0;
             bool ok = true;
             for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
-                const int ntile = item / p.n_ttiles, ttile = item % p.n_ttiles;
-                int b;
+                int nt, j0, ttile, b;
+                decode(item, nt, j0, ttile);
                 long long t0, t1;
-                locate_tile(p.tab, ttile, kTcTileN, b, t0, t1);
+                locate_tile(p.tab, ttile, kTcTileM, b, t0, t1);
+                const uint32_t w_bytes = (uint32_t)nt * kTcTileK * 2u;  // one weight tile of this item
+                const CUtensorMap *mg = nt == 128 ? &map_wg : &map_wg_half;
+                const CUtensorMap *mu = nt == 128 ? &map_wu : &map_wu_half;
                 for (int kb = 0; kb < n_kblocks; ++kb, ++kc) {
-                    const int s = kc % kTcStages;
-                    if (!tc_mbar_wait(tc_smem_u32(&s_empty[s]), ((kc / kTcStages) & 1) ^ 1, abort_flag)) {
+                    if (!tc_mbar_wait(tc_smem_u32(&s_empty[s]), par ^ 1, abort_flag)) {
                         ok = false;
                         break;
                     }
                     const uint32_t bar = tc_smem_u32(&s_full[s]);
-                    const uint32_t dst = smem0 + (uint32_t)s * kTcStageBytes;
-                    tc_mbar_expect_tx(bar, gated ? kTcStageBytes : 2 * kTcTileBytes);
-                    tc_tma_load(dst, &map_wg, kb * kTcTileK, ntile * kTcTileM, bar);
-                    if (gated) tc_tma_load(dst + kTcTileBytes, &map_wu, kb * kTcTileK, ntile * kTcTileM, bar);
-                    tc_tma_load(dst + 2 * kTcTileBytes, &map_x, kb * kTcTileK, (int)t0, bar);
+                    const uint32_t dst = smem0 + (uint32_t)s * stage_bytes;
+                    tc_mbar_expect_tx(bar, kTcTileBytes + (gated ? 2u : 1u) * w_bytes);
+                    tc_tma_load(dst, &map_x, kb * kTcTileK, (int)t0, bar);
+                    tc_tma_load(dst + kTcTileBytes, mg, kb * kTcTileK, j0, bar);
+                    if (gated) tc_tma_load(dst + kTcTileBytes + w_bytes, mu, kb * kTcTileK, j0, bar);
+                    if (++s == n_stages) {
+                        s = 0;
+                        par ^= 1;
+                    }
                 }
             }
             if (!ok) *abort_flag = 1;
             // never leave with copies in flight: the last armed use of every stage must have landed
-            for (int i = max(0, kc - kTcStages); i < kc; ++i)
-                {
+            for (int i = max(0, kc - n_stages); i < kc; ++i) {
                 int never = 0;  // these copies land by themselves: wait for them even after an abort
-                if (!tc_mbar_wait(tc_smem_u32(&s_full[i % kTcStages]), (i / kTcStages) & 1, &never)) *abort_flag = 1;
+                if (!tc_mbar_wait(tc_smem_u32(&s_full[i % n_stages]), (i / n_stages) & 1, &never)) *abort_flag = 1;
             }
         }
     } else if (warp == 1) {
         // ---- MMA issuer ------------------------------------------------------------------------
         if (lane == 0) {
-            int kc = 0, it = 0;
+            int it = 0;
+            int s = 0;
+            uint32_t par = 0;
             bool ok = true;
             for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++it) {
                 const int a = it & 1;
-                // the epilogue must have drained this accumulator pair (fresh barrier: parity 1 passes)
+                // the epilogue must have drained this accumulator (fresh barrier: parity 1 passes)
                 if (!tc_mbar_wait(tc_smem_u32(&s_acc_empty[a]), ((it >> 1) & 1) ^ 1, abort_flag)) {
                     ok = false;
                     break;
                 }
                 tc_fence_after();
-                const uint32_t d_gate = tmem_base + (uint32_t)a * 256u, d_up = d_gate + 128u;
-                for (int kb = 0; kb < n_kblocks; ++kb, ++kc) {
-                    const int s = kc % kTcStages;
-                    if (!tc_mbar_wait(tc_smem_u32(&s_full[s]), (kc / kTcStages) & 1, abort_flag)) {
+                const uint32_t d_acc = tmem_base + (uint32_t)a * 256u;
+                const uint32_t idesc = item < p.n_full ? p.idesc : p.idesc_half;
+                for (int kb = 0; kb < n_kblocks; ++kb) {
+                    if (!tc_mbar_wait(tc_smem_u32(&s_full[s]), par, abort_flag)) {
                         ok = false;
                         break;
                     }
                     tc_fence_after();
-                    const uint32_t base = smem0 + (uint32_t)s * kTcStageBytes;
-                    const uint64_t dg = tc_smem_desc(base), du = tc_smem_desc(base + kTcTileBytes),
-                                   dx = tc_smem_desc(base + 2 * kTcTileBytes);
+                    const uint32_t base = smem0 + (uint32_t)s * stage_bytes;
+                    // A = the token tile (128 rows), B = the w_gate rows with the w_up rows right behind them:
+                    // one instruction of N = 2 nt columns (gate | up) per 16-wide K step
+                    const uint64_t dx = tc_smem_desc(base), dw = tc_smem_desc(base + kTcTileBytes);
 #pragma unroll
-                    for (int k = 0; k < kTcTileK / 16; ++k) {
-                        // advancing K by 16 bf16 = 32 bytes = 2 descriptor units inside the swizzled row
-                        const uint32_t acc = (kb > 0 || k > 0) ? 1u : 0u;
-                        tc_mma(d_gate, dg + 2 * k, dx + 2 * k, acc, p.idesc);
-                        if (gated) tc_mma(d_up, du + 2 * k, dx + 2 * k, acc, p.idesc);
-                    }
+                    for (int k = 0; k < kTcTileK / 16; ++k)  // +32 bytes = 2 descriptor units inside the swizzled row
+                        tc_mma(d_acc, dx + 2 * k, dw + 2 * k, (kb > 0 || k > 0) ? 1u : 0u, idesc);
                     tc_commit(tc_smem_u32(&s_empty[s]));  // the stage is free once these MMAs have read it
+                    if (++s == n_stages) {
+                        s = 0;
+                        par ^= 1;
+                    }
                 }
-                if (ok) tc_commit(tc_smem_u32(&s_acc_full[a]));  // accumulators complete
+                if (ok) tc_commit(tc_smem_u32(&s_acc_full[a]));  // accumulator complete
             }
             if (!ok) *abort_flag = 1;
         }
     } else {
-        // ---- epilogue warps (2..5): warp w may touch TMEM lanes 32 (w % 4) .. +31 -------------------
+        // ---- epilogue warps (2..5): warp w may touch TMEM lanes 32 (w % 4) .. +31 = 32 tokens ------------
         const int quarter = warp & 3;
+        const bool b16 = lane & 16, b8 = lane & 8, b4 = lane & 4, b2 = lane & 2;
+        const int my_val = (b16 ? 8 : 0) + (b8 ? 4 : 0) + (b4 ? 2 : 0) + (b2 ? 1 : 0);
+        const int e = (warp - 2) * 32 + lane;  // 0..127: the neuron of the tile this thread finishes
         int it = 0;
         bool ok = true;
         for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++it) {
             const int a = it & 1;
-            const int ntile = item / p.n_ttiles, ttile = item % p.n_ttiles;
-            int b;
+            int nt, jbase, ttile, b;
+            decode(item, nt, jbase, ttile);
             long long t0, t1;
-            locate_tile(p.tab, ttile, kTcTileN, b, t0, t1);
-            const int ncols = (int)(t1 - t0);
+            locate_tile(p.tab, ttile, kTcTileM, b, t0, t1);
+            const int row = quarter * 32 + lane;          // this thread's token within the tile
+            const bool tok_ok = row < (int)(t1 - t0);     // rows past the prompt's end belong to nobody
             if (!tc_mbar_wait(tc_smem_u32(&s_acc_full[a]), (it >> 1) & 1, abort_flag)) {
                 ok = false;
                 break;
             }
             tc_fence_after();
-            const uint32_t t_gate = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)a * 256u;
-            const uint32_t t_up = t_gate + 128u;
-            float sum = 0.f;
-            const int jrow = ntile * kTcTileM + quarter * 32 + lane;
-            for (int c0 = 0; c0 < ncols; c0 += 16) {  // uniform per warp: ncols is
+            const uint32_t t_acc = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)a * 256u;
+            for (int c0 = 0; c0 < nt; c0 += 16) {
                 uint32_t rg[16], ru[16];
-                tc_ld16(t_gate + c0, rg);
+                tc_ld16(t_acc + c0, rg);
                 if (gated) {
-                    tc_ld16(t_up + c0, ru);
+                    tc_ld16(t_acc + nt + c0, ru);
                 } else {
 #pragma unroll
                     for (int c = 0; c < 16; ++c) ru[c] = 0u;
                 }
                 tc_wait_ld();
+                float z[16], q[16];
 #pragma unroll
                 for (int c = 0; c < 16; ++c) {
-                    if (c0 + c < ncols) {
-                        const float z = neuron_value_f(p.act, __uint_as_float(rg[c]), __uint_as_float(ru[c]));
-                        sum = fmaf(z, z, sum);
-                        if (p.z_out && jrow < p.d_ff) {  // a warp writes 32 consecutive neurons of one token
-                            const size_t at = (size_t)(t0 + c0 + c) * p.d_ff + jrow;
-                            if (p.dtype == CLADA_BF16)
-                                static_cast<__nv_bfloat16 *>(p.z_out)[at] = __float2bfloat16_rn(z);
-                            else
-                                static_cast<__half *>(p.z_out)[at] = __float2half_rn(z);
-                        }
+                    z[c] = tok_ok ? neuron_value_f(p.act, __uint_as_float(rg[c]), __uint_as_float(ru[c])) : 0.f;
+                    q[c] = z[c] * z[c];
+                }
+                if (p.z_out && tok_ok) {  // 16 consecutive neurons of this token: two 16-byte stores
+                    const int j0 = jbase + c0;
+                    uint16_t *dst = static_cast<uint16_t *>(p.z_out) + (size_t)(t0 + row) * p.d_ff + j0;
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        if (j0 + 8 * h + 8 > p.d_ff) continue;  // d_ff is a multiple of 8 when Z is asked for
+                        const uint2 lo = pack4_16bit(p.dtype, make_float4(z[8 * h], z[8 * h + 1], z[8 * h + 2], z[8 * h + 3]));
+                        const uint2 hi = pack4_16bit(p.dtype, make_float4(z[8 * h + 4], z[8 * h + 5], z[8 * h + 6], z[8 * h + 7]));
+                        *reinterpret_cast<uint4 *>(dst + 8 * h) = make_uint4(lo.x, lo.y, hi.x, hi.y);
                     }
                 }
+                // Sum of z^2 over the warp's 32 tokens for each of the 16 neurons: a halving butterfly (16
+                // shuffles) that leaves the total of neuron my_val on every lane.  Fixed order.
+                float v8[8], v4[4], v2[2], v1;
+#pragma unroll
+                for (int i = 0; i < 8; ++i)
+                    v8[i] = (b16 ? q[i + 8] : q[i]) + __shfl_xor_sync(0xffffffffu, b16 ? q[i] : q[i + 8], 16);
+#pragma unroll
+                for (int i = 0; i < 4; ++i)
+                    v4[i] = (b8 ? v8[i + 4] : v8[i]) + __shfl_xor_sync(0xffffffffu, b8 ? v8[i] : v8[i + 4], 8);
+#pragma unroll
+                for (int i = 0; i < 2; ++i)
+                    v2[i] = (b4 ? v4[i + 2] : v4[i]) + __shfl_xor_sync(0xffffffffu, b4 ? v4[i] : v4[i + 2], 4);
+                v1 = (b2 ? v2[1] : v2[0]) + __shfl_xor_sync(0xffffffffu, b2 ? v2[0] : v2[1], 2);
+                v1 += __shfl_xor_sync(0xffffffffu, v1, 1);
+                if ((lane & 1) == 0) s_col[a][quarter][c0 + my_val] = v1;
             }
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) tc_mbar_arrive(tc_smem_u32(&s_acc_empty[a]));
-            const int j = ntile * kTcTileM + quarter * 32 + lane;
-            if (j < p.d_ff) p.partials[(size_t)ttile * p.d_ff + j] = sum;
+            if (lane == 0) tc_mbar_arrive(tc_smem_u32(&s_acc_empty[a]));  // the accumulator may be overwritten
+            // the four warps' token groups, added in warp order; s_col alternates with the accumulator, so a
+            // warp that runs ahead writes the other half while this one is still being read
+            // (an mbarrier rather than a hardware barrier: its wait is bounded like every other one here)
+            if (lane == 0) tc_mbar_arrive(tc_smem_u32(&s_epi[a]));
+            if (!tc_mbar_wait(tc_smem_u32(&s_epi[a]), (it >> 1) & 1, abort_flag)) {
+                ok = false;
+                break;
+            }
+            const int j = jbase + e;
+            if (e < nt && j < p.d_ff)
+                p.partials[(size_t)ttile * p.d_ff + j] = ((s_col[a][0][e] + s_col[a][1][e]) + s_col[a][2][e]) + s_col[a][3][e];
         }
         if (!ok) *abort_flag = 1;
     }
@@ -318,12 +381,13 @@ static int encode_fn(EncodeTiledFn *out) {
     return CLADA_OK;
 }
 
-// Row-major bf16 or fp16 matrix [rows, cols] as a 2-D tensor map with a {64, 128} box and 128-byte swizzle;
+// Row-major bf16 or fp16 matrix [rows, cols] as a 2-D tensor map with a {64, box_rows} box and 128-byte swizzle;
 // out-of-range rows and columns read as zero.
-static int make_map(EncodeTiledFn enc, CUtensorMap *map, const void *base, long long rows, int cols, int dtype) {
+static int make_map(EncodeTiledFn enc, CUtensorMap *map, const void *base, long long rows, int cols, int dtype,
+                    int box_rows = kTcTileM) {
     const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
     const cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
-    const cuuint32_t box[2] = {(cuuint32_t)kTcTileK, (cuuint32_t)kTcTileM};
+    const cuuint32_t box[2] = {(cuuint32_t)kTcTileK, (cuuint32_t)box_rows};
     const cuuint32_t estr[2] = {1, 1};
     const CUtensorMapDataType et = dtype == CLADA_F16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
     const CUresult r = enc(map, et, 2, const_cast<void *>(base), dims, strides, box, estr,
@@ -340,7 +404,7 @@ int run_prefix_partials_tc(const clada_layer *layer, const void *X, const SeqTab
                            float *partials, int32_t *status, cudaStream_t st, void *z_out) {
     static bool configured[64] = {};
     int n_ttiles = 0;
-    for (int b = 0; b < tab.B; ++b) n_ttiles += tiles_of(tab.off[b + 1] - tab.off[b], kTcTileN);
+    for (int b = 0; b < tab.B; ++b) n_ttiles += tiles_of(tab.off[b + 1] - tab.off[b], kTcTileM);
     if (n_ttiles == 0) return CLADA_OK;
     DeviceInfo di;
     int rc = device_info(&di);
@@ -348,32 +412,44 @@ int run_prefix_partials_tc(const clada_layer *layer, const void *X, const SeqTab
     EncodeTiledFn enc;
     rc = encode_fn(&enc);
     if (rc != CLADA_OK) return rc;
-    CUtensorMap map_x, map_wg, map_wu;
+    const bool gated = act_is_gated(layer->activation);
+    CUtensorMap map_x, map_wg, map_wu, map_wg_half, map_wu_half;
+    // without a gate projection the w_up maps are never used by the kernel: give them w_gate's address
+    const void *wu = gated ? layer->w_up : layer->w_gate;
     if ((rc = make_map(enc, &map_x, X, T_total, layer->d_model, layer->dtype)) != CLADA_OK) return rc;
-    if ((rc = make_map(enc, &map_wg, layer->w_gate, layer->d_ff, layer->d_model, layer->dtype)) != CLADA_OK) return rc;
-    // without a gate projection the w_up map is never used by the kernel: give it w_gate's address
-    const void *wu = act_is_gated(layer->activation) ? layer->w_up : layer->w_gate;
-    if ((rc = make_map(enc, &map_wu, wu, layer->d_ff, layer->d_model, layer->dtype)) != CLADA_OK) return rc;
+    if ((rc = make_map(enc, &map_wg, layer->w_gate, layer->d_ff, layer->d_model, layer->dtype, 128)) != CLADA_OK) return rc;
+    if ((rc = make_map(enc, &map_wu, wu, layer->d_ff, layer->d_model, layer->dtype, 128)) != CLADA_OK) return rc;
+    if ((rc = make_map(enc, &map_wg_half, layer->w_gate, layer->d_ff, layer->d_model, layer->dtype, 64)) != CLADA_OK) return rc;
+    if ((rc = make_map(enc, &map_wu_half, wu, layer->d_ff, layer->d_model, layer->dtype, 64)) != CLADA_OK) return rc;
     TcParams p;
     p.d_model = layer->d_model;
     p.d_ff = layer->d_ff;
-    p.n_ntiles = (layer->d_ff + kTcTileM - 1) / kTcTileM;
+    p.n_ntiles = (layer->d_ff + 127) / 128;
     p.n_ttiles = n_ttiles;
+    // The items left over after the last full wave of CTAs run as 64-neuron halves when they then still fit one
+    // wave: that wave takes half the time.  (Halves read more bytes per flop, so only the tail is split.)
+    const long long items = (long long)p.n_ntiles * n_ttiles;
+    const long long rest = items % di.num_sms;
+    const long long split = (items > di.num_sms && 2 * rest <= di.num_sms) ? rest : 0;
+    p.n_full = (int)(items - split);
+    p.n_half = (int)(2 * split);
     p.partials = partials;
     p.status = status;
     p.act = layer->activation;
     p.z_out = z_out;
     p.dtype = layer->dtype;
-    p.idesc = layer->dtype == CLADA_F16 ? kTcInstrDescF16 : kTcInstrDescBf16;
+    p.idesc = tc_instr_desc(layer->dtype, gated ? 256 : 128);  // gate | up columns in one instruction
+    p.idesc_half = tc_instr_desc(layer->dtype, gated ? 128 : 64);
     p.tab = tab;
-    const size_t smem = (size_t)kTcStages * kTcStageBytes + 1024;
+    const uint32_t stage_bytes = kTcTileBytes + (gated ? 2u : 1u) * kTcTileBytes;
+    p.n_stages = std::min<int>(kTcMaxStages, (int)(kTcRingBytes / stage_bytes));
+    const size_t smem = (size_t)kTcRingBytes + 1024;
     if (!configured[di.device & 63]) {
         CLADA_CUDA_TRY(cudaFuncSetAttribute(prefix_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
         configured[di.device & 63] = true;
     }
-    const long long items = (long long)p.n_ntiles * n_ttiles;
-    const int grid = (int)std::min<long long>(items, di.num_sms);
-    prefix_tc_kernel<<<grid, kTcThreads, smem, st>>>(map_x, map_wg, map_wu, p);
+    const int grid = (int)std::min<long long>((long long)p.n_full + p.n_half, di.num_sms);
+    prefix_tc_kernel<<<grid, kTcThreads, smem, st>>>(map_x, map_wg, map_wu, map_wg_half, map_wu_half, p);
     CLADA_CUDA_TRY(cudaGetLastError());
     return CLADA_OK;
 }
@@ -568,7 +644,7 @@ int run_down_tc(const clada_layer *layer, const void *w_down, const void *Z, lon
     p.n_dtiles = (layer->d_model + kTcTileN - 1) / kTcTileN;
     p.y = Y;
     p.y_dtype = y_dtype;
-    p.idesc = layer->dtype == CLADA_F16 ? kTcInstrDescF16 : kTcInstrDescBf16;
+    p.idesc = tc_instr_desc(layer->dtype, kTcTileN);
     p.status = status;
     const size_t smem = (size_t)kDnStages * kDnStageBytes + 1024;
     if (!configured[di.device & 63]) {
