@@ -27,7 +27,6 @@
 namespace clada {
 
 constexpr int kTcTileM = 128;   // rows of the A tile = TMEM lanes (tokens; also the most neurons per tile)
-constexpr int kTcTileN = 128;   // columns of a down-projection tile
 constexpr int kTcTileK = 64;    // K block: 64 16-bit elements = 128 bytes = one swizzle row
 constexpr int kTcMaxStages = 8;
 constexpr int kTcThreads = 192;
@@ -458,16 +457,18 @@ int run_prefix_partials_tc(const clada_layer *layer, const void *X, const SeqTab
 //   Y[t, i] = sum_j Z[t, j] * W_out[i, j]      (Z: hidden activations, W_out in the paper's [d_model, d_ff] layout)
 // Both operands are K-major (d_ff contiguous), so the tiles, descriptors and the role split are those of
 // the statistics kernel: tokens are the M dimension (TMEM lanes), output columns the N dimension, one
-// accumulator per tile, two in flight.  The epilogue thread that owns token t writes its row of the tile.
+// accumulator per tile (256 output columns, or 128 for short prompts), two in flight.  The epilogue thread
+// that owns token t writes its row of the tile.
 
-constexpr int kDnStages = 6;
-constexpr uint32_t kDnStageBytes = 2 * kTcTileBytes;  // Z tile | W_out tile
-constexpr uint32_t kDnTmemCols = 256;                 // two 128-column accumulators
+constexpr int kDnMaxStages = 6;
+constexpr uint32_t kDnTmemCols = 512;                 // two accumulators of up to 256 columns
 
 struct DownParams {
     int d_model, d_ff;
     long long T;
     int n_ttiles, n_dtiles;
+    int nd;        // output columns per tile: 256 (fewer bytes read per flop), or 128 when 256 would leave SMs idle
+    int n_stages;
     void *y;
     int y_dtype;
     uint32_t idesc;
@@ -479,16 +480,18 @@ down_tc_kernel(const __grid_constant__ CUtensorMap map_z, const __grid_constant_
                const DownParams p) {
     extern __shared__ unsigned char tc_smem_raw[];
     const uint32_t smem0 = (tc_smem_u32(tc_smem_raw) + 1023u) & ~1023u;
-    __shared__ __align__(8) uint64_t s_full[kDnStages], s_empty[kDnStages], s_acc_full[2], s_acc_empty[2];
+    __shared__ __align__(8) uint64_t s_full[kDnMaxStages], s_empty[kDnMaxStages], s_acc_full[2], s_acc_empty[2];
     __shared__ uint32_t s_tmem_base;
     __shared__ int s_abort;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int n_items = p.n_ttiles * p.n_dtiles;
+    const int nd = p.nd, n_stages = p.n_stages;
+    const uint32_t stage_bytes = kTcTileBytes + (uint32_t)nd * kTcTileK * 2u;  // Z tile | W_out tile
     const int n_kblocks = (p.d_ff + kTcTileK - 1) / kTcTileK;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < kDnStages; ++s) {
+        for (int s = 0; s < n_stages; ++s) {
             tc_mbar_init(tc_smem_u32(&s_full[s]), 1);
             tc_mbar_init(tc_smem_u32(&s_empty[s]), 1);
         }
@@ -515,31 +518,38 @@ down_tc_kernel(const __grid_constant__ CUtensorMap map_z, const __grid_constant_
     if (warp == 0) {
         if (lane == 0) {
             int kc = 0;
+            int s = 0;  // ring position and the parity of its current use, kept incrementally
+            uint32_t par = 0;
             bool ok = true;
             for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
                 const int dtile = item / p.n_ttiles, ttile = item % p.n_ttiles;
                 for (int kb = 0; kb < n_kblocks; ++kb, ++kc) {
-                    const int s = kc % kDnStages;
-                    if (!tc_mbar_wait(tc_smem_u32(&s_empty[s]), ((kc / kDnStages) & 1) ^ 1, abort_flag)) {
+                    if (!tc_mbar_wait(tc_smem_u32(&s_empty[s]), par ^ 1, abort_flag)) {
                         ok = false;
                         break;
                     }
                     const uint32_t bar = tc_smem_u32(&s_full[s]);
-                    const uint32_t dst = smem0 + (uint32_t)s * kDnStageBytes;
-                    tc_mbar_expect_tx(bar, kDnStageBytes);
+                    const uint32_t dst = smem0 + (uint32_t)s * stage_bytes;
+                    tc_mbar_expect_tx(bar, stage_bytes);
                     tc_tma_load(dst, &map_z, kb * kTcTileK, ttile * kTcTileM, bar);
-                    tc_tma_load(dst + kTcTileBytes, &map_w, kb * kTcTileK, dtile * kTcTileN, bar);
+                    tc_tma_load(dst + kTcTileBytes, &map_w, kb * kTcTileK, dtile * nd, bar);
+                    if (++s == n_stages) {
+                        s = 0;
+                        par ^= 1;
+                    }
                 }
             }
             if (!ok) *abort_flag = 1;
-            for (int i = max(0, kc - kDnStages); i < kc; ++i) {
+            for (int i = max(0, kc - n_stages); i < kc; ++i) {
                 int never = 0;  // these copies land by themselves: wait for them even after an abort
-                if (!tc_mbar_wait(tc_smem_u32(&s_full[i % kDnStages]), (i / kDnStages) & 1, &never)) *abort_flag = 1;
+                if (!tc_mbar_wait(tc_smem_u32(&s_full[i % n_stages]), (i / n_stages) & 1, &never)) *abort_flag = 1;
             }
         }
     } else if (warp == 1) {
         if (lane == 0) {
-            int kc = 0, it = 0;
+            int it = 0;
+            int s = 0;
+            uint32_t par = 0;
             bool ok = true;
             for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++it) {
                 const int a = it & 1;
@@ -548,20 +558,23 @@ down_tc_kernel(const __grid_constant__ CUtensorMap map_z, const __grid_constant_
                     break;
                 }
                 tc_fence_after();
-                const uint32_t d_acc = tmem_base + (uint32_t)a * 128u;
-                for (int kb = 0; kb < n_kblocks; ++kb, ++kc) {
-                    const int s = kc % kDnStages;
-                    if (!tc_mbar_wait(tc_smem_u32(&s_full[s]), (kc / kDnStages) & 1, abort_flag)) {
+                const uint32_t d_acc = tmem_base + (uint32_t)a * 256u;
+                for (int kb = 0; kb < n_kblocks; ++kb) {
+                    if (!tc_mbar_wait(tc_smem_u32(&s_full[s]), par, abort_flag)) {
                         ok = false;
                         break;
                     }
                     tc_fence_after();
-                    const uint32_t base = smem0 + (uint32_t)s * kDnStageBytes;
+                    const uint32_t base = smem0 + (uint32_t)s * stage_bytes;
                     const uint64_t dz = tc_smem_desc(base), dw = tc_smem_desc(base + kTcTileBytes);
 #pragma unroll
                     for (int k = 0; k < kTcTileK / 16; ++k)
                         tc_mma(d_acc, dz + 2 * k, dw + 2 * k, (kb > 0 || k > 0) ? 1u : 0u, p.idesc);
                     tc_commit(tc_smem_u32(&s_empty[s]));
+                    if (++s == n_stages) {
+                        s = 0;
+                        par ^= 1;
+                    }
                 }
                 if (ok) tc_commit(tc_smem_u32(&s_acc_full[a]));
             }
@@ -579,10 +592,10 @@ down_tc_kernel(const __grid_constant__ CUtensorMap map_z, const __grid_constant_
                 break;
             }
             tc_fence_after();
-            const uint32_t t_acc = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)a * 128u;
+            const uint32_t t_acc = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)a * 256u;
             const long long t = (long long)ttile * kTcTileM + quarter * 32 + lane;
-            const int i0 = dtile * kTcTileN;
-            const int ncols = min(kTcTileN, p.d_model - i0);  // a multiple of 8 (d_model is)
+            const int i0 = dtile * nd;
+            const int ncols = min(nd, p.d_model - i0);  // a multiple of 8 (d_model is)
             for (int c0 = 0; c0 < ncols; c0 += 16) {           // uniform per warp
                 uint32_t r[16];
                 tc_ld16(t_acc + c0, r);
@@ -635,18 +648,22 @@ int run_down_tc(const clada_layer *layer, const void *w_down, const void *Z, lon
     if (rc != CLADA_OK) return rc;
     CUtensorMap map_z, map_w;
     if ((rc = make_map(enc, &map_z, Z, T, layer->d_ff, layer->dtype)) != CLADA_OK) return rc;
-    if ((rc = make_map(enc, &map_w, w_down, layer->d_model, layer->d_ff, layer->dtype)) != CLADA_OK) return rc;
     DownParams p;
     p.d_model = layer->d_model;
     p.d_ff = layer->d_ff;
     p.T = T;
     p.n_ttiles = (int)((T + kTcTileM - 1) / kTcTileM);
-    p.n_dtiles = (layer->d_model + kTcTileN - 1) / kTcTileN;
+    // 256 output columns per tile unless that leaves SMs without a tile
+    p.nd = (long long)p.n_ttiles * ((layer->d_model + 255) / 256) >= di.num_sms ? 256 : 128;
+    p.n_dtiles = (layer->d_model + p.nd - 1) / p.nd;
+    const uint32_t dn_stage = kTcTileBytes + (uint32_t)p.nd * kTcTileK * 2u;
+    p.n_stages = std::min<int>(kDnMaxStages, (int)(kTcRingBytes / dn_stage));
     p.y = Y;
     p.y_dtype = y_dtype;
-    p.idesc = tc_instr_desc(layer->dtype, kTcTileN);
+    p.idesc = tc_instr_desc(layer->dtype, p.nd);
     p.status = status;
-    const size_t smem = (size_t)kDnStages * kDnStageBytes + 1024;
+    if ((rc = make_map(enc, &map_w, w_down, layer->d_model, layer->d_ff, layer->dtype, p.nd)) != CLADA_OK) return rc;
+    const size_t smem = (size_t)kTcRingBytes + 1024;
     if (!configured[di.device & 63]) {
         CLADA_CUDA_TRY(cudaFuncSetAttribute(down_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
         configured[di.device & 63] = true;

@@ -150,10 +150,11 @@ def test_chunked_statistics_equal_whole_prompt(clada, oracle, name, kw):
     assert torch.allclose(scores, whole, rtol=2e-6, atol=0)
 
 
-def test_prefill_full_width_c2(clada, oracle):
-    """The benchmark's layer at full width, 512-token prompt: sampled rows of Z and Y against the oracle."""
+@pytest.mark.parametrize("T", [512, 2048])
+def test_prefill_full_width_c2(clada, oracle, T):
+    """The benchmark's layer at full width: sampled rows of Z and Y against the oracle.  512 tokens run the down
+    projection in 128-column tiles, 2048 tokens in 256-column tiles."""
     w = wl.WORKLOADS["c2_llama2_7b_layer"]
-    T = 512
     weights = wl.layer_weights(w, 0, "cuda")
     layer = gpu_layer(weights, clada)
     X = wl.hidden_states(w, 0, "prefix", 0, T, "cuda", wl.channel_scale(w, "cuda"))
@@ -170,7 +171,7 @@ def test_prefill_full_width_c2(clada, oracle):
     clada.clada_prefix_scores(layer, X, [0, T], whole, ws, status)
     torch.cuda.synchronize()
     assert int(status.item()) == 0 and torch.equal(scores, whole)      # one chunk: the very same sums
-    rows = [0, 127, 128, 300, 511]
+    rows = [0, 127, 128, 300, T - 1]
     W_in, V_in, W_out = oracle_weights(weights)
     Xn = wl.to_numpy_bits(X[rows])
     Z_or = oracle.prefill_hidden(Xn, W_in, V_in, round_z=True)
