@@ -1,20 +1,26 @@
-// Prefill statistics (Eq. neuron_activation) on the 5th-generation tensor cores, bf16 inputs:
-//   gate[j,t] = w_gate_j . x_t,  up[j,t] = w_up_j . x_t   (fp32 accumulators in tensor memory)
-//   partial[tile, j] = sum_{t in tile} (silu(gate[j,t]) * up[j,t])^2
+// Prefill statistics (Eq. neuron_activation) on the 5th-generation tensor cores, bf16 or fp16 inputs:
+//   gate[t,j] = x_t . w_gate_j,  up[t,j] = x_t . w_up_j   (fp32 accumulator in tensor memory)
+//   partial[tile, j] = sum_{t in tile} z[t,j]^2,  z = value of neuron j for token t in the layer's FFN form
+// and, on request, the hidden activations z[t,j] themselves (the dense prefill FFN's first half).
 //
-// Neurons are the M dimension (128 per tile = the 128 TMEM lanes), tokens the N dimension (128 per
-// tile = 128 TMEM columns), d_model the K dimension.  The epilogue thread that owns lane j therefore
-// walks its own row of both accumulators and adds z^2 over the tile's tokens serially in a register:
-// no cross-lane reduction, no z ever written.  A token tile never leaves its prompt; columns beyond
-// the prompt's end are skipped.
+// Tokens are the M dimension (128 per tile = the 128 TMEM lanes), d_model the K dimension, and the B operand is
+// a tile of w_gate rows with the same neurons' w_up rows right behind it in shared memory: ONE instruction of
+// N = 256 columns (gate | up) per 16-wide K step reads 12 KB of operands per MFLOP instead of the 16 KB two
+// N = 128 instructions would, and the epilogue thread that owns token t finds gate and up of a neuron in its own
+// lane.  The sum over a tile's tokens is then a sum over lanes: a halving butterfly per 16 neurons (16 shuffles),
+// the four warps' results combined through shared memory in warp order (deterministic).
 //
 // One persistent CTA per SM, 192 threads:
-//   warp 0      TMA producer: per 64-wide K block three 128 x 64 bf16 tiles (w_gate, w_up, X), 128-byte
-//               swizzle, into a 4-stage shared-memory ring (mbarrier full/empty);
-//   warp 1      allocates 512 TMEM columns (two accumulator pairs), issues tcgen05.mma (M128 N128 K16,
-//               kind::f16) for gate and up from one elected thread, commits stages and accumulators;
-//   warps 2-5   epilogue: tcgen05.ld 32x32b.x16 of both accumulators, silu * up, square, sum; the
-//               second accumulator pair lets tile i+1's MMAs run under tile i's epilogue.
+//   warp 0      TMA producer: per 64-wide K block the token tile and the two weight tiles, 128-byte swizzle, into a
+//               4-stage shared-memory ring (mbarrier full/empty);
+//   warp 1      allocates 512 TMEM columns (two accumulators), issues tcgen05.mma (M128 N256 K16, kind::f16) from
+//               one elected thread, commits stages and accumulators;
+//   warps 2-5   epilogue: tcgen05.ld 32x32b.x16 of gate and up columns, neuron value, optional store of 16
+//               consecutive neurons of the thread's token, squares, butterfly; the second accumulator lets tile
+//               i+1's MMAs run under tile i's epilogue.
+// Work items are (128 neurons x 128 tokens), neuron tile major; a token tile never leaves its prompt and rows
+// past the prompt's end count as zero.  The items left after the last full wave of CTAs are issued as two
+// 64-neuron halves each (N = 128) when they then fit one wave, which halves that wave's time.
 // Every wait is bounded; on expiry the CTA raises CLADA_STATUS_TIMEOUT, drains its copies and frees TMEM.
 #include <cuda.h>
 #include <math.h>
