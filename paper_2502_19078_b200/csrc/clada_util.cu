@@ -93,7 +93,7 @@ const char *clada_status_string(int code) {
         case CLADA_ERR_DTYPE: return "unknown or unsupported dtype";
         case CLADA_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
         case CLADA_ERR_CUDA: return "CUDA runtime error (see clada_last_cuda_error)";
-        case CLADA_ERR_UNSUPPORTED: return "size beyond what the kernels support";
+        case CLADA_ERR_UNSUPPORTED: return "size, element type or option beyond what the kernels support";
         default: return "unknown status";
     }
 }

@@ -181,3 +181,34 @@ def test_prefill_full_width_c2(clada, oracle, T):
     Yg = Y[rows].cpu().numpy().astype(np.float64)
     assert rel_inf(Yg, oracle.down_proj(Zg, W_out)) <= DOWN_TOL
     assert rel_inf(Yg, oracle.down_proj(Z_or, W_out)) <= FFN_TOL
+
+
+def test_new_entry_points_refuse_what_they_cannot_do(clada):
+    """Host-side checks: nothing is launched, the context stays usable."""
+    w32 = wl.scaled(wl.WORKLOADS["c1_small_f32"], d_model=64, d_ff=96)
+    l32 = gpu_layer(wl.layer_weights(w32, 0), clada)
+    ws = clada.new_workspace(l32, 1, 16)
+    X = torch.zeros(16, 64, device="cuda")
+    sumsq = torch.zeros(1, 96, device="cuda")
+    Z32 = torch.empty(16, 96, device="cuda")
+    with pytest.raises(clada.CladaError, match="support"):          # hidden activations: 16-bit layers only
+        clada.clada_prefix_accumulate(l32, X, [0, 16], sumsq, ws, Z32)
+    with pytest.raises(clada.CladaError, match="support"):
+        clada.clada_prefill_down(l32, torch.zeros(64, 96, device="cuda"), Z32, torch.empty(16, 64, device="cuda"))
+    clada.clada_prefix_accumulate(l32, X, [0, 16], sumsq, ws, None)      # statistics alone work for fp32
+    wb = wl.scaled(wl.WORKLOADS["c2_llama2_7b_layer"], d_model=64, d_ff=100)   # d_ff % 8 != 0
+    lb = gpu_layer(wl.layer_weights(wb, 0), clada)
+    wsb = clada.new_workspace(lb, 1, 16)
+    Xb = torch.zeros(16, 64, dtype=torch.bfloat16, device="cuda")
+    Zb = torch.empty(16, 100, dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(clada.CladaError, match="shape"):
+        clada.clada_prefix_accumulate(lb, Xb, [0, 16], torch.zeros(1, 100, device="cuda"), wsb, Zb)
+    with pytest.raises(clada.CladaError, match="shape"):
+        clada.clada_prefill_down(lb, torch.zeros(64, 100, dtype=torch.bfloat16, device="cuda"), Zb,
+                                 torch.empty(16, 64, device="cuda"))
+    big = torch.ones(1, 16385, device="cuda")                             # the list sort holds 16384 keys
+    with pytest.raises(clada.CladaError, match="support"):
+        clada.clada_nested_build(big, torch.ones(1, device="cuda"), 0.8, 0.12,
+                                 torch.empty(1, 16385, dtype=torch.int32, device="cuda"),
+                                 torch.empty(1, 4, dtype=torch.int32, device="cuda"))
+    torch.cuda.synchronize()
