@@ -87,10 +87,32 @@ cogload_kernel(const T *__restrict__ logits, int64_t V, int64_t row_stride,
     const T *row = logits + (size_t)b * row_stride;
     const int tid = threadIdx.x;
     pdl_launch_dependents();
+    // First cluster phase: "every CTA of the cluster has started", which a write into another CTA's shared
+    // memory needs.  Arrive now, wait only just before that write: by then the phase has long completed.
+    asm volatile("barrier.cluster.arrive.relaxed.aligned;" ::: "memory");
     pdl_wait();
 
     SoftStat st = stat_empty();
     bool bad = false;
+
+    // Loads that only the last steps need are issued first, so that their latency hides under the row's:
+    // the chosen token and its logit (two dependent loads), and the first adjustment operands per thread.
+    int32_t tok = 0;
+    bool tok_ok = false;
+    float tok_logit = 0.f;
+    float adj_base = 0.f, adj_lambda = 0.f, adj_gamma = 0.f;
+    if (slice == 0) {
+        if (tid == 0) {
+            tok = token_id[b];
+            tok_ok = tok >= 0 && tok < V;
+            if (tok_ok) tok_logit = load_logit(row, tok);
+        }
+        if (tau_base != nullptr && tid < L) {
+            adj_base = tau_base[(size_t)b * L + tid];
+            adj_lambda = lambda[tid];
+            adj_gamma = gamma[tid];
+        }
+    }
 
     // The row as scalar head (up to the first 16-byte boundary), 16-byte vectors, scalar tail; the
     // vectors are dealt to the slices in contiguous runs, head and tail go to slice 0.
@@ -138,7 +160,7 @@ cogload_kernel(const T *__restrict__ logits, int64_t V, int64_t row_stride,
         st = ((tid & o) == 0) ? stat_merge(st, other) : stat_merge(other, st);
     }
     __shared__ SoftStat s_stat[kCogThreads / kWarp];
-    __shared__ SoftStat s_slice;  // this CTA's slice, read by rank 0
+    __shared__ SoftStat s_all[kCogMaxCluster];  // on rank 0: every slice's statistic, written by its owner
     __shared__ int s_bad;
     __shared__ float s_out[2];
     if (tid == 0) s_bad = 0;
@@ -157,14 +179,18 @@ cogload_kernel(const T *__restrict__ logits, int64_t V, int64_t row_stride,
             tot = ((tid & o) == 0) ? stat_merge(tot, other) : stat_merge(other, tot);
         }
         if (s_bad) tot.z = NAN;  // carries the non-finite flag to rank 0
-        if (tid == 0) s_slice = tot;
+        // every CTA started (first phase) before anyone writes into rank 0's shared memory
+        asm volatile("barrier.cluster.wait.aligned;" ::: "memory");
+        if (tid == 0) *cluster.map_shared_rank(&s_all[slice], 0) = tot;
+    } else {
+        asm volatile("barrier.cluster.wait.aligned;" ::: "memory");
     }
-    cluster.sync();
+    cluster.sync();  // the statistics have landed; the other CTAs are done and may leave
     if (slice == 0) {
         if (tid < kWarp) {
-            // lane r fetches slice r's statistic over distributed shared memory, then a butterfly merges them
+            // lane r takes slice r's statistic, then a butterfly merges them
             SoftStat tot = stat_empty();
-            if (tid < n_slices) tot = *cluster.map_shared_rank(&s_slice, tid);
+            if (tid < n_slices) tot = s_all[tid];
 #pragma unroll
             for (int o = kCogMaxCluster / 2; o > 0; o >>= 1) {
                 SoftStat other;
@@ -182,12 +208,11 @@ cogload_kernel(const T *__restrict__ logits, int64_t V, int64_t row_stride,
                 } else {
                     const float logz = logf(tot.z);
                     h = logz - tot.w / tot.z;
-                    const int32_t tok = token_id[b];
-                    if (tok < 0 || tok >= V) {
+                    if (!tok_ok) {
                         flags |= CLADA_STATUS_BAD_TOKEN;
                         s = NAN;
                     } else {
-                        s = (tot.m + logz) - load_logit(row, tok);
+                        s = (tot.m + logz) - tok_logit;
                     }
                 }
                 surprisal[b] = s;
@@ -202,7 +227,13 @@ cogload_kernel(const T *__restrict__ logits, int64_t V, int64_t row_stride,
         if (tau_base != nullptr) {
             __syncthreads();
             const float s = s_out[0], h = s_out[1];
-            for (int l = tid; l < L; l += kCogThreads) {
+            if (tid < L) {  // operands fetched at the start
+                float mult = 1.0f;
+                if (s > tau_s) mult = __fadd_rn(mult, adj_lambda);
+                if (h > tau_H) mult = __fadd_rn(mult, adj_gamma);
+                tau_final[(size_t)b * L + tid] = __fmul_rn(adj_base, mult);
+            }
+            for (int l = tid + kCogThreads; l < L; l += kCogThreads) {
                 float mult = 1.0f;
                 if (s > tau_s) mult = __fadd_rn(mult, lambda[l]);
                 if (h > tau_H) mult = __fadd_rn(mult, gamma[l]);
@@ -210,7 +241,6 @@ cogload_kernel(const T *__restrict__ logits, int64_t V, int64_t row_stride,
             }
         }
     }
-    cluster.sync();  // no CTA leaves while rank 0 may still read its shared memory
 }
 
 __global__ void adjust_threshold_kernel(const float *__restrict__ tau_base,
