@@ -200,7 +200,8 @@ class Job:
 
     @property
     def launches_per_step(self) -> int:
-        return 2 + len(self.w.sparsities) * (3 + 2 * self.N)
+        # prefix (2) + per sparsity: guard band (candidates, refine, finish), select, N x (cogload, FFN)
+        return 2 + len(self.w.sparsities) * (4 + 2 * self.N)
 
     def tokens_per_step(self) -> int:
         return len(self.w.sparsities) * self.N
@@ -305,7 +306,7 @@ class StackJob:
 
     @property
     def launches_per_step(self) -> int:
-        return self.L * 6 + self.N * (1 + self.L)
+        return self.L * 7 + self.N * (1 + self.L)
 
     def tokens_per_step(self) -> int:
         return self.N

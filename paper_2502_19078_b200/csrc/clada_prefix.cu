@@ -206,15 +206,26 @@ template <> struct Widen<__nv_bfloat16> {
     }
 };
 
-// One CTA per candidate (grid-stride).  The candidate's gate and up rows are widened to fp64 once into
-// shared memory; each of the 32 warps takes every 32nd token of the prompt, lanes split d_model by
-// 16-byte vectors, products and sums in fp64.  Warp and CTA sums are taken in a fixed order.
+// How many CTAs share one candidate's prompt: with fewer candidates than CTAs, each candidate's tokens are
+// dealt to several CTAs (the partial sums meet in guard_finish_kernel), so the whole GPU works on the band.
+constexpr int kRefMaxUnits = 512;  // (candidate, split) partial sums held in the workspace
+__host__ __device__ inline int guard_splits(int total, int n_ctas) {
+    if (total <= 0 || total >= n_ctas) return 1;
+    int s = n_ctas / total;
+    if (s > 32) s = 32;
+    while (s > 1 && total * s > kRefMaxUnits) --s;
+    return s;
+}
+
+// One CTA per (candidate, split) (grid-stride).  The candidate's gate and up rows are widened to fp64 once
+// into shared memory; each of the 32 warps takes every (32 * splits)-th token of the prompt, lanes split
+// d_model by 16-byte vectors, products and sums in fp64.  Warp and CTA sums are taken in a fixed order.
 template <typename T>
 __global__ void __launch_bounds__(kRefThreads)
 guard_refine_kernel(const T *__restrict__ X, const T *__restrict__ Wg, const T *__restrict__ Wu,
                     const T *__restrict__ Wd_t, int d_model, int d_ff, const SeqTable tab,
                     const int *__restrict__ n_cand, const int2 *__restrict__ cand,
-                    float *__restrict__ scores, int act) {
+                    float *__restrict__ scores, int act, double2 *__restrict__ part) {
     constexpr int E = Elem<T>::kPerVec;
     constexpr int kWarps = kRefThreads / kWarp;
     extern __shared__ __align__(16) double s_rows[];  // gate row | up row, fp64
@@ -223,7 +234,9 @@ guard_refine_kernel(const T *__restrict__ X, const T *__restrict__ Wg, const T *
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int vpr = d_model / E;
     const int total = *n_cand;
-    for (int c = blockIdx.x; c < total; c += gridDim.x) {
+    const int S = guard_splits(total, (int)gridDim.x);
+    for (int unit = blockIdx.x; unit < total * S; unit += gridDim.x) {
+        const int c = unit / S, split = unit % S;
         const int b = cand[c].x, j = cand[c].y;
         const uint4 *wg = reinterpret_cast<const uint4 *>(Wg + (size_t)j * d_model);
         const uint4 *wu = reinterpret_cast<const uint4 *>(Wu + (size_t)j * d_model);
@@ -245,7 +258,7 @@ guard_refine_kernel(const T *__restrict__ X, const T *__restrict__ Wg, const T *
         }
         __syncthreads();
         double zz = 0.0;
-        for (long long t = tab.off[b] + warp; t < tab.off[b + 1]; t += kWarps) {
+        for (long long t = tab.off[b] + warp + (long long)kWarps * split; t < tab.off[b + 1]; t += (long long)kWarps * S) {
             const uint4 *x = reinterpret_cast<const uint4 *>(X + (size_t)t * d_model);
             double g = 0.0, u = 0.0;
 #pragma unroll 4
@@ -282,9 +295,25 @@ guard_refine_kernel(const T *__restrict__ X, const T *__restrict__ Wg, const T *
                 a += s_zz[w];
                 n2 += s_nn[w];
             }
-            scores[(size_t)b * d_ff + j] = (float)(sqrt(a) * sqrt(n2));
+            if (S == 1)
+                scores[(size_t)b * d_ff + j] = (float)(sqrt(a) * sqrt(n2));
+            else
+                part[unit] = make_double2(a, n2);  // this split's share of the sum over tokens
         }
         __syncthreads();
+    }
+}
+
+// The splits of a candidate added in split order (only launched work when candidates were split).
+__global__ void guard_finish_kernel(const int *__restrict__ n_cand, const int2 *__restrict__ cand, int n_ctas, int d_ff,
+                                    const double2 *__restrict__ part, float *__restrict__ scores) {
+    const int total = *n_cand;
+    const int S = guard_splits(total, n_ctas);
+    if (S == 1) return;
+    for (int c = blockIdx.x * blockDim.x + threadIdx.x; c < total; c += gridDim.x * blockDim.x) {
+        double a = 0.0;
+        for (int s = 0; s < S; ++s) a += part[c * S + s].x;
+        scores[(size_t)cand[c].x * d_ff + cand[c].y] = (float)(sqrt(a) * sqrt(part[c * S].y));
     }
 }
 
@@ -454,12 +483,14 @@ int clada_refine_scores(const clada_layer *layer, const void *X, const int64_t *
     rc = build_table(seq_offsets, B, &tab, &n_mtiles);
     if (rc != CLADA_OK) return rc;
     if (!ws || (reinterpret_cast<uintptr_t>(ws) & 255u)) return CLADA_ERR_WORKSPACE;
-    // candidate counter + list live behind the partials region of clada_prefix_scores
+    // candidate counter, split partial sums and candidate list live behind the partials region of clada_prefix_scores
     const size_t off = kWsCtrlBytes + partials_bytes(n_mtiles, layer->d_ff);
-    const size_t need = off + 256 + (size_t)B * layer->d_ff * sizeof(int2);
+    const size_t part_bytes = kRefMaxUnits * sizeof(double2);
+    const size_t need = off + 256 + part_bytes + (size_t)B * layer->d_ff * sizeof(int2);
     if (ws_bytes < need) return CLADA_ERR_WORKSPACE;
     int *n_cand = reinterpret_cast<int *>(static_cast<char *>(ws) + off);
-    int2 *cand = reinterpret_cast<int2 *>(static_cast<char *>(ws) + off + 256);
+    double2 *part = reinterpret_cast<double2 *>(static_cast<char *>(ws) + off + 256);
+    int2 *cand = reinterpret_cast<int2 *>(static_cast<char *>(ws) + off + 256 + part_bytes);
     GuardMults gm;
     gm.n = n_guard;
     for (int g = 0; g < 8; ++g) gm.m[g] = g < n_guard ? guard_mults[g] : 0.f;
@@ -489,17 +520,19 @@ int clada_refine_scores(const clada_layer *layer, const void *X, const int64_t *
         guard_refine_kernel<float><<<grid, kRefThreads, rows_smem, st>>>(
             static_cast<const float *>(X), static_cast<const float *>(layer->w_gate),
             static_cast<const float *>(layer->w_up), static_cast<const float *>(layer->w_down_t),
-            layer->d_model, layer->d_ff, tab, n_cand, cand, scores, layer->activation);
+            layer->d_model, layer->d_ff, tab, n_cand, cand, scores, layer->activation, part);
     else if (layer->dtype == CLADA_BF16)
         guard_refine_kernel<__nv_bfloat16><<<grid, kRefThreads, rows_smem, st>>>(
             static_cast<const __nv_bfloat16 *>(X), static_cast<const __nv_bfloat16 *>(layer->w_gate),
             static_cast<const __nv_bfloat16 *>(layer->w_up), static_cast<const __nv_bfloat16 *>(layer->w_down_t),
-            layer->d_model, layer->d_ff, tab, n_cand, cand, scores, layer->activation);
+            layer->d_model, layer->d_ff, tab, n_cand, cand, scores, layer->activation, part);
     else
         guard_refine_kernel<__half><<<grid, kRefThreads, rows_smem, st>>>(
             static_cast<const __half *>(X), static_cast<const __half *>(layer->w_gate),
             static_cast<const __half *>(layer->w_up), static_cast<const __half *>(layer->w_down_t),
-            layer->d_model, layer->d_ff, tab, n_cand, cand, scores, layer->activation);
+            layer->d_model, layer->d_ff, tab, n_cand, cand, scores, layer->activation, part);
+    CLADA_CUDA_TRY(cudaGetLastError());
+    guard_finish_kernel<<<2, 256, 0, st>>>(n_cand, cand, grid, layer->d_ff, part, scores);
     CLADA_CUDA_TRY(cudaGetLastError());
     return CLADA_OK;
 }

@@ -111,7 +111,8 @@ size_t clada_workspace_bytes(const clada_layer *layer, int32_t B, int64_t T_tota
     size_t tiles = (size_t)(T_total / 64) + (size_t)B + 1;
     size_t prefix = (tiles * (size_t)layer->d_ff * sizeof(float) + 255) & ~(size_t)255;
     // guard band: candidate list (int32 pairs) per (sequence, neuron), worst case all of them
-    size_t refine = (size_t)B * (size_t)layer->d_ff * 2 * sizeof(int32_t) + 256;
+    // plus its counter (256 bytes) and up to 512 split partial sums (two doubles each)
+    size_t refine = (size_t)B * (size_t)layer->d_ff * 2 * sizeof(int32_t) + 256 + 512 * 16;
     size_t scratch = decode > prefix + refine ? decode : prefix + refine;
     return kWsCtrlBytes + ((scratch + 255) & ~(size_t)255);
 }
