@@ -232,11 +232,12 @@ class Job:
     def io_tensors(self):
         return [self.X, self.xs, self.logits, self.tokens], self.y
 
-    def ffn_only_loop(self):
-        """The FFN launches of one sparsity level back to back (for the kernel's own duration)."""
+    def ffn_only_loop(self, r: int = 0):
+        """The FFN launches of one sparsity level at its baseline threshold back to back (for the kernel's
+        own duration)."""
         for t in range(self.N):
             self.clada.clada_sparse_ffn_decode(self.layers[t % N_COPIES], self.xs[t:t + 1], self.scores,
-                                               self.tau_base[0], 1, self.y[0, t:t + 1], self.ws)
+                                               self.tau_base[r], 1, self.y[0, t:t + 1], self.ws)
 
 
 class StackJob:
@@ -405,6 +406,19 @@ def run_ours(args):
             ffn_run = ffn_graph.replay
         ffn_run()
         ffn_ms = _timed(ffn_run, 5, lambda: None) / (5 * job.ffn_launches_per_loop)
+        # the same for the other sparsity levels of the workload (single-layer job only)
+        other_ffn_ms = []
+        if isinstance(job, Job):
+            for r in range(1, len(w.sparsities)):
+                fr = (lambda rr: (lambda: job.ffn_only_loop(rr)))(r)
+                fr()
+                if args.graph:
+                    og = torch.cuda.CUDAGraph()
+                    with torch.cuda.graph(og, stream=stream):
+                        fr()
+                    fr = og.replay
+                fr()
+                other_ffn_ms.append(_timed(fr, 5, lambda: None) / (5 * job.ffn_launches_per_loop))
         # the prefix statistics alone (tensor-core contraction), for its own roofline line
         pf = job.prefix_once
         pf()
@@ -496,6 +510,15 @@ def run_ours(args):
                             "flop": prefix_flop},
         "clocks": clocks, "device_status_word": status,
     }
+    if other_ffn_ms:
+        per = [{"sparsity": w.sparsities[0], "kept_neurons": kept_base, "us_per_launch": ffn_ms * 1e3,
+                "achieved": achieved, "frac": achieved / peak}]
+        for r, t_ms in enumerate(other_ffn_ms, start=1):
+            kr = w.d_ff - w.k_cut(w.sparsities[r])
+            br = kr * rows * w.d_model * eb + w.d_ff * 4 + w.d_model * eb + w.d_model * 4
+            per.append({"sparsity": w.sparsities[r], "kept_neurons": kr, "us_per_launch": t_ms * 1e3,
+                        "achieved": br / (t_ms * 1e-3) / 1e9, "frac": br / (t_ms * 1e-3) / 1e9 / peak})
+        line["roofline"]["by_sparsity"] = per
     if nested_value is not None:
         # list entries instead of the score vector: 4 bytes per kept neuron
         nb = kept_base * rows * w.d_model * eb + kept_base * 4 + w.d_model * eb + w.d_model * 4
