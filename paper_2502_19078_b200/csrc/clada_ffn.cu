@@ -397,7 +397,7 @@ sparse_ffn_kernel(const FfnParams p, const int n_stages) {
     if (timed_out && p.status) atomicOr(p.status, CLADA_STATUS_TIMEOUT);
 
     // ---- epilogue: grid barrier, deterministic column reduction ---------------------------------
-    if (!grid_barrier(p.ctrl, (unsigned)n_ctas)) {
+    if (!grid_barrier(p.ctrl, (unsigned)n_ctas, kConsumers)) {
         if (tid == 0 && p.status) atomicOr(p.status, CLADA_STATUS_TIMEOUT);
         return;
     }

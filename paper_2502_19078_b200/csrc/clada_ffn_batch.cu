@@ -359,7 +359,7 @@ sparse_ffn_batch_kernel(const FfnBatchParams p, const int n_stages) {
     if (timed_out && p.status) atomicOr(p.status, CLADA_STATUS_TIMEOUT);
 
     // ---- epilogue: grid barrier, deterministic column reduction per sequence ----------------------
-    if (!grid_barrier(p.ctrl, (unsigned)n_ctas)) {
+    if (!grid_barrier(p.ctrl, (unsigned)n_ctas, kConsumers)) {
         if (tid == 0 && p.status) atomicOr(p.status, CLADA_STATUS_TIMEOUT);
         return;
     }

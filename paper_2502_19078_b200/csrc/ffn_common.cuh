@@ -9,8 +9,10 @@ namespace clada {
 constexpr unsigned kBarrierSpinLimit = 1u << 22;  // polls of an L2 word: gives up after ~1 s at most
 
 // Bounded grid-wide barrier on two self-resetting counters in the workspace control block.
-// Returns false if the wait expired.
-static __device__ bool grid_barrier(WsCtrl *ctrl, unsigned n_ctas) {
+// Returns false if the wait expired.  Thread 0 arrives and polls; the departure count (whose last
+// increment resets both counters for the next launch) is another round trip to L2 that nothing waits
+// for, so a thread of the otherwise idle producer warp takes it after the CTA has been released.
+static __device__ bool grid_barrier(WsCtrl *ctrl, unsigned n_ctas, int depart_tid) {
     __shared__ int s_ok;
     __syncthreads();
     if (threadIdx.x == 0) {
@@ -27,17 +29,18 @@ static __device__ bool grid_barrier(WsCtrl *ctrl, unsigned n_ctas) {
             }
         }
         s_ok = ok;
-        if (ok) {
-            const unsigned left = atomicAdd(&ctrl->depart, 1u);
-            if (left == n_ctas - 1) {  // last one out: everyone has seen arrive == n_ctas
-                ctrl->arrive = 0;
-                ctrl->depart = 0;
-                __threadfence();
-            }
-        }
     }
     __syncthreads();
-    return s_ok != 0;
+    const bool ok = s_ok != 0;
+    if ((int)threadIdx.x == depart_tid && ok) {
+        const unsigned left = atomicAdd(&ctrl->depart, 1u);
+        if (left == n_ctas - 1) {  // last one out: everyone has seen arrive == n_ctas
+            ctrl->arrive = 0;
+            ctrl->depart = 0;
+            __threadfence();
+        }
+    }
+    return ok;
 }
 
 // ---- mbarrier / bulk-copy primitives (bounded waits) -------------------------------------------
