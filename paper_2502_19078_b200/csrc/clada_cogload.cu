@@ -1,9 +1,10 @@
 // Per-token cognitive load (Eqs. surprisal, entropy) and the token-aware threshold
 // (Eq. final_threshold).
 //
-// One CTA per vocabulary row.  Each thread streams 16-byte vectors of logits and keeps a running
-// (max m, Z = sum e^{l-m}, W = sum e^{l-m}(l-m)); triples are merged by warp shuffles, then across
-// warps through shared memory, always in the same order.  With logZ = log Z:
+// A cluster of CTAs per vocabulary row.  Each thread streams 16-byte vectors of logits and keeps a running
+// (max m, Z = sum e^{l-m}, W = sum e^{l-m}(l-m)).  At each level (CTA, then cluster) the maximum is reduced
+// first, every statistic is moved to it once, and Z and W are summed, always in the same order.  With
+// logZ = log Z:
 //   surprisal = m + logZ - l[token],   entropy = logZ - W / Z.
 #include <math.h>
 
@@ -32,14 +33,6 @@ __device__ __forceinline__ void stat_rebase(SoftStat &a, float m_new) {
     a.w = (a.w + dm * a.z) * sc;
     a.z = a.z * sc;
     a.m = m_new;
-}
-
-__device__ __forceinline__ SoftStat stat_merge(SoftStat a, SoftStat b) {
-    const float m = fmaxf(a.m, b.m);
-    if (m == -INFINITY) return a;
-    stat_rebase(a, m);
-    stat_rebase(b, m);
-    return SoftStat{m, a.z + b.z, a.w + b.w};
 }
 
 template <int N>
@@ -150,34 +143,46 @@ cogload_kernel(const T *__restrict__ logits, int64_t V, int64_t row_stride,
         stat_add(st, l, bad);
     }
 
-    // warp, CTA, then cluster merge, each in a fixed order
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-        SoftStat other;
-        other.m = __shfl_xor_sync(0xffffffffu, st.m, o);
-        other.z = __shfl_xor_sync(0xffffffffu, st.z, o);
-        other.w = __shfl_xor_sync(0xffffffffu, st.w, o);
-        st = ((tid & o) == 0) ? stat_merge(st, other) : stat_merge(other, st);
-    }
-    __shared__ SoftStat s_stat[kCogThreads / kWarp];
+    // CTA reduction, in a fixed order.  Merging statistics pairwise costs two exponentials per merge on a
+    // serial chain (13 levels from thread to row); instead the maximum is reduced first (compares only),
+    // every thread moves its statistic to it once, and Z and W are then plain sums.
+    __shared__ float s_max[kCogThreads / kWarp];
+    __shared__ float2 s_zw[kCogThreads / kWarp];
     __shared__ SoftStat s_all[kCogMaxCluster];  // on rank 0: every slice's statistic, written by its owner
     __shared__ int s_bad;
     __shared__ float s_out[2];
+    float wm = st.m;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) wm = fmaxf(wm, __shfl_xor_sync(0xffffffffu, wm, o));
     if (tid == 0) s_bad = 0;
+    if ((tid & 31) == 0) s_max[tid >> 5] = wm;
     __syncthreads();
     if (bad) atomicOr(&s_bad, 1);
-    if ((tid & 31) == 0) s_stat[tid >> 5] = st;
-    __syncthreads();
-    if (tid < kWarp) {  // warp 0 merges the 16 warp statistics by butterfly (same bits on every lane)
-        SoftStat tot = tid < kCogThreads / kWarp ? s_stat[tid] : stat_empty();
+    float cm = s_max[0];
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-            SoftStat other;
-            other.m = __shfl_xor_sync(0xffffffffu, tot.m, o);
-            other.z = __shfl_xor_sync(0xffffffffu, tot.z, o);
-            other.w = __shfl_xor_sync(0xffffffffu, tot.w, o);
-            tot = ((tid & o) == 0) ? stat_merge(tot, other) : stat_merge(other, tot);
+    for (int w = 1; w < kCogThreads / kWarp; ++w) cm = fmaxf(cm, s_max[w]);
+    float z = 0.f, wsum = 0.f;
+    if (st.z > 0.f) {  // (a thread without finite logits adds nothing; cm is finite here)
+        const float dm = st.m - cm;  // <= 0
+        const float sc = expf(dm);
+        z = st.z * sc;
+        wsum = (st.w + dm * st.z) * sc;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        z += __shfl_xor_sync(0xffffffffu, z, o);
+        wsum += __shfl_xor_sync(0xffffffffu, wsum, o);
+    }
+    if ((tid & 31) == 0) s_zw[tid >> 5] = make_float2(z, wsum);
+    __syncthreads();
+    if (tid < kWarp) {  // warp 0 adds the 16 warp sums by butterfly (same bits on every lane)
+        float2 v = tid < kCogThreads / kWarp ? s_zw[tid] : make_float2(0.f, 0.f);
+#pragma unroll
+        for (int o = 8; o > 0; o >>= 1) {
+            v.x += __shfl_xor_sync(0xffffffffu, v.x, o);
+            v.y += __shfl_xor_sync(0xffffffffu, v.y, o);
         }
+        SoftStat tot = SoftStat{cm, v.x, v.y};
         if (s_bad) tot.z = NAN;  // carries the non-finite flag to rank 0
         // every CTA started (first phase) before anyone writes into rank 0's shared memory
         asm volatile("barrier.cluster.wait.aligned;" ::: "memory");
@@ -188,17 +193,25 @@ cogload_kernel(const T *__restrict__ logits, int64_t V, int64_t row_stride,
     cluster.sync();  // the statistics have landed; the other CTAs are done and may leave
     if (slice == 0) {
         if (tid < kWarp) {
-            // lane r takes slice r's statistic, then a butterfly merges them
-            SoftStat tot = stat_empty();
-            if (tid < n_slices) tot = s_all[tid];
+            // lane r takes slice r's statistic; maximum first, one move per lane, then sums
+            SoftStat mine = stat_empty();
+            if (tid < n_slices) mine = s_all[tid];
+            float rm = mine.m;
+#pragma unroll
+            for (int o = kCogMaxCluster / 2; o > 0; o >>= 1) rm = fmaxf(rm, __shfl_xor_sync(0xffffffffu, rm, o));
+            float rz = mine.z, rw = mine.w;  // a NaN Z (non-finite flag) stays NaN through the sums
+            if (mine.z > 0.f) {
+                const float dm = mine.m - rm;
+                const float sc = expf(dm);
+                rz = mine.z * sc;
+                rw = (mine.w + dm * mine.z) * sc;
+            }
 #pragma unroll
             for (int o = kCogMaxCluster / 2; o > 0; o >>= 1) {
-                SoftStat other;
-                other.m = __shfl_xor_sync(0xffffffffu, tot.m, o);
-                other.z = __shfl_xor_sync(0xffffffffu, tot.z, o);
-                other.w = __shfl_xor_sync(0xffffffffu, tot.w, o);
-                tot = ((tid & o) == 0) ? stat_merge(tot, other) : stat_merge(other, tot);
+                rz += __shfl_xor_sync(0xffffffffu, rz, o);
+                rw += __shfl_xor_sync(0xffffffffu, rw, o);
             }
+            const SoftStat tot = SoftStat{rm, rz, rw};
             if (tid == 0) {
                 int flags = 0;
                 float s, h;
