@@ -42,6 +42,12 @@ struct FfnParams {
     const int32_t *level;   // one int in 0..3
 };
 
+// floor(n * c / n_ctas): where CTA c's even share of n items starts.  n <= 69632 and c <= n_ctas (a few
+// hundred), so the product fits 32 bits and the division is the cheap one.
+__device__ __forceinline__ int split_at(int n, int c, int n_ctas) {
+    return (int)(((unsigned)n * (unsigned)c) / (unsigned)n_ctas);
+}
+
 constexpr int G = 4;                          // neurons per CTA-wide reduction
 constexpr int kMaxBatches = 4;                // prologue batches: d_ff <= 4 * 32 * kFfnThreads
 
@@ -117,8 +123,8 @@ sparse_ffn_kernel(const FfnParams p, const int n_stages) {
         bool bad = lv < 0 || lv > 3 || n < 0 || n > F;
         n = min(max(n, 0), F);
         n_act_o = n;
-        r0_o = (int)(((int64_t)n * cta) / n_ctas);
-        r1_o = (int)(((int64_t)n * (cta + 1)) / n_ctas);
+        r0_o = split_at(n, cta, n_ctas);
+        r1_o = split_at(n, cta + 1, n_ctas);
         for (int i = tid; i < r1_o - r0_o; i += kFfnThreads) {
             const int j = p.order[r0_o + i];
             bad |= j < 0 || j >= F;
@@ -203,10 +209,10 @@ sparse_ffn_kernel(const FfnParams p, const int n_stages) {
         first_rank[bt] = n_act + wbase + incl - cnt;
         n_act += btot;
     }
-    const int r0 = (int)(((int64_t)n_act * cta) / n_ctas);
-    const int r1 = (int)(((int64_t)n_act * (cta + 1)) / n_ctas);
-    const int m0 = (int)(((int64_t)F * cta) / n_ctas);  // slice of the mask this CTA writes
-    const int m1 = (int)(((int64_t)F * (cta + 1)) / n_ctas);
+    const int r0 = split_at(n_act, cta, n_ctas);
+    const int r1 = split_at(n_act, cta + 1, n_ctas);
+    const int m0 = split_at(F, cta, n_ctas);  // slice of the mask this CTA writes
+    const int m1 = split_at(F, cta + 1, n_ctas);
     // Only two or three chunks hold this CTA's share: the warp that owns such a chunk writes it out
     // with one lane per neuron.
 #pragma unroll
@@ -243,7 +249,7 @@ sparse_ffn_kernel(const FfnParams p, const int n_stages) {
         // Nothing is kept (every CTA sees the same count): y = 0, written slice by slice, and there are
         // no partial sums to combine, so the grid barrier is skipped as well.
         const int ng = d / 4;  // output in groups of 4 columns
-        const int q0 = (int)(((int64_t)ng * cta) / n_ctas), q1 = (int)(((int64_t)ng * (cta + 1)) / n_ctas);
+        const int q0 = split_at(ng, cta, n_ctas), q1 = split_at(ng, cta + 1, n_ctas);
         for (int q = q0 + tid; q < q1; q += kFfnThreads) {
             if (p.y_dtype == CLADA_F32)
                 reinterpret_cast<float4 *>(p.y)[q] = make_float4(0.f, 0.f, 0.f, 0.f);
