@@ -218,3 +218,45 @@ def test_nested_decode_bad_inputs_are_clamped_and_reported(clada):
                                          torch.tensor([1], dtype=torch.int32, device="cuda"), y, ws, None, status)
     torch.cuda.synchronize()
     assert int(status.item()) == 0 and torch.all(y == 0)
+
+
+def test_many_launches_share_one_workspace(clada):
+    """Three hundred launches of every decode flavour back to back on ONE workspace (score scan, nested list,
+    nothing kept, a tile of four sequences): the grid barrier's counters must be back at zero after each, the
+    status word stays clear, and every flavour returns the same bits every time."""
+    w = wl.scaled(wl.WORKLOADS["c2_llama2_7b_layer"], d_model=1024, d_ff=2400)
+    weights = wl.layer_weights(w, 0)
+    layer = gpu_layer(weights, clada)
+    B = 4
+    g = torch.Generator().manual_seed(5)
+    scores = (torch.rand(B, w.d_ff, generator=g) + 0.5).cuda()
+    tau = torch.empty(B, dtype=torch.float32, device="cuda")
+    clada.clada_tau_from_sparsity(scores, 0.4, tau)
+    tau_none = torch.full((B,), 10.0, device="cuda")
+    order = torch.empty(B, w.d_ff, dtype=torch.int32, device="cuda")
+    counts = torch.empty(B, 4, dtype=torch.int32, device="cuda")
+    clada.clada_nested_build(scores, tau, 0.1, 0.03, order, counts)
+    level = torch.tensor([0, 1, 2, 3], dtype=torch.int32, device="cuda")
+    x = torch.stack([wl.hidden_states(w, 0, "decode", b, 1, "cpu", wl.channel_scale(w))[0] for b in range(B)]).cuda()
+    ws = clada.new_workspace(layer, B, 0)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    outs = {k: torch.empty(B, w.d_model, dtype=torch.float32, device="cuda") for k in ("scan1", "nested", "none", "tile")}
+    first = None
+    for it in range(75):
+        clada.clada_sparse_ffn_decode(layer, x[:1], scores[:1], tau[:1], 1, outs["scan1"][:1], ws, status=status)
+        clada.clada_sparse_ffn_decode_nested(layer, x, order, counts, level, outs["nested"], ws, None, status)
+        clada.clada_sparse_ffn_decode(layer, x[:1], scores[:1], tau_none[:1], 1, outs["none"][:1], ws, status=status)
+        clada.clada_sparse_ffn_decode(layer, x, scores, tau, 1, outs["tile"], ws, status=status)
+        if it == 0:
+            torch.cuda.synchronize()
+            first = {k: v.clone() for k, v in outs.items()}
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    assert torch.all(outs["none"][:1] == 0)
+    for k in outs:
+        rows = slice(0, 1) if k in ("scan1", "none") else slice(0, B)
+        assert torch.equal(outs[k][rows], first[k][rows]), k
+    # the tile's first sequence and the single-sequence launch keep the same neurons
+    assert torch.allclose(outs["tile"][0], outs["scan1"][0], rtol=0, atol=1e-5 * float(outs["scan1"][0].abs().max()))
+    # the control words are back at zero
+    assert int(ws[:16].view(torch.int32).abs().sum().item()) == 0
