@@ -419,6 +419,14 @@ def run_ours(args):
                     fr = og.replay
                 fr()
                 other_ffn_ms.append(_timed(fr, 5, lambda: None) / (5 * job.ffn_launches_per_loop))
+        # read-only streaming bandwidth of this machine (the peak file's figure is a read + write copy)
+        probe = torch.empty(1 << 30, dtype=torch.uint8, device=dev)
+        probe.zero_()
+        sink = torch.zeros(1, dtype=torch.int32, device=dev)
+        rd = lambda: clada.clada_stream_read_probe(probe, sink)
+        rd()
+        read_gbs = probe.numel() / (_timed(rd, 10, lambda: None) / 10 * 1e-3) / 1e9
+        del probe
         # the prefix statistics alone (tensor-core contraction), for its own roofline line
         pf = job.prefix_once
         pf()
@@ -502,6 +510,7 @@ def run_ours(args):
         "roofline": {"bound": "hbm", "kernel": "sparse_ffn_kernel", "achieved": achieved, "peak": peak,
                      "unit": "GB/s", "frac": achieved / peak, "peak_kind": peak_kind,
                      "traffic": FFN_NCU_TRAFFIC_BYTES if w.name == WORKLOAD else None,
+                     "read_only_stream_gbs": read_gbs, "frac_of_read_only_stream": achieved / read_gbs,
                      "bytes_per_launch": ffn_bytes, "us_per_launch": ffn_ms * 1e3,
                      "kept_neurons": kept_base},
         "prefix_roofline": {"bound": "tensor", "kernel": "prefix_tc_kernel (+finalize)", "ms": prefix_ms,

@@ -100,6 +100,13 @@ size_t clada_workspace_bytes(const clada_layer *layer, int32_t B, int64_t T_tota
  * a CLADA_STATUS_TIMEOUT.  ws must be 256-byte aligned. */
 int clada_workspace_init(void *ws, size_t ws_bytes, void *stream);
 
+/* Measuring aid (the paper has no counterpart): reads `bytes` of device memory
+ * at buf once (16-byte aligned, 16-byte loads that do not allocate in L1, as the
+ * decode kernel's) and xors everything into *sink (device) so the reads are
+ * kept.  Timed by the caller, it gives the read-only streaming bandwidth of the
+ * device, the ceiling for the sparse FFN's weight rows. */
+int clada_stream_read_probe(const void *buf, size_t bytes, uint32_t *sink, void *stream);
+
 /* out[j] = ||W_out,j||_2 = the l2 norm of row j of w_down_t, fp32.  Once per
  * layer; the second factor of Eq. neuron_activation. */
 int clada_down_norms(const clada_layer *layer, float *out /*[d_ff]*/, void *stream);

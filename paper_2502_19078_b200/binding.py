@@ -71,6 +71,7 @@ def load() -> ctypes.CDLL:
     L.clada_sparse_ffn_decode.argtypes = [lp, vp, i32, vp, vp, i64, vp, i32, vp, vp, vp, vp, sz, vp, vp]
     L.clada_sparse_ffn_decode_static.argtypes = [lp, vp, i32, vp, vp, i64, vp, i32, vp, vp, vp, vp, vp]
     L.clada_sparse_ffn_decode_layers.argtypes = [vp, i32, vp, i32, vp, vp, vp, i32, vp, sz, vp, vp]
+    L.clada_stream_read_probe.argtypes = [vp, sz, vp, vp]
     L.clada_prefix_accumulate.argtypes = [lp, vp, vp, i32, vp, vp, vp, sz, vp, vp]
     L.clada_prefix_finish.argtypes = [lp, vp, i32, vp, vp]
     L.clada_prefill_down.argtypes = [lp, vp, vp, i64, vp, i32, vp, vp]
@@ -427,3 +428,10 @@ def clada_prefill_down(layer: Layer, w_down, Z, Y, status=None, stream=None) -> 
     _check(load().clada_prefill_down(layer.ref, _ptr(w_down, layer.dtype, "w_down"), _ptr(Z, layer.dtype, "Z"),
                                      Z.shape[0], _ptr(Y, name="Y"), _dtype_code(Y.dtype),
                                      _ptr(status, torch.int32, "status"), _stream(stream)), "clada_prefill_down")
+
+
+def clada_stream_read_probe(buf: torch.Tensor, sink: torch.Tensor, stream=None) -> None:
+    """Read `buf` once with streaming 16-byte loads (a measuring aid); `sink` is one int32 on the device."""
+    _check(load().clada_stream_read_probe(_ptr(buf, name="buf"), buf.numel() * buf.element_size(),
+                                          _ptr(sink, torch.int32, "sink"), _stream(stream)),
+           "clada_stream_read_probe")

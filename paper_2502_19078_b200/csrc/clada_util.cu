@@ -80,6 +80,32 @@ __global__ void down_norms_kernel(const T *__restrict__ w, int d_model, int d_ff
 
 using namespace clada;
 
+namespace clada {
+// Measuring aid: read a buffer once with the decode kernel's kind of load (16 bytes per thread, no L1
+// allocation), eight loads in flight per thread, and fold it into one word per CTA so that nothing is
+// optimised away.  Gives the read-only streaming bandwidth the sparse FFN's rows could at best arrive at.
+__global__ void __launch_bounds__(512) stream_read_kernel(const uint4 *__restrict__ buf, size_t n_vec,
+                                                          uint32_t *__restrict__ sink) {
+    const size_t stride = (size_t)gridDim.x * blockDim.x;
+    uint32_t acc = 0;
+    size_t v = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    for (; v + 7 * stride < n_vec; v += 8 * stride) {
+        uint4 q[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) q[u] = ldg_stream(buf + v + u * stride);
+#pragma unroll
+        for (int u = 0; u < 8; ++u) acc ^= q[u].x ^ q[u].y ^ q[u].z ^ q[u].w;
+    }
+    for (; v < n_vec; v += stride) {
+        const uint4 q = ldg_stream(buf + v);
+        acc ^= q.x ^ q.y ^ q.z ^ q.w;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) acc ^= __shfl_xor_sync(0xffffffffu, acc, o);
+    if ((threadIdx.x & 31) == 0) atomicXor(sink, acc);
+}
+}  // namespace clada
+
 extern "C" {
 
 int clada_version(void) { return 100; }
@@ -140,6 +166,18 @@ int clada_down_norms(const clada_layer *layer, float *out, void *stream) {
     else
         down_norms_kernel<__half><<<blocks, threads, 0, st>>>(
             static_cast<const __half *>(layer->w_down_t), layer->d_model, layer->d_ff, out);
+    CLADA_CUDA_TRY(cudaGetLastError());
+    return CLADA_OK;
+}
+
+int clada_stream_read_probe(const void *buf, size_t bytes, uint32_t *sink, void *stream) {
+    if (!buf || !sink) return CLADA_ERR_NULL;
+    if (bytes < 16 || !aligned16(buf)) return CLADA_ERR_ALIGN;
+    DeviceInfo di;
+    int rc = device_info(&di);
+    if (rc != CLADA_OK) return rc;
+    stream_read_kernel<<<di.num_sms * 4, 512, 0, static_cast<cudaStream_t>(stream)>>>(
+        static_cast<const uint4 *>(buf), bytes / 16, sink);
     CLADA_CUDA_TRY(cudaGetLastError());
     return CLADA_OK;
 }
