@@ -331,7 +331,7 @@ int clada_prefill_down(const clada_layer *layer, const void *w_down, const void 
  *              (1+lambda)+gamma} in fp32 -- bit for bit the thresholds that
  *              clada_adjust_threshold produces, so order[b][0 .. counts[b][k])
  *              is exactly the kept set clada_select would give at level k.
- *   d_ff <= 16384 (the sort runs in one CTA's shared memory); otherwise
+ *   d_ff <= 32768 (every CTA holds the score vector in shared memory); otherwise
  *   CLADA_ERR_UNSUPPORTED.  Nothing is allocated.
  *
  * clada_cogload_level, per decode step: clada_cogload plus

@@ -34,7 +34,7 @@ def _thresholds(tau_base, lam, gam):
     return [np.float32(np.float32(tau_base) * m) for m in mults]
 
 
-@pytest.mark.parametrize("F", [1, 2, 33, 1376, 4097, 11008, 16384])
+@pytest.mark.parametrize("F", [1, 2, 33, 1376, 4097, 11008, 16384, 28672])
 @pytest.mark.parametrize("lam,gam", [(LAM, GAM), (-0.3, -0.1)])
 def test_nested_build_bit_exact(clada, oracle, F, lam, gam):
     B = 3

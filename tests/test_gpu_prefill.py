@@ -206,9 +206,9 @@ def test_new_entry_points_refuse_what_they_cannot_do(clada):
     with pytest.raises(clada.CladaError, match="shape"):
         clada.clada_prefill_down(lb, torch.zeros(64, 100, dtype=torch.bfloat16, device="cuda"), Zb,
                                  torch.empty(16, 64, device="cuda"))
-    big = torch.ones(1, 16385, device="cuda")                             # the list sort holds 16384 keys
+    big = torch.ones(1, 32769, device="cuda")                             # the list build holds 32768 scores per CTA
     with pytest.raises(clada.CladaError, match="support"):
         clada.clada_nested_build(big, torch.ones(1, device="cuda"), 0.8, 0.12,
-                                 torch.empty(1, 16385, dtype=torch.int32, device="cuda"),
+                                 torch.empty(1, 32769, dtype=torch.int32, device="cuda"),
                                  torch.empty(1, 4, dtype=torch.int32, device="cuda"))
     torch.cuda.synchronize()
