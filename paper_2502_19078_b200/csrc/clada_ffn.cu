@@ -71,7 +71,8 @@ sparse_ffn_kernel(const FfnParams p, const int n_stages) {
     const uint32_t ring = smem_u32(smem_raw);
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem_raw + (size_t)n_stages * stage_bytes);
     const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + kMaxStages);
-    unsigned *s_bal = reinterpret_cast<unsigned *>(bars + 2 * kMaxStages);  // keep-bits word per chunk
+    const uint32_t sbar = smem_u32(bars + 2 * kMaxStages);  // completion of the score vector's bulk copy
+    unsigned *s_bal = reinterpret_cast<unsigned *>(bars + 2 * kMaxStages + 1);  // keep-bits word per chunk
     int *s_list = reinterpret_cast<int *>(s_bal + chunks);
     __shared__ int s_wtot[kFfnWarps];
     __shared__ float s_tau;
@@ -83,6 +84,7 @@ sparse_ffn_kernel(const FfnParams p, const int n_stages) {
             mbar_init(full0 + 8 * s, 1);            // the producer's expect_tx arrival
             mbar_init(empty0 + 8 * s, kConsWarps);  // one arrival per consumer warp
         }
+        mbar_init(sbar, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     pdl_wait();  // everything below may read what the previous kernel wrote
@@ -134,6 +136,14 @@ sparse_ffn_kernel(const FfnParams p, const int n_stages) {
     } else {
     const bool vec_ok = (reinterpret_cast<uintptr_t>(p.scores) & 15u) == 0;
     const int n_batches = (chunks + kFfnThreads - 1) / kFfnThreads;
+    // The score vector comes in as ONE bulk copy into the (still idle) ring when it is aligned and fits: 148 CTAs
+    // each pulling the same 44 KB through L2 with per-thread loads took ~2.4 us, the copy engine's stream about
+    // half that.  Otherwise the threads load their chunks themselves.
+    const bool bulk_scores = vec_ok && (F & 3) == 0 && (size_t)F * 4 <= (size_t)n_stages * stage_bytes;
+    if (bulk_scores && tid == kConsumers) {
+        mbar_expect_tx(sbar, (uint32_t)F * 4u);
+        bulk_load_row_hint(ring, p.scores, (uint32_t)F * 4u, sbar, keep_policy);
+    }
     {
         int slot = tid + (cta * 37) % kFfnThreads;
         if (slot >= kFfnThreads) slot -= kFfnThreads;
@@ -145,7 +155,7 @@ sparse_ffn_kernel(const FfnParams p, const int n_stages) {
             const bool has = q < chunks;
             const int j0 = q * kWarp;
             float4 v[8];
-            if (has) {
+            if (has && !bulk_scores) {
                 if (vec_ok && j0 + kWarp <= F) {
 #pragma unroll
                     for (int u = 0; u < 8; ++u)
@@ -164,6 +174,19 @@ sparse_ffn_kernel(const FfnParams p, const int n_stages) {
             if (bt == 0) {  // the threshold arrives while the score loads are in flight
                 __syncthreads();
                 tau = s_tau;
+                if (bulk_scores && !mbar_wait(sbar, 0) && tid == 0 && p.status) atomicOr(p.status, CLADA_STATUS_TIMEOUT);
+            }
+            if (has && bulk_scores) {
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    if (j0 + 4 * u < F) {  // F is a multiple of 4 here: a vector is all in or all out
+                        const uint4 r = lds128(ring + (uint32_t)(j0 + 4 * u) * 4u);
+                        v[u] = make_float4(__uint_as_float(r.x), __uint_as_float(r.y), __uint_as_float(r.z),
+                                           __uint_as_float(r.w));
+                    } else {
+                        v[u] = make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
+                    }
+                }
             }
             if (has) {
                 unsigned w = 0;
@@ -447,7 +470,7 @@ static int launch_variant(const FfnParams &p, cudaStream_t st) {
     if (rc != CLADA_OK) return rc;
     auto kern = sparse_ffn_kernel<T, NV, GATED>;
     const size_t stage_bytes = (GATED ? 3 : 2) * (size_t)(p.d_model / E) * 16;
-    const size_t tail = 2 * kMaxStages * sizeof(uint64_t) + (size_t)((p.d_ff + 31) / 32) * sizeof(unsigned) +
+    const size_t tail = (2 * kMaxStages + 1) * sizeof(uint64_t) + (size_t)((p.d_ff + 31) / 32) * sizeof(unsigned) +
                         (size_t)(p.d_ff / di.num_sms + 2) * sizeof(int);
     const size_t budget = (size_t)di.max_smem_optin - 2048;  // leave room for the static arrays
     if (budget < tail + G * stage_bytes) return CLADA_ERR_UNSUPPORTED;  // a group needs G stages at once
