@@ -338,6 +338,117 @@ class StackJob:
             self.clada.clada_sparse_ffn_decode_layers(self.stack, self.xs[t], self.scores, self.tau_base, self.y[t], self.ws)
 
 
+class BatchJob:
+    """One layer of a batched workload (c4: 8 sequences, c5: 16, each with its own prompt, scores, threshold and
+    mask): prefix statistics of all prompts, then N decode steps of (cogload+adjust for the batch, sparse FFN for
+    the batch in tiles of sequences).  Informational: the metric's workload is the single-sequence layer."""
+    layers_run = 1
+    ffn_kernel = "sparse_ffn_batch_kernel (one call = all tiles of the batch)"
+    N_DECODE = 32      # decode steps per timed step (the workloads' 256-512 would only repeat these)
+    N_LOGITS = 8       # distinct logit rows per sequence, cycled
+
+    def __init__(self, clada, w, dev, rank: int):
+        self.clada, self.w, self.dev = clada, w, dev
+        B = self.B = w.batch
+        self.N = self.N_DECODE
+        lengths = wl.prefix_lengths(w)
+        self.off = wl.seq_offsets(lengths)
+        self.T = self.off[-1]
+        weights = wl.layer_weights(w, 0, dev)
+        self.layer = clada.Layer(weights["w_gate"], weights["w_up"], weights["w_down"].t().contiguous(),
+                                 activation=w.activation)
+        norms = torch.empty(w.d_ff, dtype=torch.float32, device=dev)
+        clada.clada_down_norms(self.layer, norms)
+        self.layer.set_down_norm(norms)
+        scale = wl.channel_scale(w, dev)
+        seq0 = rank * B    # a rank's sequences differ from the other ranks'
+        self.X = torch.cat([wl.hidden_states(w, 0, "prefix", seq0 + b, n, dev, scale) for b, n in enumerate(lengths)])
+        self.xs = torch.stack([wl.hidden_states(w, 0, "decode", seq0 + b, self.N, dev, scale) for b in range(B)],
+                              dim=1).contiguous()                                        # [N, B, d]
+        lg = [wl.decode_logits(w, seq0 + b, self.N_LOGITS, dev) for b in range(B)]
+        self.logits = torch.stack(lg, dim=1).contiguous()                               # [N_LOGITS, B, V]
+        self.tokens = torch.stack([wl.chosen_tokens(w, lg[b], seq0 + b) for b in range(B)], dim=1).contiguous()
+        f32 = dict(dtype=torch.float32, device=dev)
+        self.ws = clada.new_workspace(self.layer, B, self.T)
+        self.scores = torch.empty(B, w.d_ff, **f32)
+        self.mask = torch.empty(B, w.d_ff, dtype=torch.uint8, device=dev)
+        self.idx = torch.empty(B, w.d_ff, dtype=torch.int32, device=dev)
+        self.count = torch.empty(B, dtype=torch.int32, device=dev)
+        self.status = torch.zeros(1, dtype=torch.int32, device=dev)
+        self.lam = torch.full((1,), LAMBDA, **f32)
+        self.gam = torch.full((1,), GAMMA, **f32)
+        self.s = torch.empty(self.N_LOGITS, B, **f32)
+        self.h = torch.empty(self.N_LOGITS, B, **f32)
+        self.tau_final = torch.empty(B, 1, **f32)
+        self.tau_base = torch.empty(B, 1, **f32)
+        self.y = torch.empty(self.N, B, w.d_model, **f32)
+        self.guard = [1.0, 1.0 + LAMBDA, 1.0 + GAMMA, 1.0 + LAMBDA + GAMMA]
+        self.rho = w.sparsities[0]
+        clada.clada_prefix_scores(self.layer, self.X, self.off, self.scores, self.ws)
+        clada.clada_tau_from_sparsity(self.scores, self.rho, self.tau_base.view(B))
+        clada.clada_cogload(self.logits.view(-1, w.vocab), self.tokens.view(-1), self.s.view(-1), self.h.view(-1))
+        clada.clada_select(self.scores, self.tau_base.view(B), 1, self.mask, None, self.count)
+        torch.cuda.synchronize()
+        self.tau_s = wl.universal_threshold(self.s.flatten().tolist())
+        self.tau_H = wl.universal_threshold(self.h.flatten().tolist())
+        # rows one layer-step at the baseline thresholds has to read: the union of a tile's kept sets, per tile
+        bt = 4 if w.d_model * w.elem_bytes <= 8192 else 2
+        m = self.mask.bool()
+        self.union_rows = sum(int(m[b0:b0 + bt].any(dim=0).sum()) for b0 in range(0, B, bt))
+        self.tile = bt
+
+    step_note = property(lambda self: f"prefix statistics, guard band, select for {self.B} prompts; then {self.N} x "
+                                      f"(cogload+adjust for the batch, sparse FFN in tiles of {self.tile} sequences)")
+    l2_note = "inputs larger than L2: every layer-step streams the union of its tiles' kept rows (see bytes_per_launch)"
+    ffn_launches_per_loop = property(lambda self: self.N)
+    prefix_flop = property(lambda self: (2.0 if self.w.activation == 2 else 4.0) * self.T * self.w.d_model * self.w.d_ff)
+
+    @property
+    def ffn_bytes_per_launch(self):
+        w, eb = self.w, self.w.elem_bytes
+        return self.union_rows * 3 * w.d_model * eb + self.B * (w.d_ff * 4 + w.d_model * eb + w.d_model * 4)
+
+    def step(self):
+        c, B = self.clada, self.B
+        c.clada_prefix_select(self.layer, self.X, self.off, self.tau_base.view(B), self.guard, self.scores, self.mask,
+                              self.idx, self.count, self.ws, self.status)
+        for t in range(self.N):
+            r = t % self.N_LOGITS
+            c.clada_cogload_adjust(self.logits[r], self.tokens[r], self.tau_base, self.lam, self.gam, self.tau_s,
+                                   self.tau_H, self.s[r], self.h[r], self.tau_final, self.status)
+            c.clada_sparse_ffn_decode(self.layer, self.xs[t], self.scores, self.tau_final.view(B), 1, self.y[t],
+                                      self.ws, status=self.status)
+
+    @property
+    def launches_per_step(self) -> int:
+        tiles = (self.B + self.tile - 1) // self.tile
+        return 7 + self.N * (1 + tiles)
+
+    def tokens_per_step(self) -> int:
+        return self.B * self.N
+
+    def kept_per_token(self):
+        c, B = self.clada, self.B
+        tot = 0
+        for r in range(self.N_LOGITS):
+            c.clada_cogload_adjust(self.logits[r], self.tokens[r], self.tau_base, self.lam, self.gam, self.tau_s,
+                                   self.tau_H, self.s[r], self.h[r], self.tau_final)
+            c.clada_select(self.scores, self.tau_final.view(B), 1, None, None, self.count)
+            tot += int(self.count.sum().item())
+        return tot / (self.N_LOGITS * B)
+
+    def prefix_once(self):
+        self.clada.clada_prefix_scores(self.layer, self.X, self.off, self.scores, self.ws, self.status)
+
+    def io_tensors(self):
+        return [self.X, self.xs, self.logits, self.tokens], self.y
+
+    def ffn_only_loop(self):
+        for t in range(self.N):
+            self.clada.clada_sparse_ffn_decode(self.layer, self.xs[t], self.scores, self.tau_base.view(self.B), 1,
+                                               self.y[t], self.ws)
+
+
 def _timed(fn, steps, dist_barrier):
     start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     dist_barrier()
@@ -372,7 +483,7 @@ def run_ours(args):
     barrier()
     clada.load()
     w = wl.WORKLOADS[args.workload]
-    job = (StackJob if w.n_layers > 1 else Job)(clada, w, dev, rank)
+    job = (BatchJob if w.batch > 1 else StackJob if w.n_layers > 1 else Job)(clada, w, dev, rank)
 
     stream = torch.cuda.Stream()
     graph = None
@@ -493,6 +604,8 @@ def run_ours(args):
     # + scores + x in + y out
     rows = 2 if w.activation == 2 else 3
     ffn_bytes = kept_base * rows * w.d_model * eb + w.d_ff * 4 + w.d_model * eb + w.d_model * 4
+    if hasattr(job, "ffn_bytes_per_launch"):  # a batch: the union of each tile's kept rows
+        ffn_bytes = job.ffn_bytes_per_launch
     achieved = ffn_bytes / (ffn_ms * 1e-3) / 1e9
     h2d = sum(x.numel() * x.element_size() for x in host_in)
     d2h = hy.numel() * hy.element_size()
@@ -501,13 +614,13 @@ def run_ours(args):
         "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": w.name, "d_model": w.d_model, "d_ff": w.d_ff, "layers": w.n_layers, "prefix_tokens": job.T,
-                   "decode_tokens_per_sparsity": job.N, "sparsities": list(w.sparsities), "batch": 1,
+        "config": {"workload": w.name, "d_model": w.d_model, "d_ff": w.d_ff, "layers": getattr(job, "layers_run", w.n_layers), "prefix_tokens": job.T,
+                   "decode_tokens_per_sparsity": job.N, "sparsities": list(w.sparsities), "batch": w.batch,
                    "l2": job.l2_note, "cuda_graph": bool(args.graph), "avg_kept_neurons_per_token": kept,
                    "step": job.step_note},
         "e2e": {"value": e2e_value, "unit": "tokens/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
         "gpu_launches": job.launches_per_step * args.steps,
-        "roofline": {"bound": "hbm", "kernel": "sparse_ffn_kernel", "achieved": achieved, "peak": peak,
+        "roofline": {"bound": "hbm", "kernel": getattr(job, "ffn_kernel", "sparse_ffn_kernel"), "achieved": achieved, "peak": peak,
                      "unit": "GB/s", "frac": achieved / peak, "peak_kind": peak_kind,
                      "traffic": FFN_NCU_TRAFFIC_BYTES if w.name == WORKLOAD else None,
                      "read_only_stream_gbs": read_gbs, "frac_of_read_only_stream": achieved / read_gbs,
@@ -639,7 +752,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-graph", dest="graph", action="store_false")
-    ap.add_argument("--workload", default=WORKLOAD, choices=[WORKLOAD, "c3_llama2_7b_stack", "v1_opt_2p7b_layer", "v2_gemma_2b_layer"],
+    ap.add_argument("--workload", default=WORKLOAD, choices=[WORKLOAD, "c3_llama2_7b_stack", "c4_llama3_8b_b8", "c5_13b_b16", "v1_opt_2p7b_layer",
+                             "v2_gemma_2b_layer"],
                     help="the metric's workload (default); the 32-layer stack or the OPT- / Gemma-shaped "
                          "layers (other FFN forms) for information")
     args = ap.parse_args()

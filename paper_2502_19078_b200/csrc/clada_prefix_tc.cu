@@ -50,6 +50,7 @@ struct TcParams {
     uint32_t idesc_half;  // instruction descriptor of a 64-neuron item
     int n_ntiles;   // neuron tiles of 128
     int n_ttiles;   // token tiles over all prompts
+    int t_group;    // token tiles per group (their rows, t_group * 128 * d_model elements, should stay in L2)
     float *partials;  // [n_ttiles, d_ff]
     int32_t *status;
     void *z_out;    // [T_total, d_ff] in the layer's element type, or null: the hidden activations themselves
@@ -156,16 +157,30 @@ prefix_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
     const uint32_t stage_bytes = kTcTileBytes + (gated ? 2u : 1u) * kTcTileBytes;  // ring stride: a full item's stage
     const int n_stages = p.n_stages;
     // item -> (neurons per tile, first neuron, token tile)
+    // Items run in groups of t_group token tiles: within a group all neuron tiles follow one another, token tile
+    // fastest, so the CTAs of a wave share weight tiles and the group's token rows (sized to stay in L2) are
+    // re-read from L2, not from HBM, by every neuron tile.
+    auto tile_of = [&](int f, int &ntile, int &ttile) {
+        const int per_group = p.n_ntiles * p.t_group;
+        int g = f / per_group;
+        const int n_groups = (p.n_ttiles + p.t_group - 1) / p.t_group;
+        if (g > n_groups - 1) g = n_groups - 1;
+        const int gs = min(p.t_group, p.n_ttiles - g * p.t_group);  // the last group may be smaller
+        const int rem = f - g * per_group;
+        ntile = rem / gs;
+        ttile = g * p.t_group + rem % gs;
+    };
     auto decode = [&](int item, int &nt, int &j0, int &ttile) {
+        int ntile;
         if (item < p.n_full) {
             nt = 128;
-            j0 = (item / p.n_ttiles) * 128;
-            ttile = item % p.n_ttiles;
+            tile_of(item, ntile, ttile);
+            j0 = ntile * 128;
         } else {
-            const int h = item - p.n_full, f = p.n_full + (h >> 1);
+            const int h = item - p.n_full;
             nt = 64;
-            j0 = (f / p.n_ttiles) * 128 + (h & 1) * 64;
-            ttile = f % p.n_ttiles;
+            tile_of(p.n_full + (h >> 1), ntile, ttile);
+            j0 = ntile * 128 + (h & 1) * 64;
         }
     };
 
@@ -431,6 +446,10 @@ int run_prefix_partials_tc(const clada_layer *layer, const void *X, const SeqTab
     p.d_ff = layer->d_ff;
     p.n_ntiles = (layer->d_ff + 127) / 128;
     p.n_ttiles = n_ttiles;
+    {   // about 40 MB of token rows per group
+        const long long tile_bytes = (long long)kTcTileM * layer->d_model * 2;
+        p.t_group = (int)std::max<long long>(1, std::min<long long>(n_ttiles, (40ll << 20) / tile_bytes));
+    }
     // The items left over after the last full wave of CTAs run as 64-neuron halves when they then still fit one
     // wave: that wave takes half the time.  (Halves read more bytes per flop, so only the tail is split.)
     const long long items = (long long)p.n_ntiles * n_ttiles;
@@ -473,6 +492,7 @@ struct DownParams {
     int d_model, d_ff;
     long long T;
     int n_ttiles, n_dtiles;
+    int t_group;   // token tiles per group: a group's rows of Z stay in L2 while every output tile reads them
     int nd;        // output columns per tile: 256 (fewer bytes read per flop), or 128 when 256 would leave SMs idle
     int n_stages;
     void *y;
@@ -493,6 +513,17 @@ down_tc_kernel(const __grid_constant__ CUtensorMap map_z, const __grid_constant_
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int n_items = p.n_ttiles * p.n_dtiles;
     const int nd = p.nd, n_stages = p.n_stages;
+    // items in groups of t_group token tiles; within a group output tile by output tile, token tile fastest
+    auto tile_of = [&](int f, int &dtile, int &ttile) {
+        const int per_group = p.n_dtiles * p.t_group;
+        int g = f / per_group;
+        const int n_groups = (p.n_ttiles + p.t_group - 1) / p.t_group;
+        if (g > n_groups - 1) g = n_groups - 1;
+        const int gs = min(p.t_group, p.n_ttiles - g * p.t_group);
+        const int rem = f - g * per_group;
+        dtile = rem / gs;
+        ttile = g * p.t_group + rem % gs;
+    };
     const uint32_t stage_bytes = kTcTileBytes + (uint32_t)nd * kTcTileK * 2u;  // Z tile | W_out tile
     const int n_kblocks = (p.d_ff + kTcTileK - 1) / kTcTileK;
 
@@ -528,7 +559,8 @@ down_tc_kernel(const __grid_constant__ CUtensorMap map_z, const __grid_constant_
             uint32_t par = 0;
             bool ok = true;
             for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
-                const int dtile = item / p.n_ttiles, ttile = item % p.n_ttiles;
+                int dtile, ttile;
+                tile_of(item, dtile, ttile);
                 for (int kb = 0; kb < n_kblocks; ++kb, ++kc) {
                     if (!tc_mbar_wait(tc_smem_u32(&s_empty[s]), par ^ 1, abort_flag)) {
                         ok = false;
@@ -592,7 +624,8 @@ down_tc_kernel(const __grid_constant__ CUtensorMap map_z, const __grid_constant_
         bool ok = true;
         for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++it) {
             const int a = it & 1;
-            const int dtile = item / p.n_ttiles, ttile = item % p.n_ttiles;
+            int dtile, ttile;
+            tile_of(item, dtile, ttile);
             if (!tc_mbar_wait(tc_smem_u32(&s_acc_full[a]), (it >> 1) & 1, abort_flag)) {
                 ok = false;
                 break;
@@ -659,6 +692,10 @@ int run_down_tc(const clada_layer *layer, const void *w_down, const void *Z, lon
     p.d_ff = layer->d_ff;
     p.T = T;
     p.n_ttiles = (int)((T + kTcTileM - 1) / kTcTileM);
+    {   // about 40 MB of hidden-activation rows per group
+        const long long tile_bytes = (long long)kTcTileM * layer->d_ff * 2;
+        p.t_group = (int)std::max<long long>(1, std::min<long long>(p.n_ttiles, (40ll << 20) / tile_bytes));
+    }
     // 256 output columns per tile unless that leaves SMs without a tile
     p.nd = (long long)p.n_ttiles * ((layer->d_model + 255) / 256) >= di.num_sms ? 256 : 128;
     p.n_dtiles = (layer->d_model + p.nd - 1) / p.nd;
