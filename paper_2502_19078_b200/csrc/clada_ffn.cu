@@ -136,6 +136,7 @@ sparse_ffn_kernel(const FfnParams p, const int n_stages) {
     } else {
     const bool vec_ok = (reinterpret_cast<uintptr_t>(p.scores) & 15u) == 0;
     const int n_batches = (chunks + kFfnThreads - 1) / kFfnThreads;
+    unsigned bal[kMaxBatches];  // keep bits of this thread's chunk in every batch
     // The score vector comes in as ONE bulk copy into the (still idle) ring when it is aligned and fits: 148 CTAs
     // each pulling the same 44 KB through L2 with per-thread loads took ~2.4 us, the copy engine's stream about
     // half that.  Otherwise the threads load their chunks themselves.
@@ -145,30 +146,23 @@ sparse_ffn_kernel(const FfnParams p, const int n_stages) {
         bulk_load_row_hint(ring, p.scores, (uint32_t)F * 4u, sbar, keep_policy);
     }
     {
-        int slot = tid + (cta * 37) % kFfnThreads;
-        if (slot >= kFfnThreads) slot -= kFfnThreads;
+        // A warp tests 32 chunks.  For chunk c every lane holds ONE neuron's score -- consecutive addresses, so a
+        // load is one 128-byte line from global memory and conflict-free from shared memory -- and the chunk's
+        // keep-bits word is the warp's ballot.  (One 128-byte chunk per lane, the first layout, made every load
+        // touch 32 lines, or hit one bank 32 times: 1.6 us of the prologue.)
         float tau = 0.f;
+        const float kNoNeuron = __int_as_float(0x7fc00000);  // NaN: no threshold keeps a position past d_ff
 #pragma unroll
         for (int bt = 0; bt < kMaxBatches; ++bt) {
+            bal[bt] = 0u;
             if (bt >= n_batches) continue;  // uniform
-            const int q = bt * kFfnThreads + slot;
-            const bool has = q < chunks;
-            const int j0 = q * kWarp;
-            float4 v[8];
-            if (has && !bulk_scores) {
-                if (vec_ok && j0 + kWarp <= F) {
+            const int q0 = bt * kFfnThreads + warp * kWarp;  // the warp's first chunk of this batch
+            float v[kWarp];
+            if (!bulk_scores) {
 #pragma unroll
-                    for (int u = 0; u < 8; ++u)
-                        v[u] = ld_keep4(reinterpret_cast<const float4 *>(p.scores + j0) + u, keep_policy);
-                } else {
-#pragma unroll
-                    for (int u = 0; u < 8; ++u) {
-                        const int j = j0 + 4 * u;
-                        v[u].x = (j < F) ? ld_keep(p.scores + j, keep_policy) : -INFINITY;
-                        v[u].y = (j + 1 < F) ? ld_keep(p.scores + j + 1, keep_policy) : -INFINITY;
-                        v[u].z = (j + 2 < F) ? ld_keep(p.scores + j + 2, keep_policy) : -INFINITY;
-                        v[u].w = (j + 3 < F) ? ld_keep(p.scores + j + 3, keep_policy) : -INFINITY;
-                    }
+                for (int c = 0; c < kWarp; ++c) {
+                    const int j = (q0 + c) * kWarp + lane;
+                    v[c] = (q0 + c < chunks && j < F) ? ld_keep(p.scores + j, keep_policy) : kNoNeuron;
                 }
             }
             if (bt == 0) {  // the threshold arrives while the score loads are in flight
@@ -176,42 +170,27 @@ sparse_ffn_kernel(const FfnParams p, const int n_stages) {
                 tau = s_tau;
                 if (bulk_scores && !mbar_wait(sbar, 0) && tid == 0 && p.status) atomicOr(p.status, CLADA_STATUS_TIMEOUT);
             }
-            if (has && bulk_scores) {
+            if (bulk_scores) {
 #pragma unroll
-                for (int u = 0; u < 8; ++u) {
-                    if (j0 + 4 * u < F) {  // F is a multiple of 4 here: a vector is all in or all out
-                        const uint4 r = lds128(ring + (uint32_t)(j0 + 4 * u) * 4u);
-                        v[u] = make_float4(__uint_as_float(r.x), __uint_as_float(r.y), __uint_as_float(r.z),
-                                           __uint_as_float(r.w));
-                    } else {
-                        v[u] = make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
-                    }
+                for (int c = 0; c < kWarp; ++c) {
+                    const int j = (q0 + c) * kWarp + lane;
+                    v[c] = (q0 + c < chunks && j < F) ? lds_f32(ring + (uint32_t)j * 4u) : kNoNeuron;
                 }
             }
-            if (has) {
-                unsigned w = 0;
+            // lane c keeps the word of chunk q0 + c: thread tid owns chunk bt * kFfnThreads + tid, as below
 #pragma unroll
-                for (int u = 0; u < 8; ++u) {
-                    w |= (v[u].x >= tau ? 1u : 0u) << (4 * u);
-                    w |= (v[u].y >= tau ? 1u : 0u) << (4 * u + 1);
-                    w |= (v[u].z >= tau ? 1u : 0u) << (4 * u + 2);
-                    w |= (v[u].w >= tau ? 1u : 0u) << (4 * u + 3);
-                }
-                s_bal[q] = w;
+            for (int c = 0; c < kWarp; ++c) {
+                const unsigned w = __ballot_sync(0xffffffffu, v[c] >= tau);
+                if (lane == c) bal[bt] = w;
             }
         }
     }
-    __syncthreads();
-    unsigned bal[kMaxBatches];
     int first_rank[kMaxBatches];  // rank of this thread's chunk's first kept neuron
     int n_act = 0;
 #pragma unroll
     for (int bt = 0; bt < kMaxBatches; ++bt) {
-        bal[bt] = 0u;
         first_rank[bt] = 0;
         if (bt >= n_batches) continue;  // uniform
-        const int q = bt * kFfnThreads + tid;  // this thread's chunk
-        if (q < chunks) bal[bt] = s_bal[q];
         const int cnt = __popc(bal[bt]);
         int incl = cnt;
 #pragma unroll
