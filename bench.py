@@ -35,7 +35,7 @@ LAMBDA, GAMMA = 0.80, 0.12
 N_COPIES = 4
 # DRAM read + write bytes of one sparse_ffn_kernel launch at the baseline threshold of this workload, from the ncu
 # capture summarised in profiles/sparse_ffn_kernel_c2_full.md.  Must go back to None whenever that kernel changes.
-FFN_NCU_TRAFFIC_BYTES = 165.9e6   # mean of the two captured launches (166.0 and 165.7 MB)
+FFN_NCU_TRAFFIC_BYTES = None
 
 
 def _peaks():

@@ -157,12 +157,21 @@ sparse_ffn_kernel(const FfnParams p, const int n_stages) {
             bal[bt] = 0u;
             if (bt >= n_batches) continue;  // uniform
             const int q0 = bt * kFfnThreads + warp * kWarp;  // the warp's first chunk of this batch
+            const bool any = q0 < chunks;                    // warp-uniform: warps past the vector's end do nothing
+            // all 32 chunks whole and inside the vector: no per-element checks, constant offsets
+            const bool whole = q0 + kWarp <= chunks && (q0 + kWarp) * kWarp <= F;
             float v[kWarp];
-            if (!bulk_scores) {
+            if (!bulk_scores && any) {
+                if (whole) {
+                    const float *src = p.scores + (size_t)q0 * kWarp + lane;
 #pragma unroll
-                for (int c = 0; c < kWarp; ++c) {
-                    const int j = (q0 + c) * kWarp + lane;
-                    v[c] = (q0 + c < chunks && j < F) ? ld_keep(p.scores + j, keep_policy) : kNoNeuron;
+                    for (int c = 0; c < kWarp; ++c) v[c] = ld_keep(src + c * kWarp, keep_policy);
+                } else {
+#pragma unroll
+                    for (int c = 0; c < kWarp; ++c) {
+                        const int j = (q0 + c) * kWarp + lane;
+                        v[c] = (q0 + c < chunks && j < F) ? ld_keep(p.scores + j, keep_policy) : kNoNeuron;
+                    }
                 }
             }
             if (bt == 0) {  // the threshold arrives while the score loads are in flight
@@ -170,11 +179,18 @@ sparse_ffn_kernel(const FfnParams p, const int n_stages) {
                 tau = s_tau;
                 if (bulk_scores && !mbar_wait(sbar, 0) && tid == 0 && p.status) atomicOr(p.status, CLADA_STATUS_TIMEOUT);
             }
+            if (!any) continue;
             if (bulk_scores) {
+                if (whole) {
+                    const uint32_t src = ring + (uint32_t)(q0 * kWarp + lane) * 4u;
 #pragma unroll
-                for (int c = 0; c < kWarp; ++c) {
-                    const int j = (q0 + c) * kWarp + lane;
-                    v[c] = (q0 + c < chunks && j < F) ? lds_f32(ring + (uint32_t)j * 4u) : kNoNeuron;
+                    for (int c = 0; c < kWarp; ++c) v[c] = lds_f32(src + (uint32_t)c * (kWarp * 4u));
+                } else {
+#pragma unroll
+                    for (int c = 0; c < kWarp; ++c) {
+                        const int j = (q0 + c) * kWarp + lane;
+                        v[c] = (q0 + c < chunks && j < F) ? lds_f32(ring + (uint32_t)j * 4u) : kNoNeuron;
+                    }
                 }
             }
             // lane c keeps the word of chunk q0 + c: thread tid owns chunk bt * kFfnThreads + tid, as below
