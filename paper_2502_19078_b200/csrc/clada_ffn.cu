@@ -2,9 +2,10 @@
 //   kept = { j : A_j >= tau_final },  y = sum_{j in kept} silu(w_gate_j . x) (w_up_j . x) w_down_t[j,:]
 //
 // One persistent cooperative kernel per (layer, sequence), one CTA per SM:
-//   prologue  every CTA tests all F scores against tau (each thread owns whole 32-neuron chunks, so all
-//             its loads are independent: one memory round trip), a block scan ranks the chunks, and the
-//             CTA takes an equal share [r0, r1) of the kept neurons in ascending order;
+//   prologue  every CTA tests all F scores against tau (the vector arrives as one bulk copy into the idle
+//             ring; a warp tests 32 chunks of 32 neurons with one ballot each), a block scan ranks the
+//             chunks, and the CTA takes an equal share [r0, r1) of the kept neurons in ascending order,
+//             or, given a nested index list, simply copies its share of the list's head;
 //   stream    a producer thread copies the three contiguous rows of each kept neuron into a ring of
 //             shared-memory stages with bulk asynchronous copies (mbarrier-tracked), which keeps
 //             ~200 KB of HBM requests in flight per SM whatever the consumers are doing.  Consumer
@@ -111,10 +112,8 @@ sparse_ffn_kernel(const FfnParams p, const int n_stages) {
     }
 
     // ---- prologue: threshold test, ranks, this CTA's share of the kept list ---------------------
-    // A batch is one 32-neuron chunk per thread (eight independent 16-byte loads); F <= 32 * kFfnThreads
-    // needs a single batch.  Which chunk a thread LOADS is rotated by the CTA index, so that the 148
-    // CTAs do not all ask L2 for the same line at the same moment; the keep-bits words go through
-    // shared memory and are ranked in natural order by a block-wide scan.
+    // A batch is one 32-neuron chunk per thread; F <= 32 * kFfnThreads needs a single batch.  The keep-bits
+    // words stay in registers (thread tid owns chunk tid of the batch) and are ranked by a block-wide scan.
     int n_act_o = 0, r0_o = 0, r1_o = 0;
     if (nested) {
         // The list exists already: this CTA copies its share of the leading n_act entries.  A count or
