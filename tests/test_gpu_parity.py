@@ -333,6 +333,16 @@ def test_sparse_ffn_bf16_shapes(clada, oracle, d, F):
     assert worst <= FFN_TOL_F32
 
 
+@pytest.mark.parametrize("d,F", [(64, 17409), (64, 20000), (32, 40001)])
+def test_sparse_ffn_wide_layers(clada, oracle, d, F):
+    """More than 17408 neurons: the score test runs in two or three batches of 544 chunks per CTA, with a ragged
+    last chunk; masks, index lists and outputs as for the narrow layers."""
+    w = _small("c2_llama2_7b_layer", d_model=d, d_ff=F)
+    worst, excused, mismatched = _ffn_case(clada, oracle, w, 0.40, 4, prefix=20)
+    assert mismatched == 0
+    assert worst <= FFN_TOL_F32
+
+
 @pytest.mark.parametrize("d,F", [(16, 40), (512, 1376), (1032, 300), (4096, 300)])
 def test_sparse_ffn_f32_shapes(clada, oracle, d, F):
     w = _small("c1_small_f32", d_model=d, d_ff=F)
