@@ -486,7 +486,8 @@ def test_algorithm2_loop_config1(clada, oracle):
 # ------------------------------------------------------------------------------------------------
 
 @pytest.mark.parametrize("name,d,F,B", [("c4_llama3_8b_b8", 1024, 1800, 7), ("c5_13b_b16", 5120, 700, 5),
-                                        ("c1_small_f32", 512, 1376, 6), ("c4_llama3_8b_b8", 4096, 1000, 4)])
+                                        ("c1_small_f32", 512, 1376, 6), ("c4_llama3_8b_b8", 4096, 1000, 4),
+                                        ("c4_llama3_8b_b8", 64, 20001, 5)])
 def test_sparse_ffn_batched_tiles(clada, oracle, name, d, F, B):
     """Per-sequence scores and thresholds, including a sequence that keeps nothing and one that keeps all:
     every y_b must be the sum over its own kept set although the tile streams the union."""
