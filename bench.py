@@ -757,10 +757,20 @@ def main():
                     help="the metric's workload (default); the 32-layer stack or the OPT- / Gemma-shaped "
                          "layers (other FFN forms) for information")
     args = ap.parse_args()
+    if args.gpus < 1:
+        ap.error("--gpus must be at least 1")
     if args.impl == "reference":
         run_reference(args)
+    elif args.gpus > 1 and not sharding.under_launcher():
+        # started by hand rather than by torchrun: become the launcher of one rank per GPU
+        try:
+            rc = sharding.launch_ranks(args.gpus, [os.path.abspath(__file__)] + sys.argv[1:],
+                                       devices_available=torch.cuda.device_count())
+        except ValueError as e:
+            sys.exit(f"bench.py: {e}")
+        sys.exit(rc)
     else:
-        run_ours(args)
+        run_ours(args)      # one rank; the world size is the launcher's (RANK / WORLD_SIZE)
 
 
 if __name__ == "__main__":
