@@ -263,7 +263,14 @@ int clada_sparse_ffn_decode_layers(const clada_layer *layers, int32_t L, const v
  * itself allocates nothing.
  *  - Limits: d_model <= 8192 and a device with at most 160 SMs; beyond that the
  *    call returns CLADA_ERR_UNSUPPORTED (clada_last_cuda_error() says why)
- *    and enqueues nothing.
+ *    and enqueues nothing.  Every refusal happens before the first enqueue.
+ *  - Batches: the array holds 160 x 8192 fp32 partial outputs, i.e. one row per
+ *    (SM, sequence of a tile).  B >= 2 therefore runs in the largest tiles of
+ *    sequences (4, 2 or 1 per launch) that fit: on a 148-SM device tiles of 4 up
+ *    to d_model 2048, tiles of 2 up to d_model 4096, one sequence per launch
+ *    above that.  Results per sequence are those of clada_sparse_ffn_decode;
+ *    smaller tiles only read the shared weight rows once per tile instead of
+ *    once per larger tile.
  *  - The first call on a device looks up the array's device address; make that
  *    first call outside any stream capture.
  *  - All calls share the one array and it keeps the previous call's contents;

@@ -509,30 +509,45 @@ static int launch_ffn(const FfnParams &p, cudaStream_t st) {
 
 using namespace clada;
 
-static int decode_with_workspace(const clada_layer *layer, const void *x, int32_t B, const float *scores,
-                                 const float *tau_final, int64_t tau_stride, void *y, int32_t y_dtype,
-                                 uint8_t *mask_out, int32_t *idx_out, int32_t *count_out, void *ws,
-                                 size_t ws_bytes, int32_t *status, void *stream) {
+// Host-side checks of a decode call; nothing is enqueued here.
+static int decode_validate(const clada_layer *layer, const void *x, int32_t B, const float *scores,
+                           const float *tau_final, int64_t tau_stride, const void *y, int32_t y_dtype) {
     int rc = validate_layer(layer, false);
     if (rc != CLADA_OK) return rc;
     if (!x || !scores || !tau_final || !y) return CLADA_ERR_NULL;
     if (B <= 0 || tau_stride < 0) return CLADA_ERR_SHAPE;
     if (!dtype_ok(y_dtype)) return CLADA_ERR_DTYPE;
     if (!aligned16(x) || !aligned16(y)) return CLADA_ERR_ALIGN;
-    if (!ws || (reinterpret_cast<uintptr_t>(ws) & 255u)) return CLADA_ERR_WORKSPACE;
-    DeviceInfo di;
-    rc = device_info(&di);
-    if (rc != CLADA_OK) return rc;
-    const size_t need = kWsCtrlBytes + (size_t)di.num_sms * (B >= 4 ? 4 : B >= 2 ? 2 : 1) * layer->d_model * sizeof(float);
-    if (ws_bytes < need) return CLADA_ERR_WORKSPACE;
+    if (layer->d_ff > kMaxBatches * kWarp * kFfnThreads) return CLADA_ERR_UNSUPPORTED;
+    return CLADA_OK;
+}
 
+// Sequences per launch for the next `remaining` sequences of a batch, at most max_tile (4, 2 or 1): a tile
+// kernel that takes 4 sequences of this layer also takes 2.
+static int decode_tile(const clada_layer *layer, int remaining, int max_tile) {
+    const int bt = ffn_batch_tile(layer, remaining);
+    return bt < max_tile ? bt : max_tile;
+}
+
+// Scratch bytes a decode call needs when its tiles hold at most max_tile sequences: the control words and
+// one fp32 partial output row per (CTA, sequence of the tile).
+static size_t decode_scratch_bytes(const clada_layer *layer, int32_t B, int num_sms, int max_tile) {
+    return kWsCtrlBytes + (size_t)num_sms * decode_tile(layer, B, max_tile) * layer->d_model * sizeof(float);
+}
+
+// The launches of a validated decode call whose scratch holds tiles of up to max_tile sequences.
+static int decode_enqueue(const clada_layer *layer, const void *x, int32_t B, const float *scores,
+                          const float *tau_final, int64_t tau_stride, void *y, int32_t y_dtype,
+                          uint8_t *mask_out, int32_t *idx_out, int32_t *count_out, void *ws, int max_tile,
+                          int32_t *status, void *stream) {
+    int rc;
     const size_t esz = elem_size(layer->dtype);
     const size_t ysz = elem_size(y_dtype);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     int b = 0;
     while (b < B) {
         // Tiles of 4 or 2 sequences read each row of the union of their kept sets once.
-        const int bt = ffn_batch_tile(layer, B - b);
+        const int bt = decode_tile(layer, B - b, max_tile);
         if (bt > 1) {
             if (mask_out || idx_out || count_out) {  // the tile kernel computes y only
                 rc = clada_select(scores + (size_t)b * layer->d_ff, bt, layer->d_ff, tau_final + (size_t)b * tau_stride,
@@ -576,6 +591,21 @@ static int decode_with_workspace(const clada_layer *layer, const void *x, int32_
         ++b;
     }
     return CLADA_OK;
+}
+
+static int decode_with_workspace(const clada_layer *layer, const void *x, int32_t B, const float *scores,
+                                 const float *tau_final, int64_t tau_stride, void *y, int32_t y_dtype,
+                                 uint8_t *mask_out, int32_t *idx_out, int32_t *count_out, void *ws,
+                                 size_t ws_bytes, int32_t *status, void *stream) {
+    int rc = decode_validate(layer, x, B, scores, tau_final, tau_stride, y, y_dtype);
+    if (rc != CLADA_OK) return rc;
+    if (!ws || (reinterpret_cast<uintptr_t>(ws) & 255u)) return CLADA_ERR_WORKSPACE;
+    DeviceInfo di;
+    rc = device_info(&di);
+    if (rc != CLADA_OK) return rc;
+    if (ws_bytes < decode_scratch_bytes(layer, B, di.num_sms, 4)) return CLADA_ERR_WORKSPACE;
+    return decode_enqueue(layer, x, B, scores, tau_final, tau_stride, y, y_dtype, mask_out, idx_out, count_out, ws,
+                          4, status, stream);
 }
 
 extern "C" int clada_sparse_ffn_decode(const clada_layer *layer, const void *x, int32_t B,
@@ -632,8 +662,9 @@ extern "C" int clada_sparse_ffn_decode_nested(const clada_layer *layer, const vo
     return CLADA_OK;
 }
 
-// One decode step of a whole stack: the per-layer call in a native loop (one C call per token instead
-// of one per layer); the launches chain with programmatic dependent launch.
+// One decode step of a whole stack.  A single sequence runs all layers in one persistent launch
+// (clada_ffn_stack.cu); a batch runs the per-layer call in a native loop (one C call per token instead
+// of one per layer; the launches chain with programmatic dependent launch).
 extern "C" int clada_sparse_ffn_decode_layers(const clada_layer *layers, int32_t L, const void *x, int32_t B,
                                               const float *scores, const float *tau_final, void *y,
                                               int32_t y_dtype, void *ws, size_t ws_bytes, int32_t *status,
@@ -648,8 +679,13 @@ extern "C" int clada_sparse_ffn_decode_layers(const clada_layer *layers, int32_t
             layers[l].dtype != layers[0].dtype)
             return CLADA_ERR_SHAPE;
     }
+    if (!aligned16(x) || !aligned16(y)) return CLADA_ERR_ALIGN;
+    if (!ws || (reinterpret_cast<uintptr_t>(ws) & 255u)) return CLADA_ERR_WORKSPACE;
     const size_t d = (size_t)layers[0].d_model, F = (size_t)layers[0].d_ff;
     const size_t x_layer = (size_t)B * d * elem_size(layers[0].dtype), y_layer = (size_t)B * d * elem_size(y_dtype);
+    if (ffn_stack_supported(layers, L, B, ws_bytes))
+        return launch_ffn_stack(layers, L, x, x_layer, scores, tau_final, 1, y, y_layer, y_dtype, ws, status,
+                                static_cast<cudaStream_t>(stream));
     for (int l = 0; l < L; ++l) {
         int rc = decode_with_workspace(&layers[l], static_cast<const char *>(x) + l * x_layer, B,
                                        scores + (size_t)l * B * F, tau_final + l, L,
@@ -696,11 +732,19 @@ extern "C" int clada_sparse_ffn_decode_static(const clada_layer *layer, const vo
                                               int64_t tau_stride, void *y, int32_t y_dtype,
                                               uint8_t *mask_out, int32_t *idx_out, int32_t *count_out,
                                               int32_t *status, void *stream) {
-    if (!layer) return CLADA_ERR_NULL;
-    DeviceInfo di;
-    int rc = device_info(&di);
+    // Everything that can be refused is refused before the first enqueue.
+    int rc = decode_validate(layer, x, B, scores, tau_final, tau_stride, y, y_dtype);
     if (rc != CLADA_OK) return rc;
-    if (layer->d_model > kStaticMaxDModel || di.num_sms > kStaticMaxSms) {
+    DeviceInfo di;
+    rc = device_info(&di);
+    if (rc != CLADA_OK) return rc;
+    // The largest tile of sequences whose partial rows fit the array: a batch that the workspace entry would
+    // cut into tiles of 4 runs here in tiles of 2, or one sequence per launch, when the array is too small
+    // for more (same results per sequence; the weight rows are then read once per smaller tile).
+    int max_tile = 4;
+    while (max_tile > 1 && decode_scratch_bytes(layer, B, di.num_sms, max_tile) > kStaticScratchBytes) max_tile >>= 1;
+    if (layer->d_model > kStaticMaxDModel || di.num_sms > kStaticMaxSms ||
+        decode_scratch_bytes(layer, B, di.num_sms, max_tile) > kStaticScratchBytes) {
         set_last_cuda_error(cudaErrorInvalidValue,
                             "clada_sparse_ffn_decode_static: d_model > 8192 or more than 160 SMs exceeds the "
                             "built-in scratch; use clada_sparse_ffn_decode with a workspace");
@@ -712,6 +756,6 @@ extern "C" int clada_sparse_ffn_decode_static(const clada_layer *layer, const vo
     // The array keeps whatever the last call left.  The control words must start at zero (they are
     // zero after a clean call, not after one that timed out), so clear them in stream order.
     CLADA_CUDA_TRY(cudaMemsetAsync(scratch, 0, kWsCtrlBytes, static_cast<cudaStream_t>(stream)));
-    return decode_with_workspace(layer, x, B, scores, tau_final, tau_stride, y, y_dtype, mask_out, idx_out,
-                                 count_out, scratch, kStaticScratchBytes, status, stream);
+    return decode_enqueue(layer, x, B, scores, tau_final, tau_stride, y, y_dtype, mask_out, idx_out, count_out,
+                          scratch, max_tile, status, stream);
 }

@@ -1,0 +1,612 @@
+// Sparse gated FFN of one decode token through a whole stack of layers in ONE persistent launch
+// (Algorithm 2, generation phase: the loop over layers inside a decode step):
+//   for l = 0 .. L-1:  kept_l = { j : A_lj >= tau_l },
+//                      y_l = sum_{j in kept_l} silu(w_gate_lj . x_l) (w_up_lj . x_l) w_down_t_l[j,:]
+//
+// A launch per layer pays, per layer, for what does not move weight bytes: the launch ramp, the score
+// test, the first rows' latency, the slowest CTA's tail, a grid barrier and the column sums.  Here the
+// weight stream never stops at a layer boundary.  One cooperative CTA per SM, as in the per-layer kernel:
+//   producer  one thread walks layer after layer: the layer's x (one ring stage), then the three rows of
+//             every kept neuron of this CTA's share, as bulk asynchronous copies into the ring.  It runs
+//             ahead of the consumers by the ring's depth, across layer boundaries.
+//   consumers 512 threads.  Per layer: x from its stage into registers, the share's neurons four per
+//             CTA-wide reduction, the CTA's partial y to global memory, ARRIVE at the grid barrier, then
+//             -- while the other CTAs arrive -- the score test and the share list of layer l + 2, then
+//             WAIT at the barrier and sum a slice of columns over all CTAs' partials in CTA order.
+//             All of this takes the consumers less time than the ring holds rows for, so the copies
+//             into the ring go on while they are away from it.
+// Kept lists are built two layers ahead in a double buffer, partial rows are double buffered by barrier
+// number, every wait is bounded, and the summation order is fixed: results repeat bit for bit.
+#include <math.h>
+
+#include "common.cuh"
+#include "ffn_common.cuh"
+
+namespace clada {
+
+constexpr int kMaxStackLayers = 128;  // layers per launch (their weight pointers travel as kernel parameters)
+constexpr int kStackMaxBatches = 4;   // score-test batches: d_ff <= 4 * 32 * kConsumers
+constexpr int GS = 4;                 // neurons per CTA-wide reduction
+
+struct StackLayers {
+    const void *w[kMaxStackLayers][3];  // w_gate, w_up, w_down_t of every layer
+};
+
+struct StackParams {
+    const char *x;        // layer l reads x + l * x_stride (bytes)
+    size_t x_stride;
+    const float *scores;  // layer l: scores + l * d_ff
+    const float *tau;     // layer l: tau[l * tau_stride]
+    long long tau_stride;
+    char *y;              // layer l writes y + l * y_stride (bytes)
+    size_t y_stride;
+    int y_dtype;
+    float *partials;      // [2][gridDim.x][d_model]
+    WsCtrl *ctrl;
+    int32_t *status;
+    int d_model, d_ff, L;
+    int act;
+};
+
+__device__ __forceinline__ int stack_split_at(int n, int c, int n_ctas) {
+    return (int)(((unsigned)n * (unsigned)c) / (unsigned)n_ctas);
+}
+
+__device__ __forceinline__ void consumer_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kConsumers) : "memory"); }
+
+// Score test of one layer by the 512 consumer threads: keep bits A_j >= tau (one ballot per 32-neuron
+// chunk, coalesced loads), block-wide ranks, and this CTA's equal share [r0, r1) of the kept neurons in
+// ascending order written to list[].  Returns the layer's kept count; *my_n = r1 - r0.
+__device__ __forceinline__ int build_share_list(const float *__restrict__ scores, const float tau, const int F,
+                                                const int cta, const int n_ctas, int *list, int *s_wtot,
+                                                int *my_n, const uint64_t keep_policy) {
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int chunks = (F + kWarp - 1) / kWarp;
+    const int n_batches = (chunks + kConsumers - 1) / kConsumers;
+    const float kNoNeuron = __int_as_float(0x7fc00000);  // NaN: no threshold keeps a position past d_ff
+    unsigned bal[kStackMaxBatches];
+    int first_rank[kStackMaxBatches];
+    int n_act = 0;
+#pragma unroll
+    for (int bt = 0; bt < kStackMaxBatches; ++bt) {
+        bal[bt] = 0u;
+        first_rank[bt] = 0;
+        if (bt >= n_batches) continue;  // uniform
+        const int q0 = bt * kConsumers + warp * kWarp;  // the warp's first chunk of this batch
+        if (q0 < chunks) {
+            const bool whole = q0 + kWarp <= chunks && (q0 + kWarp) * kWarp <= F;
+#pragma unroll
+            for (int c0 = 0; c0 < kWarp; c0 += 8) {  // eight loads in flight per lane
+                float v[8];
+                if (whole) {
+                    const float *src = scores + (size_t)(q0 + c0) * kWarp + lane;
+#pragma unroll
+                    for (int c = 0; c < 8; ++c) v[c] = ld_keep(src + c * kWarp, keep_policy);
+                } else {
+#pragma unroll
+                    for (int c = 0; c < 8; ++c) {
+                        const int j = (q0 + c0 + c) * kWarp + lane;
+                        v[c] = (q0 + c0 + c < chunks && j < F) ? ld_keep(scores + j, keep_policy) : kNoNeuron;
+                    }
+                }
+#pragma unroll
+                for (int c = 0; c < 8; ++c) {
+                    const unsigned w = __ballot_sync(0xffffffffu, v[c] >= tau);
+                    if (lane == c0 + c) bal[bt] = w;  // lane c keeps the word of chunk q0 + c
+                }
+            }
+        }
+        const int cnt = __popc(bal[bt]);
+        int incl = cnt;
+#pragma unroll
+        for (int o = 1; o < kWarp; o <<= 1) {
+            const int t = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += t;
+        }
+        consumer_sync();  // s_wtot free again (also orders the previous user of list[] before the writes below)
+        if (lane == kWarp - 1) s_wtot[warp] = incl;
+        consumer_sync();
+        int wbase = 0, btot = 0;
+#pragma unroll
+        for (int w = 0; w < kConsWarps; ++w) {
+            const int v = s_wtot[w];
+            wbase += (w < warp) ? v : 0;
+            btot += v;
+        }
+        first_rank[bt] = n_act + wbase + incl - cnt;
+        n_act += btot;
+    }
+    const int r0 = stack_split_at(n_act, cta, n_ctas);
+    const int r1 = stack_split_at(n_act, cta + 1, n_ctas);
+#pragma unroll
+    for (int bt = 0; bt < kStackMaxBatches; ++bt) {
+        if (bt >= n_batches) continue;  // uniform
+        const int q = bt * kConsumers + tid;
+        const int fr = first_rank[bt];
+        const bool in_share = q < chunks && fr < r1 && fr + __popc(bal[bt]) > r0;
+        unsigned todo = __ballot_sync(0xffffffffu, in_share);
+        while (todo) {
+            const int t = __ffs(todo) - 1;
+            todo &= todo - 1;
+            const unsigned wb = __shfl_sync(0xffffffffu, bal[bt], t);
+            const int wfr = __shfl_sync(0xffffffffu, fr, t);
+            const int j = (bt * kConsumers + (warp * kWarp + t)) * kWarp + lane;
+            const int rank = wfr + __popc(wb & ((1u << lane) - 1u));
+            if (((wb >> lane) & 1u) && rank >= r0 && rank < r1) list[rank - r0] = j;
+        }
+    }
+    *my_n = r1 - r0;
+    return n_act;
+}
+
+template <typename T, int NV, bool GATED>
+__global__ void __launch_bounds__(kFfnThreads, 1)
+sparse_ffn_stack_kernel(const StackParams p, const __grid_constant__ StackLayers lay, const int n_stages,
+                        const int list_cap) {
+    constexpr int E = Elem<T>::kPerVec;
+    constexpr int P = Pairs<T>::kPairs;
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int cta = blockIdx.x, n_ctas = gridDim.x;
+    const int F = p.d_ff, d = p.d_model, L = p.L;
+    const int vpr = d / E;  // 16-byte vectors per row
+    const uint32_t row_bytes = (uint32_t)vpr * 16u;
+    constexpr uint32_t kRows = GATED ? 3u : 2u;
+    const uint32_t stage_bytes = kRows * row_bytes;
+    const uint32_t down_off = (kRows - 1u) * row_bytes;
+
+    // dynamic shared memory: ring | full[kMaxStages] | empty[kMaxStages] | list-ready[2] | list-done[2] |
+    // lists[2][list_cap]
+    const uint32_t ring = smem_u32(smem_raw);
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem_raw + (size_t)n_stages * stage_bytes);
+    const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + kMaxStages);
+    const uint32_t lbar0 = smem_u32(bars + 2 * kMaxStages);      // consumers -> producer: the list of a layer is written
+    const uint32_t pbar0 = smem_u32(bars + 2 * kMaxStages + 2);  // producer -> consumers: done with that list
+    int *s_list = reinterpret_cast<int *>(bars + 2 * kMaxStages + 4);
+    __shared__ int s_wtot[kConsWarps];
+    __shared__ int s_nact[2], s_myn[2];  // per list buffer: the layer's kept count, this CTA's share
+    __shared__ int s_ok;
+    __shared__ __align__(16) float s_dot[2][2 * GS][kConsWarps];
+
+    pdl_launch_dependents();
+    if (tid == kConsumers) {
+        for (int s = 0; s < n_stages; ++s) {
+            mbar_init(full0 + 8 * s, 1);            // the producer's expect_tx arrival
+            mbar_init(empty0 + 8 * s, kConsWarps);  // one arrival per consumer warp
+        }
+        mbar_init(lbar0, 1);
+        mbar_init(lbar0 + 8, 1);
+        mbar_init(pbar0, 1);
+        mbar_init(pbar0 + 8, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    pdl_wait();      // everything below may read what the previous kernel wrote
+    __syncthreads();  // the mbarriers exist
+
+    bool timed_out = false;
+
+    if (warp == kConsWarps) {
+        // ---- producer -----------------------------------------------------------------------------
+        if (lane == 0) {
+            const uint64_t stream_policy = policy_evict_first();
+            const uint64_t keep_policy = policy_evict_last();
+            long long issued = 0;
+            int s = 0;  // ring position and the parity of its current use, kept incrementally
+            uint32_t par = 0;
+            for (int l = 0; l < L && !timed_out; ++l) {
+                const int lb = l & 1;
+                if (!mbar_wait(lbar0 + 8 * lb, (uint32_t)(l >> 1) & 1u)) {  // layer l's list is in buffer lb
+                    timed_out = true;
+                    break;
+                }
+                const int my_n = s_myn[lb];
+                if (s_nact[lb] == 0 || my_n == 0) {  // nothing of this layer for this CTA
+                    mbar_arrive(pbar0 + 8 * lb);
+                    continue;
+                }
+                const int *list = s_list + lb * list_cap;
+                const char *Wg = static_cast<const char *>(lay.w[l][0]);
+                const char *Wu = static_cast<const char *>(lay.w[l][1]);
+                const char *Wd = static_cast<const char *>(lay.w[l][2]);
+                for (int i = -1; i < my_n; ++i) {  // i = -1: the layer's x takes a stage of its own
+                    if (!mbar_wait(empty0 + 8 * s, par ^ 1)) {  // a fresh barrier passes parity 1 at once
+                        timed_out = true;
+                        break;
+                    }
+                    const uint32_t dst = ring + (uint32_t)s * stage_bytes, bar = full0 + 8 * s;
+                    if (i < 0) {
+                        mbar_expect_tx(bar, row_bytes);
+                        bulk_load_row_hint(dst, p.x + (size_t)l * p.x_stride, row_bytes, bar, keep_policy);
+                    } else {
+                        const size_t off = (size_t)list[i] * row_bytes;
+                        mbar_expect_tx(bar, stage_bytes);
+                        bulk_load_row_hint(dst, Wg + off, row_bytes, bar, stream_policy);
+                        if (GATED) bulk_load_row_hint(dst + row_bytes, Wu + off, row_bytes, bar, stream_policy);
+                        bulk_load_row_hint(dst + down_off, Wd + off, row_bytes, bar, stream_policy);
+                    }
+                    ++issued;
+                    if (++s == n_stages) {
+                        s = 0;
+                        par ^= 1;
+                    }
+                }
+                if (!timed_out) mbar_arrive(pbar0 + 8 * lb);  // buffer lb may take the list of layer l + 2
+            }
+            // Never leave with copies in flight: the last use of every stage must have landed.
+            const long long first = issued > n_stages ? issued - n_stages : 0;
+            for (long long i = first; i < issued; ++i)
+                if (!mbar_wait(full0 + 8 * (int)(i % n_stages), (uint32_t)(i / n_stages) & 1u)) timed_out = true;
+            if (timed_out && p.status) atomicOr(p.status, CLADA_STATUS_TIMEOUT);
+        }
+        return;
+    }
+
+    // ---- consumers ------------------------------------------------------------------------------------
+    const uint64_t keep_policy = policy_evict_last();
+    bool vok[NV];
+#pragma unroll
+    for (int i = 0; i < NV; ++i) vok[i] = tid + i * kConsumers < vpr;
+
+    // The lists of layers 0 and 1 come first; from then on the list of layer l + 2 is built inside layer l.
+    for (int l = 0; l < 2 && l < L; ++l) {
+        const float tau = ld_keep(p.tau + (size_t)l * p.tau_stride, keep_policy);
+        int my_n;
+        const int n_act = build_share_list(p.scores + (size_t)l * F, tau, F, cta, n_ctas, s_list + l * list_cap,
+                                           s_wtot, &my_n, keep_policy);
+        if (tid == 0) {
+            s_nact[l] = n_act;
+            s_myn[l] = my_n;
+        }
+        consumer_sync();  // the list and its counts are written
+        if (tid == 0) mbar_arrive(lbar0 + 8 * l);
+    }
+
+    const bool b16 = lane & 16, b8 = lane & 8, b4 = lane & 4;
+    int cs = 0;  // ring position of the next stage to consume, and the parity of its use
+    uint32_t cpar = 0;
+    unsigned epoch = 0;  // grid barriers passed so far (layers that kept something)
+    for (int l = 0; l < L; ++l) {
+        const int lb = l & 1;
+        const int n_act = s_nact[lb], my_n = s_myn[lb];
+        char *yl = p.y + (size_t)l * p.y_stride;
+        float next_tau = 0.f;
+        if (l + 2 < L) next_tau = ld_keep(p.tau + (size_t)(l + 2) * p.tau_stride, keep_policy);  // used after the layer
+        if (n_act > 0) {
+            // x of this thread's columns, from the stage the producer filled ahead of the layer's rows
+            float2 xr[NV][P];
+#pragma unroll
+            for (int i = 0; i < NV; ++i)
+#pragma unroll
+                for (int e = 0; e < P; ++e) xr[i][e] = make_float2(0.f, 0.f);
+            if (my_n > 0) {
+                if (!timed_out && !mbar_wait(full0 + 8 * cs, cpar)) timed_out = true;
+                const uint32_t xa = ring + (uint32_t)cs * stage_bytes;
+#pragma unroll
+                for (int i = 0; i < NV; ++i)
+                    if (vok[i]) Pairs<T>::unpack(lds128(xa + (uint32_t)(tid + i * kConsumers) * 16u), xr[i]);
+                __syncwarp();
+                if (lane == 0) mbar_arrive(empty0 + 8 * cs);
+                if (++cs == n_stages) {
+                    cs = 0;
+                    cpar ^= 1;
+                }
+            }
+            float2 acc[NV][P];
+#pragma unroll
+            for (int i = 0; i < NV; ++i)
+#pragma unroll
+                for (int e = 0; e < P; ++e) acc[i][e] = make_float2(0.f, 0.f);
+            int buf = 0;
+            for (int g0 = 0; g0 < my_n; g0 += GS, buf ^= 1) {
+                float pd[2 * GS];
+                uint32_t st_addr[GS];
+                int st_idx[GS];
+#pragma unroll
+                for (int g = 0; g < GS; ++g) {
+                    const int i = g0 + g;
+                    float2 sg = make_float2(0.f, 0.f), su = make_float2(0.f, 0.f);
+                    st_idx[g] = cs;
+                    st_addr[g] = ring + (uint32_t)cs * stage_bytes;
+                    if (i < my_n) {
+                        if (!timed_out && !mbar_wait(full0 + 8 * cs, cpar)) timed_out = true;
+                        if (++cs == n_stages) {
+                            cs = 0;
+                            cpar ^= 1;
+                        }
+#pragma unroll
+                        for (int k = 0; k < NV; ++k) {
+                            if (!vok[k]) continue;
+                            const uint32_t a = st_addr[g] + (uint32_t)(tid + k * kConsumers) * 16u;
+                            float2 fg[P], fu[P];
+                            Pairs<T>::unpack(lds128(a), fg);
+                            if (GATED) Pairs<T>::unpack(lds128(a + row_bytes), fu);
+#pragma unroll
+                            for (int e = 0; e < P; ++e) {
+                                sg = __ffma2_rn(fg[e], xr[k][e], sg);
+                                if (GATED) su = __ffma2_rn(fu[e], xr[k][e], su);
+                            }
+                        }
+                    }
+                    pd[2 * g] = sg.x + sg.y;
+                    pd[2 * g + 1] = su.x + su.y;
+                }
+                // Warp sums of the 8 values by a halving butterfly (9 shuffles): after it every lane of
+                // quad q holds the warp total of value q.  Fixed order, so results repeat bit for bit.
+                float b[4], c[2], v8;
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const float send = b16 ? pd[i] : pd[i + 4];
+                    b[i] = (b16 ? pd[i + 4] : pd[i]) + __shfl_xor_sync(0xffffffffu, send, 16);
+                }
+#pragma unroll
+                for (int i = 0; i < 2; ++i) {
+                    const float send = b8 ? b[i] : b[i + 2];
+                    c[i] = (b8 ? b[i + 2] : b[i]) + __shfl_xor_sync(0xffffffffu, send, 8);
+                }
+                v8 = (b4 ? c[1] : c[0]) + __shfl_xor_sync(0xffffffffu, b4 ? c[0] : c[1], 4);
+                v8 += __shfl_xor_sync(0xffffffffu, v8, 2);
+                v8 += __shfl_xor_sync(0xffffffffu, v8, 1);
+                // lane 4q holds value index: bit4 -> +4, bit3 -> +2, bit2 -> +1
+                if ((lane & 3) == 0) s_dot[buf][(b16 ? 4 : 0) + (b8 ? 2 : 0) + (b4 ? 1 : 0)][warp] = v8;
+                consumer_sync();
+                // Cross-warp sums: lane l adds 4 consecutive warps of value l/4, the quad finishes by
+                // butterfly; then gate lanes form the neuron value h.
+                float tot;
+                {
+                    const float4 q4 = *reinterpret_cast<const float4 *>(&s_dot[buf][lane >> 2][(lane & 3) * 4]);
+                    tot = (q4.x + q4.y) + (q4.z + q4.w);
+                    tot += __shfl_xor_sync(0xffffffffu, tot, 1);
+                    tot += __shfl_xor_sync(0xffffffffu, tot, 2);
+                }
+                const float up = __shfl_xor_sync(0xffffffffu, tot, 4);  // value 2g+1 sits 4 lanes above value 2g
+                const float hval = neuron_value_f(p.act, tot, up);      // meaningful on lanes 8g..8g+3
+#pragma unroll
+                for (int g = 0; g < GS; ++g) {
+                    const float h = __shfl_sync(0xffffffffu, hval, 8 * g);
+                    if (g0 + g >= my_n) continue;
+                    const float2 h2 = make_float2(h, h);
+#pragma unroll
+                    for (int k = 0; k < NV; ++k) {
+                        if (!vok[k]) continue;
+                        float2 fd[P];
+                        Pairs<T>::unpack(lds128(st_addr[g] + down_off + (uint32_t)(tid + k * kConsumers) * 16u), fd);
+#pragma unroll
+                        for (int e = 0; e < P; ++e) acc[k][e] = __ffma2_rn(h2, fd[e], acc[k][e]);
+                    }
+                }
+                // hand the stages back to the producer
+                __syncwarp();
+                if (lane == 0) {
+#pragma unroll
+                    for (int g = 0; g < GS; ++g)
+                        if (g0 + g < my_n) mbar_arrive(empty0 + 8 * st_idx[g]);
+                }
+            }
+            // partial y of this CTA, into the buffer of this barrier number
+            float *mine = p.partials + ((size_t)(epoch & 1u) * n_ctas + cta) * d;
+#pragma unroll
+            for (int i = 0; i < NV; ++i) {
+                if (!vok[i]) continue;
+                float4 *dst = reinterpret_cast<float4 *>(mine + (size_t)(tid + i * kConsumers) * E);
+#pragma unroll
+                for (int e = 0; e < P; e += 2)
+                    dst[e / 2] = make_float4(acc[i][e].x, acc[i][e].y, acc[i][e + 1].x, acc[i][e + 1].y);
+            }
+            consumer_sync();  // every consumer's part of the row is written
+            if (tid == 0) {   // arrive; the wait comes after the next list
+                __threadfence();
+                atomicAdd(&p.ctrl->arrive, 1u);
+            }
+        }
+
+        // ---- the list of layer l + 2 replaces layer l's (its rows have all been consumed) ----------------
+        if (l + 2 < L) {
+            // The producer has read this buffer's counts (it may not have if the layer gave it nothing to copy).
+            if (!timed_out && !mbar_wait(pbar0 + 8 * lb, (uint32_t)(l >> 1) & 1u)) timed_out = true;
+            int nn;
+            const int na = build_share_list(p.scores + (size_t)(l + 2) * F, next_tau, F, cta, n_ctas,
+                                            s_list + lb * list_cap, s_wtot, &nn, keep_policy);
+            consumer_sync();  // everyone has read s_nact / s_myn of layer l, and the list is written
+            if (tid == 0) {
+                s_nact[lb] = na;
+                s_myn[lb] = nn;
+            }
+            consumer_sync();
+            if (tid == 0) mbar_arrive(lbar0 + 8 * lb);
+        }
+
+        if (n_act == 0) {
+            // Nothing is kept (every CTA sees the same count): y = 0, written slice by slice; no partial
+            // sums exist, so this layer has no grid barrier.
+            const int ng = d / 4;
+            const int q0 = stack_split_at(ng, cta, n_ctas), q1 = stack_split_at(ng, cta + 1, n_ctas);
+            for (int q = q0 + tid; q < q1; q += kConsumers) {
+                if (p.y_dtype == CLADA_F32)
+                    reinterpret_cast<float4 *>(yl)[q] = make_float4(0.f, 0.f, 0.f, 0.f);
+                else
+                    reinterpret_cast<uint2 *>(yl)[q] = make_uint2(0u, 0u);
+            }
+            continue;
+        }
+
+        // ---- wait for every CTA's partial row of this layer, then the column sums ------------------------
+        if (tid == 0) {
+            const unsigned target = (epoch + 1u) * (unsigned)n_ctas;
+            unsigned spins = 0, seen;
+            int ok = 1;
+            for (;;) {
+                asm volatile("ld.acquire.gpu.u32 %0, [%1];" : "=r"(seen) : "l"(&p.ctrl->arrive) : "memory");
+                if (seen >= target) break;
+                if (timed_out || ++spins > kBarrierSpinLimit) {
+                    ok = 0;
+                    break;
+                }
+            }
+            s_ok = ok;
+        }
+        consumer_sync();
+        if (s_ok == 0) timed_out = true;
+        consumer_sync();  // s_ok is free for the next layer
+        const float *part = p.partials + (size_t)(epoch & 1u) * n_ctas * d;
+        ++epoch;
+        // columns in groups of 4 (float4); a warp sums one group: lane l adds partial rows l, l+32, ...
+        // in order (five loads in flight at a time), then the 32 lane sums combine by butterfly.
+        const int ngroups = d / 4;
+        for (int q = cta + warp * n_ctas; q < ngroups; q += n_ctas * kConsWarps) {
+            float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
+            for (int rb = 0; rb < n_ctas; rb += 5 * kWarp) {
+                float4 v[5];
+#pragma unroll
+                for (int u = 0; u < 5; ++u) {
+                    const int r = rb + u * kWarp + lane;
+                    v[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+                    if (r < n_ctas) v[u] = __ldcg(reinterpret_cast<const float4 *>(part + (size_t)r * d) + q);
+                }
+#pragma unroll
+                for (int u = 0; u < 5; ++u) {
+                    s.x += v[u].x; s.y += v[u].y; s.z += v[u].z; s.w += v[u].w;
+                }
+            }
+            s.x = warp_sum(s.x); s.y = warp_sum(s.y); s.z = warp_sum(s.z); s.w = warp_sum(s.w);
+            if (lane == 0) {
+                if (p.y_dtype == CLADA_F32)
+                    reinterpret_cast<float4 *>(yl)[q] = s;
+                else
+                    reinterpret_cast<uint2 *>(yl)[q] = pack4_16bit(p.y_dtype, s);
+            }
+        }
+    }
+    if (tid == 0) {
+        if (timed_out) {
+            if (p.status) atomicOr(p.status, CLADA_STATUS_TIMEOUT);
+        } else {
+            // The counters go back to zero for the next launch: the last CTA out resets them (every CTA has
+            // then seen its last barrier complete).
+            const unsigned left = atomicAdd(&p.ctrl->depart, 1u);
+            if (left == (unsigned)n_ctas - 1u) {
+                p.ctrl->arrive = 0;
+                p.ctrl->depart = 0;
+                __threadfence();
+            }
+        }
+    }
+}
+
+// ---- host side ------------------------------------------------------------------------------
+
+// Ring stages and dynamic shared memory of a launch; n_stages < GS means the kernel cannot take the layer
+// (a reduction group holds GS stages at once; the x stage is handed back before the group starts).
+static void stack_smem_plan(const DeviceInfo &di, int d_model, int d_ff, int dtype, bool gated, int *n_stages,
+                            int *list_cap, size_t *smem, size_t *budget) {
+    const size_t stage_bytes = (gated ? 3 : 2) * (size_t)d_model * elem_size(dtype);
+    *list_cap = d_ff / di.num_sms + 2;
+    const size_t tail = (2 * kMaxStages + 4) * sizeof(uint64_t) + 2 * (size_t)*list_cap * sizeof(int);
+    *budget = (size_t)di.max_smem_optin - 2048;  // leave room for the static arrays
+    int n = *budget > tail ? (int)((*budget - tail) / stage_bytes) : 0;
+    if (n > kMaxStages) n = kMaxStages;
+    *n_stages = n;
+    *smem = (size_t)n * stage_bytes + tail;
+}
+
+template <typename T, int NV, bool GATED>
+static int launch_stack_variant(const StackParams &p, const StackLayers &lay, int dtype, cudaStream_t st) {
+    static bool configured[64] = {};
+    DeviceInfo di;
+    int rc = device_info(&di);
+    if (rc != CLADA_OK) return rc;
+    auto kern = sparse_ffn_stack_kernel<T, NV, GATED>;
+    int n_stages, list_cap;
+    size_t smem, budget;
+    stack_smem_plan(di, p.d_model, p.d_ff, dtype, GATED, &n_stages, &list_cap, &smem, &budget);
+    if (n_stages < GS) return CLADA_ERR_UNSUPPORTED;
+    if (!configured[di.device & 63]) {
+        CLADA_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)budget));
+        configured[di.device & 63] = true;
+    }
+    StackParams params = p;
+    StackLayers layers = lay;
+    int stages_arg = n_stages, cap_arg = list_cap;
+    void *args[] = {&params, &layers, &stages_arg, &cap_arg};
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(di.num_sms);  // one CTA per SM
+    cfg.blockDim = dim3(kFfnThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeCooperative;  // all CTAs co-resident: the grid barriers cannot starve
+    attr[0].val.cooperative = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 2;
+    CLADA_CUDA_TRY(cudaLaunchKernelExC(&cfg, reinterpret_cast<const void *>(kern), args));
+    return CLADA_OK;
+}
+
+template <typename T>
+static int launch_stack_typed(const StackParams &p, const StackLayers &lay, int dtype, cudaStream_t st) {
+    constexpr int E = Elem<T>::kPerVec;
+    const int vpr = p.d_model / E;
+    const bool gated = act_is_gated(p.act);
+    if (vpr <= kConsumers)
+        return gated ? launch_stack_variant<T, 1, true>(p, lay, dtype, st)
+                     : launch_stack_variant<T, 1, false>(p, lay, dtype, st);
+    if (vpr <= 2 * kConsumers)
+        return gated ? launch_stack_variant<T, 2, true>(p, lay, dtype, st)
+                     : launch_stack_variant<T, 2, false>(p, lay, dtype, st);
+    return CLADA_ERR_UNSUPPORTED;
+}
+
+bool ffn_stack_supported(const clada_layer *layers, int L, int B, size_t ws_bytes) {
+    if (B != 1 || L < 2) return false;
+    if (layers[0].d_ff > kStackMaxBatches * kWarp * kConsumers) return false;
+    for (int l = 1; l < L; ++l)
+        if (layers[l].activation != layers[0].activation) return false;
+    DeviceInfo di;
+    if (device_info(&di) != CLADA_OK) return false;
+    int n_stages, list_cap;
+    size_t smem, budget;
+    stack_smem_plan(di, layers[0].d_model, layers[0].d_ff, layers[0].dtype, act_is_gated(layers[0].activation), &n_stages,
+                    &list_cap, &smem, &budget);
+    if (n_stages < GS) return false;
+    return ws_bytes >= kWsCtrlBytes + 2 * (size_t)di.num_sms * layers[0].d_model * sizeof(float);
+}
+
+// One sequence through L validated layers of one shape, dtype and FFN form: launches of up to
+// kMaxStackLayers layers each.  Strides in bytes (x, y) and elements (tau).
+int launch_ffn_stack(const clada_layer *layers, int L, const void *x, size_t x_stride, const float *scores,
+                     const float *tau, long long tau_stride, void *y, size_t y_stride, int y_dtype, void *ws,
+                     int32_t *status, cudaStream_t st) {
+    for (int l0 = 0; l0 < L; l0 += kMaxStackLayers) {
+        const int n = L - l0 < kMaxStackLayers ? L - l0 : kMaxStackLayers;
+        StackLayers lay = {};
+        for (int l = 0; l < n; ++l) {
+            lay.w[l][0] = layers[l0 + l].w_gate;
+            lay.w[l][1] = layers[l0 + l].w_up;
+            lay.w[l][2] = layers[l0 + l].w_down_t;
+        }
+        StackParams p;
+        p.x = static_cast<const char *>(x) + (size_t)l0 * x_stride;
+        p.x_stride = x_stride;
+        p.scores = scores + (size_t)l0 * layers[0].d_ff;
+        p.tau = tau + (size_t)l0 * tau_stride;
+        p.tau_stride = tau_stride;
+        p.y = static_cast<char *>(y) + (size_t)l0 * y_stride;
+        p.y_stride = y_stride;
+        p.y_dtype = y_dtype;
+        p.partials = reinterpret_cast<float *>(static_cast<char *>(ws) + kWsCtrlBytes);
+        p.ctrl = static_cast<WsCtrl *>(ws);
+        p.status = status;
+        p.d_model = layers[0].d_model;
+        p.d_ff = layers[0].d_ff;
+        p.L = n;
+        p.act = layers[0].activation;
+        const int rc = layers[0].dtype == CLADA_F32    ? launch_stack_typed<float>(p, lay, CLADA_F32, st)
+                       : layers[0].dtype == CLADA_BF16 ? launch_stack_typed<__nv_bfloat16>(p, lay, CLADA_BF16, st)
+                                                       : launch_stack_typed<__half>(p, lay, CLADA_F16, st);
+        if (rc != CLADA_OK) return rc;
+    }
+    return CLADA_OK;
+}
+
+}  // namespace clada

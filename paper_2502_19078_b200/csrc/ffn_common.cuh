@@ -160,4 +160,12 @@ int ffn_batch_tile(const clada_layer *layer, int remaining);
 int launch_ffn_batch(const clada_layer *layer, int bt, const void *x, const float *scores, const float *tau,
                      long long tau_stride, void *y, int y_dtype, void *ws, int32_t *status, cudaStream_t st);
 
+// One sequence through a stack of layers in one persistent launch (clada_ffn_stack.cu): whether the stack
+// kernel takes this call (one sequence, at least two layers of one FFN form, a workspace with two partial
+// rows per SM), and the launch (x / y strides in bytes, tau stride in elements).
+bool ffn_stack_supported(const clada_layer *layers, int L, int B, size_t ws_bytes);
+int launch_ffn_stack(const clada_layer *layers, int L, const void *x, size_t x_stride, const float *scores,
+                     const float *tau, long long tau_stride, void *y, size_t y_stride, int y_dtype, void *ws,
+                     int32_t *status, cudaStream_t st);
+
 }  // namespace clada

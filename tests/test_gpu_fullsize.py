@@ -6,8 +6,12 @@ The oracle cannot redo a whole stack in fp64, so at full size it checks
   * the sparse FFN output on whole tokens, with scores drawn by the shared generator (both sides then take
     the same keep decisions by construction), for sampled sequences of a batch;
   * cognitive load and threshold adjustment on every row of a step;
-and, on the Llama-2-7B-shaped layer that the benchmark times, the complete chain (prefix statistics of the
-512-token prompt -> calibrated threshold -> guard band -> masks at the four threshold levels -> FFN outputs).
+and the complete chain at full width (prefix statistics of whole prompts -> calibrated threshold -> guard band ->
+masks at the four threshold levels -> FFN outputs, the oracle scoring ALL neurons): on the Llama-2-7B-shaped layer
+that the benchmark times (512 tokens), on a layer of the 32-layer stack (2048 tokens), on two sequences of the
+batch of 8 (14336 neurons, 1024 tokens, tiles of 4 sequences) and on the shortest and the longest prompt of the
+ragged batch of 16 (5120 x 13824, up to 4096 tokens, tiles of 2) -- each with the paper's coefficients and with a
+small pair under which every level keeps thousands of neurons.
 Inputs are drawn on the GPU by the shared generator and copied bit for bit to the oracle's side.
 """
 import numpy as np
@@ -204,6 +208,111 @@ def test_c5_batch16_ragged(clada, oracle):
     for rho in (0.30, 0.60):
         _ffn_synthetic_scores(clada, oracle, w, 2, seqs=[3], n_steps=1, rho=rho)
     _cogload_all_rows(clada, oracle, w, n_steps=1)
+
+
+def _fp32_levels(lam, gam):
+    """The four multipliers Eq. final_threshold can produce, formed as the adjustment forms them (fp32, left to
+    right): level = I(s > tau_s) + 2 I(H > tau_H)."""
+    one, lam, gam = np.float32(1.0), np.float32(lam), np.float32(gam)
+    return [one, one + lam, one + gam, (one + lam) + gam]
+
+
+def _full_chain(clada, oracle, w, layer_idx, seqs, rho, coeffs, n_tokens=1):
+    """Prefix statistics -> calibrated threshold -> guard band -> the masks at the four threshold levels -> FFN
+    outputs, on a whole batch of prompts at full width, compared with the oracle on the sequences `seqs`: the
+    oracle scores ALL d_ff neurons of those prompts.  `coeffs` lists (lambda, gamma) pairs; each pair gets its own
+    guard band and its own four levels.  Returns the numbers of excused neurons and of kept neurons seen."""
+    lengths = wl.prefix_lengths(w)
+    off = wl.seq_offsets(lengths)
+    B, F = len(lengths), w.d_ff
+    layer, weights = _layer_on_gpu(clada, w, layer_idx)
+    W_in, V_in, W_out = (wl.to_numpy_bits(weights[k]) for k in ("w_gate", "w_up", "w_down"))
+    scale = wl.channel_scale(w, "cuda")
+    X = torch.cat([wl.hidden_states(w, layer_idx, "prefix", b, n, "cuda", scale) for b, n in enumerate(lengths)])
+    xs = torch.stack([wl.hidden_states(w, layer_idx, "decode", b, n_tokens, "cuda", scale) for b in range(B)], dim=1)
+    ws = clada.new_workspace(layer, B, off[-1])
+    scores = torch.empty(B, F, dtype=torch.float32, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    clada.clada_prefix_scores(layer, X, off, scores, ws, status)
+    tau_base = torch.empty(B, dtype=torch.float32, device="cuda")
+    clada.clada_tau_from_sparsity(scores, rho, tau_base)
+    torch.cuda.synchronize()
+    A_gpu = scores.cpu().numpy().astype(np.float64)
+    A_or = {}
+    for b in seqs:
+        A_or[b] = oracle.neuron_scores(wl.to_numpy_bits(X[off[b]:off[b + 1]]), [0, lengths[b]], W_in, V_in, W_out)[0]
+        assert np.max(np.abs(A_gpu[b] - A_or[b]) / A_or[b]) <= SCORE_TOL, (w.name, layer_idx, b)
+    tb = tau_base.cpu().numpy()
+    mask = torch.empty(B, F, dtype=torch.uint8, device="cuda")
+    idx = torch.empty(B, F, dtype=torch.int32, device="cuda")
+    count = torch.empty(B, dtype=torch.int32, device="cuda")
+    y = torch.empty(B, w.d_model, dtype=torch.float32, device="cuda")
+    excused_total, kept_seen = 0, []
+    for lam, gam in coeffs:
+        levels = _fp32_levels(lam, gam)
+        clada.clada_prefix_select(layer, X, off, tau_base, [float(m) for m in levels], scores, mask, idx, count, ws,
+                                  status)
+        torch.cuda.synchronize()
+        for b in seqs:   # baseline masks of the prefill phase
+            e, m = compare_masks(mask[b].cpu().numpy(), A_or[b], float(tb[b]))
+            assert m == 0, (w.name, layer_idx, b, "baseline")
+            excused_total += e
+            n = int(count[b])
+            np.testing.assert_array_equal(idx[b, :n].cpu().numpy(), np.nonzero(mask[b].cpu().numpy())[0])
+        for k, mult in enumerate(levels):
+            tau_k = (tb * mult).astype(np.float32)           # one fp32 product, as the adjustment forms it
+            t = k % n_tokens
+            clada.clada_sparse_ffn_decode(layer, xs[t].contiguous(), scores, torch.from_numpy(tau_k).cuda(), 1, y, ws,
+                                          mask, None, count, status)
+            torch.cuda.synchronize()
+            for b in seqs:
+                m_gpu = mask[b].cpu().numpy()
+                e, m = compare_masks(m_gpu, A_or[b], float(tau_k[b]))
+                assert m == 0, (w.name, layer_idx, b, lam, gam, k)
+                excused_total += e
+                assert int(count[b]) == int(m_gpu.sum())
+                kept_seen.append(int(count[b]))
+                if e == 0:
+                    y_or, _, n_or = oracle.sparse_ffn(wl.to_numpy_bits(xs[t, b]), W_in, V_in, W_out, A_or[b],
+                                                      float(tau_k[b]))
+                    assert n_or == int(count[b])
+                    if n_or:
+                        assert rel_inf(y[b].cpu().numpy(), y_or) <= FFN_TOL_F32, (w.name, layer_idx, b, lam, gam, k)
+    assert int(status.item()) == 0
+    print(f"{w.name} layer {layer_idx}: sequences {list(seqs)}, excused neurons {excused_total}, "
+          f"kept counts {sorted(set(kept_seen))}")
+    return excused_total, kept_seen
+
+
+# The paper's coefficients (0.80 / 0.12), under which the raised thresholds cut nearly everything on these
+# synthetic layers, and a small pair under which all four levels keep thousands of neurons.
+CHAIN_COEFFS = [(0.80, 0.12), (0.02, 0.01)]
+
+
+def test_c3_full_chain_2048_tokens(clada, oracle):
+    """One layer of the 32-layer stack workload: all 11008 neurons scored by the oracle over the 2048-token prompt."""
+    w = wl.WORKLOADS["c3_llama2_7b_stack"]
+    _, kept = _full_chain(clada, oracle, w, 15, seqs=[0], rho=0.40, coeffs=CHAIN_COEFFS, n_tokens=2)
+    assert max(kept) == w.d_ff - w.k_cut(0.40) or abs(max(kept) - (w.d_ff - w.k_cut(0.40))) <= 2
+    assert sum(1 for k in kept if k > 1000) >= 5
+
+
+def test_c4_full_chain_two_sequences_of_the_batch(clada, oracle):
+    """Batch of 8 prompts of 1024 tokens on the 14336-neuron layer; the tile kernel's masks and outputs for two of
+    its sequences (one from each tile of 4) against the oracle's scores of all neurons."""
+    w = wl.WORKLOADS["c4_llama3_8b_b8"]
+    _, kept = _full_chain(clada, oracle, w, 1, seqs=[1, 6], rho=0.40, coeffs=CHAIN_COEFFS)
+    assert sum(1 for k in kept if k > 1000) >= 10
+
+
+def test_c5_full_chain_shortest_and_longest_prompt(clada, oracle):
+    """Batch of 16 ragged prompts on the 5120 x 13824 layer (tiles of 2 sequences): the shortest and the longest
+    prompt (up to 4096 tokens) against the oracle's scores of all neurons."""
+    w = wl.WORKLOADS["c5_13b_b16"]
+    lengths = wl.prefix_lengths(w)
+    shortest, longest = int(np.argmin(lengths)), int(np.argmax(lengths))
+    _, kept = _full_chain(clada, oracle, w, 2, seqs=[shortest, longest], rho=0.30, coeffs=CHAIN_COEFFS)
+    assert sum(1 for k in kept if k > 1000) >= 10
 
 
 def test_c2_threshold_search_full_width(clada, oracle):
