@@ -6,17 +6,18 @@
 // A launch per layer pays, per layer, for what does not move weight bytes: the launch ramp, the score
 // test, the first rows' latency, the slowest CTA's tail, a grid barrier and the column sums.  Here the
 // weight stream never stops at a layer boundary.  One cooperative CTA per SM, as in the per-layer kernel:
+//   scanner   one warp builds the kept lists: it tests a layer's scores against its threshold and writes
+//             this CTA's equal share of the kept neurons into one of four list buffers, up to four layers
+//             ahead of the layer being streamed, so the score test is never on anybody's path.
 //   producer  one thread walks layer after layer: the layer's x (one ring stage), then the three rows of
 //             every kept neuron of this CTA's share, as bulk asynchronous copies into the ring.  It runs
 //             ahead of the consumers by the ring's depth, across layer boundaries.
 //   consumers 512 threads.  Per layer: x from its stage into registers, the share's neurons four per
-//             CTA-wide reduction, the CTA's partial y to global memory, ARRIVE at the grid barrier, then
-//             -- while the other CTAs arrive -- the score test and the share list of layer l + 2, then
-//             WAIT at the barrier and sum a slice of columns over all CTAs' partials in CTA order.
-//             All of this takes the consumers less time than the ring holds rows for, so the copies
-//             into the ring go on while they are away from it.
-// Kept lists are built two layers ahead in a double buffer, partial rows are double buffered by barrier
-// number, every wait is bounded, and the summation order is fixed: results repeat bit for bit.
+//             CTA-wide reduction, the CTA's partial y to global memory, a grid barrier, then a slice of
+//             columns summed over all CTAs' partials in CTA order.  While they are at the barrier the
+//             copies of the next layer's rows go on into the ring.
+// Partial rows are double buffered by barrier number, every wait is bounded, and the summation order is
+// that of the per-layer kernel: results repeat bit for bit and equal the per-layer call's.
 #include <math.h>
 
 #include "common.cuh"
@@ -25,7 +26,7 @@
 namespace clada {
 
 constexpr int kMaxStackLayers = 128;  // layers per launch (their weight pointers travel as kernel parameters)
-constexpr int kStackMaxBatches = 4;   // score-test batches: d_ff <= 4 * 32 * kConsumers
+constexpr int kStackMaxDff = 65536;    // the scanner parks one keep word per 32 neurons in shared memory
 constexpr int GS = 4;                 // neurons per CTA-wide reduction
 
 struct StackLayers {
@@ -48,99 +49,107 @@ struct StackParams {
     int act;
 };
 
+// Tracing build (-DCLADA_STACK_TRACE, off by default): every CTA records %globaltimer stamps per layer into a
+// caller-provided device buffer [n_ctas][L][kTraceSlots] set with clada_stack_trace_buffer().  Slots: 0 layer
+// start (x in registers), 1 rows consumed, 2 arrived at the barrier, 3 unused, 4 barrier passed,
+// 5 column sums written, 6 producer's first copy of the layer, 7 its last, 8 ns the producer waited for free
+// stages, 9 ns consumer thread 0 waited for full stages.
+#ifdef CLADA_STACK_TRACE
+constexpr int kTraceSlots = 10;
+__device__ unsigned long long *g_stack_trace = nullptr;
+__device__ __forceinline__ unsigned long long trace_now() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
+}
+#define STACK_TRACE(l, slot, value)                                                                   \
+    do {                                                                                              \
+        if (g_stack_trace) g_stack_trace[((size_t)blockIdx.x * p.L + (l)) * kTraceSlots + (slot)] = (value); \
+    } while (0)
+#else
+#define STACK_TRACE(l, slot, value) \
+    do {                            \
+    } while (0)
+#endif
+
 __device__ __forceinline__ int stack_split_at(int n, int c, int n_ctas) {
     return (int)(((unsigned)n * (unsigned)c) / (unsigned)n_ctas);
 }
 
 __device__ __forceinline__ void consumer_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kConsumers) : "memory"); }
 
-// Score test of one layer by the 512 consumer threads: keep bits A_j >= tau (one ballot per 32-neuron
-// chunk, coalesced loads), block-wide ranks, and this CTA's equal share [r0, r1) of the kept neurons in
-// ascending order written to list[].  Returns the layer's kept count; *my_n = r1 - r0.
-__device__ __forceinline__ int build_share_list(const float *__restrict__ scores, const float tau, const int F,
-                                                const int cta, const int n_ctas, int *list, int *s_wtot,
-                                                int *my_n, const uint64_t keep_policy) {
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+constexpr int kStackThreads = kConsumers + 96;  // consumers + producer warp + scanner warp + epilogue warp
+constexpr int kScanWarp = kConsWarps + 1;
+constexpr int kEpiWarp = kConsWarps + 2;
+constexpr int kListBufs = 4;                    // kept lists are built up to four layers ahead
+
+// Score test of one layer by ONE warp (the scanner): keep bits A_j >= tau, one ballot per 32-neuron chunk with
+// coalesced loads (32 chunks = 1024 neurons per round, all loads of a round in flight together), the chunk words
+// parked in keep[]; then the ranks again from the parked words, and this CTA's equal share [r0, r1) of the kept
+// neurons, ascending, written to list[].  Returns the layer's kept count; *my_n = r1 - r0.
+__device__ __forceinline__ int scan_share_list(const float *__restrict__ scores, const float tau, const int F,
+                                               const int cta, const int n_ctas, int *list, unsigned *keep,
+                                               int *my_n, const uint64_t keep_policy) {
+    const int lane = threadIdx.x & 31;
     const int chunks = (F + kWarp - 1) / kWarp;
-    const int n_batches = (chunks + kConsumers - 1) / kConsumers;
     const float kNoNeuron = __int_as_float(0x7fc00000);  // NaN: no threshold keeps a position past d_ff
-    unsigned bal[kStackMaxBatches];
-    int first_rank[kStackMaxBatches];
     int n_act = 0;
+    for (int q0 = 0; q0 < chunks; q0 += kWarp) {
+        const bool whole = q0 + kWarp <= chunks && (q0 + kWarp) * kWarp <= F;
+        float v[kWarp];
+        if (whole) {
+            const float *src = scores + (size_t)q0 * kWarp + lane;
 #pragma unroll
-    for (int bt = 0; bt < kStackMaxBatches; ++bt) {
-        bal[bt] = 0u;
-        first_rank[bt] = 0;
-        if (bt >= n_batches) continue;  // uniform
-        const int q0 = bt * kConsumers + warp * kWarp;  // the warp's first chunk of this batch
-        if (q0 < chunks) {
-            const bool whole = q0 + kWarp <= chunks && (q0 + kWarp) * kWarp <= F;
+            for (int c = 0; c < kWarp; ++c) v[c] = ld_keep(src + c * kWarp, keep_policy);
+        } else {
 #pragma unroll
-            for (int c0 = 0; c0 < kWarp; c0 += 8) {  // eight loads in flight per lane
-                float v[8];
-                if (whole) {
-                    const float *src = scores + (size_t)(q0 + c0) * kWarp + lane;
-#pragma unroll
-                    for (int c = 0; c < 8; ++c) v[c] = ld_keep(src + c * kWarp, keep_policy);
-                } else {
-#pragma unroll
-                    for (int c = 0; c < 8; ++c) {
-                        const int j = (q0 + c0 + c) * kWarp + lane;
-                        v[c] = (q0 + c0 + c < chunks && j < F) ? ld_keep(scores + j, keep_policy) : kNoNeuron;
-                    }
-                }
-#pragma unroll
-                for (int c = 0; c < 8; ++c) {
-                    const unsigned w = __ballot_sync(0xffffffffu, v[c] >= tau);
-                    if (lane == c0 + c) bal[bt] = w;  // lane c keeps the word of chunk q0 + c
-                }
+            for (int c = 0; c < kWarp; ++c) {
+                const int j = (q0 + c) * kWarp + lane;
+                v[c] = (q0 + c < chunks && j < F) ? ld_keep(scores + j, keep_policy) : kNoNeuron;
             }
         }
-        const int cnt = __popc(bal[bt]);
+        unsigned mine = 0u;
+#pragma unroll
+        for (int c = 0; c < kWarp; ++c) {
+            const unsigned w = __ballot_sync(0xffffffffu, v[c] >= tau);
+            if (lane == c) mine = w;  // lane c keeps the word of chunk q0 + c
+        }
+        if (q0 + lane < chunks) keep[q0 + lane] = mine;
+        n_act += __popc(mine);
+    }
+    n_act = warp_sum(n_act);
+    __syncwarp();
+    const int r0 = stack_split_at(n_act, cta, n_ctas);
+    const int r1 = stack_split_at(n_act, cta + 1, n_ctas);
+    int base = 0;
+    for (int q0 = 0; q0 < chunks && base < r1; q0 += kWarp) {
+        const unsigned w = q0 + lane < chunks ? keep[q0 + lane] : 0u;
+        const int cnt = __popc(w);
         int incl = cnt;
 #pragma unroll
         for (int o = 1; o < kWarp; o <<= 1) {
             const int t = __shfl_up_sync(0xffffffffu, incl, o);
             if (lane >= o) incl += t;
         }
-        consumer_sync();  // s_wtot free again (also orders the previous user of list[] before the writes below)
-        if (lane == kWarp - 1) s_wtot[warp] = incl;
-        consumer_sync();
-        int wbase = 0, btot = 0;
-#pragma unroll
-        for (int w = 0; w < kConsWarps; ++w) {
-            const int v = s_wtot[w];
-            wbase += (w < warp) ? v : 0;
-            btot += v;
+        const int fr = base + incl - cnt;  // rank of this chunk's first kept neuron
+        if (fr < r1 && fr + cnt > r0) {    // at most a few chunks hold the share: their lanes walk the bits
+            unsigned rest = w;
+            int rank = fr;
+            while (rest) {
+                const int b = __ffs(rest) - 1;
+                rest &= rest - 1;
+                if (rank >= r0 && rank < r1) list[rank - r0] = (q0 + lane) * kWarp + b;
+                ++rank;
+            }
         }
-        first_rank[bt] = n_act + wbase + incl - cnt;
-        n_act += btot;
-    }
-    const int r0 = stack_split_at(n_act, cta, n_ctas);
-    const int r1 = stack_split_at(n_act, cta + 1, n_ctas);
-#pragma unroll
-    for (int bt = 0; bt < kStackMaxBatches; ++bt) {
-        if (bt >= n_batches) continue;  // uniform
-        const int q = bt * kConsumers + tid;
-        const int fr = first_rank[bt];
-        const bool in_share = q < chunks && fr < r1 && fr + __popc(bal[bt]) > r0;
-        unsigned todo = __ballot_sync(0xffffffffu, in_share);
-        while (todo) {
-            const int t = __ffs(todo) - 1;
-            todo &= todo - 1;
-            const unsigned wb = __shfl_sync(0xffffffffu, bal[bt], t);
-            const int wfr = __shfl_sync(0xffffffffu, fr, t);
-            const int j = (bt * kConsumers + (warp * kWarp + t)) * kWarp + lane;
-            const int rank = wfr + __popc(wb & ((1u << lane) - 1u));
-            if (((wb >> lane) & 1u) && rank >= r0 && rank < r1) list[rank - r0] = j;
-        }
+        base += __shfl_sync(0xffffffffu, incl, kWarp - 1);
     }
     *my_n = r1 - r0;
     return n_act;
 }
 
 template <typename T, int NV, bool GATED>
-__global__ void __launch_bounds__(kFfnThreads, 1)
+__global__ void __launch_bounds__(kStackThreads, 1)
 sparse_ffn_stack_kernel(const StackParams p, const __grid_constant__ StackLayers lay, const int n_stages,
                         const int list_cap) {
     constexpr int E = Elem<T>::kPerVec;
@@ -155,17 +164,19 @@ sparse_ffn_stack_kernel(const StackParams p, const __grid_constant__ StackLayers
     const uint32_t stage_bytes = kRows * row_bytes;
     const uint32_t down_off = (kRows - 1u) * row_bytes;
 
-    // dynamic shared memory: ring | full[kMaxStages] | empty[kMaxStages] | list-ready[2] | list-done[2] |
-    // lists[2][list_cap]
+    // dynamic shared memory: ring | full[kMaxStages] | empty[kMaxStages] | list-ready[4] | list-free[4] |
+    // lists[4][list_cap] | keep words of the layer being scanned
     const uint32_t ring = smem_u32(smem_raw);
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem_raw + (size_t)n_stages * stage_bytes);
     const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + kMaxStages);
-    const uint32_t lbar0 = smem_u32(bars + 2 * kMaxStages);      // consumers -> producer: the list of a layer is written
-    const uint32_t pbar0 = smem_u32(bars + 2 * kMaxStages + 2);  // producer -> consumers: done with that list
-    int *s_list = reinterpret_cast<int *>(bars + 2 * kMaxStages + 4);
-    __shared__ int s_wtot[kConsWarps];
-    __shared__ int s_nact[2], s_myn[2];  // per list buffer: the layer's kept count, this CTA's share
-    __shared__ int s_ok;
+    const uint32_t lready0 = smem_u32(bars + 2 * kMaxStages);             // scanner -> producer, consumers
+    const uint32_t lfree0 = smem_u32(bars + 2 * kMaxStages + kListBufs);  // producer, consumers, epilogue -> scanner
+    const uint32_t pdone = smem_u32(bars + 2 * kMaxStages + 2 * kListBufs);      // consumers -> epilogue: partial row stored
+    const uint32_t bdone = smem_u32(bars + 2 * kMaxStages + 2 * kListBufs + 1);  // epilogue -> consumers: barrier passed
+    int *s_list = reinterpret_cast<int *>(bars + 2 * kMaxStages + 2 * kListBufs + 2);
+    unsigned *s_keep = reinterpret_cast<unsigned *>(s_list + kListBufs * list_cap);
+    __shared__ int s_nact[kListBufs], s_myn[kListBufs];  // per list buffer: the layer's kept count, this CTA's share
+    __shared__ int s_cur[2][3];                          // consumers' copy for the current layer (+ give-up flag)
     __shared__ __align__(16) float s_dot[2][2 * GS][kConsWarps];
 
     pdl_launch_dependents();
@@ -174,16 +185,136 @@ sparse_ffn_stack_kernel(const StackParams p, const __grid_constant__ StackLayers
             mbar_init(full0 + 8 * s, 1);            // the producer's expect_tx arrival
             mbar_init(empty0 + 8 * s, kConsWarps);  // one arrival per consumer warp
         }
-        mbar_init(lbar0, 1);
-        mbar_init(lbar0 + 8, 1);
-        mbar_init(pbar0, 1);
-        mbar_init(pbar0 + 8, 1);
+        for (int k = 0; k < kListBufs; ++k) {
+            mbar_init(lready0 + 8 * k, 1);  // the scanner
+            mbar_init(lfree0 + 8 * k, 3);   // the producer, consumer thread 0 and the epilogue warp
+        }
+        mbar_init(pdone, kConsWarps);
+        mbar_init(bdone, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     pdl_wait();      // everything below may read what the previous kernel wrote
     __syncthreads();  // the mbarriers exist
 
     bool timed_out = false;
+
+    if (warp == kScanWarp) {
+        // ---- scanner: the kept list of every layer, up to four layers ahead of its use --------------------
+        const uint64_t keep_policy = policy_evict_last();
+        for (int l = 0; l < L; ++l) {
+            const int k = l & (kListBufs - 1);
+            // buffer k last held layer l - 4: the producer has issued its rows, the consumers have its counts
+            if (l >= kListBufs && !mbar_wait(lfree0 + 8 * k, (uint32_t)((l >> 2) - 1) & 1u)) {
+                timed_out = true;
+                break;
+            }
+            const float tau = ld_keep(p.tau + (size_t)l * p.tau_stride, keep_policy);
+            int my_n;
+            const int n_act = scan_share_list(p.scores + (size_t)l * F, tau, F, cta, n_ctas, s_list + k * list_cap,
+                                              s_keep, &my_n, keep_policy);
+            if (lane == 0) {
+                s_nact[k] = n_act;
+                s_myn[k] = my_n;
+            }
+            __syncwarp();  // every lane's list entries are written before lane 0 announces them
+            if (lane == 0) mbar_arrive(lready0 + 8 * k);
+        }
+        if (timed_out && lane == 0 && p.status) atomicOr(p.status, CLADA_STATUS_TIMEOUT);
+        return;
+    }
+
+    if (warp == kEpiWarp) {
+        // ---- epilogue warp: grid barrier and column sums of every layer, off the consumers' path ----------
+        // Per layer that kept something (barrier number e): wait until this CTA's consumers have stored their
+        // partial row, arrive at the device-wide count, wait for every CTA, tell the consumers (who may then
+        // reuse the other partial buffer), and sum this CTA's slice of columns over all partial rows in CTA
+        // order.  A layer that kept nothing gets its zeros from here.
+        unsigned epoch = 0;
+        const int ngroups = d / 4;
+        for (int l = 0; l < L; ++l) {
+            const int k = l & (kListBufs - 1);
+            if (!timed_out && !mbar_wait(lready0 + 8 * k, (uint32_t)(l >> 2) & 1u)) timed_out = true;
+            const int n_act = timed_out ? 0 : s_nact[k];
+            __syncwarp();
+            if (lane == 0) mbar_arrive(lfree0 + 8 * k);
+            char *yl = p.y + (size_t)l * p.y_stride;
+            if (n_act == 0) {
+                const int q0 = stack_split_at(ngroups, cta, n_ctas), q1 = stack_split_at(ngroups, cta + 1, n_ctas);
+                for (int q = q0 + lane; q < q1; q += kWarp) {
+                    if (p.y_dtype == CLADA_F32)
+                        reinterpret_cast<float4 *>(yl)[q] = make_float4(0.f, 0.f, 0.f, 0.f);
+                    else
+                        reinterpret_cast<uint2 *>(yl)[q] = make_uint2(0u, 0u);
+                }
+                continue;
+            }
+            if (!timed_out && !mbar_wait(pdone, epoch & 1u)) timed_out = true;
+            int ok = 1;
+            if (lane == 0) {
+                // release at device scope: the consumers' row (ordered before this by their arrivals on the
+                // shared-memory barrier) is visible to whoever sees the count
+                asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(&p.ctrl->arrive) : "memory");
+                STACK_TRACE(l, 2, trace_now());
+                const unsigned target = (epoch + 1u) * (unsigned)n_ctas;
+                unsigned spins = 0, seen;
+                for (;;) {
+                    asm volatile("ld.acquire.gpu.u32 %0, [%1];" : "=r"(seen) : "l"(&p.ctrl->arrive) : "memory");
+                    if (seen >= target) break;
+                    if (timed_out || ++spins > kBarrierSpinLimit) {
+                        ok = 0;
+                        break;
+                    }
+                }
+                STACK_TRACE(l, 4, trace_now());
+            }
+            ok = __shfl_sync(0xffffffffu, ok, 0);
+            if (!ok) timed_out = true;
+            if (lane == 0) mbar_arrive(bdone);  // every CTA has arrived: all column sums of the layer before are done
+            const float *part = p.partials + (size_t)(epoch & 1u) * n_ctas * d;
+            ++epoch;
+            // columns in groups of 4 (float4): lane l adds partial rows l, l+32, ... in order (five loads in
+            // flight at a time), then the 32 lane sums combine by butterfly.
+            for (int q = cta; q < ngroups; q += n_ctas) {
+                float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
+                for (int rb = 0; rb < n_ctas; rb += 5 * kWarp) {
+                    float4 v[5];
+#pragma unroll
+                    for (int u = 0; u < 5; ++u) {
+                        const int r = rb + u * kWarp + lane;
+                        v[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+                        if (r < n_ctas) v[u] = __ldcg(reinterpret_cast<const float4 *>(part + (size_t)r * d) + q);
+                    }
+#pragma unroll
+                    for (int u = 0; u < 5; ++u) {
+                        s.x += v[u].x; s.y += v[u].y; s.z += v[u].z; s.w += v[u].w;
+                    }
+                }
+                s.x = warp_sum(s.x); s.y = warp_sum(s.y); s.z = warp_sum(s.z); s.w = warp_sum(s.w);
+                if (lane == 0) {
+                    if (p.y_dtype == CLADA_F32)
+                        reinterpret_cast<float4 *>(yl)[q] = s;
+                    else
+                        reinterpret_cast<uint2 *>(yl)[q] = pack4_16bit(p.y_dtype, s);
+                }
+            }
+            if (lane == 0) STACK_TRACE(l, 5, trace_now());
+        }
+        if (lane == 0) {
+            if (timed_out) {
+                if (p.status) atomicOr(p.status, CLADA_STATUS_TIMEOUT);
+            } else {
+                // The counters go back to zero for the next launch: the last CTA out resets them (every CTA
+                // has then seen its last barrier complete).
+                const unsigned left = atomicAdd(&p.ctrl->depart, 1u);
+                if (left == (unsigned)n_ctas - 1u) {
+                    p.ctrl->arrive = 0;
+                    p.ctrl->depart = 0;
+                    __threadfence();
+                }
+            }
+        }
+        return;
+    }
 
     if (warp == kConsWarps) {
         // ---- producer -----------------------------------------------------------------------------
@@ -194,25 +325,35 @@ sparse_ffn_stack_kernel(const StackParams p, const __grid_constant__ StackLayers
             int s = 0;  // ring position and the parity of its current use, kept incrementally
             uint32_t par = 0;
             for (int l = 0; l < L && !timed_out; ++l) {
-                const int lb = l & 1;
-                if (!mbar_wait(lbar0 + 8 * lb, (uint32_t)(l >> 1) & 1u)) {  // layer l's list is in buffer lb
+                const int k = l & (kListBufs - 1);
+                if (!mbar_wait(lready0 + 8 * k, (uint32_t)(l >> 2) & 1u)) {  // layer l's list is in buffer k
                     timed_out = true;
                     break;
                 }
-                const int my_n = s_myn[lb];
-                if (s_nact[lb] == 0 || my_n == 0) {  // nothing of this layer for this CTA
-                    mbar_arrive(pbar0 + 8 * lb);
+                const int my_n = s_myn[k];
+                if (s_nact[k] == 0 || my_n == 0) {  // nothing of this layer for this CTA
+                    mbar_arrive(lfree0 + 8 * k);
                     continue;
                 }
-                const int *list = s_list + lb * list_cap;
+                const int *list = s_list + k * list_cap;
                 const char *Wg = static_cast<const char *>(lay.w[l][0]);
                 const char *Wu = static_cast<const char *>(lay.w[l][1]);
                 const char *Wd = static_cast<const char *>(lay.w[l][2]);
+#ifdef CLADA_STACK_TRACE
+                unsigned long long waited = 0;
+#endif
                 for (int i = -1; i < my_n; ++i) {  // i = -1: the layer's x takes a stage of its own
+#ifdef CLADA_STACK_TRACE
+                    const unsigned long long w0 = trace_now();
+#endif
                     if (!mbar_wait(empty0 + 8 * s, par ^ 1)) {  // a fresh barrier passes parity 1 at once
                         timed_out = true;
                         break;
                     }
+#ifdef CLADA_STACK_TRACE
+                    waited += trace_now() - w0;
+                    if (i == -1) STACK_TRACE(l, 6, trace_now());
+#endif
                     const uint32_t dst = ring + (uint32_t)s * stage_bytes, bar = full0 + 8 * s;
                     if (i < 0) {
                         mbar_expect_tx(bar, row_bytes);
@@ -230,7 +371,11 @@ sparse_ffn_stack_kernel(const StackParams p, const __grid_constant__ StackLayers
                         par ^= 1;
                     }
                 }
-                if (!timed_out) mbar_arrive(pbar0 + 8 * lb);  // buffer lb may take the list of layer l + 2
+#ifdef CLADA_STACK_TRACE
+                STACK_TRACE(l, 7, trace_now());
+                STACK_TRACE(l, 8, waited);
+#endif
+                if (!timed_out) mbar_arrive(lfree0 + 8 * k);  // the list has been read to its end
             }
             // Never leave with copies in flight: the last use of every stage must have landed.
             const long long first = issued > n_stages ? issued - n_stages : 0;
@@ -242,254 +387,172 @@ sparse_ffn_stack_kernel(const StackParams p, const __grid_constant__ StackLayers
     }
 
     // ---- consumers ------------------------------------------------------------------------------------
-    const uint64_t keep_policy = policy_evict_last();
     bool vok[NV];
 #pragma unroll
     for (int i = 0; i < NV; ++i) vok[i] = tid + i * kConsumers < vpr;
-
-    // The lists of layers 0 and 1 come first; from then on the list of layer l + 2 is built inside layer l.
-    for (int l = 0; l < 2 && l < L; ++l) {
-        const float tau = ld_keep(p.tau + (size_t)l * p.tau_stride, keep_policy);
-        int my_n;
-        const int n_act = build_share_list(p.scores + (size_t)l * F, tau, F, cta, n_ctas, s_list + l * list_cap,
-                                           s_wtot, &my_n, keep_policy);
-        if (tid == 0) {
-            s_nact[l] = n_act;
-            s_myn[l] = my_n;
-        }
-        consumer_sync();  // the list and its counts are written
-        if (tid == 0) mbar_arrive(lbar0 + 8 * l);
-    }
-
     const bool b16 = lane & 16, b8 = lane & 8, b4 = lane & 4;
     int cs = 0;  // ring position of the next stage to consume, and the parity of its use
     uint32_t cpar = 0;
     unsigned epoch = 0;  // grid barriers passed so far (layers that kept something)
     for (int l = 0; l < L; ++l) {
-        const int lb = l & 1;
-        const int n_act = s_nact[lb], my_n = s_myn[lb];
-        char *yl = p.y + (size_t)l * p.y_stride;
-        float next_tau = 0.f;
-        if (l + 2 < L) next_tau = ld_keep(p.tau + (size_t)(l + 2) * p.tau_stride, keep_policy);  // used after the layer
-        if (n_act > 0) {
-            // x of this thread's columns, from the stage the producer filled ahead of the layer's rows
-            float2 xr[NV][P];
+        // Thread 0 takes the layer's counts from the scanner's buffer and hands them (and whether it gave up
+        // waiting) to the others, so that all consumers take the same path through the layer.
+        if (tid == 0) {
+            const int k = l & (kListBufs - 1);
+            if (!timed_out && !mbar_wait(lready0 + 8 * k, (uint32_t)(l >> 2) & 1u)) timed_out = true;
+            s_cur[l & 1][0] = timed_out ? 0 : s_nact[k];
+            s_cur[l & 1][1] = timed_out ? 0 : s_myn[k];
+            s_cur[l & 1][2] = timed_out ? 1 : 0;
+            mbar_arrive(lfree0 + 8 * k);  // the consumers are done with this buffer
+        }
+        consumer_sync();
+        const int n_act = s_cur[l & 1][0], my_n = s_cur[l & 1][1];
+        if (s_cur[l & 1][2]) timed_out = true;
+        if (n_act == 0) continue;  // nothing is kept (every CTA sees the same count): the epilogue warp writes y = 0
+        // x of this thread's columns, from the stage the producer filled ahead of the layer's rows
+        float2 xr[NV][P];
+#pragma unroll
+        for (int i = 0; i < NV; ++i)
+#pragma unroll
+            for (int e = 0; e < P; ++e) xr[i][e] = make_float2(0.f, 0.f);
+        if (my_n > 0) {
+            if (!timed_out && !mbar_wait(full0 + 8 * cs, cpar)) timed_out = true;
+            const uint32_t xa = ring + (uint32_t)cs * stage_bytes;
 #pragma unroll
             for (int i = 0; i < NV; ++i)
-#pragma unroll
-                for (int e = 0; e < P; ++e) xr[i][e] = make_float2(0.f, 0.f);
-            if (my_n > 0) {
-                if (!timed_out && !mbar_wait(full0 + 8 * cs, cpar)) timed_out = true;
-                const uint32_t xa = ring + (uint32_t)cs * stage_bytes;
-#pragma unroll
-                for (int i = 0; i < NV; ++i)
-                    if (vok[i]) Pairs<T>::unpack(lds128(xa + (uint32_t)(tid + i * kConsumers) * 16u), xr[i]);
-                __syncwarp();
-                if (lane == 0) mbar_arrive(empty0 + 8 * cs);
-                if (++cs == n_stages) {
-                    cs = 0;
-                    cpar ^= 1;
-                }
+                if (vok[i]) Pairs<T>::unpack(lds128(xa + (uint32_t)(tid + i * kConsumers) * 16u), xr[i]);
+            __syncwarp();
+            if (lane == 0) mbar_arrive(empty0 + 8 * cs);
+            if (++cs == n_stages) {
+                cs = 0;
+                cpar ^= 1;
             }
-            float2 acc[NV][P];
+        }
+        float2 acc[NV][P];
 #pragma unroll
-            for (int i = 0; i < NV; ++i)
+        for (int i = 0; i < NV; ++i)
 #pragma unroll
-                for (int e = 0; e < P; ++e) acc[i][e] = make_float2(0.f, 0.f);
-            int buf = 0;
-            for (int g0 = 0; g0 < my_n; g0 += GS, buf ^= 1) {
-                float pd[2 * GS];
-                uint32_t st_addr[GS];
-                int st_idx[GS];
+            for (int e = 0; e < P; ++e) acc[i][e] = make_float2(0.f, 0.f);
+#ifdef CLADA_STACK_TRACE
+        unsigned long long cwait = 0;
+        if (tid == 0) STACK_TRACE(l, 0, trace_now());
+#endif
+        int buf = 0;
+        for (int g0 = 0; g0 < my_n; g0 += GS, buf ^= 1) {
+            float pd[2 * GS];
+            uint32_t st_addr[GS];
+            int st_idx[GS];
 #pragma unroll
-                for (int g = 0; g < GS; ++g) {
-                    const int i = g0 + g;
-                    float2 sg = make_float2(0.f, 0.f), su = make_float2(0.f, 0.f);
-                    st_idx[g] = cs;
-                    st_addr[g] = ring + (uint32_t)cs * stage_bytes;
-                    if (i < my_n) {
-                        if (!timed_out && !mbar_wait(full0 + 8 * cs, cpar)) timed_out = true;
-                        if (++cs == n_stages) {
-                            cs = 0;
-                            cpar ^= 1;
-                        }
-#pragma unroll
-                        for (int k = 0; k < NV; ++k) {
-                            if (!vok[k]) continue;
-                            const uint32_t a = st_addr[g] + (uint32_t)(tid + k * kConsumers) * 16u;
-                            float2 fg[P], fu[P];
-                            Pairs<T>::unpack(lds128(a), fg);
-                            if (GATED) Pairs<T>::unpack(lds128(a + row_bytes), fu);
-#pragma unroll
-                            for (int e = 0; e < P; ++e) {
-                                sg = __ffma2_rn(fg[e], xr[k][e], sg);
-                                if (GATED) su = __ffma2_rn(fu[e], xr[k][e], su);
-                            }
-                        }
+            for (int g = 0; g < GS; ++g) {
+                const int i = g0 + g;
+                float2 sg = make_float2(0.f, 0.f), su = make_float2(0.f, 0.f);
+                st_idx[g] = cs;
+                st_addr[g] = ring + (uint32_t)cs * stage_bytes;
+                if (i < my_n) {
+#ifdef CLADA_STACK_TRACE
+                    const unsigned long long w0 = trace_now();
+#endif
+                    if (!timed_out && !mbar_wait(full0 + 8 * cs, cpar)) timed_out = true;
+#ifdef CLADA_STACK_TRACE
+                    cwait += trace_now() - w0;
+#endif
+                    if (++cs == n_stages) {
+                        cs = 0;
+                        cpar ^= 1;
                     }
-                    pd[2 * g] = sg.x + sg.y;
-                    pd[2 * g + 1] = su.x + su.y;
-                }
-                // Warp sums of the 8 values by a halving butterfly (9 shuffles): after it every lane of
-                // quad q holds the warp total of value q.  Fixed order, so results repeat bit for bit.
-                float b[4], c[2], v8;
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const float send = b16 ? pd[i] : pd[i + 4];
-                    b[i] = (b16 ? pd[i + 4] : pd[i]) + __shfl_xor_sync(0xffffffffu, send, 16);
-                }
-#pragma unroll
-                for (int i = 0; i < 2; ++i) {
-                    const float send = b8 ? b[i] : b[i + 2];
-                    c[i] = (b8 ? b[i + 2] : b[i]) + __shfl_xor_sync(0xffffffffu, send, 8);
-                }
-                v8 = (b4 ? c[1] : c[0]) + __shfl_xor_sync(0xffffffffu, b4 ? c[0] : c[1], 4);
-                v8 += __shfl_xor_sync(0xffffffffu, v8, 2);
-                v8 += __shfl_xor_sync(0xffffffffu, v8, 1);
-                // lane 4q holds value index: bit4 -> +4, bit3 -> +2, bit2 -> +1
-                if ((lane & 3) == 0) s_dot[buf][(b16 ? 4 : 0) + (b8 ? 2 : 0) + (b4 ? 1 : 0)][warp] = v8;
-                consumer_sync();
-                // Cross-warp sums: lane l adds 4 consecutive warps of value l/4, the quad finishes by
-                // butterfly; then gate lanes form the neuron value h.
-                float tot;
-                {
-                    const float4 q4 = *reinterpret_cast<const float4 *>(&s_dot[buf][lane >> 2][(lane & 3) * 4]);
-                    tot = (q4.x + q4.y) + (q4.z + q4.w);
-                    tot += __shfl_xor_sync(0xffffffffu, tot, 1);
-                    tot += __shfl_xor_sync(0xffffffffu, tot, 2);
-                }
-                const float up = __shfl_xor_sync(0xffffffffu, tot, 4);  // value 2g+1 sits 4 lanes above value 2g
-                const float hval = neuron_value_f(p.act, tot, up);      // meaningful on lanes 8g..8g+3
-#pragma unroll
-                for (int g = 0; g < GS; ++g) {
-                    const float h = __shfl_sync(0xffffffffu, hval, 8 * g);
-                    if (g0 + g >= my_n) continue;
-                    const float2 h2 = make_float2(h, h);
 #pragma unroll
                     for (int k = 0; k < NV; ++k) {
                         if (!vok[k]) continue;
-                        float2 fd[P];
-                        Pairs<T>::unpack(lds128(st_addr[g] + down_off + (uint32_t)(tid + k * kConsumers) * 16u), fd);
+                        const uint32_t a = st_addr[g] + (uint32_t)(tid + k * kConsumers) * 16u;
+                        float2 fg[P], fu[P];
+                        Pairs<T>::unpack(lds128(a), fg);
+                        if (GATED) Pairs<T>::unpack(lds128(a + row_bytes), fu);
 #pragma unroll
-                        for (int e = 0; e < P; ++e) acc[k][e] = __ffma2_rn(h2, fd[e], acc[k][e]);
+                        for (int e = 0; e < P; ++e) {
+                            sg = __ffma2_rn(fg[e], xr[k][e], sg);
+                            if (GATED) su = __ffma2_rn(fu[e], xr[k][e], su);
+                        }
                     }
                 }
-                // hand the stages back to the producer
-                __syncwarp();
-                if (lane == 0) {
+                pd[2 * g] = sg.x + sg.y;
+                pd[2 * g + 1] = su.x + su.y;
+            }
+            // Warp sums of the 8 values by a halving butterfly (9 shuffles): after it every lane of
+            // quad q holds the warp total of value q.  Fixed order, so results repeat bit for bit.
+            float b[4], c[2], v8;
 #pragma unroll
-                    for (int g = 0; g < GS; ++g)
-                        if (g0 + g < my_n) mbar_arrive(empty0 + 8 * st_idx[g]);
-                }
+            for (int i = 0; i < 4; ++i) {
+                const float send = b16 ? pd[i] : pd[i + 4];
+                b[i] = (b16 ? pd[i + 4] : pd[i]) + __shfl_xor_sync(0xffffffffu, send, 16);
             }
-            // partial y of this CTA, into the buffer of this barrier number
-            float *mine = p.partials + ((size_t)(epoch & 1u) * n_ctas + cta) * d;
 #pragma unroll
-            for (int i = 0; i < NV; ++i) {
-                if (!vok[i]) continue;
-                float4 *dst = reinterpret_cast<float4 *>(mine + (size_t)(tid + i * kConsumers) * E);
-#pragma unroll
-                for (int e = 0; e < P; e += 2)
-                    dst[e / 2] = make_float4(acc[i][e].x, acc[i][e].y, acc[i][e + 1].x, acc[i][e + 1].y);
+            for (int i = 0; i < 2; ++i) {
+                const float send = b8 ? b[i] : b[i + 2];
+                c[i] = (b8 ? b[i + 2] : b[i]) + __shfl_xor_sync(0xffffffffu, send, 8);
             }
-            consumer_sync();  // every consumer's part of the row is written
-            if (tid == 0) {   // arrive; the wait comes after the next list
-                __threadfence();
-                atomicAdd(&p.ctrl->arrive, 1u);
-            }
-        }
-
-        // ---- the list of layer l + 2 replaces layer l's (its rows have all been consumed) ----------------
-        if (l + 2 < L) {
-            // The producer has read this buffer's counts (it may not have if the layer gave it nothing to copy).
-            if (!timed_out && !mbar_wait(pbar0 + 8 * lb, (uint32_t)(l >> 1) & 1u)) timed_out = true;
-            int nn;
-            const int na = build_share_list(p.scores + (size_t)(l + 2) * F, next_tau, F, cta, n_ctas,
-                                            s_list + lb * list_cap, s_wtot, &nn, keep_policy);
-            consumer_sync();  // everyone has read s_nact / s_myn of layer l, and the list is written
-            if (tid == 0) {
-                s_nact[lb] = na;
-                s_myn[lb] = nn;
-            }
+            v8 = (b4 ? c[1] : c[0]) + __shfl_xor_sync(0xffffffffu, b4 ? c[0] : c[1], 4);
+            v8 += __shfl_xor_sync(0xffffffffu, v8, 2);
+            v8 += __shfl_xor_sync(0xffffffffu, v8, 1);
+            // lane 4q holds value index: bit4 -> +4, bit3 -> +2, bit2 -> +1
+            if ((lane & 3) == 0) s_dot[buf][(b16 ? 4 : 0) + (b8 ? 2 : 0) + (b4 ? 1 : 0)][warp] = v8;
             consumer_sync();
-            if (tid == 0) mbar_arrive(lbar0 + 8 * lb);
-        }
-
-        if (n_act == 0) {
-            // Nothing is kept (every CTA sees the same count): y = 0, written slice by slice; no partial
-            // sums exist, so this layer has no grid barrier.
-            const int ng = d / 4;
-            const int q0 = stack_split_at(ng, cta, n_ctas), q1 = stack_split_at(ng, cta + 1, n_ctas);
-            for (int q = q0 + tid; q < q1; q += kConsumers) {
-                if (p.y_dtype == CLADA_F32)
-                    reinterpret_cast<float4 *>(yl)[q] = make_float4(0.f, 0.f, 0.f, 0.f);
-                else
-                    reinterpret_cast<uint2 *>(yl)[q] = make_uint2(0u, 0u);
+            // Cross-warp sums: lane l adds 4 consecutive warps of value l/4, the quad finishes by
+            // butterfly; then gate lanes form the neuron value h.
+            float tot;
+            {
+                const float4 q4 = *reinterpret_cast<const float4 *>(&s_dot[buf][lane >> 2][(lane & 3) * 4]);
+                tot = (q4.x + q4.y) + (q4.z + q4.w);
+                tot += __shfl_xor_sync(0xffffffffu, tot, 1);
+                tot += __shfl_xor_sync(0xffffffffu, tot, 2);
             }
-            continue;
-        }
-
-        // ---- wait for every CTA's partial row of this layer, then the column sums ------------------------
-        if (tid == 0) {
-            const unsigned target = (epoch + 1u) * (unsigned)n_ctas;
-            unsigned spins = 0, seen;
-            int ok = 1;
-            for (;;) {
-                asm volatile("ld.acquire.gpu.u32 %0, [%1];" : "=r"(seen) : "l"(&p.ctrl->arrive) : "memory");
-                if (seen >= target) break;
-                if (timed_out || ++spins > kBarrierSpinLimit) {
-                    ok = 0;
-                    break;
-                }
-            }
-            s_ok = ok;
-        }
-        consumer_sync();
-        if (s_ok == 0) timed_out = true;
-        consumer_sync();  // s_ok is free for the next layer
-        const float *part = p.partials + (size_t)(epoch & 1u) * n_ctas * d;
-        ++epoch;
-        // columns in groups of 4 (float4); a warp sums one group: lane l adds partial rows l, l+32, ...
-        // in order (five loads in flight at a time), then the 32 lane sums combine by butterfly.
-        const int ngroups = d / 4;
-        for (int q = cta + warp * n_ctas; q < ngroups; q += n_ctas * kConsWarps) {
-            float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
-            for (int rb = 0; rb < n_ctas; rb += 5 * kWarp) {
-                float4 v[5];
+            const float up = __shfl_xor_sync(0xffffffffu, tot, 4);  // value 2g+1 sits 4 lanes above value 2g
+            const float hval = neuron_value_f(p.act, tot, up);      // meaningful on lanes 8g..8g+3
 #pragma unroll
-                for (int u = 0; u < 5; ++u) {
-                    const int r = rb + u * kWarp + lane;
-                    v[u] = make_float4(0.f, 0.f, 0.f, 0.f);
-                    if (r < n_ctas) v[u] = __ldcg(reinterpret_cast<const float4 *>(part + (size_t)r * d) + q);
-                }
+            for (int g = 0; g < GS; ++g) {
+                const float h = __shfl_sync(0xffffffffu, hval, 8 * g);
+                if (g0 + g >= my_n) continue;
+                const float2 h2 = make_float2(h, h);
 #pragma unroll
-                for (int u = 0; u < 5; ++u) {
-                    s.x += v[u].x; s.y += v[u].y; s.z += v[u].z; s.w += v[u].w;
+                for (int k = 0; k < NV; ++k) {
+                    if (!vok[k]) continue;
+                    float2 fd[P];
+                    Pairs<T>::unpack(lds128(st_addr[g] + down_off + (uint32_t)(tid + k * kConsumers) * 16u), fd);
+#pragma unroll
+                    for (int e = 0; e < P; ++e) acc[k][e] = __ffma2_rn(h2, fd[e], acc[k][e]);
                 }
             }
-            s.x = warp_sum(s.x); s.y = warp_sum(s.y); s.z = warp_sum(s.z); s.w = warp_sum(s.w);
+            // hand the stages back to the producer
+            __syncwarp();
             if (lane == 0) {
-                if (p.y_dtype == CLADA_F32)
-                    reinterpret_cast<float4 *>(yl)[q] = s;
-                else
-                    reinterpret_cast<uint2 *>(yl)[q] = pack4_16bit(p.y_dtype, s);
+#pragma unroll
+                for (int g = 0; g < GS; ++g)
+                    if (g0 + g < my_n) mbar_arrive(empty0 + 8 * st_idx[g]);
             }
         }
-    }
-    if (tid == 0) {
-        if (timed_out) {
-            if (p.status) atomicOr(p.status, CLADA_STATUS_TIMEOUT);
-        } else {
-            // The counters go back to zero for the next launch: the last CTA out resets them (every CTA has
-            // then seen its last barrier complete).
-            const unsigned left = atomicAdd(&p.ctrl->depart, 1u);
-            if (left == (unsigned)n_ctas - 1u) {
-                p.ctrl->arrive = 0;
-                p.ctrl->depart = 0;
-                __threadfence();
-            }
+#ifdef CLADA_STACK_TRACE
+        if (tid == 0) {
+            STACK_TRACE(l, 1, trace_now());
+            STACK_TRACE(l, 9, cwait);
         }
+#endif
+        // Partial y of this CTA, into the buffer of this barrier number.  The buffer was last read for the
+        // column sums of the barrier two back; all of those are done once every CTA has passed the barrier
+        // before this one, which the epilogue warp reports.
+        if (epoch >= 1u && !timed_out && !mbar_wait(bdone, (epoch - 1u) & 1u)) timed_out = true;
+        float *mine = p.partials + ((size_t)(epoch & 1u) * n_ctas + cta) * d;
+        ++epoch;
+#pragma unroll
+        for (int i = 0; i < NV; ++i) {
+            if (!vok[i]) continue;
+            float4 *dst = reinterpret_cast<float4 *>(mine + (size_t)(tid + i * kConsumers) * E);
+#pragma unroll
+            for (int e = 0; e < P; e += 2)
+                dst[e / 2] = make_float4(acc[i][e].x, acc[i][e].y, acc[i][e + 1].x, acc[i][e + 1].y);
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(pdone);  // this warp's part of the row is stored: on to the next layer
     }
+    if (timed_out && tid == 0 && p.status) atomicOr(p.status, CLADA_STATUS_TIMEOUT);
 }
 
 // ---- host side ------------------------------------------------------------------------------
@@ -500,7 +563,8 @@ static void stack_smem_plan(const DeviceInfo &di, int d_model, int d_ff, int dty
                             int *list_cap, size_t *smem, size_t *budget) {
     const size_t stage_bytes = (gated ? 3 : 2) * (size_t)d_model * elem_size(dtype);
     *list_cap = d_ff / di.num_sms + 2;
-    const size_t tail = (2 * kMaxStages + 4) * sizeof(uint64_t) + 2 * (size_t)*list_cap * sizeof(int);
+    const size_t tail = (2 * kMaxStages + 2 * kListBufs + 2) * sizeof(uint64_t) + kListBufs * (size_t)*list_cap * sizeof(int) +
+                        (size_t)((d_ff + 31) / 32) * sizeof(unsigned);
     *budget = (size_t)di.max_smem_optin - 2048;  // leave room for the static arrays
     int n = *budget > tail ? (int)((*budget - tail) / stage_bytes) : 0;
     if (n > kMaxStages) n = kMaxStages;
@@ -529,7 +593,7 @@ static int launch_stack_variant(const StackParams &p, const StackLayers &lay, in
     void *args[] = {&params, &layers, &stages_arg, &cap_arg};
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(di.num_sms);  // one CTA per SM
-    cfg.blockDim = dim3(kFfnThreads);
+    cfg.blockDim = dim3(kStackThreads);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = st;
     cudaLaunchAttribute attr[2];
@@ -559,7 +623,7 @@ static int launch_stack_typed(const StackParams &p, const StackLayers &lay, int 
 
 bool ffn_stack_supported(const clada_layer *layers, int L, int B, size_t ws_bytes) {
     if (B != 1 || L < 2) return false;
-    if (layers[0].d_ff > kStackMaxBatches * kWarp * kConsumers) return false;
+    if (layers[0].d_ff > kStackMaxDff) return false;
     for (int l = 1; l < L; ++l)
         if (layers[l].activation != layers[0].activation) return false;
     DeviceInfo di;
@@ -610,3 +674,11 @@ int launch_ffn_stack(const clada_layer *layers, int L, const void *x, size_t x_s
 }
 
 }  // namespace clada
+
+#ifdef CLADA_STACK_TRACE
+// Tracing build only: where the stack kernel writes its time stamps (NULL switches tracing off).
+extern "C" int clada_stack_trace_buffer(unsigned long long *buf) {
+    CLADA_CUDA_TRY(cudaMemcpyToSymbol(clada::g_stack_trace, &buf, sizeof buf));
+    return CLADA_OK;
+}
+#endif
