@@ -78,9 +78,11 @@ __device__ __forceinline__ int stack_split_at(int n, int c, int n_ctas) {
 
 __device__ __forceinline__ void consumer_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kConsumers) : "memory"); }
 
-constexpr int kStackThreads = kConsumers + 96;  // consumers + producer warp + scanner warp + epilogue warp
+constexpr int kEpiWarps = 2;
+constexpr int kStackThreads = kConsumers + 64 + kEpiWarps * kWarp;  // consumers, producer, scanner, epilogue warps
 constexpr int kScanWarp = kConsWarps + 1;
-constexpr int kEpiWarp = kConsWarps + 2;
+constexpr int kEpiWarp = kConsWarps + 2;  // first epilogue warp
+__device__ __forceinline__ void epilogue_sync() { asm volatile("bar.sync 2, %0;" ::"n"(kEpiWarps * kWarp) : "memory"); }
 constexpr int kListBufs = 4;                    // kept lists are built up to four layers ahead
 
 // Score test of one layer by ONE warp (the scanner): keep bits A_j >= tau, one ballot per 32-neuron chunk with
@@ -177,6 +179,7 @@ sparse_ffn_stack_kernel(const StackParams p, const __grid_constant__ StackLayers
     unsigned *s_keep = reinterpret_cast<unsigned *>(s_list + kListBufs * list_cap);
     __shared__ int s_nact[kListBufs], s_myn[kListBufs];  // per list buffer: the layer's kept count, this CTA's share
     __shared__ int s_cur[2][3];                          // consumers' copy for the current layer (+ give-up flag)
+    __shared__ int s_ecur[2][3];                         // the epilogue warps' copy
     __shared__ __align__(16) float s_dot[2][2 * GS][kConsWarps];
 
     pdl_launch_dependents();
@@ -223,24 +226,31 @@ sparse_ffn_stack_kernel(const StackParams p, const __grid_constant__ StackLayers
         return;
     }
 
-    if (warp == kEpiWarp) {
-        // ---- epilogue warp: grid barrier and column sums of every layer, off the consumers' path ----------
+    if (warp >= kEpiWarp) {
+        // ---- epilogue warps: grid barrier and column sums of every layer, off the consumers' path ----------
         // Per layer that kept something (barrier number e): wait until this CTA's consumers have stored their
         // partial row, arrive at the device-wide count, wait for every CTA, tell the consumers (who may then
         // reuse the other partial buffer), and sum this CTA's slice of columns over all partial rows in CTA
         // order.  A layer that kept nothing gets its zeros from here.
+        const int et = tid - kEpiWarp * kWarp, ew = warp - kEpiWarp;
         unsigned epoch = 0;
         const int ngroups = d / 4;
         for (int l = 0; l < L; ++l) {
-            const int k = l & (kListBufs - 1);
-            if (!timed_out && !mbar_wait(lready0 + 8 * k, (uint32_t)(l >> 2) & 1u)) timed_out = true;
-            const int n_act = timed_out ? 0 : s_nact[k];
-            __syncwarp();
-            if (lane == 0) mbar_arrive(lfree0 + 8 * k);
+            // the first epilogue thread takes the layer's kept count (and whether it gave up waiting) for all
+            if (et == 0) {
+                const int k = l & (kListBufs - 1);
+                if (!timed_out && !mbar_wait(lready0 + 8 * k, (uint32_t)(l >> 2) & 1u)) timed_out = true;
+                s_ecur[l & 1][0] = timed_out ? 0 : s_nact[k];
+                s_ecur[l & 1][1] = timed_out ? 1 : 0;
+                mbar_arrive(lfree0 + 8 * k);
+            }
+            epilogue_sync();
+            const int n_act = s_ecur[l & 1][0];
+            if (s_ecur[l & 1][1]) timed_out = true;
             char *yl = p.y + (size_t)l * p.y_stride;
             if (n_act == 0) {
                 const int q0 = stack_split_at(ngroups, cta, n_ctas), q1 = stack_split_at(ngroups, cta + 1, n_ctas);
-                for (int q = q0 + lane; q < q1; q += kWarp) {
+                for (int q = q0 + et; q < q1; q += kEpiWarps * kWarp) {
                     if (p.y_dtype == CLADA_F32)
                         reinterpret_cast<float4 *>(yl)[q] = make_float4(0.f, 0.f, 0.f, 0.f);
                     else
@@ -248,9 +258,8 @@ sparse_ffn_stack_kernel(const StackParams p, const __grid_constant__ StackLayers
                 }
                 continue;
             }
-            if (!timed_out && !mbar_wait(pdone, epoch & 1u)) timed_out = true;
-            int ok = 1;
-            if (lane == 0) {
+            if (et == 0) {
+                if (!timed_out && !mbar_wait(pdone, epoch & 1u)) timed_out = true;
                 // release at device scope: the consumers' row (ordered before this by their arrivals on the
                 // shared-memory barrier) is visible to whoever sees the count
                 asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(&p.ctrl->arrive) : "memory");
@@ -261,20 +270,21 @@ sparse_ffn_stack_kernel(const StackParams p, const __grid_constant__ StackLayers
                     asm volatile("ld.acquire.gpu.u32 %0, [%1];" : "=r"(seen) : "l"(&p.ctrl->arrive) : "memory");
                     if (seen >= target) break;
                     if (timed_out || ++spins > kBarrierSpinLimit) {
-                        ok = 0;
+                        timed_out = true;
                         break;
                     }
                 }
                 STACK_TRACE(l, 4, trace_now());
+                s_ecur[l & 1][2] = timed_out ? 1 : 0;
+                mbar_arrive(bdone);  // every CTA has arrived: all column sums of the layer before are done
             }
-            ok = __shfl_sync(0xffffffffu, ok, 0);
-            if (!ok) timed_out = true;
-            if (lane == 0) mbar_arrive(bdone);  // every CTA has arrived: all column sums of the layer before are done
+            epilogue_sync();
+            if (s_ecur[l & 1][2]) timed_out = true;
             const float *part = p.partials + (size_t)(epoch & 1u) * n_ctas * d;
             ++epoch;
-            // columns in groups of 4 (float4): lane l adds partial rows l, l+32, ... in order (five loads in
-            // flight at a time), then the 32 lane sums combine by butterfly.
-            for (int q = cta; q < ngroups; q += n_ctas) {
+            // columns in groups of 4 (float4), a warp per group: lane l adds partial rows l, l+32, ... in order
+            // (five loads in flight at a time), then the 32 lane sums combine by butterfly.
+            for (int q = cta + ew * n_ctas; q < ngroups; q += kEpiWarps * n_ctas) {
                 float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
                 for (int rb = 0; rb < n_ctas; rb += 5 * kWarp) {
                     float4 v[5];
@@ -297,9 +307,10 @@ sparse_ffn_stack_kernel(const StackParams p, const __grid_constant__ StackLayers
                         reinterpret_cast<uint2 *>(yl)[q] = pack4_16bit(p.y_dtype, s);
                 }
             }
-            if (lane == 0) STACK_TRACE(l, 5, trace_now());
+            if (et == 0) STACK_TRACE(l, 5, trace_now());
         }
-        if (lane == 0) {
+        epilogue_sync();  // every epilogue warp has read its last partial rows
+        if (et == 0) {
             if (timed_out) {
                 if (p.status) atomicOr(p.status, CLADA_STATUS_TIMEOUT);
             } else {
