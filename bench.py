@@ -8,13 +8,17 @@ One step = one pass of the whole path over one batch of synthetic input:
 The layer exists in several identical copies at different addresses and decode step t reads copy
 t mod n, so that no step can be served from L2 (one copy's kept rows are 135-162 MB, L2 is 126 MB).
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--no-graph] [--workload NAME]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--no-graph] [--workload NAME] [--no-info]
 
 Prints ONE JSON line (rank 0).  `--impl reference` times the CPU oracle on a bounded sample.
+Beside the step's throughput the line carries the FFN kernels timed alone (the per-layer launch the step uses, and
+the persistent launch that takes a whole stack of layers), each as the median of several samples taken while the
+clocks are being recorded, and -- unless --no-info -- the same figures on the other workloads' layers.
 """
 from __future__ import annotations
 
 import argparse
+import hashlib
 import json
 import os
 import subprocess
@@ -33,9 +37,41 @@ WORKLOAD = "c2_llama2_7b_layer"
 METRIC = "sparse_ffn_decode_tokens_per_s"
 LAMBDA, GAMMA = 0.80, 0.12
 N_COPIES = 4
-# DRAM read + write bytes of one sparse_ffn_kernel launch at the baseline threshold of this workload, from the ncu
-# capture summarised in profiles/sparse_ffn_kernel_c2_full.md.  Must go back to None whenever that kernel changes.
-FFN_NCU_TRAFFIC_BYTES = 166.0e6   # both captured launches: 162.47 MB read + 3.52 MB written
+STACK_PASSES = 32      # layer passes per persistent launch in the single-layer workloads' stack measurement
+PROFILES = os.path.join(ROOT, "profiles")
+CSRC = os.path.join(ROOT, "paper_2502_19078_b200", "csrc")
+# sources a kernel's code comes from: the DRAM traffic on record for it counts only while these are unchanged
+KERNEL_SOURCES = {
+    "sparse_ffn_kernel": ["clada_ffn.cu", "ffn_common.cuh", "common.cuh"],
+    "sparse_ffn_stack_kernel": ["clada_ffn_stack.cu", "ffn_common.cuh", "common.cuh"],
+}
+
+
+def sources_hash(kernel: str) -> str:
+    h = hashlib.sha256()
+    for name in KERNEL_SOURCES[kernel]:
+        with open(os.path.join(CSRC, name), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()
+
+
+def recorded_traffic(kernel: str, workload: str):
+    """DRAM read + write bytes per launch (or per layer pass) of `kernel` from the ncu capture on record under
+    profiles/ (written by paper_2502_19078_b200.ncu_summary), or None when there is no record for this workload
+    or the kernel's sources have changed since the counters were taken."""
+    path = os.path.join(PROFILES, f"traffic_{kernel}.txt")
+    try:
+        rec = {}
+        with open(path) as f:
+            for line in f:
+                if ":" in line and not line.startswith("#"):
+                    k, v = line.split(":", 1)
+                    rec[k.strip()] = v.strip()
+        if rec.get("workload") != workload or rec.get("sources_sha256") != sources_hash(kernel):
+            return None
+        return float(rec["dram_bytes_per_unit"])
+    except Exception:
+        return None
 
 
 def _peaks():
@@ -136,10 +172,15 @@ class Job:
         self.status = torch.zeros(1, dtype=torch.int32, device=dev)
         self.lam = torch.full((1,), LAMBDA, **f32)
         self.gam = torch.full((1,), GAMMA, **f32)
+        self.zero = torch.zeros(1, **f32)
         self.s = torch.empty(self.N, **f32)
         self.h = torch.empty(self.N, **f32)
         self.tau_final = torch.empty(1, 1, **f32)
         self.y = torch.empty(len(w.sparsities), self.N, w.d_model, **f32)
+        # the persistent stack launch on this layer: STACK_PASSES layer passes over the rotating copies
+        self.stack = clada.LayerStack([self.layers[i % N_COPIES] for i in range(STACK_PASSES)])
+        self.stack_scores = torch.empty(STACK_PASSES, 1, w.d_ff, **f32)
+        self.stack_tau = torch.empty(1, STACK_PASSES, **f32)
         self.guard = [1.0, 1.0 + LAMBDA, 1.0 + GAMMA, 1.0 + LAMBDA + GAMMA]
         # calibration (stands in for the offline threshold search; not part of a step)
         clada.clada_prefix_scores(self.layers[0], self.X, self.off, self.scores, self.ws)
@@ -183,16 +224,19 @@ class Job:
             self.clada.clada_sparse_ffn_decode_nested(self.layers[t % N_COPIES], self.xs[t:t + 1], self.order[0],
                                                       self.ncounts[0], self.level, self.y[0, t:t + 1], self.ws)
 
-    def step(self):
+    def step(self, adapt: bool = True):
+        """One pass of the whole path.  adapt=False runs it with lambda = gamma = 0 (the paper's ablation row
+        without semantic adaptation): every token then decodes at the configured baseline sparsity."""
         c, w = self.clada, self.w
         L0 = self.layers[0]
+        lam, gam = (self.lam, self.gam) if adapt else (self.zero, self.zero)
         c.clada_prefix_scores(L0, self.X, self.off, self.scores, self.ws, self.status)
         for r, rho in enumerate(w.sparsities):
             tb = self.tau_base[r]
             c.clada_refine_scores(L0, self.X, self.off, tb.view(1), self.guard, 1e-4, self.scores, self.ws, self.status)
             c.clada_select(self.scores, tb.view(1), 1, self.mask, self.idx, self.count)
             for t in range(self.N):
-                c.clada_cogload_adjust(self.logits[t:t + 1], self.tokens[t:t + 1], tb, self.lam, self.gam,
+                c.clada_cogload_adjust(self.logits[t:t + 1], self.tokens[t:t + 1], tb, lam, gam,
                                        self.tau_s, self.tau_H, self.s[t:t + 1], self.h[t:t + 1], self.tau_final,
                                        self.status)
                 c.clada_sparse_ffn_decode(self.layers[t % N_COPIES], self.xs[t:t + 1], self.scores, self.tau_final, 1,
@@ -238,6 +282,20 @@ class Job:
         for t in range(self.N):
             self.clada.clada_sparse_ffn_decode(self.layers[t % N_COPIES], self.xs[t:t + 1], self.scores,
                                                self.tau_base[r], 1, self.y[0, t:t + 1], self.ws)
+
+    stack_passes_per_loop = property(lambda self: (self.N // STACK_PASSES) * STACK_PASSES)
+
+    def stack_prepare(self, r: int = 0):
+        self.stack_scores.copy_(self.scores.expand(STACK_PASSES, 1, -1))
+        self.stack_tau.copy_(self.tau_base[r].expand(1, STACK_PASSES))
+
+    def ffn_stack_loop(self):
+        """The same layer passes (token t on copy t mod n, baseline threshold) through the persistent stack
+        launch: STACK_PASSES passes per launch (call stack_prepare first)."""
+        for t0 in range(0, self.stack_passes_per_loop, STACK_PASSES):
+            self.clada.clada_sparse_ffn_decode_layers(self.stack, self.xs[t0:t0 + STACK_PASSES].unsqueeze(1),
+                                                      self.stack_scores, self.stack_tau,
+                                                      self.y[0, t0:t0 + STACK_PASSES].unsqueeze(1), self.ws)
 
 
 class StackJob:
@@ -307,7 +365,7 @@ class StackJob:
 
     @property
     def launches_per_step(self) -> int:
-        return self.L * 7 + self.N * (1 + self.L)
+        return self.L * 7 + self.N * 2      # per token: cogload+adjust, one persistent FFN launch
 
     def tokens_per_step(self) -> int:
         return self.N
@@ -332,10 +390,19 @@ class StackJob:
     def io_tensors(self):
         return [self.X, self.xs, self.logits, self.tokens], self.y
 
+    ffn_kernel = "sparse_ffn_stack_kernel (one launch = all layers of a token)"
+
     def ffn_only_loop(self):
-        """Eight tokens x 32 layers at the baseline thresholds."""
+        """Eight tokens x 32 layers at the baseline thresholds: one persistent launch per token."""
         for t in range(8):
             self.clada.clada_sparse_ffn_decode_layers(self.stack, self.xs[t], self.scores, self.tau_base, self.y[t], self.ws)
+
+    def ffn_per_layer_loop(self):
+        """The same passes as one launch per layer."""
+        for t in range(8):
+            for l in range(self.L):
+                self.clada.clada_sparse_ffn_decode(self.layers[l], self.xs[t, l], self.scores[l], self.tau_base[:, l],
+                                                   self.L, self.y[t, l], self.ws)
 
 
 class BatchJob:
@@ -449,6 +516,27 @@ class BatchJob:
                                                self.y[t], self.ws)
 
 
+FFN_INNER = 12      # replays per sample of an FFN-only loop (a sample lasts 40-60 ms; seven samples per figure)
+
+
+def _graphed(fn, stream, use_graph):
+    """fn run once to warm up, then (with use_graph) captured; returns the callable to time."""
+    fn()
+    if not use_graph:
+        return fn
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=stream):
+        fn()
+    g.replay()
+    return g.replay
+
+
+def _median_ms(run, inner=1, repeats=7):
+    """Median over `repeats` samples of the device time of one run (each sample times `inner` runs)."""
+    samples = sorted(_timed(run, inner, lambda: None) / inner for _ in range(repeats))
+    return samples[len(samples) // 2]
+
+
 def _timed(fn, steps, dist_barrier):
     start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     dist_barrier()
@@ -460,6 +548,39 @@ def _timed(fn, steps, dist_barrier):
     torch.cuda.synchronize()
     dist_barrier()
     return start.elapsed_time(end)
+
+
+def other_workloads_info(clada, dev, stream, use_graph, peak, read_gbs):
+    """FFN-only figures on the other workloads' layers, for information: the 32-layer stack (eight tokens, one
+    persistent launch per token, and the same passes as one launch per layer) and one layer of each batched
+    workload (the batch's call = its tiles of sequences, bytes = the union of each tile's kept rows)."""
+    out = {}
+    for name in ("c3_llama2_7b_stack", "c4_llama3_8b_b8", "c5_13b_b16"):
+        w = wl.WORKLOADS[name]
+        job = (BatchJob if w.batch > 1 else StackJob)(clada, w, dev, 0)
+        t_ms = _median_ms(_graphed(job.ffn_only_loop, stream, use_graph), inner=3) / job.ffn_launches_per_loop
+        kept = w.d_ff - w.k_cut(w.sparsities[0])
+        if w.batch > 1:
+            nbytes = job.ffn_bytes_per_launch
+            rec = {"kernel": job.ffn_kernel, "layers_run": 1, "batch": w.batch, "tile": job.tile,
+                   "sparsity": w.sparsities[0], "us_per_batch_call": t_ms * 1e3, "bytes_per_batch_call": nbytes,
+                   "union_rows": job.union_rows}
+        else:
+            nbytes = kept * 3 * w.d_model * w.elem_bytes + w.d_ff * 4 + w.d_model * w.elem_bytes + w.d_model * 4
+            t_layer = _median_ms(_graphed(job.ffn_per_layer_loop, stream, use_graph), inner=3) / job.ffn_launches_per_loop
+            rec = {"kernel": "sparse_ffn_stack_kernel", "layers": job.L, "sparsity": w.sparsities[0], "kept_neurons": kept,
+                   "us_per_layer_pass": t_ms * 1e3, "bytes_per_layer_pass": nbytes,
+                   "ffn_only_tokens_per_s": 1.0 / (t_ms * 1e-3 * job.L),
+                   "per_layer_launch": {"kernel": "sparse_ffn_kernel", "us_per_launch": t_layer * 1e3,
+                                        "achieved": nbytes / (t_layer * 1e-3) / 1e9,
+                                        "frac": nbytes / (t_layer * 1e-3) / 1e9 / peak}}
+        gbs = nbytes / (t_ms * 1e-3) / 1e9
+        rec.update({"achieved": gbs, "unit": "GB/s", "frac": gbs / peak, "frac_of_read_only_stream": gbs / read_gbs,
+                    "device_status_word": int(job.status.item())})
+        out[name] = rec
+        del job
+        torch.cuda.empty_cache()
+    return out
 
 
 def run_ours(args):
@@ -507,29 +628,34 @@ def run_ours(args):
         ms = _timed(run, args.steps, barrier)
         clocks = sampler.stop() if rank == 0 else None
 
-        # the FFN kernel alone, same launches, for the roofline
-        ffn_run = job.ffn_only_loop
-        job.ffn_only_loop()
-        if args.graph:
-            ffn_graph = torch.cuda.CUDAGraph()
-            with torch.cuda.graph(ffn_graph, stream=stream):
-                job.ffn_only_loop()
-            ffn_run = ffn_graph.replay
-        ffn_run()
-        ffn_ms = _timed(ffn_run, 5, lambda: None) / (5 * job.ffn_launches_per_loop)
-        # the same for the other sparsity levels of the workload (single-layer job only)
-        other_ffn_ms = []
+        # the step without semantic adaptation (lambda = gamma = 0): every token at the configured sparsity
+        base_ms = None
         if isinstance(job, Job):
-            for r in range(1, len(w.sparsities)):
-                fr = (lambda rr: (lambda: job.ffn_only_loop(rr)))(r)
-                fr()
-                if args.graph:
-                    og = torch.cuda.CUDAGraph()
-                    with torch.cuda.graph(og, stream=stream):
-                        fr()
-                    fr = og.replay
-                fr()
-                other_ffn_ms.append(_timed(fr, 5, lambda: None) / (5 * job.ffn_launches_per_loop))
+            base_run = _graphed(lambda: job.step(adapt=False), stream, args.graph)
+            for _ in range(2):
+                base_run()
+            base_ms = _timed(base_run, args.steps, barrier)
+
+        # The FFN kernels alone, for the roofline: the same launches back to back at the baseline threshold,
+        # median of several samples, all inside one recorded window of the clocks.
+        roof_sampler = ClockSampler(local)
+        if rank == 0:
+            roof_sampler.start()
+        n_sp = len(w.sparsities) if isinstance(job, Job) else 1
+        ffn_ms, stack_ms = [], []
+        for r in range(n_sp):
+            fr = _graphed((lambda rr: (lambda: job.ffn_only_loop(rr)))(r) if isinstance(job, Job) else job.ffn_only_loop,
+                          stream, args.graph)
+            ffn_ms.append(_median_ms(fr, inner=FFN_INNER) / job.ffn_launches_per_loop)
+            if hasattr(job, "ffn_stack_loop"):
+                job.stack_prepare(r)
+                sr = _graphed(job.ffn_stack_loop, stream, args.graph)
+                stack_ms.append(_median_ms(sr, inner=FFN_INNER) / job.stack_passes_per_loop)
+        per_layer_ms = None
+        if hasattr(job, "ffn_per_layer_loop"):
+            pr = _graphed(job.ffn_per_layer_loop, stream, args.graph)
+            per_layer_ms = _median_ms(pr, inner=FFN_INNER) / job.ffn_launches_per_loop
+        roof_clocks = roof_sampler.stop() if rank == 0 else None
         # read-only streaming bandwidth of this machine (the peak file's figure is a read + write copy)
         probe = torch.empty(1 << 30, dtype=torch.uint8, device=dev)
         probe.zero_()
@@ -580,8 +706,11 @@ def run_ours(args):
                     job.ffn_only_loop_nested()
                 nf_run = nf_graph.replay
             nf_run()
-            nested_ffn_ms = _timed(nf_run, 5, lambda: None) / (5 * job.ffn_launches_per_loop)
+            nested_ffn_ms = _median_ms(nf_run, inner=FFN_INNER) / job.ffn_launches_per_loop
         status = int(job.status.item())
+        info = None
+        if rank == 0 and world == 1 and w.name == WORKLOAD and args.info:
+            info = other_workloads_info(clada, dev, stream, args.graph, _peaks()[0], read_gbs)
 
     # every rank ran its own sequence; the job's rate is all ranks' tokens over the slowest rank's time
     tokens_rank = job.tokens_per_step() * args.steps
@@ -590,6 +719,9 @@ def run_ours(args):
     nested_value = None
     if nested_ms is not None:
         nested_value, nested_ms = sharding.whole_job_rate(tokens_rank, nested_ms, dev)
+    base_value = None
+    if base_ms is not None:
+        base_value, base_ms = sharding.whole_job_rate(tokens_rank, base_ms, dev)
 
     peak, peak_kind = _peaks()
     prefix_flop = job.prefix_flop
@@ -600,47 +732,83 @@ def run_ours(args):
     except Exception:
         bf16_peak, bf16_kind = 1590.0, "fallback"
     eb = w.elem_bytes
-    # algorithmic bytes of one FFN launch: three rows per kept neuron (two without a gate projection)
+    # algorithmic bytes of one FFN layer pass: three rows per kept neuron (two without a gate projection)
     # + scores + x in + y out
     rows = 2 if w.activation == 2 else 3
-    ffn_bytes = kept_base * rows * w.d_model * eb + w.d_ff * 4 + w.d_model * eb + w.d_model * 4
-    if hasattr(job, "ffn_bytes_per_launch"):  # a batch: the union of each tile's kept rows
-        ffn_bytes = job.ffn_bytes_per_launch
-    achieved = ffn_bytes / (ffn_ms * 1e-3) / 1e9
+
+    def pass_bytes(kept_neurons):
+        return kept_neurons * rows * w.d_model * eb + w.d_ff * 4 + w.d_model * eb + w.d_model * 4
+
+    def figures(nbytes, t_ms):
+        gbs = nbytes / (t_ms * 1e-3) / 1e9
+        return {"achieved": gbs, "frac": gbs / peak, "frac_of_read_only_stream": gbs / read_gbs}
+
+    ffn_bytes = job.ffn_bytes_per_launch if hasattr(job, "ffn_bytes_per_launch") else pass_bytes(kept_base)
+    sample_note = f"median of 7 samples of {FFN_INNER} replays of the loop's CUDA graph, clocks recorded over all of them"
+    per_launch = {"kernel": "sparse_ffn_kernel", "call": "clada_sparse_ffn_decode: one launch per layer pass",
+                  **figures(ffn_bytes, ffn_ms[0]), "bytes_per_launch": ffn_bytes, "us_per_launch": ffn_ms[0] * 1e3,
+                  "kept_neurons": kept_base, "traffic": recorded_traffic("sparse_ffn_kernel", w.name)}
+    if isinstance(job, Job):
+        per_launch["by_sparsity"] = [
+            {"sparsity": w.sparsities[r], "kept_neurons": w.d_ff - w.k_cut(w.sparsities[r]), "us_per_launch": t * 1e3,
+             **figures(pass_bytes(w.d_ff - w.k_cut(w.sparsities[r])), t)} for r, t in enumerate(ffn_ms)]
+    common = {"bound": "hbm", "peak": peak, "unit": "GB/s", "peak_kind": peak_kind, "read_only_stream_gbs": read_gbs,
+              "samples": sample_note, "clocks": roof_clocks}
+    if stack_ms:
+        # The persistent launch that takes a whole stack of layers is the library's decode path for a model's
+        # layers; on this one-layer workload it runs STACK_PASSES passes per launch over the rotating copies.
+        # The timed step itself launches per layer (its figures: per_layer_launch).
+        roofline = {**common, "kernel": "sparse_ffn_stack_kernel",
+                    "call": f"clada_sparse_ffn_decode_layers: one persistent launch per {STACK_PASSES} layer passes "
+                            f"(the same passes as per_layer_launch: token t on copy t mod {N_COPIES})",
+                    **figures(pass_bytes(kept_base), stack_ms[0]), "bytes_per_launch": pass_bytes(kept_base) * STACK_PASSES,
+                    "bytes_per_layer_pass": pass_bytes(kept_base), "us_per_layer_pass": stack_ms[0] * 1e3,
+                    "us_per_launch": stack_ms[0] * 1e3 * STACK_PASSES, "kept_neurons": kept_base,
+                    "traffic": (lambda t: None if t is None else t * STACK_PASSES)(
+                        recorded_traffic("sparse_ffn_stack_kernel", w.name)),
+                    "by_sparsity": [
+                        {"sparsity": w.sparsities[r], "kept_neurons": w.d_ff - w.k_cut(w.sparsities[r]),
+                         "us_per_layer_pass": t * 1e3, **figures(pass_bytes(w.d_ff - w.k_cut(w.sparsities[r])), t)}
+                        for r, t in enumerate(stack_ms)],
+                    "per_layer_launch": per_launch}
+    elif isinstance(job, StackJob):
+        roofline = {**common, "kernel": "sparse_ffn_stack_kernel",
+                    "call": "clada_sparse_ffn_decode_layers: one persistent launch per token (all layers)",
+                    **figures(ffn_bytes, ffn_ms[0]), "bytes_per_launch": ffn_bytes * job.L, "bytes_per_layer_pass": ffn_bytes,
+                    "us_per_layer_pass": ffn_ms[0] * 1e3, "us_per_launch": ffn_ms[0] * 1e3 * job.L, "kept_neurons": kept_base,
+                    "traffic": None,
+                    "per_layer_launch": {"kernel": "sparse_ffn_kernel", "call": "clada_sparse_ffn_decode per layer",
+                                         **figures(ffn_bytes, per_layer_ms), "us_per_launch": per_layer_ms * 1e3}}
+    else:
+        roofline = {**common, **per_launch, "kernel": getattr(job, "ffn_kernel", "sparse_ffn_kernel")}
     h2d = sum(x.numel() * x.element_size() for x in host_in)
     d2h = hy.numel() * hy.element_size()
 
     line = {
         "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
-        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "vs_baseline": None, "dtype": w.dtype, "data": "synthetic",
         "config": {"workload": w.name, "d_model": w.d_model, "d_ff": w.d_ff, "layers": getattr(job, "layers_run", w.n_layers), "prefix_tokens": job.T,
                    "decode_tokens_per_sparsity": job.N, "sparsities": list(w.sparsities), "batch": w.batch,
                    "l2": job.l2_note, "cuda_graph": bool(args.graph), "avg_kept_neurons_per_token": kept,
-                   "step": job.step_note},
+                   "lambda": LAMBDA, "gamma": GAMMA, "step": job.step_note},
         "e2e": {"value": e2e_value, "unit": "tokens/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
         "gpu_launches": job.launches_per_step * args.steps,
-        "roofline": {"bound": "hbm", "kernel": getattr(job, "ffn_kernel", "sparse_ffn_kernel"), "achieved": achieved, "peak": peak,
-                     "unit": "GB/s", "frac": achieved / peak, "peak_kind": peak_kind,
-                     "traffic": FFN_NCU_TRAFFIC_BYTES if w.name == WORKLOAD else None,
-                     "read_only_stream_gbs": read_gbs, "frac_of_read_only_stream": achieved / read_gbs,
-                     "bytes_per_launch": ffn_bytes, "us_per_launch": ffn_ms * 1e3,
-                     "kept_neurons": kept_base},
+        "roofline": roofline,
         "prefix_roofline": {"bound": "tensor", "kernel": "prefix_tc_kernel (+finalize)", "ms": prefix_ms,
                             "achieved": prefix_flop / (prefix_ms * 1e-3) / 1e12, "peak": bf16_peak, "unit": "TFLOP/s",
                             "frac": prefix_flop / (prefix_ms * 1e-3) / 1e12 / bf16_peak, "peak_kind": bf16_kind,
                             "flop": prefix_flop},
         "clocks": clocks, "device_status_word": status,
     }
-    if other_ffn_ms:
-        per = [{"sparsity": w.sparsities[0], "kept_neurons": kept_base, "us_per_launch": ffn_ms * 1e3,
-                "achieved": achieved, "frac": achieved / peak}]
-        for r, t_ms in enumerate(other_ffn_ms, start=1):
-            kr = w.d_ff - w.k_cut(w.sparsities[r])
-            br = kr * rows * w.d_model * eb + w.d_ff * 4 + w.d_model * eb + w.d_model * 4
-            per.append({"sparsity": w.sparsities[r], "kept_neurons": kr, "us_per_launch": t_ms * 1e3,
-                        "achieved": br / (t_ms * 1e-3) / 1e9, "frac": br / (t_ms * 1e-3) / 1e9 / peak})
-        line["roofline"]["by_sparsity"] = per
+    if base_value is not None:
+        # lambda = gamma = 0 (the paper's ablation without semantic adaptation): the same step with every token
+        # at the configured baseline sparsities, i.e. the kept sets the roofline figures are taken on
+        line["value_baseline_only"] = {"value": base_value, "unit": "tokens/s", "ms_per_step": base_ms / args.steps,
+                                       "kept_neurons_per_token": [w.d_ff - w.k_cut(r) for r in w.sparsities],
+                                       "lambda": 0.0, "gamma": 0.0}
+    if info:
+        line["other_workloads"] = info
     if nested_value is not None:
         # list entries instead of the score vector: 4 bytes per kept neuron
         nb = kept_base * rows * w.d_model * eb + kept_base * 4 + w.d_model * eb + w.d_model * 4
@@ -752,6 +920,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-graph", dest="graph", action="store_false")
+    ap.add_argument("--no-info", dest="info", action="store_false",
+                    help="leave out the informational figures on the other workloads' layers")
     ap.add_argument("--workload", default=WORKLOAD, choices=[WORKLOAD, "c3_llama2_7b_stack", "c4_llama3_8b_b8", "c5_13b_b16", "v1_opt_2p7b_layer",
                              "v2_gemma_2b_layer"],
                     help="the metric's workload (default); the 32-layer stack or the OPT- / Gemma-shaped "

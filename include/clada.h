@@ -107,6 +107,23 @@ int clada_workspace_init(void *ws, size_t ws_bytes, void *stream);
  * device, the ceiling for the sparse FFN's weight rows. */
 int clada_stream_read_probe(const void *buf, size_t bytes, uint32_t *sink, void *stream);
 
+/* Self-test of the bounded device-side waits (the paper has no counterpart).
+ * Every wait inside the decode kernels -- for a ring stage's mbarrier, for the
+ * grid barrier -- gives up after a bounded number of polls and reports
+ * CLADA_STATUS_TIMEOUT instead of hanging.  This call makes both kinds of wait
+ * run out on purpose, in a form that cannot hang: two small CTAs wait on a
+ * shared-memory barrier that nobody arrives at, then meet at the workspace's
+ * grid barrier, which is told to expect one CTA more than the grid has.
+ *   poll_limit  polls per wait before giving up, 1 .. 2^20 (a few thousand is plenty)
+ *   report      out [2] int32, device: report[0] = 1 if the mbarrier wait gave up,
+ *               report[1] = 1 if the grid barrier gave up (both are expected)
+ *   status      optional device word; CLADA_STATUS_TIMEOUT is or-ed into it
+ * Afterwards the workspace's control words are left as a timed-out decode
+ * kernel leaves them (non-zero): call clada_workspace_init before the next
+ * decode on this workspace, exactly as after a real CLADA_STATUS_TIMEOUT. */
+int clada_selftest_bounded_waits(void *ws, size_t ws_bytes, uint32_t poll_limit, int32_t *report,
+                                 int32_t *status, void *stream);
+
 /* out[j] = ||W_out,j||_2 = the l2 norm of row j of w_down_t, fp32.  Once per
  * layer; the second factor of Eq. neuron_activation. */
 int clada_down_norms(const clada_layer *layer, float *out /*[d_ff]*/, void *stream);
@@ -332,7 +349,9 @@ int clada_prefill_down(const clada_layer *layer, const void *w_down, const void 
  *   tau_base   sequence b reads tau_base[b * tau_stride], device
  *   lambda, gamma  the layer's coefficients (host values, signed)
  *   order  out [B, d_ff] int32, device: neurons by descending score, equal
- *              scores by ascending index
+ *              scores by ascending index; zero scores of either sign come after
+ *              every positive one and NaN scores last of all, which is where
+ *              the comparison A_j >= tau puts them
  *   counts out [B, 4] int32, device: counts[b][k] = |{ j : A_bj >= tau_k }|,
  *              tau_k = fl32(tau_base_b * m_k), m = {1, 1+lambda, 1+gamma,
  *              (1+lambda)+gamma} in fp32 -- bit for bit the thresholds that

@@ -23,7 +23,7 @@ _INT_RETURNING = [
     "clada_workspace_init", "clada_down_norms", "clada_prefix_scores", "clada_refine_scores",
     "clada_select", "clada_prefix_select", "clada_tau_from_sparsity", "clada_cogload",
     "clada_adjust_threshold", "clada_cogload_adjust", "clada_sparse_ffn_decode",
-    "clada_sparse_ffn_decode_static", "clada_sparse_ffn_decode_layers", "clada_cett_threshold_search",
+    "clada_sparse_ffn_decode_static", "clada_sparse_ffn_decode_layers", "clada_selftest_bounded_waits", "clada_cett_threshold_search",
     "clada_cett_curve",
 ]
 
@@ -59,6 +59,7 @@ def load() -> ctypes.CDLL:
     L.clada_workspace_bytes.argtypes = [lp, i32, i64]
     L.clada_workspace_bytes.restype = sz
     L.clada_workspace_init.argtypes = [vp, sz, vp]
+    L.clada_selftest_bounded_waits.argtypes = [vp, sz, ctypes.c_uint32, vp, vp, vp]
     L.clada_down_norms.argtypes = [lp, vp, vp]
     L.clada_prefix_scores.argtypes = [lp, vp, vp, i32, vp, vp, sz, vp, vp]
     L.clada_refine_scores.argtypes = [lp, vp, vp, i32, vp, vp, i32, f32, vp, vp, sz, vp, vp]
@@ -197,6 +198,12 @@ def new_workspace(layer: Layer, B: int, T_total: int, stream=None) -> torch.Tens
     ws = torch.empty(clada_workspace_bytes(layer, B, T_total), dtype=torch.uint8, device=layer.w_gate.device)
     clada_workspace_init(ws, stream)
     return ws
+
+
+def clada_selftest_bounded_waits(ws, poll_limit: int, report, status=None, stream=None) -> None:
+    _check(load().clada_selftest_bounded_waits(_ptr(ws, torch.uint8, "ws"), ws.numel(), int(poll_limit),
+                                               _ptr(report, torch.int32, "report"), _ptr(status, torch.int32, "status"),
+                                               _stream(stream)), "clada_selftest_bounded_waits")
 
 
 def clada_down_norms(layer: Layer, out: torch.Tensor, stream=None) -> None:

@@ -12,7 +12,7 @@
 // Rank sort: a neuron's place in the list is the number of neurons that come before it -- those with a larger
 // score, or an equal score and a smaller index -- so every place can be computed independently and exactly.
 // A sequence is shared by several CTAs; each holds the whole score vector in shared memory (as bit patterns:
-// scores are norms, non-negative, so their patterns order them) and ranks its slice, one warp per neuron, lanes
+// scores are norms, so the patterns of the positive ones order them; see score_key for the rest) and ranks its slice, one warp per neuron, lanes
 // striding over the vector.  The four counts come from the first CTA of the sequence by a block-wide sum.  The
 // multipliers are formed on the host exactly as the adjustment kernel forms them (fp32, one addition at a time),
 // the thresholds with one fp32 multiplication.
@@ -31,6 +31,14 @@ struct NestMults {
     float m[4];
 };
 
+// Sort key of a score: scores are norms, so the bit patterns of the positive ones order them.  What is not a
+// positive number is put where the selection A_j >= tau puts it: NaN compares false with every threshold and
+// sorts after everything (key 0); zero of either sign and anything negative sort just before it (key 1).
+__device__ __forceinline__ unsigned score_key(float a) {
+    if (a > 0.f) return __float_as_uint(a) + 1u;
+    return a != a ? 0u : 1u;
+}
+
 __global__ void __launch_bounds__(kNestThreads)
 nested_build_kernel(const float *__restrict__ scores, int d_ff, const float *__restrict__ tau_base,
                     long long tau_stride, const NestMults mults, int32_t *__restrict__ order,
@@ -39,7 +47,7 @@ nested_build_kernel(const float *__restrict__ scores, int d_ff, const float *__r
     __shared__ int s_part[kNestThreads / kWarp][4];
     const int b = blockIdx.y, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const float *A = scores + (size_t)b * d_ff;
-    for (int i = tid; i < d_ff; i += kNestThreads) s_key[i] = __float_as_uint(A[i]);
+    for (int i = tid; i < d_ff; i += kNestThreads) s_key[i] = score_key(A[i]);
     __syncthreads();
     const int e0 = (int)(((long long)d_ff * blockIdx.x) / gridDim.x);
     const int e1 = (int)(((long long)d_ff * (blockIdx.x + 1)) / gridDim.x);
@@ -80,7 +88,7 @@ nested_build_kernel(const float *__restrict__ scores, int d_ff, const float *__r
         for (int k = 0; k < 4; ++k) tau[k] = __fmul_rn(tau_base[(size_t)b * tau_stride], mults.m[k]);
         int c[4] = {0, 0, 0, 0};
         for (int i = tid; i < d_ff; i += kNestThreads) {
-            const float a = __uint_as_float(s_key[i]);
+            const float a = A[i];
 #pragma unroll
             for (int k = 0; k < 4; ++k) c[k] += (a >= tau[k]) ? 1 : 0;
         }
@@ -114,14 +122,14 @@ nested_sort_kernel(const float *__restrict__ scores, int d_ff, int n_pow2, const
     float tau[4];
 #pragma unroll
     for (int k = 0; k < 4; ++k) tau[k] = __fmul_rn(tau_base[(size_t)b * tau_stride], mults.m[k]);
-    // Scores are norms (non-negative), so their bit patterns order them; complementing the pattern turns
-    // the ascending network into descending score, and the index in the low word breaks ties upward.
+    // Complementing the score's key turns the ascending network into descending score, and the index in the
+    // low word breaks ties upward.
     int c[4] = {0, 0, 0, 0};
     for (int i = tid; i < n_pow2; i += kNestThreads) {
         unsigned long long key = ~0ull;  // padding sorts last
         if (i < d_ff) {
             const float a = A[i];
-            key = ((unsigned long long)(~__float_as_uint(a)) << 32) | (unsigned)i;
+            key = ((unsigned long long)(~score_key(a)) << 32) | (unsigned)i;
 #pragma unroll
             for (int k = 0; k < 4; ++k) c[k] += (a >= tau[k]) ? 1 : 0;
         }

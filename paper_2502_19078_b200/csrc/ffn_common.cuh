@@ -12,7 +12,8 @@ constexpr unsigned kBarrierSpinLimit = 1u << 22;  // polls of an L2 word: gives 
 // Returns false if the wait expired.  Thread 0 arrives and polls; the departure count (whose last
 // increment resets both counters for the next launch) is another round trip to L2 that nothing waits
 // for, so a thread of the otherwise idle producer warp takes it after the CTA has been released.
-static __device__ bool grid_barrier(WsCtrl *ctrl, unsigned n_ctas, int depart_tid) {
+static __device__ bool grid_barrier(WsCtrl *ctrl, unsigned n_ctas, int depart_tid,
+                                    unsigned spin_limit = kBarrierSpinLimit) {
     __shared__ int s_ok;
     __syncthreads();
     if (threadIdx.x == 0) {
@@ -23,7 +24,7 @@ static __device__ bool grid_barrier(WsCtrl *ctrl, unsigned n_ctas, int depart_ti
         for (;;) {
             asm volatile("ld.acquire.gpu.u32 %0, [%1];" : "=r"(seen) : "l"(&ctrl->arrive) : "memory");
             if (seen >= n_ctas) break;
-            if (++spins > kBarrierSpinLimit) {
+            if (++spins > spin_limit) {
                 ok = 0;
                 break;
             }
@@ -69,9 +70,9 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
     return ok != 0;
 }
 constexpr unsigned kMbarSpinLimit = 1u << 20;  // tries of at most ~1 us each: about a second
-// Waits for the phase with the given parity; gives up (returns false) after kMbarSpinLimit tries.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
-    for (unsigned i = 0; i < kMbarSpinLimit; ++i)
+// Waits for the phase with the given parity; gives up (returns false) after `limit` tries.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, unsigned limit = kMbarSpinLimit) {
+    for (unsigned i = 0; i < limit; ++i)
         if (mbar_try_wait(bar, parity)) return true;
     return false;
 }

@@ -63,6 +63,41 @@ def test_nested_build_bit_exact(clada, oracle, F, lam, gam):
             np.testing.assert_array_equal(mask[0].cpu().numpy(), listed)
 
 
+@pytest.mark.parametrize("F", [200, 11008, 16384])
+@pytest.mark.parametrize("B", [1, 40])
+def test_nested_build_puts_non_numbers_where_the_selection_puts_them(clada, F, B):
+    """A NaN score is cut by every threshold (A_j >= tau is false), a zero of either sign only by positive ones:
+    the list must order them so that order[:counts[k]] is still exactly clada_select's kept set -- on both the
+    rank-sort and the bitonic route (B = 40 wide sequences takes the latter)."""
+    g = torch.Generator().manual_seed(F + B)
+    scores = (torch.rand(B, F, generator=g) * 0.2 + 0.9).float()
+    scores[0, 3] = float("nan")
+    scores[0, F - 1] = float("nan")
+    scores[0, 7] = -0.0
+    scores[0, 9] = 0.0
+    scores[-1, 0] = float("nan")
+    tau_base = torch.full((B,), 0.95, dtype=torch.float32)
+    order = torch.empty(B, F, dtype=torch.int32, device="cuda")
+    counts = torch.empty(B, 4, dtype=torch.int32, device="cuda")
+    sd = scores.cuda()
+    clada.clada_nested_build(sd, tau_base.cuda(), LAM, GAM, order, counts)
+    mask = torch.empty(1, F, dtype=torch.uint8, device="cuda")
+    cnt = torch.empty(1, dtype=torch.int32, device="cuda")
+    for b in (0, B - 1):
+        o = order[b].cpu().numpy()
+        assert sorted(o.tolist()) == list(range(F))                  # a permutation
+        nan_idx = set(np.nonzero(np.isnan(scores[b].numpy()))[0].tolist())
+        assert set(o[F - len(nan_idx):].tolist()) == nan_idx         # the NaNs come last
+        for k, tau in enumerate(_thresholds(0.95, LAM, GAM)):
+            clada.clada_select(sd[b:b + 1], torch.tensor([tau]).cuda(), 1, mask, None, cnt)
+            n = int(counts[b, k])
+            assert n == int(cnt.item())
+            kept = np.zeros(F, dtype=np.uint8)
+            kept[o[:n]] = 1
+            np.testing.assert_array_equal(kept, mask[0].cpu().numpy())
+    torch.cuda.synchronize()
+
+
 def test_cogload_level_matches_adjustment(clada, oracle):
     w = wl.WORKLOADS["c2_llama2_7b_layer"]
     n = 16
