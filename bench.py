@@ -516,7 +516,8 @@ class BatchJob:
                                                self.y[t], self.ws)
 
 
-FFN_INNER = 12      # replays per sample of an FFN-only loop (a sample lasts 40-60 ms; seven samples per figure)
+FFN_INNER = 12      # replays per sample of an FFN-only loop (a sample lasts 40-60 ms)
+FFN_REPEATS = 7     # samples per figure
 
 
 def _graphed(fn, stream, use_graph):
@@ -531,8 +532,9 @@ def _graphed(fn, stream, use_graph):
     return g.replay
 
 
-def _median_ms(run, inner=1, repeats=7):
+def _median_ms(run, inner=1, repeats=None):
     """Median over `repeats` samples of the device time of one run (each sample times `inner` runs)."""
+    repeats = FFN_REPEATS if repeats is None else repeats
     samples = sorted(_timed(run, inner, lambda: None) / inner for _ in range(repeats))
     return samples[len(samples) // 2]
 
@@ -744,7 +746,7 @@ def run_ours(args):
         return {"achieved": gbs, "frac": gbs / peak, "frac_of_read_only_stream": gbs / read_gbs}
 
     ffn_bytes = job.ffn_bytes_per_launch if hasattr(job, "ffn_bytes_per_launch") else pass_bytes(kept_base)
-    sample_note = f"median of 7 samples of {FFN_INNER} replays of the loop's CUDA graph, clocks recorded over all of them"
+    sample_note = f"median of {FFN_REPEATS} samples of {FFN_INNER} replays of the loop's CUDA graph, clocks recorded over all of them"
     per_launch = {"kernel": "sparse_ffn_kernel", "call": "clada_sparse_ffn_decode: one launch per layer pass",
                   **figures(ffn_bytes, ffn_ms[0]), "bytes_per_launch": ffn_bytes, "us_per_launch": ffn_ms[0] * 1e3,
                   "kept_neurons": kept_base, "traffic": recorded_traffic("sparse_ffn_kernel", w.name)}
@@ -922,11 +924,17 @@ def main():
     ap.add_argument("--no-graph", dest="graph", action="store_false")
     ap.add_argument("--no-info", dest="info", action="store_false",
                     help="leave out the informational figures on the other workloads' layers")
+    ap.add_argument("--quick", action="store_true",
+                    help="for profiler captures: one replay per sample of the FFN-only loops and no informational "
+                         "workloads (the figures of such a run are not bench values)")
     ap.add_argument("--workload", default=WORKLOAD, choices=[WORKLOAD, "c3_llama2_7b_stack", "c4_llama3_8b_b8", "c5_13b_b16", "v1_opt_2p7b_layer",
                              "v2_gemma_2b_layer"],
                     help="the metric's workload (default); the 32-layer stack or the OPT- / Gemma-shaped "
                          "layers (other FFN forms) for information")
     args = ap.parse_args()
+    if args.quick:
+        global FFN_INNER, FFN_REPEATS
+        FFN_INNER, FFN_REPEATS, args.info = 1, 1, False
     if args.gpus < 1:
         ap.error("--gpus must be at least 1")
     if args.impl == "reference":
