@@ -31,7 +31,7 @@ struct FfnParams {
     uint8_t *mask_out;    // [d_ff] or null
     int32_t *idx_out;     // [d_ff] or null
     int32_t *count_out;   // one int or null
-    float *partials;      // [gridDim.x, d_model]
+    float *partials;      // [gridDim.x, consumer groups, d_model]
     WsCtrl *ctrl;
     int32_t *status;
     int d_model, d_ff;
@@ -49,10 +49,10 @@ __device__ __forceinline__ int split_at(int n, int c, int n_ctas) {
     return (int)(((unsigned)n * (unsigned)c) / (unsigned)n_ctas);
 }
 
-constexpr int G = 4;                          // neurons per CTA-wide reduction
+constexpr int G = GS;                         // neurons per group-wide reduction (a reduction holds G stages)
 constexpr int kMaxBatches = 4;                // prologue batches: d_ff <= 4 * 32 * kFfnThreads
 
-template <typename T, int NV, bool GATED>
+template <typename T, int NV, bool GATED, int GROUPS>
 __global__ void __launch_bounds__(kFfnThreads, 1)
 sparse_ffn_kernel(const FfnParams p, const int n_stages) {
     constexpr int E = Elem<T>::kPerVec;
@@ -77,13 +77,15 @@ sparse_ffn_kernel(const FfnParams p, const int n_stages) {
     int *s_list = reinterpret_cast<int *>(s_bal + chunks);
     __shared__ int s_wtot[kFfnWarps];
     __shared__ float s_tau;
-    __shared__ __align__(16) float s_dot[2][2 * G][kConsWarps];
+    __shared__ __align__(16) float s_dot[kDotFloats];
+    constexpr int GT = kConsumers / GROUPS;  // threads per consumer group (the producer warp counts as none)
+    const int grp = tid < kConsumers ? tid / GT : 0, gt = tid - grp * GT;
 
     pdl_launch_dependents();  // the next kernel in the stream may be scheduled as SMs free up
     if (tid == kConsumers) {  // the producer warp sets the ring up while the others start loading
         for (int s = 0; s < n_stages; ++s) {
             mbar_init(full0 + 8 * s, 1);            // the producer's expect_tx arrival
-            mbar_init(empty0 + 8 * s, kConsWarps);  // one arrival per consumer warp
+            mbar_init(empty0 + 8 * s, kConsWarps / GROUPS);  // one arrival per warp of the group that owns the stage
         }
         mbar_init(sbar, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -104,7 +106,7 @@ sparse_ffn_kernel(const FfnParams p, const int n_stages) {
     bool vok[NV];
 #pragma unroll
     for (int i = 0; i < NV; ++i) {
-        const int v = tid + i * kConsumers;
+        const int v = gt + i * GT;
         vok[i] = tid < kConsumers && v < vpr;
         uint4 q = make_uint4(0, 0, 0, 0);
         if (vok[i]) q = *(reinterpret_cast<const uint4 *>(p.x) + v);
@@ -317,101 +319,16 @@ sparse_ffn_kernel(const FfnParams p, const int n_stages) {
         for (int i = 0; i < NV; ++i)
 #pragma unroll
             for (int e = 0; e < P; ++e) acc[i][e] = make_float2(0.f, 0.f);
-        const bool b16 = lane & 16, b8 = lane & 8, b4 = lane & 4;
-        int buf = 0;
         int cs = 0;           // ring position of the next neuron to consume, and the parity of its use
         uint32_t cpar = 0;
-        for (int g0 = 0; g0 < my_n; g0 += G, buf ^= 1) {
-            float pd[2 * G];
-            uint32_t st_addr[G];
-            int st_idx[G];
-#pragma unroll
-            for (int g = 0; g < G; ++g) {
-                const int i = g0 + g;
-                float2 sg = make_float2(0.f, 0.f), su = make_float2(0.f, 0.f);
-                st_idx[g] = cs;
-                st_addr[g] = ring + (uint32_t)cs * stage_bytes;
-                if (i < my_n) {
-                    if (!timed_out && !mbar_wait(full0 + 8 * cs, cpar)) timed_out = true;
-                    if (++cs == n_stages) {
-                        cs = 0;
-                        cpar ^= 1;
-                    }
-#pragma unroll
-                    for (int k = 0; k < NV; ++k) {
-                        if (!vok[k]) continue;
-                        const uint32_t a = st_addr[g] + (uint32_t)(tid + k * kConsumers) * 16u;
-                        float2 fg[P], fu[P];
-                        Pairs<T>::unpack(lds128(a), fg);
-                        if (GATED) Pairs<T>::unpack(lds128(a + row_bytes), fu);
-#pragma unroll
-                        for (int e = 0; e < P; ++e) {
-                            sg = __ffma2_rn(fg[e], xr[k][e], sg);
-                            if (GATED) su = __ffma2_rn(fu[e], xr[k][e], su);
-                        }
-                    }
-                }
-                pd[2 * g] = sg.x + sg.y;
-                pd[2 * g + 1] = su.x + su.y;
-            }
-            // Warp sums of the 8 values by a halving butterfly (9 shuffles): after it every lane of
-            // quad q holds the warp total of value q.  Fixed order, so results repeat bit for bit.
-            float b[4], c[2], v8;
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const float send = b16 ? pd[i] : pd[i + 4];
-                b[i] = (b16 ? pd[i + 4] : pd[i]) + __shfl_xor_sync(0xffffffffu, send, 16);
-            }
-#pragma unroll
-            for (int i = 0; i < 2; ++i) {
-                const float send = b8 ? b[i] : b[i + 2];
-                c[i] = (b8 ? b[i + 2] : b[i]) + __shfl_xor_sync(0xffffffffu, send, 8);
-            }
-            v8 = (b4 ? c[1] : c[0]) + __shfl_xor_sync(0xffffffffu, b4 ? c[0] : c[1], 4);
-            v8 += __shfl_xor_sync(0xffffffffu, v8, 2);
-            v8 += __shfl_xor_sync(0xffffffffu, v8, 1);
-            // lane 4q holds value index: bit4 -> +4, bit3 -> +2, bit2 -> +1
-            if ((lane & 3) == 0) s_dot[buf][(b16 ? 4 : 0) + (b8 ? 2 : 0) + (b4 ? 1 : 0)][warp] = v8;
-            asm volatile("bar.sync 1, %0;" ::"n"(kConsumers) : "memory");
-            // Cross-warp sums: lane l adds 4 consecutive warps of value l/4 (16 warps = 4 lanes per
-            // value), the quad finishes by butterfly; then gate lanes form h = silu(gate) * up.
-            float tot;
-            {
-                const float4 q4 = *reinterpret_cast<const float4 *>(&s_dot[buf][lane >> 2][(lane & 3) * 4]);
-                tot = (q4.x + q4.y) + (q4.z + q4.w);
-                tot += __shfl_xor_sync(0xffffffffu, tot, 1);
-                tot += __shfl_xor_sync(0xffffffffu, tot, 2);
-            }
-            const float up = __shfl_xor_sync(0xffffffffu, tot, 4);  // value 2g+1 sits 4 lanes above value 2g
-            const float hval = neuron_value_f(p.act, tot, up);          // meaningful on lanes 8g..8g+3
-#pragma unroll
-            for (int g = 0; g < G; ++g) {
-                const float h = __shfl_sync(0xffffffffu, hval, 8 * g);
-                if (g0 + g >= my_n) continue;
-                const float2 h2 = make_float2(h, h);
-#pragma unroll
-                for (int k = 0; k < NV; ++k) {
-                    if (!vok[k]) continue;
-                    float2 fd[P];
-                    Pairs<T>::unpack(lds128(st_addr[g] + down_off + (uint32_t)(tid + k * kConsumers) * 16u), fd);
-#pragma unroll
-                    for (int e = 0; e < P; ++e) acc[k][e] = __ffma2_rn(h2, fd[e], acc[k][e]);
-                }
-            }
-            // hand the stages back to the producer
-            __syncwarp();
-            if (lane == 0) {
-#pragma unroll
-                for (int g = 0; g < G; ++g)
-                    if (g0 + g < my_n) mbar_arrive(empty0 + 8 * st_idx[g]);
-            }
-        }
-        // partial y of this CTA
-        float *mine = p.partials + (size_t)cta * d;
+        consume_share<T, NV, GATED, GROUPS>(my_n, p.act, ring, stage_bytes, row_bytes, down_off, full0, empty0, n_stages,
+                                            cs, cpar, xr, vok, acc, s_dot, timed_out);
+        // partial y of this consumer group
+        float *mine = p.partials + ((size_t)cta * GROUPS + grp) * d;
 #pragma unroll
         for (int i = 0; i < NV; ++i) {
             if (!vok[i]) continue;
-            float4 *dst = reinterpret_cast<float4 *>(mine + (size_t)(tid + i * kConsumers) * E);
+            float4 *dst = reinterpret_cast<float4 *>(mine + (size_t)(gt + i * GT) * E);
 #pragma unroll
             for (int e = 0; e < P; e += 2)
                 dst[e / 2] = make_float4(acc[i][e].x, acc[i][e].y, acc[i][e + 1].x, acc[i][e + 1].y);
@@ -424,18 +341,20 @@ sparse_ffn_kernel(const FfnParams p, const int n_stages) {
         if (tid == 0 && p.status) atomicOr(p.status, CLADA_STATUS_TIMEOUT);
         return;
     }
-    // columns in groups of 4 (float4); a warp sums one group: lane l adds partial rows l, l+32, ...
-    // in order (five loads in flight at a time), then the 32 lane sums combine by butterfly.
+    // columns in groups of 4 (float4); a warp sums one group: lane l adds partial rows l, l+32, ... (one row
+    // per CTA and consumer group) in order (five loads in flight at a time), then the 32 lane sums combine by
+    // butterfly.
     const int ngroups = d / 4;
+    const int n_rows = n_ctas * GROUPS;
     for (int q = cta + warp * n_ctas; q < ngroups; q += n_ctas * kFfnWarps) {
         float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
-        for (int rb = 0; rb < n_ctas; rb += 5 * kWarp) {
+        for (int rb = 0; rb < n_rows; rb += 5 * kWarp) {
             float4 v[5];
 #pragma unroll
             for (int u = 0; u < 5; ++u) {
                 const int r = rb + u * kWarp + lane;
                 v[u] = make_float4(0.f, 0.f, 0.f, 0.f);
-                if (r < n_ctas) v[u] = __ldcg(reinterpret_cast<const float4 *>(p.partials + (size_t)r * d) + q);
+                if (r < n_rows) v[u] = __ldcg(reinterpret_cast<const float4 *>(p.partials + (size_t)r * d) + q);
             }
 #pragma unroll
             for (int u = 0; u < 5; ++u) {
@@ -455,14 +374,14 @@ sparse_ffn_kernel(const FfnParams p, const int n_stages) {
 
 // ---- host side ------------------------------------------------------------------------------
 
-template <typename T, int NV, bool GATED>
+template <typename T, int NV, bool GATED, int GROUPS>
 static int launch_variant(const FfnParams &p, cudaStream_t st) {
     constexpr int E = Elem<T>::kPerVec;
     static bool configured[64] = {};
     DeviceInfo di;
     int rc = device_info(&di);
     if (rc != CLADA_OK) return rc;
-    auto kern = sparse_ffn_kernel<T, NV, GATED>;
+    auto kern = sparse_ffn_kernel<T, NV, GATED, GROUPS>;
     const size_t stage_bytes = (GATED ? 3 : 2) * (size_t)(p.d_model / E) * 16;
     const size_t tail = (2 * kMaxStages + 1) * sizeof(uint64_t) + (size_t)((p.d_ff + 31) / 32) * sizeof(unsigned) +
                         (size_t)(p.d_ff / di.num_sms + 2) * sizeof(int);
@@ -500,8 +419,11 @@ static int launch_ffn(const FfnParams &p, cudaStream_t st) {
     const int vpr = p.d_model / E;
     if (p.d_ff > kMaxBatches * kWarp * kFfnThreads) return CLADA_ERR_UNSUPPORTED;
     const bool gated = act_is_gated(p.act);
-    if (vpr <= kConsumers) return gated ? launch_variant<T, 1, true>(p, st) : launch_variant<T, 1, false>(p, st);
-    if (vpr <= 2 * kConsumers) return gated ? launch_variant<T, 2, true>(p, st) : launch_variant<T, 2, false>(p, st);
+    if (vpr <= kConsumers / 2)  // narrow rows: two consumer groups of 256 threads, one vector per thread
+        return gated ? launch_variant<T, 1, true, 2>(p, st) : launch_variant<T, 1, false, 2>(p, st);
+    if (vpr <= kConsumers) return gated ? launch_variant<T, 1, true, 1>(p, st) : launch_variant<T, 1, false, 1>(p, st);
+    if (vpr <= 2 * kConsumers)  // wide rows: two vectors per thread
+        return gated ? launch_variant<T, 2, true, 1>(p, st) : launch_variant<T, 2, false, 1>(p, st);
     return CLADA_ERR_UNSUPPORTED;
 }
 
@@ -532,7 +454,12 @@ static int decode_tile(const clada_layer *layer, int remaining, int max_tile) {
 // Scratch bytes a decode call needs when its tiles hold at most max_tile sequences: the control words and
 // one fp32 partial output row per (CTA, sequence of the tile).
 static size_t decode_scratch_bytes(const clada_layer *layer, int32_t B, int num_sms, int max_tile) {
-    return kWsCtrlBytes + (size_t)num_sms * decode_tile(layer, B, max_tile) * layer->d_model * sizeof(float);
+    const int tile = decode_tile(layer, B, max_tile);
+    const int vpr = layer->d_model / (layer->dtype == CLADA_F32 ? 4 : 8);
+    // a single sequence's launch writes one row per consumer group; sequences left over after the tiles run singly
+    const int rows = tile > 1 ? tile : 1;
+    const int single_rows = (tile == 1 || B % tile != 0) ? ffn_groups(vpr) : 1;
+    return kWsCtrlBytes + (size_t)num_sms * (rows > single_rows ? rows : single_rows) * layer->d_model * sizeof(float);
 }
 
 // The launches of a validated decode call whose scratch holds tiles of up to max_tile sequences.
@@ -633,7 +560,7 @@ extern "C" int clada_sparse_ffn_decode_nested(const clada_layer *layer, const vo
     DeviceInfo di;
     rc = device_info(&di);
     if (rc != CLADA_OK) return rc;
-    if (ws_bytes < kWsCtrlBytes + (size_t)di.num_sms * layer->d_model * sizeof(float)) return CLADA_ERR_WORKSPACE;
+    if (ws_bytes < decode_scratch_bytes(layer, 1, di.num_sms, 1)) return CLADA_ERR_WORKSPACE;
     const size_t esz = elem_size(layer->dtype), ysz = elem_size(y_dtype);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     for (int b = 0; b < B; ++b) {

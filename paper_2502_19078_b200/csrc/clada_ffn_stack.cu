@@ -27,7 +27,6 @@ namespace clada {
 
 constexpr int kMaxStackLayers = 128;  // layers per launch (their weight pointers travel as kernel parameters)
 constexpr int kStackMaxDff = 65536;    // the scanner parks one keep word per 32 neurons in shared memory
-constexpr int GS = 4;                 // neurons per CTA-wide reduction
 
 struct StackLayers {
     const void *w[kMaxStackLayers][3];  // w_gate, w_up, w_down_t of every layer
@@ -42,7 +41,7 @@ struct StackParams {
     char *y;              // layer l writes y + l * y_stride (bytes)
     size_t y_stride;
     int y_dtype;
-    float *partials;      // [2][gridDim.x][d_model]
+    float *partials;      // [2][gridDim.x][consumer groups][d_model]
     WsCtrl *ctrl;
     int32_t *status;
     int d_model, d_ff, L;
@@ -150,7 +149,7 @@ __device__ __forceinline__ int scan_share_list(const float *__restrict__ scores,
     return n_act;
 }
 
-template <typename T, int NV, bool GATED>
+template <typename T, int NV, bool GATED, int GROUPS>
 __global__ void __launch_bounds__(kStackThreads, 1)
 sparse_ffn_stack_kernel(const StackParams p, const __grid_constant__ StackLayers lay, const int n_stages,
                         const int list_cap) {
@@ -180,13 +179,13 @@ sparse_ffn_stack_kernel(const StackParams p, const __grid_constant__ StackLayers
     __shared__ int s_nact[kListBufs], s_myn[kListBufs];  // per list buffer: the layer's kept count, this CTA's share
     __shared__ int s_cur[2][3];                          // consumers' copy for the current layer (+ give-up flag)
     __shared__ int s_ecur[2][3];                         // the epilogue warps' copy
-    __shared__ __align__(16) float s_dot[2][2 * GS][kConsWarps];
+    __shared__ __align__(16) float s_dot[kDotFloats];
 
     pdl_launch_dependents();
     if (tid == kConsumers) {
         for (int s = 0; s < n_stages; ++s) {
             mbar_init(full0 + 8 * s, 1);            // the producer's expect_tx arrival
-            mbar_init(empty0 + 8 * s, kConsWarps);  // one arrival per consumer warp
+            mbar_init(empty0 + 8 * s, kConsWarps / GROUPS);  // one arrival per warp of the group that owns the stage
         }
         for (int k = 0; k < kListBufs; ++k) {
             mbar_init(lready0 + 8 * k, 1);  // the scanner
@@ -280,19 +279,20 @@ sparse_ffn_stack_kernel(const StackParams p, const __grid_constant__ StackLayers
             }
             epilogue_sync();
             if (s_ecur[l & 1][2]) timed_out = true;
-            const float *part = p.partials + (size_t)(epoch & 1u) * n_ctas * d;
+            const int n_rows = n_ctas * GROUPS;  // one partial row per (CTA, consumer group)
+            const float *part = p.partials + (size_t)(epoch & 1u) * n_rows * d;
             ++epoch;
             // columns in groups of 4 (float4), a warp per group: lane l adds partial rows l, l+32, ... in order
             // (five loads in flight at a time), then the 32 lane sums combine by butterfly.
             for (int q = cta + ew * n_ctas; q < ngroups; q += kEpiWarps * n_ctas) {
                 float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
-                for (int rb = 0; rb < n_ctas; rb += 5 * kWarp) {
+                for (int rb = 0; rb < n_rows; rb += 5 * kWarp) {
                     float4 v[5];
 #pragma unroll
                     for (int u = 0; u < 5; ++u) {
                         const int r = rb + u * kWarp + lane;
                         v[u] = make_float4(0.f, 0.f, 0.f, 0.f);
-                        if (r < n_ctas) v[u] = __ldcg(reinterpret_cast<const float4 *>(part + (size_t)r * d) + q);
+                        if (r < n_rows) v[u] = __ldcg(reinterpret_cast<const float4 *>(part + (size_t)r * d) + q);
                     }
 #pragma unroll
                     for (int u = 0; u < 5; ++u) {
@@ -398,10 +398,11 @@ sparse_ffn_stack_kernel(const StackParams p, const __grid_constant__ StackLayers
     }
 
     // ---- consumers ------------------------------------------------------------------------------------
+    constexpr int GT = kConsumers / GROUPS;  // threads per consumer group
+    const int grp = tid / GT, gt = tid - grp * GT;
     bool vok[NV];
 #pragma unroll
-    for (int i = 0; i < NV; ++i) vok[i] = tid + i * kConsumers < vpr;
-    const bool b16 = lane & 16, b8 = lane & 8, b4 = lane & 4;
+    for (int i = 0; i < NV; ++i) vok[i] = gt + i * GT < vpr;
     int cs = 0;  // ring position of the next stage to consume, and the parity of its use
     uint32_t cpar = 0;
     unsigned epoch = 0;  // grid barriers passed so far (layers that kept something)
@@ -419,7 +420,7 @@ sparse_ffn_stack_kernel(const StackParams p, const __grid_constant__ StackLayers
         consumer_sync();
         const int n_act = s_cur[l & 1][0], my_n = s_cur[l & 1][1];
         if (s_cur[l & 1][2]) timed_out = true;
-        if (n_act == 0) continue;  // nothing is kept (every CTA sees the same count): the epilogue warp writes y = 0
+        if (n_act == 0) continue;  // nothing is kept (every CTA sees the same count): the epilogue warps write y = 0
         // x of this thread's columns, from the stage the producer filled ahead of the layer's rows
         float2 xr[NV][P];
 #pragma unroll
@@ -431,9 +432,10 @@ sparse_ffn_stack_kernel(const StackParams p, const __grid_constant__ StackLayers
             const uint32_t xa = ring + (uint32_t)cs * stage_bytes;
 #pragma unroll
             for (int i = 0; i < NV; ++i)
-                if (vok[i]) Pairs<T>::unpack(lds128(xa + (uint32_t)(tid + i * kConsumers) * 16u), xr[i]);
+                if (vok[i]) Pairs<T>::unpack(lds128(xa + (uint32_t)(gt + i * GT) * 16u), xr[i]);
+            if (GROUPS > 1) consumer_sync();  // both groups have read x; the first group's warps hand the stage back
             __syncwarp();
-            if (lane == 0) mbar_arrive(empty0 + 8 * cs);
+            if (lane == 0 && grp == 0) mbar_arrive(empty0 + 8 * cs);
             if (++cs == n_stages) {
                 cs = 0;
                 cpar ^= 1;
@@ -447,115 +449,26 @@ sparse_ffn_stack_kernel(const StackParams p, const __grid_constant__ StackLayers
 #ifdef CLADA_STACK_TRACE
         unsigned long long cwait = 0;
         if (tid == 0) STACK_TRACE(l, 0, trace_now());
-#endif
-        int buf = 0;
-        for (int g0 = 0; g0 < my_n; g0 += GS, buf ^= 1) {
-            float pd[2 * GS];
-            uint32_t st_addr[GS];
-            int st_idx[GS];
-#pragma unroll
-            for (int g = 0; g < GS; ++g) {
-                const int i = g0 + g;
-                float2 sg = make_float2(0.f, 0.f), su = make_float2(0.f, 0.f);
-                st_idx[g] = cs;
-                st_addr[g] = ring + (uint32_t)cs * stage_bytes;
-                if (i < my_n) {
-#ifdef CLADA_STACK_TRACE
-                    const unsigned long long w0 = trace_now();
-#endif
-                    if (!timed_out && !mbar_wait(full0 + 8 * cs, cpar)) timed_out = true;
-#ifdef CLADA_STACK_TRACE
-                    cwait += trace_now() - w0;
-#endif
-                    if (++cs == n_stages) {
-                        cs = 0;
-                        cpar ^= 1;
-                    }
-#pragma unroll
-                    for (int k = 0; k < NV; ++k) {
-                        if (!vok[k]) continue;
-                        const uint32_t a = st_addr[g] + (uint32_t)(tid + k * kConsumers) * 16u;
-                        float2 fg[P], fu[P];
-                        Pairs<T>::unpack(lds128(a), fg);
-                        if (GATED) Pairs<T>::unpack(lds128(a + row_bytes), fu);
-#pragma unroll
-                        for (int e = 0; e < P; ++e) {
-                            sg = __ffma2_rn(fg[e], xr[k][e], sg);
-                            if (GATED) su = __ffma2_rn(fu[e], xr[k][e], su);
-                        }
-                    }
-                }
-                pd[2 * g] = sg.x + sg.y;
-                pd[2 * g + 1] = su.x + su.y;
-            }
-            // Warp sums of the 8 values by a halving butterfly (9 shuffles): after it every lane of
-            // quad q holds the warp total of value q.  Fixed order, so results repeat bit for bit.
-            float b[4], c[2], v8;
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const float send = b16 ? pd[i] : pd[i + 4];
-                b[i] = (b16 ? pd[i + 4] : pd[i]) + __shfl_xor_sync(0xffffffffu, send, 16);
-            }
-#pragma unroll
-            for (int i = 0; i < 2; ++i) {
-                const float send = b8 ? b[i] : b[i + 2];
-                c[i] = (b8 ? b[i + 2] : b[i]) + __shfl_xor_sync(0xffffffffu, send, 8);
-            }
-            v8 = (b4 ? c[1] : c[0]) + __shfl_xor_sync(0xffffffffu, b4 ? c[0] : c[1], 4);
-            v8 += __shfl_xor_sync(0xffffffffu, v8, 2);
-            v8 += __shfl_xor_sync(0xffffffffu, v8, 1);
-            // lane 4q holds value index: bit4 -> +4, bit3 -> +2, bit2 -> +1
-            if ((lane & 3) == 0) s_dot[buf][(b16 ? 4 : 0) + (b8 ? 2 : 0) + (b4 ? 1 : 0)][warp] = v8;
-            consumer_sync();
-            // Cross-warp sums: lane l adds 4 consecutive warps of value l/4, the quad finishes by
-            // butterfly; then gate lanes form the neuron value h.
-            float tot;
-            {
-                const float4 q4 = *reinterpret_cast<const float4 *>(&s_dot[buf][lane >> 2][(lane & 3) * 4]);
-                tot = (q4.x + q4.y) + (q4.z + q4.w);
-                tot += __shfl_xor_sync(0xffffffffu, tot, 1);
-                tot += __shfl_xor_sync(0xffffffffu, tot, 2);
-            }
-            const float up = __shfl_xor_sync(0xffffffffu, tot, 4);  // value 2g+1 sits 4 lanes above value 2g
-            const float hval = neuron_value_f(p.act, tot, up);      // meaningful on lanes 8g..8g+3
-#pragma unroll
-            for (int g = 0; g < GS; ++g) {
-                const float h = __shfl_sync(0xffffffffu, hval, 8 * g);
-                if (g0 + g >= my_n) continue;
-                const float2 h2 = make_float2(h, h);
-#pragma unroll
-                for (int k = 0; k < NV; ++k) {
-                    if (!vok[k]) continue;
-                    float2 fd[P];
-                    Pairs<T>::unpack(lds128(st_addr[g] + down_off + (uint32_t)(tid + k * kConsumers) * 16u), fd);
-#pragma unroll
-                    for (int e = 0; e < P; ++e) acc[k][e] = __ffma2_rn(h2, fd[e], acc[k][e]);
-                }
-            }
-            // hand the stages back to the producer
-            __syncwarp();
-            if (lane == 0) {
-#pragma unroll
-                for (int g = 0; g < GS; ++g)
-                    if (g0 + g < my_n) mbar_arrive(empty0 + 8 * st_idx[g]);
-            }
-        }
-#ifdef CLADA_STACK_TRACE
+        consume_share<T, NV, GATED, GROUPS>(my_n, p.act, ring, stage_bytes, row_bytes, down_off, full0, empty0, n_stages,
+                                            cs, cpar, xr, vok, acc, s_dot, timed_out, &cwait);
         if (tid == 0) {
             STACK_TRACE(l, 1, trace_now());
             STACK_TRACE(l, 9, cwait);
         }
+#else
+        consume_share<T, NV, GATED, GROUPS>(my_n, p.act, ring, stage_bytes, row_bytes, down_off, full0, empty0, n_stages,
+                                            cs, cpar, xr, vok, acc, s_dot, timed_out);
 #endif
-        // Partial y of this CTA, into the buffer of this barrier number.  The buffer was last read for the
-        // column sums of the barrier two back; all of those are done once every CTA has passed the barrier
-        // before this one, which the epilogue warp reports.
+        // Partial y of this consumer group, into the buffer of this barrier number.  The buffer was last read
+        // for the column sums of the barrier two back; all of those are done once every CTA has passed the
+        // barrier before this one, which the epilogue warps report.
         if (epoch >= 1u && !timed_out && !mbar_wait(bdone, (epoch - 1u) & 1u)) timed_out = true;
-        float *mine = p.partials + ((size_t)(epoch & 1u) * n_ctas + cta) * d;
+        float *mine = p.partials + (((size_t)(epoch & 1u) * n_ctas + cta) * GROUPS + grp) * d;
         ++epoch;
 #pragma unroll
         for (int i = 0; i < NV; ++i) {
             if (!vok[i]) continue;
-            float4 *dst = reinterpret_cast<float4 *>(mine + (size_t)(tid + i * kConsumers) * E);
+            float4 *dst = reinterpret_cast<float4 *>(mine + (size_t)(gt + i * GT) * E);
 #pragma unroll
             for (int e = 0; e < P; e += 2)
                 dst[e / 2] = make_float4(acc[i][e].x, acc[i][e].y, acc[i][e + 1].x, acc[i][e + 1].y);
@@ -565,8 +478,6 @@ sparse_ffn_stack_kernel(const StackParams p, const __grid_constant__ StackLayers
     }
     if (timed_out && tid == 0 && p.status) atomicOr(p.status, CLADA_STATUS_TIMEOUT);
 }
-
-// ---- host side ------------------------------------------------------------------------------
 
 // Ring stages and dynamic shared memory of a launch; n_stages < GS means the kernel cannot take the layer
 // (a reduction group holds GS stages at once; the x stage is handed back before the group starts).
@@ -583,13 +494,13 @@ static void stack_smem_plan(const DeviceInfo &di, int d_model, int d_ff, int dty
     *smem = (size_t)n * stage_bytes + tail;
 }
 
-template <typename T, int NV, bool GATED>
+template <typename T, int NV, bool GATED, int GROUPS>
 static int launch_stack_variant(const StackParams &p, const StackLayers &lay, int dtype, cudaStream_t st) {
     static bool configured[64] = {};
     DeviceInfo di;
     int rc = device_info(&di);
     if (rc != CLADA_OK) return rc;
-    auto kern = sparse_ffn_stack_kernel<T, NV, GATED>;
+    auto kern = sparse_ffn_stack_kernel<T, NV, GATED, GROUPS>;
     int n_stages, list_cap;
     size_t smem, budget;
     stack_smem_plan(di, p.d_model, p.d_ff, dtype, GATED, &n_stages, &list_cap, &smem, &budget);
@@ -623,12 +534,15 @@ static int launch_stack_typed(const StackParams &p, const StackLayers &lay, int 
     constexpr int E = Elem<T>::kPerVec;
     const int vpr = p.d_model / E;
     const bool gated = act_is_gated(p.act);
+    if (vpr <= kConsumers / 2)  // narrow rows: two consumer groups of 256 threads, one vector per thread
+        return gated ? launch_stack_variant<T, 1, true, 2>(p, lay, dtype, st)
+                     : launch_stack_variant<T, 1, false, 2>(p, lay, dtype, st);
     if (vpr <= kConsumers)
-        return gated ? launch_stack_variant<T, 1, true>(p, lay, dtype, st)
-                     : launch_stack_variant<T, 1, false>(p, lay, dtype, st);
-    if (vpr <= 2 * kConsumers)
-        return gated ? launch_stack_variant<T, 2, true>(p, lay, dtype, st)
-                     : launch_stack_variant<T, 2, false>(p, lay, dtype, st);
+        return gated ? launch_stack_variant<T, 1, true, 1>(p, lay, dtype, st)
+                     : launch_stack_variant<T, 1, false, 1>(p, lay, dtype, st);
+    if (vpr <= 2 * kConsumers)  // wide rows: two vectors per thread
+        return gated ? launch_stack_variant<T, 2, true, 1>(p, lay, dtype, st)
+                     : launch_stack_variant<T, 2, false, 1>(p, lay, dtype, st);
     return CLADA_ERR_UNSUPPORTED;
 }
 
@@ -644,7 +558,8 @@ bool ffn_stack_supported(const clada_layer *layers, int L, int B, size_t ws_byte
     stack_smem_plan(di, layers[0].d_model, layers[0].d_ff, layers[0].dtype, act_is_gated(layers[0].activation), &n_stages,
                     &list_cap, &smem, &budget);
     if (n_stages < GS) return false;
-    return ws_bytes >= kWsCtrlBytes + 2 * (size_t)di.num_sms * layers[0].d_model * sizeof(float);
+    const int vpr = layers[0].d_model / (layers[0].dtype == CLADA_F32 ? 4 : 8);
+    return ws_bytes >= kWsCtrlBytes + 2 * (size_t)di.num_sms * ffn_groups(vpr) * layers[0].d_model * sizeof(float);
 }
 
 // One sequence through L validated layers of one shape, dtype and FFN form: launches of up to

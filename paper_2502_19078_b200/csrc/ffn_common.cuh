@@ -155,6 +155,171 @@ constexpr int kFfnThreads = kConsumers + 32;  // + one producer warp
 constexpr int kFfnWarps = kFfnThreads / kWarp;
 constexpr int kMaxStages = 16;
 
+// ---- the consumers' loop over one share of kept neurons (single-sequence kernels) -----------------------
+//
+// The 512 consumer threads work as GROUPS groups of GT = 512 / GROUPS threads.  A group owns every GROUPS-th
+// chunk of GS = 4 consecutive neurons of the share; within a group thread gt owns the 16-byte column vectors
+// gt, gt + GT, ... of every row (x and the partial y of those columns stay in registers).  Per chunk: the gate
+// and up dot products of its four neurons from the staged rows (packed two-wide FMAs), ONE group-wide reduction
+// of the eight values (halving butterfly in the warp, then across the group's warps through shared memory, fixed
+// order), the neuron values, and the four down rows scaled into the partial y.  With two groups one group's
+// reduction latency hides under the other's arithmetic, and a row of at most 256 vectors keeps every thread busy.
+// A group never reads the other group's stages, but it watches each of them land before it moves past.
+// A stage is handed back by the warps of the group that owns its neuron (kConsWarps / GROUPS arrivals per stage;
+// a group needs GS <= n_stages stages at once, which the launch checks).
+constexpr int GS = 4;  // neurons per group-wide reduction
+
+__device__ __forceinline__ void group_sync(int grp, int n_threads) {
+    asm volatile("bar.sync %0, %1;" ::"r"(4 + grp), "r"(n_threads) : "memory");  // named barriers 4, 5
+}
+
+template <typename T, int NV, bool GATED, int GROUPS>
+__device__ __forceinline__ void consume_share(const int my_n, const int act, const uint32_t ring,
+                                              const uint32_t stage_bytes, const uint32_t row_bytes,
+                                              const uint32_t down_off, const uint32_t full0, const uint32_t empty0,
+                                              const int n_stages, int &cs, uint32_t &cpar,
+                                              const float2 (&xr)[NV][Pairs<T>::kPairs], const bool (&vok)[NV],
+                                              float2 (&acc)[NV][Pairs<T>::kPairs], float *s_dot, bool &timed_out,
+                                              unsigned long long *waited_ns = nullptr) {
+    constexpr int P = Pairs<T>::kPairs;
+    constexpr int GT = kConsumers / GROUPS;  // threads per group
+    constexpr int GW = GT / kWarp;           // warps per group
+    constexpr int PER = GW / 4;              // warps each lane adds in the cross-warp sum (4 lanes per value)
+    static_assert(GROUPS == 1 || GROUPS == 2, "one or two consumer groups");
+    const int tid = threadIdx.x, lane = tid & 31;
+    const int grp = tid / GT, gt = tid - grp * GT, gw = gt >> 5;
+    float(*dot)[2 * GS][GW] = reinterpret_cast<float(*)[2 * GS][GW]>(s_dot + (size_t)grp * 2 * 2 * GS * GW);
+    const bool b16 = lane & 16, b8 = lane & 8, b4 = lane & 4;
+    int buf = 0;
+    for (int g0 = 0, chunk = 0; g0 < my_n; g0 += GS, ++chunk) {
+        if (GROUPS > 1 && (chunk & (GROUPS - 1)) != grp) {
+            // The other group's chunk.  Its stages are not read here and not handed back from here, but each
+            // one's copy is seen to land: bulk copies may complete out of order, and a wait by parity for the
+            // NEXT use of a stage would pass at once if this use had not even completed yet.
+#pragma unroll
+            for (int g = 0; g < GS; ++g) {
+                if (g0 + g >= my_n) break;
+                if (!timed_out && !mbar_wait(full0 + 8 * cs, cpar)) timed_out = true;
+                if (++cs == n_stages) {
+                    cs = 0;
+                    cpar ^= 1;
+                }
+            }
+            continue;
+        }
+        float pd[2 * GS];
+        uint32_t st_addr[GS];
+        int st_idx[GS];
+#pragma unroll
+        for (int g = 0; g < GS; ++g) {
+            const int i = g0 + g;
+            float2 sg = make_float2(0.f, 0.f), su = make_float2(0.f, 0.f);
+            st_idx[g] = cs;
+            st_addr[g] = ring + (uint32_t)cs * stage_bytes;
+            if (i < my_n) {
+#ifdef CLADA_STACK_TRACE
+                unsigned long long w0 = 0;
+                if (waited_ns) asm volatile("mov.u64 %0, %globaltimer;" : "=l"(w0));
+#endif
+                if (!timed_out && !mbar_wait(full0 + 8 * cs, cpar)) timed_out = true;
+#ifdef CLADA_STACK_TRACE
+                if (waited_ns) {
+                    unsigned long long w1;
+                    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(w1));
+                    *waited_ns += w1 - w0;
+                }
+#endif
+                if (++cs == n_stages) {
+                    cs = 0;
+                    cpar ^= 1;
+                }
+#pragma unroll
+                for (int k = 0; k < NV; ++k) {
+                    if (!vok[k]) continue;
+                    const uint32_t a = st_addr[g] + (uint32_t)(gt + k * GT) * 16u;
+                    float2 fg[P], fu[P];
+                    Pairs<T>::unpack(lds128(a), fg);
+                    if (GATED) Pairs<T>::unpack(lds128(a + row_bytes), fu);
+#pragma unroll
+                    for (int e = 0; e < P; ++e) {
+                        sg = __ffma2_rn(fg[e], xr[k][e], sg);
+                        if (GATED) su = __ffma2_rn(fu[e], xr[k][e], su);
+                    }
+                }
+            }
+            pd[2 * g] = sg.x + sg.y;
+            pd[2 * g + 1] = su.x + su.y;
+        }
+        // Warp sums of the 8 values by a halving butterfly (9 shuffles): after it every lane of
+        // quad q holds the warp total of value q.  Fixed order, so results repeat bit for bit.
+        float b[4], c[2], v8;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const float send = b16 ? pd[i] : pd[i + 4];
+            b[i] = (b16 ? pd[i + 4] : pd[i]) + __shfl_xor_sync(0xffffffffu, send, 16);
+        }
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+            const float send = b8 ? b[i] : b[i + 2];
+            c[i] = (b8 ? b[i + 2] : b[i]) + __shfl_xor_sync(0xffffffffu, send, 8);
+        }
+        v8 = (b4 ? c[1] : c[0]) + __shfl_xor_sync(0xffffffffu, b4 ? c[0] : c[1], 4);
+        v8 += __shfl_xor_sync(0xffffffffu, v8, 2);
+        v8 += __shfl_xor_sync(0xffffffffu, v8, 1);
+        // lane 4q holds value index: bit4 -> +4, bit3 -> +2, bit2 -> +1
+        if ((lane & 3) == 0) dot[buf][(b16 ? 4 : 0) + (b8 ? 2 : 0) + (b4 ? 1 : 0)][gw] = v8;
+        if (GROUPS == 1)
+            asm volatile("bar.sync 1, %0;" ::"n"(kConsumers) : "memory");
+        else
+            group_sync(grp, GT);
+        // Cross-warp sums: lane l adds PER consecutive warps of value l/4 (4 lanes per value), the quad
+        // finishes by butterfly; then gate lanes form the neuron value h.
+        float tot;
+        if (PER == 4) {
+            const float4 q4 = *reinterpret_cast<const float4 *>(&dot[buf][lane >> 2][(lane & 3) * 4]);
+            tot = (q4.x + q4.y) + (q4.z + q4.w);
+        } else {
+            const float2 q2 = *reinterpret_cast<const float2 *>(&dot[buf][lane >> 2][(lane & 3) * 2]);
+            tot = q2.x + q2.y;
+        }
+        tot += __shfl_xor_sync(0xffffffffu, tot, 1);
+        tot += __shfl_xor_sync(0xffffffffu, tot, 2);
+        const float up = __shfl_xor_sync(0xffffffffu, tot, 4);  // value 2g+1 sits 4 lanes above value 2g
+        const float hval = neuron_value_f(act, tot, up);        // meaningful on lanes 8g..8g+3
+#pragma unroll
+        for (int g = 0; g < GS; ++g) {
+            const float h = __shfl_sync(0xffffffffu, hval, 8 * g);
+            if (g0 + g >= my_n) continue;
+            const float2 h2 = make_float2(h, h);
+#pragma unroll
+            for (int k = 0; k < NV; ++k) {
+                if (!vok[k]) continue;
+                float2 fd[P];
+                Pairs<T>::unpack(lds128(st_addr[g] + down_off + (uint32_t)(gt + k * GT) * 16u), fd);
+#pragma unroll
+                for (int e = 0; e < P; ++e) acc[k][e] = __ffma2_rn(h2, fd[e], acc[k][e]);
+            }
+        }
+        // hand the stages back to the producer
+        __syncwarp();
+        if (lane == 0) {
+#pragma unroll
+            for (int g = 0; g < GS; ++g)
+                if (g0 + g < my_n) mbar_arrive(empty0 + 8 * st_idx[g]);
+        }
+        buf ^= 1;
+    }
+}
+
+// Shared-memory floats consume_share needs for its cross-warp sums (all groups, two buffers each).
+constexpr int kDotFloats = 2 * 2 * GS * kConsWarps;
+
+// Consumer groups for a row of vpr 16-byte vectors: two groups of 256 threads when a group covers the row with one
+// vector per thread (otherwise half the 512 threads would own nothing), else one group of 512.  Measured: with two
+// vectors per thread in two groups (rows of 257-512 vectors) a group holds its four stages twice as long and the
+// 4096-wide layers lose 6 % against one group; at 256 vectors two groups gain 9-13 %.
+__host__ __device__ inline int ffn_groups(int vpr) { return vpr <= kConsumers / 2 ? 2 : 1; }
+
 // Batched decode (clada_ffn_batch.cu): how many sequences the next launch should take (4, 2 or 1 = use
 // the single-sequence kernel), and the launch itself for a tile of 2 or 4 sequences.
 int ffn_batch_tile(const clada_layer *layer, int remaining);

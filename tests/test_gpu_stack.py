@@ -145,12 +145,13 @@ def test_stack_kernel_repeats_on_one_workspace(clada):
 
 
 def test_stack_call_falls_back_to_the_loop(clada):
-    """A batch, or a workspace too small for two partial rows per SM, takes the per-layer loop: same results."""
+    """A batch, or a workspace too small for the stack launch's double-buffered partial rows, takes the per-layer
+    loop: same results."""
     L, d, F = 3, 1024, 600
     w, weights, layers, scores, tau, x = _stack_case(clada, "c2_llama2_7b_layer", d, F, L)
     stack = clada.LayerStack(layers)
     sms = torch.cuda.get_device_properties(0).multi_processor_count
-    small = torch.zeros(256 + sms * d * 4, dtype=torch.uint8, device="cuda")      # one row per SM only
+    small = torch.zeros(256 + sms * 2 * d * 4, dtype=torch.uint8, device="cuda")  # room for one layer's rows only
     y_small = torch.empty(L, 1, d, device="cuda")
     clada.clada_sparse_ffn_decode_layers(stack, x.cuda(), scores.cuda(), tau.cuda(), y_small, small)
     y_stack, y_ref, _ = _run_both(clada, layers, x, scores, tau)
@@ -190,3 +191,47 @@ def test_stack_kernel_full_size_layers(clada, oracle):
             y_or, _, n = oracle.sparse_ffn(wl.to_numpy_bits(xs[t, i, 0]), W_in, V_in, W_out, sc[i, 0], float(tb[0, i]))
             assert n == F - w.k_cut(0.4)
             assert rel_inf(ys[t, i, 0].cpu().numpy(), y_or) <= FFN_TOL_F32, (l, t)
+
+
+@pytest.mark.parametrize("name,d,F", [("v2_gemma_2b_layer", 2048, 16384),      # two consumer groups, ring of 16 stages
+                                      ("c2_llama2_7b_layer", 4096, 11008),     # one group, ring of 9 stages
+                                      ("c5_13b_b16", 5120, 13824)])            # two vectors per thread, 7 stages
+def test_many_launches_back_to_back_at_full_width(clada, name, d, F):
+    """Hundreds of launches queued without a host synchronisation, each CTA's share several times the ring's
+    depth: every launch must give the bits of a launch that ran alone, and no bounded wait may expire.  (Bulk
+    copies complete out of order; a consumer group that moved past a stage before its copy had landed would
+    take the next use's parity for granted -- this is the case that catches it.)"""
+    w = wl.scaled(wl.WORKLOADS[name], d_model=d, d_ff=F)
+    L = 4
+    layers = []
+    for l in range(L):
+        wt = wl.layer_weights(w, l, "cuda")
+        layers.append(clada.Layer(wt["w_gate"], wt["w_up"] if w.activation != 2 else None,
+                                  wt["w_down"].t().contiguous(), activation=w.activation))
+    stack = clada.LayerStack(layers)
+    g = torch.Generator(device="cuda").manual_seed(F)
+    scores = torch.rand(L, 1, F, generator=g, device="cuda") + 0.5
+    tau = torch.empty(1, L, device="cuda")
+    for l in range(L):
+        clada.clada_tau_from_sparsity(scores[l], 0.4, tau[:, l])
+    scale = wl.channel_scale(w, "cuda")
+    x = torch.stack([wl.hidden_states(w, l, "decode", 0, 1, "cuda", scale) for l in range(L)])   # [L, 1, d]
+    ws = clada.new_workspace(layers[0], 1, 0)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    y_alone = torch.empty(L, 1, d, device="cuda")
+    for l in range(L):
+        clada.clada_sparse_ffn_decode(layers[l], x[l], scores[l], tau[:, l], L, y_alone[l], ws, status=status)
+        torch.cuda.synchronize()
+    n_rep = 48
+    y_loop = torch.empty(n_rep, L, 1, d, device="cuda")
+    y_stack = torch.empty(n_rep, L, 1, d, device="cuda")
+    for r in range(n_rep):
+        for l in range(L):
+            clada.clada_sparse_ffn_decode(layers[l], x[l], scores[l], tau[:, l], L, y_loop[r, l], ws, status=status)
+    for r in range(n_rep):
+        clada.clada_sparse_ffn_decode_layers(stack, x, scores, tau, y_stack[r], ws, status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    assert float(y_alone.abs().max()) > 0
+    assert torch.equal(y_loop, y_alone.expand(n_rep, L, 1, d))
+    assert torch.equal(y_stack, y_alone.expand(n_rep, L, 1, d))
