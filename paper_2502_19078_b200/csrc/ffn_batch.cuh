@@ -1,0 +1,178 @@
+// Pieces shared by the two batched decode kernels (CUDA-core tile kernel, tensor-core tile kernel): the launch
+// parameters, the prologue that builds a CTA's share of the union of a tile's kept sets, and the epilogue that
+// sums the CTAs' partial outputs.
+#pragma once
+
+#include "common.cuh"
+#include "ffn_common.cuh"
+
+namespace clada {
+
+struct FfnBatchParams {
+    const void *w_gate, *w_up, *w_down_t;
+    const void *x;           // sequence b at x + b * x_stride (bytes)
+    size_t x_stride;
+    const float *scores;     // [BT, d_ff]
+    const float *tau;        // sequence b at tau[b * tau_stride]
+    long long tau_stride;
+    void *y;                 // sequence b at y + b * y_stride (bytes)
+    size_t y_stride;
+    int y_dtype;
+    float *partials;         // [gridDim.x, BT, d_model]
+    WsCtrl *ctrl;
+    int32_t *status;
+    int d_model, d_ff;
+    int act;                 // clada_activation of the layer
+};
+
+constexpr int kBatchMaxBatches = 4;  // prologue batches: d_ff <= 4 * 32 * kFfnThreads
+
+// Prologue of a tile of BT sequences, run by all kFfnThreads threads of the CTA: every sequence's keep bits
+// A_bj >= tau_b per 32-neuron chunk (s_balb), their union (s_bal), the union's ranks by a block scan, and this
+// CTA's equal share of the union in ascending order: s_list[i] = neuron, s_keep[i] = bit b set iff sequence b
+// keeps it.  s_tau must hold the BT thresholds (visible to all threads).  Returns the share's size.
+template <int BT>
+__device__ __forceinline__ int batch_union_share(const FfnBatchParams &p, const float *s_tau, unsigned *s_bal,
+                                                 unsigned *s_balb, int *s_list, int *s_keep, int *s_wtot,
+                                                 const uint64_t keep_policy) {
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int cta = blockIdx.x, n_ctas = gridDim.x;
+    const int F = p.d_ff;
+    const int chunks = (F + kWarp - 1) / kWarp;
+    // ---- prologue: keep-bits per sequence, their union, ranks of the union -----------------------
+    const int n_batches = (chunks + kFfnThreads - 1) / kFfnThreads;
+    {
+        int slot = tid + (cta * 37) % kFfnThreads;
+        if (slot >= kFfnThreads) slot -= kFfnThreads;
+        for (int bt = 0; bt < n_batches; ++bt) {
+            const int q = bt * kFfnThreads + slot;
+            if (q >= chunks) continue;
+            const int j0 = q * kWarp;
+            unsigned wu = 0;
+#pragma unroll
+            for (int b = 0; b < BT; ++b) {
+                const float *sc = p.scores + (size_t)b * F;
+                const float tau = s_tau[b];
+                unsigned w = 0;
+                if (((reinterpret_cast<uintptr_t>(sc) & 15u) == 0) && j0 + kWarp <= F) {
+                    float4 v[8];
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) v[u] = ld_keep4(reinterpret_cast<const float4 *>(sc + j0) + u, keep_policy);
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) {
+                        w |= (v[u].x >= tau ? 1u : 0u) << (4 * u);
+                        w |= (v[u].y >= tau ? 1u : 0u) << (4 * u + 1);
+                        w |= (v[u].z >= tau ? 1u : 0u) << (4 * u + 2);
+                        w |= (v[u].w >= tau ? 1u : 0u) << (4 * u + 3);
+                    }
+                } else {
+                    for (int u = 0; u < kWarp; ++u)
+                        if (j0 + u < F && ld_keep(sc + j0 + u, keep_policy) >= tau) w |= 1u << u;
+                }
+                s_balb[b * chunks + q] = w;
+                wu |= w;
+            }
+            s_bal[q] = wu;
+        }
+    }
+    __syncthreads();
+    unsigned bal[kBatchMaxBatches];
+    int first_rank[kBatchMaxBatches];
+    int n_act = 0;
+#pragma unroll
+    for (int bt = 0; bt < kBatchMaxBatches; ++bt) {
+        bal[bt] = 0u;
+        first_rank[bt] = 0;
+        if (bt >= n_batches) continue;  // uniform
+        const int q = bt * kFfnThreads + tid;
+        if (q < chunks) bal[bt] = s_bal[q];
+        const int cnt = __popc(bal[bt]);
+        int incl = cnt;
+#pragma unroll
+        for (int o = 1; o < kWarp; o <<= 1) {
+            const int t = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += t;
+        }
+        if (bt > 0) __syncthreads();
+        if (lane == kWarp - 1) s_wtot[warp] = incl;
+        __syncthreads();
+        int wbase = 0, btot = 0;
+#pragma unroll
+        for (int w = 0; w < kFfnWarps; ++w) {
+            const int v = s_wtot[w];
+            wbase += (w < warp) ? v : 0;
+            btot += v;
+        }
+        first_rank[bt] = n_act + wbase + incl - cnt;
+        n_act += btot;
+    }
+    const int r0 = (int)(((int64_t)n_act * cta) / n_ctas);
+    const int r1 = (int)(((int64_t)n_act * (cta + 1)) / n_ctas);
+#pragma unroll
+    for (int bt = 0; bt < kBatchMaxBatches; ++bt) {
+        if (bt >= n_batches) continue;  // uniform
+        const int q = bt * kFfnThreads + tid;
+        const int fr = first_rank[bt];
+        const bool in_share = q < chunks && fr < r1 && fr + __popc(bal[bt]) > r0;
+        unsigned todo = __ballot_sync(0xffffffffu, in_share);
+        while (todo) {
+            const int t = __ffs(todo) - 1;
+            todo &= todo - 1;
+            const unsigned wb = __shfl_sync(0xffffffffu, bal[bt], t);
+            const int wfr = __shfl_sync(0xffffffffu, fr, t);
+            const int qq = bt * kFfnThreads + warp * kWarp + t;
+            const int rank = wfr + __popc(wb & ((1u << lane) - 1u));
+            if (((wb >> lane) & 1u) && rank >= r0 && rank < r1) {
+                int bits = 0;
+#pragma unroll
+                for (int b = 0; b < BT; ++b) bits |= (int)((s_balb[b * chunks + qq] >> lane) & 1u) << b;
+                s_list[rank - r0] = qq * kWarp + lane;
+                s_keep[rank - r0] = bits;
+            }
+        }
+    }
+    return r1 - r0;
+}
+
+// Epilogue of a tile: after the grid barrier every CTA sums a slice of (sequence, column group) pairs over all
+// CTAs' partial rows [n_ctas][BT][d_model] in CTA order (a warp per group of 4 columns: lane l adds rows l,
+// l+32, ..., then the 32 lane sums combine by butterfly) and writes y.
+template <int BT>
+__device__ __forceinline__ void batch_column_sums(const FfnBatchParams &p) {
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int cta = blockIdx.x, n_ctas = gridDim.x, d = p.d_model;
+    const int ngroups = d / 4;
+    for (int it = cta + warp * n_ctas; it < BT * ngroups; it += n_ctas * kFfnWarps) {
+        const int b = it / ngroups, q = it % ngroups;
+        float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int rb = 0; rb < n_ctas; rb += 5 * kWarp) {
+            float4 v[5];
+#pragma unroll
+            for (int u = 0; u < 5; ++u) {
+                const int r = rb + u * kWarp + lane;
+                v[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (r < n_ctas)
+                    v[u] = __ldcg(reinterpret_cast<const float4 *>(p.partials + ((size_t)r * BT + b) * d) + q);
+            }
+#pragma unroll
+            for (int u = 0; u < 5; ++u) {
+                s.x += v[u].x; s.y += v[u].y; s.z += v[u].z; s.w += v[u].w;
+            }
+        }
+        s.x = warp_sum(s.x); s.y = warp_sum(s.y); s.z = warp_sum(s.z); s.w = warp_sum(s.w);
+        if (lane == 0) {
+            char *yb = static_cast<char *>(p.y) + b * p.y_stride;
+            if (p.y_dtype == CLADA_F32) {
+                reinterpret_cast<float4 *>(yb)[q] = s;
+            } else {
+                reinterpret_cast<uint2 *>(yb)[q] = pack4_16bit(p.y_dtype, s);
+            }
+        }
+    }
+}
+
+// The tensor-core tile kernel (clada_ffn_batch_tc.cu): whether it takes this layer and tile, and its launch.
+bool ffn_batch_tc_supported(const clada_layer *layer, int bt);
+int launch_ffn_batch_tc(const FfnBatchParams &p, int dtype, int bt, cudaStream_t st);
+
+}  // namespace clada
