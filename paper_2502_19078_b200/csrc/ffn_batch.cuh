@@ -31,7 +31,7 @@ constexpr int kBatchMaxBatches = 4;  // prologue batches: d_ff <= 4 * 32 * kFfnT
 // A_bj >= tau_b per 32-neuron chunk (s_balb), their union (s_bal), the union's ranks by a block scan, and this
 // CTA's equal share of the union in ascending order: s_list[i] = neuron, s_keep[i] = bit b set iff sequence b
 // keeps it.  s_tau must hold the BT thresholds (visible to all threads).  Returns the share's size.
-template <int BT>
+template <int BT, int NT = kFfnThreads>
 __device__ __forceinline__ int batch_union_share(const FfnBatchParams &p, const float *s_tau, unsigned *s_bal,
                                                  unsigned *s_balb, int *s_list, int *s_keep, int *s_wtot,
                                                  const uint64_t keep_policy) {
@@ -40,12 +40,12 @@ __device__ __forceinline__ int batch_union_share(const FfnBatchParams &p, const 
     const int F = p.d_ff;
     const int chunks = (F + kWarp - 1) / kWarp;
     // ---- prologue: keep-bits per sequence, their union, ranks of the union -----------------------
-    const int n_batches = (chunks + kFfnThreads - 1) / kFfnThreads;
+    const int n_batches = (chunks + NT - 1) / NT;
     {
-        int slot = tid + (cta * 37) % kFfnThreads;
-        if (slot >= kFfnThreads) slot -= kFfnThreads;
+        int slot = tid + (cta * 37) % NT;
+        if (slot >= NT) slot -= NT;
         for (int bt = 0; bt < n_batches; ++bt) {
-            const int q = bt * kFfnThreads + slot;
+            const int q = bt * NT + slot;
             if (q >= chunks) continue;
             const int j0 = q * kWarp;
             unsigned wu = 0;
@@ -84,7 +84,7 @@ __device__ __forceinline__ int batch_union_share(const FfnBatchParams &p, const 
         bal[bt] = 0u;
         first_rank[bt] = 0;
         if (bt >= n_batches) continue;  // uniform
-        const int q = bt * kFfnThreads + tid;
+        const int q = bt * NT + tid;
         if (q < chunks) bal[bt] = s_bal[q];
         const int cnt = __popc(bal[bt]);
         int incl = cnt;
@@ -98,7 +98,7 @@ __device__ __forceinline__ int batch_union_share(const FfnBatchParams &p, const 
         __syncthreads();
         int wbase = 0, btot = 0;
 #pragma unroll
-        for (int w = 0; w < kFfnWarps; ++w) {
+        for (int w = 0; w < (NT / kWarp); ++w) {
             const int v = s_wtot[w];
             wbase += (w < warp) ? v : 0;
             btot += v;
@@ -111,7 +111,7 @@ __device__ __forceinline__ int batch_union_share(const FfnBatchParams &p, const 
 #pragma unroll
     for (int bt = 0; bt < kBatchMaxBatches; ++bt) {
         if (bt >= n_batches) continue;  // uniform
-        const int q = bt * kFfnThreads + tid;
+        const int q = bt * NT + tid;
         const int fr = first_rank[bt];
         const bool in_share = q < chunks && fr < r1 && fr + __popc(bal[bt]) > r0;
         unsigned todo = __ballot_sync(0xffffffffu, in_share);
@@ -120,7 +120,7 @@ __device__ __forceinline__ int batch_union_share(const FfnBatchParams &p, const 
             todo &= todo - 1;
             const unsigned wb = __shfl_sync(0xffffffffu, bal[bt], t);
             const int wfr = __shfl_sync(0xffffffffu, fr, t);
-            const int qq = bt * kFfnThreads + warp * kWarp + t;
+            const int qq = bt * NT + warp * kWarp + t;
             const int rank = wfr + __popc(wb & ((1u << lane) - 1u));
             if (((wb >> lane) & 1u) && rank >= r0 && rank < r1) {
                 int bits = 0;
@@ -137,12 +137,12 @@ __device__ __forceinline__ int batch_union_share(const FfnBatchParams &p, const 
 // Epilogue of a tile: after the grid barrier every CTA sums a slice of (sequence, column group) pairs over all
 // CTAs' partial rows [n_ctas][BT][d_model] in CTA order (a warp per group of 4 columns: lane l adds rows l,
 // l+32, ..., then the 32 lane sums combine by butterfly) and writes y.
-template <int BT>
+template <int BT, int NT = kFfnThreads>
 __device__ __forceinline__ void batch_column_sums(const FfnBatchParams &p) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int cta = blockIdx.x, n_ctas = gridDim.x, d = p.d_model;
     const int ngroups = d / 4;
-    for (int it = cta + warp * n_ctas; it < BT * ngroups; it += n_ctas * kFfnWarps) {
+    for (int it = cta + warp * n_ctas; it < BT * ngroups; it += n_ctas * (NT / kWarp)) {
         const int b = it / ngroups, q = it % ngroups;
         float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
         for (int rb = 0; rb < n_ctas; rb += 5 * kWarp) {

@@ -58,6 +58,10 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
 __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
+#ifndef CLADA_MBAR_SUSPEND_NS
+#define CLADA_MBAR_SUSPEND_NS 1000
+#endif
+constexpr unsigned kMbarSuspendNs = CLADA_MBAR_SUSPEND_NS;  // a try may suspend the thread for about this long
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
     uint32_t ok;
     asm volatile(
@@ -65,7 +69,7 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
         "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(ok)
-        : "r"(bar), "r"(parity), "r"(1000u)  // suspend for at most ~1 us per try
+        : "r"(bar), "r"(parity), "r"(kMbarSuspendNs)
         : "memory");
     return ok != 0;
 }
