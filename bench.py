@@ -410,7 +410,7 @@ class BatchJob:
     mask): prefix statistics of all prompts, then N decode steps of (cogload+adjust for the batch, sparse FFN for
     the batch in tiles of sequences).  Informational: the metric's workload is the single-sequence layer."""
     layers_run = 1
-    ffn_kernel = "sparse_ffn_batch_kernel (one call = all tiles of the batch)"
+    ffn_kernel = "sparse_ffn_batch_tc_kernel (one call = keep words of the batch + all its tiles)"
     N_DECODE = 32      # decode steps per timed step (the workloads' 256-512 would only repeat these)
     N_LOGITS = 8       # distinct logit rows per sequence, cycled
 
@@ -489,7 +489,7 @@ class BatchJob:
     @property
     def launches_per_step(self) -> int:
         tiles = (self.B + self.tile - 1) // self.tile
-        return 7 + self.N * (1 + tiles)
+        return 7 + self.N * (2 + tiles)      # cogload+adjust, keep words, the tiles
 
     def tokens_per_step(self) -> int:
         return self.B * self.N

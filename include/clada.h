@@ -283,8 +283,9 @@ int clada_sparse_ffn_decode_layers(const clada_layer *layers, int32_t L, const v
  *    and enqueues nothing.  Every refusal happens before the first enqueue.
  *  - Batches: the array holds 160 x 8192 fp32 partial outputs, i.e. one row per
  *    (SM, sequence of a tile).  B >= 2 therefore runs in the largest tiles of
- *    sequences (4, 2 or 1 per launch) that fit: on a 148-SM device tiles of 4 up
- *    to d_model 2048, tiles of 2 up to d_model 4096, one sequence per launch
+ *    sequences (4, 2 or 1 per launch) that fit, together with the batch's keep
+ *    bits (4 bytes per sequence and 32 neurons): on a 148-SM device tiles of 4
+ *    up to d_model 2048, tiles of 2 up to d_model 4096, one sequence per launch
  *    above that.  Results per sequence are those of clada_sparse_ffn_decode;
  *    smaller tiles only read the shared weight rows once per tile instead of
  *    once per larger tile.

@@ -459,7 +459,8 @@ static size_t decode_scratch_bytes(const clada_layer *layer, int32_t B, int num_
     // a single sequence's launch writes one row per consumer group; sequences left over after the tiles run singly
     const int rows = tile > 1 ? tile : 1;
     const int single_rows = (tile == 1 || B % tile != 0) ? ffn_groups(vpr) : 1;
-    return kWsCtrlBytes + (size_t)num_sms * (rows > single_rows ? rows : single_rows) * layer->d_model * sizeof(float);
+    return kWsCtrlBytes + (size_t)num_sms * (rows > single_rows ? rows : single_rows) * layer->d_model * sizeof(float) +
+           (tile > 1 ? keep_words_bytes_of(B, layer->d_ff) : 0);  // the batch's keep words sit behind the partial rows
 }
 
 // The launches of a validated decode call whose scratch holds tiles of up to max_tile sequences.
@@ -471,6 +472,19 @@ static int decode_enqueue(const clada_layer *layer, const void *x, int32_t B, co
     const size_t esz = elem_size(layer->dtype);
     const size_t ysz = elem_size(y_dtype);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    // Tiles of sequences: the keep bits of the whole batch are computed once, into the end of the scratch, and
+    // every CTA of every tile launch reads those words instead of testing the score vectors itself.
+    unsigned *words = nullptr;
+    if (decode_tile(layer, B, max_tile) > 1) {
+        DeviceInfo di;
+        rc = device_info(&di);
+        if (rc != CLADA_OK) return rc;
+        const size_t total = decode_scratch_bytes(layer, B, di.num_sms, max_tile);
+        words = reinterpret_cast<unsigned *>(static_cast<char *>(ws) + total - keep_words_bytes_of(B, layer->d_ff));
+        rc = launch_keep_words(scores, B, layer->d_ff, tau_final, tau_stride, words, st);
+        if (rc != CLADA_OK) return rc;
+    }
+    const size_t chunks = (size_t)(layer->d_ff + 31) / 32;
     int b = 0;
     while (b < B) {
         // Tiles of 4 or 2 sequences read each row of the union of their kept sets once.
@@ -485,7 +499,8 @@ static int decode_enqueue(const clada_layer *layer, const void *x, int32_t B, co
             }
             rc = launch_ffn_batch(layer, bt, static_cast<const char *>(x) + (size_t)b * layer->d_model * esz,
                                   scores + (size_t)b * layer->d_ff, tau_final + (size_t)b * tau_stride, tau_stride,
-                                  static_cast<char *>(y) + (size_t)b * layer->d_model * ysz, y_dtype, ws, status, st);
+                                  static_cast<char *>(y) + (size_t)b * layer->d_model * ysz, y_dtype, ws,
+                                  words + (size_t)b * chunks, status, st);
             if (rc != CLADA_OK) return rc;
             b += bt;
             continue;

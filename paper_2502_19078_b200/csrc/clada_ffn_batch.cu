@@ -257,7 +257,59 @@ sparse_ffn_batch_kernel(const FfnBatchParams p, const int n_stages) {
 }
 
 
+// One thread per (sequence, 32-neuron chunk): eight 16-byte loads, one keep word.
+__global__ void __launch_bounds__(256)
+keep_words_kernel(const float *__restrict__ scores, int B, int d_ff, const float *__restrict__ tau,
+                  long long tau_stride, unsigned *__restrict__ words) {
+    pdl_launch_dependents();
+    pdl_wait();
+    const int chunks = (d_ff + kWarp - 1) / kWarp;
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= B * chunks) return;
+    const int b = i / chunks, q = i - b * chunks;
+    const float *sc = scores + (size_t)b * d_ff;
+    const float t = tau[(size_t)b * tau_stride];
+    const int j0 = q * kWarp;
+    unsigned w = 0;
+    if (((reinterpret_cast<uintptr_t>(sc) & 15u) == 0) && j0 + kWarp <= d_ff) {
+        float4 v[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) v[u] = __ldg(reinterpret_cast<const float4 *>(sc + j0) + u);
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            w |= (v[u].x >= t ? 1u : 0u) << (4 * u);
+            w |= (v[u].y >= t ? 1u : 0u) << (4 * u + 1);
+            w |= (v[u].z >= t ? 1u : 0u) << (4 * u + 2);
+            w |= (v[u].w >= t ? 1u : 0u) << (4 * u + 3);
+        }
+    } else {
+        for (int u = 0; u < kWarp; ++u)
+            if (j0 + u < d_ff && sc[j0 + u] >= t) w |= 1u << u;
+    }
+    words[i] = w;
+}
+
 // ---- host side ------------------------------------------------------------------------------
+
+size_t keep_words_bytes_of(int B, int d_ff) { return keep_words_bytes(B, d_ff); }
+
+int launch_keep_words(const float *scores, int B, int d_ff, const float *tau, long long tau_stride, unsigned *words,
+                      cudaStream_t st) {
+    const int chunks = (d_ff + kWarp - 1) / kWarp;
+    const int n = B * chunks;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((n + 255) / 256);
+    cfg.blockDim = dim3(256);
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    void *args[] = {&scores, &B, &d_ff, &tau, &tau_stride, &words};
+    CLADA_CUDA_TRY(cudaLaunchKernelExC(&cfg, reinterpret_cast<const void *>(keep_words_kernel), args));
+    return CLADA_OK;
+}
 
 template <typename T, int NV, int BT>
 static int launch_batch_variant(const FfnBatchParams &p, cudaStream_t st) {
@@ -308,7 +360,8 @@ int ffn_batch_tile(const clada_layer *layer, int remaining) {
 }
 
 int launch_ffn_batch(const clada_layer *layer, int bt, const void *x, const float *scores, const float *tau,
-                     long long tau_stride, void *y, int y_dtype, void *ws, int32_t *status, cudaStream_t st) {
+                     long long tau_stride, void *y, int y_dtype, void *ws, const unsigned *keep_words,
+                     int32_t *status, cudaStream_t st) {
     FfnBatchParams p;
     p.w_gate = layer->w_gate;
     p.w_up = layer->w_up;
@@ -316,6 +369,7 @@ int launch_ffn_batch(const clada_layer *layer, int bt, const void *x, const floa
     p.x = x;
     p.x_stride = (size_t)layer->d_model * elem_size(layer->dtype);
     p.scores = scores;
+    p.keep_words = keep_words;
     p.tau = tau;
     p.tau_stride = tau_stride;
     p.y = y;

@@ -119,6 +119,7 @@ sparse_ffn_batch_tc_kernel(const FfnBatchParams p, const int n_stages) {
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     pdl_wait();
+    TC_TRACE(255, 0);
 
     const uint64_t keep_policy = policy_evict_last();
     if (tid < BT) s_tau[tid] = ld_keep(p.tau + (size_t)tid * p.tau_stride, keep_policy);
@@ -130,6 +131,7 @@ sparse_ffn_batch_tc_kernel(const FfnBatchParams p, const int n_stages) {
 
     const int my_n = batch_union_share<BT, kConsumers>(p, s_tau, s_bal, s_balb, s_list, s_keep, s_wtot, keep_policy);
     __syncthreads();  // list, keep bits and the mbarriers are ready
+    TC_TRACE(255, 1);
 
     // ---- the copies (thread 0) -----------------------------------------------------------------------------
     // Warp 0 issues: lane l copies row l % n_rows of neuron first + l / n_rows (one bulk copy per lane, so a
@@ -164,6 +166,7 @@ sparse_ffn_batch_tc_kernel(const FfnBatchParams p, const int n_stages) {
             afrag[j] = *(reinterpret_cast<const uint4 *>(static_cast<const char *>(p.x) + g * p.x_stride) + v);
     }
 
+    TC_TRACE(255, 2);
     bool timed_out = false;
     float2 acc[BT][NV][P];
 #pragma unroll
@@ -269,6 +272,7 @@ sparse_ffn_batch_tc_kernel(const FfnBatchParams p, const int n_stages) {
         }
         TC_TRACE(g0 / CH, 6);
     }
+    TC_TRACE(255, 3);
     // Never leave with copies in flight.  Every copy issued was waited for above, unless a wait gave up: then
     // thread 0 waits (bounded again) for the last ring's worth.
     if (timed_out && tid == 0) {
@@ -288,13 +292,16 @@ sparse_ffn_batch_tc_kernel(const FfnBatchParams p, const int n_stages) {
         }
     }
     if (timed_out && p.status) atomicOr(p.status, CLADA_STATUS_TIMEOUT);
+    TC_TRACE(255, 4);
 
     // ---- epilogue: grid barrier, deterministic column reduction per sequence ----------------------
     if (!grid_barrier(p.ctrl, (unsigned)n_ctas, kWarp)) {
         if (tid == 0 && p.status) atomicOr(p.status, CLADA_STATUS_TIMEOUT);
         return;
     }
+    TC_TRACE(255, 5);
     batch_column_sums<BT, kConsumers>(p);
+    TC_TRACE(255, 6);
 }
 
 // ---- host side ------------------------------------------------------------------------------

@@ -131,8 +131,10 @@ size_t clada_workspace_bytes(const clada_layer *layer, int32_t B, int64_t T_tota
     DeviceInfo di;
     int sms = 148;
     if (device_info(&di) == CLADA_OK) sms = di.num_sms;
-    // decode: one fp32 partial output row per persistent CTA (at most 4 CTAs per SM)
-    size_t decode = (size_t)sms * 4 * (size_t)layer->d_model * sizeof(float);
+    // decode: at most four fp32 partial output rows per persistent CTA (a tile of 4 sequences; two consumer groups
+    // in two buffers for the stack launch), then the keep words of the batch (4 bytes per sequence and 32 neurons)
+    size_t decode = (size_t)sms * 4 * (size_t)layer->d_model * sizeof(float) +
+                    ((((size_t)B * ((size_t)(layer->d_ff + 31) / 32) * sizeof(unsigned)) + 255) & ~(size_t)255);
     // prefix: one fp32 partial sum of squares per (token tile, neuron); tiles hold 64 tokens
     size_t tiles = (size_t)(T_total / 64) + (size_t)B + 1;
     size_t prefix = (tiles * (size_t)layer->d_ff * sizeof(float) + 255) & ~(size_t)255;

@@ -13,6 +13,7 @@ struct FfnBatchParams {
     const void *x;           // sequence b at x + b * x_stride (bytes)
     size_t x_stride;
     const float *scores;     // [BT, d_ff]
+    const unsigned *keep_words;  // [BT, chunks] keep bits A_bj >= tau_b per 32-neuron chunk, or null: test the scores here
     const float *tau;        // sequence b at tau[b * tau_stride]
     long long tau_stride;
     void *y;                 // sequence b at y + b * y_stride (bytes)
@@ -51,9 +52,15 @@ __device__ __forceinline__ int batch_union_share(const FfnBatchParams &p, const 
             unsigned wu = 0;
 #pragma unroll
             for (int b = 0; b < BT; ++b) {
+                unsigned w = 0;
+                if (p.keep_words) {  // the words of the whole batch were computed once by keep_words_kernel
+                    w = p.keep_words[(size_t)b * chunks + q];
+                    s_balb[b * chunks + q] = w;
+                    wu |= w;
+                    continue;
+                }
                 const float *sc = p.scores + (size_t)b * F;
                 const float tau = s_tau[b];
-                unsigned w = 0;
                 if (((reinterpret_cast<uintptr_t>(sc) & 15u) == 0) && j0 + kWarp <= F) {
                     float4 v[8];
 #pragma unroll
@@ -169,6 +176,14 @@ __device__ __forceinline__ void batch_column_sums(const FfnBatchParams &p) {
             }
         }
     }
+}
+
+// Keep bits of a whole batch, once per decode call: words[b][q] bit u = (scores[b][32 q + u] >= tau_b).  Every CTA
+// of every tile launch then reads 4 bytes per (sequence, chunk) instead of testing 128 bytes of scores.
+int launch_keep_words(const float *scores, int B, int d_ff, const float *tau, long long tau_stride, unsigned *words,
+                      cudaStream_t st);
+inline size_t keep_words_bytes(int B, int d_ff) {
+    return (((size_t)B * ((d_ff + 31) / 32) * sizeof(unsigned)) + 255) & ~(size_t)255;
 }
 
 // The tensor-core tile kernel (clada_ffn_batch_tc.cu): whether it takes this layer and tile, and its launch.

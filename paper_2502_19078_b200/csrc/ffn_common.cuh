@@ -328,7 +328,13 @@ __host__ __device__ inline int ffn_groups(int vpr) { return vpr <= kConsumers / 
 // the single-sequence kernel), and the launch itself for a tile of 2 or 4 sequences.
 int ffn_batch_tile(const clada_layer *layer, int remaining);
 int launch_ffn_batch(const clada_layer *layer, int bt, const void *x, const float *scores, const float *tau,
-                     long long tau_stride, void *y, int y_dtype, void *ws, int32_t *status, cudaStream_t st);
+                     long long tau_stride, void *y, int y_dtype, void *ws, const unsigned *keep_words,
+                     int32_t *status, cudaStream_t st);
+// Keep bits of a whole batch for the tile launches (clada_ffn_batch.cu): the kernel's launch and the bytes of
+// workspace its output takes (a multiple of 256).
+int launch_keep_words(const float *scores, int B, int d_ff, const float *tau, long long tau_stride, unsigned *words,
+                      cudaStream_t st);
+size_t keep_words_bytes_of(int B, int d_ff);
 
 // One sequence through a stack of layers in one persistent launch (clada_ffn_stack.cu): whether the stack
 // kernel takes this call (one sequence, at least two layers of one FFN form, a workspace with two partial
