@@ -183,14 +183,13 @@ sparse_ffn_batch_tc_kernel(const FfnBatchParams p, const int n_stages) {
     for (int g0 = 0; g0 < my_n; g0 += CH) {
         const int nn = min(CH, my_n - g0);
         TC_TRACE(g0 / CH, 0);
-        // the chunk's stages
-        uint32_t st_addr[CH];
+        // the chunk's stages: neuron q of the chunk sits in stage s0 + q (wrapped)
+        const int s0 = cs;
         {
             int s = cs;
             uint32_t par = cpar;
 #pragma unroll
             for (int q = 0; q < CH; ++q) {
-                st_addr[q] = ring + (uint32_t)s * stage_bytes;
                 if (q < nn) {
                     if (!timed_out && !mbar_wait(full0 + 8 * s, par)) timed_out = true;
                     if (++s == n_stages) {
@@ -202,16 +201,16 @@ sparse_ffn_batch_tc_kernel(const FfnBatchParams p, const int n_stages) {
             cs = s;
             cpar = par;
         }
+        auto stage_addr = [&](int q) {
+            const int s = s0 + q;
+            return ring + (uint32_t)(s < n_stages ? s : s - n_stages) * stage_bytes;
+        };
         TC_TRACE(g0 / CH, 1);
         // ---- gate | up of four neurons for all sequences: one chain of warp-level MMAs per accumulator ----
         float d0[4] = {0.f, 0.f, 0.f, 0.f}, d1[4] = {0.f, 0.f, 0.f, 0.f};
         {
             const bool row_ok = nb < nn && (g < 4 || gated);
-            uint32_t brow = st_addr[0];
-            if (CH > 1 && nb == 1) brow = st_addr[1];
-            if (CH > 2 && nb == 2) brow = st_addr[2];
-            if (CH > 3 && nb == 3) brow = st_addr[3];
-            brow += b_off;
+            const uint32_t brow = stage_addr(nb) + b_off;
 #pragma unroll
             for (int j = 0; j < NPS; ++j) {
                 const int v = 4 * (warp + kConsWarps * j) + t;
@@ -263,7 +262,7 @@ sparse_ffn_batch_tc_kernel(const FfnBatchParams p, const int n_stages) {
             for (int k = 0; k < NV; ++k) {
                 if (!vok[k]) continue;
                 float2 fd[P];
-                Pairs<T>::unpack(lds128(st_addr[q] + down_off + (uint32_t)(tid + k * kConsumers) * 16u), fd);
+                Pairs<T>::unpack(lds128(stage_addr(q) + down_off + (uint32_t)(tid + k * kConsumers) * 16u), fd);
 #pragma unroll
                 for (int b = 0; b < BT; ++b)
 #pragma unroll
