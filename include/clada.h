@@ -248,7 +248,12 @@ int clada_cogload_adjust(const void *logits, int32_t logits_dtype, int32_t B, in
  *   y        out [B, d_model], y_dtype fp32, bf16 or fp16
  *   mask_out / idx_out / count_out: optional (NULL), as in clada_select
  * Accumulation is fp32 in a fixed order: results are bit-identical run to run.
- * The workspace must have been initialised with clada_workspace_init. */
+ * A batch runs in tiles of 4 or 2 sequences that read the union of their kept
+ * rows once (16-bit layers: gate / up contractions on the tensor cores with
+ * short fp32 accumulation chains, same 1e-5 as the CUDA-core path), preceded by
+ * one small launch that tests the batch's scores once.
+ * The workspace (clada_workspace_bytes(layer, B, 0) bytes at least) must have
+ * been initialised with clada_workspace_init. */
 int clada_sparse_ffn_decode(const clada_layer *layer, const void *x, int32_t B,
                             const float *scores /*[B,d_ff]*/, const float *tau_final,
                             int64_t tau_stride, void *y, int32_t y_dtype,
@@ -257,13 +262,19 @@ int clada_sparse_ffn_decode(const clada_layer *layer, const void *x, int32_t B,
 
 /* Algorithm 2's sparse forward pass over a stack of L layers for one decode
  * step: clada_sparse_ffn_decode for l = 0 .. L-1 in one call.
- *   layers     HOST array of L layers of one shape and dtype
+ *   layers     HOST array of L layers of one shape, dtype and FFN form
  *   x          [L, B, d_model]: the input hidden state of every layer (this path has
  *              no attention, residual or norm between FFNs, so each layer's input is given)
  *   scores     [L, B, d_ff]
  *   tau_final  [B, L] as clada_adjust_threshold writes it
  *   y          out [L, B, d_model]
- * All layers are validated before anything is enqueued. */
+ * All layers are validated before anything is enqueued.
+ * One sequence (B = 1, L >= 2) runs all layers in ONE persistent launch (up to
+ * 128 layers per launch): the weight stream does not stop at layer
+ * boundaries, the outputs are bit for bit those of the per-layer call.  This
+ * needs the workspace clada_workspace_bytes(layer, 1, 0) gives; with a smaller
+ * one, for a batch, or for rows too wide for a ring of four stages
+ * (d_model 8192 in 16-bit types) the call runs the per-layer launches in a loop. */
 int clada_sparse_ffn_decode_layers(const clada_layer *layers, int32_t L, const void *x, int32_t B,
                                    const float *scores, const float *tau_final, void *y,
                                    int32_t y_dtype, void *ws, size_t ws_bytes, int32_t *status,
