@@ -408,9 +408,9 @@ class StackJob:
 class BatchJob:
     """One layer of a batched workload (c4: 8 sequences, c5: 16, each with its own prompt, scores, threshold and
     mask): prefix statistics of all prompts, then N decode steps of (cogload+adjust for the batch, sparse FFN for
-    the batch in tiles of sequences).  Informational: the metric's workload is the single-sequence layer."""
+    the batch: one dense pass over the layer per 16 sequences).  Informational: the metric's workload is the
+    single-sequence layer."""
     layers_run = 1
-    ffn_kernel = "sparse_ffn_batch_tc_kernel (one call = keep words of the batch + all its tiles)"
     N_DECODE = 32      # decode steps per timed step (the workloads' 256-512 would only repeat these)
     N_LOGITS = 8       # distinct logit rows per sequence, cycled
 
@@ -458,15 +458,30 @@ class BatchJob:
         torch.cuda.synchronize()
         self.tau_s = wl.universal_threshold(self.s.flatten().tolist())
         self.tau_H = wl.universal_threshold(self.h.flatten().tolist())
-        # rows one layer-step at the baseline thresholds has to read: the union of a tile's kept sets, per tile
-        bt = 4 if w.d_model * w.elem_bytes <= 8192 else 2
+        # Rows one layer-step at the baseline thresholds has to read: per launch, the union of the kept sets of the
+        # launch's sequences (the library takes 16 sequences per dense pass from 5 sequences on -- the pass reads
+        # every row of the layer, its union or not -- and tiles of 4 or 2 below that).
+        tile = 4 if w.d_model * w.elem_bytes <= 8192 else 2
+        self.launch_sizes, rest = [], B
+        while rest > 0:
+            n = min(rest, 16) if rest >= 5 and w.dtype != "f32" else min(rest, tile)
+            self.launch_sizes.append(n)
+            rest -= n
         m = self.mask.bool()
-        self.union_rows = sum(int(m[b0:b0 + bt].any(dim=0).sum()) for b0 in range(0, B, bt))
-        self.tile = bt
+        self.union_rows, b0 = 0, 0
+        for n in self.launch_sizes:
+            self.union_rows += int(m[b0:b0 + n].any(dim=0).sum())
+            b0 += n
+        self.dense = max(self.launch_sizes) > 4
 
+    ffn_kernel = property(lambda self: "sparse_ffn_batch_dense_kernel (one call = one dense pass per 16 sequences)"
+                          if self.dense else
+                          "sparse_ffn_batch_tc_kernel (one call = keep words of the batch + all its tiles)")
     step_note = property(lambda self: f"prefix statistics, guard band, select for {self.B} prompts; then {self.N} x "
-                                      f"(cogload+adjust for the batch, sparse FFN in tiles of {self.tile} sequences)")
-    l2_note = "inputs larger than L2: every layer-step streams the union of its tiles' kept rows (see bytes_per_launch)"
+                                      f"(cogload+adjust for the batch, sparse FFN for the batch in launches of "
+                                      f"{self.launch_sizes} sequences)")
+    l2_note = ("inputs larger than L2: every layer-step streams the layer (dense pass) or the union of its tiles' "
+               "kept rows (see bytes_per_launch)")
     ffn_launches_per_loop = property(lambda self: self.N)
     prefix_flop = property(lambda self: (2.0 if self.w.activation == 2 else 4.0) * self.T * self.w.d_model * self.w.d_ff)
 
@@ -488,8 +503,8 @@ class BatchJob:
 
     @property
     def launches_per_step(self) -> int:
-        tiles = (self.B + self.tile - 1) // self.tile
-        return 7 + self.N * (2 + tiles)      # cogload+adjust, keep words, the tiles
+        keep_words = 0 if all(n > 4 or n == 1 for n in self.launch_sizes) else 1
+        return 7 + self.N * (1 + keep_words + len(self.launch_sizes))      # cogload+adjust, keep words, the FFN launches
 
     def tokens_per_step(self) -> int:
         return self.B * self.N
@@ -555,7 +570,8 @@ def _timed(fn, steps, dist_barrier):
 def other_workloads_info(clada, dev, stream, use_graph, peak, read_gbs):
     """FFN-only figures on the other workloads' layers, for information: the 32-layer stack (eight tokens, one
     persistent launch per token, and the same passes as one launch per layer) and one layer of each batched
-    workload (the batch's call = its tiles of sequences, bytes = the union of each tile's kept rows)."""
+    workload (the batch's call = one dense pass per 16 sequences; bytes = the union of the kept rows of each
+    launch's sequences, which the pass reads along with the few rows nobody keeps)."""
     out = {}
     for name in ("c3_llama2_7b_stack", "c4_llama3_8b_b8", "c5_13b_b16"):
         w = wl.WORKLOADS[name]
@@ -564,7 +580,7 @@ def other_workloads_info(clada, dev, stream, use_graph, peak, read_gbs):
         kept = w.d_ff - w.k_cut(w.sparsities[0])
         if w.batch > 1:
             nbytes = job.ffn_bytes_per_launch
-            rec = {"kernel": job.ffn_kernel, "layers_run": 1, "batch": w.batch, "tile": job.tile,
+            rec = {"kernel": job.ffn_kernel, "layers_run": 1, "batch": w.batch, "sequences_per_launch": job.launch_sizes,
                    "sparsity": w.sparsities[0], "us_per_batch_call": t_ms * 1e3, "bytes_per_batch_call": nbytes,
                    "union_rows": job.union_rows}
         else:

@@ -29,17 +29,15 @@
 
 #include "common.cuh"
 #include "prefix_common.cuh"
+#include "tc_common.cuh"
 
 namespace clada {
 
-constexpr int kTcTileM = 128;   // rows of the A tile = TMEM lanes (tokens; also the most neurons per tile)
-constexpr int kTcTileK = 64;    // K block: 64 16-bit elements = 128 bytes = one swizzle row
 constexpr int kTcMaxStages = 8;
 constexpr int kTcThreads = 192;
 constexpr uint32_t kTcTileBytes = kTcTileM * kTcTileK * 2;       // 16 KiB: a 128-row tile
 constexpr uint32_t kTcRingBytes = 192 * 1024;                    // shared-memory ring of the statistics kernel
 constexpr uint32_t kTcTmemCols = 512;                            // two accumulators of up to 256 columns
-constexpr unsigned kTcSpinLimit = 1u << 20;
 
 struct TcParams {
     int d_model, d_ff;
@@ -59,84 +57,6 @@ struct TcParams {
     int act;        // clada_activation; the non-gated form skips the w_up tiles and their MMAs
     SeqTable tab;
 };
-
-__device__ __forceinline__ uint32_t tc_smem_u32(const void *p) {
-    return static_cast<uint32_t>(__cvta_generic_to_shared(p));
-}
-__device__ __forceinline__ void tc_mbar_init(uint32_t bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void tc_mbar_arrive(uint32_t bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void tc_mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-// Bounded wait for the phase of the given parity; false if it gave up or another role raised the
-// abort flag.  Each try suspends for at most ~1 us (the hint), so the bound is about a second.
-__device__ __forceinline__ bool tc_mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag) {
-    for (unsigned i = 0; i < kTcSpinLimit; ++i) {
-        uint32_t ok;
-        asm volatile(
-            "{\n\t.reg .pred p;\n\t"
-            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
-            "selp.u32 %0, 1, 0, p;\n\t}"
-            : "=r"(ok)
-            : "r"(bar), "r"(parity), "r"(1000u)
-            : "memory");
-        if (ok) return true;
-        if (*abort_flag) return false;
-    }
-    return false;
-}
-// 2-D tiled TMA load (no multicast): box {64 elements, 128 rows} at element c0 of row c1.
-__device__ __forceinline__ void tc_tma_load(uint32_t dst, const CUtensorMap *map, int c0, int c1, uint32_t bar) {
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-        ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1)
-        : "memory");
-}
-// Shared-memory matrix descriptor: K-major tile of 128-byte rows, 128-byte swizzle, 8-row groups
-// 1024 bytes apart (stride byte offset), version 1 (sm_100).  Fields are in 16-byte units.
-__device__ __forceinline__ uint64_t tc_smem_desc(uint32_t addr) {
-    uint64_t d = 0;
-    d |= (uint64_t)((addr >> 4) & 0x3fffu);  // start address
-    d |= (uint64_t)1 << 16;                  // leading byte offset (unused with swizzle): 1
-    d |= (uint64_t)(1024 >> 4) << 32;        // stride byte offset
-    d |= (uint64_t)1 << 46;                  // descriptor version
-    d |= (uint64_t)2 << 61;                  // SWIZZLE_128B
-    return d;
-}
-// Instruction descriptor, kind::f16: D fp32, A and B of one 16-bit type (format code 1 = bf16, 0 = fp16,
-// the same for both operands), both K-major, N = 128, M = 128.
-__host__ __device__ constexpr uint32_t tc_instr_desc(int dtype, int n_cols) {
-    return (1u << 4) | (dtype == CLADA_F16 ? 0u : ((1u << 7) | (1u << 10))) | ((uint32_t)(n_cols >> 3) << 17) |
-           ((uint32_t)(kTcTileM >> 4) << 24);
-}
-__device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t accumulate,
-                                       uint32_t idesc) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
-        : "memory");
-}
-// Arrive on an mbarrier once all MMAs issued so far by this thread have completed.
-__device__ __forceinline__ void tc_commit(uint32_t bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_ld16(uint32_t taddr, uint32_t (&r)[16]) {
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
-        : "r"(taddr));
-}
-__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-
 
 __global__ void __launch_bounds__(kTcThreads, 1)
 prefix_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_wg,
@@ -382,43 +302,6 @@ prefix_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
 
 
 // ---- host side ------------------------------------------------------------------------------
-
-typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
-                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-// The driver's tensor-map encoder, fetched through the runtime (the library does not link libcuda).
-static int encode_fn(EncodeTiledFn *out) {
-    static EncodeTiledFn cached = nullptr;
-    if (!cached) {
-        void *fn = nullptr;
-        cudaDriverEntryPointQueryResult q;
-        CLADA_CUDA_TRY(cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q));
-        if (q != cudaDriverEntryPointSuccess || !fn) return CLADA_ERR_UNSUPPORTED;
-        cached = reinterpret_cast<EncodeTiledFn>(fn);
-    }
-    *out = cached;
-    return CLADA_OK;
-}
-
-// Row-major bf16 or fp16 matrix [rows, cols] as a 2-D tensor map with a {64, box_rows} box and 128-byte swizzle;
-// out-of-range rows and columns read as zero.
-static int make_map(EncodeTiledFn enc, CUtensorMap *map, const void *base, long long rows, int cols, int dtype,
-                    int box_rows = kTcTileM) {
-    const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
-    const cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
-    const cuuint32_t box[2] = {(cuuint32_t)kTcTileK, (cuuint32_t)box_rows};
-    const cuuint32_t estr[2] = {1, 1};
-    const CUtensorMapDataType et = dtype == CLADA_F16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
-    const CUresult r = enc(map, et, 2, const_cast<void *>(base), dims, strides, box, estr,
-                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    if (r != CUDA_SUCCESS) {
-        set_last_cuda_error(cudaErrorInvalidValue, "cuTensorMapEncodeTiled");
-        return CLADA_ERR_CUDA;
-    }
-    return CLADA_OK;
-}
 
 int run_prefix_partials_tc(const clada_layer *layer, const void *X, const SeqTable &tab, long long T_total,
                            float *partials, int32_t *status, cudaStream_t st, void *z_out) {

@@ -2,7 +2,10 @@
 #include <stdio.h>
 #include <string.h>
 
+#include <algorithm>
+
 #include "common.cuh"
+#include "ffn_batch.cuh"
 
 namespace clada {
 
@@ -135,6 +138,12 @@ size_t clada_workspace_bytes(const clada_layer *layer, int32_t B, int64_t T_tota
     // in two buffers for the stack launch), then the keep words of the batch (4 bytes per sequence and 32 neurons)
     size_t decode = (size_t)sms * 4 * (size_t)layer->d_model * sizeof(float) +
                     ((((size_t)B * ((size_t)(layer->d_ff + 31) / 32) * sizeof(unsigned)) + 255) & ~(size_t)255);
+    // a dense pass over the layer for 5-16 sequences: a partial output per group of CTAs and the groups' hidden activations
+    if (B >= kDenseMinSeqs) {
+        const size_t dense = ffn_batch_dense_scratch_bytes(layer, B < kDenseMaxSeqs ? B : kDenseMaxSeqs);
+        // sequences past a multiple of 16 may still run as tiles, whose keep words sit behind the launch scratch
+        decode = std::max(decode, dense + ((((size_t)B * ((size_t)(layer->d_ff + 31) / 32) * sizeof(unsigned)) + 255) & ~(size_t)255));
+    }
     // prefix: one fp32 partial sum of squares per (token tile, neuron); tiles hold 64 tokens
     size_t tiles = (size_t)(T_total / 64) + (size_t)B + 1;
     size_t prefix = (tiles * (size_t)layer->d_ff * sizeof(float) + 255) & ~(size_t)255;

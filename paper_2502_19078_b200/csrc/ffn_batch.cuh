@@ -190,4 +190,14 @@ inline size_t keep_words_bytes(int B, int d_ff) {
 bool ffn_batch_tc_supported(const clada_layer *layer, int bt);
 int launch_ffn_batch_tc(const FfnBatchParams &p, int dtype, int bt, cudaStream_t st);
 
+// The dense pass for 4-16 sequences of a 16-bit layer (clada_ffn_batch_dense.cu): every row of the layer is read
+// once for the whole launch.  Below kDenseMinSeqs sequences the union of the kept sets leaves enough of the layer
+// out for the tile kernels, which read only the union, to win.
+constexpr int kDenseMinSeqs = 5;
+constexpr int kDenseMaxSeqs = 16;
+bool ffn_batch_dense_supported(const clada_layer *layer, int B);
+size_t ffn_batch_dense_scratch_bytes(const clada_layer *layer, int B);
+int launch_ffn_batch_dense(const clada_layer *layer, int B, const void *x, const float *scores, const float *tau,
+                           long long tau_stride, void *y, int y_dtype, void *ws, int32_t *status, cudaStream_t st);
+
 }  // namespace clada

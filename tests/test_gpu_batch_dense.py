@@ -1,0 +1,129 @@
+"""GPU parity of the dense pass of batched decode: 5-16 sequences of a 16-bit layer go through the layer in one
+launch (tensor cores, per-sequence masks applied to the hidden activations), every sequence compared with the
+oracle's masked FFN for its own scores and threshold.  Same tolerances as the other FFN parity tests.
+"""
+import numpy as np
+import pytest
+import torch
+
+from paper_2502_19078_b200 import workloads as wl
+from tests._util import gpu_layer, oracle_weights, rel_inf
+
+pytestmark = pytest.mark.gpu
+
+FFN_TOL_F32 = 1e-5
+FFN_TOL_16_OUT = 2e-2
+
+
+@pytest.fixture(scope="module")
+def clada():
+    from paper_2502_19078_b200 import binding, build
+    build.build()
+    binding.load()
+    return binding
+
+
+def _case(clada, oracle, name, kw, B, act=0, y_dtypes=(torch.float32,), seed=0, outputs=False):
+    w = wl.scaled(wl.WORKLOADS[name], batch=B, **kw)
+    d, F = w.d_model, w.d_ff
+    weights = wl.layer_weights(w, 0)
+    layer = gpu_layer(weights, clada, activation=act)
+    W_in, V_in, W_out = oracle_weights(weights, act)
+    rng = np.random.default_rng(seed + 1000 * B + d + F)
+    scores = (rng.random((B, F)) + 0.5).astype(np.float32)
+    taus = (0.7 + 0.6 * rng.random(B)).astype(np.float32)
+    taus[1] = np.inf          # keeps nothing
+    taus[2] = 0.0             # keeps everything
+    xs = torch.stack([wl.hidden_states(w, 0, "decode", b, 1)[0] for b in range(B)])
+    ws = clada.new_workspace(layer, B, 0)
+    sc_d, tau_d = torch.from_numpy(scores).cuda(), torch.from_numpy(taus).cuda()
+    expected = [oracle.sparse_ffn(wl.to_numpy_bits(xs[b]), W_in, V_in, W_out, scores[b].astype(np.float64),
+                                  float(taus[b]), act=act) for b in range(B)]
+    for y_dtype in y_dtypes:
+        tol = FFN_TOL_F32 if y_dtype == torch.float32 else FFN_TOL_16_OUT
+        y = torch.full((B, d), float("nan"), dtype=y_dtype, device="cuda")
+        status = torch.zeros(1, dtype=torch.int32, device="cuda")
+        if outputs:
+            mask = torch.empty(B, F, dtype=torch.uint8, device="cuda")
+            idx = torch.full((B, F), -1, dtype=torch.int32, device="cuda")
+            count = torch.empty(B, dtype=torch.int32, device="cuda")
+            clada.clada_sparse_ffn_decode(layer, xs.cuda(), sc_d, tau_d, 1, y, ws, mask, idx, count, status)
+        else:
+            clada.clada_sparse_ffn_decode(layer, xs.cuda(), sc_d, tau_d, 1, y, ws, None, None, None, status)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        worst = 0.0
+        for b in range(B):
+            y_or, m_or, n_or = expected[b]
+            if outputs:
+                assert int(count[b]) == n_or
+                np.testing.assert_array_equal(mask[b].cpu().numpy(), m_or)
+            got = y[b].float().cpu().numpy()
+            assert np.all(np.isfinite(got)), b
+            if n_or == 0:
+                assert np.all(got == 0), b
+            else:
+                err = rel_inf(got, y_or)
+                worst = max(worst, err)
+                assert err <= tol, (b, y_dtype, err)
+        # the same call again gives the same bits (fixed summation orders, counters back at zero)
+        y2 = torch.empty_like(y)
+        clada.clada_sparse_ffn_decode(layer, xs.cuda(), sc_d, tau_d, 1, y2, ws, None, None, None, status)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0 and torch.equal(y, y2)
+    return worst
+
+
+@pytest.mark.parametrize("name,kw,B", [
+    ("c4_llama3_8b_b8", {"d_model": 1024, "d_ff": 1800}, 8),      # 13 neurons per CTA, 8 column tiles
+    ("c5_13b_b16", {"d_model": 5120, "d_ff": 700}, 16),           # 40 column tiles, 10 per member
+    ("c2_llama2_7b_layer", {"d_model": 520, "d_ff": 777}, 5),     # d_model not a multiple of 64: ragged K block, ragged tile
+    ("c2_llama2_7b_layer", {"d_model": 64, "d_ff": 100}, 6),      # fewer neurons than CTAs, one column tile
+    ("c4_llama3_8b_b8", {"d_model": 2048, "d_ff": 9000}, 9),      # 61 neurons per CTA: three padded rows per box
+    ("c4_llama3_8b_b8", {"d_model": 256, "d_ff": 18900}, 7),      # 128 neurons per CTA, the most a launch takes
+])
+def test_dense_pass_matches_oracle(clada, oracle, name, kw, B):
+    _case(clada, oracle, name, kw, B, y_dtypes=(torch.float32, torch.bfloat16), outputs=(B == 8))
+
+
+@pytest.mark.parametrize("B", [17, 20, 33])
+def test_batches_beyond_sixteen_sequences(clada, oracle, B):
+    """16 sequences per dense launch; what is left over runs densely too (5 or more), as tiles, or singly."""
+    _case(clada, oracle, "c2_llama2_7b_layer", {"d_model": 1024, "d_ff": 1500}, B, outputs=True)
+
+
+@pytest.mark.parametrize("act", [1, 2])
+def test_dense_pass_other_ffn_forms(clada, oracle, act):
+    _case(clada, oracle, "v1_opt_2p7b_layer", {"d_ff": 1300}, 8, act=act)
+
+
+def test_dense_pass_fp16_layer(clada, oracle):
+    _case(clada, oracle, "c5_13b_b16", {"d_model": 1024, "d_ff": 2100, "dtype": "f16"}, 12,
+          y_dtypes=(torch.float32, torch.float16))
+
+
+def test_dense_pass_full_width_sampled(clada, oracle):
+    """c5's width (d_model 5120, d_ff 13824, 16 sequences) in the launch configuration the benchmark times:
+    three sequences checked against the oracle (one that keeps nothing, one that keeps all, one at 40 %)."""
+    w = wl.WORKLOADS["c5_13b_b16"]
+    B, d, F = 16, w.d_model, w.d_ff
+    weights = wl.layer_weights(w, 0)
+    layer = gpu_layer(weights, clada)
+    W_in, V_in, W_out = oracle_weights(weights)
+    rng = np.random.default_rng(5)
+    scores = (rng.random((B, F)) + 0.5).astype(np.float32)
+    taus = np.full(B, 0.9, dtype=np.float32)
+    taus[1], taus[2] = np.inf, 0.0
+    xs = torch.stack([wl.hidden_states(w, 0, "decode", b, 1)[0] for b in range(B)])
+    ws = clada.new_workspace(layer, B, 0)
+    y = torch.empty(B, d, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    clada.clada_sparse_ffn_decode(layer, xs.cuda(), torch.from_numpy(scores).cuda(), torch.from_numpy(taus).cuda(), 1,
+                                  y, ws, None, None, None, status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    assert bool((y[1] == 0).all())
+    for b in (2, 7, 15):
+        y_or, _, n_or = oracle.sparse_ffn(wl.to_numpy_bits(xs[b]), W_in, V_in, W_out, scores[b].astype(np.float64),
+                                          float(taus[b]))
+        assert n_or > 0 and rel_inf(y[b].cpu().numpy(), y_or) <= FFN_TOL_F32, b
