@@ -11,15 +11,19 @@
 //   h         one epilogue thread per neuron: gate / up of its 16 sequences from TMEM, neuron value, keep bits from
 //             the score vectors, and h split exactly into three 16-bit parts (h = h1 + h2 + h3 to fp32 precision),
 //             because the second contraction takes 16-bit operands and y is held to 1e-5.
-//   phase 2   D2[column, b] = sum_j W_down_t[j, column] * h[b, j]   A = down rows as they lie in memory (MN-major:
-//             columns contiguous), B = the three parts of h (K-major), accumulated in one TMEM tile per 128 columns.
+//   phase 2   D2[column, (part, b)] = sum_j W_down_t[j, column] * h_part[b, j]   A = down rows as they lie in memory
+//             (MN-major: columns contiguous), B = the three parts of h as 48 rows (K-major): ONE instruction of N = 48
+//             per 16 neurons and 128 columns, the three column groups added by the epilogue.  (Layers so wide that 48
+//             TMEM columns per tile do not fit issue three N = 16 instructions into one column group instead.)
 //
 // Work split: 4 consecutive CTAs form a group.  Member m of group g streams the gate / up rows of its own
-// rows_blk neurons (phase 1), the four members exchange their parts of h through global memory (a byte counter
-// per group in the control block, bounded wait; the producer keeps prefetching meanwhile), and in phase 2 member
-// m streams column slice m (a quarter of d_model) of the down rows of all four members' neurons.  Every weight
-// byte is read once, and a group writes ONE partial output [B, d_model] instead of one per CTA.  After a grid
-// barrier all threads sum the groups' partials in group order and write y.
+// rows_blk neurons (phase 1), the four members exchange their parts of h through global memory (each writes its
+// slice of the operand image, a byte counter per group in the control block, bounded wait; the producer keeps
+// prefetching meanwhile), and in phase 2 member m streams column slice m (a quarter of d_model) of the down rows
+// of all four members' neurons, column tile by column tile, so that a finished tile's partial output is stored
+// while the next tile streams.  Every weight byte is read once, and a group writes ONE partial output
+// [B, d_model] instead of one per CTA.  After a grid barrier all threads sum the groups' partials in group order
+// and write y.
 //
 // One persistent CTA per SM, 192 threads: warp 0 TMA producer (64-column boxes of rows_blk rows, 128-byte swizzle,
 // mbarrier ring), warp 1 TMEM allocation + MMA issue from one thread, warps 2-5 epilogues.  Every wait is bounded;
@@ -44,10 +48,34 @@ constexpr int kBdMaxRows = 128;      // neurons per CTA (TMEM lanes)
 constexpr int kBdMaxTiles = 24;      // 128-column tiles per member: 24 * 16 TMEM columns
 constexpr int kBdParts = 3;          // 16-bit parts of h
 constexpr uint32_t kBdTmemCols = 512;
-constexpr uint32_t kBdP2Col = 2 * kBdSeqs * kBdKSplit;  // phase-2 accumulators start behind the phase-1 columns
+constexpr uint32_t kBdImgBlock = kBdParts * 2048;  // bytes of a 64-neuron block of the h image: 48 rows of 128 bytes
 constexpr int kBdGroupWord0 = 8;     // group byte counters: control-block words 8..63
 constexpr int kBdMaxGroups = 4 * (64 - kBdGroupWord0);
 constexpr unsigned kBdGroupSpinLimit = 1u << 22;
+
+// Opt-in timeline (-DCLADA_BD_TRACE): %globaltimer stamps per CTA, 64 slots, written by the thread that passes the point.
+#ifdef CLADA_BD_TRACE
+__device__ unsigned long long *g_bd_trace = nullptr;  // [n_ctas][64]
+#define BD_TRACE(slot)                                                \
+    do {                                                              \
+        if (g_bd_trace) {                                             \
+            unsigned long long t_;                                    \
+            asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t_));     \
+            g_bd_trace[(size_t)blockIdx.x * 64 + (slot)] = t_;        \
+        }                                                             \
+    } while (0)
+#define BD_CLOCK(slot)                                                           \
+    do {                                                                         \
+        if (g_bd_trace) g_bd_trace[(size_t)blockIdx.x * 64 + (slot)] = clock64(); \
+    } while (0)
+#else
+#define BD_TRACE(slot) \
+    do {               \
+    } while (0)
+#define BD_CLOCK(slot) \
+    do {               \
+    } while (0)
+#endif
 
 struct BdParams {
     int d_model, d_ff, B;
@@ -57,7 +85,8 @@ struct BdParams {
     int n_stages;
     int n_tiles, tps;    // 128-column tiles of d_model; tiles per member
     int act, dtype;
-    uint32_t idesc_p1, idesc_p2;
+    int wide;            // phase 2 with one N = 48 instruction per K step (48 TMEM columns per tile fit), else three of N = 16
+    uint32_t idesc_p1, idesc_p2, idesc_p2w;
     const float *scores;  // [B, d_ff]
     const float *tau;
     long long tau_stride;
@@ -65,7 +94,7 @@ struct BdParams {
     size_t y_stride;
     int y_dtype;
     float *partials;      // [n_groups, B, d_model]
-    unsigned char *himg;  // [n_groups] images of the phase-2 B operand: 3 parts x K blocks x (16 rows x 128 bytes)
+    unsigned char *himg;  // [n_groups] images of the phase-2 B operand: K blocks x (3 parts x 16 rows x 128 bytes)
     WsCtrl *ctrl;
     int32_t *status;
 };
@@ -91,11 +120,12 @@ __device__ __forceinline__ uint64_t bd_smem_desc_mn(uint32_t addr, uint32_t lbo_
     d |= (uint64_t)2 << 61;
     return d;
 }
-// Byte offset of element (row n of 16, k) in the K-major, 128-byte-swizzled image of a [16, K] operand: blocks of 64
-// k (2048 bytes), two 8-row atoms per block, 16-byte chunks XORed with the row inside the atom.
+// Byte offset of element (row n of 48 = 16 part + sequence, k) in the K-major, 128-byte-swizzled image of the
+// [48, K] operand: blocks of 64 k, six 8-row atoms of 1024 bytes per block, 16-byte chunks XORed with the row
+// inside the atom.
 __device__ __forceinline__ uint32_t bd_himg_off(int k, int n) {
     const int kb = k >> 6, kk = k & 63;
-    return (uint32_t)kb * 2048u + (uint32_t)(n >> 3) * 1024u + (uint32_t)(n & 7) * 128u +
+    return (uint32_t)kb * kBdImgBlock + (uint32_t)(n >> 3) * 1024u + (uint32_t)(n & 7) * 128u +
            (uint32_t)(((kk >> 3) ^ (n & 7)) << 4) + (uint32_t)(kk & 7) * 2u;
 }
 __device__ __forceinline__ uint16_t bd_to16(int dtype, float v, float &back) {
@@ -108,6 +138,34 @@ __device__ __forceinline__ uint16_t bd_to16(int dtype, float v, float &back) {
     back = __bfloat162float(h);
     return __bfloat16_as_ushort(h);
 }
+// The MMAs of one phase-2 stage (up to 8 K steps of 16 neurons), issued back to back from descriptors computed
+// beforehand: the issuing thread's own instructions between two MMAs are what limits their rate.
+//   da: MN-major descriptor of the stage's first 16 rows (the next K step lies 2048 bytes on);
+//   dh: K-major descriptor of the first K step's rows of the h image, kq its K step inside the 64-neuron block
+//       (the next step lies 32 bytes on, after the fourth step of a block the next block follows).
+template <bool WIDE>
+__device__ __forceinline__ void bd_issue_stage(uint32_t d_y, uint64_t da, uint64_t dh, int kq, int ksteps, uint32_t acc,
+                                               uint32_t idesc) {
+    constexpr uint64_t kBlkStep = (kBdImgBlock >> 4) - 6;
+    uint64_t dhv[kBdMaxRows / 16];
+#pragma unroll
+    for (int k = 0; k < kBdMaxRows / 16; ++k) {
+        dhv[k] = dh;
+        dh += ((kq + k) & 3) == 3 ? kBlkStep : 2;
+    }
+#pragma unroll
+    for (int k = 0; k < kBdMaxRows / 16; ++k) {
+        if (k < ksteps) {
+            if (WIDE) {
+                tc_mma(d_y, da + 128 * k, dhv[k], k > 0 ? 1u : acc, idesc);
+            } else {  // the parts' rows lie 2048 bytes apart
+                tc_mma(d_y, da + 128 * k, dhv[k], k > 0 ? 1u : acc, idesc);
+                tc_mma(d_y, da + 128 * k, dhv[k] + 128, 1u, idesc);
+                tc_mma(d_y, da + 128 * k, dhv[k] + 256, 1u, idesc);
+            }
+        }
+    }
+}
 __device__ __forceinline__ void bd_epi_sync() { asm volatile("bar.sync 2, 128;" ::: "memory"); }
 
 __global__ void __launch_bounds__(kBdThreads, 1)
@@ -116,7 +174,8 @@ sparse_ffn_batch_dense_kernel(const __grid_constant__ CUtensorMap map_x, const _
                               const BdParams p) {
     extern __shared__ unsigned char bd_smem_raw[];
     const uint32_t smem0 = (tc_smem_u32(bd_smem_raw) + 1023u) & ~1023u;
-    __shared__ __align__(8) uint64_t s_full[kBdMaxStages], s_empty[kBdMaxStages], s_p1_full, s_h_ready, s_p2_full;
+    __shared__ __align__(8) uint64_t s_full[kBdMaxStages], s_empty[kBdMaxStages], s_p1_full, s_h_own, s_h_all,
+        s_tile_full[kBdMaxTiles];
     __shared__ uint32_t s_tmem_base;
     __shared__ int s_abort, s_group_ok;
 
@@ -131,7 +190,7 @@ sparse_ffn_batch_dense_kernel(const __grid_constant__ CUtensorMap map_x, const _
     const uint32_t slot_bytes = (uint32_t)p.rpad * 128u;        // where the next box of a stage starts
     const uint32_t stage_bytes = 2u * slot_bytes + 2048u;       // gate | up | x   or   down columns 0-63 | 64-127
     const int kimg_blocks = (kBdMembers * p.rpad + 63) / 64;
-    const uint32_t part_bytes = (uint32_t)kimg_blocks * 2048u;
+    const uint32_t img_bytes = (uint32_t)kimg_blocks * kBdImgBlock;
     const uint32_t himg_s = smem0 + (uint32_t)n_stages * stage_bytes;  // the group's h image in shared memory
     const int t0 = mem * p.tps;
     const int nt = max(0, min(p.tps, p.n_tiles - t0));          // this member's column tiles in phase 2
@@ -143,8 +202,9 @@ sparse_ffn_batch_dense_kernel(const __grid_constant__ CUtensorMap map_x, const _
             tc_mbar_init(tc_smem_u32(&s_empty[s]), 1);
         }
         tc_mbar_init(tc_smem_u32(&s_p1_full), 1);
-        tc_mbar_init(tc_smem_u32(&s_h_ready), 128);
-        tc_mbar_init(tc_smem_u32(&s_p2_full), 1);
+        tc_mbar_init(tc_smem_u32(&s_h_own), 128);
+        tc_mbar_init(tc_smem_u32(&s_h_all), 128);
+        for (int t = 0; t < kBdMaxTiles; ++t) tc_mbar_init(tc_smem_u32(&s_tile_full[t]), 1);
         s_abort = 0;
         s_group_ok = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -174,6 +234,7 @@ sparse_ffn_batch_dense_kernel(const __grid_constant__ CUtensorMap map_x, const _
     volatile int *abort_flag = &s_abort;
     pdl_launch_dependents();
     pdl_wait();  // x, the scores and the thresholds may come from the launch before
+    if (threadIdx.x == 0) BD_TRACE(0);
 
     if (active && warp == 0) {
         // ---- TMA producer ----------------------------------------------------------------------
@@ -198,24 +259,28 @@ sparse_ffn_batch_dense_kernel(const __grid_constant__ CUtensorMap map_x, const _
                     par ^= 1;
                 }
             }
-            for (int mm = 0; mm < kBdMembers && ok; ++mm) {  // phase 2: a member's rows x one column tile per stage
+            BD_TRACE(14);
+            // Phase 2, one column tile of one member's rows per stage: first this CTA's own rows for every tile (their
+            // h is here before the group's exchange is over), then tile by tile the other three members' rows.
+            auto issue_p2 = [&](int mm, int t) -> bool {
+                if (!tc_mbar_wait(tc_smem_u32(&s_empty[s]), par ^ 1, abort_flag)) return false;
                 const int rows0 = (grp * kBdMembers + mm) * p.rows_blk;
-                for (int t = 0; t < nt; ++t, ++kc) {
-                    if (!tc_mbar_wait(tc_smem_u32(&s_empty[s]), par ^ 1, abort_flag)) {
-                        ok = false;
-                        break;
-                    }
-                    const uint32_t bar = tc_smem_u32(&s_full[s]);
-                    const uint32_t dst = smem0 + (uint32_t)s * stage_bytes;
-                    tc_mbar_expect_tx(bar, 2u * box_bytes);
-                    bd_tma_load(dst, &map_wd, (t0 + t) * kTcTileM, rows0, bar, stream_policy);
-                    bd_tma_load(dst + slot_bytes, &map_wd, (t0 + t) * kTcTileM + 64, rows0, bar, stream_policy);
-                    if (++s == n_stages) {
-                        s = 0;
-                        par ^= 1;
-                    }
+                const uint32_t bar = tc_smem_u32(&s_full[s]);
+                const uint32_t dst = smem0 + (uint32_t)s * stage_bytes;
+                tc_mbar_expect_tx(bar, 2u * box_bytes);
+                bd_tma_load(dst, &map_wd, (t0 + t) * kTcTileM, rows0, bar, stream_policy);
+                bd_tma_load(dst + slot_bytes, &map_wd, (t0 + t) * kTcTileM + 64, rows0, bar, stream_policy);
+                ++kc;
+                if (++s == n_stages) {
+                    s = 0;
+                    par ^= 1;
                 }
-            }
+                return true;
+            };
+            for (int t = 0; t < nt && ok; ++t) ok = issue_p2(mem, t);
+            for (int t = 0; t < nt && ok; ++t)
+                for (int mo = 0; mo < kBdMembers - 1 && ok; ++mo) ok = issue_p2(mo + (mo >= mem ? 1 : 0), t);
+            BD_TRACE(15);
             if (!ok) *abort_flag = 1;
             for (int i = max(0, kc - n_stages); i < kc; ++i) {  // never leave with copies in flight
                 int never = 0;
@@ -228,59 +293,77 @@ sparse_ffn_batch_dense_kernel(const __grid_constant__ CUtensorMap map_x, const _
             int s = 0;
             uint32_t par = 0;
             bool ok = true;
+            // One thread issues every MMA, so its instruction count per MMA bounds the rate (an MMA of N <= 48 takes
+            // the tensor pipe ~44 cycles): descriptors are advanced by additions, never rebuilt.
+            const uint64_t desc0 = tc_smem_desc(smem0);  // K-major descriptor of the ring's first byte
+            const uint64_t stage16 = stage_bytes >> 4, slot16 = slot_bytes >> 4;
+            uint64_t dstage = desc0;                     // descriptor of the current stage's first byte
             for (int kb = 0; kb < n_kblocks && ok; ++kb) {
                 if (!tc_mbar_wait(tc_smem_u32(&s_full[s]), par, abort_flag)) {
                     ok = false;
                     break;
                 }
                 tc_fence_after();
-                const uint32_t base = smem0 + (uint32_t)s * stage_bytes;
-                const uint64_t dg = tc_smem_desc(base), du = tc_smem_desc(base + slot_bytes),
-                               dx = tc_smem_desc(base + 2u * slot_bytes);
+                if (kb == 0) BD_TRACE(1);
+                const uint64_t dg = dstage, du = dstage + slot16, dx = dstage + 2 * slot16;
                 const uint32_t d_g = tmem_base + (uint32_t)(kb % kBdKSplit) * (2 * kBdSeqs);  // this K split's columns
+                const uint32_t acc0 = kb >= kBdKSplit ? 1u : 0u;
 #pragma unroll
                 for (int k = 0; k < kTcTileK / 16; ++k) {
-                    const uint32_t acc = (kb >= kBdKSplit || k > 0) ? 1u : 0u;
-                    tc_mma(d_g, dg + 2 * k, dx + 2 * k, acc, p.idesc_p1);
-                    if (gated) tc_mma(d_g + kBdSeqs, du + 2 * k, dx + 2 * k, acc, p.idesc_p1);
+                    tc_mma(d_g, dg + 2 * k, dx + 2 * k, k > 0 ? 1u : acc0, p.idesc_p1);
+                    if (gated) tc_mma(d_g + kBdSeqs, du + 2 * k, dx + 2 * k, k > 0 ? 1u : acc0, p.idesc_p1);
                 }
                 tc_commit(tc_smem_u32(&s_empty[s]));
+                dstage += stage16;
                 if (++s == n_stages) {
                     s = 0;
                     par ^= 1;
+                    dstage = desc0;
                 }
             }
             if (ok) tc_commit(tc_smem_u32(&s_p1_full));
-            // the group's h must be in shared memory before the down rows can be multiplied
-            if (ok && !tc_mbar_wait(tc_smem_u32(&s_h_ready), 0, abort_flag)) ok = false;
-            tc_fence_after();
+            BD_TRACE(2);
+            // Phase 2 writes over the phase-1 columns: the epilogue has read them before it lets s_h_own complete.
+            // A: the stage's two boxes as one MN-major tile, 16 rows (2048 bytes) further per K step.  B: the h image,
+            // 32 bytes further per K step and from the fourth step of a 64-neuron block on to the next block.
             const int ksteps = p.rpad / 16;
-            for (int mm = 0; mm < kBdMembers && ok; ++mm) {
-                for (int t = 0; t < nt; ++t) {
-                    if (!tc_mbar_wait(tc_smem_u32(&s_full[s]), par, abort_flag)) {
-                        ok = false;
-                        break;
-                    }
-                    tc_fence_after();
-                    const uint32_t base = smem0 + (uint32_t)s * stage_bytes;
-                    const uint32_t d_y = tmem_base + kBdP2Col + (uint32_t)t * kBdSeqs;
-                    for (int k = 0; k < ksteps; ++k) {
-                        const uint64_t da = bd_smem_desc_mn(base + (uint32_t)k * 2048u, slot_bytes);
-                        const int kk = mm * p.rpad + k * 16;  // position of these 16 neurons in the group's h
-                        const uint32_t hb = himg_s + (uint32_t)(kk >> 6) * 2048u + (uint32_t)((kk & 63) >> 4) * 32u;
-#pragma unroll
-                        for (int part = 0; part < kBdParts; ++part)
-                            tc_mma(d_y, da, tc_smem_desc(hb + (uint32_t)part * part_bytes),
-                                   (mm > 0 || k > 0 || part > 0) ? 1u : 0u, p.idesc_p2);
-                    }
-                    tc_commit(tc_smem_u32(&s_empty[s]));
-                    if (++s == n_stages) {
-                        s = 0;
-                        par ^= 1;
-                    }
+            const uint32_t tile_cols = p.wide ? kBdParts * kBdSeqs : kBdSeqs;
+            const uint64_t dmn0 = bd_smem_desc_mn(smem0, slot_bytes);
+            const uint64_t dh0 = tc_smem_desc(himg_s);
+            uint64_t dstage2 = dmn0 + (uint64_t)s * stage16;
+            auto run_p2 = [&](int mm, int t, uint32_t acc) -> bool {  // the MMAs of one stage
+                if (!tc_mbar_wait(tc_smem_u32(&s_full[s]), par, abort_flag)) return false;
+                tc_fence_after();
+                if (acc && t < 8) BD_CLOCK(16 + 6 * t + 2 * (mm - (mm > mem ? 1 : 0)));
+                const uint32_t d_y = tmem_base + (uint32_t)t * tile_cols;
+                const int kk16 = mm * ksteps;  // first K step of member mm in the group's h
+                const uint64_t dh = dh0 + (uint64_t)(kk16 >> 2) * (kBdImgBlock >> 4) + (uint64_t)(kk16 & 3) * 2;
+                if (p.wide)
+                    bd_issue_stage<true>(d_y, dstage2, dh, kk16 & 3, ksteps, acc, p.idesc_p2w);
+                else
+                    bd_issue_stage<false>(d_y, dstage2, dh, kk16 & 3, ksteps, acc, p.idesc_p2);
+                tc_commit(tc_smem_u32(&s_empty[s]));
+                if (acc && t < 8) BD_CLOCK(17 + 6 * t + 2 * (mm - (mm > mem ? 1 : 0)));
+                dstage2 += stage16;
+                if (++s == n_stages) {
+                    s = 0;
+                    par ^= 1;
+                    dstage2 = dmn0;
                 }
+                return true;
+            };
+            // this CTA's own part of h is in shared memory first; the other members' parts follow the exchange
+            if (ok && !tc_mbar_wait(tc_smem_u32(&s_h_own), 0, abort_flag)) ok = false;
+            tc_fence_after();
+            BD_TRACE(3);
+            for (int t = 0; t < nt && ok; ++t) ok = run_p2(mem, t, 0u);
+            if (ok && !tc_mbar_wait(tc_smem_u32(&s_h_all), 0, abort_flag)) ok = false;
+            tc_fence_after();
+            for (int t = 0; t < nt && ok; ++t) {
+                for (int mo = 0; mo < kBdMembers - 1 && ok; ++mo) ok = run_p2(mo + (mo >= mem ? 1 : 0), t, 1u);
+                if (ok) tc_commit(tc_smem_u32(&s_tile_full[t]));  // this tile's partial output is complete
             }
-            if (ok) tc_commit(tc_smem_u32(&s_p2_full));
+            BD_TRACE(4);
             if (!ok) *abort_flag = 1;
         }
     } else if (active) {
@@ -298,6 +381,7 @@ sparse_ffn_batch_dense_kernel(const __grid_constant__ CUtensorMap map_x, const _
         bool ok = tc_mbar_wait(tc_smem_u32(&s_p1_full), 0, abort_flag);
         tc_fence_after();
         const uint32_t t_lane = tmem_base + ((uint32_t)(quarter * 32) << 16);
+        if (etid == 0) BD_TRACE(5);
         if (ok) {
             float g[kBdSeqs], u[kBdSeqs];
 #pragma unroll
@@ -315,23 +399,39 @@ sparse_ffn_batch_dense_kernel(const __grid_constant__ CUtensorMap map_x, const _
                 }
             }
             if (r < p.rpad) {  // rows rows_blk .. rpad-1 are the zero padding of the K steps
-                unsigned char *img = p.himg + (size_t)grp * kBdParts * part_bytes;
-                const int k = mem * p.rpad + r;
+                const int k = mem * p.rpad + r;  // this CTA's slice of the image, written where phase 2 reads it
 #pragma unroll
                 for (int b = 0; b < kBdSeqs; ++b) {
                     float h = ((keep >> b) & 1u) ? neuron_value_f(p.act, g[b], u[b]) : 0.f;
-                    const uint32_t off = bd_himg_off(k, b);
 #pragma unroll
                     for (int part = 0; part < kBdParts; ++part) {
                         float back;
                         const uint16_t bits = bd_to16(p.dtype, h, back);
                         h -= back;
-                        *reinterpret_cast<uint16_t *>(img + (size_t)part * part_bytes + off) = bits;
+                        asm volatile("st.shared.u16 [%0], %1;" ::"r"(himg_s + bd_himg_off(k, part * kBdSeqs + b)), "h"(bits)
+                                     : "memory");
                     }
                 }
             }
+        }
+        if (ok) {  // the MMA thread may start on this CTA's own down rows
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            tc_fence_before();  // phase 2 writes over the TMEM columns this thread has read
+            tc_mbar_arrive(tc_smem_u32(&s_h_own));
+        }
+        bd_epi_sync();
+        unsigned char *img = p.himg + (size_t)grp * img_bytes;
+        const int cpr = p.rpad / 8;                       // 16-byte chunks of a member's slice per image row
+        const int n_chunks = kBdParts * kBdSeqs * cpr;
+        if (ok) {  // the slice goes to global memory for the other three members
+            for (int i = etid; i < n_chunks; i += 128) {
+                const int n = i / cpr, c = i - n * cpr;
+                const uint32_t off = bd_himg_off(mem * p.rpad + 8 * c, n);
+                __stcg(reinterpret_cast<uint4 *>(img + off), lds128(himg_s + off));
+            }
             __threadfence();
         }
+        if (etid == 0) BD_TRACE(6);
         bd_epi_sync();
         // group exchange: one byte counter per group; every member adds 1 when its part of h is in global memory
         if (etid == 0) {
@@ -350,42 +450,61 @@ sparse_ffn_batch_dense_kernel(const __grid_constant__ CUtensorMap map_x, const _
                 }
             }
             s_group_ok = gok;
+            BD_TRACE(7);
         }
         bd_epi_sync();
         ok = ok && s_group_ok != 0;
         if (ok) {
-            const uint4 *src = reinterpret_cast<const uint4 *>(p.himg + (size_t)grp * kBdParts * part_bytes);
-            const int n_vec = (int)(kBdParts * part_bytes / 16u);
-            for (int i = etid; i < n_vec; i += 128) {
-                const uint4 v = __ldcg(src + i);
-                asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(himg_s + (uint32_t)i * 16u), "r"(v.x), "r"(v.y),
-                             "r"(v.z), "r"(v.w)
+            for (int i = etid; i < (kBdMembers - 1) * n_chunks; i += 128) {  // the other members' slices
+                const int mo = i / n_chunks, rem = i - mo * n_chunks;
+                const int m2 = mo + (mo >= mem ? 1 : 0);
+                const int n = rem / cpr, c = rem - n * cpr;
+                const uint32_t off = bd_himg_off(m2 * p.rpad + 8 * c, n);
+                const uint4 v = __ldcg(reinterpret_cast<const uint4 *>(img + off));
+                asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(himg_s + off), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w)
                              : "memory");
             }
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-            tc_mbar_arrive(tc_smem_u32(&s_h_ready));
-            // ---- phase 2 epilogue: this member's column tiles of the group's partial output ----------
-            ok = tc_mbar_wait(tc_smem_u32(&s_p2_full), 0, abort_flag);
-            tc_fence_after();
-            if (ok) {
-                for (int t = 0; t < nt; ++t) {
-                    uint32_t ry[16];
-                    tc_ld16(t_lane + kBdP2Col + (uint32_t)t * kBdSeqs, ry);
+            tc_mbar_arrive(tc_smem_u32(&s_h_all));
+            if (etid == 0) BD_TRACE(8);
+            // ---- phase 2 epilogue: each column tile of the group's partial output as soon as it is complete ----------
+            for (int t = 0; t < nt && ok; ++t) {
+                ok = tc_mbar_wait(tc_smem_u32(&s_tile_full[t]), 0, abort_flag);
+                tc_fence_after();
+                if (t == 0 && etid == 0) BD_TRACE(9);
+                if (!ok) break;
+                uint32_t ry[16];
+                float yv[kBdSeqs];
+                if (p.wide) {  // the three parts' column groups, added in part order
+                    uint32_t r2[16], r3[16];
+                    tc_ld16(t_lane + (uint32_t)t * (kBdParts * kBdSeqs), ry);
+                    tc_ld16(t_lane + (uint32_t)t * (kBdParts * kBdSeqs) + kBdSeqs, r2);
+                    tc_ld16(t_lane + (uint32_t)t * (kBdParts * kBdSeqs) + 2 * kBdSeqs, r3);
                     tc_wait_ld();
-                    const int i = (t0 + t) * kTcTileM + r;
-                    if (i < p.d_model) {
 #pragma unroll
-                        for (int b = 0; b < kBdSeqs; ++b)
-                            if (b < p.B) p.partials[((size_t)grp * p.B + b) * p.d_model + i] = __uint_as_float(ry[b]);
-                    }
+                    for (int b = 0; b < kBdSeqs; ++b)
+                        yv[b] = (__uint_as_float(ry[b]) + __uint_as_float(r2[b])) + __uint_as_float(r3[b]);
+                } else {
+                    tc_ld16(t_lane + (uint32_t)t * kBdSeqs, ry);
+                    tc_wait_ld();
+#pragma unroll
+                    for (int b = 0; b < kBdSeqs; ++b) yv[b] = __uint_as_float(ry[b]);
+                }
+                const int i = (t0 + t) * kTcTileM + r;
+                if (i < p.d_model) {
+#pragma unroll
+                    for (int b = 0; b < kBdSeqs; ++b)
+                        if (b < p.B) p.partials[((size_t)grp * p.B + b) * p.d_model + i] = yv[b];
                 }
             }
         }
+        if (etid == 0) BD_TRACE(10);
         if (!ok) *abort_flag = 1;
     }
 
     tc_fence_before();
     __syncthreads();
+    if (threadIdx.x == 0) BD_TRACE(11);
     if (threadIdx.x == 0 && s_abort && p.status) atomicOr(p.status, CLADA_STATUS_TIMEOUT);
     if (warp == 1) {
         tc_fence_after();
@@ -396,6 +515,7 @@ sparse_ffn_batch_dense_kernel(const __grid_constant__ CUtensorMap map_x, const _
         if (threadIdx.x == 0 && p.status) atomicOr(p.status, CLADA_STATUS_TIMEOUT);
         return;
     }
+    if (threadIdx.x == 0) BD_TRACE(12);
     if (cta == 0 && threadIdx.x < 64 - kBdGroupWord0)  // every member has passed its group's counter: clear them
         reinterpret_cast<unsigned *>(p.ctrl)[kBdGroupWord0 + threadIdx.x] = 0u;
     const int d4 = p.d_model / 4;
@@ -420,6 +540,7 @@ sparse_ffn_batch_dense_kernel(const __grid_constant__ CUtensorMap map_x, const _
             reinterpret_cast<uint2 *>(yb)[q] = pack4_16bit(p.y_dtype, s);
         }
     }
+    if (threadIdx.x == 0) BD_TRACE(13);
 }
 
 // ---- host side ------------------------------------------------------------------------------
@@ -445,7 +566,7 @@ static bool bd_plan(const clada_layer *layer, int B, const DeviceInfo &di, BdPla
     if (pl->tps > kBdMaxTiles) return false;
     const size_t stage_bytes = 2 * (size_t)pl->rpad * 128 + 2048;
     const size_t kimg_blocks = ((size_t)kBdMembers * pl->rpad + 63) / 64;
-    pl->himg_bytes = kBdParts * kimg_blocks * 2048;
+    pl->himg_bytes = kimg_blocks * kBdImgBlock;
     const size_t budget = (size_t)di.max_smem_optin - 1024;  // static arrays: barriers and flags
     // behind the ring: the h image; at least 16 KB, because a phase-1 A tile is always 128 rows high and with few
     // neurons per CTA the tile of the last stage reaches past its own slot
@@ -506,6 +627,8 @@ int launch_ffn_batch_dense(const clada_layer *layer, int B, const void *x, const
     p.dtype = layer->dtype;
     p.idesc_p1 = tc_instr_desc(layer->dtype, kBdSeqs);
     p.idesc_p2 = tc_instr_desc(layer->dtype, kBdSeqs) | (1u << 15);  // A (the down rows) is MN-major
+    p.idesc_p2w = tc_instr_desc(layer->dtype, kBdParts * kBdSeqs) | (1u << 15);
+    p.wide = pl.tps * kBdParts * kBdSeqs <= (int)kBdTmemCols ? 1 : 0;
     p.scores = scores;
     p.tau = tau;
     p.tau_stride = tau_stride;
@@ -539,3 +662,10 @@ int launch_ffn_batch_dense(const clada_layer *layer, int B, const void *x, const
 }
 
 }  // namespace clada
+
+#ifdef CLADA_BD_TRACE
+extern "C" int clada_bd_trace_buffer(unsigned long long *buf) {
+    CLADA_CUDA_TRY(cudaMemcpyToSymbol(clada::g_bd_trace, &buf, sizeof buf));
+    return CLADA_OK;
+}
+#endif
