@@ -237,7 +237,7 @@ extern "C" int clada_sparse_ffn_decode_layers(const clada_layer *layers, int32_t
     const size_t d = (size_t)layers[0].d_model, F = (size_t)layers[0].d_ff;
     const size_t x_layer = (size_t)B * d * elem_size(layers[0].dtype), y_layer = (size_t)B * d * elem_size(y_dtype);
     if (ffn_stack_supported(layers, L, B, ws_bytes))
-        return launch_ffn_stack(layers, L, x, x_layer, scores, tau_final, 1, y, y_layer, y_dtype, ws, status,
+        return launch_ffn_stack(layers, L, x, x_layer, scores, tau_final, 1, y, y_layer, y_dtype, ws, ws_bytes, status,
                                 static_cast<cudaStream_t>(stream));
     for (int l = 0; l < L; ++l) {
         int rc = decode_with_workspace(&layers[l], static_cast<const char *>(x) + l * x_layer, B,

@@ -42,6 +42,8 @@ struct StackParams {
     size_t y_stride;
     int y_dtype;
     float *partials;      // [2][gridDim.x][consumer groups][d_model]
+    const unsigned *keep_words;  // [L][chunks of 32 neurons] keep bits A_lj >= tau_l from keep_words_kernel, or null:
+                                 // the scanner tests the score vectors itself
     WsCtrl *ctrl;
     int32_t *status;
     int d_model, d_ff, L;
@@ -88,13 +90,25 @@ constexpr int kListBufs = 4;                    // kept lists are built up to fo
 // coalesced loads (32 chunks = 1024 neurons per round, all loads of a round in flight together), the chunk words
 // parked in keep[]; then the ranks again from the parked words, and this CTA's equal share [r0, r1) of the kept
 // neurons, ascending, written to list[].  Returns the layer's kept count; *my_n = r1 - r0.
-__device__ __forceinline__ int scan_share_list(const float *__restrict__ scores, const float tau, const int F,
-                                               const int cta, const int n_ctas, int *list, unsigned *keep,
-                                               int *my_n, const uint64_t keep_policy) {
+__device__ __forceinline__ int scan_share_list(const float *__restrict__ scores, const unsigned *__restrict__ words,
+                                               const float tau, const int F, const int cta, const int n_ctas,
+                                               int *list, unsigned *keep, int *my_n, const uint64_t keep_policy) {
     const int lane = threadIdx.x & 31;
     const int chunks = (F + kWarp - 1) / kWarp;
     const float kNoNeuron = __int_as_float(0x7fc00000);  // NaN: no threshold keeps a position past d_ff
     int n_act = 0;
+    if (words) {  // the layer's keep words are there already (4 bytes per chunk instead of 128 bytes of scores)
+        for (int q0 = 0; q0 < chunks; q0 += 4 * kWarp) {
+            unsigned w[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) w[u] = q0 + u * kWarp + lane < chunks ? __ldcg(words + q0 + u * kWarp + lane) : 0u;
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                if (q0 + u * kWarp + lane < chunks) keep[q0 + u * kWarp + lane] = w[u];
+                n_act += __popc(w[u]);
+            }
+        }
+    } else
     for (int q0 = 0; q0 < chunks; q0 += kWarp) {
         const bool whole = q0 + kWarp <= chunks && (q0 + kWarp) * kWarp <= F;
         float v[kWarp];
@@ -212,8 +226,9 @@ sparse_ffn_stack_kernel(const StackParams p, const __grid_constant__ StackLayers
             }
             const float tau = ld_keep(p.tau + (size_t)l * p.tau_stride, keep_policy);
             int my_n;
-            const int n_act = scan_share_list(p.scores + (size_t)l * F, tau, F, cta, n_ctas, s_list + k * list_cap,
-                                              s_keep, &my_n, keep_policy);
+            const int n_act = scan_share_list(p.scores + (size_t)l * F,
+                                              p.keep_words ? p.keep_words + (size_t)l * ((F + kWarp - 1) / kWarp) : nullptr,
+                                              tau, F, cta, n_ctas, s_list + k * list_cap, s_keep, &my_n, keep_policy);
             if (lane == 0) {
                 s_nact[k] = n_act;
                 s_myn[k] = my_n;
@@ -566,7 +581,16 @@ bool ffn_stack_supported(const clada_layer *layers, int L, int B, size_t ws_byte
 // kMaxStackLayers layers each.  Strides in bytes (x, y) and elements (tau).
 int launch_ffn_stack(const clada_layer *layers, int L, const void *x, size_t x_stride, const float *scores,
                      const float *tau, long long tau_stride, void *y, size_t y_stride, int y_dtype, void *ws,
-                     int32_t *status, cudaStream_t st) {
+                     size_t ws_bytes, int32_t *status, cudaStream_t st) {
+    DeviceInfo di;
+    int rc0 = device_info(&di);
+    if (rc0 != CLADA_OK) return rc0;
+    // Behind the partial rows, when the workspace has the room: the keep words of every layer of a launch, written
+    // by one small kernel before it, so that the scanner warp reads 4 bytes per 32 neurons instead of their scores.
+    const int vpr0 = layers[0].d_model / (layers[0].dtype == CLADA_F32 ? 4 : 8);
+    const size_t words_at = kWsCtrlBytes + 2 * (size_t)di.num_sms * ffn_groups(vpr0) * layers[0].d_model * sizeof(float);
+    const bool have_words =
+        ws_bytes >= words_at + keep_words_bytes_of(L < kMaxStackLayers ? L : kMaxStackLayers, layers[0].d_ff);
     for (int l0 = 0; l0 < L; l0 += kMaxStackLayers) {
         const int n = L - l0 < kMaxStackLayers ? L - l0 : kMaxStackLayers;
         StackLayers lay = {};
@@ -585,6 +609,13 @@ int launch_ffn_stack(const clada_layer *layers, int L, const void *x, size_t x_s
         p.y_stride = y_stride;
         p.y_dtype = y_dtype;
         p.partials = reinterpret_cast<float *>(static_cast<char *>(ws) + kWsCtrlBytes);
+        p.keep_words = nullptr;
+        if (have_words) {
+            unsigned *words = reinterpret_cast<unsigned *>(static_cast<char *>(ws) + words_at);
+            const int rcw = launch_keep_words(p.scores, n, layers[0].d_ff, p.tau, tau_stride, words, st);
+            if (rcw != CLADA_OK) return rcw;
+            p.keep_words = words;
+        }
         p.ctrl = static_cast<WsCtrl *>(ws);
         p.status = status;
         p.d_model = layers[0].d_model;

@@ -342,6 +342,6 @@ size_t keep_words_bytes_of(int B, int d_ff);
 bool ffn_stack_supported(const clada_layer *layers, int L, int B, size_t ws_bytes);
 int launch_ffn_stack(const clada_layer *layers, int L, const void *x, size_t x_stride, const float *scores,
                      const float *tau, long long tau_stride, void *y, size_t y_stride, int y_dtype, void *ws,
-                     int32_t *status, cudaStream_t st);
+                     size_t ws_bytes, int32_t *status, cudaStream_t st);
 
 }  // namespace clada
