@@ -166,7 +166,8 @@ constexpr int kMaxStages = 16;
 // gt, gt + GT, ... of every row (x and the partial y of those columns stay in registers).  Per chunk: the gate
 // and up dot products of its four neurons from the staged rows (packed two-wide FMAs), ONE group-wide reduction
 // of the eight values (halving butterfly in the warp, then across the group's warps through shared memory, fixed
-// order), the neuron values, and the four down rows scaled into the partial y.  With two groups one group's
+// order), the neuron values, and the four down rows scaled into the partial y.  (Without a gate projection and with
+// one vector per thread a chunk is EIGHT neurons: the eight values are their gate sums.)  With two groups one group's
 // reduction latency hides under the other's arithmetic, and a row of at most 256 vectors keeps every thread busy.
 // A group never reads the other group's stages, but it watches each of them land before it moves past.
 // A stage is handed back by the warps of the group that owns its neuron (kConsWarps / GROUPS arrivals per stage;
@@ -190,18 +191,22 @@ __device__ __forceinline__ void consume_share(const int my_n, const int act, con
     constexpr int GW = GT / kWarp;           // warps per group
     constexpr int PER = GW / 4;              // warps each lane adds in the cross-warp sum (4 lanes per value)
     static_assert(GROUPS == 1 || GROUPS == 2, "one or two consumer groups");
+    // Neurons per chunk (= per group-wide reduction of eight values): four with a gate and an up value each, or,
+    // without a gate projection, eight when a row is one vector per thread (the ring then holds twelve stages or
+    // more): rows that narrow are bound by the reduction's latency, not by their bytes.
+    constexpr int NPC = (!GATED && NV == 1) ? 2 * GS : GS;
     const int tid = threadIdx.x, lane = tid & 31;
     const int grp = tid / GT, gt = tid - grp * GT, gw = gt >> 5;
     float(*dot)[2 * GS][GW] = reinterpret_cast<float(*)[2 * GS][GW]>(s_dot + (size_t)grp * 2 * 2 * GS * GW);
     const bool b16 = lane & 16, b8 = lane & 8, b4 = lane & 4;
     int buf = 0;
-    for (int g0 = 0, chunk = 0; g0 < my_n; g0 += GS, ++chunk) {
+    for (int g0 = 0, chunk = 0; g0 < my_n; g0 += NPC, ++chunk) {
         if (GROUPS > 1 && (chunk & (GROUPS - 1)) != grp) {
             // The other group's chunk.  Its stages are not read here and not handed back from here, but each
             // one's copy is seen to land: bulk copies may complete out of order, and a wait by parity for the
             // NEXT use of a stage would pass at once if this use had not even completed yet.
 #pragma unroll
-            for (int g = 0; g < GS; ++g) {
+            for (int g = 0; g < NPC; ++g) {
                 if (g0 + g >= my_n) break;
                 if (!timed_out && !mbar_wait(full0 + 8 * cs, cpar)) timed_out = true;
                 if (++cs == n_stages) {
@@ -212,10 +217,10 @@ __device__ __forceinline__ void consume_share(const int my_n, const int act, con
             continue;
         }
         float pd[2 * GS];
-        uint32_t st_addr[GS];
-        int st_idx[GS];
+        uint32_t st_addr[NPC];
+        int st_idx[NPC];
 #pragma unroll
-        for (int g = 0; g < GS; ++g) {
+        for (int g = 0; g < NPC; ++g) {
             const int i = g0 + g;
             float2 sg = make_float2(0.f, 0.f), su = make_float2(0.f, 0.f);
             st_idx[g] = cs;
@@ -251,8 +256,12 @@ __device__ __forceinline__ void consume_share(const int my_n, const int act, con
                     }
                 }
             }
-            pd[2 * g] = sg.x + sg.y;
-            pd[2 * g + 1] = su.x + su.y;
+            if (NPC == GS) {
+                pd[2 * g] = sg.x + sg.y;
+                pd[2 * g + 1] = su.x + su.y;
+            } else {
+                pd[g] = sg.x + sg.y;  // no up values: the eight slots hold eight neurons' gate sums
+            }
         }
         // Warp sums of the 8 values by a halving butterfly (9 shuffles): after it every lane of
         // quad q holds the warp total of value q.  Fixed order, so results repeat bit for bit.
@@ -289,10 +298,10 @@ __device__ __forceinline__ void consume_share(const int my_n, const int act, con
         tot += __shfl_xor_sync(0xffffffffu, tot, 1);
         tot += __shfl_xor_sync(0xffffffffu, tot, 2);
         const float up = __shfl_xor_sync(0xffffffffu, tot, 4);  // value 2g+1 sits 4 lanes above value 2g
-        const float hval = neuron_value_f(act, tot, up);        // meaningful on lanes 8g..8g+3
+        const float hval = neuron_value_f(act, tot, up);        // meaningful on lanes 8g..8g+3 (4g..4g+3 without up values)
 #pragma unroll
-        for (int g = 0; g < GS; ++g) {
-            const float h = __shfl_sync(0xffffffffu, hval, 8 * g);
+        for (int g = 0; g < NPC; ++g) {
+            const float h = __shfl_sync(0xffffffffu, hval, (NPC == GS ? 8 : 4) * g);
             if (g0 + g >= my_n) continue;
             const float2 h2 = make_float2(h, h);
 #pragma unroll
@@ -308,7 +317,7 @@ __device__ __forceinline__ void consume_share(const int my_n, const int act, con
         __syncwarp();
         if (lane == 0) {
 #pragma unroll
-            for (int g = 0; g < GS; ++g)
+            for (int g = 0; g < NPC; ++g)
                 if (g0 + g < my_n) mbar_arrive(empty0 + 8 * st_idx[g]);
         }
         buf ^= 1;
