@@ -41,18 +41,7 @@ STACK_PASSES = 32      # layer passes per persistent launch in the single-layer 
 PROFILES = os.path.join(ROOT, "profiles")
 CSRC = os.path.join(ROOT, "paper_2502_19078_b200", "csrc")
 # sources a kernel's code comes from: the DRAM traffic on record for it counts only while these are unchanged
-KERNEL_SOURCES = {
-    "sparse_ffn_kernel": ["clada_ffn.cu", "ffn_common.cuh", "common.cuh"],
-    "sparse_ffn_stack_kernel": ["clada_ffn_stack.cu", "ffn_common.cuh", "common.cuh"],
-}
-
-
-def sources_hash(kernel: str) -> str:
-    h = hashlib.sha256()
-    for name in KERNEL_SOURCES[kernel]:
-        with open(os.path.join(CSRC, name), "rb") as f:
-            h.update(f.read())
-    return h.hexdigest()
+from paper_2502_19078_b200.ncu_summary import KERNEL_SOURCES, sources_hash  # noqa: E402  (one list for both sides)
 
 
 def recorded_traffic(kernel: str, workload: str):
@@ -474,6 +463,7 @@ class BatchJob:
             b0 += n
         self.dense = max(self.launch_sizes) > 4
 
+    traffic_kernel = property(lambda self: "sparse_ffn_batch_dense_kernel" if self.dense else "sparse_ffn_batch_tc_kernel")
     ffn_kernel = property(lambda self: "sparse_ffn_batch_dense_kernel (one call = one dense pass per 16 sequences)"
                           if self.dense else
                           "sparse_ffn_batch_tc_kernel (one call = keep words of the batch + all its tiles)")
@@ -582,7 +572,7 @@ def other_workloads_info(clada, dev, stream, use_graph, peak, read_gbs):
             nbytes = job.ffn_bytes_per_launch
             rec = {"kernel": job.ffn_kernel, "layers_run": 1, "batch": w.batch, "sequences_per_launch": job.launch_sizes,
                    "sparsity": w.sparsities[0], "us_per_batch_call": t_ms * 1e3, "bytes_per_batch_call": nbytes,
-                   "union_rows": job.union_rows}
+                   "union_rows": job.union_rows, "traffic": recorded_traffic(job.traffic_kernel, name)}
         else:
             nbytes = kept * 3 * w.d_model * w.elem_bytes + w.d_ff * 4 + w.d_model * w.elem_bytes + w.d_model * 4
             t_layer = _median_ms(_graphed(job.ffn_per_layer_loop, stream, use_graph), inner=3) / job.ffn_launches_per_loop
@@ -622,6 +612,8 @@ def run_ours(args):
     barrier()
     clada.load()
     w = wl.WORKLOADS[args.workload]
+    if args.batch:
+        w = wl.scaled(w, batch=args.batch)
     job = (BatchJob if w.batch > 1 else StackJob if w.n_layers > 1 else Job)(clada, w, dev, rank)
 
     stream = torch.cuda.Stream()
@@ -765,7 +757,8 @@ def run_ours(args):
     sample_note = f"median of {FFN_REPEATS} samples of {FFN_INNER} replays of the loop's CUDA graph, clocks recorded over all of them"
     per_launch = {"kernel": "sparse_ffn_kernel", "call": "clada_sparse_ffn_decode: one launch per layer pass",
                   **figures(ffn_bytes, ffn_ms[0]), "bytes_per_launch": ffn_bytes, "us_per_launch": ffn_ms[0] * 1e3,
-                  "kept_neurons": kept_base, "traffic": recorded_traffic("sparse_ffn_kernel", w.name)}
+                  "kept_neurons": kept_base,
+                  "traffic": recorded_traffic(getattr(job, "traffic_kernel", "sparse_ffn_kernel"), w.name)}
     if isinstance(job, Job):
         per_launch["by_sparsity"] = [
             {"sparsity": w.sparsities[r], "kept_neurons": w.d_ff - w.k_cut(w.sparsities[r]), "us_per_launch": t * 1e3,
@@ -940,6 +933,8 @@ def main():
     ap.add_argument("--no-graph", dest="graph", action="store_false")
     ap.add_argument("--no-info", dest="info", action="store_false",
                     help="leave out the informational figures on the other workloads' layers")
+    ap.add_argument("--batch", type=int, default=0,
+                    help="sequences per batch for the batched workloads instead of the workload's own (e.g. 4: the tile kernel)")
     ap.add_argument("--quick", action="store_true",
                     help="for profiler captures: one replay per sample of the FFN-only loops and no informational "
                          "workloads (the figures of such a run are not bench values)")

@@ -248,12 +248,17 @@ int clada_cogload_adjust(const void *logits, int32_t logits_dtype, int32_t B, in
  *   y        out [B, d_model], y_dtype fp32, bf16 or fp16
  *   mask_out / idx_out / count_out: optional (NULL), as in clada_select
  * Accumulation is fp32 in a fixed order: results are bit-identical run to run.
- * A batch runs in tiles of 4 or 2 sequences that read the union of their kept
- * rows once (16-bit layers: gate / up contractions on the tensor cores with
- * short fp32 accumulation chains, same 1e-5 as the CUDA-core path), preceded by
- * one small launch that tests the batch's scores once.
+ * A batch of a 16-bit layer with d_ff <= 128 x (SM count) runs 16 sequences at
+ * a time through ONE dense pass over the layer while 5 or more are left (the
+ * union of that many kept sets is nearly the whole layer; both contractions on
+ * the tensor cores, the hidden activations carried exactly as three 16-bit
+ * parts, each sequence's mask applied to its own activations: same 1e-5 as the
+ * CUDA-core path).  What is left, and every batch of other layers, runs in tiles
+ * of 4 or 2 sequences that read the union of their kept rows once, preceded by
+ * one small launch that tests the tiled sequences' scores once.
  * The workspace (clada_workspace_bytes(layer, B, 0) bytes at least) must have
- * been initialised with clada_workspace_init. */
+ * been initialised with clada_workspace_init; with a workspace too small for the
+ * dense pass's scratch but large enough for tiles the call uses tiles. */
 int clada_sparse_ffn_decode(const clada_layer *layer, const void *x, int32_t B,
                             const float *scores /*[B,d_ff]*/, const float *tau_final,
                             int64_t tau_stride, void *y, int32_t y_dtype,
@@ -271,7 +276,9 @@ int clada_sparse_ffn_decode(const clada_layer *layer, const void *x, int32_t B,
  * All layers are validated before anything is enqueued.
  * One sequence (B = 1, L >= 2) runs all layers in ONE persistent launch (up to
  * 128 layers per launch): the weight stream does not stop at layer
- * boundaries, the outputs are bit for bit those of the per-layer call.  This
+ * boundaries, the outputs are bit for bit those of the per-layer call.  One
+ * small launch before it tests every layer's scores against its threshold
+ * (4 bytes per 32 neurons, kept behind the partial rows in the workspace).  This
  * needs the workspace clada_workspace_bytes(layer, 1, 0) gives; with a smaller
  * one, for a batch, or for rows too wide for a ring of four stages
  * (d_model 8192 in 16-bit types) the call runs the per-layer launches in a loop. */
@@ -292,14 +299,17 @@ int clada_sparse_ffn_decode_layers(const clada_layer *layers, int32_t L, const v
  *  - Limits: d_model <= 8192 and a device with at most 160 SMs; beyond that the
  *    call returns CLADA_ERR_UNSUPPORTED (clada_last_cuda_error() says why)
  *    and enqueues nothing.  Every refusal happens before the first enqueue.
- *  - Batches: the array holds 160 x 8192 fp32 partial outputs, i.e. one row per
- *    (SM, sequence of a tile).  B >= 2 therefore runs in the largest tiles of
- *    sequences (4, 2 or 1 per launch) that fit, together with the batch's keep
- *    bits (4 bytes per sequence and 32 neurons): on a 148-SM device tiles of 4
- *    up to d_model 2048, tiles of 2 up to d_model 4096, one sequence per launch
- *    above that.  Results per sequence are those of clada_sparse_ffn_decode;
- *    smaller tiles only read the shared weight rows once per tile instead of
- *    once per larger tile.
+ *  - Batches: the array holds 160 x 8192 fp32 partial outputs.  B >= 2 runs in
+ *    the largest launches whose scratch fits: the dense pass of
+ *    clada_sparse_ffn_decode (SMs / 4 x B x d_model fp32 values plus SMs / 4
+ *    images of the hidden activations of up to 48 KB: on a 148-SM device 8
+ *    sequences fit up to d_model 2048, at 4096 they do not), else
+ *    the largest tiles of sequences (4, 2 or 1 per launch; one row per SM and
+ *    sequence of a tile, together with the batch's keep bits, 4 bytes per
+ *    sequence and 32 neurons: tiles of 4 up to d_model 2048, tiles of 2 up to
+ *    d_model 4096, one sequence per launch above that).  Results per sequence
+ *    are those of clada_sparse_ffn_decode; smaller launches only read the
+ *    shared weight rows once per launch instead of once per larger one.
  *  - The first call on a device looks up the array's device address; make that
  *    first call outside any stream capture.
  *  - All calls share the one array and it keeps the previous call's contents;

@@ -22,6 +22,9 @@ CSRC = os.path.join(ROOT, "paper_2502_19078_b200", "csrc")
 KERNEL_SOURCES = {
     "sparse_ffn_kernel": ["clada_ffn.cu", "ffn_common.cuh", "common.cuh"],
     "sparse_ffn_stack_kernel": ["clada_ffn_stack.cu", "ffn_common.cuh", "common.cuh"],
+    "sparse_ffn_batch_dense_kernel": ["clada_ffn_batch_dense.cu", "tc_common.cuh", "ffn_batch.cuh", "ffn_common.cuh",
+                                      "common.cuh"],
+    "sparse_ffn_batch_tc_kernel": ["clada_ffn_batch_tc.cu", "ffn_batch.cuh", "ffn_common.cuh", "common.cuh"],
 }
 _UNIT = {"byte": 1.0, "Kbyte": 1e3, "Mbyte": 1e6, "Gbyte": 1e9}
 
