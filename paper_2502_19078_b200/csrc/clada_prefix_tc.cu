@@ -171,10 +171,18 @@ prefix_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
     } else if (warp == 1) {
         // ---- MMA issuer ------------------------------------------------------------------------
         if (lane == 0) {
+            // One thread issues every MMA of the CTA, and its own instructions between two MMAs are what paces
+            // them (a lone thread issues an instruction every ~5 cycles): nothing in the K loop is recomputed --
+            // the stage's descriptors and barrier addresses advance by additions.
             int it = 0;
             int s = 0;
             uint32_t par = 0;
             bool ok = true;
+            const uint64_t desc0 = tc_smem_desc(smem0);          // descriptor of the ring's first byte
+            const uint64_t stage16 = stage_bytes >> 4, tile16 = kTcTileBytes >> 4;
+            const uint32_t full0 = tc_smem_u32(&s_full[0]), empty0 = tc_smem_u32(&s_empty[0]);
+            uint64_t dstage = desc0;
+            uint32_t full_s = full0, empty_s = empty0;
             for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++it) {
                 const int a = it & 1;
                 // the epilogue must have drained this accumulator (fresh barrier: parity 1 passes)
@@ -185,23 +193,32 @@ prefix_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                 tc_fence_after();
                 const uint32_t d_acc = tmem_base + (uint32_t)a * 256u;
                 const uint32_t idesc = item < p.n_full ? p.idesc : p.idesc_half;
+                uint32_t acc = 0u;  // the item's first MMA overwrites the accumulator
                 for (int kb = 0; kb < n_kblocks; ++kb) {
-                    if (!tc_mbar_wait(tc_smem_u32(&s_full[s]), par, abort_flag)) {
+                    if (!tc_mbar_wait(full_s, par, abort_flag)) {
                         ok = false;
                         break;
                     }
                     tc_fence_after();
-                    const uint32_t base = smem0 + (uint32_t)s * stage_bytes;
                     // A = the token tile (128 rows), B = the w_gate rows with the w_up rows right behind them:
-                    // one instruction of N = 2 nt columns (gate | up) per 16-wide K step
-                    const uint64_t dx = tc_smem_desc(base), dw = tc_smem_desc(base + kTcTileBytes);
-#pragma unroll
-                    for (int k = 0; k < kTcTileK / 16; ++k)  // +32 bytes = 2 descriptor units inside the swizzled row
-                        tc_mma(d_acc, dx + 2 * k, dw + 2 * k, (kb > 0 || k > 0) ? 1u : 0u, idesc);
-                    tc_commit(tc_smem_u32(&s_empty[s]));  // the stage is free once these MMAs have read it
+                    // one instruction of N = 2 nt columns (gate | up) per 16-wide K step (+32 bytes = 2 descriptor
+                    // units inside the swizzled row)
+                    const uint64_t dx = dstage, dw = dstage + tile16;
+                    tc_mma(d_acc, dx, dw, acc, idesc);
+                    tc_mma(d_acc, dx + 2, dw + 2, 1u, idesc);
+                    tc_mma(d_acc, dx + 4, dw + 4, 1u, idesc);
+                    tc_mma(d_acc, dx + 6, dw + 6, 1u, idesc);
+                    acc = 1u;
+                    tc_commit(empty_s);  // the stage is free once these MMAs have read it
+                    dstage += stage16;
+                    full_s += 8;
+                    empty_s += 8;
                     if (++s == n_stages) {
                         s = 0;
                         par ^= 1;
+                        dstage = desc0;
+                        full_s = full0;
+                        empty_s = empty0;
                     }
                 }
                 if (ok) tc_commit(tc_smem_u32(&s_acc_full[a]));  // accumulator complete
@@ -472,6 +489,12 @@ down_tc_kernel(const __grid_constant__ CUtensorMap map_z, const __grid_constant_
             int s = 0;
             uint32_t par = 0;
             bool ok = true;
+            // descriptors and barrier addresses advance by additions (see prefix_tc_kernel's issuer)
+            const uint64_t desc0 = tc_smem_desc(smem0);
+            const uint64_t stage16 = stage_bytes >> 4, tile16 = kTcTileBytes >> 4;
+            const uint32_t full0 = tc_smem_u32(&s_full[0]), empty0 = tc_smem_u32(&s_empty[0]);
+            uint64_t dstage = desc0;
+            uint32_t full_s = full0, empty_s = empty0;
             for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++it) {
                 const int a = it & 1;
                 if (!tc_mbar_wait(tc_smem_u32(&s_acc_empty[a]), ((it >> 1) & 1) ^ 1, abort_flag)) {
@@ -480,21 +503,29 @@ down_tc_kernel(const __grid_constant__ CUtensorMap map_z, const __grid_constant_
                 }
                 tc_fence_after();
                 const uint32_t d_acc = tmem_base + (uint32_t)a * 256u;
+                uint32_t acc = 0u;
                 for (int kb = 0; kb < n_kblocks; ++kb) {
-                    if (!tc_mbar_wait(tc_smem_u32(&s_full[s]), par, abort_flag)) {
+                    if (!tc_mbar_wait(full_s, par, abort_flag)) {
                         ok = false;
                         break;
                     }
                     tc_fence_after();
-                    const uint32_t base = smem0 + (uint32_t)s * stage_bytes;
-                    const uint64_t dz = tc_smem_desc(base), dw = tc_smem_desc(base + kTcTileBytes);
-#pragma unroll
-                    for (int k = 0; k < kTcTileK / 16; ++k)
-                        tc_mma(d_acc, dz + 2 * k, dw + 2 * k, (kb > 0 || k > 0) ? 1u : 0u, p.idesc);
-                    tc_commit(tc_smem_u32(&s_empty[s]));
+                    const uint64_t dz = dstage, dw = dstage + tile16;
+                    tc_mma(d_acc, dz, dw, acc, p.idesc);
+                    tc_mma(d_acc, dz + 2, dw + 2, 1u, p.idesc);
+                    tc_mma(d_acc, dz + 4, dw + 4, 1u, p.idesc);
+                    tc_mma(d_acc, dz + 6, dw + 6, 1u, p.idesc);
+                    acc = 1u;
+                    tc_commit(empty_s);
+                    dstage += stage16;
+                    full_s += 8;
+                    empty_s += 8;
                     if (++s == n_stages) {
                         s = 0;
                         par ^= 1;
+                        dstage = desc0;
+                        full_s = full0;
+                        empty_s = empty0;
                     }
                 }
                 if (ok) tc_commit(tc_smem_u32(&s_acc_full[a]));
