@@ -136,6 +136,8 @@ prefix_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
             int s = 0;   // ring position and the parity of its current use
             uint32_t par = 0;
             bool ok = true;
+            const uint32_t full0 = tc_smem_u32(&s_full[0]), empty0 = tc_smem_u32(&s_empty[0]);
+            uint32_t full_s = full0, empty_s = empty0, dst_s = smem0;
             for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
                 int nt, j0, ttile, b;
                 decode(item, nt, j0, ttile);
@@ -144,20 +146,29 @@ prefix_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                 const uint32_t w_bytes = (uint32_t)nt * kTcTileK * 2u;  // one weight tile of this item
                 const CUtensorMap *mg = nt == 128 ? &map_wg : &map_wg_half;
                 const CUtensorMap *mu = nt == 128 ? &map_wu : &map_wu_half;
-                for (int kb = 0; kb < n_kblocks; ++kb, ++kc) {
-                    if (!tc_mbar_wait(tc_smem_u32(&s_empty[s]), par ^ 1, abort_flag)) {
+                const uint32_t tx_bytes = kTcTileBytes + (gated ? 2u : 1u) * w_bytes;
+                const uint32_t up_off = kTcTileBytes + w_bytes;
+                const int row0 = (int)t0;
+                int c0 = 0;  // first column of the K block
+                // like the MMA issuer, this thread's own instructions per K block count: nothing is recomputed
+                for (int kb = 0; kb < n_kblocks; ++kb, ++kc, c0 += kTcTileK) {
+                    if (!tc_mbar_wait(empty_s, par ^ 1, abort_flag)) {
                         ok = false;
                         break;
                     }
-                    const uint32_t bar = tc_smem_u32(&s_full[s]);
-                    const uint32_t dst = smem0 + (uint32_t)s * stage_bytes;
-                    tc_mbar_expect_tx(bar, kTcTileBytes + (gated ? 2u : 1u) * w_bytes);
-                    tc_tma_load(dst, &map_x, kb * kTcTileK, (int)t0, bar);
-                    tc_tma_load(dst + kTcTileBytes, mg, kb * kTcTileK, j0, bar);
-                    if (gated) tc_tma_load(dst + kTcTileBytes + w_bytes, mu, kb * kTcTileK, j0, bar);
+                    tc_mbar_expect_tx(full_s, tx_bytes);
+                    tc_tma_load(dst_s, &map_x, c0, row0, full_s);
+                    tc_tma_load(dst_s + kTcTileBytes, mg, c0, j0, full_s);
+                    if (gated) tc_tma_load(dst_s + up_off, mu, c0, j0, full_s);
+                    dst_s += stage_bytes;
+                    full_s += 8;
+                    empty_s += 8;
                     if (++s == n_stages) {
                         s = 0;
                         par ^= 1;
+                        dst_s = smem0;
+                        full_s = full0;
+                        empty_s = empty0;
                     }
                 }
             }
