@@ -128,3 +128,32 @@ def test_dense_pass_full_width_sampled(clada, oracle):
         y_or, _, n_or = oracle.sparse_ffn(wl.to_numpy_bits(xs[b]), W_in, V_in, W_out, scores[b].astype(np.float64),
                                           float(taus[b]))
         assert n_or > 0 and rel_inf(y[b].cpu().numpy(), y_or) <= FFN_TOL_F32, b
+
+
+def test_stack_call_with_a_batch_runs_dense_passes(clada, oracle):
+    """clada_sparse_ffn_decode_layers with 6 sequences: every layer takes the dense pass with tau_final read at
+    stride L; same bits as the per-layer calls, and one (layer, sequence) checked against the oracle."""
+    L, B = 3, 6
+    w = wl.scaled(wl.WORKLOADS["c3_llama2_7b_stack"], d_model=1024, d_ff=1100, batch=B)
+    weights = [wl.layer_weights(w, l) for l in range(L)]
+    layers = [gpu_layer(wt, clada) for wt in weights]
+    stack = clada.LayerStack(layers)
+    ws = clada.new_workspace(layers[0], B, 0)
+    g = torch.Generator(device="cuda").manual_seed(3)
+    scores = torch.rand(L, B, w.d_ff, generator=g, device="cuda") + 0.5
+    tau = torch.rand(B, L, generator=g, device="cuda") * 0.5 + 0.75
+    x_h = torch.stack([torch.stack([wl.hidden_states(w, l, "decode", b, 1)[0] for b in range(B)]) for l in range(L)])
+    x = x_h.cuda()
+    y_stack = torch.empty(L, B, w.d_model, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    clada.clada_sparse_ffn_decode_layers(stack, x, scores, tau, y_stack, ws, status)
+    y_ref = torch.empty_like(y_stack)
+    for l in range(L):
+        clada.clada_sparse_ffn_decode(layers[l], x[l], scores[l], tau[:, l], L, y_ref[l], ws)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0 and torch.equal(y_stack, y_ref)
+    l, b = 2, 4
+    W_in, V_in, W_out = oracle_weights(weights[l])
+    y_or, _, n_or = oracle.sparse_ffn(wl.to_numpy_bits(x_h[l, b]), W_in, V_in, W_out,
+                                      scores[l, b].cpu().numpy().astype(np.float64), float(tau[b, l].item()))
+    assert n_or > 0 and rel_inf(y_stack[l, b].cpu().numpy(), y_or) <= FFN_TOL_F32
