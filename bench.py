@@ -686,14 +686,41 @@ def run_ours(args):
         host_in = [t.cpu().pin_memory() for t in dev_in]
         hy = torch.empty(dev_out.shape, dtype=dev_out.dtype).pin_memory()
 
+        # Pipelined across steps: the inputs of step i+1 cross PCIe (copy stream, into staging buffers on the device)
+        # while step i computes; a step waits for its own inputs, moves them from staging into the tensors the
+        # launches read (device-to-device), runs, and reads its result back.  Every step's inputs and result
+        # travel inside the timed region; a run of K steps issues K+1 input copies (the last one for nobody).
+        copy_stream = torch.cuda.Stream(device=dev)
+        staging = [torch.empty_like(t) for t in dev_in]
+        h2d_done, staging_free = torch.cuda.Event(), torch.cuda.Event()
+        e2e_state = {"primed": False}
+
+        def start_h2d():
+            copy_stream.wait_event(staging_free)
+            with torch.cuda.stream(copy_stream):
+                for st_, ht in zip(staging, host_in):
+                    st_.copy_(ht, non_blocking=True)
+                h2d_done.record(copy_stream)
+
         def e2e_step():
-            for dt, ht in zip(dev_in, host_in):
-                dt.copy_(ht, non_blocking=True)
+            cur = torch.cuda.current_stream()
+            if not e2e_state["primed"]:      # the first step of a run: its own copy, nothing to overlap with
+                staging_free.record(cur)
+                start_h2d()
+                e2e_state["primed"] = True
+            cur.wait_event(h2d_done)
+            for dt, st_ in zip(dev_in, staging):
+                dt.copy_(st_, non_blocking=True)
+            staging_free.record(cur)
+            start_h2d()
             run()
             hy.copy_(dev_out, non_blocking=True)
 
         e2e_step()
+        torch.cuda.synchronize()
+        e2e_state["primed"] = False          # the timed run starts with nothing in flight
         e2e_ms = _timed(e2e_step, args.steps, barrier)
+        torch.cuda.synchronize()
 
         # the same step over nested index lists, reported beside the headline (not in place of it)
         nested_ms = nested_ffn_ms = None
@@ -803,7 +830,8 @@ def run_ours(args):
                    "decode_tokens_per_sparsity": job.N, "sparsities": list(w.sparsities), "batch": w.batch,
                    "l2": job.l2_note, "cuda_graph": bool(args.graph), "avg_kept_neurons_per_token": kept,
                    "lambda": LAMBDA, "gamma": GAMMA, "step": job.step_note},
-        "e2e": {"value": e2e_value, "unit": "tokens/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+        "e2e": {"value": e2e_value, "unit": "tokens/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "pipelined": "inputs of step i+1 are copied (pinned host -> device staging) while step i computes"},
         "gpu_launches": job.launches_per_step * args.steps,
         "roofline": roofline,
         "prefix_roofline": {"bound": "tensor", "kernel": "prefix_tc_kernel (+finalize)", "ms": prefix_ms,
