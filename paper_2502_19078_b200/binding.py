@@ -14,7 +14,7 @@ from typing import Optional, Sequence
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libclada.so")
+LIB_PATH = os.environ.get("CLADA_LIB") or os.path.join(_HERE, "libclada.so")   # CLADA_LIB: another build of the library
 
 CLADA_F32, CLADA_BF16, CLADA_F16 = 0, 1, 2
 STATUS_BAD_TOKEN, STATUS_NONFINITE_LOGIT, STATUS_TIMEOUT = 1, 2, 4

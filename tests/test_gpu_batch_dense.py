@@ -103,11 +103,13 @@ def test_dense_pass_fp16_layer(clada, oracle):
           y_dtypes=(torch.float32, torch.float16))
 
 
-def test_dense_pass_full_width_sampled(clada, oracle):
-    """c5's width (d_model 5120, d_ff 13824, 16 sequences) in the launch configuration the benchmark times:
-    three sequences checked against the oracle (one that keeps nothing, one that keeps all, one at 40 %)."""
-    w = wl.WORKLOADS["c5_13b_b16"]
-    B, d, F = 16, w.d_model, w.d_ff
+@pytest.mark.parametrize("name,picks", [("c5_13b_b16", (2, 7, 15)), ("c4_llama3_8b_b8", (0, 2, 5))])
+def test_dense_pass_full_width_sampled(clada, oracle, name, picks):
+    """The batched workloads' own widths and batch sizes (c5: d_model 5120, d_ff 13824, 16 sequences; c4: 4096,
+    14336, 8) in the launch configuration the benchmark times: three sequences checked against the oracle (among
+    them one that keeps all), and the one that keeps nothing is zero."""
+    w = wl.WORKLOADS[name]
+    B, d, F = w.batch, w.d_model, w.d_ff
     weights = wl.layer_weights(w, 0)
     layer = gpu_layer(weights, clada)
     W_in, V_in, W_out = oracle_weights(weights)
@@ -124,7 +126,7 @@ def test_dense_pass_full_width_sampled(clada, oracle):
     torch.cuda.synchronize()
     assert int(status.item()) == 0
     assert bool((y[1] == 0).all())
-    for b in (2, 7, 15):
+    for b in picks:
         y_or, _, n_or = oracle.sparse_ffn(wl.to_numpy_bits(xs[b]), W_in, V_in, W_out, scores[b].astype(np.float64),
                                           float(taus[b]))
         assert n_or > 0 and rel_inf(y[b].cpu().numpy(), y_or) <= FFN_TOL_F32, b
