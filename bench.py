@@ -48,19 +48,19 @@ def recorded_traffic(kernel: str, workload: str):
     """DRAM read + write bytes per launch (or per layer pass) of `kernel` from the ncu capture on record under
     profiles/ (written by paper_2502_19078_b200.ncu_summary), or None when there is no record for this workload
     or the kernel's sources have changed since the counters were taken."""
-    path = os.path.join(PROFILES, f"traffic_{kernel}.txt")
-    try:
-        rec = {}
-        with open(path) as f:
-            for line in f:
-                if ":" in line and not line.startswith("#"):
-                    k, v = line.split(":", 1)
-                    rec[k.strip()] = v.strip()
-        if rec.get("workload") != workload or rec.get("sources_sha256") != sources_hash(kernel):
-            return None
-        return float(rec["dram_bytes_per_unit"])
-    except Exception:
-        return None
+    for name in (f"traffic_{kernel}_{workload}.txt", f"traffic_{kernel}.txt"):
+        try:
+            rec = {}
+            with open(os.path.join(PROFILES, name)) as f:
+                for line in f:
+                    if ":" in line and not line.startswith("#"):
+                        k, v = line.split(":", 1)
+                        rec[k.strip()] = v.strip()
+            if rec.get("workload") == workload and rec.get("sources_sha256") == sources_hash(kernel):
+                return float(rec["dram_bytes_per_unit"])
+        except Exception:
+            pass
+    return None
 
 
 def _peaks():

@@ -65,6 +65,8 @@ def main(argv=None):
     ap.add_argument("--workload", required=True)
     ap.add_argument("--units-per-launch", type=int, default=1, help="layer passes one captured launch processes")
     ap.add_argument("--note", default="")
+    ap.add_argument("--per-workload", action="store_true",
+                    help="write traffic_<kernel>_<workload>.txt (a second workload's record beside the kernel's first)")
     args = ap.parse_args(argv)
     launches = read_raw_csv(args.csv, args.kernel)
     if not launches:
@@ -72,7 +74,8 @@ def main(argv=None):
     rd = [l["dram__bytes_read.sum"] for l in launches]
     wr = [l["dram__bytes_write.sum"] for l in launches]
     per_unit = (sum(rd) + sum(wr)) / len(launches) / args.units_per_launch
-    path = os.path.join(ROOT, "profiles", f"traffic_{args.kernel}.txt")
+    name = f"traffic_{args.kernel}_{args.workload}.txt" if args.per_workload else f"traffic_{args.kernel}.txt"
+    path = os.path.join(ROOT, "profiles", name)
     with open(path, "w") as f:
         f.write("# DRAM traffic of one kernel from an ncu capture (dram__bytes_read.sum + dram__bytes_write.sum),\n"
                 "# written by python -m paper_2502_19078_b200.ncu_summary; bench.py reports it while the hash matches.\n")
