@@ -82,6 +82,8 @@ def _case(clada, oracle, name, kw, B, act=0, y_dtypes=(torch.float32,), seed=0, 
     ("c4_llama3_8b_b8", {"d_model": 2048, "d_ff": 9000}, 9),      # 61 neurons per CTA: three padded rows per box
     ("c4_llama3_8b_b8", {"d_model": 256, "d_ff": 18900}, 7),      # 128 neurons per CTA, the most a launch takes
     ("c5_13b_b16", {"d_model": 8192, "d_ff": 600}, 6),            # 16 column tiles per member: three N = 16 instructions per K step
+    ("c2_llama2_7b_layer", {"d_model": 8, "d_ff": 5}, 5),         # one K block of 8 columns, members 1-3 without a column tile
+    ("c2_llama2_7b_layer", {"d_model": 72, "d_ff": 130}, 16),     # one neuron per CTA, ragged everything
 ])
 def test_dense_pass_matches_oracle(clada, oracle, name, kw, B):
     _case(clada, oracle, name, kw, B, y_dtypes=(torch.float32, torch.bfloat16), outputs=(B == 8))
