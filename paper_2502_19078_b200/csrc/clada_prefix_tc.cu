@@ -10,14 +10,15 @@
 // lane.  The sum over a tile's tokens is then a sum over lanes: a halving butterfly per 16 neurons (16 shuffles),
 // the four warps' results combined through shared memory in warp order (deterministic).
 //
-// One persistent CTA per SM, 192 threads:
+// One persistent CTA per SM, 320 threads:
 //   warp 0      TMA producer: per 64-wide K block the token tile and the two weight tiles, 128-byte swizzle, into a
 //               4-stage shared-memory ring (mbarrier full/empty);
 //   warp 1      allocates 512 TMEM columns (two accumulators), issues tcgen05.mma (M128 N256 K16, kind::f16) from
 //               one elected thread, commits stages and accumulators;
-//   warps 2-5   epilogue: tcgen05.ld 32x32b.x16 of gate and up columns, neuron value, optional store of 16
-//               consecutive neurons of the thread's token, squares, butterfly; the second accumulator lets tile
-//               i+1's MMAs run under tile i's epilogue.
+//   warps 2-9   epilogue (two warps per quarter of the TMEM lanes, alternate groups of 16 neurons): tcgen05.ld
+//               32x32b.x16 of gate and up columns, neuron value, optional store of 16 consecutive neurons of the
+//               thread's token, squares, butterfly; the second accumulator lets tile i+1's MMAs run under tile
+//               i's epilogue, and eight warps halve what is exposed after a CTA's last tile.
 // Work items are (128 neurons x 128 tokens), neuron tile major; a token tile never leaves its prompt and rows
 // past the prompt's end count as zero.  The items left after the last full wave of CTAs are issued as two
 // 64-neuron halves each (N = 128) when they then fit one wave, which halves that wave's time.
@@ -35,6 +36,8 @@ namespace clada {
 
 constexpr int kTcMaxStages = 8;
 constexpr int kTcThreads = 192;
+constexpr int kTcEpiWarps = 8;                    // prefix_tc_kernel: two epilogue warps per TMEM lane quarter
+constexpr int kTcPfThreads = 64 + 32 * kTcEpiWarps;
 constexpr uint32_t kTcTileBytes = kTcTileM * kTcTileK * 2;       // 16 KiB: a 128-row tile
 constexpr uint32_t kTcRingBytes = 192 * 1024;                    // shared-memory ring of the statistics kernel
 constexpr uint32_t kTcTmemCols = 512;                            // two accumulators of up to 256 columns
@@ -58,7 +61,7 @@ struct TcParams {
     SeqTable tab;
 };
 
-__global__ void __launch_bounds__(kTcThreads, 1)
+__global__ void __launch_bounds__(kTcPfThreads, 1)
 prefix_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_wg,
                  const __grid_constant__ CUtensorMap map_wu, const __grid_constant__ CUtensorMap map_wg_half,
                  const __grid_constant__ CUtensorMap map_wu_half, const TcParams p) {
@@ -111,8 +114,8 @@ prefix_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
         }
         for (int a = 0; a < 2; ++a) {
             tc_mbar_init(tc_smem_u32(&s_acc_full[a]), 1);
-            tc_mbar_init(tc_smem_u32(&s_acc_empty[a]), 4);  // one arrival per epilogue warp
-            tc_mbar_init(tc_smem_u32(&s_epi[a]), 4);
+            tc_mbar_init(tc_smem_u32(&s_acc_empty[a]), kTcEpiWarps);  // one arrival per epilogue warp
+            tc_mbar_init(tc_smem_u32(&s_epi[a]), kTcEpiWarps);
         }
         s_abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -237,8 +240,10 @@ prefix_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
             if (!ok) *abort_flag = 1;
         }
     } else {
-        // ---- epilogue warps (2..5): warp w may touch TMEM lanes 32 (w % 4) .. +31 = 32 tokens ------------
+        // ---- epilogue warps (2..9): warp w may touch TMEM lanes 32 (w % 4) .. +31 = 32 tokens; the two warps of a
+        // lane quarter take alternate groups of 16 columns ------------
         const int quarter = warp & 3;
+        const int col_half = (warp - 2) >> 2;
         const bool b16 = lane & 16, b8 = lane & 8, b4 = lane & 4, b2 = lane & 2;
         const int my_val = (b16 ? 8 : 0) + (b8 ? 4 : 0) + (b4 ? 2 : 0) + (b2 ? 1 : 0);
         const int e = (warp - 2) * 32 + lane;  // 0..127: the neuron of the tile this thread finishes
@@ -258,7 +263,7 @@ prefix_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
             }
             tc_fence_after();
             const uint32_t t_acc = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)a * 256u;
-            for (int c0 = 0; c0 < nt; c0 += 16) {
+            for (int c0 = 16 * col_half; c0 < nt; c0 += 32) {
                 uint32_t rg[16], ru[16];
                 tc_ld16(t_acc + c0, rg);
                 if (gated) {
@@ -313,7 +318,7 @@ prefix_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                 break;
             }
             const int j = jbase + e;
-            if (e < nt && j < p.d_ff)
+            if (col_half == 0 && e < nt && j < p.d_ff)
                 p.partials[(size_t)ttile * p.d_ff + j] = ((s_col[a][0][e] + s_col[a][1][e]) + s_col[a][2][e]) + s_col[a][3][e];
         }
         if (!ok) *abort_flag = 1;
@@ -384,7 +389,7 @@ int run_prefix_partials_tc(const clada_layer *layer, const void *X, const SeqTab
         configured[di.device & 63] = true;
     }
     const int grid = (int)std::min<long long>((long long)p.n_full + p.n_half, di.num_sms);
-    prefix_tc_kernel<<<grid, kTcThreads, smem, st>>>(map_x, map_wg, map_wu, map_wg_half, map_wu_half, p);
+    prefix_tc_kernel<<<grid, kTcPfThreads, smem, st>>>(map_x, map_wg, map_wu, map_wg_half, map_wu_half, p);
     CLADA_CUDA_TRY(cudaGetLastError());
     return CLADA_OK;
 }
