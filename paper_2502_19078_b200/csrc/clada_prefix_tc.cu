@@ -36,7 +36,7 @@ namespace clada {
 
 constexpr int kTcMaxStages = 8;
 constexpr int kTcThreads = 192;
-constexpr int kTcEpiWarps = 8;                    // prefix_tc_kernel: two epilogue warps per TMEM lane quarter
+constexpr int kTcEpiWarps = 8;   // prefix_tc_kernel: epilogue warps, a multiple of 4 (TMEM lane quarters); 12 and 16 measured the same
 constexpr int kTcPfThreads = 64 + 32 * kTcEpiWarps;
 constexpr uint32_t kTcTileBytes = kTcTileM * kTcTileK * 2;       // 16 KiB: a 128-row tile
 constexpr uint32_t kTcRingBytes = 192 * 1024;                    // shared-memory ring of the statistics kernel
@@ -263,7 +263,7 @@ prefix_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
             }
             tc_fence_after();
             const uint32_t t_acc = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)a * 256u;
-            for (int c0 = 16 * col_half; c0 < nt; c0 += 32) {
+            for (int c0 = 16 * col_half; c0 < nt; c0 += 4 * kTcEpiWarps) {
                 uint32_t rg[16], ru[16];
                 tc_ld16(t_acc + c0, rg);
                 if (gated) {
