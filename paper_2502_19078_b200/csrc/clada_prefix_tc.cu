@@ -474,22 +474,31 @@ down_tc_kernel(const __grid_constant__ CUtensorMap map_z, const __grid_constant_
             int s = 0;  // ring position and the parity of its current use, kept incrementally
             uint32_t par = 0;
             bool ok = true;
+            // nothing in the K loop is recomputed (see prefix_tc_kernel): addresses advance by additions
+            const uint32_t full0 = tc_smem_u32(&s_full[0]), empty0 = tc_smem_u32(&s_empty[0]);
+            uint32_t full_s = full0, empty_s = empty0, dst_s = smem0;
             for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
                 int dtile, ttile;
                 tile_of(item, dtile, ttile);
-                for (int kb = 0; kb < n_kblocks; ++kb, ++kc) {
-                    if (!tc_mbar_wait(tc_smem_u32(&s_empty[s]), par ^ 1, abort_flag)) {
+                const int row_z = ttile * kTcTileM, row_w = dtile * nd;
+                int c0 = 0;
+                for (int kb = 0; kb < n_kblocks; ++kb, ++kc, c0 += kTcTileK) {
+                    if (!tc_mbar_wait(empty_s, par ^ 1, abort_flag)) {
                         ok = false;
                         break;
                     }
-                    const uint32_t bar = tc_smem_u32(&s_full[s]);
-                    const uint32_t dst = smem0 + (uint32_t)s * stage_bytes;
-                    tc_mbar_expect_tx(bar, stage_bytes);
-                    tc_tma_load(dst, &map_z, kb * kTcTileK, ttile * kTcTileM, bar);
-                    tc_tma_load(dst + kTcTileBytes, &map_w, kb * kTcTileK, dtile * nd, bar);
+                    tc_mbar_expect_tx(full_s, stage_bytes);
+                    tc_tma_load(dst_s, &map_z, c0, row_z, full_s);
+                    tc_tma_load(dst_s + kTcTileBytes, &map_w, c0, row_w, full_s);
+                    dst_s += stage_bytes;
+                    full_s += 8;
+                    empty_s += 8;
                     if (++s == n_stages) {
                         s = 0;
                         par ^= 1;
+                        dst_s = smem0;
+                        full_s = full0;
+                        empty_s = empty0;
                     }
                 }
             }
