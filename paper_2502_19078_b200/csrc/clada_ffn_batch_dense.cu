@@ -141,18 +141,10 @@ __device__ __forceinline__ uint16_t bd_to16(int dtype, float v, float &back) {
 // The MMAs of one phase-2 stage (up to 8 K steps of 16 neurons), issued back to back from descriptors computed
 // beforehand: the issuing thread's own instructions between two MMAs are what limits their rate.
 //   da: MN-major descriptor of the stage's first 16 rows (the next K step lies 2048 bytes on);
-//   dh: K-major descriptor of the first K step's rows of the h image, kq its K step inside the 64-neuron block
-//       (the next step lies 32 bytes on, after the fourth step of a block the next block follows).
+//   dhv: the K-major descriptors of the member's K steps in the h image, computed once per launch and member.
 template <bool WIDE>
-__device__ __forceinline__ void bd_issue_stage(uint32_t d_y, uint64_t da, uint64_t dh, int kq, int ksteps, uint32_t acc,
-                                               uint32_t idesc) {
-    constexpr uint64_t kBlkStep = (kBdImgBlock >> 4) - 6;
-    uint64_t dhv[kBdMaxRows / 16];
-#pragma unroll
-    for (int k = 0; k < kBdMaxRows / 16; ++k) {
-        dhv[k] = dh;
-        dh += ((kq + k) & 3) == 3 ? kBlkStep : 2;
-    }
+__device__ __forceinline__ void bd_issue_stage(uint32_t d_y, uint64_t da, const uint64_t (&dhv)[kBdMaxRows / 16], int ksteps,
+                                               uint32_t acc, uint32_t idesc) {
 #pragma unroll
     for (int k = 0; k < kBdMaxRows / 16; ++k) {
         if (k < ksteps) {
@@ -164,6 +156,15 @@ __device__ __forceinline__ void bd_issue_stage(uint32_t d_y, uint64_t da, uint64
                 tc_mma(d_y, da + 128 * k, dhv[k] + 256, 1u, idesc);
             }
         }
+    }
+}
+// The K-major descriptors of a member's K steps in the h image: the next step lies 32 bytes on, after the fourth
+// step of a 64-neuron block the next block follows.
+__device__ __forceinline__ void bd_member_descs(uint64_t dh0, int mm, int ksteps, uint64_t (&dhv)[kBdMaxRows / 16]) {
+#pragma unroll
+    for (int k = 0; k < kBdMaxRows / 16; ++k) {
+        const int kk16 = mm * ksteps + k;
+        dhv[k] = dh0 + (uint64_t)(kk16 >> 2) * (kBdImgBlock >> 4) + (uint64_t)(kk16 & 3) * 2;
     }
 }
 __device__ __forceinline__ void bd_epi_sync() { asm volatile("bar.sync 2, 128;" ::: "memory"); }
@@ -331,19 +332,15 @@ sparse_ffn_batch_dense_kernel(const __grid_constant__ CUtensorMap map_x, const _
             const uint64_t dmn0 = bd_smem_desc_mn(smem0, slot_bytes);
             const uint64_t dh0 = tc_smem_desc(himg_s);
             uint64_t dstage2 = dmn0 + (uint64_t)s * stage16;
-            auto run_p2 = [&](int mm, int t, uint32_t acc) -> bool {  // the MMAs of one stage
+            auto run_p2 = [&](const uint64_t (&dhv)[kBdMaxRows / 16], int t, uint32_t acc) -> bool {  // the MMAs of one stage
                 if (!tc_mbar_wait(tc_smem_u32(&s_full[s]), par, abort_flag)) return false;
                 tc_fence_after();
-                if (acc && t < 8) BD_CLOCK(16 + 6 * t + 2 * (mm - (mm > mem ? 1 : 0)));
                 const uint32_t d_y = tmem_base + (uint32_t)t * tile_cols;
-                const int kk16 = mm * ksteps;  // first K step of member mm in the group's h
-                const uint64_t dh = dh0 + (uint64_t)(kk16 >> 2) * (kBdImgBlock >> 4) + (uint64_t)(kk16 & 3) * 2;
                 if (p.wide)
-                    bd_issue_stage<true>(d_y, dstage2, dh, kk16 & 3, ksteps, acc, p.idesc_p2w);
+                    bd_issue_stage<true>(d_y, dstage2, dhv, ksteps, acc, p.idesc_p2w);
                 else
-                    bd_issue_stage<false>(d_y, dstage2, dh, kk16 & 3, ksteps, acc, p.idesc_p2);
+                    bd_issue_stage<false>(d_y, dstage2, dhv, ksteps, acc, p.idesc_p2);
                 tc_commit(tc_smem_u32(&s_empty[s]));
-                if (acc && t < 8) BD_CLOCK(17 + 6 * t + 2 * (mm - (mm > mem ? 1 : 0)));
                 dstage2 += stage16;
                 if (++s == n_stages) {
                     s = 0;
@@ -352,15 +349,22 @@ sparse_ffn_batch_dense_kernel(const __grid_constant__ CUtensorMap map_x, const _
                 }
                 return true;
             };
+            // the B descriptors of the four members' K steps stay in registers for the whole phase
+            uint64_t dh_own[kBdMaxRows / 16], dh_oth[kBdMembers - 1][kBdMaxRows / 16];
+            bd_member_descs(dh0, mem, ksteps, dh_own);
+#pragma unroll
+            for (int mo = 0; mo < kBdMembers - 1; ++mo) bd_member_descs(dh0, mo + (mo >= mem ? 1 : 0), ksteps, dh_oth[mo]);
             // this CTA's own part of h is in shared memory first; the other members' parts follow the exchange
             if (ok && !tc_mbar_wait(tc_smem_u32(&s_h_own), 0, abort_flag)) ok = false;
             tc_fence_after();
             BD_TRACE(3);
-            for (int t = 0; t < nt && ok; ++t) ok = run_p2(mem, t, 0u);
+            for (int t = 0; t < nt && ok; ++t) ok = run_p2(dh_own, t, 0u);
             if (ok && !tc_mbar_wait(tc_smem_u32(&s_h_all), 0, abort_flag)) ok = false;
             tc_fence_after();
             for (int t = 0; t < nt && ok; ++t) {
-                for (int mo = 0; mo < kBdMembers - 1 && ok; ++mo) ok = run_p2(mo + (mo >= mem ? 1 : 0), t, 1u);
+#pragma unroll
+                for (int mo = 0; mo < kBdMembers - 1; ++mo)
+                    if (ok) ok = run_p2(dh_oth[mo], t, 1u);
                 if (ok) tc_commit(tc_smem_u32(&s_tile_full[t]));  // this tile's partial output is complete
             }
             BD_TRACE(4);
