@@ -48,7 +48,9 @@ def build(force: bool = False, verbose: bool = False) -> str:
     from concurrent.futures import ThreadPoolExecutor
     os.makedirs(OBJ_DIR, exist_ok=True)
     newest_header = max(os.path.getmtime(h) for h in _headers())
-    base = [_nvcc()] + NVCC_FLAGS + ["-I", INCLUDE, "-I", CSRC]
+    # CLADA_NVCC_FLAGS: extra compiler flags for an opt-in build, e.g. -DCLADA_NVTX (NVTX ranges around the C
+    # entry points) or -DCLADA_STACK_TRACE / -DCLADA_BD_TRACE (in-kernel time stamps); rebuild with --force
+    base = [_nvcc()] + NVCC_FLAGS + os.environ.get("CLADA_NVCC_FLAGS", "").split() + ["-I", INCLUDE, "-I", CSRC]
     if verbose:
         base += ["-Xptxas", "-v"]
     jobs, objs = [], []

@@ -17,6 +17,7 @@
 #include <algorithm>
 
 #include "common.cuh"
+#include "nvtx_ranges.cuh"
 #include "prefix_common.cuh"
 
 namespace clada {
@@ -220,6 +221,7 @@ size_t clada_cett_workspace_bytes(const clada_layer *layer, const int64_t *seq_o
 int clada_cett_threshold_search(const clada_layer *layer, const void *X, const int64_t *seq_offsets, int32_t B,
                                 float bound, float *tau_base, float *mean_cett, float *scores, void *ws,
                                 size_t ws_bytes, int32_t *status, void *stream) {
+    CLADA_RANGE("clada_cett_threshold_search");
     (void)status;
     int rc = validate_layer(layer, true);
     if (rc != CLADA_OK) return rc;
@@ -298,6 +300,7 @@ int clada_cett_threshold_search(const clada_layer *layer, const void *X, const i
 // k = 0 .. d_ff, read back from the workspace of the last clada_cett_threshold_search on the same arguments.
 int clada_cett_curve(const clada_layer *layer, const int64_t *seq_offsets, int32_t B, int32_t sample,
                      const void *ws, size_t ws_bytes, double *cum_out, int32_t *order_out, void *stream) {
+    CLADA_RANGE("clada_cett_curve");
     if (!layer || !ws || !cum_out) return CLADA_ERR_NULL;
     int rc = check_offsets(seq_offsets, B);
     if (rc != CLADA_OK) return rc;

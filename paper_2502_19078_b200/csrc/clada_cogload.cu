@@ -11,6 +11,7 @@
 #include <cooperative_groups.h>
 
 #include "common.cuh"
+#include "nvtx_ranges.cuh"
 
 namespace cg = cooperative_groups;
 
@@ -322,6 +323,7 @@ extern "C" {
 int clada_cogload(const void *logits, int32_t logits_dtype, int32_t B, int64_t V, int64_t row_stride,
                   const int32_t *token_id, float *surprisal, float *entropy, int32_t *status,
                   void *stream) {
+    CLADA_RANGE("clada_cogload");
     return launch_cogload(logits, logits_dtype, B, V, row_stride, token_id, surprisal, entropy, status,
                           nullptr, nullptr, nullptr, 0.f, 0.f, 0, nullptr, nullptr, stream);
 }
@@ -331,6 +333,7 @@ int clada_cogload(const void *logits, int32_t logits_dtype, int32_t B, int64_t V
 int clada_cogload_level(const void *logits, int32_t logits_dtype, int32_t B, int64_t V, int64_t row_stride,
                         const int32_t *token_id, float tau_s, float tau_H, float *surprisal, float *entropy,
                         int32_t *level, int32_t *status, void *stream) {
+    CLADA_RANGE("clada_cogload_level");
     if (!level) return CLADA_ERR_NULL;
     return launch_cogload(logits, logits_dtype, B, V, row_stride, token_id, surprisal, entropy, status,
                           nullptr, nullptr, nullptr, tau_s, tau_H, 0, nullptr, level, stream);
@@ -339,6 +342,7 @@ int clada_cogload_level(const void *logits, int32_t logits_dtype, int32_t B, int
 int clada_adjust_threshold(const float *tau_base, const float *lambda, const float *gamma, float tau_s,
                            float tau_H, const float *surprisal, const float *entropy, int32_t B,
                            int32_t L, float *tau_final, void *stream) {
+    CLADA_RANGE("clada_adjust_threshold");
     if (!tau_base || !lambda || !gamma || !surprisal || !entropy || !tau_final) return CLADA_ERR_NULL;
     if (B <= 0 || L <= 0) return CLADA_ERR_SHAPE;
     const int threads = 128;
@@ -354,6 +358,7 @@ int clada_cogload_adjust(const void *logits, int32_t logits_dtype, int32_t B, in
                          const float *lambda, const float *gamma, float tau_s, float tau_H, int32_t L,
                          float *surprisal, float *entropy, float *tau_final, int32_t *status,
                          void *stream) {
+    CLADA_RANGE("clada_cogload_adjust");
     if (!tau_base || !lambda || !gamma || !tau_final) return CLADA_ERR_NULL;
     if (L <= 0) return CLADA_ERR_SHAPE;
     return launch_cogload(logits, logits_dtype, B, V, row_stride, token_id, surprisal, entropy, status,

@@ -4,6 +4,7 @@
 #include <algorithm>
 
 #include "common.cuh"
+#include "nvtx_ranges.cuh"
 #include "ffn_batch.cuh"
 #include "ffn_common.cuh"
 #include "ffn_single.cuh"
@@ -168,6 +169,7 @@ extern "C" int clada_sparse_ffn_decode(const clada_layer *layer, const void *x, 
                                        void *y, int32_t y_dtype, uint8_t *mask_out, int32_t *idx_out,
                                        int32_t *count_out, void *ws, size_t ws_bytes, int32_t *status,
                                        void *stream) {
+    CLADA_RANGE("clada_sparse_ffn_decode");
     return decode_with_workspace(layer, x, B, scores, tau_final, tau_stride, y, y_dtype, mask_out, idx_out,
                                  count_out, ws, ws_bytes, status, stream);
 }
@@ -178,6 +180,7 @@ extern "C" int clada_sparse_ffn_decode_nested(const clada_layer *layer, const vo
                                               const int32_t *order, const int32_t *counts, const int32_t *level,
                                               void *y, int32_t y_dtype, int32_t *count_out, void *ws,
                                               size_t ws_bytes, int32_t *status, void *stream) {
+    CLADA_RANGE("clada_sparse_ffn_decode_nested");
     int rc = validate_layer(layer, false);
     if (rc != CLADA_OK) return rc;
     if (!x || !order || !counts || !level || !y) return CLADA_ERR_NULL;
@@ -222,6 +225,7 @@ extern "C" int clada_sparse_ffn_decode_layers(const clada_layer *layers, int32_t
                                               const float *scores, const float *tau_final, void *y,
                                               int32_t y_dtype, void *ws, size_t ws_bytes, int32_t *status,
                                               void *stream) {
+    CLADA_RANGE("clada_sparse_ffn_decode_layers");
     if (!layers || !x || !scores || !tau_final || !y) return CLADA_ERR_NULL;
     if (L <= 0 || B <= 0) return CLADA_ERR_SHAPE;
     if (!dtype_ok(y_dtype)) return CLADA_ERR_DTYPE;
@@ -285,6 +289,7 @@ extern "C" int clada_sparse_ffn_decode_static(const clada_layer *layer, const vo
                                               int64_t tau_stride, void *y, int32_t y_dtype,
                                               uint8_t *mask_out, int32_t *idx_out, int32_t *count_out,
                                               int32_t *status, void *stream) {
+    CLADA_RANGE("clada_sparse_ffn_decode_static");
     // Everything that can be refused is refused before the first enqueue.
     int rc = decode_validate(layer, x, B, scores, tau_final, tau_stride, y, y_dtype);
     if (rc != CLADA_OK) return rc;

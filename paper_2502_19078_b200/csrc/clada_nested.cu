@@ -21,6 +21,7 @@
 #include <algorithm>
 
 #include "common.cuh"
+#include "nvtx_ranges.cuh"
 
 namespace clada {
 
@@ -174,6 +175,7 @@ using namespace clada;
 extern "C" int clada_nested_build(const float *scores, int32_t B, int32_t d_ff, const float *tau_base,
                                   int64_t tau_stride, float lambda, float gamma, int32_t *order, int32_t *counts,
                                   void *stream) {
+    CLADA_RANGE("clada_nested_build");
     if (!scores || !tau_base || !order || !counts) return CLADA_ERR_NULL;
     if (B <= 0 || d_ff <= 0 || tau_stride < 0) return CLADA_ERR_SHAPE;
     if (d_ff > kNestMaxN || B > 65535) return CLADA_ERR_UNSUPPORTED;

@@ -9,6 +9,7 @@
 #include <math.h>
 
 #include "common.cuh"
+#include "nvtx_ranges.cuh"
 #include "prefix_common.cuh"
 
 namespace clada {
@@ -387,6 +388,7 @@ extern "C" {
 
 int clada_prefix_scores(const clada_layer *layer, const void *X, const int64_t *seq_offsets, int32_t B,
                         float *scores, void *ws, size_t ws_bytes, int32_t *status, void *stream) {
+    CLADA_RANGE("clada_prefix_scores");
     (void)status;
     int rc = validate_layer(layer, true);
     if (rc != CLADA_OK) return rc;
@@ -409,6 +411,7 @@ int clada_prefix_scores(const clada_layer *layer, const void *X, const int64_t *
 
 int clada_prefix_accumulate(const clada_layer *layer, const void *X, const int64_t *seq_offsets, int32_t B,
                             float *sumsq, void *Z, void *ws, size_t ws_bytes, int32_t *status, void *stream) {
+    CLADA_RANGE("clada_prefix_accumulate");
     int rc = validate_layer(layer, false);
     if (rc != CLADA_OK) return rc;
     if (!X || !sumsq) return CLADA_ERR_NULL;
@@ -445,6 +448,7 @@ int clada_prefix_accumulate(const clada_layer *layer, const void *X, const int64
 }
 
 int clada_prefix_finish(const clada_layer *layer, const float *sumsq, int32_t B, float *scores, void *stream) {
+    CLADA_RANGE("clada_prefix_finish");
     int rc = validate_layer(layer, true);
     if (rc != CLADA_OK) return rc;
     if (!sumsq || !scores) return CLADA_ERR_NULL;
@@ -458,6 +462,7 @@ int clada_prefix_finish(const clada_layer *layer, const float *sumsq, int32_t B,
 
 int clada_prefill_down(const clada_layer *layer, const void *w_down, const void *Z, int64_t T, void *Y,
                        int32_t y_dtype, int32_t *status, void *stream) {
+    CLADA_RANGE("clada_prefill_down");
     int rc = validate_layer(layer, false);
     if (rc != CLADA_OK) return rc;
     if (!w_down || !Z || !Y) return CLADA_ERR_NULL;
@@ -472,6 +477,7 @@ int clada_prefill_down(const clada_layer *layer, const void *w_down, const void 
 int clada_refine_scores(const clada_layer *layer, const void *X, const int64_t *seq_offsets, int32_t B,
                         const float *tau_base, const float *guard_mults, int32_t n_guard, float rel_band,
                         float *scores, void *ws, size_t ws_bytes, int32_t *status, void *stream) {
+    CLADA_RANGE("clada_refine_scores");
     (void)status;
     int rc = validate_layer(layer, false);
     if (rc != CLADA_OK) return rc;
@@ -541,6 +547,7 @@ int clada_prefix_select(const clada_layer *layer, const void *X, const int64_t *
                         const float *tau_base, const float *guard_mults, int32_t n_guard, float *scores,
                         uint8_t *mask, int32_t *idx, int32_t *count, void *ws, size_t ws_bytes,
                         int32_t *status, void *stream) {
+    CLADA_RANGE("clada_prefix_select");
     int rc = clada_prefix_scores(layer, X, seq_offsets, B, scores, ws, ws_bytes, status, stream);
     if (rc != CLADA_OK || !tau_base) return rc;
     if (n_guard > 0 && guard_mults) {

@@ -3,6 +3,7 @@
 #include <math.h>
 
 #include "common.cuh"
+#include "nvtx_ranges.cuh"
 
 namespace clada {
 
@@ -108,6 +109,7 @@ extern "C" {
 
 int clada_select(const float *scores, int32_t B, int32_t d_ff, const float *tau, int64_t tau_stride,
                  uint8_t *mask, int32_t *idx, int32_t *count, void *stream) {
+    CLADA_RANGE("clada_select");
     if (!scores || !tau) return CLADA_ERR_NULL;
     if (B <= 0 || d_ff <= 0 || tau_stride < 0) return CLADA_ERR_SHAPE;
     select_kernel<<<B, kSelThreads, 0, static_cast<cudaStream_t>(stream)>>>(scores, d_ff, tau, tau_stride,
@@ -118,6 +120,7 @@ int clada_select(const float *scores, int32_t B, int32_t d_ff, const float *tau,
 
 int clada_tau_from_sparsity(const float *scores, int32_t B, int32_t d_ff, float rho, float *tau_base,
                             void *stream) {
+    CLADA_RANGE("clada_tau_from_sparsity");
     if (!scores || !tau_base) return CLADA_ERR_NULL;
     if (B <= 0 || d_ff <= 0 || !(rho >= 0.f && rho <= 1.f)) return CLADA_ERR_SHAPE;
     const int k_cut = (int)floor((double)rho * d_ff + 0.5);

@@ -5,6 +5,7 @@
 #include <algorithm>
 
 #include "common.cuh"
+#include "nvtx_ranges.cuh"
 #include "ffn_batch.cuh"
 
 namespace clada {
@@ -164,6 +165,7 @@ int clada_workspace_init(void *ws, size_t ws_bytes, void *stream) {
 }
 
 int clada_down_norms(const clada_layer *layer, float *out, void *stream) {
+    CLADA_RANGE("clada_down_norms");
     int rc = validate_layer(layer, false);
     if (rc != CLADA_OK) return rc;
     if (!out) return CLADA_ERR_NULL;
