@@ -448,12 +448,12 @@ class BatchJob:
         self.tau_s = wl.universal_threshold(self.s.flatten().tolist())
         self.tau_H = wl.universal_threshold(self.h.flatten().tolist())
         # Rows one layer-step at the baseline thresholds has to read: per launch, the union of the kept sets of the
-        # launch's sequences (the library takes 16 sequences per dense pass from 5 sequences on -- the pass reads
+        # launch's sequences (the library takes 16 sequences per dense pass from 3 sequences on -- the pass reads
         # every row of the layer, its union or not -- and tiles of 4 or 2 below that).
         tile = 4 if w.d_model * w.elem_bytes <= 8192 else 2
         self.launch_sizes, rest = [], B
         while rest > 0:
-            n = min(rest, 16) if rest >= 5 and w.dtype != "f32" else min(rest, tile)
+            n = min(rest, 16) if rest >= 3 and w.dtype != "f32" else min(rest, tile)
             self.launch_sizes.append(n)
             rest -= n
         m = self.mask.bool()
@@ -962,7 +962,7 @@ def main():
     ap.add_argument("--no-info", dest="info", action="store_false",
                     help="leave out the informational figures on the other workloads' layers")
     ap.add_argument("--batch", type=int, default=0,
-                    help="sequences per batch for the batched workloads instead of the workload's own (e.g. 4: the tile kernel)")
+                    help="sequences per batch for the batched workloads instead of the workload's own (e.g. 2: the tile kernel)")
     ap.add_argument("--quick", action="store_true",
                     help="for profiler captures: one replay per sample of the FFN-only loops and no informational "
                          "workloads (the figures of such a run are not bench values)")

@@ -249,8 +249,8 @@ int clada_cogload_adjust(const void *logits, int32_t logits_dtype, int32_t B, in
  *   mask_out / idx_out / count_out: optional (NULL), as in clada_select
  * Accumulation is fp32 in a fixed order: results are bit-identical run to run.
  * A batch of a 16-bit layer with d_ff <= 128 x (SM count) runs 16 sequences at
- * a time through ONE dense pass over the layer while 5 or more are left (the
- * union of that many kept sets is nearly the whole layer; both contractions on
+ * a time through ONE dense pass over the layer while 3 or more are left (at 40-60 %
+ * sparsity the union of that many kept sets is most of the layer; both contractions on
  * the tensor cores, the hidden activations carried exactly as three 16-bit
  * parts, each sequence's mask applied to its own activations: same 1e-5 as the
  * CUDA-core path).  What is left, and every batch of other layers, runs in tiles

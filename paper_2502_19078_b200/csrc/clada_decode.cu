@@ -1,5 +1,5 @@
 // The decode entry points of the C ABI: host-side checks, the choice of launches for a batch (one dense pass for
-// 4-16 sequences of a 16-bit layer, else tiles of 4 or 2 sequences, else one launch per sequence), the scratch
+// 3-16 sequences of a 16-bit layer, else tiles of 4 or 2 sequences, else one launch per sequence), the scratch
 // each choice needs, and the entry that allocates nothing.
 #include <algorithm>
 
@@ -24,13 +24,17 @@ static int decode_validate(const clada_layer *layer, const void *x, int32_t B, c
     return CLADA_OK;
 }
 
-// Sequences per launch for the next `remaining` sequences of a batch, at most max_tile (16, 4, 2 or 1): five or
+// Sequences per launch for the next `remaining` sequences of a batch, at most max_tile (16, 4, 2 or 1): three or
 // more sequences of a 16-bit layer go through the layer in one dense pass, up to 16 per launch; otherwise tiles of
 // 4 or 2 read the union of their kept sets (a tile kernel that takes 4 sequences of this layer also takes 2).
-static int decode_tile(const clada_layer *layer, int remaining, int max_tile) {
+static int decode_tile(const clada_layer *layer, int remaining, int max_tile, bool *dense) {
+    *dense = false;
     if (max_tile >= kDenseMaxSeqs && remaining >= kDenseMinSeqs) {
         const int n = remaining < kDenseMaxSeqs ? remaining : kDenseMaxSeqs;
-        if (ffn_batch_dense_supported(layer, n)) return n;
+        if (ffn_batch_dense_supported(layer, n)) {
+            *dense = true;
+            return n;
+        }
     }
     const int bt = ffn_batch_tile(layer, remaining);
     return bt < max_tile ? bt : (max_tile < 4 ? max_tile : 4);
@@ -39,8 +43,9 @@ static int decode_tile(const clada_layer *layer, int remaining, int max_tile) {
 // Whether any launch of the call is a tile of 2 or 4 sequences (those read the batch's keep words).
 static bool decode_has_tiles(const clada_layer *layer, int32_t B, int max_tile) {
     for (int b = 0; b < B;) {
-        const int bt = decode_tile(layer, B - b, max_tile);
-        if (bt > 1 && bt <= 4) return true;
+        bool dense;
+        const int bt = decode_tile(layer, B - b, max_tile, &dense);
+        if (bt > 1 && !dense) return true;
         b += bt;
     }
     return false;
@@ -55,9 +60,10 @@ static size_t decode_scratch_bytes(const clada_layer *layer, int32_t B, int num_
     size_t launch = 0;
     bool tiles = false;
     for (int b = 0; b < B;) {
-        const int bt = decode_tile(layer, B - b, max_tile);
+        bool dense;
+        const int bt = decode_tile(layer, B - b, max_tile, &dense);
         size_t need;
-        if (bt > 4) {
+        if (dense) {
             need = ffn_batch_dense_scratch_bytes(layer, bt);
         } else {
             need = (size_t)num_sms * (bt > 1 ? bt : ffn_groups(vpr)) * layer->d_model * sizeof(float);
@@ -95,7 +101,8 @@ static int decode_enqueue(const clada_layer *layer, const void *x, int32_t B, co
     int b = 0;
     while (b < B) {
         // Tiles of 4 or 2 sequences read each row of the union of their kept sets once.
-        const int bt = decode_tile(layer, B - b, max_tile);
+        bool dense;
+        const int bt = decode_tile(layer, B - b, max_tile, &dense);
         if (bt > 1) {
             if (mask_out || idx_out || count_out) {  // the batch kernels compute y only
                 rc = clada_select(scores + (size_t)b * layer->d_ff, bt, layer->d_ff, tau_final + (size_t)b * tau_stride,
@@ -104,7 +111,7 @@ static int decode_enqueue(const clada_layer *layer, const void *x, int32_t B, co
                                   count_out ? count_out + b : nullptr, stream);
                 if (rc != CLADA_OK) return rc;
             }
-            if (bt > 4)
+            if (dense)
                 rc = launch_ffn_batch_dense(layer, bt, static_cast<const char *>(x) + (size_t)b * layer->d_model * esz,
                                             scores + (size_t)b * layer->d_ff, tau_final + (size_t)b * tau_stride,
                                             tau_stride, static_cast<char *>(y) + (size_t)b * layer->d_model * ysz,

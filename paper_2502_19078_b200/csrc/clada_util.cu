@@ -141,7 +141,7 @@ size_t clada_workspace_bytes(const clada_layer *layer, int32_t B, int64_t T_tota
                     ((((size_t)B * ((size_t)(layer->d_ff + 31) / 32) * sizeof(unsigned)) + 255) & ~(size_t)255);
     // one sequence through a stack of layers: the keep words of up to 128 layers behind the partial rows
     decode = std::max(decode, (size_t)sms * 4 * (size_t)layer->d_model * sizeof(float) + keep_words_bytes(128, layer->d_ff));
-    // a dense pass over the layer for 5-16 sequences: a partial output per group of CTAs and the groups' hidden activations
+    // a dense pass over the layer for 3-16 sequences: a partial output per group of CTAs and the groups' hidden activations
     if (B >= kDenseMinSeqs) {
         const size_t dense = ffn_batch_dense_scratch_bytes(layer, B < kDenseMaxSeqs ? B : kDenseMaxSeqs);
         // sequences past a multiple of 16 may still run as tiles, whose keep words sit behind the launch scratch

@@ -1,4 +1,4 @@
-"""GPU parity of the dense pass of batched decode: 5-16 sequences of a 16-bit layer go through the layer in one
+"""GPU parity of the dense pass of batched decode: 3-16 sequences of a 16-bit layer go through the layer in one
 launch (tensor cores, per-sequence masks applied to the hidden activations), every sequence compared with the
 oracle's masked FFN for its own scores and threshold.  Same tolerances as the other FFN parity tests.
 """
@@ -82,6 +82,8 @@ def _case(clada, oracle, name, kw, B, act=0, y_dtypes=(torch.float32,), seed=0, 
     ("c4_llama3_8b_b8", {"d_model": 2048, "d_ff": 9000}, 9),      # 61 neurons per CTA: three padded rows per box
     ("c4_llama3_8b_b8", {"d_model": 256, "d_ff": 18900}, 7),      # 128 neurons per CTA, the most a launch takes
     ("c5_13b_b16", {"d_model": 8192, "d_ff": 600}, 6),            # 16 column tiles per member: three N = 16 instructions per K step
+    ("c4_llama3_8b_b8", {"d_model": 4096, "d_ff": 1000}, 4),      # the smallest batches that take the dense pass
+    ("c2_llama2_7b_layer", {"d_model": 1024, "d_ff": 900}, 3),
     ("c2_llama2_7b_layer", {"d_model": 8, "d_ff": 5}, 5),         # one K block of 8 columns, members 1-3 without a column tile
     ("c2_llama2_7b_layer", {"d_model": 72, "d_ff": 130}, 16),     # one neuron per CTA, ragged everything
 ])
@@ -89,9 +91,9 @@ def test_dense_pass_matches_oracle(clada, oracle, name, kw, B):
     _case(clada, oracle, name, kw, B, y_dtypes=(torch.float32, torch.bfloat16), outputs=(B == 8))
 
 
-@pytest.mark.parametrize("B", [17, 20, 33])
+@pytest.mark.parametrize("B", [17, 18, 20, 33])
 def test_batches_beyond_sixteen_sequences(clada, oracle, B):
-    """16 sequences per dense launch; what is left over runs densely too (5 or more), as tiles, or singly."""
+    """16 sequences per dense launch; what is left over runs densely too (3 or more), as a tile of two, or singly."""
     _case(clada, oracle, "c2_llama2_7b_layer", {"d_model": 1024, "d_ff": 1500}, B, outputs=True)
 
 

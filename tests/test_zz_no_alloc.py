@@ -9,8 +9,9 @@ run that stops at the first failure has already run everything else; it also pas
 fresh process, where its first call is the one that looks up the scratch address.
 
 The workspace entry is itself checked against the oracle elsewhere (tests/test_gpu_parity.py); the batch
-cases here check both entries against the oracle as well, because the fixed array forces the static entry
-into smaller tiles of sequences than the workspace entry takes (other CTA shares, so other rounding).
+cases here check both entries against the oracle as well, because the fixed array can force the static entry
+into smaller launches than the workspace entry takes (tiles instead of the dense pass, or smaller tiles: other
+CTA shares, so other rounding).
 """
 import numpy as np
 import pytest
@@ -54,8 +55,8 @@ def _run(clada, entry, layer, x, scores, tau, y_dtype, ws):
     ("c1_small_f32", 512, 1376, 2, torch.float32),
     ("c2_llama2_7b_layer", 4096, 900, 2, torch.bfloat16),
     ("c2_llama2_7b_layer", 4096, 900, 1, torch.float32),       # the single-sequence kernel on the array
-    ("c2_llama2_7b_layer", 4096, 900, 3, torch.float32),       # a tile of 2 and the odd sequence
-    ("c2_llama2_7b_layer", 4096, 900, 4, torch.float32),       # workspace: one tile of 4; static: two tiles of 2
+    ("c2_llama2_7b_layer", 4096, 900, 3, torch.float32),       # three sequences: one dense pass in both entries
+    ("c2_llama2_7b_layer", 4096, 900, 4, torch.float32),
     ("c2_llama2_7b_layer", 4096, 900, 8, torch.float32),       # the Llama-3-8B workload's batch
     ("c5_13b_b16", 5120, 700, 2, torch.float32),               # wider than a tile of 2 fits: one sequence per launch
     ("c2_llama2_7b_layer", 2048, 1200, 5, torch.float32),      # narrow enough for tiles of 4 on the array
