@@ -229,7 +229,7 @@ sparse_ffn_kernel(const FfnParams p, const int n_stages) {
             const int j = (bt * kFfnThreads + (warp * kWarp + t)) * kWarp + lane;
             const bool keep = (wb >> lane) & 1u;
             const int rank = wfr + __popc(wb & ((1u << lane) - 1u));
-            if (keep && rank >= r0 && rank < r1) {
+            if (keep && rank >= r0 && rank < r1 && guard_slot(rank, F, p.status)) {
                 s_list[rank - r0] = j;
                 if (p.idx_out) p.idx_out[rank] = j;
             }
@@ -275,7 +275,7 @@ sparse_ffn_kernel(const FfnParams p, const int n_stages) {
                     timed_out = true;
                     break;
                 }
-                const size_t off = (size_t)s_list[i] * row_bytes;
+                const size_t off = (size_t)guard_row(s_list[i], p.d_ff, p.status) * row_bytes;
                 const uint32_t dst = ring + (uint32_t)s * stage_bytes, bar = full0 + 8 * s;
                 mbar_expect_tx(bar, stage_bytes);
                 bulk_load_row_hint(dst, Wg + off, row_bytes, bar, stream_policy);

@@ -94,7 +94,7 @@ sparse_ffn_batch_kernel(const FfnBatchParams p, const int n_stages) {
                     timed_out = true;
                     break;
                 }
-                const size_t off = (size_t)s_list[i] * row_bytes;
+                const size_t off = (size_t)guard_row(s_list[i], p.d_ff, p.status) * row_bytes;
                 const uint32_t dst = ring + (uint32_t)s * stage_bytes, bar = full0 + 8 * s;
                 mbar_expect_tx(bar, stage_bytes);
                 bulk_load_row_hint(dst, Wg + off, row_bytes, bar, stream_policy);

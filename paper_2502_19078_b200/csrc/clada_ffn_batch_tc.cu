@@ -146,7 +146,7 @@ sparse_ffn_batch_tc_kernel(const FfnBatchParams p, const int n_stages) {
         __syncwarp();
         if (on) {
             const void *base = r == 0 ? p.w_gate : (r + 1 == (int)n_rows ? p.w_down_t : p.w_up);
-            const char *src = static_cast<const char *>(base) + (size_t)s_list[i] * row_bytes;
+            const char *src = static_cast<const char *>(base) + (size_t)guard_row(s_list[i], p.d_ff, p.status) * row_bytes;
             bulk_load_row_hint(ring + (uint32_t)s * stage_bytes + (uint32_t)r * pitch, src, row_bytes, bar,
                                policy_evict_first());
         }

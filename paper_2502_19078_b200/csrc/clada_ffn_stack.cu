@@ -385,7 +385,7 @@ sparse_ffn_stack_kernel(const StackParams p, const __grid_constant__ StackLayers
                         mbar_expect_tx(bar, row_bytes);
                         bulk_load_row_hint(dst, p.x + (size_t)l * p.x_stride, row_bytes, bar, keep_policy);
                     } else {
-                        const size_t off = (size_t)list[i] * row_bytes;
+                        const size_t off = (size_t)guard_row(list[i], p.d_ff, p.status) * row_bytes;
                         mbar_expect_tx(bar, stage_bytes);
                         bulk_load_row_hint(dst, Wg + off, row_bytes, bar, stream_policy);
                         if (GATED) bulk_load_row_hint(dst + row_bytes, Wu + off, row_bytes, bar, stream_policy);

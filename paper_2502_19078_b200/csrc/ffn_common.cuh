@@ -101,6 +101,30 @@ __device__ __forceinline__ void bulk_load_row_hint(uint32_t dst, const void *src
         ::"r"(dst), "l"(src), "r"(bytes), "r"(bar), "l"(policy)
         : "memory");
 }
+// A neuron index on its way into a row address.  The lists the kernels build hold indices below d_ff by
+// construction, so the release build passes them through; a -DCLADA_DEBUG_BOUNDS build checks every one, records
+// CLADA_STATUS_BAD_INDEX in the call's status word and reads row 0 instead (never a trap, never a skipped copy:
+// the stage's byte count stays what its barrier expects).
+__device__ __forceinline__ int guard_row(int j, int d_ff, int32_t *status) {
+#ifdef CLADA_DEBUG_BOUNDS
+    if ((unsigned)j >= (unsigned)d_ff) {
+        if (status) atomicOr(status, CLADA_STATUS_BAD_INDEX);
+        return 0;
+    }
+#endif
+    return j;
+}
+// A slot of a list about to be written: always true in the release build; the checking build records an
+// out-of-range slot and the caller skips the store.
+__device__ __forceinline__ bool guard_slot(int i, int n, int32_t *status) {
+#ifdef CLADA_DEBUG_BOUNDS
+    if ((unsigned)i >= (unsigned)n) {
+        if (status) atomicOr(status, CLADA_STATUS_BAD_INDEX);
+        return false;
+    }
+#endif
+    return true;
+}
 __device__ __forceinline__ float ld_keep(const float *p, uint64_t policy) {
     float v;
     asm volatile("ld.global.L2::cache_hint.f32 %0, [%1], %2;" : "=f"(v) : "l"(p), "l"(policy));
