@@ -349,14 +349,23 @@ int clada_sparse_ffn_decode_static(const clada_layer *layer, const void *x, int3
  *   the decode path's w_down_t is its transpose), tensor cores, fp32
  *   accumulation.  bf16 / fp16 layers; d_ff a multiple of 8; all pointers
  *   16-byte aligned.  Together with Z from clada_prefix_accumulate this is the
- *   layer's dense prefill output. */
+ *   layer's dense prefill output.
+ *   ws / ws_bytes: optional workspace (NULL, 0: none).  A short prompt has fewer
+ *   output tiles than the device has SMs; with a workspace of
+ *   clada_workspace_bytes(layer, 1, T) bytes the K dimension (d_ff) of each tile
+ *   is then split among up to 8 CTAs, whose fp32 partial outputs are added in a
+ *   fixed order (same result on every call; it differs from the unsplit sum only
+ *   by fp32 rounding).  A workspace too small for that is not an error: the call
+ *   runs unsplit.  CLADA_ERR_WORKSPACE: ws not 256-byte aligned or smaller than
+ *   its control block. */
 int clada_prefix_accumulate(const clada_layer *layer, const void *X, const int64_t *seq_offsets,
                             int32_t B, float *sumsq, void *Z, void *ws, size_t ws_bytes,
                             int32_t *status, void *stream);
 int clada_prefix_finish(const clada_layer *layer, const float *sumsq, int32_t B, float *scores,
                         void *stream);
 int clada_prefill_down(const clada_layer *layer, const void *w_down, const void *Z, int64_t T,
-                       void *Y, int32_t y_dtype, int32_t *status, void *stream);
+                       void *Y, int32_t y_dtype, void *ws, size_t ws_bytes, int32_t *status,
+                       void *stream);
 
 /* ---- Nested index lists: the masks of Eq. final_threshold in compressed form ----
  *

@@ -75,7 +75,7 @@ def load() -> ctypes.CDLL:
     L.clada_stream_read_probe.argtypes = [vp, sz, vp, vp]
     L.clada_prefix_accumulate.argtypes = [lp, vp, vp, i32, vp, vp, vp, sz, vp, vp]
     L.clada_prefix_finish.argtypes = [lp, vp, i32, vp, vp]
-    L.clada_prefill_down.argtypes = [lp, vp, vp, i64, vp, i32, vp, vp]
+    L.clada_prefill_down.argtypes = [lp, vp, vp, i64, vp, i32, vp, sz, vp, vp]
     L.clada_nested_build.argtypes = [vp, i32, i32, vp, i64, f32, f32, vp, vp, vp]
     L.clada_cogload_level.argtypes = [vp, i32, i32, i64, i64, vp, f32, f32, vp, vp, vp, vp, vp]
     L.clada_sparse_ffn_decode_nested.argtypes = [lp, vp, i32, vp, vp, vp, vp, i32, vp, vp, sz, vp, vp]
@@ -430,10 +430,11 @@ def clada_prefix_finish(layer: Layer, sumsq, scores, stream=None) -> None:
                                       _ptr(scores, torch.float32, "scores"), _stream(stream)), "clada_prefix_finish")
 
 
-def clada_prefill_down(layer: Layer, w_down, Z, Y, status=None, stream=None) -> None:
-    """Y [T, d_model] = Z [T, d_ff] w_down^T, w_down [d_model, d_ff] in the paper's layout."""
+def clada_prefill_down(layer: Layer, w_down, Z, Y, status=None, stream=None, ws=None) -> None:
+    """Y [T, d_model] = Z [T, d_ff] w_down^T, w_down [d_model, d_ff] in the paper's layout; ws: optional workspace."""
     _check(load().clada_prefill_down(layer.ref, _ptr(w_down, layer.dtype, "w_down"), _ptr(Z, layer.dtype, "Z"),
                                      Z.shape[0], _ptr(Y, name="Y"), _dtype_code(Y.dtype),
+                                     ws.data_ptr() if ws is not None else None, ws.numel() if ws is not None else 0,
                                      _ptr(status, torch.int32, "status"), _stream(stream)), "clada_prefill_down")
 
 

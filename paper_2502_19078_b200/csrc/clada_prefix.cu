@@ -461,7 +461,7 @@ int clada_prefix_finish(const clada_layer *layer, const float *sumsq, int32_t B,
 }
 
 int clada_prefill_down(const clada_layer *layer, const void *w_down, const void *Z, int64_t T, void *Y,
-                       int32_t y_dtype, int32_t *status, void *stream) {
+                       int32_t y_dtype, void *ws, size_t ws_bytes, int32_t *status, void *stream) {
     CLADA_RANGE("clada_prefill_down");
     int rc = validate_layer(layer, false);
     if (rc != CLADA_OK) return rc;
@@ -471,7 +471,11 @@ int clada_prefill_down(const clada_layer *layer, const void *w_down, const void 
     if (!dtype_ok(y_dtype)) return CLADA_ERR_DTYPE;
     if (layer->d_ff % 8 != 0) return CLADA_ERR_SHAPE;  // rows of Z and of w_down must be 16-byte multiples
     if (!aligned16(w_down) || !aligned16(Z) || !aligned16(Y)) return CLADA_ERR_ALIGN;
-    return run_down_tc(layer, w_down, Z, T, Y, y_dtype, status, static_cast<cudaStream_t>(stream));
+    if (ws && ((reinterpret_cast<uintptr_t>(ws) & 255u) || ws_bytes < kWsCtrlBytes)) return CLADA_ERR_WORKSPACE;
+    // the scratch behind the workspace's control block (which this call leaves alone) holds split partial outputs
+    void *scratch = ws ? static_cast<char *>(ws) + kWsCtrlBytes : nullptr;
+    return run_down_tc(layer, w_down, Z, T, Y, y_dtype, scratch, ws ? ws_bytes - kWsCtrlBytes : 0, status,
+                       static_cast<cudaStream_t>(stream));
 }
 
 int clada_refine_scores(const clada_layer *layer, const void *X, const int64_t *seq_offsets, int32_t B,

@@ -400,8 +400,12 @@ int run_prefix_partials_tc(const clada_layer *layer, const void *X, const SeqTab
 // the statistics kernel: tokens are the M dimension (TMEM lanes), output columns the N dimension, one
 // accumulator per tile (256 output columns, or 128 for short prompts), two in flight.  The epilogue thread
 // that owns token t writes its row of the tile.
+// Short prompts have fewer tiles than the device has SMs, and a tile's time is its number of K blocks whatever
+// its width: given scratch, the K dimension of every tile is then split among n_split CTAs, each writes its fp32
+// partial tile to the scratch, and down_reduce_kernel adds the partials in split order and writes Y.
 
 constexpr int kDnMaxStages = 6;
+constexpr int kDnMaxSplit = 8;                        // CTAs per output tile along K, at most
 constexpr uint32_t kDnTmemCols = 512;                 // two accumulators of up to 256 columns
 
 struct DownParams {
@@ -411,6 +415,9 @@ struct DownParams {
     int t_group;   // token tiles per group: a group's rows of Z stay in L2 while every output tile reads them
     int nd;        // output columns per tile: 256 (fewer bytes read per flop), or 128 when 256 would leave SMs idle
     int n_stages;
+    int n_split;   // CTAs per tile along K (1: no split, Y is written directly)
+    int kb_split;  // K blocks per split
+    float *partials;  // [n_split, T, d_model] fp32 when n_split > 1
     void *y;
     int y_dtype;
     uint32_t idesc;
@@ -427,7 +434,8 @@ down_tc_kernel(const __grid_constant__ CUtensorMap map_z, const __grid_constant_
     __shared__ int s_abort;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int n_items = p.n_ttiles * p.n_dtiles;
+    const int n_tiles = p.n_ttiles * p.n_dtiles;
+    const int n_items = n_tiles * p.n_split;  // item = split * n_tiles + tile: a wave's CTAs walk the same K range
     const int nd = p.nd, n_stages = p.n_stages;
     // items in groups of t_group token tiles; within a group output tile by output tile, token tile fastest
     auto tile_of = [&](int f, int &dtile, int &ttile) {
@@ -442,6 +450,13 @@ down_tc_kernel(const __grid_constant__ CUtensorMap map_z, const __grid_constant_
     };
     const uint32_t stage_bytes = kTcTileBytes + (uint32_t)nd * kTcTileK * 2u;  // Z tile | W_out tile
     const int n_kblocks = (p.d_ff + kTcTileK - 1) / kTcTileK;
+    // K blocks [kb_lo, kb_hi) of an item (never empty: the host sees to that)
+    auto k_range = [&](int item, int &tile, int &kb_lo, int &kb_hi) {
+        const int sp = item / n_tiles;
+        tile = item - sp * n_tiles;
+        kb_lo = sp * p.kb_split;
+        kb_hi = min(n_kblocks, kb_lo + p.kb_split);
+    };
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < n_stages; ++s) {
@@ -478,11 +493,12 @@ down_tc_kernel(const __grid_constant__ CUtensorMap map_z, const __grid_constant_
             const uint32_t full0 = tc_smem_u32(&s_full[0]), empty0 = tc_smem_u32(&s_empty[0]);
             uint32_t full_s = full0, empty_s = empty0, dst_s = smem0;
             for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
-                int dtile, ttile;
-                tile_of(item, dtile, ttile);
+                int dtile, ttile, tile, kb_lo, kb_hi;
+                k_range(item, tile, kb_lo, kb_hi);
+                tile_of(tile, dtile, ttile);
                 const int row_z = ttile * kTcTileM, row_w = dtile * nd;
-                int c0 = 0;
-                for (int kb = 0; kb < n_kblocks; ++kb, ++kc, c0 += kTcTileK) {
+                int c0 = kb_lo * kTcTileK;
+                for (int kb = kb_lo; kb < kb_hi; ++kb, ++kc, c0 += kTcTileK) {
                     if (!tc_mbar_wait(empty_s, par ^ 1, abort_flag)) {
                         ok = false;
                         break;
@@ -529,7 +545,9 @@ down_tc_kernel(const __grid_constant__ CUtensorMap map_z, const __grid_constant_
                 tc_fence_after();
                 const uint32_t d_acc = tmem_base + (uint32_t)a * 256u;
                 uint32_t acc = 0u;
-                for (int kb = 0; kb < n_kblocks; ++kb) {
+                int tile, kb_lo, kb_hi;
+                k_range(item, tile, kb_lo, kb_hi);
+                for (int kb = kb_lo; kb < kb_hi; ++kb) {
                     if (!tc_mbar_wait(full_s, par, abort_flag)) {
                         ok = false;
                         break;
@@ -563,8 +581,11 @@ down_tc_kernel(const __grid_constant__ CUtensorMap map_z, const __grid_constant_
         bool ok = true;
         for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++it) {
             const int a = it & 1;
-            int dtile, ttile;
-            tile_of(item, dtile, ttile);
+            int dtile, ttile, tile, kb_lo, kb_hi;
+            k_range(item, tile, kb_lo, kb_hi);
+            tile_of(tile, dtile, ttile);
+            // a split item's fp32 partial tile goes to its split's copy of the output, added up afterwards
+            float *part = p.n_split > 1 ? p.partials + (size_t)(item / n_tiles) * (size_t)p.T * p.d_model : nullptr;
             if (!tc_mbar_wait(tc_smem_u32(&s_acc_full[a]), (it >> 1) & 1, abort_flag)) {
                 ok = false;
                 break;
@@ -587,7 +608,11 @@ down_tc_kernel(const __grid_constant__ CUtensorMap map_z, const __grid_constant_
                         const float4 hi = make_float4(__uint_as_float(r[8 * h + 4]), __uint_as_float(r[8 * h + 5]),
                                                       __uint_as_float(r[8 * h + 6]), __uint_as_float(r[8 * h + 7]));
                         const size_t at = (size_t)t * p.d_model + i0 + c0 + 8 * h;
-                        if (p.y_dtype == CLADA_F32) {
+                        if (part) {
+                            float4 *dst = reinterpret_cast<float4 *>(part + at);
+                            dst[0] = lo;
+                            dst[1] = hi;
+                        } else if (p.y_dtype == CLADA_F32) {
                             float4 *dst = reinterpret_cast<float4 *>(static_cast<float *>(p.y) + at);
                             dst[0] = lo;
                             dst[1] = hi;
@@ -614,8 +639,41 @@ down_tc_kernel(const __grid_constant__ CUtensorMap map_z, const __grid_constant_
     }
 }
 
+// Y = the sum of the splits' fp32 partial outputs, in split order (fixed: results repeat bit for bit).
+__global__ void __launch_bounds__(256)
+down_reduce_kernel(const float4 *__restrict__ partials, int n_split, size_t n4, void *y, int y_dtype) {
+    const size_t i = (size_t)blockIdx.x * 256 + threadIdx.x;
+    pdl_wait();  // launched while the contraction still runs: its partial outputs are complete from here on
+    if (i >= n4) return;
+    float4 s = __ldcg(partials + i);
+    for (int k = 1; k < n_split; ++k) {
+        const float4 v = __ldcg(partials + (size_t)k * n4 + i);
+        s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
+    }
+    if (y_dtype == CLADA_F32)
+        static_cast<float4 *>(y)[i] = s;
+    else
+        static_cast<uint2 *>(y)[i] = pack4_16bit(y_dtype, s);
+}
+
+// CTAs per tile along K for a prompt of T tokens: 1 unless tiles of 256 output columns leave at least half of the
+// SMs without one; at most kDnMaxSplit, and no split may be empty.
+static int down_split(const clada_layer *layer, long long T, int num_sms) {
+    const long long tiles = ((T + kTcTileM - 1) / kTcTileM) * ((layer->d_model + 255) / 256);
+    if (tiles <= 0 || 2 * tiles > num_sms) return 1;
+    const int n_kblocks = (layer->d_ff + kTcTileK - 1) / kTcTileK;
+    int n = (int)std::min<long long>(kDnMaxSplit, num_sms / tiles);
+    while (n > 1 && (n - 1) * ((n_kblocks + n - 1) / n) >= n_kblocks) --n;
+    return n;
+}
+
+size_t down_split_scratch_bytes(const clada_layer *layer, long long T, int num_sms) {
+    const int n = down_split(layer, T, num_sms);
+    return n > 1 ? (size_t)n * (size_t)T * layer->d_model * sizeof(float) : 0;
+}
+
 int run_down_tc(const clada_layer *layer, const void *w_down, const void *Z, long long T, void *Y, int y_dtype,
-                int32_t *status, cudaStream_t st) {
+                void *scratch, size_t scratch_bytes, int32_t *status, cudaStream_t st) {
     static bool configured[64] = {};
     if (T <= 0) return CLADA_OK;
     DeviceInfo di;
@@ -635,9 +693,17 @@ int run_down_tc(const clada_layer *layer, const void *w_down, const void *Z, lon
         const long long tile_bytes = (long long)kTcTileM * layer->d_ff * 2;
         p.t_group = (int)std::max<long long>(1, std::min<long long>(p.n_ttiles, (40ll << 20) / tile_bytes));
     }
-    // 256 output columns per tile unless that leaves SMs without a tile
-    p.nd = (long long)p.n_ttiles * ((layer->d_model + 255) / 256) >= di.num_sms ? 256 : 128;
+    // 256 output columns per tile unless that leaves SMs without a tile -- or, given scratch, with K split among
+    // as many CTAs per tile as fit the device
+    p.n_split = 1;
+    {
+        const size_t need = down_split_scratch_bytes(layer, T, di.num_sms);
+        if (scratch && need > 0 && scratch_bytes >= need) p.n_split = down_split(layer, T, di.num_sms);
+    }
+    p.nd = p.n_split > 1 || (long long)p.n_ttiles * ((layer->d_model + 255) / 256) >= di.num_sms ? 256 : 128;
     p.n_dtiles = (layer->d_model + p.nd - 1) / p.nd;
+    p.kb_split = (((layer->d_ff + kTcTileK - 1) / kTcTileK) + p.n_split - 1) / p.n_split;
+    p.partials = static_cast<float *>(scratch);
     const uint32_t dn_stage = kTcTileBytes + (uint32_t)p.nd * kTcTileK * 2u;
     p.n_stages = std::min<int>(kDnMaxStages, (int)(kTcRingBytes / dn_stage));
     p.y = Y;
@@ -650,10 +716,24 @@ int run_down_tc(const clada_layer *layer, const void *w_down, const void *Z, lon
         CLADA_CUDA_TRY(cudaFuncSetAttribute(down_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
         configured[di.device & 63] = true;
     }
-    const long long items = (long long)p.n_ttiles * p.n_dtiles;
+    const long long items = (long long)p.n_ttiles * p.n_dtiles * p.n_split;
     const int grid = (int)std::min<long long>(items, di.num_sms);
     down_tc_kernel<<<grid, kTcThreads, smem, st>>>(map_z, map_w, p);
     CLADA_CUDA_TRY(cudaGetLastError());
+    if (p.n_split > 1) {
+        const size_t n4 = (size_t)T * layer->d_model / 4;  // d_model is a multiple of 8
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)((n4 + 255) / 256));
+        cfg.blockDim = dim3(256);
+        cfg.stream = st;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;  // hide the launch latency
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        CLADA_CUDA_TRY(cudaLaunchKernelEx(&cfg, down_reduce_kernel, static_cast<const float4 *>(scratch), p.n_split, n4, Y,
+                                          y_dtype));
+    }
     return CLADA_OK;
 }
 

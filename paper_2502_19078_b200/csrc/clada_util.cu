@@ -7,6 +7,7 @@
 #include "common.cuh"
 #include "nvtx_ranges.cuh"
 #include "ffn_batch.cuh"
+#include "prefix_common.cuh"
 
 namespace clada {
 
@@ -154,6 +155,8 @@ size_t clada_workspace_bytes(const clada_layer *layer, int32_t B, int64_t T_tota
     // plus its counter (256 bytes) and up to 512 split partial sums (two doubles each)
     size_t refine = (size_t)B * (size_t)layer->d_ff * 2 * sizeof(int32_t) + 256 + 512 * 16;
     size_t scratch = decode > prefix + refine ? decode : prefix + refine;
+    // dense prefill down projection of a short prompt: the fp32 partial outputs of its K splits
+    if (layer->dtype != CLADA_F32) scratch = std::max(scratch, down_split_scratch_bytes(layer, T_total, sms));
     return kWsCtrlBytes + ((scratch + 255) & ~(size_t)255);
 }
 

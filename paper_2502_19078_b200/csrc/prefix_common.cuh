@@ -44,9 +44,11 @@ size_t prefix_partials_bytes_cuda_core(const int64_t *seq_offsets, int32_t B, in
 int run_prefix_partials_tc(const clada_layer *layer, const void *X, const SeqTable &tab, long long T_total,
                            float *partials, int32_t *status, cudaStream_t st, void *z_out = nullptr);
 
-// Y [T, d_model] = Z [T, d_ff] . w_down[d_model, d_ff]^T on the tensor cores (16-bit element types).
+// Y [T, d_model] = Z [T, d_ff] . w_down[d_model, d_ff]^T on the tensor cores (16-bit element types).  scratch
+// (optional, 16-byte aligned): down_split_scratch_bytes() bytes let a short prompt's tiles be split along K.
 int run_down_tc(const clada_layer *layer, const void *w_down, const void *Z, long long T, void *Y, int y_dtype,
-                int32_t *status, cudaStream_t st);
+                void *scratch, size_t scratch_bytes, int32_t *status, cudaStream_t st);
+size_t down_split_scratch_bytes(const clada_layer *layer, long long T, int num_sms);
 constexpr int kTcTokenTile = 128;
 
 }  // namespace clada

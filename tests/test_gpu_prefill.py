@@ -59,7 +59,8 @@ def test_prefill_ffn_parity(clada, oracle, dtype, act, d, F, lengths):
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
     clada.clada_prefix_accumulate(layer, X.cuda(), off, sumsq, ws, Z, status)
     clada.clada_prefix_finish(layer, sumsq, scores)
-    clada.clada_prefill_down(layer, weights["w_down"].cuda().contiguous(), Z, Y, status)
+    # with the workspace these few tiles are split along K (five CTAs per tile at d_ff 304, three at 136)
+    clada.clada_prefill_down(layer, weights["w_down"].cuda().contiguous(), Z, Y, status, ws=ws)
     torch.cuda.synchronize()
     assert int(status.item()) == 0
     W_in, V_in, W_out = oracle_weights(weights, act)
@@ -115,6 +116,47 @@ def test_prefill_output_types_and_ragged_columns(clada, oracle):
     assert rel_inf(Y32.cpu().numpy().astype(np.float64), Y_own) <= DOWN_TOL
 
 
+@pytest.mark.parametrize("d,F,T", [(512, 1000, 300),     # 6 tiles x 8 splits of 2 K blocks, the last one ragged
+                                   (1024, 4160, 128),    # 4 tiles x 8 splits of 9 K blocks (the last: 2)
+                                   (2048, 704, 600)])    # 40 tiles x 3 splits of 4 K blocks (the last: 3)
+def test_prefill_down_split_along_k(clada, oracle, d, F, T):
+    """A short prompt's down projection with a workspace: every output tile's K range is split among several CTAs
+    and their fp32 partial outputs are added in a fixed order.  Against the oracle's projection of the same Z,
+    against the unsplit call (fp32 rounding apart), bit-identical on repetition, in fp32 and bf16 outputs, and
+    rows past T stay untouched."""
+    w = wl.scaled(wl.WORKLOADS["c2_llama2_7b_layer"], d_model=d, d_ff=F)
+    weights = wl.layer_weights(w, 0)
+    layer = gpu_layer(weights, clada)
+    g = torch.Generator().manual_seed(11)
+    Z = (torch.randn(T, F, generator=g) * 0.5).to(torch.bfloat16).cuda()
+    wd = weights["w_down"].cuda().contiguous()
+    ws = clada.new_workspace(layer, 1, T)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    Y_plain = torch.empty(T, d, dtype=torch.float32, device="cuda")
+    clada.clada_prefill_down(layer, wd, Z, Y_plain, status)
+    Y_split = torch.full((T + 2, d), 7.0, dtype=torch.float32, device="cuda")
+    clada.clada_prefill_down(layer, wd, Z, Y_split[:T], status, ws=ws)
+    Y_again = torch.empty(T, d, dtype=torch.float32, device="cuda")
+    clada.clada_prefill_down(layer, wd, Z, Y_again, status, ws=ws)
+    Y16 = torch.full((T + 2, d), 7.0, dtype=torch.bfloat16, device="cuda")
+    clada.clada_prefill_down(layer, wd, Z, Y16[:T], status, ws=ws)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    assert torch.equal(Y_split[:T], Y_again) and torch.all(Y_split[T:] == 7.0) and torch.all(Y16[T:] == 7.0)
+    assert torch.equal(Y16[:T], Y_split[:T].to(torch.bfloat16))
+    Y_own = oracle.down_proj(_widen(Z), oracle_weights(weights)[2])
+    assert rel_inf(Y_split[:T].cpu().numpy().astype(np.float64), Y_own) <= DOWN_TOL
+    assert rel_inf(Y_plain.cpu().numpy().astype(np.float64), Y_own) <= DOWN_TOL
+    assert not torch.equal(Y_plain, Y_split[:T]) or F <= 64      # the split really ran (another summation order)
+    # the workspace's control block is left as it was: a decode on it still works
+    x = wl.hidden_states(w, 0, "decode", 0, 1)[0].cuda()
+    y = torch.empty(1, d, device="cuda")
+    clada.clada_sparse_ffn_decode(layer, x[None], torch.ones(1, F, device="cuda"), torch.zeros(1, device="cuda"), 1, y, ws,
+                                  None, None, None, status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0 and bool(torch.isfinite(y).all())
+
+
 @pytest.mark.parametrize("name,kw", [("c2_llama2_7b_layer", {"d_model": 256, "d_ff": 300}),
                                      ("c1_small_f32", {"d_model": 72, "d_ff": 130})])
 def test_chunked_statistics_equal_whole_prompt(clada, oracle, name, kw):
@@ -153,8 +195,9 @@ def test_chunked_statistics_equal_whole_prompt(clada, oracle, name, kw):
 
 @pytest.mark.parametrize("T", [512, 2048])
 def test_prefill_full_width_c2(clada, oracle, T):
-    """The benchmark's layer at full width: sampled rows of Z and Y against the oracle.  512 tokens run the down
-    projection in 128-column tiles, 2048 tokens in 256-column tiles."""
+    """The benchmark's layer at full width: sampled rows of Z and Y against the oracle.  2048 tokens run the down
+    projection in 256-column tiles; 512 tokens too, given the workspace, with every tile's K range split between
+    two CTAs (and in 128-column tiles, unsplit, without the workspace: both are checked)."""
     w = wl.WORKLOADS["c2_llama2_7b_layer"]
     weights = wl.layer_weights(w, 0, "cuda")
     layer = gpu_layer(weights, clada)
@@ -165,7 +208,9 @@ def test_prefill_full_width_c2(clada, oracle, T):
     Y = torch.empty(T, w.d_model, dtype=torch.float32, device="cuda")
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
     clada.clada_prefix_accumulate(layer, X, [0, T], sumsq, ws, Z, status)
-    clada.clada_prefill_down(layer, weights["w_down"].contiguous(), Z, Y, status)
+    clada.clada_prefill_down(layer, weights["w_down"].contiguous(), Z, Y, status, ws=ws)
+    Y_plain = torch.empty_like(Y)
+    clada.clada_prefill_down(layer, weights["w_down"].contiguous(), Z, Y_plain, status)
     scores = torch.empty(1, w.d_ff, dtype=torch.float32, device="cuda")
     clada.clada_prefix_finish(layer, sumsq, scores)
     whole = torch.empty(1, w.d_ff, dtype=torch.float32, device="cuda")
@@ -179,9 +224,12 @@ def test_prefill_full_width_c2(clada, oracle, T):
     Zg = _widen(Z[rows])
     diff = np.abs(Zg - Z_or)
     assert np.all(diff <= _ulp(Z_or, "bf16") * 1.0001 + 2e-5 * np.max(np.abs(Z_or))) and np.mean(diff > 0) <= 0.03
-    Yg = Y[rows].cpu().numpy().astype(np.float64)
-    assert rel_inf(Yg, oracle.down_proj(Zg, W_out)) <= DOWN_TOL
-    assert rel_inf(Yg, oracle.down_proj(Z_or, W_out)) <= FFN_TOL
+    Y_own = oracle.down_proj(Zg, W_out)
+    for Yt in (Y, Y_plain):
+        Yg = Yt[rows].cpu().numpy().astype(np.float64)
+        assert rel_inf(Yg, Y_own) <= DOWN_TOL
+        assert rel_inf(Yg, oracle.down_proj(Z_or, W_out)) <= FFN_TOL
+    assert torch.equal(Y, Y_plain) == (T == 2048)      # enough tiles for every SM: the workspace changes nothing
 
 
 def test_new_entry_points_refuse_what_they_cannot_do(clada):
