@@ -434,7 +434,7 @@ def clada_prefill_down(layer: Layer, w_down, Z, Y, status=None, stream=None, ws=
     """Y [T, d_model] = Z [T, d_ff] w_down^T, w_down [d_model, d_ff] in the paper's layout; ws: optional workspace."""
     _check(load().clada_prefill_down(layer.ref, _ptr(w_down, layer.dtype, "w_down"), _ptr(Z, layer.dtype, "Z"),
                                      Z.shape[0], _ptr(Y, name="Y"), _dtype_code(Y.dtype),
-                                     ws.data_ptr() if ws is not None else None, ws.numel() if ws is not None else 0,
+                                     _ptr(ws, torch.uint8, "ws"), ws.numel() if ws is not None else 0,
                                      _ptr(status, torch.int32, "status"), _stream(stream)), "clada_prefill_down")
 
 

@@ -255,6 +255,19 @@ def test_new_entry_points_refuse_what_they_cannot_do(clada):
     with pytest.raises(clada.CladaError, match="shape"):
         clada.clada_prefill_down(lb, torch.zeros(64, 100, dtype=torch.bfloat16, device="cuda"), Zb,
                                  torch.empty(16, 64, device="cuda"))
+    w8 = wl.scaled(wl.WORKLOADS["c2_llama2_7b_layer"], d_model=64, d_ff=104)
+    l8 = gpu_layer(wl.layer_weights(w8, 0), clada)
+    ws8 = clada.new_workspace(l8, 1, 16)
+    Z8 = torch.zeros(16, 104, dtype=torch.bfloat16, device="cuda")
+    wd8 = torch.zeros(64, 104, dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(clada.CladaError, match="workspace"):             # a workspace off its 256-byte boundary
+        clada.clada_prefill_down(l8, wd8, Z8, torch.empty(16, 64, device="cuda"), ws=ws8[16:])
+    with pytest.raises(clada.CladaError, match="workspace"):             # smaller than its control block
+        clada.clada_prefill_down(l8, wd8, Z8, torch.empty(16, 64, device="cuda"), ws=ws8[:128])
+    Y8 = torch.full((16, 64), 5.0, device="cuda")
+    clada.clada_prefill_down(l8, wd8, Z8, Y8, ws=ws8[:256])               # too small to split: runs unsplit
+    torch.cuda.synchronize()
+    assert bool((Y8 == 0).all())
     big = torch.ones(1, 32769, device="cuda")                             # the list build holds 32768 scores per CTA
     with pytest.raises(clada.CladaError, match="support"):
         clada.clada_nested_build(big, torch.ones(1, device="cuda"), 0.8, 0.12,
